@@ -1,0 +1,164 @@
+/*
+ * lpmm.h - C ABI of the B200 (sm_100a) fused 4-bit AdamW step.
+ *
+ * Implements the hot path of "Memory Efficient Optimizers with 4-bit States" (arXiv 2309.01507):
+ * Alg. 3 (compressed Adam) with Eq. 1, decoupled weight decay, the first moment kept as
+ * B128/DE (Sec. 3, App. D.2) and the second moment as Rank-1/Linear (Sec. 4.1, 4.2), B128/Linear
+ * for one-dimensional tensors (Sec. 4.2) and fp32 states for tensors of <= 4096 elements (App. C.1).
+ *
+ * Conventions
+ *  - Pointers named d_* are DEVICE pointers, h_* are HOST pointers; everything else is host memory.
+ *  - The caller owns every device buffer (parameters, gradients, the state arena). The library
+ *    allocates no device memory; it owns only the small host-side handle (lpmm_state).
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream). Work is
+ *    enqueued on it and the call returns without synchronizing unless stated otherwise.
+ *  - Every function validates its arguments on the host before launching anything and returns a
+ *    negative lpmm_status on error; nothing throws, traps or exits. Launch failures are reported
+ *    as LPMM_ERR_CUDA (see lpmm_last_cuda_error()).
+ *  - Tensors are row-major and contiguous. Codes are 4-bit; element 2k of the flattened tensor sits
+ *    in bits 0-3 of byte k and element 2k+1 in bits 4-7; ceil(numel/2) bytes per moment.
+ *  - NaN/Inf gradients are not detected; the result is then unspecified (but nothing faults).
+ *  - There is no CPU fallback: without a CUDA device every launching call returns LPMM_ERR_CUDA.
+ */
+#ifndef LPMM_H
+#define LPMM_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t lpmm_status;
+#define LPMM_OK 0
+#define LPMM_ERR_INVALID_ARG (-1)     /* null pointer, non-positive size, bad enum, bad hyper-parameter */
+#define LPMM_ERR_UNSUPPORTED (-2)     /* a combination this build does not implement */
+#define LPMM_ERR_ALIGNMENT (-3)       /* a device pointer is not 16-byte aligned */
+#define LPMM_ERR_ARENA_TOO_SMALL (-4) /* arena_bytes < lpmm_state_bytes() */
+#define LPMM_ERR_CUDA (-5)            /* a CUDA runtime call or launch failed */
+
+typedef enum { LPMM_F32 = 0, LPMM_BF16 = 1 } lpmm_dtype;
+typedef enum { LPMM_NORM_BLOCK = 0, LPMM_NORM_RANK1 = 1 } lpmm_norm;          /* Sec. 2.2 / Sec. 4.2 */
+typedef enum { LPMM_MAP_DE_SIGNED = 0, LPMM_MAP_LINEAR_NOZERO = 1 } lpmm_map; /* App. D.2 / Sec. 4.1 */
+typedef enum { LPMM_V_RANK1 = 0, LPMM_V_BLOCK = 1 } lpmm_vmode;               /* second-moment normalizer for 2-D tensors */
+
+/* lpmm_shape.flags */
+#define LPMM_FORCE_QUANT 1u /* quantize even if numel <= min_quant_numel */
+#define LPMM_FORCE_FP32 2u  /* keep fp32 states whatever the size */
+
+/* lpmm_quantize flags */
+#define LPMM_Q_GIVEN_SCALES 1u /* use the scales already in d_scale0/d_scale1 instead of recomputing them */
+
+typedef struct {
+    int64_t rows, cols; /* ndim 1: rows = numel, cols = 1; ndim 2: rows x cols, row-major */
+    int32_t ndim;       /* 1 or 2 */
+    uint32_t flags;
+} lpmm_shape;
+
+typedef struct {
+    int32_t bits;            /* 4 */
+    int32_t m_block;         /* first-moment block size B (Sec. 3: 128) */
+    int32_t v_block;         /* second-moment block size for 1-D tensors and LPMM_V_BLOCK (Sec. 4.2: 128) */
+    int32_t v_mode;          /* lpmm_vmode */
+    int64_t min_quant_numel; /* tensors with numel <= this keep fp32 states (App. C.1: 4096) */
+} lpmm_config;
+
+typedef struct lpmm_state lpmm_state; /* opaque host handle */
+
+/* State kind chosen per tensor (App. C.1 size rule; Sec. 4.2: a tensor that is 1-D, or has an
+ * extent of 1, uses block-wise normalization for v). */
+#define LPMM_KIND_FP32 0
+#define LPMM_KIND_BLOCK 1
+#define LPMM_KIND_RANK1 2
+
+/* Size in bytes of the device arena that holds the states of n tensors (codes, scales, fp32 states
+ * of small tensors, the device-side tensor table and the per-step scratch for the rank-1 maxima).
+ * Host-only; launches nothing. */
+lpmm_status lpmm_state_bytes(const lpmm_config* cfg, const lpmm_shape* shapes, int32_t n, size_t* arena_bytes);
+
+/* Alg. 1 / Alg. 3 "initial state 0": lays the arena out and enqueues its initialisation on `stream`
+ * (first-moment codes = the table's zero entry, second-moment codes 0, every scale 0, fp32 states 0;
+ * a zero scale dequantizes to exactly 0 whatever the code). d_arena must be 256-byte aligned and stay
+ * alive until lpmm_state_destroy. *out receives the handle. */
+lpmm_status lpmm_state_init(const lpmm_config* cfg, const lpmm_shape* shapes, int32_t n,
+                            void* d_arena, size_t arena_bytes, lpmm_state** out, void* stream);
+
+/* Re-creates a handle over an arena that already holds states (checkpoint restore): the arena bytes
+ * are a copy of an arena previously produced with the same cfg/shapes, `phase` is the value
+ * lpmm_state_phase() returned when that copy was taken. Only the tensor table is rewritten. */
+lpmm_status lpmm_state_attach(const lpmm_config* cfg, const lpmm_shape* shapes, int32_t n,
+                              void* d_arena, size_t arena_bytes, int32_t phase, lpmm_state** out, void* stream);
+
+/* One fused step of Alg. 3 over every tensor of the state: decompress m, v; Eq. 1 moment updates,
+ * bias correction, decoupled decay w <- w (1 - lr*wd), update w <- w - lr * m^/(sqrt(v^) + eps) with
+ * the un-quantized new moments; new block / row / column maxima; compress to the nearest code.
+ *   d_params[i] : device pointer to tensor i's fp32 parameters (updated in place)
+ *   d_grads[i]  : device pointer to tensor i's gradient in grad_dtype (read only)
+ * Both arrays are HOST arrays of n device pointers, each 16-byte aligned. step is t >= 1.
+ * Requires 0 <= beta1, beta2 < 1, lr >= 0, eps >= 0, weight_decay >= 0, all finite.
+ * Kernels launched: one pass over the rank-1 tensors that reduces the new row/column maxima, one
+ * small pass that inverts them, one pass over all tensors that updates and re-quantizes. */
+lpmm_status lpmm_adamw4_step(lpmm_state* st, void* const* d_params, const void* const* d_grads,
+                             int32_t grad_dtype, float lr, float beta1, float beta2, float eps,
+                             float weight_decay, int64_t step, void* stream);
+
+/* The same step for callers whose parameters and gradients live in HOST memory (optimizer
+ * offloading): copies every tensor's parameters and gradient into the caller's device staging
+ * buffers, runs lpmm_adamw4_step there and copies the updated parameters back, all on `stream`.
+ *   h_params[i], h_grads[i] : host pointers (pinned memory makes the copies asynchronous)
+ *   d_param_stage / d_grad_stage : device buffers of at least lpmm_stage_bytes() bytes each
+ * Returns after enqueueing; synchronize the stream before reading h_params. */
+lpmm_status lpmm_adamw4_step_host(lpmm_state* st, void* const* h_params, const void* const* h_grads,
+                                  int32_t grad_dtype, float lr, float beta1, float beta2, float eps,
+                                  float weight_decay, int64_t step,
+                                  void* d_param_stage, void* d_grad_stage, size_t stage_bytes, void* stream);
+
+/* Bytes needed by each staging buffer of lpmm_adamw4_step_host (tensors packed at 256-byte
+ * boundaries, 4 bytes per element). */
+lpmm_status lpmm_stage_bytes(const lpmm_state* st, size_t* bytes);
+
+/* Stand-alone quantizer Q = M o N of Sec. 2.2 for a rows x cols fp32 tensor (cols = 1 for 1-D).
+ *   norm BLOCK : d_scale0 receives ceil(numel/block) block maxima of |x| (block = 128 or 2048)
+ *   norm RANK1 : d_scale0 receives the rows row maxima, d_scale1 the cols column maxima (Sec. 4.2)
+ *   map DE_SIGNED (signed input) or LINEAR_NOZERO (meant for non-negative input: RANK1 takes |x|,
+ *       BLOCK keeps the sign and sends negative values to code 0)
+ * n = x * (1/scale) in fp32 (a scale below FLT_MIN counts as 0 and gives n = 0), code = nearest
+ * table entry, exact, lower entry on a tie. d_codes receives ceil(numel/2) bytes. RANK1 + DE_SIGNED
+ * is LPMM_ERR_UNSUPPORTED. With LPMM_Q_GIVEN_SCALES the scale buffers are inputs. */
+lpmm_status lpmm_quantize(const float* d_x, int64_t rows, int64_t cols, int32_t norm, int32_t map,
+                          int32_t block, uint32_t flags, uint8_t* d_codes, float* d_scale0, float* d_scale1,
+                          void* stream);
+
+/* Dequantizer of Sec. 2.2: d_out[i] = T(code_i) * scale_i, scale_i = block maximum or min(r, c). */
+lpmm_status lpmm_dequantize(const uint8_t* d_codes, const float* d_scale0, const float* d_scale1,
+                            int64_t rows, int64_t cols, int32_t norm, int32_t map, int32_t block,
+                            float* d_out, void* stream);
+
+/* Device pointers into the arena for tensor i's current state (for inspection and parity checks).
+ * Pointers that do not apply to the tensor's kind are set to NULL. Sizes: codes ceil(numel/2) bytes;
+ * m_scale ceil(numel/m_block); BLOCK v_scale0 ceil(numel/v_block); RANK1 v_scale0 rows, v_scale1 cols;
+ * FP32 m32/v32 numel floats. Valid until the next step (rank-1 scales alternate between two buffers). */
+lpmm_status lpmm_state_view(const lpmm_state* st, int32_t tensor, int32_t* kind,
+                            const uint8_t** m_codes, const float** m_scale,
+                            const uint8_t** v_codes, const float** v_scale0, const float** v_scale1,
+                            const float** m32, const float** v32);
+
+/* 0 or 1: which of the two rank-1 scale buffers is current. Save it with a copy of the arena. */
+int32_t lpmm_state_phase(const lpmm_state* st);
+
+/* Number of kernels and memsets the last lpmm_adamw4_step on this state enqueued. */
+int32_t lpmm_state_last_launches(const lpmm_state* st);
+
+/* Frees the host handle only; the arena stays the caller's. NULL is allowed. */
+void lpmm_state_destroy(lpmm_state* st);
+
+const char* lpmm_status_string(lpmm_status s);
+
+/* The cudaError_t (as int) of the most recent failed CUDA call made by this library in this thread. */
+int32_t lpmm_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LPMM_H */

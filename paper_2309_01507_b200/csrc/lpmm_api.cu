@@ -1,0 +1,455 @@
+// Host side of the C ABI declared in include/lpmm.h: argument validation, arena layout, the
+// device-side tensor table and the launch sequence of one step. No device memory is allocated here.
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/lpmm.h"
+#include "lpmm_internal.h"
+
+using namespace lpmm;
+
+namespace {
+
+thread_local int32_t g_last_cuda_error = 0;
+
+lpmm_status cuda_fail(cudaError_t e) {
+    g_last_cuda_error = (int32_t)e;
+    return LPMM_ERR_CUDA;
+}
+#define LPMM_CUDA(call)                                   \
+    do {                                                  \
+        cudaError_t e__ = (call);                         \
+        if (e__ != cudaSuccess) return cuda_fail(e__);    \
+    } while (0)
+
+constexpr size_t kAlign = 256;
+size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+struct TensorLayout {
+    int32_t kind;       // K_* of lpmm_internal.h
+    int64_t rows, cols, numel;
+    size_t m_codes, m_scale, v_codes, v_bscale, m32, v32;  // byte offsets into the arena (0 = unused)
+    int64_t rc_index;   // float index of this tensor's [r | c] inside each rank-1 scale buffer
+    int32_t c_off;
+};
+
+struct Layout {
+    std::vector<TensorLayout> t;
+    size_t descs = 0, params = 0, grads = 0, tiles1 = 0, tiles2 = 0;
+    size_t rc[2] = {0, 0}, rcp = 0;
+    int64_t rc_floats = 0;
+    size_t total = 0;
+};
+
+int public_kind(int32_t k) {
+    if (k == K_FP32) return LPMM_KIND_FP32;
+    if (k == K_BLOCK) return LPMM_KIND_BLOCK;
+    return LPMM_KIND_RANK1;
+}
+
+lpmm_status validate_config(const lpmm_config* cfg, const lpmm_shape* shapes, int32_t n) {
+    if (!cfg || !shapes || n <= 0) return LPMM_ERR_INVALID_ARG;
+    if (cfg->min_quant_numel < 0) return LPMM_ERR_INVALID_ARG;
+    if (cfg->v_mode != LPMM_V_RANK1 && cfg->v_mode != LPMM_V_BLOCK) return LPMM_ERR_INVALID_ARG;
+    if (cfg->bits != 4) return LPMM_ERR_UNSUPPORTED;
+    if (cfg->m_block != 128 || cfg->v_block != 128) return LPMM_ERR_UNSUPPORTED;
+    for (int32_t i = 0; i < n; ++i) {
+        const lpmm_shape& s = shapes[i];
+        if (s.rows <= 0 || s.cols <= 0) return LPMM_ERR_INVALID_ARG;
+        if (s.ndim != 1 && s.ndim != 2) return (s.ndim >= 3) ? LPMM_ERR_UNSUPPORTED : LPMM_ERR_INVALID_ARG;
+        if (s.ndim == 1 && s.cols != 1) return LPMM_ERR_INVALID_ARG;
+        if ((s.flags & LPMM_FORCE_QUANT) && (s.flags & LPMM_FORCE_FP32)) return LPMM_ERR_INVALID_ARG;
+        if (s.rows > (int64_t)1 << 40 || s.cols > (int64_t)1 << 40 || s.rows > ((int64_t)1 << 40) / s.cols)
+            return LPMM_ERR_INVALID_ARG;  // numel overflow guard
+        if (s.rows + s.cols > (int64_t)1 << 30) return LPMM_ERR_UNSUPPORTED;
+    }
+    return LPMM_OK;
+}
+
+int32_t choose_kind(const lpmm_config& cfg, const lpmm_shape& s) {
+    const int64_t numel = s.rows * s.cols;
+    if (s.flags & LPMM_FORCE_FP32) return K_FP32;
+    if (!(s.flags & LPMM_FORCE_QUANT) && numel <= cfg.min_quant_numel) return K_FP32;  // App. C.1
+    if (s.ndim == 1 || s.rows == 1 || s.cols == 1 || cfg.v_mode == LPMM_V_BLOCK) return K_BLOCK;  // Sec. 4.2
+    return (s.cols % 128 == 0) ? K_RANK1_FAST : K_RANK1_FLAT;
+}
+
+void compute_layout(const lpmm_config& cfg, const lpmm_shape* shapes, int32_t n, Layout* L) {
+    L->t.resize(n);
+    size_t off = kAlign;  // header block
+    L->descs = off;  off = align_up(off + sizeof(TensorDesc) * n);
+    L->params = off; off = align_up(off + sizeof(void*) * n);
+    L->grads = off;  off = align_up(off + sizeof(void*) * n);
+    L->tiles1 = off; off = align_up(off + sizeof(int32_t) * (n + 1));
+    L->tiles2 = off; off = align_up(off + sizeof(int32_t) * (n + 1));
+    int64_t rc = 0;
+    for (int32_t i = 0; i < n; ++i) {
+        TensorLayout& t = L->t[i];
+        t = TensorLayout{};
+        t.rows = shapes[i].rows; t.cols = shapes[i].cols; t.numel = t.rows * t.cols;
+        t.kind = choose_kind(cfg, shapes[i]);
+        if (t.kind == K_RANK1_FAST || t.kind == K_RANK1_FLAT) {
+            t.rc_index = rc;
+            t.c_off = (int32_t)((t.rows + 3) / 4 * 4);
+            rc += t.c_off + (t.cols + 3) / 4 * 4;
+            rc = (rc + 63) / 64 * 64;  // 256-byte granules so r and c always start 16-byte aligned
+        }
+    }
+    L->rc_floats = rc;
+    L->rc[0] = off; off = align_up(off + sizeof(float) * rc);
+    L->rc[1] = off; off = align_up(off + sizeof(float) * rc);
+    L->rcp = off;   off = align_up(off + sizeof(float) * rc);
+    for (int32_t i = 0; i < n; ++i) {
+        TensorLayout& t = L->t[i];
+        if (t.kind == K_FP32) {
+            t.m32 = off; off = align_up(off + sizeof(float) * t.numel);
+            t.v32 = off; off = align_up(off + sizeof(float) * t.numel);
+        } else {
+            const size_t code_bytes = (size_t)((t.numel + 1) / 2);
+            const size_t nblk = (size_t)((t.numel + 127) / 128);
+            t.m_codes = off; off = align_up(off + code_bytes);
+            t.v_codes = off; off = align_up(off + code_bytes);
+            t.m_scale = off; off = align_up(off + sizeof(float) * nblk);
+            if (t.kind == K_BLOCK) { t.v_bscale = off; off = align_up(off + sizeof(float) * nblk); }
+        }
+    }
+    L->total = off;
+}
+
+}  // namespace
+
+struct lpmm_state {
+    lpmm_config cfg;
+    int32_t n;
+    Layout L;
+    char* arena;
+    size_t arena_bytes;
+    int32_t phase;
+    int32_t grid1, grid2, total1, total2;
+    int32_t last_launches;
+    bool ptrs_valid;
+    std::vector<void*> params, grads;  // what the device-side pointer arrays currently hold
+    size_t stage_bytes;
+    std::vector<size_t> stage_off;
+};
+
+namespace {
+
+// Fills descriptors and tile tables, and uploads them. Tile sizes adapt to the amount of work so that
+// small parameter sets still spread over the whole GPU.
+lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
+    int dev = 0, sms = 0, occ1 = 1, occ2 = 1;
+    LPMM_CUDA(cudaGetDevice(&dev));
+    LPMM_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    LPMM_CUDA(step_kernel_occupancy(&occ1, &occ2));
+    if (occ1 < 1) occ1 = 1;
+    if (occ2 < 1) occ2 = 1;
+    const int32_t n = st->n;
+    int64_t total_elems = 0;
+    for (int32_t i = 0; i < n; ++i) total_elems += st->L.t[i].numel;
+    // aim at >= 4 tiles per resident CTA, tiles between 2 Ki and 32 Ki elements (powers of two)
+    int64_t target = total_elems / (4LL * sms * occ2);
+    int64_t tile_elems = 2048;
+    while (tile_elems * 2 <= target && tile_elems < 32768) tile_elems *= 2;
+
+    std::vector<TensorDesc> descs(n);
+    std::vector<int32_t> t1(n + 1, 0), t2(n + 1, 0);
+    char* A = st->arena;
+    for (int32_t i = 0; i < n; ++i) {
+        const TensorLayout& t = st->L.t[i];
+        TensorDesc& d = descs[i];
+        std::memset(&d, 0, sizeof(d));
+        d.rows = t.rows; d.cols = t.cols; d.numel = t.numel; d.kind = t.kind; d.c_off = t.c_off;
+        int64_t tiles = 0;
+        if (t.kind == K_FP32) {
+            d.m32 = reinterpret_cast<float*>(A + t.m32);
+            d.v32 = reinterpret_cast<float*>(A + t.v32);
+        } else {
+            d.m_codes = reinterpret_cast<uint8_t*>(A + t.m_codes);
+            d.v_codes = reinterpret_cast<uint8_t*>(A + t.v_codes);
+            d.m_scale = reinterpret_cast<float*>(A + t.m_scale);
+            if (t.kind == K_BLOCK) d.v_bscale = reinterpret_cast<float*>(A + t.v_bscale);
+            if (t.kind == K_RANK1_FAST || t.kind == K_RANK1_FLAT) {
+                d.rc[0] = reinterpret_cast<float*>(A + st->L.rc[0]) + t.rc_index;
+                d.rc[1] = reinterpret_cast<float*>(A + st->L.rc[1]) + t.rc_index;
+                d.rcp_new = reinterpret_cast<float*>(A + st->L.rcp) + t.rc_index;
+            }
+        }
+        if (t.kind == K_RANK1_FAST) {
+            d.wx = (t.cols % 1024 == 0) ? 4 : (t.cols % 512 == 0) ? 2 : 1;
+            const int64_t tile_cols = (int64_t)kWarpElems * d.wx;
+            int64_t tr = tile_elems / tile_cols;
+            if (tr < kWarps / d.wx) tr = kWarps / d.wx;
+            d.tile_rows = (int32_t)tr;
+            d.tiles_x = (int32_t)((t.cols + tile_cols - 1) / tile_cols);
+            tiles = (int64_t)d.tiles_x * ((t.rows + tr - 1) / tr);
+        } else {
+            int64_t chunks = tile_elems / (kWarps * kWarpElems);
+            if (chunks < 1) chunks = 1;
+            d.flat_chunks = (int32_t)chunks;
+            const int64_t per_tile = chunks * kWarps * kWarpElems;
+            tiles = (t.numel + per_tile - 1) / per_tile;
+        }
+        if (t2[i] + tiles > 0x7fffffffLL) return LPMM_ERR_UNSUPPORTED;
+        t2[i + 1] = t2[i] + (int32_t)tiles;
+        const bool rank1 = (t.kind == K_RANK1_FAST || t.kind == K_RANK1_FLAT);
+        t1[i + 1] = t1[i] + (rank1 ? (int32_t)tiles : 0);
+    }
+    st->total1 = t1[n];
+    st->total2 = t2[n];
+    st->grid1 = st->total1 < sms * occ1 ? st->total1 : sms * occ1;
+    st->grid2 = st->total2 < sms * occ2 ? st->total2 : sms * occ2;
+    LPMM_CUDA(cudaMemcpyAsync(A + st->L.descs, descs.data(), sizeof(TensorDesc) * n, cudaMemcpyHostToDevice, s));
+    LPMM_CUDA(cudaMemcpyAsync(A + st->L.tiles1, t1.data(), sizeof(int32_t) * (n + 1), cudaMemcpyHostToDevice, s));
+    LPMM_CUDA(cudaMemcpyAsync(A + st->L.tiles2, t2.data(), sizeof(int32_t) * (n + 1), cudaMemcpyHostToDevice, s));
+    // the vectors above are pageable memory: the runtime stages such copies before returning
+    return LPMM_OK;
+}
+
+lpmm_status make_state(const lpmm_config* cfg, const lpmm_shape* shapes, int32_t n, void* d_arena, size_t arena_bytes,
+                       bool fresh, int32_t phase, lpmm_state** out, void* stream) {
+    if (!out) return LPMM_ERR_INVALID_ARG;
+    *out = nullptr;
+    lpmm_status v = validate_config(cfg, shapes, n);
+    if (v != LPMM_OK) return v;
+    if (!d_arena) return LPMM_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(d_arena) % kAlign != 0) return LPMM_ERR_ALIGNMENT;
+    if (phase != 0 && phase != 1) return LPMM_ERR_INVALID_ARG;
+    lpmm_state* st = new (std::nothrow) lpmm_state();
+    if (!st) return LPMM_ERR_INVALID_ARG;
+    st->cfg = *cfg;
+    st->n = n;
+    compute_layout(*cfg, shapes, n, &st->L);
+    if (arena_bytes < st->L.total) { delete st; return LPMM_ERR_ARENA_TOO_SMALL; }
+    st->arena = static_cast<char*>(d_arena);
+    st->arena_bytes = arena_bytes;
+    st->phase = phase;
+    st->last_launches = 0;
+    st->ptrs_valid = false;
+    st->params.assign(n, nullptr);
+    st->grads.assign(n, nullptr);
+    st->stage_off.resize(n);
+    size_t so = 0;
+    for (int32_t i = 0; i < n; ++i) { st->stage_off[i] = so; so = align_up(so + 4 * (size_t)st->L.t[i].numel); }
+    st->stage_bytes = so;
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    lpmm_status rc = LPMM_OK;
+    if (fresh) {
+        // s_0 = 0 (Alg. 1): every scale 0, second-moment codes 0, fp32 states 0 ...
+        cudaError_t e = cudaMemsetAsync(d_arena, 0, st->L.total, s);
+        // ... and first-moment codes = 7, the zero entry of the signed table (an odd tail keeps nibble 0).
+        for (int32_t i = 0; i < n && e == cudaSuccess; ++i) {
+            const TensorLayout& t = st->L.t[i];
+            if (t.kind == K_FP32) continue;
+            e = cudaMemsetAsync(st->arena + t.m_codes, 0x77, (size_t)(t.numel / 2), s);
+            if (e == cudaSuccess && (t.numel & 1))
+                e = cudaMemsetAsync(st->arena + t.m_codes + t.numel / 2, 0x07, 1, s);
+        }
+        if (e != cudaSuccess) rc = cuda_fail(e);
+    }
+    if (rc == LPMM_OK) rc = build_tables(st, s);
+    if (rc != LPMM_OK) { delete st; return rc; }
+    *out = st;
+    return LPMM_OK;
+}
+
+bool finite_nonneg(float x) { return std::isfinite(x) && x >= 0.0f; }
+
+}  // namespace
+
+extern "C" {
+
+lpmm_status lpmm_state_bytes(const lpmm_config* cfg, const lpmm_shape* shapes, int32_t n, size_t* arena_bytes) {
+    if (!arena_bytes) return LPMM_ERR_INVALID_ARG;
+    lpmm_status v = validate_config(cfg, shapes, n);
+    if (v != LPMM_OK) return v;
+    Layout L;
+    compute_layout(*cfg, shapes, n, &L);
+    *arena_bytes = L.total;
+    return LPMM_OK;
+}
+
+lpmm_status lpmm_state_init(const lpmm_config* cfg, const lpmm_shape* shapes, int32_t n,
+                            void* d_arena, size_t arena_bytes, lpmm_state** out, void* stream) {
+    return make_state(cfg, shapes, n, d_arena, arena_bytes, true, 0, out, stream);
+}
+
+lpmm_status lpmm_state_attach(const lpmm_config* cfg, const lpmm_shape* shapes, int32_t n,
+                              void* d_arena, size_t arena_bytes, int32_t phase, lpmm_state** out, void* stream) {
+    return make_state(cfg, shapes, n, d_arena, arena_bytes, false, phase, out, stream);
+}
+
+lpmm_status lpmm_adamw4_step(lpmm_state* st, void* const* d_params, const void* const* d_grads,
+                             int32_t grad_dtype, float lr, float beta1, float beta2, float eps,
+                             float weight_decay, int64_t step, void* stream) {
+    if (!st || !d_params || !d_grads) return LPMM_ERR_INVALID_ARG;
+    if (grad_dtype != LPMM_F32 && grad_dtype != LPMM_BF16) return LPMM_ERR_INVALID_ARG;
+    if (step < 1) return LPMM_ERR_INVALID_ARG;
+    if (!finite_nonneg(lr) || !finite_nonneg(eps) || !finite_nonneg(weight_decay)) return LPMM_ERR_INVALID_ARG;
+    if (!finite_nonneg(beta1) || !finite_nonneg(beta2) || beta1 >= 1.0f || beta2 >= 1.0f) return LPMM_ERR_INVALID_ARG;
+    const int32_t n = st->n;
+    bool changed = !st->ptrs_valid;
+    for (int32_t i = 0; i < n; ++i) {
+        if (!d_params[i] || !d_grads[i]) return LPMM_ERR_INVALID_ARG;
+        if (!aligned16(d_params[i]) || !aligned16(d_grads[i])) return LPMM_ERR_ALIGNMENT;
+        if (d_params[i] != st->params[i] || d_grads[i] != st->grads[i]) changed = true;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int32_t launches = 0;
+    if (changed) {
+        for (int32_t i = 0; i < n; ++i) { st->params[i] = d_params[i]; st->grads[i] = const_cast<void*>(d_grads[i]); }
+        st->ptrs_valid = false;
+        LPMM_CUDA(cudaMemcpyAsync(st->arena + st->L.params, st->params.data(), sizeof(void*) * n, cudaMemcpyHostToDevice, s));
+        LPMM_CUDA(cudaMemcpyAsync(st->arena + st->L.grads, st->grads.data(), sizeof(void*) * n, cudaMemcpyHostToDevice, s));
+        st->ptrs_valid = true;
+    }
+
+    StepArgs a;
+    a.descs = reinterpret_cast<const TensorDesc*>(st->arena + st->L.descs);
+    a.params = reinterpret_cast<float* const*>(st->arena + st->L.params);
+    a.grads = reinterpret_cast<const void* const*>(st->arena + st->L.grads);
+    a.n_tensors = n;
+    a.phase = st->phase;
+    a.h.lr = lr; a.h.beta1 = beta1; a.h.beta2 = beta2; a.h.eps = eps;
+    a.h.omb1 = 1.0f - beta1;
+    a.h.omb2 = 1.0f - beta2;
+    a.h.bc1 = (float)(1.0 - std::pow((double)beta1, (double)step));   // Eq. 1: 1 - beta^t
+    a.h.bc2 = (float)(1.0 - std::pow((double)beta2, (double)step));
+    a.h.decay = 1.0f - lr * weight_decay;
+    const bool bf16 = (grad_dtype == LPMM_BF16);
+
+    if (st->total1 > 0) {
+        float* rc_new = reinterpret_cast<float*>(st->arena + st->L.rc[st->phase ^ 1]);
+        LPMM_CUDA(cudaMemsetAsync(rc_new, 0, sizeof(float) * st->L.rc_floats, s));
+        a.tile_start = reinterpret_cast<const int32_t*>(st->arena + st->L.tiles1);
+        a.total_tiles = st->total1;
+        LPMM_CUDA(launch_pass1(a, bf16, st->grid1, s));
+        LPMM_CUDA(launch_rcp(rc_new, reinterpret_cast<float*>(st->arena + st->L.rcp), st->L.rc_floats, s));
+        launches += 3;
+    }
+    a.tile_start = reinterpret_cast<const int32_t*>(st->arena + st->L.tiles2);
+    a.total_tiles = st->total2;
+    LPMM_CUDA(launch_pass2(a, bf16, st->grid2, s));
+    launches += 1;
+    st->phase ^= 1;
+    st->last_launches = launches;
+    return LPMM_OK;
+}
+
+lpmm_status lpmm_stage_bytes(const lpmm_state* st, size_t* bytes) {
+    if (!st || !bytes) return LPMM_ERR_INVALID_ARG;
+    *bytes = st->stage_bytes;
+    return LPMM_OK;
+}
+
+lpmm_status lpmm_adamw4_step_host(lpmm_state* st, void* const* h_params, const void* const* h_grads,
+                                  int32_t grad_dtype, float lr, float beta1, float beta2, float eps,
+                                  float weight_decay, int64_t step,
+                                  void* d_param_stage, void* d_grad_stage, size_t stage_bytes, void* stream) {
+    if (!st || !h_params || !h_grads || !d_param_stage || !d_grad_stage) return LPMM_ERR_INVALID_ARG;
+    if (grad_dtype != LPMM_F32 && grad_dtype != LPMM_BF16) return LPMM_ERR_INVALID_ARG;
+    if (stage_bytes < st->stage_bytes) return LPMM_ERR_ARENA_TOO_SMALL;
+    if (!aligned16(d_param_stage) || !aligned16(d_grad_stage)) return LPMM_ERR_ALIGNMENT;
+    const int32_t n = st->n;
+    for (int32_t i = 0; i < n; ++i) if (!h_params[i] || !h_grads[i]) return LPMM_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t gsz = (grad_dtype == LPMM_BF16) ? 2 : 4;
+    std::vector<void*> dp(n);
+    std::vector<const void*> dg(n);
+    for (int32_t i = 0; i < n; ++i) {
+        const size_t numel = (size_t)st->L.t[i].numel;
+        dp[i] = static_cast<char*>(d_param_stage) + st->stage_off[i];
+        dg[i] = static_cast<char*>(d_grad_stage) + st->stage_off[i];
+        LPMM_CUDA(cudaMemcpyAsync(dp[i], h_params[i], 4 * numel, cudaMemcpyHostToDevice, s));
+        LPMM_CUDA(cudaMemcpyAsync(const_cast<void*>(dg[i]), h_grads[i], gsz * numel, cudaMemcpyHostToDevice, s));
+    }
+    lpmm_status rc = lpmm_adamw4_step(st, dp.data(), dg.data(), grad_dtype, lr, beta1, beta2, eps, weight_decay, step, stream);
+    if (rc != LPMM_OK) return rc;
+    for (int32_t i = 0; i < n; ++i)
+        LPMM_CUDA(cudaMemcpyAsync(h_params[i], dp[i], 4 * (size_t)st->L.t[i].numel, cudaMemcpyDeviceToHost, s));
+    return LPMM_OK;
+}
+
+lpmm_status lpmm_quantize(const float* d_x, int64_t rows, int64_t cols, int32_t norm, int32_t map,
+                          int32_t block, uint32_t flags, uint8_t* d_codes, float* d_scale0, float* d_scale1,
+                          void* stream) {
+    if (!d_x || !d_codes || !d_scale0 || rows <= 0 || cols <= 0) return LPMM_ERR_INVALID_ARG;
+    if (norm != LPMM_NORM_BLOCK && norm != LPMM_NORM_RANK1) return LPMM_ERR_INVALID_ARG;
+    if (map != LPMM_MAP_DE_SIGNED && map != LPMM_MAP_LINEAR_NOZERO) return LPMM_ERR_INVALID_ARG;
+    if (flags & ~LPMM_Q_GIVEN_SCALES) return LPMM_ERR_INVALID_ARG;
+    if (rows > ((int64_t)1 << 40) / cols) return LPMM_ERR_INVALID_ARG;
+    if (norm == LPMM_NORM_RANK1) {
+        if (!d_scale1) return LPMM_ERR_INVALID_ARG;
+        if (map != LPMM_MAP_LINEAR_NOZERO) return LPMM_ERR_UNSUPPORTED;
+    } else if (block != 128 && block != 2048) {
+        return LPMM_ERR_UNSUPPORTED;
+    }
+    LPMM_CUDA(launch_quantize(d_x, rows, cols, norm, map, block, (flags & LPMM_Q_GIVEN_SCALES) != 0, d_codes,
+                              d_scale0, d_scale1, static_cast<cudaStream_t>(stream)));
+    return LPMM_OK;
+}
+
+lpmm_status lpmm_dequantize(const uint8_t* d_codes, const float* d_scale0, const float* d_scale1,
+                            int64_t rows, int64_t cols, int32_t norm, int32_t map, int32_t block,
+                            float* d_out, void* stream) {
+    if (!d_codes || !d_scale0 || !d_out || rows <= 0 || cols <= 0) return LPMM_ERR_INVALID_ARG;
+    if (norm != LPMM_NORM_BLOCK && norm != LPMM_NORM_RANK1) return LPMM_ERR_INVALID_ARG;
+    if (map != LPMM_MAP_DE_SIGNED && map != LPMM_MAP_LINEAR_NOZERO) return LPMM_ERR_INVALID_ARG;
+    if (rows > ((int64_t)1 << 40) / cols) return LPMM_ERR_INVALID_ARG;
+    if (norm == LPMM_NORM_RANK1) {
+        if (!d_scale1) return LPMM_ERR_INVALID_ARG;
+        if (map != LPMM_MAP_LINEAR_NOZERO) return LPMM_ERR_UNSUPPORTED;
+    } else if (block != 128 && block != 2048) {
+        return LPMM_ERR_UNSUPPORTED;
+    }
+    LPMM_CUDA(launch_dequantize(d_codes, d_scale0, d_scale1, rows, cols, norm, map, block, d_out,
+                                static_cast<cudaStream_t>(stream)));
+    return LPMM_OK;
+}
+
+lpmm_status lpmm_state_view(const lpmm_state* st, int32_t tensor, int32_t* kind,
+                            const uint8_t** m_codes, const float** m_scale,
+                            const uint8_t** v_codes, const float** v_scale0, const float** v_scale1,
+                            const float** m32, const float** v32) {
+    if (!st || tensor < 0 || tensor >= st->n) return LPMM_ERR_INVALID_ARG;
+    const TensorLayout& t = st->L.t[tensor];
+    const char* A = st->arena;
+    const bool q = (t.kind != K_FP32);
+    const bool r1 = (t.kind == K_RANK1_FAST || t.kind == K_RANK1_FLAT);
+    if (kind) *kind = public_kind(t.kind);
+    if (m_codes) *m_codes = q ? reinterpret_cast<const uint8_t*>(A + t.m_codes) : nullptr;
+    if (m_scale) *m_scale = q ? reinterpret_cast<const float*>(A + t.m_scale) : nullptr;
+    if (v_codes) *v_codes = q ? reinterpret_cast<const uint8_t*>(A + t.v_codes) : nullptr;
+    const float* rc = reinterpret_cast<const float*>(A + st->L.rc[st->phase]) + t.rc_index;
+    if (v_scale0) *v_scale0 = r1 ? rc : (t.kind == K_BLOCK ? reinterpret_cast<const float*>(A + t.v_bscale) : nullptr);
+    if (v_scale1) *v_scale1 = r1 ? rc + t.c_off : nullptr;
+    if (m32) *m32 = q ? nullptr : reinterpret_cast<const float*>(A + t.m32);
+    if (v32) *v32 = q ? nullptr : reinterpret_cast<const float*>(A + t.v32);
+    return LPMM_OK;
+}
+
+int32_t lpmm_state_phase(const lpmm_state* st) { return st ? st->phase : -1; }
+
+int32_t lpmm_state_last_launches(const lpmm_state* st) { return st ? st->last_launches : 0; }
+
+void lpmm_state_destroy(lpmm_state* st) { delete st; }
+
+const char* lpmm_status_string(lpmm_status s) {
+    switch (s) {
+        case LPMM_OK: return "ok";
+        case LPMM_ERR_INVALID_ARG: return "invalid argument";
+        case LPMM_ERR_UNSUPPORTED: return "unsupported configuration";
+        case LPMM_ERR_ALIGNMENT: return "pointer not sufficiently aligned";
+        case LPMM_ERR_ARENA_TOO_SMALL: return "arena or staging buffer too small";
+        case LPMM_ERR_CUDA: return "CUDA runtime error";
+        default: return "unknown status";
+    }
+}
+
+int32_t lpmm_last_cuda_error(void) { return g_last_cuda_error; }
+
+}  // extern "C"

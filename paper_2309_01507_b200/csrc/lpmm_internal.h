@@ -1,0 +1,62 @@
+// Internal structures shared by the host API and the kernels of the fused step.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "lpmm_device.cuh"
+
+namespace lpmm {
+
+// Work kinds inside the step kernels. RANK1_FAST needs cols % 128 == 0 (a 128-block then lies inside
+// one row and every row starts on a 16-byte boundary of every operand); other 2-D shapes take the
+// element-indexed RANK1_FLAT path.
+enum : int32_t { K_FP32 = 0, K_BLOCK = 1, K_RANK1_FAST = 2, K_RANK1_FLAT = 3 };
+
+constexpr int kThreads = 256;          // threads per CTA in the step kernels
+constexpr int kWarps = kThreads / 32;
+constexpr int kLaneElems = 8;          // consecutive elements per lane
+constexpr int kWarpElems = 32 * kLaneElems;  // 256: two 128-element blocks per warp
+
+// One entry of the device-side tensor table (lives at the head of the arena).
+struct TensorDesc {
+    uint8_t* m_codes;   // ceil(numel/2) bytes
+    float* m_scale;     // ceil(numel/128) block maxima of |m|
+    uint8_t* v_codes;
+    float* v_bscale;    // K_BLOCK: ceil(numel/128) block maxima of v
+    float* rc[2];       // K_RANK1_*: two buffers of [r (rows, padded to 4) | c (cols)]
+    float* rcp_new;     // K_RANK1_*: reciprocals of the new r, c (same layout), per-step scratch
+    float* m32;         // K_FP32
+    float* v32;
+    int64_t rows, cols, numel;
+    int32_t kind;
+    int32_t c_off;      // float offset of c inside rc[] and rcp_new
+    int32_t wx;         // K_RANK1_FAST: warps across a tile (1, 2 or 4); tile is 256*wx columns wide
+    int32_t tiles_x;    // K_RANK1_FAST: column tiles
+    int32_t tile_rows;  // K_RANK1_FAST: rows per tile
+    int32_t flat_chunks;  // other kinds: 256-element chunks per warp per tile
+    int32_t pad[2];
+};
+
+struct StepArgs {
+    const TensorDesc* descs;
+    float* const* params;        // n device pointers, fp32
+    const void* const* grads;    // n device pointers
+    const int32_t* tile_start;   // n + 1 prefix sums of tiles (pass-specific)
+    int32_t n_tensors;
+    int32_t total_tiles;
+    int32_t phase;               // rc[phase] holds the current r, c; rc[1 - phase] receives the new ones
+    Hyper h;
+};
+
+cudaError_t launch_pass1(const StepArgs& a, bool bf16, int grid, cudaStream_t s);
+cudaError_t launch_pass2(const StepArgs& a, bool bf16, int grid, cudaStream_t s);
+cudaError_t launch_rcp(const float* src, float* dst, int64_t n, cudaStream_t s);
+cudaError_t step_kernel_occupancy(int* pass1_blocks_per_sm, int* pass2_blocks_per_sm);
+
+cudaError_t launch_quantize(const float* x, int64_t rows, int64_t cols, int norm, int map, int block,
+                            bool given, uint8_t* codes, float* s0, float* s1, cudaStream_t s);
+cudaError_t launch_dequantize(const uint8_t* codes, const float* s0, const float* s1, int64_t rows, int64_t cols,
+                              int norm, int map, int block, float* out, cudaStream_t s);
+
+}  // namespace lpmm

@@ -1,0 +1,444 @@
+// Kernels of the fused 4-bit AdamW step (Alg. 3 with Eq. 1) for sm_100a.
+//
+// One step is three launches over a device-side tensor table:
+//   pass 1  (rank-1 tensors only) recomputes the new second moment v_t from the gradient and the old
+//           codes and reduces its row and column maxima r', c' (Sec. 4.2) with an unsigned atomicMax
+//           on the float bit patterns (v_t >= 0);
+//   rcp     inverts r', c' once (1/s, or 0 for a scale below FLT_MIN);
+//   pass 2  (all tensors) dequantizes m and v, applies the moment updates, bias correction, decoupled
+//           decay and the parameter update, reduces each 128-block's |m_t| maximum inside 16 lanes,
+//           and re-quantizes both moments to the nearest code, two codes per byte.
+// Work is cut into tiles; tile -> tensor is a binary search over prefix sums, so one launch covers
+// every tensor. A lane always owns 8 consecutive elements: 32 B of fp32 parameters, 16 B of bf16 (32 B
+// of fp32) gradient and one 32-bit word of each moment's codes; 16 lanes own one 128-element block.
+#include "lpmm_internal.h"
+
+namespace lpmm {
+
+namespace {
+
+__device__ __forceinline__ int find_tensor(const int32_t* __restrict__ start, int n, int tile) {
+    int lo = 0, hi = n;  // invariant: start[lo] <= tile < start[hi]
+    while (hi - lo > 1) {
+        int mid = (lo + hi) >> 1;
+        if (__ldg(start + mid) <= tile) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+// ---- 8-element loads ------------------------------------------------------------------------
+
+__device__ __forceinline__ void load8_f32(const float* p, float (&x)[8]) {
+    float4 a = __ldg(reinterpret_cast<const float4*>(p));
+    float4 b = __ldg(reinterpret_cast<const float4*>(p) + 1);
+    x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+}
+__device__ __forceinline__ void load8_rw(const float* p, float (&x)[8]) {  // read-modify-write data: no __ldg
+    float4 a = *reinterpret_cast<const float4*>(p);
+    float4 b = *(reinterpret_cast<const float4*>(p) + 1);
+    x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+}
+__device__ __forceinline__ void store8_f32(float* p, const float (&x)[8]) {
+    *reinterpret_cast<float4*>(p) = make_float4(x[0], x[1], x[2], x[3]);
+    *(reinterpret_cast<float4*>(p) + 1) = make_float4(x[4], x[5], x[6], x[7]);
+}
+__device__ __forceinline__ void load8_bf16(const uint16_t* p, float (&x)[8]) {
+    uint4 r = __ldg(reinterpret_cast<const uint4*>(p));
+    x[0] = bf16_lo(r.x); x[1] = bf16_hi(r.x); x[2] = bf16_lo(r.y); x[3] = bf16_hi(r.y);
+    x[4] = bf16_lo(r.z); x[5] = bf16_hi(r.z); x[6] = bf16_lo(r.w); x[7] = bf16_hi(r.w);
+}
+template <bool BF16>
+__device__ __forceinline__ void load8_grad(const void* g, int64_t e, float (&x)[8]) {
+    if (BF16) load8_bf16(reinterpret_cast<const uint16_t*>(g) + e, x);
+    else load8_f32(reinterpret_cast<const float*>(g) + e, x);
+}
+template <bool BF16>
+__device__ __forceinline__ float load1_grad(const void* g, int64_t e) {
+    if (BF16) return __uint_as_float(((uint32_t)__ldg(reinterpret_cast<const uint16_t*>(g) + e)) << 16);
+    return __ldg(reinterpret_cast<const float*>(g) + e);
+}
+
+// Guarded variants for the ragged end of a tensor: elements at or beyond `numel` read as zero.
+template <bool BF16>
+__device__ __forceinline__ void load8_grad_guard(const void* g, int64_t e, int64_t numel, float (&x)[8]) {
+#pragma unroll
+    for (int k = 0; k < 8; ++k) x[k] = (e + k < numel) ? load1_grad<BF16>(g, e + k) : 0.0f;
+}
+__device__ __forceinline__ void load8_guard(const float* p, int64_t e, int64_t numel, float (&x)[8]) {
+#pragma unroll
+    for (int k = 0; k < 8; ++k) x[k] = (e + k < numel) ? p[e + k] : 0.0f;
+}
+__device__ __forceinline__ void store8_guard(float* p, int64_t e, int64_t numel, const float (&x)[8]) {
+#pragma unroll
+    for (int k = 0; k < 8; ++k) if (e + k < numel) p[e + k] = x[k];
+}
+// 8 codes of elements e..e+7 (e is a multiple of 8); bytes beyond the tensor read as 0.
+__device__ __forceinline__ uint32_t load_codes_guard(const uint8_t* codes, int64_t e, int64_t numel) {
+    int64_t nbytes = (numel + 1) >> 1;
+    uint32_t q = 0;
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+        int64_t byte = (e >> 1) + b;
+        if (byte < nbytes) q |= ((uint32_t)codes[byte]) << (8 * b);
+    }
+    return q;
+}
+// Stores the codes of the valid elements; a trailing odd element leaves its byte's high nibble 0.
+__device__ __forceinline__ void store_codes_guard(uint8_t* codes, int64_t e, int64_t numel, uint32_t q) {
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+        int64_t lo = e + 2 * b;
+        if (lo < numel) {
+            uint32_t byte = (q >> (8 * b)) & 0xffu;
+            if (lo + 1 >= numel) byte &= 0x0fu;
+            codes[lo >> 1] = (uint8_t)byte;
+        }
+    }
+}
+
+// ---- per-lane arithmetic ----------------------------------------------------------------------
+
+// Dequantize (Sec. 2.2), update the moments (Eq. 1) and the parameters for 8 elements.
+// vs[k] is the old scale of element k's second moment, am the old scale of its first-moment block.
+__device__ __forceinline__ void moments_and_update8(float (&w)[8], const float (&g)[8], uint32_t qm, uint32_t qv,
+                                                    float am, const float (&vs)[8], const Hyper& h,
+                                                    const float* s_de, float (&mt)[8], float (&vt)[8]) {
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        float m = __fmul_rn(s_de[(qm >> (4 * k)) & 15u], am);
+        float v = __fmul_rn(lin_value((qv >> (4 * k)) & 15u), vs[k]);
+        mt[k] = ema_m(m, g[k], h);
+        vt[k] = ema_v(v, g[k], h);
+        w[k] = adam_update(w[k], mt[k], vt[k], h);
+    }
+}
+
+__device__ __forceinline__ float absmax8(const float (&x)[8]) {
+    float a = 0.0f;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) a = fmaxf(a, fabsf(x[k]));
+    return a;
+}
+
+__device__ __forceinline__ uint32_t quantize8_de(const float (&x)[8], float rcp) {
+    uint32_t q = 0;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) q |= de_nearest(__fmul_rn(x[k], rcp)) << (4 * k);
+    return q;
+}
+__device__ __forceinline__ uint32_t quantize8_lin(const float (&x)[8], const float (&rcp)[8]) {
+    uint32_t q = 0;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) q |= lin_nearest(__fmul_rn(x[k], rcp[k])) << (4 * k);
+    return q;
+}
+
+// ---- pass 2, rank-1 tensors with cols % 128 == 0 ---------------------------------------------------
+
+template <bool BF16>
+__device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __restrict__ w, const void* __restrict__ g,
+                                                 int tile, int phase, const Hyper& h, const float* s_de) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int wx = d.wx, wy_count = kWarps / wx;
+    const int tx = tile % d.tiles_x, ty = tile / d.tiles_x;
+    const int64_t col0 = (int64_t)tx * (kWarpElems * wx) + (warp % wx) * kWarpElems + lane * kLaneElems;
+    const bool active = col0 < d.cols;
+    const float* rc_old = d.rc[phase];
+    const float* rcp_new = d.rcp_new;
+    float* m_scale = d.m_scale;
+
+    float c_old[8], c_rcp[8];
+    if (active) {
+        load8_f32(rc_old + d.c_off + col0, c_old);
+        load8_f32(rcp_new + d.c_off + col0, c_rcp);
+    }
+    const int64_t row_end = min((int64_t)(ty + 1) * d.tile_rows, d.rows);
+    for (int64_t i = (int64_t)ty * d.tile_rows + warp / wx; i < row_end; i += wy_count) {
+        float wv[8], gv[8], mt[8], vt[8], vs[8], vr[8];
+        uint32_t qm = 0, qv = 0;
+        float am_new = 0.0f;
+        const int64_t e = i * d.cols + col0;
+        if (active) {
+            load8_rw(w + e, wv);
+            load8_grad<BF16>(g, e, gv);
+            qm = __ldg(reinterpret_cast<const uint32_t*>(d.m_codes + (e >> 1)));
+            qv = __ldg(reinterpret_cast<const uint32_t*>(d.v_codes + (e >> 1)));
+            const float am = m_scale[e >> 7];
+            const float r_old = __ldg(rc_old + i);
+            const float r_rcp = __ldg(rcp_new + i);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                vs[k] = fminf(r_old, c_old[k]);      // Sec. 4.2: scale = min(r_i, c_j)
+                vr[k] = fmaxf(r_rcp, c_rcp[k]);      // 1/min(r', c') = max(1/r', 1/c')
+            }
+            moments_and_update8(wv, gv, qm, qv, am, vs, h, s_de, mt, vt);
+            store8_f32(w + e, wv);
+            am_new = absmax8(mt);
+        }
+        am_new = half_warp_max(am_new);              // all 32 lanes take part in the shuffles
+        if (active) {
+            if ((lane & 15) == 0) m_scale[e >> 7] = am_new;
+            *reinterpret_cast<uint32_t*>(d.m_codes + (e >> 1)) = quantize8_de(mt, scale_rcp(am_new));
+            *reinterpret_cast<uint32_t*>(d.v_codes + (e >> 1)) = quantize8_lin(vt, vr);
+        }
+    }
+}
+
+// ---- pass 2, flat (element-indexed) tensors: block-wise v, or rank-1 with arbitrary cols ------
+
+template <bool BF16, bool RANK1>
+__device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restrict__ w, const void* __restrict__ g,
+                                           int tile, int phase, const Hyper& h, const float* s_de) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const float* rc_old = d.rc[phase];
+    const float* rcp_new = d.rcp_new;
+    for (int c = 0; c < d.flat_chunks; ++c) {
+        const int64_t chunk = ((int64_t)tile * d.flat_chunks + c) * kWarps + warp;
+        const int64_t e = chunk * kWarpElems + lane * kLaneElems;
+        if (chunk * kWarpElems >= d.numel) break;          // uniform per warp
+        const bool full = (chunk + 1) * kWarpElems <= d.numel;
+        float wv[8], gv[8], mt[8], vt[8], vs[8], vr[8];
+        uint32_t qm, qv;
+        if (full) {
+            load8_rw(w + e, wv);
+            load8_grad<BF16>(g, e, gv);
+            qm = __ldg(reinterpret_cast<const uint32_t*>(d.m_codes + (e >> 1)));
+            qv = __ldg(reinterpret_cast<const uint32_t*>(d.v_codes + (e >> 1)));
+        } else {
+            load8_guard(w, e, d.numel, wv);
+            load8_grad_guard<BF16>(g, e, d.numel, gv);
+            qm = load_codes_guard(d.m_codes, e, d.numel);
+            qv = load_codes_guard(d.v_codes, e, d.numel);
+        }
+        const bool lane_live = e < d.numel;
+        const float am = lane_live ? d.m_scale[e >> 7] : 0.0f;
+        if (RANK1) {
+            int64_t i = e / d.cols, j = e - i * d.cols;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                if (e + k < d.numel) {
+                    vs[k] = fminf(__ldg(rc_old + i), __ldg(rc_old + d.c_off + j));
+                    vr[k] = fmaxf(__ldg(rcp_new + i), __ldg(rcp_new + d.c_off + j));
+                } else {
+                    vs[k] = 0.0f; vr[k] = 0.0f;
+                }
+                if (++j == d.cols) { j = 0; ++i; }
+            }
+        } else {
+            const float av = lane_live ? d.v_bscale[e >> 7] : 0.0f;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) vs[k] = av;
+        }
+        moments_and_update8(wv, gv, qm, qv, am, vs, h, s_de, mt, vt);
+        if (!full) {   // elements beyond the tensor must not reach a block maximum
+#pragma unroll
+            for (int k = 0; k < 8; ++k) if (e + k >= d.numel) { mt[k] = 0.0f; vt[k] = 0.0f; }
+        }
+        const float am_new = half_warp_max(absmax8(mt));
+        if (!RANK1) {
+            const float av_new = half_warp_max(absmax8(vt));
+            const float r = scale_rcp(av_new);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) vr[k] = r;
+            if (lane_live && (lane & 15) == 0) d.v_bscale[e >> 7] = av_new;
+        }
+        if (lane_live && (lane & 15) == 0) d.m_scale[e >> 7] = am_new;
+        const uint32_t qm_new = quantize8_de(mt, scale_rcp(am_new));
+        const uint32_t qv_new = quantize8_lin(vt, vr);
+        if (full) {
+            store8_f32(w + e, wv);
+            *reinterpret_cast<uint32_t*>(d.m_codes + (e >> 1)) = qm_new;
+            *reinterpret_cast<uint32_t*>(d.v_codes + (e >> 1)) = qv_new;
+        } else {
+            store8_guard(w, e, d.numel, wv);
+            store_codes_guard(d.m_codes, e, d.numel, qm_new);
+            store_codes_guard(d.v_codes, e, d.numel, qv_new);
+        }
+    }
+}
+
+// ---- pass 2, small tensors with fp32 states (App. C.1) ------------------------------------------
+
+template <bool BF16>
+__device__ __forceinline__ void pass2_fp32(const TensorDesc& d, float* __restrict__ w, const void* __restrict__ g,
+                                           int tile, const Hyper& h) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int c = 0; c < d.flat_chunks; ++c) {
+        const int64_t chunk = ((int64_t)tile * d.flat_chunks + c) * kWarps + warp;
+        const int64_t e = chunk * kWarpElems + lane * kLaneElems;
+        if (chunk * kWarpElems >= d.numel) break;
+        const bool full = (chunk + 1) * kWarpElems <= d.numel;
+        float wv[8], gv[8], m[8], v[8];
+        if (full) {
+            load8_rw(w + e, wv); load8_grad<BF16>(g, e, gv); load8_rw(d.m32 + e, m); load8_rw(d.v32 + e, v);
+        } else {
+            load8_guard(w, e, d.numel, wv); load8_grad_guard<BF16>(g, e, d.numel, gv);
+            load8_guard(d.m32, e, d.numel, m); load8_guard(d.v32, e, d.numel, v);
+        }
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            m[k] = ema_m(m[k], gv[k], h);
+            v[k] = ema_v(v[k], gv[k], h);
+            wv[k] = adam_update(wv[k], m[k], v[k], h);
+        }
+        if (full) {
+            store8_f32(w + e, wv); store8_f32(d.m32 + e, m); store8_f32(d.v32 + e, v);
+        } else {
+            store8_guard(w, e, d.numel, wv); store8_guard(d.m32, e, d.numel, m); store8_guard(d.v32, e, d.numel, v);
+        }
+    }
+}
+
+template <bool BF16>
+__global__ void __launch_bounds__(kThreads, 2) pass2_kernel(StepArgs a) {
+    __shared__ float s_de[16];
+    if (threadIdx.x < 16) s_de[threadIdx.x] = kDeTable[threadIdx.x];
+    __syncthreads();
+    for (int tile = blockIdx.x; tile < a.total_tiles; tile += gridDim.x) {
+        const int t = find_tensor(a.tile_start, a.n_tensors, tile);
+        const TensorDesc& d = a.descs[t];
+        float* w = a.params[t];
+        const void* g = a.grads[t];
+        const int local = tile - __ldg(a.tile_start + t);
+        switch (d.kind) {
+            case K_RANK1_FAST: pass2_rank1_fast<BF16>(d, w, g, local, a.phase, a.h, s_de); break;
+            case K_RANK1_FLAT: pass2_flat<BF16, true>(d, w, g, local, a.phase, a.h, s_de); break;
+            case K_BLOCK:      pass2_flat<BF16, false>(d, w, g, local, a.phase, a.h, s_de); break;
+            default:           pass2_fp32<BF16>(d, w, g, local, a.h); break;
+        }
+    }
+}
+
+// ---- pass 1: new row / column maxima of v_t for rank-1 tensors -----------------------------------
+
+template <bool BF16>
+__device__ __forceinline__ void pass1_rank1_fast(const TensorDesc& d, const void* __restrict__ g, int tile, int phase,
+                                                 const Hyper& h, float* s_col) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int wx = d.wx, wy_count = kWarps / wx;
+    const int tx = tile % d.tiles_x, ty = tile / d.tiles_x;
+    const int64_t col0 = (int64_t)tx * (kWarpElems * wx) + (warp % wx) * kWarpElems + lane * kLaneElems;
+    const bool active = col0 < d.cols;
+    const float* rc_old = d.rc[phase];
+    float* rc_new = d.rc[phase ^ 1];
+
+    float c_old[8], c_max[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) { c_old[k] = 0.0f; c_max[k] = 0.0f; }
+    if (active) load8_f32(rc_old + d.c_off + col0, c_old);
+    const int64_t row_end = min((int64_t)(ty + 1) * d.tile_rows, d.rows);
+    for (int64_t i = (int64_t)ty * d.tile_rows + warp / wx; i < row_end; i += wy_count) {
+        float r_max = 0.0f;
+        if (active) {
+            const int64_t e = i * d.cols + col0;
+            float gv[8];
+            load8_grad<BF16>(g, e, gv);
+            const uint32_t qv = __ldg(reinterpret_cast<const uint32_t*>(d.v_codes + (e >> 1)));
+            const float r_old = __ldg(rc_old + i);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                float v = __fmul_rn(lin_value((qv >> (4 * k)) & 15u), fminf(r_old, c_old[k]));
+                float vt = ema_v(v, gv[k], h);
+                r_max = fmaxf(r_max, vt);
+                c_max[k] = fmaxf(c_max[k], vt);
+            }
+        }
+        r_max = warp_max(r_max);
+        if (lane == 0 && active) atomic_max_nonneg(rc_new + i, r_max);
+    }
+    // Column maxima: combine the warps that share columns in shared memory, then one atomic per column.
+    float* mine = s_col + warp * kWarpElems + lane * kLaneElems;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) mine[k] = c_max[k];
+    __syncthreads();
+    if (warp < wx) {   // warp `warp` owns column group warp % wx == warp
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            // lane-contiguous layout for the atomics: column = lane + 32 k within the 256-column group
+            const int cc = lane + 32 * k;
+            float mx = 0.0f;
+            for (int y = 0; y < wy_count; ++y) mx = fmaxf(mx, s_col[(y * wx + warp) * kWarpElems + cc]);
+            const int64_t col = (int64_t)tx * (kWarpElems * wx) + warp * kWarpElems + cc;
+            if (col < d.cols) atomic_max_nonneg(rc_new + d.c_off + col, mx);
+        }
+    }
+    __syncthreads();
+}
+
+template <bool BF16>
+__device__ __forceinline__ void pass1_rank1_flat(const TensorDesc& d, const void* __restrict__ g, int tile, int phase,
+                                                 const Hyper& h) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const float* rc_old = d.rc[phase];
+    float* rc_new = d.rc[phase ^ 1];
+    for (int c = 0; c < d.flat_chunks; ++c) {
+        const int64_t chunk = ((int64_t)tile * d.flat_chunks + c) * kWarps + warp;
+        const int64_t e = chunk * kWarpElems + lane * kLaneElems;
+        if (chunk * kWarpElems >= d.numel) break;
+        if (e >= d.numel) continue;
+        float gv[8];
+        load8_grad_guard<BF16>(g, e, d.numel, gv);
+        const uint32_t qv = load_codes_guard(d.v_codes, e, d.numel);
+        int64_t i = e / d.cols, j = e - i * d.cols;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            if (e + k < d.numel) {
+                const float s = fminf(__ldg(rc_old + i), __ldg(rc_old + d.c_off + j));
+                const float vt = ema_v(__fmul_rn(lin_value((qv >> (4 * k)) & 15u), s), gv[k], h);
+                atomic_max_nonneg(rc_new + i, vt);
+                atomic_max_nonneg(rc_new + d.c_off + j, vt);
+            }
+            if (++j == d.cols) { j = 0; ++i; }
+        }
+    }
+}
+
+template <bool BF16>
+__global__ void __launch_bounds__(kThreads, 2) pass1_kernel(StepArgs a) {
+    __shared__ float s_col[kWarps * kWarpElems];
+    for (int tile = blockIdx.x; tile < a.total_tiles; tile += gridDim.x) {
+        const int t = find_tensor(a.tile_start, a.n_tensors, tile);
+        const TensorDesc& d = a.descs[t];
+        const void* g = a.grads[t];
+        const int local = tile - __ldg(a.tile_start + t);
+        if (d.kind == K_RANK1_FAST) pass1_rank1_fast<BF16>(d, g, local, a.phase, a.h, s_col);
+        else pass1_rank1_flat<BF16>(d, g, local, a.phase, a.h);
+    }
+}
+
+__global__ void rcp_kernel(const float* __restrict__ src, float* __restrict__ dst, int64_t n) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+        dst[i] = scale_rcp(src[i]);
+}
+
+}  // namespace
+
+cudaError_t launch_pass1(const StepArgs& a, bool bf16, int grid, cudaStream_t s) {
+    if (a.total_tiles <= 0) return cudaSuccess;
+    if (bf16) pass1_kernel<true><<<grid, kThreads, 0, s>>>(a);
+    else pass1_kernel<false><<<grid, kThreads, 0, s>>>(a);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_pass2(const StepArgs& a, bool bf16, int grid, cudaStream_t s) {
+    if (a.total_tiles <= 0) return cudaSuccess;
+    if (bf16) pass2_kernel<true><<<grid, kThreads, 0, s>>>(a);
+    else pass2_kernel<false><<<grid, kThreads, 0, s>>>(a);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_rcp(const float* src, float* dst, int64_t n, cudaStream_t s) {
+    if (n <= 0) return cudaSuccess;
+    int grid = (int)((n + 255) / 256);
+    if (grid > 2048) grid = 2048;
+    rcp_kernel<<<grid, 256, 0, s>>>(src, dst, n);
+    return cudaGetLastError();
+}
+
+cudaError_t step_kernel_occupancy(int* p1, int* p2) {
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(p1, pass1_kernel<true>, kThreads, 0);
+    if (e != cudaSuccess) return e;
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(p2, pass2_kernel<true>, kThreads, 0);
+}
+
+}  // namespace lpmm

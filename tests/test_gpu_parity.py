@@ -1,0 +1,245 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle on the same seeded inputs.
+
+Bar: packed codes and scales bit for bit; parameters within 1e-6 * max(|w|, lr) after one step from a
+shared state; over a 100-step trajectory parameters within 1e-4 and at most 1e-6 of the codes off by
+one adjacent code (none is expected: the state path never reads the parameters).
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2309_01507_b200 import lpmm, workloads
+from paper_2309_01507_b200.workloads import TensorSpec
+from parity_util import Pair, hyper_of
+
+pytestmark = pytest.mark.gpu
+
+TDE = oracle.de_map(4, True)
+TLIN = oracle.linear_map(4)
+
+
+def _mat(r, c, **kw):
+    return TensorSpec(f"m{r}x{c}", r, c, 2, **kw)
+
+
+def _vec(n, **kw):
+    return TensorSpec(f"v{n}", n, 1, 1, **kw)
+
+
+# ------------------------------------------------------------------ stand-alone quantizer
+
+def _threshold_probe():
+    pts = [0.0, -0.0, 1.0, -1.0, 1.5, -1.5, 1e-30, -1e-30, 1e-45]
+    for T in (TDE, TLIN):
+        for a, b in zip(T[:-1], T[1:]):
+            p = np.float32((float(a) + float(b)) / 2)
+            for _ in range(6):
+                p = np.nextafter(p, np.float32(-np.inf), dtype=np.float32)
+            for _ in range(13):
+                pts.append(float(p))
+                p = np.nextafter(p, np.float32(np.inf), dtype=np.float32)
+        pts += [float(t) for t in T]
+    rng = np.random.default_rng(0)
+    pts += list(rng.uniform(-1.1, 1.1, 3000))
+    x = np.array(pts, dtype=np.float32)
+    pad = (-x.size) % 128
+    return np.concatenate([x, np.zeros(pad, np.float32)])
+
+
+@pytest.mark.parametrize("map_, T", [(lpmm.MAP_DE_SIGNED, TDE), (lpmm.MAP_LINEAR_NOZERO, TLIN)])
+def test_nearest_entry_at_every_threshold(map_, T):
+    x = _threshold_probe()
+    ones = torch.ones(x.size // 128, device="cuda")
+    codes, _, _ = lpmm.quantize(torch.from_numpy(x).cuda(), lpmm.NORM_BLOCK, map_, 128, scales=(ones, None))
+    want, _ = oracle.quantize_block(x, 128, T, scale=np.ones(x.size // 128, np.float32))
+    assert np.array_equal(codes.cpu().numpy(), oracle.pack4(want))
+
+
+@pytest.mark.parametrize("numel,block", [(1, 128), (127, 128), (128, 128), (129, 128), (50265, 128), (5000, 2048),
+                                         (128 * 2000 + 3, 128), (2048 * 37 + 1111, 2048)])
+@pytest.mark.parametrize("map_", [lpmm.MAP_DE_SIGNED, lpmm.MAP_LINEAR_NOZERO])
+def test_block_quantizer_matches_oracle(numel, block, map_):
+    rng = np.random.default_rng(numel)
+    x = (rng.standard_normal(numel) * np.exp(2 * rng.standard_normal(numel))).astype(np.float32)
+    if map_ == lpmm.MAP_LINEAR_NOZERO:
+        x = x * x
+    T = TDE if map_ == lpmm.MAP_DE_SIGNED else TLIN
+    codes, s0, _ = lpmm.quantize(torch.from_numpy(x).cuda(), lpmm.NORM_BLOCK, map_, block)
+    want, ws = oracle.quantize_block(x, block, T)
+    assert np.array_equal(s0.cpu().numpy(), ws)
+    assert np.array_equal(codes.cpu().numpy(), oracle.pack4(want))
+    deq = lpmm.dequantize(codes, s0, None, numel, 1, lpmm.NORM_BLOCK, map_, block)
+    assert np.array_equal(deq.cpu().numpy(), oracle.dequantize_block(want, block, T, ws))
+    # round trip with the stored scales reproduces every code
+    codes2, _, _ = lpmm.quantize(deq, lpmm.NORM_BLOCK, map_, block, scales=(s0, None))
+    assert torch.equal(codes, codes2)
+
+
+@pytest.mark.parametrize("rows,cols", [(2, 3), (1, 300), (300, 1), (37, 53), (96, 256), (513, 1000), (1024, 4096)])
+def test_rank1_quantizer_matches_oracle(rows, cols):
+    rng = np.random.default_rng(rows * 31 + cols)
+    x = (rng.standard_normal((rows, cols)) * np.exp(rng.standard_normal((rows, 1))) *
+         np.exp(rng.standard_normal((1, cols)))).astype(np.float32) ** 2
+    x[rng.random((rows, cols)) < 0.01] = 0
+    if rows > 4:
+        x[3, :] = 0
+    codes, r, c = lpmm.quantize(torch.from_numpy(x).cuda(), lpmm.NORM_RANK1, lpmm.MAP_LINEAR_NOZERO)
+    want, wr, wc = oracle.quantize_rank1(x, TLIN)
+    assert np.array_equal(r.cpu().numpy(), wr) and np.array_equal(c.cpu().numpy(), wc)
+    assert np.array_equal(codes.cpu().numpy(), oracle.pack4(want))
+    deq = lpmm.dequantize(codes, r, c, rows, cols, lpmm.NORM_RANK1, lpmm.MAP_LINEAR_NOZERO)
+    ref = oracle.dequantize_rank1(want, TLIN, wr, wc)
+    assert np.array_equal(deq.cpu().numpy().reshape(rows, cols), ref)
+    assert np.all(ref[np.minimum(wr[:, None], wc[None, :]) > 0] > 0)     # zero-free map
+    # recomputed scales reproduce themselves and the codes (Rank-1/Linear round trip)
+    codes2, r2, c2 = lpmm.quantize(deq.reshape(rows, cols).contiguous(), lpmm.NORM_RANK1, lpmm.MAP_LINEAR_NOZERO)
+    assert torch.equal(r, r2) and torch.equal(c, c2) and torch.equal(codes, codes2)
+
+
+# ------------------------------------------------------------------ the fused step
+
+def test_single_matrix_config_ten_steps():
+    wl = workloads.single_matrix()
+    pair = Pair(wl.tensors, hyper_of(wl), workload_index=wl.index)
+    kinds = [lpmm.state_view(pair.state, i)["kind"] for i in range(2)]
+    assert kinds == [lpmm.KIND_RANK1, lpmm.KIND_BLOCK]          # bias forced onto the quantized 1-D path
+    seen_v, seen_m = set(), set()
+    for t in range(1, wl.steps + 1):
+        pair.step(t, pair.grads_for(t))
+        pair.compare(tol=1e-6)
+        seen_m |= set(np.unique(oracle.unpack4(pair.ostate[0].m_codes, 1024 * 4096)).tolist())
+        seen_v |= set(np.unique(oracle.unpack4(pair.ostate[0].v_codes, 1024 * 4096)).tolist())
+    assert seen_m == set(range(16)) and seen_v == set(range(16))
+    assert pair.state.last_launches == 4
+
+
+@pytest.mark.parametrize("grad_dtype", [torch.float32, torch.bfloat16])
+def test_shape_zoo_multi_tensor(grad_dtype):
+    specs = [_mat(96, 256), _mat(33, 77), _mat(5, 1000), _mat(130, 384), _mat(64, 1024), _mat(8, 2048),
+             _mat(1, 8192), _mat(8192, 1), _mat(300, 640), _mat(257, 129), _mat(70, 128),
+             _vec(50265), _vec(4097), _vec(4096), _vec(4096, force_quant=True), _vec(1), _vec(300),
+             _mat(16, 16), _mat(64, 64), _mat(65, 64), _vec(12345)]
+    hyper = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
+    pair = Pair(specs, hyper, grad_dtype=grad_dtype, workload_index=7)
+    for t in range(1, 6):
+        grads = pair.grads_for(t, outlier_p=0.0 if t % 2 == 0 else 1e-3)
+        if t == 3:
+            for g in grads[:4]:
+                g[: max(1, g.shape[0] // 3)] = 0           # zero rows
+            grads[11].zero_()                              # an all-zero gradient
+        if t == 4:
+            grads[0][5, 7] = 3.0e4                         # one huge outlier
+            grads[1].mul_(1e-18)                           # second moment in the denormal range
+        pair.step(t, grads)
+        pair.compare(tol=1e-6)
+
+
+def test_block_mode_for_matrices():
+    cfg = lpmm.default_config(v_mode=lpmm.V_BLOCK)
+    specs = [_mat(96, 256), _mat(133, 77), _mat(512, 1024)]
+    hyper = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0)
+    pair = Pair(specs, hyper, config=cfg, workload_index=8)
+    assert all(lpmm.state_view(pair.state, i)["kind"] == lpmm.KIND_BLOCK for i in range(3))
+    for t in range(1, 4):
+        pair.step(t, pair.grads_for(t))
+        pair.compare(tol=1e-6)
+
+
+def test_transformer_base_three_steps_one_launch_per_pass():
+    wl = workloads.transformer_base()
+    pair = Pair(wl.tensors, hyper_of(wl), workload_index=wl.index)
+    kinds = [lpmm.state_view(pair.state, i)["kind"] for i in range(len(wl.tensors))]
+    assert kinds.count(lpmm.KIND_RANK1) == 61 and kinds.count(lpmm.KIND_FP32) == 120
+    for t in range(1, 4):
+        pair.step(t, pair.grads_for(t))
+        pair.compare(tol=1e-6)
+    assert pair.state.last_launches == 4        # memset + pass 1 + reciprocal + pass 2 for all 181 tensors
+
+
+def test_sparse_token_rows_and_lm_head_bias():
+    # RoBERTa-shaped slice: token-sparse embedding gradients (90% of rows zero) and the odd-length 50265 bias.
+    specs = [TensorSpec("emb.word", 50265, 1024, 2, sparse_rows=0.9), TensorSpec("emb.pos", 514, 1024, 2),
+             TensorSpec("emb.type", 1, 1024, 2), _vec(1024), TensorSpec("fc1", 4096, 1024, 2),
+             TensorSpec("head.bias", 50265, 1, 1)]
+    hyper = dict(lr=1e-5, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
+    pair = Pair(specs, hyper, workload_index=2)
+    for t in range(1, 4):
+        pair.step(t, pair.grads_for(t))
+        pair.compare(tol=1e-6)
+    r = pair.ostate[0].v_s0
+    assert np.sum(r == 0) > 0.5 * r.size * 0.9 ** 3      # rows never touched keep scale 0 and dequantize to 0
+
+
+def test_trajectory_100_steps():
+    specs = [_mat(256, 1024), _vec(8192)]
+    hyper = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
+    pair = Pair(specs, hyper, workload_index=5)
+    for t in range(1, 101):
+        pair.step(t, pair.grads_for(t))
+        if t % 25 == 0 or t < 3:
+            pair.compare(tol=1e-4, share_params=False)       # oracle keeps its own fp32 trajectory
+    pair.compare(tol=1e-4, share_params=False)
+
+
+def test_checkpoint_attach_resumes_bit_exactly():
+    specs = [_mat(128, 512), _vec(5000), _vec(100)]
+    hyper = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
+    a = Pair(specs, hyper, workload_index=6)
+    for t in range(1, 4):
+        a.step(t, a.grads_for(t))
+    arena_copy = a.state.arena.clone()
+    phase = a.state.phase
+    params_copy = [p.clone() for p in a.params]
+    for t in range(4, 7):
+        a.step(t, a.grads_for(t))
+    resumed = lpmm.state_attach(a.config, specs, arena_copy, phase)
+    for t in range(4, 7):
+        lpmm.adamw4_step(resumed, params_copy, a.grads_for(t), step=t, **hyper)
+    torch.cuda.synchronize()
+    for i in range(len(specs)):
+        va, vb = lpmm.state_view(a.state, i), lpmm.state_view(resumed, i)
+        for k in ("m_codes", "m_scale", "v_codes", "v_s0", "v_s1", "m32", "v32"):
+            if va[k] is not None:
+                assert torch.equal(va[k], vb[k]), (i, k)
+        assert torch.equal(a.params[i], params_copy[i])
+
+
+def test_host_buffer_step_matches_device_step():
+    specs = [_mat(128, 512), _vec(5000), _vec(100)]
+    hyper = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
+    a = Pair(specs, hyper, workload_index=4)
+    b_state = lpmm.state_init(a.config, specs)
+    h_params = [p.detach().cpu().pin_memory() for p in a.params]
+    nbytes = lpmm.stage_bytes(b_state)
+    dp = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    dg = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    for t in range(1, 4):
+        grads = a.grads_for(t)
+        a.step(t, grads)
+        h_grads = [g.cpu().pin_memory() for g in grads]
+        lpmm.adamw4_step_host(b_state, h_params, h_grads, dp, dg, step=t, **hyper)
+        torch.cuda.synchronize()
+        for i in range(len(specs)):
+            assert torch.equal(h_params[i], a.params[i].cpu())
+
+
+def test_argument_errors_do_not_launch():
+    cfg = lpmm.default_config()
+    st = lpmm.state_init(cfg, [_mat(64, 128)])
+    p = torch.zeros(64, 128, device="cuda")
+    g = torch.zeros(64, 128, device="cuda")
+    ok = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0)
+    for bad in (dict(step=0), dict(step=1, beta1=1.0), dict(step=1, lr=-1.0), dict(step=1, eps=float("nan"))):
+        with pytest.raises(lpmm.LpmmError) as ei:
+            lpmm.adamw4_step(st, [p], [g], **{**ok, "step": 1, **bad})
+        assert ei.value.status == lpmm.ERR_INVALID_ARG
+    flat = torch.zeros(64 * 128 + 4, device="cuda")
+    with pytest.raises(lpmm.LpmmError) as ei:
+        lpmm.adamw4_step(st, [flat[1:64 * 128 + 1]], [g], step=1, **ok)
+    assert ei.value.status == lpmm.ERR_ALIGNMENT
+    with pytest.raises(lpmm.LpmmError) as ei:
+        lpmm.quantize(p, lpmm.NORM_RANK1, lpmm.MAP_DE_SIGNED)
+    assert ei.value.status == lpmm.ERR_UNSUPPORTED
+    torch.cuda.synchronize()
+    assert torch.count_nonzero(p) == 0
