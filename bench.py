@@ -1,0 +1,326 @@
+"""Benchmark of the fused 4-bit AdamW step (one JSON line on stdout).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+A step is one pass of the whole hot path (rank-1 maxima pass, reciprocal pass, update/re-quantize pass)
+over every tensor of the workload. The default workload is the LLaMA-7B-shaped parameter list with bf16
+gradients (6.74 G fp32 parameters, about 47.5 GB resident), far larger than L2, so no flush is needed
+between iterations. With N > 1 (one process per GPU under torch.distributed.run) every rank runs its own
+copy of the per-GPU workload with no collective inside the step (weak scaling).
+
+`--impl reference` times the CPU oracle (a deliberately plain program) on a bounded sample of the same
+workload on the host cores; under a multi-rank launch only rank 0 runs it.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "4-bit AdamW step: Gparams/s and achieved HBM GB/s vs B200 peak"
+UNIT = "Gparams/s"
+
+# Algorithmic bytes per parameter (each operand read once and written once, scales included) for a
+# 2-D rank-1 tensor: w 4+4, g 2 (bf16) or 4 (fp32), m codes 0.5+0.5, v codes 0.5+0.5, m block maxima 8/128.
+# The update/re-quantize pass moves exactly these; the maxima pass re-reads g and the v codes.
+PASS2_BYTES = {"bf16": 12.0625, "f32": 14.0625}
+PASS1_BYTES = {"bf16": 2.5, "f32": 4.5}
+# DRAM traffic of the update/re-quantize pass measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum)
+# per parameter, from the capture summarised in profiles/; None until a capture exists.
+PASS2_TRAFFIC_BYTES_PER_PARAM = {"bf16": None, "f32": None}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama_7b")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+# ----------------------------------------------------------------------------- clocks
+
+class ClockSampler:
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        import torch
+        self.proc = None
+        self.path = None
+        try:
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            ident = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
+        except Exception:
+            ident = str(device_index)
+        try:
+            fd, self.path = tempfile.mkstemp(prefix="lpmm_clocks_", suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", ident, f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self, t0: float, t1: float) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.12)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        rows = []
+        try:
+            from datetime import datetime
+            for line in open(self.path):
+                parts = [p.strip() for p in line.strip().split(",")]
+                if len(parts) < 8:
+                    continue
+                try:
+                    ts = datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                    rows.append((ts, float(parts[1]), float(parts[2]), parts[4:8]))
+                except Exception:
+                    continue
+        finally:
+            try:
+                os.unlink(self.path)
+            except Exception:
+                pass
+        inside = [r for r in rows if t0 - 0.03 <= r[0] <= t1 + 0.03] or rows
+        if not inside:
+            return out
+        sm = sorted(r[1] for r in inside)
+        out["sm_mhz"] = sm[len(sm) // 2]
+        out["sm_max_mhz"] = inside[0][2]
+        out["samples"] = len(inside)
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        out["reasons"] = [n for k, n in enumerate(names) if any(r[3][k] == "Active" for r in inside)]
+        return out
+
+
+# ----------------------------------------------------------------------------- oracle legs
+
+def oracle_sample(wl):
+    """The bounded sample of the workload the CPU oracle is timed on: its largest repeated group of
+    matrices (one attention block of the LLaMA list), or the whole list when that is small."""
+    mats = [(i, t) for i, t in enumerate(wl.tensors) if t.ndim == 2 and t.numel > 4096]
+    if wl.numel <= 80_000_000:
+        return list(enumerate(wl.tensors)), "whole workload"
+    picked, total = [], 0
+    for i, t in mats[1:]:
+        if total + t.numel > 70_000_000:
+            break
+        picked.append((i, t))
+        total += t.numel
+    return picked, f"{len(picked)} matrices of one layer ({', '.join(f'{t.rows}x{t.cols}' for _, t in picked)})"
+
+
+def time_oracle(wl, steps: int, warmup: int):
+    """Runs the oracle as it stands on the sample; returns (Gparams/s, threads, description, ms/step)."""
+    import numpy as np
+    import torch
+    import oracle
+    from paper_2309_01507_b200 import workloads
+    sample, desc = oracle_sample(wl)
+    hyper = dict(lr=wl.lr, beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps, weight_decay=wl.weight_decay)
+    gdt = torch.bfloat16 if wl.grad_dtype == "bf16" else torch.float32
+    ws, gs, sts = [], [], []
+    for i, t in sample:
+        ws.append(workloads.make_param(t, wl.index, i).numpy().ravel().copy())
+        gs.append(workloads.make_grad(t, wl.index, i, 1, dtype=gdt).float().numpy().ravel())
+        sts.append(oracle.state_init(t.rows, t.cols, oracle.kind_of(t.rows, t.cols, t.ndim, 4096, int(t.force_quant))))
+    n = sum(t.numel for _, t in sample)
+    step = 0
+    for _ in range(warmup):
+        step += 1
+        for w, g, st in zip(ws, gs, sts):
+            oracle.adamw4_step(w, g, st, step=step, **hyper)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        step += 1
+        for w, g, st in zip(ws, gs, sts):
+            oracle.adamw4_step(w, g, st, step=step, **hyper)
+    dt = time.perf_counter() - t0
+    return n * steps / dt / 1e9, oracle.threads(), f"{desc}, {n / 1e6:.1f} M params per step, {steps} step(s)", dt / steps * 1e3
+
+
+def run_reference(args):
+    from paper_2309_01507_b200 import dist, workloads
+    rank, _, _ = dist.env()
+    if rank != 0:
+        return
+    wl = workloads.WORKLOADS[args.workload]()
+    value, threads, desc, ms = time_oracle(wl, max(args.steps, 1), args.warmup)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": wl.name, "sample": desc, "grad_dtype": wl.grad_dtype},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------- the CUDA arm
+
+def run_ours(args):
+    import torch
+    from paper_2309_01507_b200 import build as cuda_build
+    from paper_2309_01507_b200 import dist, lpmm, workloads
+
+    rank, local_rank, world = dist.env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the fused step has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    cuda_build.build()
+    dist.init("nccl")
+
+    wl = workloads.WORKLOADS[args.workload]()
+    gdt = torch.bfloat16 if wl.grad_dtype == "bf16" else torch.float32
+    hyper = dict(lr=wl.lr, beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps, weight_decay=wl.weight_decay)
+    params = [workloads.make_param(t, wl.index, i, device=dev) for i, t in enumerate(wl.tensors)]
+    grads = [workloads.make_grad(t, wl.index, i, 1, device=dev, dtype=gdt) for i, t in enumerate(wl.tensors)]
+    state = lpmm.state_init(lpmm.default_config(), wl.tensors, device=dev)
+    cache = lpmm.make_ptr_cache(params, grads)
+    n_params = wl.numel
+    torch.cuda.synchronize()
+
+    step = 0
+    for _ in range(max(args.warmup, 3)):
+        step += 1
+        lpmm.adamw4_step(state, params, grads, step=step, ptr_cache=cache, **hyper)
+    torch.cuda.synchronize()
+    dist.barrier()
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    lpmm.profile(state, True)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    t_wall0 = time.time()
+    ev0.record()
+    for _ in range(args.steps):
+        step += 1
+        lpmm.adamw4_step(state, params, grads, step=step, ptr_cache=cache, **hyper)
+    ev1.record()
+    torch.cuda.synchronize()
+    t_wall1 = time.time()
+    dist.barrier()
+    clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
+    prof = lpmm.profile_read(state)
+    lpmm.profile(state, False)
+    launches = state.last_launches * args.steps
+    ms_total = dist.max_over_ranks(ev0.elapsed_time(ev1), device=dev)
+    ms_step = ms_total / args.steps
+    value = world * n_params / (ms_step * 1e-3) / 1e9
+
+    # ---- end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
+    e2e = None
+    if not args.no_e2e and args.e2e_steps > 0:
+        gsz = 2 if wl.grad_dtype == "bf16" else 4
+        nstage = lpmm.stage_bytes(state)
+        d_pstage = torch.empty(nstage, dtype=torch.uint8, device=dev)
+        d_gstage = torch.empty(nstage, dtype=torch.uint8, device=dev)
+        h_p = torch.empty(n_params, dtype=torch.float32, pin_memory=True)
+        h_g = torch.empty(n_params, dtype=gdt, pin_memory=True)
+        hp, hg, off = [], [], 0
+        for p, g in zip(params, grads):
+            k = p.numel()
+            hp.append(h_p[off:off + k]); hg.append(h_g[off:off + k])
+            hp[-1].copy_(p.reshape(-1)); hg[-1].copy_(g.reshape(-1))
+            off += k
+        torch.cuda.synchronize()
+        e2e_state = lpmm.state_init(lpmm.default_config(), wl.tensors, device=dev)
+        t = 0
+        for _ in range(1):
+            t += 1
+            lpmm.adamw4_step_host(e2e_state, hp, hg, d_pstage, d_gstage, step=t, **hyper)
+        torch.cuda.synchronize()
+        dist.barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.e2e_steps):
+            t += 1
+            lpmm.adamw4_step_host(e2e_state, hp, hg, d_pstage, d_gstage, step=t, **hyper)
+        e1.record()
+        torch.cuda.synchronize()
+        dist.barrier()
+        e2e_ms = dist.max_over_ranks(e0.elapsed_time(e1), device=dev) / args.e2e_steps
+        e2e = {"value": world * n_params / (e2e_ms * 1e-3) / 1e9, "unit": UNIT,
+               "h2d_bytes_per_step": (4 + gsz) * n_params, "d2h_bytes_per_step": 4 * n_params,
+               "ms_per_step": e2e_ms, "steps": args.e2e_steps,
+               "note": "lpmm_adamw4_step_host: pinned host params+grads copied in, updated params copied out, every step"}
+        del d_pstage, d_gstage, h_p, h_g, hp, hg, e2e_state
+
+    if rank != 0:
+        dist.shutdown()
+        return
+
+    peak, peak_kind = measured_peak()
+    p2_ms = prof["pass2_ms"] / max(prof["steps"], 1)
+    p1_ms = prof["pass1_ms"] / max(prof["steps"], 1)
+    alg_bytes = PASS2_BYTES[wl.grad_dtype] * n_params
+    achieved = alg_bytes / (p2_ms * 1e-3) / 1e9
+    traffic_pp = PASS2_TRAFFIC_BYTES_PER_PARAM[wl.grad_dtype]
+    roofline = {"bound": "hbm", "kernel": "pass2_kernel (update + re-quantize)", "achieved": achieved, "peak": peak,
+                "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                "traffic": None if traffic_pp is None else traffic_pp * n_params,
+                "algorithmic_bytes_per_launch": alg_bytes, "ms_per_launch": p2_ms,
+                "pass1_ms_per_launch": p1_ms,
+                "pass1_achieved_gbs": PASS1_BYTES[wl.grad_dtype] * n_params / (p1_ms * 1e-3) / 1e9 if p1_ms > 0 else None,
+                "step_algorithmic_gbs": alg_bytes / (ms_step * 1e-3) / 1e9,
+                "step_moved_gbs": (PASS2_BYTES[wl.grad_dtype] + PASS1_BYTES[wl.grad_dtype]) * n_params / (ms_step * 1e-3) / 1e9,
+                "frac_of_nominal_8tbs": achieved / 8000.0}
+
+    cpu = None
+    if not args.no_cpu_baseline and world == 1:
+        v, threads, desc, _ = time_oracle(wl, 2, 1)
+        cpu = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": wl.name, "tensors": len(wl.tensors), "params_per_gpu": n_params,
+                       "grad_dtype": wl.grad_dtype, "param_dtype": "f32", "m": "B128/DE 4-bit", "v": "Rank-1/Linear 4-bit",
+                       "l2": "inputs larger than L2 (47 GB resident), no flush", "parallelism": f"replicas x{world}, no collective"},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu}
+    print(json.dumps(line), flush=True)
+    dist.shutdown()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -147,7 +147,17 @@ lpmm_status lpmm_state_view(const lpmm_state* st, int32_t tensor, int32_t* kind,
 /* 0 or 1: which of the two rank-1 scale buffers is current. Save it with a copy of the arena. */
 int32_t lpmm_state_phase(const lpmm_state* st);
 
-/* Number of kernels and memsets the last lpmm_adamw4_step on this state enqueued. */
+/* Optional per-kernel timing. While enabled, every lpmm_adamw4_step records CUDA events on its stream
+ * around its three kernels (host-side event objects only; no device memory). */
+lpmm_status lpmm_state_profile(lpmm_state* st, int32_t enable);
+
+/* Waits for the recorded steps to finish, returns the summed durations in milliseconds of the rank-1
+ * maxima pass, the reciprocal pass and the update/re-quantize pass over `steps` recorded steps, and
+ * clears the record. Any output pointer may be NULL. */
+lpmm_status lpmm_state_profile_read(lpmm_state* st, double* pass1_ms, double* rcp_ms, double* pass2_ms, int32_t* steps);
+
+/* Number of kernels the last lpmm_adamw4_step on this state launched (3 when a rank-1 tensor is present,
+ * else 1; one additional memset node clears the new row/column maxima). */
 int32_t lpmm_state_last_launches(const lpmm_state* st);
 
 /* Frees the host handle only; the arena stays the caller's. NULL is allowed. */

@@ -134,6 +134,8 @@ struct lpmm_state {
     std::vector<void*> params, grads;  // what the device-side pointer arrays currently hold
     size_t stage_bytes;
     std::vector<size_t> stage_off;
+    bool profile;                          // record events around each kernel of a step
+    std::vector<cudaEvent_t> prof_events;  // 4 per recorded step: start, after pass 1, after rcp, after pass 2
 };
 
 namespace {
@@ -228,6 +230,7 @@ lpmm_status make_state(const lpmm_config* cfg, const lpmm_shape* shapes, int32_t
     st->arena_bytes = arena_bytes;
     st->phase = phase;
     st->last_launches = 0;
+    st->profile = false;
     st->ptrs_valid = false;
     st->params.assign(n, nullptr);
     st->grads.assign(n, nullptr);
@@ -322,18 +325,32 @@ lpmm_status lpmm_adamw4_step(lpmm_state* st, void* const* d_params, const void* 
     a.h.decay = 1.0f - lr * weight_decay;
     const bool bf16 = (grad_dtype == LPMM_BF16);
 
+    cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
+    if (st->profile) {
+        for (int k = 0; k < 4; ++k) {
+            LPMM_CUDA(cudaEventCreate(&ev[k]));
+            st->prof_events.push_back(ev[k]);
+        }
+    }
     if (st->total1 > 0) {
         float* rc_new = reinterpret_cast<float*>(st->arena + st->L.rc[st->phase ^ 1]);
         LPMM_CUDA(cudaMemsetAsync(rc_new, 0, sizeof(float) * st->L.rc_floats, s));
+        if (ev[0]) LPMM_CUDA(cudaEventRecord(ev[0], s));
         a.tile_start = reinterpret_cast<const int32_t*>(st->arena + st->L.tiles1);
         a.total_tiles = st->total1;
         LPMM_CUDA(launch_pass1(a, bf16, st->grid1, s));
+        if (ev[1]) LPMM_CUDA(cudaEventRecord(ev[1], s));
         LPMM_CUDA(launch_rcp(rc_new, reinterpret_cast<float*>(st->arena + st->L.rcp), st->L.rc_floats, s));
-        launches += 3;
+        launches += 2;
+    } else if (ev[0]) {
+        LPMM_CUDA(cudaEventRecord(ev[0], s));
+        LPMM_CUDA(cudaEventRecord(ev[1], s));
     }
+    if (ev[2]) LPMM_CUDA(cudaEventRecord(ev[2], s));
     a.tile_start = reinterpret_cast<const int32_t*>(st->arena + st->L.tiles2);
     a.total_tiles = st->total2;
     LPMM_CUDA(launch_pass2(a, bf16, st->grid2, s));
+    if (ev[3]) LPMM_CUDA(cudaEventRecord(ev[3], s));
     launches += 1;
     st->phase ^= 1;
     st->last_launches = launches;
@@ -432,11 +449,45 @@ lpmm_status lpmm_state_view(const lpmm_state* st, int32_t tensor, int32_t* kind,
     return LPMM_OK;
 }
 
+lpmm_status lpmm_state_profile(lpmm_state* st, int32_t enable) {
+    if (!st) return LPMM_ERR_INVALID_ARG;
+    st->profile = (enable != 0);
+    return LPMM_OK;
+}
+
+lpmm_status lpmm_state_profile_read(lpmm_state* st, double* pass1_ms, double* rcp_ms, double* pass2_ms, int32_t* steps) {
+    if (!st) return LPMM_ERR_INVALID_ARG;
+    double t[3] = {0.0, 0.0, 0.0};
+    const size_t n = st->prof_events.size() / 4;
+    lpmm_status rc = LPMM_OK;
+    for (size_t i = 0; i < n && rc == LPMM_OK; ++i) {
+        cudaEvent_t* e = &st->prof_events[4 * i];
+        cudaError_t err = cudaEventSynchronize(e[3]);
+        for (int k = 0; k < 3 && err == cudaSuccess; ++k) {
+            float ms = 0.0f;
+            err = cudaEventElapsedTime(&ms, e[k], e[k + 1]);
+            t[k] += ms;
+        }
+        if (err != cudaSuccess) rc = cuda_fail(err);
+    }
+    for (cudaEvent_t e : st->prof_events) cudaEventDestroy(e);
+    st->prof_events.clear();
+    if (pass1_ms) *pass1_ms = t[0];
+    if (rcp_ms) *rcp_ms = t[1];
+    if (pass2_ms) *pass2_ms = t[2];
+    if (steps) *steps = (int32_t)n;
+    return rc;
+}
+
 int32_t lpmm_state_phase(const lpmm_state* st) { return st ? st->phase : -1; }
 
 int32_t lpmm_state_last_launches(const lpmm_state* st) { return st ? st->last_launches : 0; }
 
-void lpmm_state_destroy(lpmm_state* st) { delete st; }
+void lpmm_state_destroy(lpmm_state* st) {
+    if (!st) return;
+    for (cudaEvent_t e : st->prof_events) cudaEventDestroy(e);
+    delete st;
+}
 
 const char* lpmm_status_string(lpmm_status s) {
     switch (s) {

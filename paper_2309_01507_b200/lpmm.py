@@ -26,6 +26,7 @@ KIND_FP32, KIND_BLOCK, KIND_RANK1 = 0, 1, 2
 EXPORTS = ("lpmm_state_bytes", "lpmm_state_init", "lpmm_state_attach", "lpmm_adamw4_step",
            "lpmm_adamw4_step_host", "lpmm_stage_bytes", "lpmm_quantize", "lpmm_dequantize",
            "lpmm_state_view", "lpmm_state_phase", "lpmm_state_last_launches", "lpmm_state_destroy",
+           "lpmm_state_profile", "lpmm_state_profile_read",
            "lpmm_status_string", "lpmm_last_cuda_error")
 
 
@@ -73,6 +74,9 @@ def lib():
         L.lpmm_quantize.argtypes = [vp, i64, i64, i32, i32, i32, u32, vp, vp, vp, vp]
         L.lpmm_dequantize.argtypes = [vp, vp, vp, i64, i64, i32, i32, i32, vp, vp]
         L.lpmm_state_view.argtypes = [vp, i32, C.POINTER(i32)] + [C.POINTER(vp)] * 7
+        L.lpmm_state_profile.argtypes = [vp, i32]
+        L.lpmm_state_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_double),
+                                              C.POINTER(i32)]
         L.lpmm_state_phase.argtypes = [vp]
         L.lpmm_state_last_launches.argtypes = [vp]
         L.lpmm_state_destroy.argtypes = [vp]
@@ -202,6 +206,18 @@ def adamw4_step(state: State, params, grads, *, lr, beta1, beta2, eps, weight_de
 def make_ptr_cache(params, grads):
     """Pre-marshalled pointer arrays for repeated steps on the same buffers (skips per-call Python work)."""
     return _ptr_array(params), _ptr_array(grads), _grad_dtype(grads)
+
+
+def profile(state: State, enable: bool) -> None:
+    _check(lib().lpmm_state_profile(state.handle, int(enable)), "lpmm_state_profile")
+
+
+def profile_read(state: State) -> dict:
+    """Summed kernel durations (ms) over the steps recorded since the last read."""
+    p1, rc, p2, n = C.c_double(), C.c_double(), C.c_double(), C.c_int32()
+    _check(lib().lpmm_state_profile_read(state.handle, C.byref(p1), C.byref(rc), C.byref(p2), C.byref(n)),
+           "lpmm_state_profile_read")
+    return {"pass1_ms": p1.value, "rcp_ms": rc.value, "pass2_ms": p2.value, "steps": n.value}
 
 
 def stage_bytes(state: State) -> int:

@@ -136,6 +136,9 @@ WORKLOADS = {
     "roberta_large": roberta_large,
     "llama_7b": llama_7b,
     "square_8192": square_8192,
+    # reduced LLaMA list (embedding, head and a few decoder layers) for profiler captures and quick checks
+    "llama_7b_1l": lambda: llama_7b(layers=1),
+    "llama_7b_4l": lambda: llama_7b(layers=4),
 }
 
 
