@@ -43,6 +43,13 @@ typedef enum { LPMM_NORM_BLOCK = 0, LPMM_NORM_RANK1 = 1 } lpmm_norm;          /*
 typedef enum { LPMM_MAP_DE_SIGNED = 0, LPMM_MAP_LINEAR_NOZERO = 1 } lpmm_map; /* App. D.2 / Sec. 4.1 */
 typedef enum { LPMM_V_RANK1 = 0, LPMM_V_BLOCK = 1 } lpmm_vmode;               /* second-moment normalizer for 2-D tensors */
 
+/* How Eq. 1's last line (bias correction, sqrt, division) is evaluated. The stored states (codes and
+ * scales) are bit-identical in both modes; only the rounding of the updated parameters differs.
+ *   FAST: lr/(1-beta1^t) and 1/(1-beta2^t) folded on the host, one approximate square root and one
+ *         approximate reciprocal per element; within 1e-6 * max(|w|, lr) of the IEEE evaluation.
+ *   IEEE: every division and the square root correctly rounded, in the order Eq. 1 writes them. */
+typedef enum { LPMM_UPDATE_FAST = 0, LPMM_UPDATE_IEEE = 1 } lpmm_update_math;
+
 /* lpmm_shape.flags */
 #define LPMM_FORCE_QUANT 1u /* quantize even if numel <= min_quant_numel */
 #define LPMM_FORCE_FP32 2u  /* keep fp32 states whatever the size */
@@ -62,6 +69,8 @@ typedef struct {
     int32_t v_block;         /* second-moment block size for 1-D tensors and LPMM_V_BLOCK (Sec. 4.2: 128) */
     int32_t v_mode;          /* lpmm_vmode */
     int64_t min_quant_numel; /* tensors with numel <= this keep fp32 states (App. C.1: 4096) */
+    int32_t update_math;     /* lpmm_update_math: arithmetic of the parameter update only */
+    int32_t reserved;        /* 0 */
 } lpmm_config;
 
 typedef struct lpmm_state lpmm_state; /* opaque host handle */

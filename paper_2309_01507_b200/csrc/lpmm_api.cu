@@ -56,6 +56,7 @@ lpmm_status validate_config(const lpmm_config* cfg, const lpmm_shape* shapes, in
     if (cfg->v_mode != LPMM_V_RANK1 && cfg->v_mode != LPMM_V_BLOCK) return LPMM_ERR_INVALID_ARG;
     if (cfg->bits != 4) return LPMM_ERR_UNSUPPORTED;
     if (cfg->m_block != 128 || cfg->v_block != 128) return LPMM_ERR_UNSUPPORTED;
+    if (cfg->update_math != LPMM_UPDATE_FAST && cfg->update_math != LPMM_UPDATE_IEEE) return LPMM_ERR_INVALID_ARG;
     for (int32_t i = 0; i < n; ++i) {
         const lpmm_shape& s = shapes[i];
         if (s.rows <= 0 || s.cols <= 0) return LPMM_ERR_INVALID_ARG;
@@ -323,6 +324,11 @@ lpmm_status lpmm_adamw4_step(lpmm_state* st, void* const* d_params, const void* 
     a.h.bc1 = (float)(1.0 - std::pow((double)beta1, (double)step));   // Eq. 1: 1 - beta^t
     a.h.bc2 = (float)(1.0 - std::pow((double)beta2, (double)step));
     a.h.decay = 1.0f - lr * weight_decay;
+    {
+        const double bc1 = 1.0 - std::pow((double)beta1, (double)step), bc2 = 1.0 - std::pow((double)beta2, (double)step);
+        a.h.step_size = (float)((double)lr / bc1);
+        a.h.rbc2 = (float)(1.0 / bc2);
+    }
     const bool bf16 = (grad_dtype == LPMM_BF16);
 
     cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
@@ -349,7 +355,7 @@ lpmm_status lpmm_adamw4_step(lpmm_state* st, void* const* d_params, const void* 
     if (ev[2]) LPMM_CUDA(cudaEventRecord(ev[2], s));
     a.tile_start = reinterpret_cast<const int32_t*>(st->arena + st->L.tiles2);
     a.total_tiles = st->total2;
-    LPMM_CUDA(launch_pass2(a, bf16, st->grid2, s));
+    LPMM_CUDA(launch_pass2(a, bf16, st->cfg.update_math == LPMM_UPDATE_IEEE, st->grid2, s));
     if (ev[3]) LPMM_CUDA(cudaEventRecord(ev[3], s));
     launches += 1;
     st->phase ^= 1;

@@ -7,6 +7,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "lpmm_de_lut.cuh"
+
 namespace lpmm {
 
 constexpr float kFltMin = 1.17549435e-38f;  // smallest normal binary32
@@ -56,6 +58,48 @@ __device__ __forceinline__ float lin_value(uint32_t q) {  // (q+1)/16, exact
     return __fmul_rn((float)(q + 1u), 0.0625f);
 }
 
+// Same value without an integer conversion: `word` holds the nibble at bits [shift, shift+4); it is
+// moved to the top of the mantissa of 1.0f (giving 1 + q/16 exactly) and 15/16 is subtracted (exact).
+template <int SHIFT>
+__device__ __forceinline__ float lin_value_at(uint32_t word) {
+    const uint32_t moved = (SHIFT <= 19) ? (word << (19 - SHIFT)) : (word >> (SHIFT - 19));
+    return __fadd_rn(__uint_as_float((moved & 0x00780000u) | 0x3f800000u), -0.9375f);
+}
+
+// Nearest linear code as the low mantissa bits of 2^23 + ceil(max(16 n - 1.5, 0)), added with
+// round-up; valid for n <= 1 + 2^-22 (then the code is at most 15). The caller removes the 2^23 pattern.
+constexpr uint32_t kMagicBits = 0x4b000000u;  // 2^23 as binary32
+__device__ __forceinline__ uint32_t lin_nearest_magic(float n) {
+    const float y = fmaxf(__fmaf_rn(n, 16.0f, -1.5f), 0.0f);
+    return __float_as_uint(__fadd_ru(y, 8388608.0f));
+}
+
+// Shared-memory image used by the step kernel: the non-negative half of kDeLut at byte 0, the negative
+// half at byte 16384 (so that the sign bit of the key selects it without an extra instruction), and the
+// 16-entry dequantization table in between.
+constexpr int kLutNegOffset = 16384;
+constexpr int kLutDeTableOffset = 1024;
+constexpr int kLutSmemBytes = kLutNegOffset + kDeLutBins * 8;
+
+__device__ __forceinline__ void load_lut_smem(unsigned char* smem) {
+    for (int i = threadIdx.x; i < kDeLutBins; i += blockDim.x) {
+        reinterpret_cast<uint2*>(smem)[i] = kDeLut[i];
+        reinterpret_cast<uint2*>(smem + kLutNegOffset)[i] = kDeLut[kDeLutBins + i];
+    }
+    if (threadIdx.x < 16) reinterpret_cast<float*>(smem + kLutDeTableOffset)[threadIdx.x] = kDeTable[threadIdx.x];
+}
+
+// Table-driven equivalent of de_nearest() for |n| < 2 (always true for m / blockmax(|m|)); NaN gives code 7.
+__device__ __forceinline__ uint32_t de_nearest_lut(float n, const unsigned char* smem) {
+    const float a = fminf(fmaxf(fabsf(n), kDeLutMinAbs), 1.9999999f);
+    const uint32_t nb = __float_as_uint(n);
+    const uint32_t cs = (__float_as_uint(a) & 0x7fffffffu) | (nb & 0x80000000u);   // copysign(a, n)
+    const uint32_t off = (cs >> 17) & 0x7ff8u;      // bit 14 = sign -> +16384; bits 3..13 = key * 8
+    const uint2 e = *reinterpret_cast<const uint2*>(smem + off - kDeLutKeyBias);
+    const uint32_t c = e.y + (a > __uint_as_float(e.x) ? 1u : 0u);
+    return c ^ ((uint32_t)((int32_t)nb >> 31) & 15u);
+}
+
 // 1/s for a usable scale, 0 for a zero or denormal one (everything under it quantizes as zero).
 __device__ __forceinline__ float scale_rcp(float s) {
     return (s >= kFltMin) ? __fdiv_rn(1.0f, s) : 0.0f;
@@ -66,6 +110,8 @@ struct Hyper {
     float omb1, omb2;  // 1 - beta, evaluated in binary32
     float bc1, bc2;    // 1 - beta^t, evaluated in binary64 on the host and rounded once
     float decay;       // 1 - lr * weight_decay
+    float step_size;   // lr / bc1, evaluated in binary64 and rounded once (fast update)
+    float rbc2;        // 1 / bc2, likewise
 };
 
 // Eq. 1 moment updates; separate roundings, in the order written there.
@@ -83,6 +129,18 @@ __device__ __forceinline__ float adam_update(float w, float mt, float vt, const 
     float denom = __fadd_rn(__fsqrt_rn(vhat), h.eps);
     float upd = __fmul_rn(h.lr, __fdiv_rn(mhat, denom));
     return __fsub_rn(__fmul_rn(w, h.decay), upd);
+}
+
+// The same update with one approximate square root and one approximate reciprocal (each within about
+// one ulp) and the constant divisions folded into host-side factors: a handful of roundings away from
+// adam_update(), far inside the 1e-6 * max(|w|, lr) parameter tolerance. The stored states never
+// depend on this function.
+__device__ __forceinline__ float adam_update_fast(float w, float mt, float vt, const Hyper& h) {
+    float sq, rc;
+    asm("sqrt.approx.f32 %0, %1;" : "=f"(sq) : "f"(__fmul_rn(vt, h.rbc2)));
+    asm("rcp.approx.f32 %0, %1;" : "=f"(rc) : "f"(__fadd_rn(sq, h.eps)));
+    const float upd = __fmul_rn(__fmul_rn(mt, h.step_size), rc);
+    return __fmaf_rn(w, h.decay, -upd);
 }
 
 __device__ __forceinline__ float bf16_lo(uint32_t pair) { return __uint_as_float(pair << 16); }

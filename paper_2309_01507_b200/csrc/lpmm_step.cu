@@ -98,18 +98,31 @@ __device__ __forceinline__ void store_codes_guard(uint8_t* codes, int64_t e, int
 
 // ---- per-lane arithmetic ----------------------------------------------------------------------
 
+__device__ __forceinline__ float lin_value_k(uint32_t word, int k) {   // k is a compile-time constant after unrolling
+    const int shift = 4 * k;
+    const uint32_t moved = (shift <= 19) ? (word << (19 - shift)) : (word >> (shift - 19));
+    return __fadd_rn(__uint_as_float((moved & 0x00780000u) | 0x3f800000u), -0.9375f);   // (q + 1) / 16, exact
+}
+
+template <bool EXACT>
+__device__ __forceinline__ float update_param(float w, float mt, float vt, const Hyper& h) {
+    return EXACT ? adam_update(w, mt, vt, h) : adam_update_fast(w, mt, vt, h);
+}
+
 // Dequantize (Sec. 2.2), update the moments (Eq. 1) and the parameters for 8 elements.
 // vs[k] is the old scale of element k's second moment, am the old scale of its first-moment block.
+template <bool EXACT>
 __device__ __forceinline__ void moments_and_update8(float (&w)[8], const float (&g)[8], uint32_t qm, uint32_t qv,
                                                     float am, const float (&vs)[8], const Hyper& h,
-                                                    const float* s_de, float (&mt)[8], float (&vt)[8]) {
+                                                    const unsigned char* s_lut, float (&mt)[8], float (&vt)[8]) {
+    const float* s_de = reinterpret_cast<const float*>(s_lut + kLutDeTableOffset);
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
         float m = __fmul_rn(s_de[(qm >> (4 * k)) & 15u], am);
-        float v = __fmul_rn(lin_value((qv >> (4 * k)) & 15u), vs[k]);
+        float v = __fmul_rn(lin_value_k(qv, k), vs[k]);
         mt[k] = ema_m(m, g[k], h);
         vt[k] = ema_v(v, g[k], h);
-        w[k] = adam_update(w[k], mt[k], vt[k], h);
+        w[k] = update_param<EXACT>(w[k], mt[k], vt[k], h);
     }
 }
 
@@ -120,75 +133,115 @@ __device__ __forceinline__ float absmax8(const float (&x)[8]) {
     return a;
 }
 
-__device__ __forceinline__ uint32_t quantize8_de(const float (&x)[8], float rcp) {
+// Eight nearest codes packed little-nibble-first: acc = acc * 16 + code, from element 7 down to 0.
+__device__ __forceinline__ uint32_t quantize8_de(const float (&x)[8], float rcp, const unsigned char* s_lut) {
     uint32_t q = 0;
 #pragma unroll
-    for (int k = 0; k < 8; ++k) q |= de_nearest(__fmul_rn(x[k], rcp)) << (4 * k);
+    for (int k = 7; k >= 0; --k) q = q * 16u + de_nearest_lut(__fmul_rn(x[k], rcp), s_lut);
     return q;
 }
 __device__ __forceinline__ uint32_t quantize8_lin(const float (&x)[8], const float (&rcp)[8]) {
     uint32_t q = 0;
 #pragma unroll
-    for (int k = 0; k < 8; ++k) q |= lin_nearest(__fmul_rn(x[k], rcp[k])) << (4 * k);
-    return q;
+    for (int k = 7; k >= 0; --k) q = q * 16u + lin_nearest_magic(__fmul_rn(x[k], rcp[k]));
+    return q - kMagicBits * 0x11111111u;   // removes the eight 2^23 patterns (mod 2^32)
 }
 
 // ---- pass 2, rank-1 tensors with cols % 128 == 0 ---------------------------------------------------
 
 template <bool BF16>
+struct RowRegs {           // one lane's share of one row: raw, still packed
+    float4 w0, w1;
+    uint4 g0, g1;          // bf16: g0 holds all 8 values; fp32: g0, g1
+    uint32_t qm, qv;
+    float am, r_old, r_rcp;
+};
+
+template <bool BF16>
+__device__ __forceinline__ void load_row(RowRegs<BF16>& r, const TensorDesc& d, const float* __restrict__ w,
+                                         const void* __restrict__ g, const float* rc_old, const float* rcp_new,
+                                         int64_t i, int64_t col0) {
+    const int64_t e = i * d.cols + col0;
+    r.w0 = *reinterpret_cast<const float4*>(w + e);
+    r.w1 = *reinterpret_cast<const float4*>(w + e + 4);
+    if (BF16) {
+        r.g0 = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(g) + e));
+    } else {
+        r.g0 = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(g) + e));
+        r.g1 = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(g) + e + 4));
+    }
+    r.qm = *reinterpret_cast<const uint32_t*>(d.m_codes + (e >> 1));
+    r.qv = *reinterpret_cast<const uint32_t*>(d.v_codes + (e >> 1));
+    r.am = d.m_scale[e >> 7];
+    r.r_old = __ldg(rc_old + i);
+    r.r_rcp = __ldg(rcp_new + i);
+}
+
+template <bool BF16>
+__device__ __forceinline__ void unpack_grad(const RowRegs<BF16>& r, float (&g)[8]) {
+    if (BF16) {
+        g[0] = bf16_lo(r.g0.x); g[1] = bf16_hi(r.g0.x); g[2] = bf16_lo(r.g0.y); g[3] = bf16_hi(r.g0.y);
+        g[4] = bf16_lo(r.g0.z); g[5] = bf16_hi(r.g0.z); g[6] = bf16_lo(r.g0.w); g[7] = bf16_hi(r.g0.w);
+    } else {
+        g[0] = __uint_as_float(r.g0.x); g[1] = __uint_as_float(r.g0.y); g[2] = __uint_as_float(r.g0.z);
+        g[3] = __uint_as_float(r.g0.w); g[4] = __uint_as_float(r.g1.x); g[5] = __uint_as_float(r.g1.y);
+        g[6] = __uint_as_float(r.g1.z); g[7] = __uint_as_float(r.g1.w);
+    }
+}
+
+template <bool BF16, bool EXACT>
 __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __restrict__ w, const void* __restrict__ g,
-                                                 int tile, int phase, const Hyper& h, const float* s_de) {
+                                                 int tile, int phase, const Hyper& h, const unsigned char* s_lut) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int wx = d.wx, wy_count = kWarps / wx;
     const int tx = tile % d.tiles_x, ty = tile / d.tiles_x;
     const int64_t col0 = (int64_t)tx * (kWarpElems * wx) + (warp % wx) * kWarpElems + lane * kLaneElems;
-    const bool active = col0 < d.cols;
+    if (col0 >= d.cols) return;   // cols % 128 == 0: a whole 16-lane group (one block) is in or out together
+    // Shuffles below use a half-warp mask, so the other half may be absent.
+    const unsigned half_mask = 0xffffu << (lane & 16);
     const float* rc_old = d.rc[phase];
     const float* rcp_new = d.rcp_new;
     float* m_scale = d.m_scale;
 
     float c_old[8], c_rcp[8];
-    if (active) {
-        load8_f32(rc_old + d.c_off + col0, c_old);
-        load8_f32(rcp_new + d.c_off + col0, c_rcp);
-    }
+    load8_f32(rc_old + d.c_off + col0, c_old);
+    load8_f32(rcp_new + d.c_off + col0, c_rcp);
     const int64_t row_end = min((int64_t)(ty + 1) * d.tile_rows, d.rows);
-    for (int64_t i = (int64_t)ty * d.tile_rows + warp / wx; i < row_end; i += wy_count) {
-        float wv[8], gv[8], mt[8], vt[8], vs[8], vr[8];
-        uint32_t qm = 0, qv = 0;
-        float am_new = 0.0f;
-        const int64_t e = i * d.cols + col0;
-        if (active) {
-            load8_rw(w + e, wv);
-            load8_grad<BF16>(g, e, gv);
-            qm = __ldg(reinterpret_cast<const uint32_t*>(d.m_codes + (e >> 1)));
-            qv = __ldg(reinterpret_cast<const uint32_t*>(d.v_codes + (e >> 1)));
-            const float am = m_scale[e >> 7];
-            const float r_old = __ldg(rc_old + i);
-            const float r_rcp = __ldg(rcp_new + i);
+    int64_t i = (int64_t)ty * d.tile_rows + warp / wx;
+    if (i >= row_end) return;
+    RowRegs<BF16> cur, nxt;
+    load_row<BF16>(cur, d, w, g, rc_old, rcp_new, i, col0);
+    for (; i < row_end; i += wy_count) {
+        const bool more = i + wy_count < row_end;
+        if (more) load_row<BF16>(nxt, d, w, g, rc_old, rcp_new, i + wy_count, col0);   // prefetch the next row
+        float wv[8] = {cur.w0.x, cur.w0.y, cur.w0.z, cur.w0.w, cur.w1.x, cur.w1.y, cur.w1.z, cur.w1.w};
+        float gv[8], mt[8], vt[8], vs[8], vr[8];
+        unpack_grad<BF16>(cur, gv);
 #pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                vs[k] = fminf(r_old, c_old[k]);      // Sec. 4.2: scale = min(r_i, c_j)
-                vr[k] = fmaxf(r_rcp, c_rcp[k]);      // 1/min(r', c') = max(1/r', 1/c')
-            }
-            moments_and_update8(wv, gv, qm, qv, am, vs, h, s_de, mt, vt);
-            store8_f32(w + e, wv);
-            am_new = absmax8(mt);
+        for (int k = 0; k < 8; ++k) {
+            vs[k] = fminf(cur.r_old, c_old[k]);      // Sec. 4.2: scale = min(r_i, c_j)
+            vr[k] = fmaxf(cur.r_rcp, c_rcp[k]);      // 1/min(r', c') = max(1/r', 1/c')
         }
-        am_new = half_warp_max(am_new);              // all 32 lanes take part in the shuffles
-        if (active) {
-            if ((lane & 15) == 0) m_scale[e >> 7] = am_new;
-            *reinterpret_cast<uint32_t*>(d.m_codes + (e >> 1)) = quantize8_de(mt, scale_rcp(am_new));
-            *reinterpret_cast<uint32_t*>(d.v_codes + (e >> 1)) = quantize8_lin(vt, vr);
-        }
+        moments_and_update8<EXACT>(wv, gv, cur.qm, cur.qv, cur.am, vs, h, s_lut, mt, vt);
+        const int64_t e = i * d.cols + col0;
+        store8_f32(w + e, wv);
+        float am_new = absmax8(mt);
+        am_new = fmaxf(am_new, __shfl_xor_sync(half_mask, am_new, 8));
+        am_new = fmaxf(am_new, __shfl_xor_sync(half_mask, am_new, 4));
+        am_new = fmaxf(am_new, __shfl_xor_sync(half_mask, am_new, 2));
+        am_new = fmaxf(am_new, __shfl_xor_sync(half_mask, am_new, 1));
+        if ((lane & 15) == 0) m_scale[e >> 7] = am_new;
+        *reinterpret_cast<uint32_t*>(d.m_codes + (e >> 1)) = quantize8_de(mt, scale_rcp(am_new), s_lut);
+        *reinterpret_cast<uint32_t*>(d.v_codes + (e >> 1)) = quantize8_lin(vt, vr);
+        if (more) cur = nxt;
     }
 }
 
 // ---- pass 2, flat (element-indexed) tensors: block-wise v, or rank-1 with arbitrary cols ------
 
-template <bool BF16, bool RANK1>
+template <bool BF16, bool RANK1, bool EXACT>
 __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restrict__ w, const void* __restrict__ g,
-                                           int tile, int phase, const Hyper& h, const float* s_de) {
+                                           int tile, int phase, const Hyper& h, const unsigned char* s_lut) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const float* rc_old = d.rc[phase];
     const float* rcp_new = d.rcp_new;
@@ -229,7 +282,7 @@ __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restric
 #pragma unroll
             for (int k = 0; k < 8; ++k) vs[k] = av;
         }
-        moments_and_update8(wv, gv, qm, qv, am, vs, h, s_de, mt, vt);
+        moments_and_update8<EXACT>(wv, gv, qm, qv, am, vs, h, s_lut, mt, vt);
         if (!full) {   // elements beyond the tensor must not reach a block maximum
 #pragma unroll
             for (int k = 0; k < 8; ++k) if (e + k >= d.numel) { mt[k] = 0.0f; vt[k] = 0.0f; }
@@ -243,7 +296,7 @@ __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restric
             if (lane_live && (lane & 15) == 0) d.v_bscale[e >> 7] = av_new;
         }
         if (lane_live && (lane & 15) == 0) d.m_scale[e >> 7] = am_new;
-        const uint32_t qm_new = quantize8_de(mt, scale_rcp(am_new));
+        const uint32_t qm_new = quantize8_de(mt, scale_rcp(am_new), s_lut);
         const uint32_t qv_new = quantize8_lin(vt, vr);
         if (full) {
             store8_f32(w + e, wv);
@@ -259,7 +312,7 @@ __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restric
 
 // ---- pass 2, small tensors with fp32 states (App. C.1) ------------------------------------------
 
-template <bool BF16>
+template <bool BF16, bool EXACT>
 __device__ __forceinline__ void pass2_fp32(const TensorDesc& d, float* __restrict__ w, const void* __restrict__ g,
                                            int tile, const Hyper& h) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -279,7 +332,7 @@ __device__ __forceinline__ void pass2_fp32(const TensorDesc& d, float* __restric
         for (int k = 0; k < 8; ++k) {
             m[k] = ema_m(m[k], gv[k], h);
             v[k] = ema_v(v[k], gv[k], h);
-            wv[k] = adam_update(wv[k], m[k], v[k], h);
+            wv[k] = update_param<EXACT>(wv[k], m[k], v[k], h);
         }
         if (full) {
             store8_f32(w + e, wv); store8_f32(d.m32 + e, m); store8_f32(d.v32 + e, v);
@@ -289,10 +342,10 @@ __device__ __forceinline__ void pass2_fp32(const TensorDesc& d, float* __restric
     }
 }
 
-template <bool BF16>
+template <bool BF16, bool EXACT>
 __global__ void __launch_bounds__(kThreads, 2) pass2_kernel(StepArgs a) {
-    __shared__ float s_de[16];
-    if (threadIdx.x < 16) s_de[threadIdx.x] = kDeTable[threadIdx.x];
+    __shared__ __align__(16) unsigned char s_lut[kLutSmemBytes];
+    load_lut_smem(s_lut);
     __syncthreads();
     for (int tile = blockIdx.x; tile < a.total_tiles; tile += gridDim.x) {
         const int t = find_tensor(a.tile_start, a.n_tensors, tile);
@@ -301,10 +354,10 @@ __global__ void __launch_bounds__(kThreads, 2) pass2_kernel(StepArgs a) {
         const void* g = a.grads[t];
         const int local = tile - __ldg(a.tile_start + t);
         switch (d.kind) {
-            case K_RANK1_FAST: pass2_rank1_fast<BF16>(d, w, g, local, a.phase, a.h, s_de); break;
-            case K_RANK1_FLAT: pass2_flat<BF16, true>(d, w, g, local, a.phase, a.h, s_de); break;
-            case K_BLOCK:      pass2_flat<BF16, false>(d, w, g, local, a.phase, a.h, s_de); break;
-            default:           pass2_fp32<BF16>(d, w, g, local, a.h); break;
+            case K_RANK1_FAST: pass2_rank1_fast<BF16, EXACT>(d, w, g, local, a.phase, a.h, s_lut); break;
+            case K_RANK1_FLAT: pass2_flat<BF16, true, EXACT>(d, w, g, local, a.phase, a.h, s_lut); break;
+            case K_BLOCK:      pass2_flat<BF16, false, EXACT>(d, w, g, local, a.phase, a.h, s_lut); break;
+            default:           pass2_fp32<BF16, EXACT>(d, w, g, local, a.h); break;
         }
     }
 }
@@ -337,7 +390,7 @@ __device__ __forceinline__ void pass1_rank1_fast(const TensorDesc& d, const void
             const float r_old = __ldg(rc_old + i);
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
-                float v = __fmul_rn(lin_value((qv >> (4 * k)) & 15u), fminf(r_old, c_old[k]));
+                float v = __fmul_rn(lin_value_k(qv, k), fminf(r_old, c_old[k]));
                 float vt = ema_v(v, gv[k], h);
                 r_max = fmaxf(r_max, vt);
                 c_max[k] = fmaxf(c_max[k], vt);
@@ -420,10 +473,15 @@ cudaError_t launch_pass1(const StepArgs& a, bool bf16, int grid, cudaStream_t s)
     return cudaGetLastError();
 }
 
-cudaError_t launch_pass2(const StepArgs& a, bool bf16, int grid, cudaStream_t s) {
+cudaError_t launch_pass2(const StepArgs& a, bool bf16, bool exact, int grid, cudaStream_t s) {
     if (a.total_tiles <= 0) return cudaSuccess;
-    if (bf16) pass2_kernel<true><<<grid, kThreads, 0, s>>>(a);
-    else pass2_kernel<false><<<grid, kThreads, 0, s>>>(a);
+    if (bf16) {
+        if (exact) pass2_kernel<true, true><<<grid, kThreads, 0, s>>>(a);
+        else pass2_kernel<true, false><<<grid, kThreads, 0, s>>>(a);
+    } else {
+        if (exact) pass2_kernel<false, true><<<grid, kThreads, 0, s>>>(a);
+        else pass2_kernel<false, false><<<grid, kThreads, 0, s>>>(a);
+    }
     return cudaGetLastError();
 }
 
@@ -438,7 +496,7 @@ cudaError_t launch_rcp(const float* src, float* dst, int64_t n, cudaStream_t s) 
 cudaError_t step_kernel_occupancy(int* p1, int* p2) {
     cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(p1, pass1_kernel<true>, kThreads, 0);
     if (e != cudaSuccess) return e;
-    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(p2, pass2_kernel<true>, kThreads, 0);
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(p2, pass2_kernel<true, false>, kThreads, 0);
 }
 
 }  // namespace lpmm

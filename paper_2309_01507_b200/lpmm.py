@@ -19,6 +19,7 @@ F32, BF16 = 0, 1
 NORM_BLOCK, NORM_RANK1 = 0, 1
 MAP_DE_SIGNED, MAP_LINEAR_NOZERO = 0, 1
 V_RANK1, V_BLOCK = 0, 1
+UPDATE_FAST, UPDATE_IEEE = 0, 1
 FORCE_QUANT, FORCE_FP32 = 1, 2
 Q_GIVEN_SCALES = 1
 KIND_FP32, KIND_BLOCK, KIND_RANK1 = 0, 1, 2
@@ -36,11 +37,11 @@ class Shape(C.Structure):
 
 class Config(C.Structure):
     _fields_ = [("bits", C.c_int32), ("m_block", C.c_int32), ("v_block", C.c_int32), ("v_mode", C.c_int32),
-                ("min_quant_numel", C.c_int64)]
+                ("min_quant_numel", C.c_int64), ("update_math", C.c_int32), ("reserved", C.c_int32)]
 
 
-def default_config(v_mode: int = V_RANK1, min_quant_numel: int = 4096) -> Config:
-    return Config(4, 128, 128, v_mode, min_quant_numel)
+def default_config(v_mode: int = V_RANK1, min_quant_numel: int = 4096, update_math: int = 0) -> Config:
+    return Config(4, 128, 128, v_mode, min_quant_numel, update_math, 0)
 
 
 class LpmmError(RuntimeError):

@@ -99,29 +99,32 @@ def test_rank1_quantizer_matches_oracle(rows, cols):
 
 # ------------------------------------------------------------------ the fused step
 
-def test_single_matrix_config_ten_steps():
+@pytest.mark.parametrize("update_math", [lpmm.UPDATE_FAST, lpmm.UPDATE_IEEE])
+def test_single_matrix_config_ten_steps(update_math):
     wl = workloads.single_matrix()
-    pair = Pair(wl.tensors, hyper_of(wl), workload_index=wl.index)
+    pair = Pair(wl.tensors, hyper_of(wl), workload_index=wl.index, config=lpmm.default_config(update_math=update_math))
     kinds = [lpmm.state_view(pair.state, i)["kind"] for i in range(2)]
     assert kinds == [lpmm.KIND_RANK1, lpmm.KIND_BLOCK]          # bias forced onto the quantized 1-D path
     seen_v, seen_m = set(), set()
     for t in range(1, wl.steps + 1):
         pair.step(t, pair.grads_for(t))
-        pair.compare(tol=1e-6)
+        # IEEE update math follows the oracle's operation order: parameters are then bit-identical too
+        pair.compare(tol=1e-6, exact_params=(update_math == lpmm.UPDATE_IEEE))
         seen_m |= set(np.unique(oracle.unpack4(pair.ostate[0].m_codes, 1024 * 4096)).tolist())
         seen_v |= set(np.unique(oracle.unpack4(pair.ostate[0].v_codes, 1024 * 4096)).tolist())
     assert seen_m == set(range(16)) and seen_v == set(range(16))
     assert pair.state.last_launches == 3
 
 
-@pytest.mark.parametrize("grad_dtype", [torch.float32, torch.bfloat16])
-def test_shape_zoo_multi_tensor(grad_dtype):
+@pytest.mark.parametrize("grad_dtype,update_math", [(torch.float32, lpmm.UPDATE_FAST), (torch.bfloat16, lpmm.UPDATE_FAST),
+                                                    (torch.float32, lpmm.UPDATE_IEEE)])
+def test_shape_zoo_multi_tensor(grad_dtype, update_math):
     specs = [_mat(96, 256), _mat(33, 77), _mat(5, 1000), _mat(130, 384), _mat(64, 1024), _mat(8, 2048),
              _mat(1, 8192), _mat(8192, 1), _mat(300, 640), _mat(257, 129), _mat(70, 128),
              _vec(50265), _vec(4097), _vec(4096), _vec(4096, force_quant=True), _vec(1), _vec(300),
              _mat(16, 16), _mat(64, 64), _mat(65, 64), _vec(12345)]
     hyper = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
-    pair = Pair(specs, hyper, grad_dtype=grad_dtype, workload_index=7)
+    pair = Pair(specs, hyper, grad_dtype=grad_dtype, workload_index=7, config=lpmm.default_config(update_math=update_math))
     for t in range(1, 6):
         grads = pair.grads_for(t, outlier_p=0.0 if t % 2 == 0 else 1e-3)
         if t == 3:
@@ -130,7 +133,9 @@ def test_shape_zoo_multi_tensor(grad_dtype):
             grads[11].zero_()                              # an all-zero gradient
         if t == 4:
             grads[0][5, 7] = 3.0e4                         # one huge outlier
-            grads[1].mul_(1e-18)                           # second moment in the denormal range
+            grads[3].mul_(1e-18)                           # second moments in the denormal range
+            grads[9].mul_(1e-18)
+            grads[12].mul_(1e-18)
         pair.step(t, grads)
         pair.compare(tol=1e-6)
 
