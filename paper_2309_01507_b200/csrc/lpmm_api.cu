@@ -355,7 +355,9 @@ lpmm_status lpmm_adamw4_step(lpmm_state* st, void* const* d_params, const void* 
     if (ev[2]) LPMM_CUDA(cudaEventRecord(ev[2], s));
     a.tile_start = reinterpret_cast<const int32_t*>(st->arena + st->L.tiles2);
     a.total_tiles = st->total2;
-    LPMM_CUDA(launch_pass2(a, bf16, st->cfg.update_math == LPMM_UPDATE_IEEE, st->grid2, s));
+    // the approximate update flushes a denormal v^ before the square root: only safe with a real eps
+    const bool ieee_update = (st->cfg.update_math == LPMM_UPDATE_IEEE) || eps < 1e-30f;
+    LPMM_CUDA(launch_pass2(a, bf16, ieee_update, st->grid2, s));
     if (ev[3]) LPMM_CUDA(cudaEventRecord(ev[3], s));
     launches += 1;
     st->phase ^= 1;

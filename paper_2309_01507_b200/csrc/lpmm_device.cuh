@@ -133,12 +133,14 @@ __device__ __forceinline__ float adam_update(float w, float mt, float vt, const 
 
 // The same update with one approximate square root and one approximate reciprocal (each within about
 // one ulp) and the constant divisions folded into host-side factors: a handful of roundings away from
-// adam_update(), far inside the 1e-6 * max(|w|, lr) parameter tolerance. The stored states never
-// depend on this function.
+// adam_update(), far inside the 1e-6 * max(|w|, lr) parameter tolerance. A denormal bias-corrected
+// second moment is flushed to zero before the square root, which is harmless once eps is added; the host
+// therefore selects adam_update() instead when eps is (almost) zero. The stored states never depend on
+// this function.
 __device__ __forceinline__ float adam_update_fast(float w, float mt, float vt, const Hyper& h) {
     float sq, rc;
-    asm("sqrt.approx.f32 %0, %1;" : "=f"(sq) : "f"(__fmul_rn(vt, h.rbc2)));
-    asm("rcp.approx.f32 %0, %1;" : "=f"(rc) : "f"(__fadd_rn(sq, h.eps)));
+    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(sq) : "f"(__fmul_rn(vt, h.rbc2)));
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rc) : "f"(__fadd_rn(sq, h.eps)));
     const float upd = __fmul_rn(__fmul_rn(mt, h.step_size), rc);
     return __fmaf_rn(w, h.decay, -upd);
 }

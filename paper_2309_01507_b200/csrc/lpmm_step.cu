@@ -98,28 +98,38 @@ __device__ __forceinline__ void store_codes_guard(uint8_t* codes, int64_t e, int
 
 // ---- per-lane arithmetic ----------------------------------------------------------------------
 
-__device__ __forceinline__ float lin_value_k(uint32_t word, int k) {   // k is a compile-time constant after unrolling
-    const int shift = 4 * k;
-    const uint32_t moved = (shift <= 19) ? (word << (19 - shift)) : (word >> (shift - 19));
-    return __fadd_rn(__uint_as_float((moved & 0x00780000u) | 0x3f800000u), -0.9375f);   // (q + 1) / 16, exact
-}
-
 template <bool EXACT>
 __device__ __forceinline__ float update_param(float w, float mt, float vt, const Hyper& h) {
     return EXACT ? adam_update(w, mt, vt, h) : adam_update_fast(w, mt, vt, h);
 }
 
+// Per-lane constants of the shuffle-based table lookups: lane l of every 16-lane group holds entry
+// l & 15 of the signed DE table and of the linear table; a code is dequantized by reading the lane whose
+// index is the code (shuffle width 16 takes the source lane modulo 16, so the nibble needs no masking).
+struct LaneTables {
+    float de;    // T_DE[lane & 15]
+    float lin;   // (lane & 15 + 1) / 16
+    unsigned mask;   // the 16 lanes of this lane's group
+};
+__device__ __forceinline__ LaneTables make_lane_tables() {
+    const int lane = threadIdx.x & 31;
+    LaneTables t;
+    t.de = kDeTable[lane & 15];
+    t.lin = __fmul_rn((float)((lane & 15) + 1), 0.0625f);
+    t.mask = 0xffffu << (lane & 16);
+    return t;
+}
+
 // Dequantize (Sec. 2.2), update the moments (Eq. 1) and the parameters for 8 elements.
-// vs[k] is the old scale of element k's second moment, am the old scale of its first-moment block.
+// m_prod is T_DE[lane & 15] * (old block scale of m); vs[k] the old scale of element k's second moment.
 template <bool EXACT>
 __device__ __forceinline__ void moments_and_update8(float (&w)[8], const float (&g)[8], uint32_t qm, uint32_t qv,
-                                                    float am, const float (&vs)[8], const Hyper& h,
-                                                    const unsigned char* s_lut, float (&mt)[8], float (&vt)[8]) {
-    const float* s_de = reinterpret_cast<const float*>(s_lut + kLutDeTableOffset);
+                                                    float m_prod, const float (&vs)[8], const Hyper& h,
+                                                    const LaneTables& lt, float (&mt)[8], float (&vt)[8]) {
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
-        float m = __fmul_rn(s_de[(qm >> (4 * k)) & 15u], am);
-        float v = __fmul_rn(lin_value_k(qv, k), vs[k]);
+        const float m = __shfl_sync(lt.mask, m_prod, (int)(qm >> (4 * k)), 16);
+        const float v = __fmul_rn(__shfl_sync(lt.mask, lt.lin, (int)(qv >> (4 * k)), 16), vs[k]);
         mt[k] = ema_m(m, g[k], h);
         vt[k] = ema_v(v, g[k], h);
         w[k] = update_param<EXACT>(w[k], mt[k], vt[k], h);
@@ -131,6 +141,13 @@ __device__ __forceinline__ float absmax8(const float (&x)[8]) {
 #pragma unroll
     for (int k = 0; k < 8; ++k) a = fmaxf(a, fabsf(x[k]));
     return a;
+}
+__device__ __forceinline__ float group_max(float x, unsigned mask) {   // over the 16 lanes of one block
+    x = fmaxf(x, __shfl_xor_sync(mask, x, 8));
+    x = fmaxf(x, __shfl_xor_sync(mask, x, 4));
+    x = fmaxf(x, __shfl_xor_sync(mask, x, 2));
+    x = fmaxf(x, __shfl_xor_sync(mask, x, 1));
+    return x;
 }
 
 // Eight nearest codes packed little-nibble-first: acc = acc * 16 + code, from element 7 down to 0.
@@ -147,6 +164,18 @@ __device__ __forceinline__ uint32_t quantize8_lin(const float (&x)[8], const flo
     return q - kMagicBits * 0x11111111u;   // removes the eight 2^23 patterns (mod 2^32)
 }
 
+template <bool BF16>
+__device__ __forceinline__ void unpack_grad8(const uint4& g0, const uint4& g1, float (&g)[8]) {
+    if (BF16) {
+        g[0] = bf16_lo(g0.x); g[1] = bf16_hi(g0.x); g[2] = bf16_lo(g0.y); g[3] = bf16_hi(g0.y);
+        g[4] = bf16_lo(g0.z); g[5] = bf16_hi(g0.z); g[6] = bf16_lo(g0.w); g[7] = bf16_hi(g0.w);
+    } else {
+        g[0] = __uint_as_float(g0.x); g[1] = __uint_as_float(g0.y); g[2] = __uint_as_float(g0.z);
+        g[3] = __uint_as_float(g0.w); g[4] = __uint_as_float(g1.x); g[5] = __uint_as_float(g1.y);
+        g[6] = __uint_as_float(g1.z); g[7] = __uint_as_float(g1.w);
+    }
+}
+
 // ---- pass 2, rank-1 tensors with cols % 128 == 0 ---------------------------------------------------
 
 template <bool BF16>
@@ -157,83 +186,100 @@ struct RowRegs {           // one lane's share of one row: raw, still packed
     float am, r_old, r_rcp;
 };
 
-template <bool BF16>
-__device__ __forceinline__ void load_row(RowRegs<BF16>& r, const TensorDesc& d, const float* __restrict__ w,
-                                         const void* __restrict__ g, const float* rc_old, const float* rcp_new,
-                                         int64_t i, int64_t col0) {
-    const int64_t e = i * d.cols + col0;
-    r.w0 = *reinterpret_cast<const float4*>(w + e);
-    r.w1 = *reinterpret_cast<const float4*>(w + e + 4);
-    if (BF16) {
-        r.g0 = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(g) + e));
-    } else {
-        r.g0 = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(g) + e));
-        r.g1 = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(g) + e + 4));
-    }
-    r.qm = *reinterpret_cast<const uint32_t*>(d.m_codes + (e >> 1));
-    r.qv = *reinterpret_cast<const uint32_t*>(d.v_codes + (e >> 1));
-    r.am = d.m_scale[e >> 7];
-    r.r_old = __ldg(rc_old + i);
-    r.r_rcp = __ldg(rcp_new + i);
-}
+// Per-lane view of a tile: base pointers at the lane's first element and 32-bit offsets from there.
+struct TileView {
+    float* w;
+    const void* g;
+    uint8_t* m_codes;
+    uint8_t* v_codes;
+    float* m_scale;
+    const float* r_old;
+    const float* r_rcp;
+    uint32_t row_step;     // elements between two rows this warp handles
+    uint32_t row_stride;   // rows between them
+};
 
 template <bool BF16>
-__device__ __forceinline__ void unpack_grad(const RowRegs<BF16>& r, float (&g)[8]) {
+__device__ __forceinline__ void load_row(RowRegs<BF16>& r, const TileView& t, uint32_t k) {
+    const uint32_t off = k * t.row_step;
+    r.w0 = *reinterpret_cast<const float4*>(t.w + off);
+    r.w1 = *reinterpret_cast<const float4*>(t.w + off + 4);
     if (BF16) {
-        g[0] = bf16_lo(r.g0.x); g[1] = bf16_hi(r.g0.x); g[2] = bf16_lo(r.g0.y); g[3] = bf16_hi(r.g0.y);
-        g[4] = bf16_lo(r.g0.z); g[5] = bf16_hi(r.g0.z); g[6] = bf16_lo(r.g0.w); g[7] = bf16_hi(r.g0.w);
+        r.g0 = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(t.g) + off));
     } else {
-        g[0] = __uint_as_float(r.g0.x); g[1] = __uint_as_float(r.g0.y); g[2] = __uint_as_float(r.g0.z);
-        g[3] = __uint_as_float(r.g0.w); g[4] = __uint_as_float(r.g1.x); g[5] = __uint_as_float(r.g1.y);
-        g[6] = __uint_as_float(r.g1.z); g[7] = __uint_as_float(r.g1.w);
+        r.g0 = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(t.g) + off));
+        r.g1 = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(t.g) + off + 4));
     }
+    r.qm = *reinterpret_cast<const uint32_t*>(t.m_codes + (off >> 1));
+    r.qv = *reinterpret_cast<const uint32_t*>(t.v_codes + (off >> 1));
+    r.am = t.m_scale[off >> 7];
+    r.r_old = __ldg(t.r_old + k * t.row_stride);
+    r.r_rcp = __ldg(t.r_rcp + k * t.row_stride);
+}
+
+template <bool BF16, bool EXACT>
+__device__ __forceinline__ void process_row(const RowRegs<BF16>& r, const TileView& t, uint32_t k,
+                                            const float (&c_old)[8], const float (&c_rcp)[8], const Hyper& h,
+                                            const LaneTables& lt, const unsigned char* s_lut) {
+    const uint32_t off = k * t.row_step;
+    float wv[8] = {r.w0.x, r.w0.y, r.w0.z, r.w0.w, r.w1.x, r.w1.y, r.w1.z, r.w1.w};
+    float gv[8], mt[8], vt[8], vs[8], vr[8];
+    unpack_grad8<BF16>(r.g0, r.g1, gv);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        vs[j] = fminf(r.r_old, c_old[j]);      // Sec. 4.2: scale = min(r_i, c_j)
+        vr[j] = fmaxf(r.r_rcp, c_rcp[j]);      // 1/min(r', c') = max(1/r', 1/c')
+    }
+    moments_and_update8<EXACT>(wv, gv, r.qm, r.qv, __fmul_rn(lt.de, r.am), vs, h, lt, mt, vt);
+    store8_f32(t.w + off, wv);
+    const float am_new = group_max(absmax8(mt), lt.mask);
+    if ((threadIdx.x & 15) == 0) t.m_scale[off >> 7] = am_new;
+    *reinterpret_cast<uint32_t*>(t.m_codes + (off >> 1)) = quantize8_de(mt, scale_rcp(am_new), s_lut);
+    *reinterpret_cast<uint32_t*>(t.v_codes + (off >> 1)) = quantize8_lin(vt, vr);
 }
 
 template <bool BF16, bool EXACT>
 __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __restrict__ w, const void* __restrict__ g,
-                                                 int tile, int phase, const Hyper& h, const unsigned char* s_lut) {
+                                                 int tile, int phase, const Hyper& h, const LaneTables& lt,
+                                                 const unsigned char* s_lut) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int wx = d.wx, wy_count = kWarps / wx;
     const int tx = tile % d.tiles_x, ty = tile / d.tiles_x;
     const int64_t col0 = (int64_t)tx * (kWarpElems * wx) + (warp % wx) * kWarpElems + lane * kLaneElems;
     if (col0 >= d.cols) return;   // cols % 128 == 0: a whole 16-lane group (one block) is in or out together
-    // Shuffles below use a half-warp mask, so the other half may be absent.
-    const unsigned half_mask = 0xffffu << (lane & 16);
-    const float* rc_old = d.rc[phase];
+    const float* rc_old = (phase ? d.rc[1] : d.rc[0]);
     const float* rcp_new = d.rcp_new;
-    float* m_scale = d.m_scale;
+    const int64_t row0 = (int64_t)ty * d.tile_rows + warp / wx;
+    const int64_t row_end = min((int64_t)(ty + 1) * d.tile_rows, d.rows);
+    if (row0 >= row_end) return;
+    const uint32_t nrows = (uint32_t)((row_end - row0 + wy_count - 1) / wy_count);
 
     float c_old[8], c_rcp[8];
     load8_f32(rc_old + d.c_off + col0, c_old);
     load8_f32(rcp_new + d.c_off + col0, c_rcp);
-    const int64_t row_end = min((int64_t)(ty + 1) * d.tile_rows, d.rows);
-    int64_t i = (int64_t)ty * d.tile_rows + warp / wx;
-    if (i >= row_end) return;
-    RowRegs<BF16> cur, nxt;
-    load_row<BF16>(cur, d, w, g, rc_old, rcp_new, i, col0);
-    for (; i < row_end; i += wy_count) {
-        const bool more = i + wy_count < row_end;
-        if (more) load_row<BF16>(nxt, d, w, g, rc_old, rcp_new, i + wy_count, col0);   // prefetch the next row
-        float wv[8] = {cur.w0.x, cur.w0.y, cur.w0.z, cur.w0.w, cur.w1.x, cur.w1.y, cur.w1.z, cur.w1.w};
-        float gv[8], mt[8], vt[8], vs[8], vr[8];
-        unpack_grad<BF16>(cur, gv);
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            vs[k] = fminf(cur.r_old, c_old[k]);      // Sec. 4.2: scale = min(r_i, c_j)
-            vr[k] = fmaxf(cur.r_rcp, c_rcp[k]);      // 1/min(r', c') = max(1/r', 1/c')
-        }
-        moments_and_update8<EXACT>(wv, gv, cur.qm, cur.qv, cur.am, vs, h, s_lut, mt, vt);
-        const int64_t e = i * d.cols + col0;
-        store8_f32(w + e, wv);
-        float am_new = absmax8(mt);
-        am_new = fmaxf(am_new, __shfl_xor_sync(half_mask, am_new, 8));
-        am_new = fmaxf(am_new, __shfl_xor_sync(half_mask, am_new, 4));
-        am_new = fmaxf(am_new, __shfl_xor_sync(half_mask, am_new, 2));
-        am_new = fmaxf(am_new, __shfl_xor_sync(half_mask, am_new, 1));
-        if ((lane & 15) == 0) m_scale[e >> 7] = am_new;
-        *reinterpret_cast<uint32_t*>(d.m_codes + (e >> 1)) = quantize8_de(mt, scale_rcp(am_new), s_lut);
-        *reinterpret_cast<uint32_t*>(d.v_codes + (e >> 1)) = quantize8_lin(vt, vr);
-        if (more) cur = nxt;
+    const int64_t e0 = row0 * d.cols + col0;
+    TileView t;
+    t.w = w + e0;
+    t.g = BF16 ? static_cast<const void*>(reinterpret_cast<const uint16_t*>(g) + e0)
+               : static_cast<const void*>(reinterpret_cast<const float*>(g) + e0);
+    t.m_codes = d.m_codes + (e0 >> 1);
+    t.v_codes = d.v_codes + (e0 >> 1);
+    t.m_scale = d.m_scale + (e0 >> 7);
+    t.r_old = rc_old + row0;
+    t.r_rcp = rcp_new + row0;
+    t.row_step = (uint32_t)(wy_count * d.cols);
+    t.row_stride = (uint32_t)wy_count;
+
+    // Two register sets alternate: while one row is processed the next one is already in flight.
+    RowRegs<BF16> ra, rb;
+    load_row<BF16>(ra, t, 0);
+    for (uint32_t k = 0; k < nrows; k += 2) {
+        const bool has_b = k + 1 < nrows;
+        if (has_b) load_row<BF16>(rb, t, k + 1);
+        process_row<BF16, EXACT>(ra, t, k, c_old, c_rcp, h, lt, s_lut);
+        if (!has_b) break;
+        if (k + 2 < nrows) load_row<BF16>(ra, t, k + 2);
+        process_row<BF16, EXACT>(rb, t, k + 1, c_old, c_rcp, h, lt, s_lut);
     }
 }
 
@@ -241,9 +287,10 @@ __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __r
 
 template <bool BF16, bool RANK1, bool EXACT>
 __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restrict__ w, const void* __restrict__ g,
-                                           int tile, int phase, const Hyper& h, const unsigned char* s_lut) {
+                                           int tile, int phase, const Hyper& h, const LaneTables& lt,
+                                           const unsigned char* s_lut) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const float* rc_old = d.rc[phase];
+    const float* rc_old = (phase ? d.rc[1] : d.rc[0]);
     const float* rcp_new = d.rcp_new;
     for (int c = 0; c < d.flat_chunks; ++c) {
         const int64_t chunk = ((int64_t)tile * d.flat_chunks + c) * kWarps + warp;
@@ -264,7 +311,10 @@ __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restric
             qv = load_codes_guard(d.v_codes, e, d.numel);
         }
         const bool lane_live = e < d.numel;
-        const float am = lane_live ? d.m_scale[e >> 7] : 0.0f;
+        // every lane of a 16-lane group that still holds an element needs the block's scale: the
+        // shuffle-based table lookup reads T[q] * scale from the group's other lanes
+        const bool group_live = (e & ~(int64_t)127) < d.numel;
+        const float am = group_live ? d.m_scale[e >> 7] : 0.0f;
         if (RANK1) {
             int64_t i = e / d.cols, j = e - i * d.cols;
 #pragma unroll
@@ -282,7 +332,7 @@ __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restric
 #pragma unroll
             for (int k = 0; k < 8; ++k) vs[k] = av;
         }
-        moments_and_update8<EXACT>(wv, gv, qm, qv, am, vs, h, s_lut, mt, vt);
+        moments_and_update8<EXACT>(wv, gv, qm, qv, __fmul_rn(lt.de, am), vs, h, lt, mt, vt);
         if (!full) {   // elements beyond the tensor must not reach a block maximum
 #pragma unroll
             for (int k = 0; k < 8; ++k) if (e + k >= d.numel) { mt[k] = 0.0f; vt[k] = 0.0f; }
@@ -347,57 +397,142 @@ __global__ void __launch_bounds__(kThreads, 2) pass2_kernel(StepArgs a) {
     __shared__ __align__(16) unsigned char s_lut[kLutSmemBytes];
     load_lut_smem(s_lut);
     __syncthreads();
+    const LaneTables lt = make_lane_tables();
     for (int tile = blockIdx.x; tile < a.total_tiles; tile += gridDim.x) {
         const int t = find_tensor(a.tile_start, a.n_tensors, tile);
-        const TensorDesc& d = a.descs[t];
+        const TensorDesc d = a.descs[t];   // by value: the fields stay in registers across the stores below
         float* w = a.params[t];
         const void* g = a.grads[t];
         const int local = tile - __ldg(a.tile_start + t);
         switch (d.kind) {
-            case K_RANK1_FAST: pass2_rank1_fast<BF16, EXACT>(d, w, g, local, a.phase, a.h, s_lut); break;
-            case K_RANK1_FLAT: pass2_flat<BF16, true, EXACT>(d, w, g, local, a.phase, a.h, s_lut); break;
-            case K_BLOCK:      pass2_flat<BF16, false, EXACT>(d, w, g, local, a.phase, a.h, s_lut); break;
+            case K_RANK1_FAST: pass2_rank1_fast<BF16, EXACT>(d, w, g, local, a.phase, a.h, lt, s_lut); break;
+            case K_RANK1_FLAT: pass2_flat<BF16, true, EXACT>(d, w, g, local, a.phase, a.h, lt, s_lut); break;
+            case K_BLOCK:      pass2_flat<BF16, false, EXACT>(d, w, g, local, a.phase, a.h, lt, s_lut); break;
             default:           pass2_fp32<BF16, EXACT>(d, w, g, local, a.h); break;
         }
     }
 }
 
 // ---- pass 1: new row / column maxima of v_t for rank-1 tensors -----------------------------------
+//
+// Maxima are idempotent, so ragged edges are handled by clamping indices onto valid rows / column
+// groups (a duplicate contributes the same value again) instead of predicating the loads.
+
+constexpr int kP1Rows = 4;   // rows a lane keeps in flight per batch
+
+template <bool BF16>
+struct P1Row {             // one lane's share of one row
+    uint4 g0, g1;          // bf16: g0 only
+    uint32_t qv;
+    float r_old;
+};
+
+struct P1View {
+    const void* g;             // at the lane's column group, row 0 of the tensor
+    const uint8_t* v_codes;
+    const float* r_old;
+    uint32_t cols;
+    uint32_t last_row;         // last valid row of the tile
+};
+
+template <bool BF16>
+__device__ __forceinline__ void load_p1_batch(P1Row<BF16> (&b)[kP1Rows], const P1View& t, uint32_t row, uint32_t stride) {
+#pragma unroll
+    for (int u = 0; u < kP1Rows; ++u) {
+        const uint32_t rr = min(row + u * stride, t.last_row);
+        const uint64_t e = (uint64_t)rr * t.cols;
+        if (BF16) {
+            b[u].g0 = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(t.g) + e));
+        } else {
+            b[u].g0 = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(t.g) + e));
+            b[u].g1 = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(t.g) + e + 4));
+        }
+        b[u].qv = __ldg(reinterpret_cast<const uint32_t*>(t.v_codes + (e >> 1)));
+        b[u].r_old = __ldg(t.r_old + rr);
+    }
+}
+
+// Maxima of four per-lane values over the warp with 6 shuffles: afterwards the lanes with
+// (lane & 7) == 0 hold the warp-wide maximum of value number 2 * bit4(lane) + bit3(lane).
+__device__ __forceinline__ float warp_max4(const float (&r)[4], int lane) {
+    const bool h16 = lane & 16, h8 = lane & 8;
+    float k0 = h16 ? r[2] : r[0], k1 = h16 ? r[3] : r[1];
+    const float s0 = h16 ? r[0] : r[2], s1 = h16 ? r[1] : r[3];
+    k0 = fmaxf(k0, __shfl_xor_sync(0xffffffffu, s0, 16));
+    k1 = fmaxf(k1, __shfl_xor_sync(0xffffffffu, s1, 16));
+    float k = h8 ? k1 : k0;
+    const float s = h8 ? k0 : k1;
+    k = fmaxf(k, __shfl_xor_sync(0xffffffffu, s, 8));
+    k = fmaxf(k, __shfl_xor_sync(0xffffffffu, k, 4));
+    k = fmaxf(k, __shfl_xor_sync(0xffffffffu, k, 2));
+    k = fmaxf(k, __shfl_xor_sync(0xffffffffu, k, 1));
+    return k;
+}
+
+template <bool BF16>
+__device__ __forceinline__ void p1_process_batch(const P1Row<BF16> (&b)[kP1Rows], const P1View& t, uint32_t row,
+                                                 uint32_t stride, const float (&c_old)[8], float (&c_max)[8],
+                                                 const Hyper& h, const LaneTables& lt, float* rc_new) {
+    const int lane = threadIdx.x & 31;
+    float r_max[kP1Rows];
+#pragma unroll
+    for (int u = 0; u < kP1Rows; ++u) {
+        float gv[8];
+        unpack_grad8<BF16>(b[u].g0, b[u].g1, gv);
+        float rm = 0.0f;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const float tl = __shfl_sync(0xffffffffu, lt.lin, (int)(b[u].qv >> (4 * k)), 16);
+            const float vt = ema_v(__fmul_rn(tl, fminf(b[u].r_old, c_old[k])), gv[k], h);
+            rm = fmaxf(rm, vt);
+            c_max[k] = fmaxf(c_max[k], vt);
+        }
+        r_max[u] = rm;
+    }
+    const float rm = warp_max4(r_max, lane);
+    const uint32_t which = ((lane >> 4) & 1) * 2 + ((lane >> 3) & 1);
+    if ((lane & 7) == 0) atomic_max_nonneg(rc_new + min(row + which * stride, t.last_row), rm);
+}
 
 template <bool BF16>
 __device__ __forceinline__ void pass1_rank1_fast(const TensorDesc& d, const void* __restrict__ g, int tile, int phase,
-                                                 const Hyper& h, float* s_col) {
+                                                 const Hyper& h, const LaneTables& lt, float* s_col) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int wx = d.wx, wy_count = kWarps / wx;
     const int tx = tile % d.tiles_x, ty = tile / d.tiles_x;
-    const int64_t col0 = (int64_t)tx * (kWarpElems * wx) + (warp % wx) * kWarpElems + lane * kLaneElems;
-    const bool active = col0 < d.cols;
-    const float* rc_old = d.rc[phase];
-    float* rc_new = d.rc[phase ^ 1];
+    int64_t col0 = (int64_t)tx * (kWarpElems * wx) + (warp % wx) * kWarpElems + lane * kLaneElems;
+    if (col0 >= d.cols) col0 -= 128;   // only when cols % 256 == 128: the upper half-warp repeats the lower one
+    const float* rc_old = (phase ? d.rc[1] : d.rc[0]);
+    float* rc_new = (phase ? d.rc[0] : d.rc[1]);
 
     float c_old[8], c_max[8];
 #pragma unroll
-    for (int k = 0; k < 8; ++k) { c_old[k] = 0.0f; c_max[k] = 0.0f; }
-    if (active) load8_f32(rc_old + d.c_off + col0, c_old);
-    const int64_t row_end = min((int64_t)(ty + 1) * d.tile_rows, d.rows);
-    for (int64_t i = (int64_t)ty * d.tile_rows + warp / wx; i < row_end; i += wy_count) {
-        float r_max = 0.0f;
-        if (active) {
-            const int64_t e = i * d.cols + col0;
-            float gv[8];
-            load8_grad<BF16>(g, e, gv);
-            const uint32_t qv = __ldg(reinterpret_cast<const uint32_t*>(d.v_codes + (e >> 1)));
-            const float r_old = __ldg(rc_old + i);
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                float v = __fmul_rn(lin_value_k(qv, k), fminf(r_old, c_old[k]));
-                float vt = ema_v(v, gv[k], h);
-                r_max = fmaxf(r_max, vt);
-                c_max[k] = fmaxf(c_max[k], vt);
-            }
-        }
-        r_max = warp_max(r_max);
-        if (lane == 0 && active) atomic_max_nonneg(rc_new + i, r_max);
+    for (int k = 0; k < 8; ++k) c_max[k] = 0.0f;
+    load8_f32(rc_old + d.c_off + col0, c_old);
+    const uint32_t row_end = (uint32_t)min((int64_t)(ty + 1) * d.tile_rows, d.rows);
+    const uint32_t stride = (uint32_t)wy_count, batch = kP1Rows * stride;
+    P1View t;
+    t.g = BF16 ? static_cast<const void*>(reinterpret_cast<const uint16_t*>(g) + col0)
+               : static_cast<const void*>(reinterpret_cast<const float*>(g) + col0);
+    t.v_codes = d.v_codes + (col0 >> 1);
+    t.r_old = rc_old;
+    t.cols = (uint32_t)d.cols;
+    t.last_row = row_end - 1;
+
+    uint32_t i = (uint32_t)((int64_t)ty * d.tile_rows) + warp / wx;   // tile_rows >= warps down, so i < row_end ... or clamped
+    P1Row<BF16> ba[kP1Rows], bb[kP1Rows];
+    load_p1_batch<BF16>(ba, t, i, stride);
+    while (true) {
+        const bool has_b = i + batch < row_end;
+        if (has_b) load_p1_batch<BF16>(bb, t, i + batch, stride);
+        p1_process_batch<BF16>(ba, t, i, stride, c_old, c_max, h, lt, rc_new);
+        if (!has_b) break;
+        i += batch;
+        const bool has_a = i + batch < row_end;
+        if (has_a) load_p1_batch<BF16>(ba, t, i + batch, stride);
+        p1_process_batch<BF16>(bb, t, i, stride, c_old, c_max, h, lt, rc_new);
+        if (!has_a) break;
+        i += batch;
     }
     // Column maxima: combine the warps that share columns in shared memory, then one atomic per column.
     float* mine = s_col + warp * kWarpElems + lane * kLaneElems;
@@ -422,8 +557,8 @@ template <bool BF16>
 __device__ __forceinline__ void pass1_rank1_flat(const TensorDesc& d, const void* __restrict__ g, int tile, int phase,
                                                  const Hyper& h) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const float* rc_old = d.rc[phase];
-    float* rc_new = d.rc[phase ^ 1];
+    const float* rc_old = (phase ? d.rc[1] : d.rc[0]);
+    float* rc_new = (phase ? d.rc[0] : d.rc[1]);
     for (int c = 0; c < d.flat_chunks; ++c) {
         const int64_t chunk = ((int64_t)tile * d.flat_chunks + c) * kWarps + warp;
         const int64_t e = chunk * kWarpElems + lane * kLaneElems;
@@ -449,12 +584,13 @@ __device__ __forceinline__ void pass1_rank1_flat(const TensorDesc& d, const void
 template <bool BF16>
 __global__ void __launch_bounds__(kThreads, 2) pass1_kernel(StepArgs a) {
     __shared__ float s_col[kWarps * kWarpElems];
+    const LaneTables lt = make_lane_tables();
     for (int tile = blockIdx.x; tile < a.total_tiles; tile += gridDim.x) {
         const int t = find_tensor(a.tile_start, a.n_tensors, tile);
-        const TensorDesc& d = a.descs[t];
+        const TensorDesc d = a.descs[t];
         const void* g = a.grads[t];
         const int local = tile - __ldg(a.tile_start + t);
-        if (d.kind == K_RANK1_FAST) pass1_rank1_fast<BF16>(d, g, local, a.phase, a.h, s_col);
+        if (d.kind == K_RANK1_FAST) pass1_rank1_fast<BF16>(d, g, local, a.phase, a.h, lt, s_col);
         else pass1_rank1_flat<BF16>(d, g, local, a.phase, a.h);
     }
 }
