@@ -324,6 +324,7 @@ lpmm_status lpmm_adamw4_step(lpmm_state* st, void* const* d_params, const void* 
     a.h.bc1 = (float)(1.0 - std::pow((double)beta1, (double)step));   // Eq. 1: 1 - beta^t
     a.h.bc2 = (float)(1.0 - std::pow((double)beta2, (double)step));
     a.h.decay = 1.0f - lr * weight_decay;
+    a.h.one = 1.0f;
     {
         const double bc1 = 1.0 - std::pow((double)beta1, (double)step), bc2 = 1.0 - std::pow((double)beta2, (double)step);
         a.h.step_size = (float)((double)lr / bc1);

@@ -58,14 +58,6 @@ __device__ __forceinline__ float lin_value(uint32_t q) {  // (q+1)/16, exact
     return __fmul_rn((float)(q + 1u), 0.0625f);
 }
 
-// Same value without an integer conversion: `word` holds the nibble at bits [shift, shift+4); it is
-// moved to the top of the mantissa of 1.0f (giving 1 + q/16 exactly) and 15/16 is subtracted (exact).
-template <int SHIFT>
-__device__ __forceinline__ float lin_value_at(uint32_t word) {
-    const uint32_t moved = (SHIFT <= 19) ? (word << (19 - SHIFT)) : (word >> (SHIFT - 19));
-    return __fadd_rn(__uint_as_float((moved & 0x00780000u) | 0x3f800000u), -0.9375f);
-}
-
 // Nearest linear code as the low mantissa bits of 2^23 + ceil(max(16 n - 1.5, 0)), added with
 // round-up; valid for n <= 1 + 2^-22 (then the code is at most 15). The caller removes the 2^23 pattern.
 constexpr uint32_t kMagicBits = 0x4b000000u;  // 2^23 as binary32
@@ -74,35 +66,37 @@ __device__ __forceinline__ uint32_t lin_nearest_magic(float n) {
     return __float_as_uint(__fadd_ru(y, 8388608.0f));
 }
 
-// Shared-memory image used by the step kernel: the non-negative half of kDeLut at byte 0, the negative
-// half at byte 16384 (so that the sign bit of the key selects it without an extra instruction), and the
-// 16-entry dequantization table in between.
-constexpr int kLutNegOffset = 16384;
-constexpr int kLutDeTableOffset = 1024;
-constexpr int kLutSmemBytes = kLutNegOffset + kDeLutBins * 8;
+// Shared-memory image of the nearest-entry table, directly indexed by the top 12 bits of n (sign, exponent,
+// three mantissa bits): 2048 eight-byte entries for n >= 0 followed by 2048 for n < 0, so that no clamping is
+// needed and every bit pattern (NaN and infinities included) stays inside the table. Entries outside the 80
+// bins of kDeLut repeat the end codes: below 2^-9 the entry 0, from 2.0 upwards the extreme entry.
+constexpr int kLutSmemBytes = 2 * 2048 * 8;
 
 __device__ __forceinline__ void load_lut_smem(unsigned char* smem) {
-    for (int i = threadIdx.x; i < kDeLutBins; i += blockDim.x) {
-        reinterpret_cast<uint2*>(smem)[i] = kDeLut[i];
-        reinterpret_cast<uint2*>(smem + kLutNegOffset)[i] = kDeLut[kDeLutBins + i];
+    constexpr uint32_t kFirst = kDeLutKeyBias / 8;            // key of 2^-9
+    for (uint32_t i = threadIdx.x; i < 4096u; i += blockDim.x) {
+        const uint32_t key = i & 2047u, neg = i >> 11;
+        uint2 e;
+        if (key < kFirst) e = make_uint2(0x7f7fffffu, neg ? 8u : 7u);
+        else if (key >= kFirst + kDeLutBins) e = make_uint2(0x7f7fffffu, 15u);
+        else e = kDeLut[neg * kDeLutBins + key - kFirst];
+        reinterpret_cast<uint2*>(smem)[i] = e;
     }
-    if (threadIdx.x < 16) reinterpret_cast<float*>(smem + kLutDeTableOffset)[threadIdx.x] = kDeTable[threadIdx.x];
 }
 
-// Table-driven equivalent of de_nearest() for |n| < 2 (always true for m / blockmax(|m|)); NaN gives code 7.
+// Table-driven equivalent of de_nearest(): one lookup, one comparison. Codes of negative values are stored
+// as 15 - code and flipped back by the final xor.
 __device__ __forceinline__ uint32_t de_nearest_lut(float n, const unsigned char* smem) {
-    const float a = fminf(fmaxf(fabsf(n), kDeLutMinAbs), 1.9999999f);
     const uint32_t nb = __float_as_uint(n);
-    const uint32_t cs = (__float_as_uint(a) & 0x7fffffffu) | (nb & 0x80000000u);   // copysign(a, n)
-    const uint32_t off = (cs >> 17) & 0x7ff8u;      // bit 14 = sign -> +16384; bits 3..13 = key * 8
-    const uint2 e = *reinterpret_cast<const uint2*>(smem + off - kDeLutKeyBias);
-    const uint32_t c = e.y + (a > __uint_as_float(e.x) ? 1u : 0u);
+    const uint2 e = *reinterpret_cast<const uint2*>(smem + ((nb >> 17) & 0x7ff8u));
+    const uint32_t c = e.y + (fabsf(n) > __uint_as_float(e.x) ? 1u : 0u);
     return c ^ ((uint32_t)((int32_t)nb >> 31) & 15u);
 }
 
-// 1/s for a usable scale, 0 for a zero or denormal one (everything under it quantizes as zero).
+// 1/s (correctly rounded) for a usable scale, 0 for a zero or denormal one (everything under it
+// quantizes as zero).
 __device__ __forceinline__ float scale_rcp(float s) {
-    return (s >= kFltMin) ? __fdiv_rn(1.0f, s) : 0.0f;
+    return (s >= kFltMin) ? __frcp_rn(s) : 0.0f;
 }
 
 struct Hyper {
@@ -112,7 +106,77 @@ struct Hyper {
     float decay;       // 1 - lr * weight_decay
     float step_size;   // lr / bc1, evaluated in binary64 and rounded once (fast update)
     float rbc2;        // 1 / bc2, likewise
+    float one;         // 1.0f, passed as data (see ema_m2)
 };
+
+// The same constants as pairs, for the packed two-lane fp32 instructions of sm_100 (mul/add/fma.f32x2:
+// two independent IEEE operations per instruction, so results are bit-identical to the scalar forms).
+struct Hyper2 {
+    float2 beta1, omb1, beta2, omb2;
+    float2 rbc2, eps, neg_step, decay, one;
+};
+__device__ __forceinline__ float2 splat(float x) { return make_float2(x, x); }
+
+// Packed operations written as PTX with an explicit rounding mode: such instructions are never
+// contracted into a fused multiply-add, which the stored states rely on.
+__device__ __forceinline__ unsigned long long pack2(float2 a) {
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a.x), "f"(a.y));
+    return r;
+}
+__device__ __forceinline__ float2 unpack2(unsigned long long r) {
+    float2 a;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(a.x), "=f"(a.y) : "l"(r));
+    return a;
+}
+__device__ __forceinline__ float2 mul2_rn(float2 a, float2 b) {
+    unsigned long long d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(pack2(a)), "l"(pack2(b)));
+    return unpack2(d);
+}
+__device__ __forceinline__ float2 add2_rn(float2 a, float2 b) {
+    unsigned long long d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(pack2(a)), "l"(pack2(b)));
+    return unpack2(d);
+}
+__device__ __forceinline__ float2 add2_ru(float2 a, float2 b) {
+    unsigned long long d;
+    asm("add.rp.f32x2 %0, %1, %2;" : "=l"(d) : "l"(pack2(a)), "l"(pack2(b)));
+    return unpack2(d);
+}
+__device__ __forceinline__ float2 fma2_rn(float2 a, float2 b, float2 c) {
+    unsigned long long d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(pack2(a)), "l"(pack2(b)), "l"(pack2(c)));
+    return unpack2(d);
+}
+__device__ __forceinline__ Hyper2 make_hyper2(const Hyper& h) {
+    Hyper2 p;
+    p.beta1 = splat(h.beta1); p.omb1 = splat(h.omb1); p.beta2 = splat(h.beta2); p.omb2 = splat(h.omb2);
+    p.rbc2 = splat(h.rbc2); p.eps = splat(h.eps); p.neg_step = splat(-h.step_size); p.decay = splat(h.decay);
+    p.one = splat(h.one);
+    return p;
+}
+// Both products must be rounded before the sum (Eq. 1 evaluated operation by operation). The assembler
+// was observed to merge a packed multiply with a following packed add into a fused multiply-add even with
+// explicit rounding modes, so the sum is written as fma(p1, 1, p2) with the 1 supplied at run time:
+// fl(p1 * 1 + p2) = fl(p1 + p2) exactly, and nothing is left to merge.
+__device__ __forceinline__ float2 ema_m2(float2 m, float2 g, const Hyper2& h) {
+    return fma2_rn(mul2_rn(h.beta1, m), h.one, mul2_rn(h.omb1, g));
+}
+__device__ __forceinline__ float2 ema_v2(float2 v, float2 g, const Hyper2& h) {
+    return fma2_rn(mul2_rn(h.beta2, v), h.one, mul2_rn(h.omb2, mul2_rn(g, g)));
+}
+// adam_update_fast() on a pair (the two approximate special-function calls stay scalar).
+__device__ __forceinline__ float2 adam_update_fast2(float2 w, float2 mt, float2 vt, const Hyper2& h) {
+    const float2 vh = mul2_rn(vt, h.rbc2);
+    float2 sq, rc;
+    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(sq.x) : "f"(vh.x));
+    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(sq.y) : "f"(vh.y));
+    const float2 den = add2_rn(sq, h.eps);
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rc.x) : "f"(den.x));
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rc.y) : "f"(den.y));
+    return fma2_rn(w, h.decay, mul2_rn(mul2_rn(mt, h.neg_step), rc));
+}
 
 // Eq. 1 moment updates; separate roundings, in the order written there.
 __device__ __forceinline__ float ema_m(float m, float g, const Hyper& h) {

@@ -120,19 +120,32 @@ __device__ __forceinline__ LaneTables make_lane_tables() {
     return t;
 }
 
-// Dequantize (Sec. 2.2), update the moments (Eq. 1) and the parameters for 8 elements.
+// Dequantize (Sec. 2.2), update the moments (Eq. 1) and the parameters for 8 elements, two at a time.
 // m_prod is T_DE[lane & 15] * (old block scale of m); vs[k] the old scale of element k's second moment.
 template <bool EXACT>
 __device__ __forceinline__ void moments_and_update8(float (&w)[8], const float (&g)[8], uint32_t qm, uint32_t qv,
                                                     float m_prod, const float (&vs)[8], const Hyper& h,
-                                                    const LaneTables& lt, float (&mt)[8], float (&vt)[8]) {
+                                                    const Hyper2& h2, const LaneTables& lt, float (&mt)[8],
+                                                    float (&vt)[8]) {
 #pragma unroll
-    for (int k = 0; k < 8; ++k) {
-        const float m = __shfl_sync(lt.mask, m_prod, (int)(qm >> (4 * k)), 16);
-        const float v = __fmul_rn(__shfl_sync(lt.mask, lt.lin, (int)(qv >> (4 * k)), 16), vs[k]);
-        mt[k] = ema_m(m, g[k], h);
-        vt[k] = ema_v(v, g[k], h);
-        w[k] = update_param<EXACT>(w[k], mt[k], vt[k], h);
+    for (int k = 0; k < 8; k += 2) {
+        const float2 m = make_float2(__shfl_sync(lt.mask, m_prod, (int)(qm >> (4 * k)), 16),
+                                     __shfl_sync(lt.mask, m_prod, (int)(qm >> (4 * k + 4)), 16));
+        const float2 tl = make_float2(__shfl_sync(lt.mask, lt.lin, (int)(qv >> (4 * k)), 16),
+                                      __shfl_sync(lt.mask, lt.lin, (int)(qv >> (4 * k + 4)), 16));
+        const float2 v = mul2_rn(tl, make_float2(vs[k], vs[k + 1]));
+        const float2 g2 = make_float2(g[k], g[k + 1]);
+        const float2 m2 = ema_m2(m, g2, h2);
+        const float2 v2 = ema_v2(v, g2, h2);
+        mt[k] = m2.x; mt[k + 1] = m2.y;
+        vt[k] = v2.x; vt[k + 1] = v2.y;
+        if (EXACT) {
+            w[k] = adam_update(w[k], m2.x, v2.x, h);
+            w[k + 1] = adam_update(w[k + 1], m2.y, v2.y, h);
+        } else {
+            const float2 w2 = adam_update_fast2(make_float2(w[k], w[k + 1]), m2, v2, h2);
+            w[k] = w2.x; w[k + 1] = w2.y;
+        }
     }
 }
 
@@ -153,14 +166,28 @@ __device__ __forceinline__ float group_max(float x, unsigned mask) {   // over t
 // Eight nearest codes packed little-nibble-first: acc = acc * 16 + code, from element 7 down to 0.
 __device__ __forceinline__ uint32_t quantize8_de(const float (&x)[8], float rcp, const unsigned char* s_lut) {
     uint32_t q = 0;
+    const float2 r2 = splat(rcp);
 #pragma unroll
-    for (int k = 7; k >= 0; --k) q = q * 16u + de_nearest_lut(__fmul_rn(x[k], rcp), s_lut);
+    for (int k = 6; k >= 0; k -= 2) {
+        const float2 n = mul2_rn(make_float2(x[k], x[k + 1]), r2);
+        q = q * 16u + de_nearest_lut(n.y, s_lut);
+        q = q * 16u + de_nearest_lut(n.x, s_lut);
+    }
     return q;
 }
+// Linear codes as the low mantissa bits of 2^23 + ceil(max(16 n - 1.5, 0)) (see lin_nearest_magic()).
 __device__ __forceinline__ uint32_t quantize8_lin(const float (&x)[8], const float (&rcp)[8]) {
     uint32_t q = 0;
+    const float2 c16 = splat(16.0f), cm = splat(-1.5f), magic = splat(8388608.0f);
 #pragma unroll
-    for (int k = 7; k >= 0; --k) q = q * 16u + lin_nearest_magic(__fmul_rn(x[k], rcp[k]));
+    for (int k = 6; k >= 0; k -= 2) {
+        float2 y = fma2_rn(mul2_rn(make_float2(x[k], x[k + 1]), make_float2(rcp[k], rcp[k + 1])), c16, cm);
+        y.x = fmaxf(y.x, 0.0f);
+        y.y = fmaxf(y.y, 0.0f);
+        const float2 t = add2_ru(y, magic);
+        q = q * 16u + __float_as_uint(t.y);
+        q = q * 16u + __float_as_uint(t.x);
+    }
     return q - kMagicBits * 0x11111111u;   // removes the eight 2^23 patterns (mod 2^32)
 }
 
@@ -199,6 +226,25 @@ struct TileView {
     uint32_t row_stride;   // rows between them
 };
 
+// Asks L2 to fetch this lane's share of row k ahead of time (no register is tied up): the later
+// loads then find their data in L2 instead of waiting for DRAM.
+constexpr uint32_t kL2Ahead = 4;   // rows
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
+template <bool BF16>
+__device__ __forceinline__ void prefetch_row(const TileView& t, uint32_t k) {
+    const uint32_t off = k * t.row_step;
+    prefetch_l2(t.w + off);
+    if (BF16) {
+        prefetch_l2(reinterpret_cast<const uint16_t*>(t.g) + off);
+    } else {
+        prefetch_l2(reinterpret_cast<const float*>(t.g) + off);
+    }
+    prefetch_l2(t.m_codes + (off >> 1));
+    prefetch_l2(t.v_codes + (off >> 1));
+    prefetch_l2(t.m_scale + (off >> 7));
+}
+
 template <bool BF16>
 __device__ __forceinline__ void load_row(RowRegs<BF16>& r, const TileView& t, uint32_t k) {
     const uint32_t off = k * t.row_step;
@@ -220,7 +266,7 @@ __device__ __forceinline__ void load_row(RowRegs<BF16>& r, const TileView& t, ui
 template <bool BF16, bool EXACT>
 __device__ __forceinline__ void process_row(const RowRegs<BF16>& r, const TileView& t, uint32_t k,
                                             const float (&c_old)[8], const float (&c_rcp)[8], const Hyper& h,
-                                            const LaneTables& lt, const unsigned char* s_lut) {
+                                            const Hyper2& h2, const LaneTables& lt, const unsigned char* s_lut) {
     const uint32_t off = k * t.row_step;
     float wv[8] = {r.w0.x, r.w0.y, r.w0.z, r.w0.w, r.w1.x, r.w1.y, r.w1.z, r.w1.w};
     float gv[8], mt[8], vt[8], vs[8], vr[8];
@@ -230,7 +276,7 @@ __device__ __forceinline__ void process_row(const RowRegs<BF16>& r, const TileVi
         vs[j] = fminf(r.r_old, c_old[j]);      // Sec. 4.2: scale = min(r_i, c_j)
         vr[j] = fmaxf(r.r_rcp, c_rcp[j]);      // 1/min(r', c') = max(1/r', 1/c')
     }
-    moments_and_update8<EXACT>(wv, gv, r.qm, r.qv, __fmul_rn(lt.de, r.am), vs, h, lt, mt, vt);
+    moments_and_update8<EXACT>(wv, gv, r.qm, r.qv, __fmul_rn(lt.de, r.am), vs, h, h2, lt, mt, vt);
     store8_f32(t.w + off, wv);
     const float am_new = group_max(absmax8(mt), lt.mask);
     if ((threadIdx.x & 15) == 0) t.m_scale[off >> 7] = am_new;
@@ -240,8 +286,8 @@ __device__ __forceinline__ void process_row(const RowRegs<BF16>& r, const TileVi
 
 template <bool BF16, bool EXACT>
 __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __restrict__ w, const void* __restrict__ g,
-                                                 int tile, int phase, const Hyper& h, const LaneTables& lt,
-                                                 const unsigned char* s_lut) {
+                                                 int tile, int phase, const Hyper& h, const Hyper2& h2,
+                                                 const LaneTables& lt, const unsigned char* s_lut) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int wx = d.wx, wy_count = kWarps / wx;
     const int tx = tile % d.tiles_x, ty = tile / d.tiles_x;
@@ -272,14 +318,18 @@ __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __r
 
     // Two register sets alternate: while one row is processed the next one is already in flight.
     RowRegs<BF16> ra, rb;
+#pragma unroll
+    for (uint32_t k = 1; k < kL2Ahead; ++k) if (k < nrows) prefetch_row<BF16>(t, k);
     load_row<BF16>(ra, t, 0);
     for (uint32_t k = 0; k < nrows; k += 2) {
         const bool has_b = k + 1 < nrows;
+        if (k + kL2Ahead < nrows) prefetch_row<BF16>(t, k + kL2Ahead);
         if (has_b) load_row<BF16>(rb, t, k + 1);
-        process_row<BF16, EXACT>(ra, t, k, c_old, c_rcp, h, lt, s_lut);
+        process_row<BF16, EXACT>(ra, t, k, c_old, c_rcp, h, h2, lt, s_lut);
         if (!has_b) break;
+        if (k + 1 + kL2Ahead < nrows) prefetch_row<BF16>(t, k + 1 + kL2Ahead);
         if (k + 2 < nrows) load_row<BF16>(ra, t, k + 2);
-        process_row<BF16, EXACT>(rb, t, k + 1, c_old, c_rcp, h, lt, s_lut);
+        process_row<BF16, EXACT>(rb, t, k + 1, c_old, c_rcp, h, h2, lt, s_lut);
     }
 }
 
@@ -287,7 +337,7 @@ __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __r
 
 template <bool BF16, bool RANK1, bool EXACT>
 __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restrict__ w, const void* __restrict__ g,
-                                           int tile, int phase, const Hyper& h, const LaneTables& lt,
+                                           int tile, int phase, const Hyper& h, const Hyper2& h2, const LaneTables& lt,
                                            const unsigned char* s_lut) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const float* rc_old = (phase ? d.rc[1] : d.rc[0]);
@@ -332,7 +382,7 @@ __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restric
 #pragma unroll
             for (int k = 0; k < 8; ++k) vs[k] = av;
         }
-        moments_and_update8<EXACT>(wv, gv, qm, qv, __fmul_rn(lt.de, am), vs, h, lt, mt, vt);
+        moments_and_update8<EXACT>(wv, gv, qm, qv, __fmul_rn(lt.de, am), vs, h, h2, lt, mt, vt);
         if (!full) {   // elements beyond the tensor must not reach a block maximum
 #pragma unroll
             for (int k = 0; k < 8; ++k) if (e + k >= d.numel) { mt[k] = 0.0f; vt[k] = 0.0f; }
@@ -398,6 +448,7 @@ __global__ void __launch_bounds__(kThreads, 2) pass2_kernel(StepArgs a) {
     load_lut_smem(s_lut);
     __syncthreads();
     const LaneTables lt = make_lane_tables();
+    const Hyper2 h2 = make_hyper2(a.h);
     for (int tile = blockIdx.x; tile < a.total_tiles; tile += gridDim.x) {
         const int t = find_tensor(a.tile_start, a.n_tensors, tile);
         const TensorDesc d = a.descs[t];   // by value: the fields stay in registers across the stores below
@@ -405,9 +456,9 @@ __global__ void __launch_bounds__(kThreads, 2) pass2_kernel(StepArgs a) {
         const void* g = a.grads[t];
         const int local = tile - __ldg(a.tile_start + t);
         switch (d.kind) {
-            case K_RANK1_FAST: pass2_rank1_fast<BF16, EXACT>(d, w, g, local, a.phase, a.h, lt, s_lut); break;
-            case K_RANK1_FLAT: pass2_flat<BF16, true, EXACT>(d, w, g, local, a.phase, a.h, lt, s_lut); break;
-            case K_BLOCK:      pass2_flat<BF16, false, EXACT>(d, w, g, local, a.phase, a.h, lt, s_lut); break;
+            case K_RANK1_FAST: pass2_rank1_fast<BF16, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut); break;
+            case K_RANK1_FLAT: pass2_flat<BF16, true, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut); break;
+            case K_BLOCK:      pass2_flat<BF16, false, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut); break;
             default:           pass2_fp32<BF16, EXACT>(d, w, g, local, a.h); break;
         }
     }
@@ -472,7 +523,7 @@ __device__ __forceinline__ float warp_max4(const float (&r)[4], int lane) {
 template <bool BF16>
 __device__ __forceinline__ void p1_process_batch(const P1Row<BF16> (&b)[kP1Rows], const P1View& t, uint32_t row,
                                                  uint32_t stride, const float (&c_old)[8], float (&c_max)[8],
-                                                 const Hyper& h, const LaneTables& lt, float* rc_new) {
+                                                 const Hyper2& h2, const LaneTables& lt, float* rc_new) {
     const int lane = threadIdx.x & 31;
     float r_max[kP1Rows];
 #pragma unroll
@@ -481,11 +532,14 @@ __device__ __forceinline__ void p1_process_batch(const P1Row<BF16> (&b)[kP1Rows]
         unpack_grad8<BF16>(b[u].g0, b[u].g1, gv);
         float rm = 0.0f;
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            const float tl = __shfl_sync(0xffffffffu, lt.lin, (int)(b[u].qv >> (4 * k)), 16);
-            const float vt = ema_v(__fmul_rn(tl, fminf(b[u].r_old, c_old[k])), gv[k], h);
-            rm = fmaxf(rm, vt);
-            c_max[k] = fmaxf(c_max[k], vt);
+        for (int k = 0; k < 8; k += 2) {
+            const float2 tl = make_float2(__shfl_sync(0xffffffffu, lt.lin, (int)(b[u].qv >> (4 * k)), 16),
+                                          __shfl_sync(0xffffffffu, lt.lin, (int)(b[u].qv >> (4 * k + 4)), 16));
+            const float2 sc = make_float2(fminf(b[u].r_old, c_old[k]), fminf(b[u].r_old, c_old[k + 1]));
+            const float2 vt = ema_v2(mul2_rn(tl, sc), make_float2(gv[k], gv[k + 1]), h2);
+            rm = fmaxf(rm, fmaxf(vt.x, vt.y));
+            c_max[k] = fmaxf(c_max[k], vt.x);
+            c_max[k + 1] = fmaxf(c_max[k + 1], vt.y);
         }
         r_max[u] = rm;
     }
@@ -496,7 +550,7 @@ __device__ __forceinline__ void p1_process_batch(const P1Row<BF16> (&b)[kP1Rows]
 
 template <bool BF16>
 __device__ __forceinline__ void pass1_rank1_fast(const TensorDesc& d, const void* __restrict__ g, int tile, int phase,
-                                                 const Hyper& h, const LaneTables& lt, float* s_col) {
+                                                 const Hyper2& h2, const LaneTables& lt, float* s_col) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int wx = d.wx, wy_count = kWarps / wx;
     const int tx = tile % d.tiles_x, ty = tile / d.tiles_x;
@@ -525,12 +579,12 @@ __device__ __forceinline__ void pass1_rank1_fast(const TensorDesc& d, const void
     while (true) {
         const bool has_b = i + batch < row_end;
         if (has_b) load_p1_batch<BF16>(bb, t, i + batch, stride);
-        p1_process_batch<BF16>(ba, t, i, stride, c_old, c_max, h, lt, rc_new);
+        p1_process_batch<BF16>(ba, t, i, stride, c_old, c_max, h2, lt, rc_new);
         if (!has_b) break;
         i += batch;
         const bool has_a = i + batch < row_end;
         if (has_a) load_p1_batch<BF16>(ba, t, i + batch, stride);
-        p1_process_batch<BF16>(bb, t, i, stride, c_old, c_max, h, lt, rc_new);
+        p1_process_batch<BF16>(bb, t, i, stride, c_old, c_max, h2, lt, rc_new);
         if (!has_a) break;
         i += batch;
     }
@@ -585,12 +639,13 @@ template <bool BF16>
 __global__ void __launch_bounds__(kThreads, 2) pass1_kernel(StepArgs a) {
     __shared__ float s_col[kWarps * kWarpElems];
     const LaneTables lt = make_lane_tables();
+    const Hyper2 h2 = make_hyper2(a.h);
     for (int tile = blockIdx.x; tile < a.total_tiles; tile += gridDim.x) {
         const int t = find_tensor(a.tile_start, a.n_tensors, tile);
         const TensorDesc d = a.descs[t];
         const void* g = a.grads[t];
         const int local = tile - __ldg(a.tile_start + t);
-        if (d.kind == K_RANK1_FAST) pass1_rank1_fast<BF16>(d, g, local, a.phase, a.h, lt, s_col);
+        if (d.kind == K_RANK1_FAST) pass1_rank1_fast<BF16>(d, g, local, a.phase, h2, lt, s_col);
         else pass1_rank1_flat<BF16>(d, g, local, a.phase, a.h);
     }
 }
