@@ -37,6 +37,7 @@ typedef int32_t lpmm_status;
 #define LPMM_ERR_ALIGNMENT (-3)       /* a device pointer is not 16-byte aligned */
 #define LPMM_ERR_ARENA_TOO_SMALL (-4) /* arena_bytes < lpmm_state_bytes() */
 #define LPMM_ERR_CUDA (-5)            /* a CUDA runtime call or launch failed */
+#define LPMM_ERR_TOO_LARGE (-6)       /* larger than the fixed capacity of lpmm_quantize_rank1_noalloc */
 
 typedef enum { LPMM_F32 = 0, LPMM_BF16 = 1 } lpmm_dtype;
 typedef enum { LPMM_NORM_BLOCK = 0, LPMM_NORM_RANK1 = 1 } lpmm_norm;          /* Sec. 2.2 / Sec. 4.2 */
@@ -138,6 +139,29 @@ lpmm_status lpmm_stage_bytes(const lpmm_state* st, size_t* bytes);
 lpmm_status lpmm_quantize(const float* d_x, int64_t rows, int64_t cols, int32_t norm, int32_t map,
                           int32_t block, uint32_t flags, uint8_t* d_codes, float* d_scale0, float* d_scale1,
                           void* stream);
+
+/* Allocation-free rank-1 quantizer. (No counterpart in the paper: this is a deployment variant of
+ * lpmm_quantize(..., LPMM_NORM_RANK1, LPMM_MAP_LINEAR_NOZERO, ...) and produces the same codes and scales.)
+ *
+ * Who it is for: callers that cannot get device memory at the moment of the call and have nothing to
+ * lend as scratch - a process whose whole GPU memory is already held by a framework's pool, a serving
+ * loop that runs under a fixed memory budget, code that must not call cudaMalloc because that call
+ * synchronizes the device. They pass only the input and the three outputs; the intermediate buffer
+ * (the reciprocals of the row and column maxima) lives in a fixed array inside the library image.
+ *
+ *  - Capacity: round_up(rows, 4) + cols <= LPMM_NOALLOC_MAX_SCALES; beyond that the call launches nothing
+ *    and returns LPMM_ERR_TOO_LARGE. The array costs LPMM_NOALLOC_MAX_SCALES * 4 bytes (1 MiB) of device
+ *    memory on every GPU that loads the library, from load until the process exits.
+ *  - The first call on each device looks up the array's device address (a host-side query, no allocation).
+ *    Make that first call before starting any stream capture on that device.
+ *  - All calls on a device share the one array and it keeps whatever the last call left there. Nothing
+ *    in it needs to start at zero (each call overwrites the part it uses before reading it; the outputs
+ *    d_scale0 / d_scale1 are cleared by the call itself). Two calls that overlap on the GPU - different
+ *    streams, or different host threads - race on it: run them one after the other.
+ *  - It calls neither cudaMalloc nor cudaFree nor any library routine that allocates. */
+#define LPMM_NOALLOC_MAX_SCALES 262144
+lpmm_status lpmm_quantize_rank1_noalloc(const float* d_x, int64_t rows, int64_t cols, uint8_t* d_codes,
+                                        float* d_scale0 /* rows */, float* d_scale1 /* cols */, void* stream);
 
 /* Dequantizer of Sec. 2.2: d_out[i] = T(code_i) * scale_i, scale_i = block maximum or min(r, c). */
 lpmm_status lpmm_dequantize(const uint8_t* d_codes, const float* d_scale0, const float* d_scale1,

@@ -419,6 +419,16 @@ lpmm_status lpmm_quantize(const float* d_x, int64_t rows, int64_t cols, int32_t 
     return LPMM_OK;
 }
 
+lpmm_status lpmm_quantize_rank1_noalloc(const float* d_x, int64_t rows, int64_t cols, uint8_t* d_codes,
+                                        float* d_scale0, float* d_scale1, void* stream) {
+    if (!d_x || !d_codes || !d_scale0 || !d_scale1 || rows <= 0 || cols <= 0) return LPMM_ERR_INVALID_ARG;
+    if (rows > ((int64_t)1 << 40) / cols) return LPMM_ERR_INVALID_ARG;
+    if ((rows + 3) / 4 * 4 + cols > LPMM_NOALLOC_MAX_SCALES) return LPMM_ERR_TOO_LARGE;
+    LPMM_CUDA(launch_quantize_rank1_noalloc(d_x, rows, cols, d_codes, d_scale0, d_scale1,
+                                            static_cast<cudaStream_t>(stream)));
+    return LPMM_OK;
+}
+
 lpmm_status lpmm_dequantize(const uint8_t* d_codes, const float* d_scale0, const float* d_scale1,
                             int64_t rows, int64_t cols, int32_t norm, int32_t map, int32_t block,
                             float* d_out, void* stream) {
@@ -506,6 +516,7 @@ const char* lpmm_status_string(lpmm_status s) {
         case LPMM_ERR_ALIGNMENT: return "pointer not sufficiently aligned";
         case LPMM_ERR_ARENA_TOO_SMALL: return "arena or staging buffer too small";
         case LPMM_ERR_CUDA: return "CUDA runtime error";
+        case LPMM_ERR_TOO_LARGE: return "size exceeds the fixed capacity of the allocation-free entry point";
         default: return "unknown status";
     }
 }

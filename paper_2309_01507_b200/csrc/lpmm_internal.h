@@ -59,4 +59,7 @@ cudaError_t launch_quantize(const float* x, int64_t rows, int64_t cols, int norm
 cudaError_t launch_dequantize(const uint8_t* codes, const float* s0, const float* s1, int64_t rows, int64_t cols,
                               int norm, int map, int block, float* out, cudaStream_t s);
 
+cudaError_t launch_quantize_rank1_noalloc(const float* x, int64_t rows, int64_t cols, uint8_t* codes, float* r,
+                                          float* c, cudaStream_t s);
+
 }  // namespace lpmm

@@ -1,5 +1,8 @@
 // Stand-alone quantizer / dequantizer kernels (Sec. 2.2: Q = M o N, x~ = N^-1 o T(q)) for sm_100a.
 // They serve inspection, checkpoint tooling and the parity tests; the fused step does not call them.
+#include <mutex>
+
+#include "../../include/lpmm.h"
 #include "lpmm_internal.h"
 
 namespace lpmm {
@@ -133,6 +136,85 @@ cudaError_t launch_dequantize(const uint8_t* codes, const float* s0, const float
     if (rank1) unmap_kernel<false, true><<<grid, kQThreads, 0, s>>>(codes, rows, cols, block, s0, s1, out);
     else if (de) unmap_kernel<true, false><<<grid, kQThreads, 0, s>>>(codes, rows, cols, block, s0, s1, out);
     else unmap_kernel<false, false><<<grid, kQThreads, 0, s>>>(codes, rows, cols, block, s0, s1, out);
+    return cudaGetLastError();
+}
+
+// ---- rank-1 quantizer whose scratch lives inside the library image ---------------------------------
+//
+// The reciprocals of the row and column maxima are computed once into a scratch array and the mapping
+// kernel reads them from there (instead of dividing twice per element). The scratch is a fixed
+// file-scope device array, so this path needs no allocation from anybody.
+
+constexpr int64_t kStaticScratchFloats = LPMM_NOALLOC_MAX_SCALES;
+static __device__ __align__(256) float g_static_scratch[kStaticScratchFloats];
+
+namespace {
+
+__global__ void rcp_to_scratch_kernel(const float* __restrict__ r, const float* __restrict__ c, int64_t rows,
+                                      int64_t c_off, int64_t cols, float* __restrict__ scratch) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < rows + cols; i += (int64_t)gridDim.x * blockDim.x) {
+        if (i < rows) scratch[i] = scale_rcp(r[i]);
+        else scratch[c_off + (i - rows)] = scale_rcp(c[i - rows]);
+    }
+}
+
+__global__ void map_rank1_scratch_kernel(const float* __restrict__ x, int64_t rows, int64_t cols, int64_t c_off,
+                                         const float* __restrict__ scratch, uint8_t* __restrict__ codes) {
+    const int64_t numel = rows * cols;
+    const int64_t nbytes = (numel + 1) >> 1;
+    for (int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; b < nbytes; b += (int64_t)gridDim.x * blockDim.x) {
+        uint32_t byte = 0;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int64_t e = 2 * b + h;
+            if (e >= numel) continue;
+            const int64_t i = e / cols, j = e - i * cols;
+            const float rcp = fmaxf(scratch[i], scratch[c_off + j]);
+            byte |= lin_nearest(__fmul_rn(fabsf(__ldg(x + e)), rcp)) << (4 * h);
+        }
+        codes[b] = (uint8_t)byte;
+    }
+}
+
+// Device address of g_static_scratch on the current device, looked up once per device. In host code the
+// array's name is only a handle for the runtime; the kernels must be given this address.
+cudaError_t static_scratch_address(float** out) {
+    constexpr int kMaxDevices = 64;
+    static float* cached[kMaxDevices] = {};
+    static std::mutex mu;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!cached[dev]) {
+        float* p = nullptr;
+        e = cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_static_scratch);
+        if (e != cudaSuccess) return e;
+        cached[dev] = p;
+    }
+    *out = cached[dev];
+    return cudaSuccess;
+}
+
+}  // namespace
+
+cudaError_t launch_quantize_rank1_noalloc(const float* x, int64_t rows, int64_t cols, uint8_t* codes, float* r,
+                                          float* c, cudaStream_t s) {
+    float* scratch = nullptr;
+    cudaError_t e = static_scratch_address(&scratch);
+    if (e != cudaSuccess) return e;
+    const int64_t c_off = (rows + 3) / 4 * 4;
+    // The outputs accumulate maxima and must start at zero; the scratch needs no clearing because the part
+    // used by this call is overwritten below before anything reads it.
+    e = cudaMemsetAsync(r, 0, sizeof(float) * rows, s);
+    if (e != cudaSuccess) return e;
+    e = cudaMemsetAsync(c, 0, sizeof(float) * cols, s);
+    if (e != cudaSuccess) return e;
+    const int64_t tiles = ((cols + kQThreads - 1) / kQThreads) * ((rows + 31) / 32);
+    rank1_scale_kernel<<<(int)(tiles < 148 * 16 ? tiles : 148 * 16), kQThreads, 0, s>>>(x, rows, cols, r, c);
+    rcp_to_scratch_kernel<<<grid_for(rows + cols), kQThreads, 0, s>>>(r, c, rows, c_off, cols, scratch);
+    map_rank1_scratch_kernel<<<grid_for((rows * cols + 1) / 2), kQThreads, 0, s>>>(x, rows, cols, c_off, scratch, codes);
     return cudaGetLastError();
 }
 

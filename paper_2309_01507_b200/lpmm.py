@@ -15,6 +15,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "liblpmm.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_ARENA_TOO_SMALL, ERR_CUDA = 0, -1, -2, -3, -4, -5
+ERR_TOO_LARGE = -6
+NOALLOC_MAX_SCALES = 262144
 F32, BF16 = 0, 1
 NORM_BLOCK, NORM_RANK1 = 0, 1
 MAP_DE_SIGNED, MAP_LINEAR_NOZERO = 0, 1
@@ -26,6 +28,7 @@ KIND_FP32, KIND_BLOCK, KIND_RANK1 = 0, 1, 2
 
 EXPORTS = ("lpmm_state_bytes", "lpmm_state_init", "lpmm_state_attach", "lpmm_adamw4_step",
            "lpmm_adamw4_step_host", "lpmm_stage_bytes", "lpmm_quantize", "lpmm_dequantize",
+           "lpmm_quantize_rank1_noalloc",
            "lpmm_state_view", "lpmm_state_phase", "lpmm_state_last_launches", "lpmm_state_destroy",
            "lpmm_state_profile", "lpmm_state_profile_read",
            "lpmm_status_string", "lpmm_last_cuda_error")
@@ -74,6 +77,7 @@ def lib():
         L.lpmm_stage_bytes.argtypes = [vp, C.POINTER(C.c_size_t)]
         L.lpmm_quantize.argtypes = [vp, i64, i64, i32, i32, i32, u32, vp, vp, vp, vp]
         L.lpmm_dequantize.argtypes = [vp, vp, vp, i64, i64, i32, i32, i32, vp, vp]
+        L.lpmm_quantize_rank1_noalloc.argtypes = [vp, i64, i64, vp, vp, vp, vp]
         L.lpmm_state_view.argtypes = [vp, i32, C.POINTER(i32)] + [C.POINTER(vp)] * 7
         L.lpmm_state_profile.argtypes = [vp, i32]
         L.lpmm_state_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_double),
@@ -260,6 +264,14 @@ def quantize(x: torch.Tensor, norm: int, map_: int, block: int = 128, scales=Non
                                    s0.data_ptr(), None if s1 is None else s1.data_ptr(), _stream_ptr(stream)),
                "lpmm_quantize")
     return codes, s0, s1
+
+
+def quantize_rank1_noalloc(x: torch.Tensor, codes: torch.Tensor, r: torch.Tensor, c: torch.Tensor, stream=None) -> None:
+    """lpmm_quantize_rank1_noalloc: the caller supplies the input and all three outputs; nothing is allocated."""
+    rows, cols = x.shape
+    with torch.cuda.device(x.device):
+        _check(lib().lpmm_quantize_rank1_noalloc(x.data_ptr(), rows, cols, codes.data_ptr(), r.data_ptr(),
+                                                 c.data_ptr(), _stream_ptr(stream)), "lpmm_quantize_rank1_noalloc")
 
 
 def dequantize(codes: torch.Tensor, s0: torch.Tensor, s1, rows: int, cols: int, norm: int, map_: int,
