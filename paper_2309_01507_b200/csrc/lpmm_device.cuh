@@ -66,31 +66,26 @@ __device__ __forceinline__ uint32_t lin_nearest_magic(float n) {
     return __float_as_uint(__fadd_ru(y, 8388608.0f));
 }
 
-// Shared-memory image of the nearest-entry table, directly indexed by the top 12 bits of n (sign, exponent,
-// three mantissa bits): 2048 eight-byte entries for n >= 0 followed by 2048 for n < 0, so that no clamping is
-// needed and every bit pattern (NaN and infinities included) stays inside the table. Entries outside the 80
-// bins of kDeLut repeat the end codes: below 2^-9 the entry 0, from 2.0 upwards the extreme entry.
+// Shared-memory image of the nearest-entry table, directly indexed by the top 12 bits of n: 2048 eight-byte
+// entries for n >= 0 followed by 2048 for n < 0, so that no clamping is needed and every bit pattern (NaN
+// and infinities included) stays inside the table.
 constexpr int kLutSmemBytes = 2 * 2048 * 8;
 
 __device__ __forceinline__ void load_lut_smem(unsigned char* smem) {
-    constexpr uint32_t kFirst = kDeLutKeyBias / 8;            // key of 2^-9
     for (uint32_t i = threadIdx.x; i < 4096u; i += blockDim.x) {
         const uint32_t key = i & 2047u, neg = i >> 11;
         uint2 e;
-        if (key < kFirst) e = make_uint2(0x7f7fffffu, neg ? 8u : 7u);
-        else if (key >= kFirst + kDeLutBins) e = make_uint2(0x7f7fffffu, 15u);
-        else e = kDeLut[neg * kDeLutBins + key - kFirst];
+        if (key < kDeLutFirstKey) e = make_uint2(0x7f7fffffu, 7u);
+        else if (key >= kDeLutFirstKey + kDeLutBins) e = make_uint2(0x7f7fffffu, neg ? 0u : 15u);
+        else e = kDeLut[neg * kDeLutBins + key - kDeLutFirstKey];
         reinterpret_cast<uint2*>(smem)[i] = e;
     }
 }
 
-// Table-driven equivalent of de_nearest(): one lookup, one comparison. Codes of negative values are stored
-// as 15 - code and flipped back by the final xor.
+// Table-driven equivalent of de_nearest(): one lookup, one comparison, one add.
 __device__ __forceinline__ uint32_t de_nearest_lut(float n, const unsigned char* smem) {
-    const uint32_t nb = __float_as_uint(n);
-    const uint2 e = *reinterpret_cast<const uint2*>(smem + ((nb >> 17) & 0x7ff8u));
-    const uint32_t c = e.y + (fabsf(n) > __uint_as_float(e.x) ? 1u : 0u);
-    return c ^ ((uint32_t)((int32_t)nb >> 31) & 15u);
+    const uint2 e = *reinterpret_cast<const uint2*>(smem + ((__float_as_uint(n) >> 17) & 0x7ff8u));
+    return e.y + (n > __uint_as_float(e.x) ? 1u : 0u);
 }
 
 // 1/s (correctly rounded) for a usable scale, 0 for a zero or denormal one (everything under it

@@ -469,38 +469,36 @@ __global__ void __launch_bounds__(kThreads, 2) pass2_kernel(StepArgs a) {
 // Maxima are idempotent, so ragged edges are handled by clamping indices onto valid rows / column
 // groups (a duplicate contributes the same value again) instead of predicating the loads.
 
-constexpr int kP1Rows = 4;   // rows a lane keeps in flight per batch
-
 template <bool BF16>
 struct P1Row {             // one lane's share of one row
     uint4 g0, g1;          // bf16: g0 only
     uint32_t qv;
-    float r_old;
 };
 
 struct P1View {
-    const void* g;             // at the lane's column group, row 0 of the tensor
-    const uint8_t* v_codes;
-    const float* r_old;
-    uint32_t cols;
-    uint32_t last_row;         // last valid row of the tile
+    const void* g;             // at the lane's first element of the tile (row i0, the lane's 8 columns)
+    const uint8_t* v_codes;    // likewise
+    uint32_t row_step;         // elements between two rows this warp handles
 };
 
 template <bool BF16>
-__device__ __forceinline__ void load_p1_batch(P1Row<BF16> (&b)[kP1Rows], const P1View& t, uint32_t row, uint32_t stride) {
-#pragma unroll
-    for (int u = 0; u < kP1Rows; ++u) {
-        const uint32_t rr = min(row + u * stride, t.last_row);
-        const uint64_t e = (uint64_t)rr * t.cols;
-        if (BF16) {
-            b[u].g0 = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(t.g) + e));
-        } else {
-            b[u].g0 = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(t.g) + e));
-            b[u].g1 = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(t.g) + e + 4));
-        }
-        b[u].qv = __ldg(reinterpret_cast<const uint32_t*>(t.v_codes + (e >> 1)));
-        b[u].r_old = __ldg(t.r_old + rr);
+__device__ __forceinline__ void load_p1_row(P1Row<BF16>& b, const P1View& t, uint32_t k) {
+    const uint32_t off = k * t.row_step;
+    if (BF16) {
+        b.g0 = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(t.g) + off));
+    } else {
+        b.g0 = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(t.g) + off));
+        b.g1 = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(t.g) + off + 4));
     }
+    b.qv = __ldg(reinterpret_cast<const uint32_t*>(t.v_codes + (off >> 1)));
+}
+
+template <bool BF16>
+__device__ __forceinline__ void prefetch_p1_row(const P1View& t, uint32_t k) {
+    const uint32_t off = k * t.row_step;
+    if (BF16) prefetch_l2(reinterpret_cast<const uint16_t*>(t.g) + off);
+    else prefetch_l2(reinterpret_cast<const float*>(t.g) + off);
+    prefetch_l2(t.v_codes + (off >> 1));
 }
 
 // Maxima of four per-lane values over the warp with 6 shuffles: afterwards the lanes with
@@ -520,33 +518,27 @@ __device__ __forceinline__ float warp_max4(const float (&r)[4], int lane) {
     return k;
 }
 
+// New second moments of one row; accumulates the column maxima and returns the lane's row maximum.
 template <bool BF16>
-__device__ __forceinline__ void p1_process_batch(const P1Row<BF16> (&b)[kP1Rows], const P1View& t, uint32_t row,
-                                                 uint32_t stride, const float (&c_old)[8], float (&c_max)[8],
-                                                 const Hyper2& h2, const LaneTables& lt, float* rc_new) {
-    const int lane = threadIdx.x & 31;
-    float r_max[kP1Rows];
+__device__ __forceinline__ float p1_process_row(const P1Row<BF16>& b, float r_old, const float (&c_old)[8],
+                                                float (&c_max)[8], const Hyper2& h2, const LaneTables& lt) {
+    float gv[8];
+    unpack_grad8<BF16>(b.g0, b.g1, gv);
+    float rm = 0.0f;
 #pragma unroll
-    for (int u = 0; u < kP1Rows; ++u) {
-        float gv[8];
-        unpack_grad8<BF16>(b[u].g0, b[u].g1, gv);
-        float rm = 0.0f;
-#pragma unroll
-        for (int k = 0; k < 8; k += 2) {
-            const float2 tl = make_float2(__shfl_sync(0xffffffffu, lt.lin, (int)(b[u].qv >> (4 * k)), 16),
-                                          __shfl_sync(0xffffffffu, lt.lin, (int)(b[u].qv >> (4 * k + 4)), 16));
-            const float2 sc = make_float2(fminf(b[u].r_old, c_old[k]), fminf(b[u].r_old, c_old[k + 1]));
-            const float2 vt = ema_v2(mul2_rn(tl, sc), make_float2(gv[k], gv[k + 1]), h2);
-            rm = fmaxf(rm, fmaxf(vt.x, vt.y));
-            c_max[k] = fmaxf(c_max[k], vt.x);
-            c_max[k + 1] = fmaxf(c_max[k + 1], vt.y);
-        }
-        r_max[u] = rm;
+    for (int k = 0; k < 8; k += 2) {
+        const float2 tl = make_float2(__shfl_sync(0xffffffffu, lt.lin, (int)(b.qv >> (4 * k)), 16),
+                                      __shfl_sync(0xffffffffu, lt.lin, (int)(b.qv >> (4 * k + 4)), 16));
+        const float2 sc = make_float2(fminf(r_old, c_old[k]), fminf(r_old, c_old[k + 1]));
+        const float2 vt = ema_v2(mul2_rn(tl, sc), make_float2(gv[k], gv[k + 1]), h2);
+        rm = fmaxf(rm, fmaxf(vt.x, vt.y));
+        c_max[k] = fmaxf(c_max[k], vt.x);
+        c_max[k + 1] = fmaxf(c_max[k + 1], vt.y);
     }
-    const float rm = warp_max4(r_max, lane);
-    const uint32_t which = ((lane >> 4) & 1) * 2 + ((lane >> 3) & 1);
-    if ((lane & 7) == 0) atomic_max_nonneg(rc_new + min(row + which * stride, t.last_row), rm);
+    return rm;
 }
+
+constexpr uint32_t kP1L2Ahead = 8;  // rows the L2 prefetch hints run ahead
 
 template <bool BF16>
 __device__ __forceinline__ void pass1_rank1_fast(const TensorDesc& d, const void* __restrict__ g, int tile, int phase,
@@ -554,57 +546,74 @@ __device__ __forceinline__ void pass1_rank1_fast(const TensorDesc& d, const void
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int wx = d.wx, wy_count = kWarps / wx;
     const int tx = tile % d.tiles_x, ty = tile / d.tiles_x;
-    int64_t col0 = (int64_t)tx * (kWarpElems * wx) + (warp % wx) * kWarpElems + lane * kLaneElems;
-    if (col0 >= d.cols) col0 -= 128;   // only when cols % 256 == 128: the upper half-warp repeats the lower one
+    const int64_t col_w = (int64_t)tx * (kWarpElems * wx) + (warp % wx) * kWarpElems;   // first column of this warp
+    int64_t col0 = col_w + lane * kLaneElems;
+    // Maxima are idempotent: when cols % 256 == 128 the upper half-warp repeats the lower one's columns.
+    if (col0 >= d.cols) col0 -= 128;
     const float* rc_old = (phase ? d.rc[1] : d.rc[0]);
     float* rc_new = (phase ? d.rc[0] : d.rc[1]);
+    const int64_t row0 = (int64_t)ty * d.tile_rows + warp / wx;
+    const int64_t row_end = min((int64_t)(ty + 1) * d.tile_rows, d.rows);
+    if (row0 >= row_end) return;                      // uniform over the warp
+    const uint32_t nrows = (uint32_t)((row_end - row0 + wy_count - 1) / wy_count);
 
     float c_old[8], c_max[8];
 #pragma unroll
     for (int k = 0; k < 8; ++k) c_max[k] = 0.0f;
     load8_f32(rc_old + d.c_off + col0, c_old);
-    const uint32_t row_end = (uint32_t)min((int64_t)(ty + 1) * d.tile_rows, d.rows);
-    const uint32_t stride = (uint32_t)wy_count, batch = kP1Rows * stride;
+    const int64_t e0 = row0 * d.cols + col0;
     P1View t;
-    t.g = BF16 ? static_cast<const void*>(reinterpret_cast<const uint16_t*>(g) + col0)
-               : static_cast<const void*>(reinterpret_cast<const float*>(g) + col0);
-    t.v_codes = d.v_codes + (col0 >> 1);
-    t.r_old = rc_old;
-    t.cols = (uint32_t)d.cols;
-    t.last_row = row_end - 1;
+    t.g = BF16 ? static_cast<const void*>(reinterpret_cast<const uint16_t*>(g) + e0)
+               : static_cast<const void*>(reinterpret_cast<const float*>(g) + e0);
+    t.v_codes = d.v_codes + (e0 >> 1);
+    t.row_step = (uint32_t)(wy_count * d.cols);
 
-    uint32_t i = (uint32_t)((int64_t)ty * d.tile_rows) + warp / wx;   // tile_rows >= warps down, so i < row_end ... or clamped
-    P1Row<BF16> ba[kP1Rows], bb[kP1Rows];
-    load_p1_batch<BF16>(ba, t, i, stride);
-    while (true) {
-        const bool has_b = i + batch < row_end;
-        if (has_b) load_p1_batch<BF16>(bb, t, i + batch, stride);
-        p1_process_batch<BF16>(ba, t, i, stride, c_old, c_max, h2, lt, rc_new);
-        if (!has_b) break;
-        i += batch;
-        const bool has_a = i + batch < row_end;
-        if (has_a) load_p1_batch<BF16>(ba, t, i + batch, stride);
-        p1_process_batch<BF16>(bb, t, i, stride, c_old, c_max, h2, lt, rc_new);
-        if (!has_a) break;
-        i += batch;
-    }
-    // Column maxima: combine the warps that share columns in shared memory, then one atomic per column.
-    float* mine = s_col + warp * kWarpElems + lane * kLaneElems;
 #pragma unroll
-    for (int k = 0; k < 8; ++k) mine[k] = c_max[k];
-    __syncthreads();
-    if (warp < wx) {   // warp `warp` owns column group warp % wx == warp
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            // lane-contiguous layout for the atomics: column = lane + 32 k within the 256-column group
-            const int cc = lane + 32 * k;
-            float mx = 0.0f;
-            for (int y = 0; y < wy_count; ++y) mx = fmaxf(mx, s_col[(y * wx + warp) * kWarpElems + cc]);
-            const int64_t col = (int64_t)tx * (kWarpElems * wx) + warp * kWarpElems + cc;
-            if (col < d.cols) atomic_max_nonneg(rc_new + d.c_off + col, mx);
+    for (uint32_t k = 1; k < kP1L2Ahead; ++k) if (k < nrows) prefetch_p1_row<BF16>(t, k);
+    // Lane j keeps the old row scale of the warp's row number base + j (32 rows per refill); a row's scale is
+    // then read with one shuffle instead of a load.
+    float r_vec = 0.0f;
+    P1Row<BF16> ra, rb;                               // two register sets alternate: the next row is always in flight
+    load_p1_row<BF16>(ra, t, 0);
+    for (uint32_t k = 0; k < nrows; k += 4) {         // four rows per trip so that their maxima reduce together
+        if ((k & 31) == 0) {
+            const uint32_t kk = min(k + lane, nrows - 1);
+            r_vec = __ldg(rc_old + row0 + (int64_t)kk * wy_count);
         }
+#pragma unroll
+        for (uint32_t u = 0; u < 4; ++u)
+            if (k + kP1L2Ahead + u < nrows) prefetch_p1_row<BF16>(t, k + kP1L2Ahead + u);
+        float r_max[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        if (k + 1 < nrows) load_p1_row<BF16>(rb, t, k + 1);
+        r_max[0] = p1_process_row<BF16>(ra, __shfl_sync(0xffffffffu, r_vec, k & 31), c_old, c_max, h2, lt);
+        if (k + 1 < nrows) {
+            if (k + 2 < nrows) load_p1_row<BF16>(ra, t, k + 2);
+            r_max[1] = p1_process_row<BF16>(rb, __shfl_sync(0xffffffffu, r_vec, (k + 1) & 31), c_old, c_max, h2, lt);
+        }
+        if (k + 2 < nrows) {
+            if (k + 3 < nrows) load_p1_row<BF16>(rb, t, k + 3);
+            r_max[2] = p1_process_row<BF16>(ra, __shfl_sync(0xffffffffu, r_vec, (k + 2) & 31), c_old, c_max, h2, lt);
+        }
+        if (k + 3 < nrows) {
+            if (k + 4 < nrows) load_p1_row<BF16>(ra, t, k + 4);
+            r_max[3] = p1_process_row<BF16>(rb, __shfl_sync(0xffffffffu, r_vec, (k + 3) & 31), c_old, c_max, h2, lt);
+        }
+        const float rm = warp_max4(r_max, lane);
+        const uint32_t kr = k + ((lane >> 4) & 1) * 2 + ((lane >> 3) & 1);   // the row whose maximum this lane holds
+        if ((lane & 7) == 0 && kr < nrows) atomic_max_nonneg(rc_new + row0 + (int64_t)kr * wy_count, rm);
     }
-    __syncthreads();
+    // Column maxima: transpose through this warp's slice of shared memory so that consecutive lanes hold
+    // consecutive columns, then one atomic per column. Only the warp itself touches its slice.
+    float* mine = s_col + warp * kWarpElems;
+    __syncwarp();
+#pragma unroll
+    for (int k = 0; k < 8; ++k) mine[lane * kLaneElems + k] = c_max[k];
+    __syncwarp();
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const int cc = lane + 32 * k;
+        if (col_w + cc < d.cols) atomic_max_nonneg(rc_new + d.c_off + col_w + cc, mine[cc]);
+    }
 }
 
 template <bool BF16>
@@ -636,7 +645,7 @@ __device__ __forceinline__ void pass1_rank1_flat(const TensorDesc& d, const void
 }
 
 template <bool BF16>
-__global__ void __launch_bounds__(kThreads, 2) pass1_kernel(StepArgs a) {
+__global__ void __launch_bounds__(kThreads, 3) pass1_kernel(StepArgs a) {
     __shared__ float s_col[kWarps * kWarpElems];
     const LaneTables lt = make_lane_tables();
     const Hyper2 h2 = make_hyper2(a.h);
