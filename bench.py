@@ -276,7 +276,7 @@ def run_ours(args):
         e2e = {"value": world * n_params / (e2e_ms * 1e-3) / 1e9, "unit": UNIT,
                "h2d_bytes_per_step": (4 + gsz) * n_params, "d2h_bytes_per_step": 4 * n_params,
                "ms_per_step": e2e_ms, "steps": args.e2e_steps,
-               "note": "lpmm_adamw4_step_host: pinned host params+grads copied in, updated params copied out, every step"}
+               "note": "lpmm_adamw4_step_host: pinned host params+grads copied in, updated params copied out, every step; copies of neighbouring tensor groups overlap the kernels"}
         del d_pstage, d_gstage, h_p, h_g, hp, hg, e2e_state
 
     if rank != 0:

@@ -115,10 +115,14 @@ lpmm_status lpmm_adamw4_step(lpmm_state* st, void* const* d_params, const void* 
 
 /* The same step for callers whose parameters and gradients live in HOST memory (optimizer
  * offloading): copies every tensor's parameters and gradient into the caller's device staging
- * buffers, runs lpmm_adamw4_step there and copies the updated parameters back, all on `stream`.
+ * buffers, runs the step there and copies the updated parameters back. The tensors are processed in
+ * groups so that copy-in, update and copy-out of neighbouring groups overlap (two internal copy
+ * streams owned by the handle, chained to `stream` by events): `stream` waits for earlier work before
+ * the first copy and is complete only after the last copy-out.
  *   h_params[i], h_grads[i] : host pointers (pinned memory makes the copies asynchronous)
  *   d_param_stage / d_grad_stage : device buffers of at least lpmm_stage_bytes() bytes each
- * Returns after enqueueing; synchronize the stream before reading h_params. */
+ * Returns after enqueueing; synchronize the stream before reading h_params. The number of kernels is
+ * three per group that holds a rank-1 tensor. */
 lpmm_status lpmm_adamw4_step_host(lpmm_state* st, void* const* h_params, const void* const* h_grads,
                                   int32_t grad_dtype, float lr, float beta1, float beta2, float eps,
                                   float weight_decay, int64_t step,
@@ -176,6 +180,11 @@ lpmm_status lpmm_state_view(const lpmm_state* st, int32_t tensor, int32_t* kind,
                             const uint8_t** m_codes, const float** m_scale,
                             const uint8_t** v_codes, const float** v_scale0, const float** v_scale1,
                             const float** m32, const float** v32);
+
+/* Reads the device-side error word of the state (synchronizes `stream`). 0 = no error; 1 = a bounded wait
+ * for an asynchronous shared-memory copy inside a step kernel expired (the affected warp stopped early, so
+ * the states written by that step are incomplete). Kernels never trap or spin without limit. */
+lpmm_status lpmm_state_device_status(lpmm_state* st, int32_t* status, void* stream);
 
 /* 0 or 1: which of the two rank-1 scale buffers is current. Save it with a copy of the arena. */
 int32_t lpmm_state_phase(const lpmm_state* st);

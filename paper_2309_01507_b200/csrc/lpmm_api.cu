@@ -1,6 +1,7 @@
 // Host side of the C ABI declared in include/lpmm.h: argument validation, arena layout, the
 // device-side tensor table and the launch sequence of one step. No device memory is allocated here.
 #include <cmath>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -135,6 +136,11 @@ struct lpmm_state {
     std::vector<void*> params, grads;  // what the device-side pointer arrays currently hold
     size_t stage_bytes;
     std::vector<size_t> stage_off;
+    int32_t pass2_variant;                 // 0 = register prefetch, 1 = bulk-copy staging
+    int32_t sms, occ1, occ2;
+    std::vector<int32_t> tiles1, tiles2;   // host copies of the tile prefix sums
+    cudaStream_t copy_in, copy_out;        // lazily created by the host-buffer entry point
+    std::vector<cudaEvent_t> host_events;
     bool profile;                          // record events around each kernel of a step
     std::vector<cudaEvent_t> prof_events;  // 4 per recorded step: start, after pass 1, after rcp, after pass 2
 };
@@ -153,10 +159,10 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
     const int32_t n = st->n;
     int64_t total_elems = 0;
     for (int32_t i = 0; i < n; ++i) total_elems += st->L.t[i].numel;
-    // aim at >= 4 tiles per resident CTA, tiles between 2 Ki and 32 Ki elements (powers of two)
+    // aim at >= 4 tiles per resident CTA, tiles between 2 Ki and 128 Ki elements (powers of two)
     int64_t target = total_elems / (4LL * sms * occ2);
     int64_t tile_elems = 2048;
-    while (tile_elems * 2 <= target && tile_elems < 32768) tile_elems *= 2;
+    while (tile_elems * 2 <= target && tile_elems < 131072) tile_elems *= 2;
 
     std::vector<TensorDesc> descs(n);
     std::vector<int32_t> t1(n + 1, 0), t2(n + 1, 0);
@@ -205,6 +211,9 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
     st->total2 = t2[n];
     st->grid1 = st->total1 < sms * occ1 ? st->total1 : sms * occ1;
     st->grid2 = st->total2 < sms * occ2 ? st->total2 : sms * occ2;
+    st->sms = sms; st->occ1 = occ1; st->occ2 = occ2;
+    st->tiles1 = t1;
+    st->tiles2 = t2;
     LPMM_CUDA(cudaMemcpyAsync(A + st->L.descs, descs.data(), sizeof(TensorDesc) * n, cudaMemcpyHostToDevice, s));
     LPMM_CUDA(cudaMemcpyAsync(A + st->L.tiles1, t1.data(), sizeof(int32_t) * (n + 1), cudaMemcpyHostToDevice, s));
     LPMM_CUDA(cudaMemcpyAsync(A + st->L.tiles2, t2.data(), sizeof(int32_t) * (n + 1), cudaMemcpyHostToDevice, s));
@@ -232,6 +241,12 @@ lpmm_status make_state(const lpmm_config* cfg, const lpmm_shape* shapes, int32_t
     st->phase = phase;
     st->last_launches = 0;
     st->profile = false;
+    st->copy_in = nullptr;
+    st->copy_out = nullptr;
+    {
+        const char* v = std::getenv("LPMM_PASS2_VARIANT");   // development switch
+        st->pass2_variant = (v && v[0] == '1') ? 1 : 0;
+    }
     st->ptrs_valid = false;
     st->params.assign(n, nullptr);
     st->grads.assign(n, nullptr);
@@ -287,14 +302,22 @@ lpmm_status lpmm_state_attach(const lpmm_config* cfg, const lpmm_shape* shapes, 
     return make_state(cfg, shapes, n, d_arena, arena_bytes, false, phase, out, stream);
 }
 
-lpmm_status lpmm_adamw4_step(lpmm_state* st, void* const* d_params, const void* const* d_grads,
-                             int32_t grad_dtype, float lr, float beta1, float beta2, float eps,
-                             float weight_decay, int64_t step, void* stream) {
-    if (!st || !d_params || !d_grads) return LPMM_ERR_INVALID_ARG;
+}  // extern "C" (reopened below)
+
+namespace {
+
+lpmm_status check_step_args(const lpmm_state* st, const void* p, const void* g, int32_t grad_dtype, float lr, float beta1,
+                            float beta2, float eps, float weight_decay, int64_t step) {
+    if (!st || !p || !g) return LPMM_ERR_INVALID_ARG;
     if (grad_dtype != LPMM_F32 && grad_dtype != LPMM_BF16) return LPMM_ERR_INVALID_ARG;
     if (step < 1) return LPMM_ERR_INVALID_ARG;
     if (!finite_nonneg(lr) || !finite_nonneg(eps) || !finite_nonneg(weight_decay)) return LPMM_ERR_INVALID_ARG;
     if (!finite_nonneg(beta1) || !finite_nonneg(beta2) || beta1 >= 1.0f || beta2 >= 1.0f) return LPMM_ERR_INVALID_ARG;
+    return LPMM_OK;
+}
+
+// Makes the device-side pointer arrays hold these parameter / gradient pointers (uploads only on change).
+lpmm_status set_pointers(lpmm_state* st, void* const* d_params, const void* const* d_grads, cudaStream_t s) {
     const int32_t n = st->n;
     bool changed = !st->ptrs_valid;
     for (int32_t i = 0; i < n; ++i) {
@@ -302,8 +325,6 @@ lpmm_status lpmm_adamw4_step(lpmm_state* st, void* const* d_params, const void* 
         if (!aligned16(d_params[i]) || !aligned16(d_grads[i])) return LPMM_ERR_ALIGNMENT;
         if (d_params[i] != st->params[i] || d_grads[i] != st->grads[i]) changed = true;
     }
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    int32_t launches = 0;
     if (changed) {
         for (int32_t i = 0; i < n; ++i) { st->params[i] = d_params[i]; st->grads[i] = const_cast<void*>(d_grads[i]); }
         st->ptrs_valid = false;
@@ -311,27 +332,84 @@ lpmm_status lpmm_adamw4_step(lpmm_state* st, void* const* d_params, const void* 
         LPMM_CUDA(cudaMemcpyAsync(st->arena + st->L.grads, st->grads.data(), sizeof(void*) * n, cudaMemcpyHostToDevice, s));
         st->ptrs_valid = true;
     }
+    return LPMM_OK;
+}
 
+StepArgs make_args(const lpmm_state* st, float lr, float beta1, float beta2, float eps, float weight_decay, int64_t step) {
     StepArgs a;
     a.descs = reinterpret_cast<const TensorDesc*>(st->arena + st->L.descs);
     a.params = reinterpret_cast<float* const*>(st->arena + st->L.params);
     a.grads = reinterpret_cast<const void* const*>(st->arena + st->L.grads);
-    a.n_tensors = n;
+    a.n_tensors = st->n;
     a.phase = st->phase;
+    a.variant = st->pass2_variant;
+    a.dev_status = reinterpret_cast<uint32_t*>(st->arena);
     a.h.lr = lr; a.h.beta1 = beta1; a.h.beta2 = beta2; a.h.eps = eps;
     a.h.omb1 = 1.0f - beta1;
     a.h.omb2 = 1.0f - beta2;
-    a.h.bc1 = (float)(1.0 - std::pow((double)beta1, (double)step));   // Eq. 1: 1 - beta^t
-    a.h.bc2 = (float)(1.0 - std::pow((double)beta2, (double)step));
+    const double bc1 = 1.0 - std::pow((double)beta1, (double)step);   // Eq. 1: 1 - beta^t
+    const double bc2 = 1.0 - std::pow((double)beta2, (double)step);
+    a.h.bc1 = (float)bc1;
+    a.h.bc2 = (float)bc2;
     a.h.decay = 1.0f - lr * weight_decay;
     a.h.one = 1.0f;
-    {
-        const double bc1 = 1.0 - std::pow((double)beta1, (double)step), bc2 = 1.0 - std::pow((double)beta2, (double)step);
-        a.h.step_size = (float)((double)lr / bc1);
-        a.h.rbc2 = (float)(1.0 / bc2);
-    }
-    const bool bf16 = (grad_dtype == LPMM_BF16);
+    a.h.step_size = (float)((double)lr / bc1);
+    a.h.rbc2 = (float)(1.0 / bc2);
+    return a;
+}
 
+// Enqueues the three kernels of one step for tensors [t0, t1). ev (4 events or nullptr) brackets the kernels.
+lpmm_status enqueue_range(lpmm_state* st, StepArgs a, int32_t t0, int32_t t1, bool bf16, bool ieee_update,
+                          cudaStream_t s, cudaEvent_t* ev, int32_t* launches) {
+    const int32_t p1_begin = st->tiles1[t0], p1_end = st->tiles1[t1];
+    if (p1_end > p1_begin) {
+        // the rank-1 scale region of these tensors is one contiguous range of the scale buffers
+        int64_t rc_begin = -1, rc_end = 0;
+        for (int32_t i = t0; i < t1; ++i) {
+            const TensorLayout& t = st->L.t[i];
+            if (t.kind != K_RANK1_FAST && t.kind != K_RANK1_FLAT) continue;
+            if (rc_begin < 0) rc_begin = t.rc_index;
+            rc_end = (t.rc_index + t.c_off + (t.cols + 3) / 4 * 4 + 63) / 64 * 64;
+        }
+        float* rc_new = reinterpret_cast<float*>(st->arena + st->L.rc[st->phase ^ 1]) + rc_begin;
+        LPMM_CUDA(cudaMemsetAsync(rc_new, 0, sizeof(float) * (size_t)(rc_end - rc_begin), s));
+        if (ev) LPMM_CUDA(cudaEventRecord(ev[0], s));
+        a.tile_start = reinterpret_cast<const int32_t*>(st->arena + st->L.tiles1);
+        a.tile_begin = p1_begin;
+        a.tile_end = p1_end;
+        const int32_t cap = st->sms * st->occ1, tiles = p1_end - p1_begin;
+        LPMM_CUDA(launch_pass1(a, bf16, tiles < cap ? tiles : cap, s));
+        if (ev) LPMM_CUDA(cudaEventRecord(ev[1], s));
+        LPMM_CUDA(launch_rcp(rc_new, reinterpret_cast<float*>(st->arena + st->L.rcp) + rc_begin, rc_end - rc_begin, s));
+        *launches += 2;
+    } else if (ev) {
+        LPMM_CUDA(cudaEventRecord(ev[0], s));
+        LPMM_CUDA(cudaEventRecord(ev[1], s));
+    }
+    if (ev) LPMM_CUDA(cudaEventRecord(ev[2], s));
+    a.tile_start = reinterpret_cast<const int32_t*>(st->arena + st->L.tiles2);
+    a.tile_begin = st->tiles2[t0];
+    a.tile_end = st->tiles2[t1];
+    const int32_t cap = st->sms * st->occ2, tiles = a.tile_end - a.tile_begin;
+    LPMM_CUDA(launch_pass2(a, bf16, ieee_update, tiles < cap ? tiles : cap, s));
+    if (ev) LPMM_CUDA(cudaEventRecord(ev[3], s));
+    *launches += 1;
+    return LPMM_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+lpmm_status lpmm_adamw4_step(lpmm_state* st, void* const* d_params, const void* const* d_grads,
+                             int32_t grad_dtype, float lr, float beta1, float beta2, float eps,
+                             float weight_decay, int64_t step, void* stream) {
+    lpmm_status rc = check_step_args(st, d_params, d_grads, grad_dtype, lr, beta1, beta2, eps, weight_decay, step);
+    if (rc != LPMM_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    rc = set_pointers(st, d_params, d_grads, s);
+    if (rc != LPMM_OK) return rc;
+    const StepArgs a = make_args(st, lr, beta1, beta2, eps, weight_decay, step);
     cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
     if (st->profile) {
         for (int k = 0; k < 4; ++k) {
@@ -339,28 +417,11 @@ lpmm_status lpmm_adamw4_step(lpmm_state* st, void* const* d_params, const void* 
             st->prof_events.push_back(ev[k]);
         }
     }
-    if (st->total1 > 0) {
-        float* rc_new = reinterpret_cast<float*>(st->arena + st->L.rc[st->phase ^ 1]);
-        LPMM_CUDA(cudaMemsetAsync(rc_new, 0, sizeof(float) * st->L.rc_floats, s));
-        if (ev[0]) LPMM_CUDA(cudaEventRecord(ev[0], s));
-        a.tile_start = reinterpret_cast<const int32_t*>(st->arena + st->L.tiles1);
-        a.total_tiles = st->total1;
-        LPMM_CUDA(launch_pass1(a, bf16, st->grid1, s));
-        if (ev[1]) LPMM_CUDA(cudaEventRecord(ev[1], s));
-        LPMM_CUDA(launch_rcp(rc_new, reinterpret_cast<float*>(st->arena + st->L.rcp), st->L.rc_floats, s));
-        launches += 2;
-    } else if (ev[0]) {
-        LPMM_CUDA(cudaEventRecord(ev[0], s));
-        LPMM_CUDA(cudaEventRecord(ev[1], s));
-    }
-    if (ev[2]) LPMM_CUDA(cudaEventRecord(ev[2], s));
-    a.tile_start = reinterpret_cast<const int32_t*>(st->arena + st->L.tiles2);
-    a.total_tiles = st->total2;
     // the approximate update flushes a denormal v^ before the square root: only safe with a real eps
     const bool ieee_update = (st->cfg.update_math == LPMM_UPDATE_IEEE) || eps < 1e-30f;
-    LPMM_CUDA(launch_pass2(a, bf16, ieee_update, st->grid2, s));
-    if (ev[3]) LPMM_CUDA(cudaEventRecord(ev[3], s));
-    launches += 1;
+    int32_t launches = 0;
+    rc = enqueue_range(st, a, 0, st->n, grad_dtype == LPMM_BF16, ieee_update, s, st->profile ? ev : nullptr, &launches);
+    if (rc != LPMM_OK) return rc;
     st->phase ^= 1;
     st->last_launches = launches;
     return LPMM_OK;
@@ -376,27 +437,75 @@ lpmm_status lpmm_adamw4_step_host(lpmm_state* st, void* const* h_params, const v
                                   int32_t grad_dtype, float lr, float beta1, float beta2, float eps,
                                   float weight_decay, int64_t step,
                                   void* d_param_stage, void* d_grad_stage, size_t stage_bytes, void* stream) {
-    if (!st || !h_params || !h_grads || !d_param_stage || !d_grad_stage) return LPMM_ERR_INVALID_ARG;
-    if (grad_dtype != LPMM_F32 && grad_dtype != LPMM_BF16) return LPMM_ERR_INVALID_ARG;
+    lpmm_status rc = check_step_args(st, h_params, h_grads, grad_dtype, lr, beta1, beta2, eps, weight_decay, step);
+    if (rc != LPMM_OK) return rc;
+    if (!d_param_stage || !d_grad_stage) return LPMM_ERR_INVALID_ARG;
     if (stage_bytes < st->stage_bytes) return LPMM_ERR_ARENA_TOO_SMALL;
     if (!aligned16(d_param_stage) || !aligned16(d_grad_stage)) return LPMM_ERR_ALIGNMENT;
     const int32_t n = st->n;
     for (int32_t i = 0; i < n; ++i) if (!h_params[i] || !h_grads[i]) return LPMM_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (!st->copy_in) LPMM_CUDA(cudaStreamCreateWithFlags(&st->copy_in, cudaStreamNonBlocking));
+    if (!st->copy_out) LPMM_CUDA(cudaStreamCreateWithFlags(&st->copy_out, cudaStreamNonBlocking));
+
+    // Tensors are cut into consecutive groups of roughly equal size. Group k+1 is copied in and group k-1 is
+    // copied out (the link is full duplex) while group k is updated: three streams chained by events.
+    std::vector<int32_t> cut(1, 0);
+    {
+        int64_t total = 0;
+        for (int32_t i = 0; i < n; ++i) total += st->L.t[i].numel;
+        const int64_t per_group = total / 16 + 1;
+        int64_t acc = 0;
+        for (int32_t i = 0; i < n; ++i) {
+            acc += st->L.t[i].numel;
+            if (acc >= per_group || i == n - 1) { cut.push_back(i + 1); acc = 0; }
+        }
+    }
+    const size_t groups = cut.size() - 1;
+    const size_t need_events = 2 * groups + 2;
+    while (st->host_events.size() < need_events) {
+        cudaEvent_t e;
+        LPMM_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+        st->host_events.push_back(e);
+    }
+    cudaEvent_t ev_start = st->host_events[2 * groups], ev_end = st->host_events[2 * groups + 1];
+
     const size_t gsz = (grad_dtype == LPMM_BF16) ? 2 : 4;
     std::vector<void*> dp(n);
     std::vector<const void*> dg(n);
     for (int32_t i = 0; i < n; ++i) {
-        const size_t numel = (size_t)st->L.t[i].numel;
         dp[i] = static_cast<char*>(d_param_stage) + st->stage_off[i];
         dg[i] = static_cast<char*>(d_grad_stage) + st->stage_off[i];
-        LPMM_CUDA(cudaMemcpyAsync(dp[i], h_params[i], 4 * numel, cudaMemcpyHostToDevice, s));
-        LPMM_CUDA(cudaMemcpyAsync(const_cast<void*>(dg[i]), h_grads[i], gsz * numel, cudaMemcpyHostToDevice, s));
     }
-    lpmm_status rc = lpmm_adamw4_step(st, dp.data(), dg.data(), grad_dtype, lr, beta1, beta2, eps, weight_decay, step, stream);
+    rc = set_pointers(st, dp.data(), dg.data(), s);
     if (rc != LPMM_OK) return rc;
-    for (int32_t i = 0; i < n; ++i)
-        LPMM_CUDA(cudaMemcpyAsync(h_params[i], dp[i], 4 * (size_t)st->L.t[i].numel, cudaMemcpyDeviceToHost, s));
+    const StepArgs a = make_args(st, lr, beta1, beta2, eps, weight_decay, step);
+    const bool ieee_update = (st->cfg.update_math == LPMM_UPDATE_IEEE) || eps < 1e-30f;
+
+    LPMM_CUDA(cudaEventRecord(ev_start, s));                       // earlier work on the caller's stream comes first
+    LPMM_CUDA(cudaStreamWaitEvent(st->copy_in, ev_start, 0));
+    LPMM_CUDA(cudaStreamWaitEvent(st->copy_out, ev_start, 0));
+    int32_t launches = 0;
+    for (size_t k = 0; k < groups; ++k) {
+        cudaEvent_t ev_in = st->host_events[2 * k], ev_done = st->host_events[2 * k + 1];
+        for (int32_t i = cut[k]; i < cut[k + 1]; ++i) {
+            const size_t numel = (size_t)st->L.t[i].numel;
+            LPMM_CUDA(cudaMemcpyAsync(dp[i], h_params[i], 4 * numel, cudaMemcpyHostToDevice, st->copy_in));
+            LPMM_CUDA(cudaMemcpyAsync(const_cast<void*>(dg[i]), h_grads[i], gsz * numel, cudaMemcpyHostToDevice, st->copy_in));
+        }
+        LPMM_CUDA(cudaEventRecord(ev_in, st->copy_in));
+        LPMM_CUDA(cudaStreamWaitEvent(s, ev_in, 0));
+        rc = enqueue_range(st, a, cut[k], cut[k + 1], grad_dtype == LPMM_BF16, ieee_update, s, nullptr, &launches);
+        if (rc != LPMM_OK) return rc;
+        LPMM_CUDA(cudaEventRecord(ev_done, s));
+        LPMM_CUDA(cudaStreamWaitEvent(st->copy_out, ev_done, 0));
+        for (int32_t i = cut[k]; i < cut[k + 1]; ++i)
+            LPMM_CUDA(cudaMemcpyAsync(h_params[i], dp[i], 4 * (size_t)st->L.t[i].numel, cudaMemcpyDeviceToHost, st->copy_out));
+    }
+    LPMM_CUDA(cudaEventRecord(ev_end, st->copy_out));
+    LPMM_CUDA(cudaStreamWaitEvent(s, ev_end, 0));                  // the caller's stream ends after the last copy-out
+    st->phase ^= 1;
+    st->last_launches = launches;
     return LPMM_OK;
 }
 
@@ -498,6 +607,16 @@ lpmm_status lpmm_state_profile_read(lpmm_state* st, double* pass1_ms, double* rc
     return rc;
 }
 
+lpmm_status lpmm_state_device_status(lpmm_state* st, int32_t* status, void* stream) {
+    if (!st || !status) return LPMM_ERR_INVALID_ARG;
+    uint32_t word = 0;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    LPMM_CUDA(cudaMemcpyAsync(&word, st->arena, sizeof(word), cudaMemcpyDeviceToHost, s));
+    LPMM_CUDA(cudaStreamSynchronize(s));
+    *status = (int32_t)word;
+    return LPMM_OK;
+}
+
 int32_t lpmm_state_phase(const lpmm_state* st) { return st ? st->phase : -1; }
 
 int32_t lpmm_state_last_launches(const lpmm_state* st) { return st ? st->last_launches : 0; }
@@ -505,6 +624,9 @@ int32_t lpmm_state_last_launches(const lpmm_state* st) { return st ? st->last_la
 void lpmm_state_destroy(lpmm_state* st) {
     if (!st) return;
     for (cudaEvent_t e : st->prof_events) cudaEventDestroy(e);
+    for (cudaEvent_t e : st->host_events) cudaEventDestroy(e);
+    if (st->copy_in) cudaStreamDestroy(st->copy_in);
+    if (st->copy_out) cudaStreamDestroy(st->copy_out);
     delete st;
 }
 

@@ -44,8 +44,10 @@ struct StepArgs {
     const void* const* grads;    // n device pointers
     const int32_t* tile_start;   // n + 1 prefix sums of tiles (pass-specific)
     int32_t n_tensors;
-    int32_t total_tiles;
+    int32_t tile_begin, tile_end;  // this launch covers tiles [tile_begin, tile_end) of the prefix table
     int32_t phase;               // rc[phase] holds the current r, c; rc[1 - phase] receives the new ones
+    int32_t variant;             // pass 2: 0 = rows prefetched into registers, 1 = rows staged by bulk copies
+    uint32_t* dev_status;        // device error word in the arena header (0 = ok)
     Hyper h;
 };
 

@@ -333,6 +333,179 @@ __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __r
     }
 }
 
+// ---- pass 2, rank-1 tensors, rows staged by bulk asynchronous copies ---------------------------------
+//
+// Each warp owns a small ring in shared memory. One lane asks the copy engine (cp.async.bulk, completion
+// counted on an mbarrier) for the warp's 256-element segment of the next rows: parameters, gradient and
+// both code words. The data of several rows is then in flight without holding registers or issue slots,
+// and the lanes read their 8 elements back with plain shared-memory loads. Nothing is shared between
+// warps, so there is no block-wide barrier; a warp reuses a slot right after its own lanes have read it.
+// Every wait is bounded: if a copy never completes, the warp records an error word and stops.
+
+constexpr int kBulkStages = 4;
+constexpr uint32_t kSpinLimit = 1u << 18;   // polls of a (self-suspending) try_wait before giving up
+constexpr uint32_t kStatusCopyTimeout = 1u;
+
+template <bool BF16>
+struct WarpStage {                                   // byte offsets inside one stage of one warp
+    static constexpr int kW = 0;                                    // 256 floats
+    static constexpr int kG = 1024;                                 // 256 bf16 / 256 floats
+    static constexpr int kQm = kG + (BF16 ? 512 : 1024);            // 128 bytes of codes
+    static constexpr int kQv = kQm + 128;
+    static constexpr int kBytes = kQv + 128;
+};
+template <bool BF16>
+constexpr int bulk_smem_bytes() {
+    return kLutSmemBytes + kWarps * kBulkStages * WarpStage<BF16>::kBytes + kWarps * kBulkStages * 8;
+}
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+// Bounded wait for the given phase parity of an mbarrier; false if it never completed.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+        uint32_t done;
+        asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+                     : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+
+struct WarpRing {
+    unsigned char* data;     // kBulkStages stages of this warp
+    uint32_t bars;           // shared address of this warp's kBulkStages mbarriers
+    uint32_t slot;           // stage that receives / delivers the next row
+    uint32_t phases;         // bit s = parity to wait for on stage s
+    bool dead;               // a wait timed out: this warp does no further work
+};
+
+// Warp-uniform description of the warp's rows in one tile (addresses at the warp's first column).
+struct BulkView {
+    const float* w;
+    const void* g;
+    const uint8_t* m_codes;
+    const uint8_t* v_codes;
+    uint32_t row_step;
+};
+
+template <bool BF16>
+__device__ __forceinline__ void bulk_issue_row(const WarpRing& r, uint32_t slot, const BulkView& t, uint32_t k) {
+    // called by one lane
+    const uint32_t off = k * t.row_step;
+    const uint32_t bar = r.bars + slot * 8;
+    const uint32_t dst = smem_u32(r.data + slot * WarpStage<BF16>::kBytes);
+    mbar_expect_tx(bar, WarpStage<BF16>::kBytes);
+    bulk_load(dst + WarpStage<BF16>::kW, t.w + off, 1024, bar);
+    if (BF16) bulk_load(dst + WarpStage<BF16>::kG, reinterpret_cast<const uint16_t*>(t.g) + off, 512, bar);
+    else bulk_load(dst + WarpStage<BF16>::kG, reinterpret_cast<const float*>(t.g) + off, 1024, bar);
+    bulk_load(dst + WarpStage<BF16>::kQm, t.m_codes + (off >> 1), 128, bar);
+    bulk_load(dst + WarpStage<BF16>::kQv, t.v_codes + (off >> 1), 128, bar);
+}
+
+template <bool BF16, bool EXACT>
+__device__ __forceinline__ void pass2_rank1_bulk(const TensorDesc& d, float* __restrict__ w, const void* __restrict__ g,
+                                                 int tile, int phase, const Hyper& h, const Hyper2& h2,
+                                                 const LaneTables& lt, const unsigned char* s_lut, WarpRing& ring,
+                                                 uint32_t* dev_status) {
+    if (ring.dead) return;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int wx = d.wx, wy_count = kWarps / wx;
+    const int tx = tile % d.tiles_x, ty = tile / d.tiles_x;
+    const int64_t col_w = (int64_t)tx * (kWarpElems * wx) + (warp % wx) * kWarpElems;   // cols % 256 == 0 here
+    const int64_t col0 = col_w + lane * kLaneElems;
+    const float* rc_old = (phase ? d.rc[1] : d.rc[0]);
+    const float* rcp_new = d.rcp_new;
+    const int64_t row0 = (int64_t)ty * d.tile_rows + warp / wx;
+    const int64_t row_end = min((int64_t)(ty + 1) * d.tile_rows, d.rows);
+    if (row0 >= row_end) return;                       // uniform over the warp
+    const uint32_t nrows = (uint32_t)((row_end - row0 + wy_count - 1) / wy_count);
+    const int64_t e_w = row0 * d.cols + col_w;         // warp's first element
+    BulkView t;
+    t.w = w + e_w;
+    t.g = BF16 ? static_cast<const void*>(reinterpret_cast<const uint16_t*>(g) + e_w)
+               : static_cast<const void*>(reinterpret_cast<const float*>(g) + e_w);
+    t.m_codes = d.m_codes + (e_w >> 1);
+    t.v_codes = d.v_codes + (e_w >> 1);
+    t.row_step = (uint32_t)(wy_count * d.cols);
+
+    if (lane == 0) {                                   // fill the ring
+        for (uint32_t k = 0; k < (uint32_t)kBulkStages && k < nrows; ++k)
+            bulk_issue_row<BF16>(ring, (ring.slot + k) % kBulkStages, t, k);
+    }
+    float c_old[8], c_rcp[8];
+    load8_f32(rc_old + d.c_off + col0, c_old);
+    load8_f32(rcp_new + d.c_off + col0, c_rcp);
+    // Per-row scalars: lane j (mod 16) keeps the values of the warp's row number base + j, 16 rows per refill;
+    // lanes 0-15 hold the first block's old scale of m, lanes 16-31 the second block's.
+    float* w_lane = w + e_w + lane * kLaneElems;
+    uint8_t* mq_lane = d.m_codes + ((e_w + lane * kLaneElems) >> 1);
+    uint8_t* vq_lane = d.v_codes + ((e_w + lane * kLaneElems) >> 1);
+    float* ms_warp = d.m_scale + (e_w >> 7);
+    float am_vec = 0.0f, ro_vec = 0.0f, rr_vec = 0.0f;
+    for (uint32_t k = 0; k < nrows; ++k) {
+        if ((k & 15) == 0) {
+            const uint32_t kk = min(k + (lane & 15), nrows - 1);
+            am_vec = ms_warp[(size_t)((kk * t.row_step) >> 7) + (lane >> 4)];
+            ro_vec = __ldg(rc_old + row0 + (int64_t)kk * wy_count);
+            rr_vec = __ldg(rcp_new + row0 + (int64_t)kk * wy_count);
+        }
+        const uint32_t slot = ring.slot;
+        if (!mbar_wait(ring.bars + slot * 8, (ring.phases >> slot) & 1u)) {
+            if (lane == 0) atomicExch(dev_status, kStatusCopyTimeout);
+            ring.dead = true;
+            return;
+        }
+        ring.phases ^= 1u << slot;
+        const unsigned char* st = ring.data + slot * WarpStage<BF16>::kBytes;
+        const float4 w0 = *reinterpret_cast<const float4*>(st + WarpStage<BF16>::kW + lane * 32);
+        const float4 w1 = *reinterpret_cast<const float4*>(st + WarpStage<BF16>::kW + lane * 32 + 16);
+        uint4 g0, g1 = make_uint4(0, 0, 0, 0);
+        if (BF16) {
+            g0 = *reinterpret_cast<const uint4*>(st + WarpStage<BF16>::kG + lane * 16);
+        } else {
+            g0 = *reinterpret_cast<const uint4*>(st + WarpStage<BF16>::kG + lane * 32);
+            g1 = *reinterpret_cast<const uint4*>(st + WarpStage<BF16>::kG + lane * 32 + 16);
+        }
+        const uint32_t qm = *reinterpret_cast<const uint32_t*>(st + WarpStage<BF16>::kQm + lane * 4);
+        const uint32_t qv = *reinterpret_cast<const uint32_t*>(st + WarpStage<BF16>::kQv + lane * 4);
+        __syncwarp();                                  // every lane has read the slot
+        if (lane == 0 && k + kBulkStages < nrows) {
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            bulk_issue_row<BF16>(ring, slot, t, k + kBulkStages);
+        }
+        ring.slot = (slot + 1 == (uint32_t)kBulkStages) ? 0u : slot + 1;
+
+        const float am = __shfl_sync(0xffffffffu, am_vec, (lane & 16) | (k & 15));
+        const float r_old = __shfl_sync(0xffffffffu, ro_vec, k & 15);
+        const float r_rcp = __shfl_sync(0xffffffffu, rr_vec, k & 15);
+        float wv[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+        float gv[8], mt[8], vt[8], vs[8], vr[8];
+        unpack_grad8<BF16>(g0, g1, gv);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            vs[j] = fminf(r_old, c_old[j]);
+            vr[j] = fmaxf(r_rcp, c_rcp[j]);
+        }
+        moments_and_update8<EXACT>(wv, gv, qm, qv, __fmul_rn(lt.de, am), vs, h, h2, lt, mt, vt);
+        const uint32_t off = k * t.row_step;
+        store8_f32(w_lane + off, wv);
+        const float am_new = group_max(absmax8(mt), lt.mask);
+        if ((lane & 15) == 0) ms_warp[(size_t)(off >> 7) + (lane >> 4)] = am_new;
+        *reinterpret_cast<uint32_t*>(mq_lane + (off >> 1)) = quantize8_de(mt, scale_rcp(am_new), s_lut);
+        *reinterpret_cast<uint32_t*>(vq_lane + (off >> 1)) = quantize8_lin(vt, vr);
+    }
+}
+
 // ---- pass 2, flat (element-indexed) tensors: block-wise v, or rank-1 with arbitrary cols ------
 
 template <bool BF16, bool RANK1, bool EXACT>
@@ -449,7 +622,7 @@ __global__ void __launch_bounds__(kThreads, 2) pass2_kernel(StepArgs a) {
     __syncthreads();
     const LaneTables lt = make_lane_tables();
     const Hyper2 h2 = make_hyper2(a.h);
-    for (int tile = blockIdx.x; tile < a.total_tiles; tile += gridDim.x) {
+    for (int tile = a.tile_begin + blockIdx.x; tile < a.tile_end; tile += gridDim.x) {
         const int t = find_tensor(a.tile_start, a.n_tensors, tile);
         const TensorDesc d = a.descs[t];   // by value: the fields stay in registers across the stores below
         float* w = a.params[t];
@@ -457,6 +630,43 @@ __global__ void __launch_bounds__(kThreads, 2) pass2_kernel(StepArgs a) {
         const int local = tile - __ldg(a.tile_start + t);
         switch (d.kind) {
             case K_RANK1_FAST: pass2_rank1_fast<BF16, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut); break;
+            case K_RANK1_FLAT: pass2_flat<BF16, true, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut); break;
+            case K_BLOCK:      pass2_flat<BF16, false, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut); break;
+            default:           pass2_fp32<BF16, EXACT>(d, w, g, local, a.h); break;
+        }
+    }
+}
+
+template <bool BF16, bool EXACT>
+__global__ void __launch_bounds__(kThreads, 2) pass2_bulk_kernel(StepArgs a) {
+    extern __shared__ __align__(128) unsigned char s_dyn[];   // [nearest-entry table | warp rings | mbarriers]
+    unsigned char* s_lut = s_dyn;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    WarpRing ring;
+    ring.data = s_dyn + kLutSmemBytes + warp * kBulkStages * WarpStage<BF16>::kBytes;
+    ring.bars = smem_u32(s_dyn + kLutSmemBytes + kWarps * kBulkStages * WarpStage<BF16>::kBytes) + warp * kBulkStages * 8;
+    ring.slot = 0;
+    ring.phases = 0;
+    ring.dead = false;
+    if (lane == 0) {
+        for (int s = 0; s < kBulkStages; ++s) mbar_init(ring.bars + s * 8, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    load_lut_smem(s_lut);
+    __syncthreads();
+    const LaneTables lt = make_lane_tables();
+    const Hyper2 h2 = make_hyper2(a.h);
+    for (int tile = a.tile_begin + blockIdx.x; tile < a.tile_end; tile += gridDim.x) {
+        const int t = find_tensor(a.tile_start, a.n_tensors, tile);
+        const TensorDesc d = a.descs[t];
+        float* w = a.params[t];
+        const void* g = a.grads[t];
+        const int local = tile - __ldg(a.tile_start + t);
+        switch (d.kind) {
+            case K_RANK1_FAST:
+                if ((d.cols & 255) == 0) pass2_rank1_bulk<BF16, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, ring, a.dev_status);
+                else pass2_rank1_fast<BF16, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut);
+                break;
             case K_RANK1_FLAT: pass2_flat<BF16, true, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut); break;
             case K_BLOCK:      pass2_flat<BF16, false, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut); break;
             default:           pass2_fp32<BF16, EXACT>(d, w, g, local, a.h); break;
@@ -649,7 +859,7 @@ __global__ void __launch_bounds__(kThreads, 3) pass1_kernel(StepArgs a) {
     __shared__ float s_col[kWarps * kWarpElems];
     const LaneTables lt = make_lane_tables();
     const Hyper2 h2 = make_hyper2(a.h);
-    for (int tile = blockIdx.x; tile < a.total_tiles; tile += gridDim.x) {
+    for (int tile = a.tile_begin + blockIdx.x; tile < a.tile_end; tile += gridDim.x) {
         const int t = find_tensor(a.tile_start, a.n_tensors, tile);
         const TensorDesc d = a.descs[t];
         const void* g = a.grads[t];
@@ -667,14 +877,27 @@ __global__ void rcp_kernel(const float* __restrict__ src, float* __restrict__ ds
 }  // namespace
 
 cudaError_t launch_pass1(const StepArgs& a, bool bf16, int grid, cudaStream_t s) {
-    if (a.total_tiles <= 0) return cudaSuccess;
+    if (a.tile_end <= a.tile_begin) return cudaSuccess;
     if (bf16) pass1_kernel<true><<<grid, kThreads, 0, s>>>(a);
     else pass1_kernel<false><<<grid, kThreads, 0, s>>>(a);
     return cudaGetLastError();
 }
 
+template <bool BF16, bool EXACT>
+cudaError_t launch_pass2_bulk_t(const StepArgs& a, int grid, cudaStream_t s) {
+    constexpr int smem = bulk_smem_bytes<BF16>();
+    cudaError_t e = cudaFuncSetAttribute(pass2_bulk_kernel<BF16, EXACT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    pass2_bulk_kernel<BF16, EXACT><<<grid, kThreads, smem, s>>>(a);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_pass2(const StepArgs& a, bool bf16, bool exact, int grid, cudaStream_t s) {
-    if (a.total_tiles <= 0) return cudaSuccess;
+    if (a.tile_end <= a.tile_begin) return cudaSuccess;
+    if (a.variant == 1) {
+        if (bf16) return exact ? launch_pass2_bulk_t<true, true>(a, grid, s) : launch_pass2_bulk_t<true, false>(a, grid, s);
+        return exact ? launch_pass2_bulk_t<false, true>(a, grid, s) : launch_pass2_bulk_t<false, false>(a, grid, s);
+    }
     if (bf16) {
         if (exact) pass2_kernel<true, true><<<grid, kThreads, 0, s>>>(a);
         else pass2_kernel<true, false><<<grid, kThreads, 0, s>>>(a);

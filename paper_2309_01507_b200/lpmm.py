@@ -30,7 +30,7 @@ EXPORTS = ("lpmm_state_bytes", "lpmm_state_init", "lpmm_state_attach", "lpmm_ada
            "lpmm_adamw4_step_host", "lpmm_stage_bytes", "lpmm_quantize", "lpmm_dequantize",
            "lpmm_quantize_rank1_noalloc",
            "lpmm_state_view", "lpmm_state_phase", "lpmm_state_last_launches", "lpmm_state_destroy",
-           "lpmm_state_profile", "lpmm_state_profile_read",
+           "lpmm_state_profile", "lpmm_state_profile_read", "lpmm_state_device_status",
            "lpmm_status_string", "lpmm_last_cuda_error")
 
 
@@ -82,6 +82,7 @@ def lib():
         L.lpmm_state_profile.argtypes = [vp, i32]
         L.lpmm_state_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_double),
                                               C.POINTER(i32)]
+        L.lpmm_state_device_status.argtypes = [vp, C.POINTER(i32), vp]
         L.lpmm_state_phase.argtypes = [vp]
         L.lpmm_state_last_launches.argtypes = [vp]
         L.lpmm_state_destroy.argtypes = [vp]
@@ -223,6 +224,13 @@ def profile_read(state: State) -> dict:
     _check(lib().lpmm_state_profile_read(state.handle, C.byref(p1), C.byref(rc), C.byref(p2), C.byref(n)),
            "lpmm_state_profile_read")
     return {"pass1_ms": p1.value, "rcp_ms": rc.value, "pass2_ms": p2.value, "steps": n.value}
+
+
+def device_status(state: State, stream=None) -> int:
+    """Device-side error word of the state (0 = ok); synchronizes the stream."""
+    out = C.c_int32()
+    _check(lib().lpmm_state_device_status(state.handle, C.byref(out), _stream_ptr(stream)), "lpmm_state_device_status")
+    return out.value
 
 
 def stage_bytes(state: State) -> int:

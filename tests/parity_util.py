@@ -56,6 +56,7 @@ class Pair:
     def compare(self, tol=1e-6, share_params=True, exact_params=False):
         """Codes and scales bit for bit; parameters within tol. Returns the worst normalised parameter error."""
         worst = 0.0
+        assert lpmm.device_status(self.state) == 0, "a step kernel reported an expired wait"
         for i, s in enumerate(self.specs):
             view = lpmm.state_view(self.state, i)
             o = self.ostate[i]
