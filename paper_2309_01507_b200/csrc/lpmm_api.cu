@@ -355,6 +355,7 @@ StepArgs make_args(const lpmm_state* st, float lr, float beta1, float beta2, flo
     a.h.one = 1.0f;
     a.h.step_size = (float)((double)lr / bc1);
     a.h.rbc2 = (float)(1.0 / bc2);
+    a.h2 = make_hyper2(a.h);
     return a;
 }
 

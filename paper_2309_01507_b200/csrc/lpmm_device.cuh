@@ -109,8 +109,9 @@ struct Hyper {
 struct Hyper2 {
     float2 beta1, omb1, beta2, omb2;
     float2 rbc2, eps, neg_step, decay, one;
+    float2 c16, cm15, magic;   // 16, -1.5 and 2^23 for the linear quantizer
 };
-__device__ __forceinline__ float2 splat(float x) { return make_float2(x, x); }
+__host__ __device__ __forceinline__ float2 splat(float x) { return make_float2(x, x); }
 
 // Packed operations written as PTX with an explicit rounding mode: such instructions are never
 // contracted into a fused multiply-add, which the stored states rely on.
@@ -144,11 +145,12 @@ __device__ __forceinline__ float2 fma2_rn(float2 a, float2 b, float2 c) {
     asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(pack2(a)), "l"(pack2(b)), "l"(pack2(c)));
     return unpack2(d);
 }
-__device__ __forceinline__ Hyper2 make_hyper2(const Hyper& h) {
+__host__ __device__ __forceinline__ Hyper2 make_hyper2(const Hyper& h) {
     Hyper2 p;
     p.beta1 = splat(h.beta1); p.omb1 = splat(h.omb1); p.beta2 = splat(h.beta2); p.omb2 = splat(h.omb2);
     p.rbc2 = splat(h.rbc2); p.eps = splat(h.eps); p.neg_step = splat(-h.step_size); p.decay = splat(h.decay);
     p.one = splat(h.one);
+    p.c16 = splat(16.0f); p.cm15 = splat(-1.5f); p.magic = splat(8388608.0f);
     return p;
 }
 // Both products must be rounded before the sum (Eq. 1 evaluated operation by operation). The assembler

@@ -49,6 +49,7 @@ struct StepArgs {
     int32_t variant;             // pass 2: 0 = rows prefetched into registers, 1 = rows staged by bulk copies
     uint32_t* dev_status;        // device error word in the arena header (0 = ok)
     Hyper h;
+    Hyper2 h2;                   // the same constants as pairs (kernel-parameter space: usable as operands)
 };
 
 cudaError_t launch_pass1(const StepArgs& a, bool bf16, int grid, cudaStream_t s);

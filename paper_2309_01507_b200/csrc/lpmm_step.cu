@@ -176,9 +176,9 @@ __device__ __forceinline__ uint32_t quantize8_de(const float (&x)[8], float rcp,
     return q;
 }
 // Linear codes as the low mantissa bits of 2^23 + ceil(max(16 n - 1.5, 0)) (see lin_nearest_magic()).
-__device__ __forceinline__ uint32_t quantize8_lin(const float (&x)[8], const float (&rcp)[8]) {
+__device__ __forceinline__ uint32_t quantize8_lin(const float (&x)[8], const float (&rcp)[8], const Hyper2& h2) {
     uint32_t q = 0;
-    const float2 c16 = splat(16.0f), cm = splat(-1.5f), magic = splat(8388608.0f);
+    const float2 c16 = h2.c16, cm = h2.cm15, magic = h2.magic;
 #pragma unroll
     for (int k = 6; k >= 0; k -= 2) {
         float2 y = fma2_rn(mul2_rn(make_float2(x[k], x[k + 1]), make_float2(rcp[k], rcp[k + 1])), c16, cm);
@@ -281,7 +281,7 @@ __device__ __forceinline__ void process_row(const RowRegs<BF16>& r, const TileVi
     const float am_new = group_max(absmax8(mt), lt.mask);
     if ((threadIdx.x & 15) == 0) t.m_scale[off >> 7] = am_new;
     *reinterpret_cast<uint32_t*>(t.m_codes + (off >> 1)) = quantize8_de(mt, scale_rcp(am_new), s_lut);
-    *reinterpret_cast<uint32_t*>(t.v_codes + (off >> 1)) = quantize8_lin(vt, vr);
+    *reinterpret_cast<uint32_t*>(t.v_codes + (off >> 1)) = quantize8_lin(vt, vr, h2);
 }
 
 template <bool BF16, bool EXACT>
@@ -502,7 +502,7 @@ __device__ __forceinline__ void pass2_rank1_bulk(const TensorDesc& d, float* __r
         const float am_new = group_max(absmax8(mt), lt.mask);
         if ((lane & 15) == 0) ms_warp[(size_t)(off >> 7) + (lane >> 4)] = am_new;
         *reinterpret_cast<uint32_t*>(mq_lane + (off >> 1)) = quantize8_de(mt, scale_rcp(am_new), s_lut);
-        *reinterpret_cast<uint32_t*>(vq_lane + (off >> 1)) = quantize8_lin(vt, vr);
+        *reinterpret_cast<uint32_t*>(vq_lane + (off >> 1)) = quantize8_lin(vt, vr, h2);
     }
 }
 
@@ -570,7 +570,7 @@ __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restric
         }
         if (lane_live && (lane & 15) == 0) d.m_scale[e >> 7] = am_new;
         const uint32_t qm_new = quantize8_de(mt, scale_rcp(am_new), s_lut);
-        const uint32_t qv_new = quantize8_lin(vt, vr);
+        const uint32_t qv_new = quantize8_lin(vt, vr, h2);
         if (full) {
             store8_f32(w + e, wv);
             *reinterpret_cast<uint32_t*>(d.m_codes + (e >> 1)) = qm_new;
@@ -621,7 +621,7 @@ __global__ void __launch_bounds__(kThreads, 2) pass2_kernel(StepArgs a) {
     load_lut_smem(s_lut);
     __syncthreads();
     const LaneTables lt = make_lane_tables();
-    const Hyper2 h2 = make_hyper2(a.h);
+    const Hyper2& h2 = a.h2;
     for (int tile = a.tile_begin + blockIdx.x; tile < a.tile_end; tile += gridDim.x) {
         const int t = find_tensor(a.tile_start, a.n_tensors, tile);
         const TensorDesc d = a.descs[t];   // by value: the fields stay in registers across the stores below
@@ -655,7 +655,7 @@ __global__ void __launch_bounds__(kThreads, 2) pass2_bulk_kernel(StepArgs a) {
     load_lut_smem(s_lut);
     __syncthreads();
     const LaneTables lt = make_lane_tables();
-    const Hyper2 h2 = make_hyper2(a.h);
+    const Hyper2& h2 = a.h2;
     for (int tile = a.tile_begin + blockIdx.x; tile < a.tile_end; tile += gridDim.x) {
         const int t = find_tensor(a.tile_start, a.n_tensors, tile);
         const TensorDesc d = a.descs[t];
@@ -858,7 +858,7 @@ template <bool BF16>
 __global__ void __launch_bounds__(kThreads, 3) pass1_kernel(StepArgs a) {
     __shared__ float s_col[kWarps * kWarpElems];
     const LaneTables lt = make_lane_tables();
-    const Hyper2 h2 = make_hyper2(a.h);
+    const Hyper2& h2 = a.h2;
     for (int tile = a.tile_begin + blockIdx.x; tile < a.tile_end; tile += gridDim.x) {
         const int t = find_tensor(a.tile_start, a.n_tensors, tile);
         const TensorDesc d = a.descs[t];
