@@ -49,6 +49,8 @@ def parse_args():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--m-block", type=int, default=128, choices=[128, 2048], help="first-moment block size")
+    ap.add_argument("--v-mode", default="rank1", choices=["rank1", "block"], help="second-moment normalizer of matrices")
     return ap.parse_args()
 
 
@@ -208,7 +210,8 @@ def run_ours(args):
     hyper = dict(lr=wl.lr, beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps, weight_decay=wl.weight_decay)
     params = [workloads.make_param(t, wl.index, i, device=dev) for i, t in enumerate(wl.tensors)]
     grads = [workloads.make_grad(t, wl.index, i, 1, device=dev, dtype=gdt) for i, t in enumerate(wl.tensors)]
-    state = lpmm.state_init(lpmm.default_config(), wl.tensors, device=dev)
+    cfg = lpmm.default_config(m_block=args.m_block, v_mode=lpmm.V_BLOCK if args.v_mode == "block" else lpmm.V_RANK1)
+    state = lpmm.state_init(cfg, wl.tensors, device=dev)
     cache = lpmm.make_ptr_cache(params, grads)
     n_params = wl.numel
     torch.cuda.synchronize()
@@ -257,7 +260,7 @@ def run_ours(args):
             hp[-1].copy_(p.reshape(-1)); hg[-1].copy_(g.reshape(-1))
             off += k
         torch.cuda.synchronize()
-        e2e_state = lpmm.state_init(lpmm.default_config(), wl.tensors, device=dev)
+        e2e_state = lpmm.state_init(cfg, wl.tensors, device=dev)
         t = 0
         for _ in range(1):
             t += 1
@@ -286,7 +289,9 @@ def run_ours(args):
     peak, peak_kind = measured_peak()
     p2_ms = prof["pass2_ms"] / max(prof["steps"], 1)
     p1_ms = prof["pass1_ms"] / max(prof["steps"], 1)
-    alg_bytes = PASS2_BYTES[wl.grad_dtype] * n_params
+    # block maxima: 8 bytes per block of m (and of v when v is block-wise; then pass 1 has nothing to do)
+    pass2_bpp = PASS2_BYTES[wl.grad_dtype] - 8 / 128 + 8 / args.m_block + (8 / 128 if args.v_mode == "block" else 0)
+    alg_bytes = pass2_bpp * n_params
     achieved = alg_bytes / (p2_ms * 1e-3) / 1e9
     traffic_pp = PASS2_TRAFFIC_BYTES_PER_PARAM[wl.grad_dtype]
     roofline = {"bound": "hbm", "kernel": "pass2_kernel (update + re-quantize)", "achieved": achieved, "peak": peak,
@@ -296,7 +301,7 @@ def run_ours(args):
                 "pass1_ms_per_launch": p1_ms,
                 "pass1_achieved_gbs": PASS1_BYTES[wl.grad_dtype] * n_params / (p1_ms * 1e-3) / 1e9 if p1_ms > 0 else None,
                 "step_algorithmic_gbs": alg_bytes / (ms_step * 1e-3) / 1e9,
-                "step_moved_gbs": (PASS2_BYTES[wl.grad_dtype] + PASS1_BYTES[wl.grad_dtype]) * n_params / (ms_step * 1e-3) / 1e9,
+                "step_moved_gbs": (pass2_bpp + (PASS1_BYTES[wl.grad_dtype] if args.v_mode == "rank1" else 0)) * n_params / (ms_step * 1e-3) / 1e9,
                 "frac_of_nominal_8tbs": achieved / 8000.0}
 
     cpu = None
@@ -308,8 +313,8 @@ def run_ours(args):
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": wl.name, "tensors": len(wl.tensors), "params_per_gpu": n_params,
-                       "grad_dtype": wl.grad_dtype, "param_dtype": "f32", "m": "B128/DE 4-bit", "v": "Rank-1/Linear 4-bit",
-                       "l2": "inputs larger than L2 (47 GB resident), no flush", "parallelism": f"replicas x{world}, no collective"},
+                       "grad_dtype": wl.grad_dtype, "param_dtype": "f32", "m": f"B{args.m_block}/DE 4-bit", "v": ("Rank-1" if args.v_mode == "rank1" else "B128") + "/Linear 4-bit",
+                       "l2": f"inputs larger than L2 ({(n_params * (8 + (2 if wl.grad_dtype == 'bf16' else 4) + 1)) / 1e9:.1f} GB touched per step), no flush", "parallelism": f"replicas x{world}, no collective"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu}
     print(json.dumps(line), flush=True)
     dist.shutdown()

@@ -66,7 +66,7 @@ typedef struct {
 
 typedef struct {
     int32_t bits;            /* 4 */
-    int32_t m_block;         /* first-moment block size B (Sec. 3: 128) */
+    int32_t m_block;         /* first-moment block size B: 128 (Sec. 3) or 2048 (the 8-bit optimizer's size, Sec. 2.2) */
     int32_t v_block;         /* second-moment block size for 1-D tensors and LPMM_V_BLOCK (Sec. 4.2: 128) */
     int32_t v_mode;          /* lpmm_vmode */
     int64_t min_quant_numel; /* tensors with numel <= this keep fp32 states (App. C.1: 4096) */

@@ -56,7 +56,7 @@ lpmm_status validate_config(const lpmm_config* cfg, const lpmm_shape* shapes, in
     if (cfg->min_quant_numel < 0) return LPMM_ERR_INVALID_ARG;
     if (cfg->v_mode != LPMM_V_RANK1 && cfg->v_mode != LPMM_V_BLOCK) return LPMM_ERR_INVALID_ARG;
     if (cfg->bits != 4) return LPMM_ERR_UNSUPPORTED;
-    if (cfg->m_block != 128 || cfg->v_block != 128) return LPMM_ERR_UNSUPPORTED;
+    if ((cfg->m_block != 128 && cfg->m_block != 2048) || cfg->v_block != 128) return LPMM_ERR_UNSUPPORTED;
     if (cfg->update_math != LPMM_UPDATE_FAST && cfg->update_math != LPMM_UPDATE_IEEE) return LPMM_ERR_INVALID_ARG;
     for (int32_t i = 0; i < n; ++i) {
         const lpmm_shape& s = shapes[i];
@@ -76,7 +76,8 @@ int32_t choose_kind(const lpmm_config& cfg, const lpmm_shape& s) {
     if (s.flags & LPMM_FORCE_FP32) return K_FP32;
     if (!(s.flags & LPMM_FORCE_QUANT) && numel <= cfg.min_quant_numel) return K_FP32;  // App. C.1
     if (s.ndim == 1 || s.rows == 1 || s.cols == 1 || cfg.v_mode == LPMM_V_BLOCK) return K_BLOCK;  // Sec. 4.2
-    return (s.cols % 128 == 0) ? K_RANK1_FAST : K_RANK1_FLAT;
+    // the tiled path needs whole first-moment blocks inside a row (and, for B2048, one block per tile width)
+    return (s.cols % cfg.m_block == 0) ? K_RANK1_FAST : K_RANK1_FLAT;
 }
 
 void compute_layout(const lpmm_config& cfg, const lpmm_shape* shapes, int32_t n, Layout* L) {
@@ -112,9 +113,10 @@ void compute_layout(const lpmm_config& cfg, const lpmm_shape* shapes, int32_t n,
         } else {
             const size_t code_bytes = (size_t)((t.numel + 1) / 2);
             const size_t nblk = (size_t)((t.numel + 127) / 128);
+            const size_t nblk_m = (size_t)((t.numel + cfg.m_block - 1) / cfg.m_block);
             t.m_codes = off; off = align_up(off + code_bytes);
             t.v_codes = off; off = align_up(off + code_bytes);
-            t.m_scale = off; off = align_up(off + sizeof(float) * nblk);
+            t.m_scale = off; off = align_up(off + sizeof(float) * nblk_m);
             if (t.kind == K_BLOCK) { t.v_bscale = off; off = align_up(off + sizeof(float) * nblk); }
         }
     }
@@ -172,6 +174,7 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
         TensorDesc& d = descs[i];
         std::memset(&d, 0, sizeof(d));
         d.rows = t.rows; d.cols = t.cols; d.numel = t.numel; d.kind = t.kind; d.c_off = t.c_off;
+        d.m_shift = (st->cfg.m_block == 2048) ? 11 : 7;
         int64_t tiles = 0;
         if (t.kind == K_FP32) {
             d.m32 = reinterpret_cast<float*>(A + t.m32);
@@ -188,7 +191,7 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
             }
         }
         if (t.kind == K_RANK1_FAST) {
-            d.wx = (t.cols % 1024 == 0) ? 4 : (t.cols % 512 == 0) ? 2 : 1;
+            d.wx = (st->cfg.m_block == 2048) ? 8 : (t.cols % 1024 == 0) ? 4 : (t.cols % 512 == 0) ? 2 : 1;
             const int64_t tile_cols = (int64_t)kWarpElems * d.wx;
             int64_t tr = tile_elems / tile_cols;
             if (tr < kWarps / d.wx) tr = kWarps / d.wx;

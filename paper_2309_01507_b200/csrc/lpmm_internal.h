@@ -21,7 +21,7 @@ constexpr int kWarpElems = 32 * kLaneElems;  // 256: two 128-element blocks per 
 // One entry of the device-side tensor table (lives at the head of the arena).
 struct TensorDesc {
     uint8_t* m_codes;   // ceil(numel/2) bytes
-    float* m_scale;     // ceil(numel/128) block maxima of |m|
+    float* m_scale;     // ceil(numel / m_block) block maxima of |m|
     uint8_t* v_codes;
     float* v_bscale;    // K_BLOCK: ceil(numel/128) block maxima of v
     float* rc[2];       // K_RANK1_*: two buffers of [r (rows, padded to 4) | c (cols)]
@@ -35,7 +35,8 @@ struct TensorDesc {
     int32_t tiles_x;    // K_RANK1_FAST: column tiles
     int32_t tile_rows;  // K_RANK1_FAST: rows per tile
     int32_t flat_chunks;  // other kinds: 256-element chunks per warp per tile
-    int32_t pad[2];
+    int32_t m_shift;    // log2 of the first-moment block size: 7 (B128) or 11 (B2048)
+    int32_t pad;
 };
 
 struct StepArgs {

@@ -163,6 +163,20 @@ __device__ __forceinline__ float group_max(float x, unsigned mask) {   // over t
     return x;
 }
 
+// Maximum over one first-moment block. B128: the 16 lanes that own it. B2048: the whole CTA (its 8 warps
+// cover exactly one block per step and move in lockstep); the two halves of s_red alternate from step to
+// step, so one barrier per step is enough.
+__device__ __forceinline__ float block_max(float x, int m_shift, const LaneTables& lt, float* s_red, uint32_t& step) {
+    if (m_shift == 7) return group_max(x, lt.mask);
+    x = warp_max(x);
+    float* slot = s_red + (step++ & 1u) * kWarps;   // the counter runs across tiles: every thread calls this equally often
+    if ((threadIdx.x & 31) == 0) slot[threadIdx.x >> 5] = x;
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < kWarps; ++i) x = fmaxf(x, slot[i]);
+    return x;
+}
+
 // Eight nearest codes packed little-nibble-first: acc = acc * 16 + code, from element 7 down to 0.
 __device__ __forceinline__ uint32_t quantize8_de(const float (&x)[8], float rcp, const unsigned char* s_lut) {
     uint32_t q = 0;
@@ -224,6 +238,9 @@ struct TileView {
     const float* r_rcp;
     uint32_t row_step;     // elements between two rows this warp handles
     uint32_t row_stride;   // rows between them
+    int m_shift;           // log2 of the first-moment block size
+    float* s_red;          // CTA scratch for B2048 block maxima
+    uint32_t* red_step;    // running count of CTA-wide reductions
 };
 
 // Asks L2 to fetch this lane's share of row k ahead of time (no register is tied up): the later
@@ -242,7 +259,7 @@ __device__ __forceinline__ void prefetch_row(const TileView& t, uint32_t k) {
     }
     prefetch_l2(t.m_codes + (off >> 1));
     prefetch_l2(t.v_codes + (off >> 1));
-    prefetch_l2(t.m_scale + (off >> 7));
+    prefetch_l2(t.m_scale + (off >> t.m_shift));
 }
 
 template <bool BF16>
@@ -258,7 +275,7 @@ __device__ __forceinline__ void load_row(RowRegs<BF16>& r, const TileView& t, ui
     }
     r.qm = *reinterpret_cast<const uint32_t*>(t.m_codes + (off >> 1));
     r.qv = *reinterpret_cast<const uint32_t*>(t.v_codes + (off >> 1));
-    r.am = t.m_scale[off >> 7];
+    r.am = t.m_scale[off >> t.m_shift];
     r.r_old = __ldg(t.r_old + k * t.row_stride);
     r.r_rcp = __ldg(t.r_rcp + k * t.row_stride);
 }
@@ -278,8 +295,8 @@ __device__ __forceinline__ void process_row(const RowRegs<BF16>& r, const TileVi
     }
     moments_and_update8<EXACT>(wv, gv, r.qm, r.qv, __fmul_rn(lt.de, r.am), vs, h, h2, lt, mt, vt);
     store8_f32(t.w + off, wv);
-    const float am_new = group_max(absmax8(mt), lt.mask);
-    if ((threadIdx.x & 15) == 0) t.m_scale[off >> 7] = am_new;
+    const float am_new = block_max(absmax8(mt), t.m_shift, lt, t.s_red, *t.red_step);
+    if ((threadIdx.x & (t.m_shift == 7 ? 15 : 2047)) == 0) t.m_scale[off >> t.m_shift] = am_new;
     *reinterpret_cast<uint32_t*>(t.m_codes + (off >> 1)) = quantize8_de(mt, scale_rcp(am_new), s_lut);
     *reinterpret_cast<uint32_t*>(t.v_codes + (off >> 1)) = quantize8_lin(vt, vr, h2);
 }
@@ -287,12 +304,15 @@ __device__ __forceinline__ void process_row(const RowRegs<BF16>& r, const TileVi
 template <bool BF16, bool EXACT>
 __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __restrict__ w, const void* __restrict__ g,
                                                  int tile, int phase, const Hyper& h, const Hyper2& h2,
-                                                 const LaneTables& lt, const unsigned char* s_lut) {
+                                                 const LaneTables& lt, const unsigned char* s_lut, float* s_red,
+                                                 uint32_t& red_step) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int wx = d.wx, wy_count = kWarps / wx;
     const int tx = tile % d.tiles_x, ty = tile / d.tiles_x;
     const int64_t col0 = (int64_t)tx * (kWarpElems * wx) + (warp % wx) * kWarpElems + lane * kLaneElems;
-    if (col0 >= d.cols) return;   // cols % 128 == 0: a whole 16-lane group (one block) is in or out together
+    // cols % 128 == 0: a whole 16-lane group (one block) is in or out together. With B2048 the tile is one
+    // block wide (wx = 8, cols % 2048 == 0), every warp is inside and all of them run the same rows.
+    if (col0 >= d.cols) return;
     const float* rc_old = (phase ? d.rc[1] : d.rc[0]);
     const float* rcp_new = d.rcp_new;
     const int64_t row0 = (int64_t)ty * d.tile_rows + warp / wx;
@@ -310,11 +330,14 @@ __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __r
                : static_cast<const void*>(reinterpret_cast<const float*>(g) + e0);
     t.m_codes = d.m_codes + (e0 >> 1);
     t.v_codes = d.v_codes + (e0 >> 1);
-    t.m_scale = d.m_scale + (e0 >> 7);
+    t.m_scale = d.m_scale + (e0 >> d.m_shift);
     t.r_old = rc_old + row0;
     t.r_rcp = rcp_new + row0;
     t.row_step = (uint32_t)(wy_count * d.cols);
     t.row_stride = (uint32_t)wy_count;
+    t.m_shift = d.m_shift;
+    t.s_red = s_red;
+    t.red_step = &red_step;
 
     // Two register sets alternate: while one row is processed the next one is already in flight.
     RowRegs<BF16> ra, rb;
@@ -511,14 +534,19 @@ __device__ __forceinline__ void pass2_rank1_bulk(const TensorDesc& d, float* __r
 template <bool BF16, bool RANK1, bool EXACT>
 __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restrict__ w, const void* __restrict__ g,
                                            int tile, int phase, const Hyper& h, const Hyper2& h2, const LaneTables& lt,
-                                           const unsigned char* s_lut) {
+                                           const unsigned char* s_lut, float* s_red, uint32_t& red_step) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const float* rc_old = (phase ? d.rc[1] : d.rc[0]);
     const float* rcp_new = d.rcp_new;
+    const int64_t m_mask = ((int64_t)1 << d.m_shift) - 1;
     for (int c = 0; c < d.flat_chunks; ++c) {
-        const int64_t chunk = ((int64_t)tile * d.flat_chunks + c) * kWarps + warp;
+        const int64_t chunk0 = ((int64_t)tile * d.flat_chunks + c) * kWarps;   // the CTA's 8 chunks = 2048 elements
+        const int64_t chunk = chunk0 + warp;
         const int64_t e = chunk * kWarpElems + lane * kLaneElems;
-        if (chunk * kWarpElems >= d.numel) break;          // uniform per warp
+        if (chunk0 * kWarpElems >= d.numel) break;          // uniform over the CTA
+        // B128: a warp past the end has nothing to do. B2048: it still joins the CTA-wide block maximum
+        // (with zeros; its loads and stores are all guarded away).
+        if (d.m_shift == 7 && chunk * kWarpElems >= d.numel) break;
         const bool full = (chunk + 1) * kWarpElems <= d.numel;
         float wv[8], gv[8], mt[8], vt[8], vs[8], vr[8];
         uint32_t qm, qv;
@@ -536,8 +564,8 @@ __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restric
         const bool lane_live = e < d.numel;
         // every lane of a 16-lane group that still holds an element needs the block's scale: the
         // shuffle-based table lookup reads T[q] * scale from the group's other lanes
-        const bool group_live = (e & ~(int64_t)127) < d.numel;
-        const float am = group_live ? d.m_scale[e >> 7] : 0.0f;
+        const bool group_live = (e & ~m_mask) < d.numel;
+        const float am = group_live ? d.m_scale[e >> d.m_shift] : 0.0f;
         if (RANK1) {
             int64_t i = e / d.cols, j = e - i * d.cols;
 #pragma unroll
@@ -560,7 +588,7 @@ __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restric
 #pragma unroll
             for (int k = 0; k < 8; ++k) if (e + k >= d.numel) { mt[k] = 0.0f; vt[k] = 0.0f; }
         }
-        const float am_new = half_warp_max(absmax8(mt));
+        const float am_new = block_max(absmax8(mt), d.m_shift, lt, s_red, red_step);
         if (!RANK1) {
             const float av_new = half_warp_max(absmax8(vt));
             const float r = scale_rcp(av_new);
@@ -568,7 +596,7 @@ __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restric
             for (int k = 0; k < 8; ++k) vr[k] = r;
             if (lane_live && (lane & 15) == 0) d.v_bscale[e >> 7] = av_new;
         }
-        if (lane_live && (lane & 15) == 0) d.m_scale[e >> 7] = am_new;
+        if (lane_live && (threadIdx.x & (d.m_shift == 7 ? 15 : 2047)) == 0) d.m_scale[e >> d.m_shift] = am_new;
         const uint32_t qm_new = quantize8_de(mt, scale_rcp(am_new), s_lut);
         const uint32_t qv_new = quantize8_lin(vt, vr, h2);
         if (full) {
@@ -618,10 +646,12 @@ __device__ __forceinline__ void pass2_fp32(const TensorDesc& d, float* __restric
 template <bool BF16, bool EXACT>
 __global__ void __launch_bounds__(kThreads, 2) pass2_kernel(StepArgs a) {
     __shared__ __align__(16) unsigned char s_lut[kLutSmemBytes];
+    __shared__ float s_red[2 * kWarps];
     load_lut_smem(s_lut);
     __syncthreads();
     const LaneTables lt = make_lane_tables();
     const Hyper2& h2 = a.h2;
+    uint32_t red_step = 0;
     for (int tile = a.tile_begin + blockIdx.x; tile < a.tile_end; tile += gridDim.x) {
         const int t = find_tensor(a.tile_start, a.n_tensors, tile);
         const TensorDesc d = a.descs[t];   // by value: the fields stay in registers across the stores below
@@ -629,9 +659,9 @@ __global__ void __launch_bounds__(kThreads, 2) pass2_kernel(StepArgs a) {
         const void* g = a.grads[t];
         const int local = tile - __ldg(a.tile_start + t);
         switch (d.kind) {
-            case K_RANK1_FAST: pass2_rank1_fast<BF16, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut); break;
-            case K_RANK1_FLAT: pass2_flat<BF16, true, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut); break;
-            case K_BLOCK:      pass2_flat<BF16, false, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut); break;
+            case K_RANK1_FAST: pass2_rank1_fast<BF16, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
+            case K_RANK1_FLAT: pass2_flat<BF16, true, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
+            case K_BLOCK:      pass2_flat<BF16, false, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
             default:           pass2_fp32<BF16, EXACT>(d, w, g, local, a.h); break;
         }
     }
@@ -642,6 +672,7 @@ __global__ void __launch_bounds__(kThreads, 2) pass2_bulk_kernel(StepArgs a) {
     extern __shared__ __align__(128) unsigned char s_dyn[];   // [nearest-entry table | warp rings | mbarriers]
     unsigned char* s_lut = s_dyn;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    __shared__ float s_red[2 * kWarps];
     WarpRing ring;
     ring.data = s_dyn + kLutSmemBytes + warp * kBulkStages * WarpStage<BF16>::kBytes;
     ring.bars = smem_u32(s_dyn + kLutSmemBytes + kWarps * kBulkStages * WarpStage<BF16>::kBytes) + warp * kBulkStages * 8;
@@ -656,6 +687,7 @@ __global__ void __launch_bounds__(kThreads, 2) pass2_bulk_kernel(StepArgs a) {
     __syncthreads();
     const LaneTables lt = make_lane_tables();
     const Hyper2& h2 = a.h2;
+    uint32_t red_step = 0;
     for (int tile = a.tile_begin + blockIdx.x; tile < a.tile_end; tile += gridDim.x) {
         const int t = find_tensor(a.tile_start, a.n_tensors, tile);
         const TensorDesc d = a.descs[t];
@@ -664,11 +696,11 @@ __global__ void __launch_bounds__(kThreads, 2) pass2_bulk_kernel(StepArgs a) {
         const int local = tile - __ldg(a.tile_start + t);
         switch (d.kind) {
             case K_RANK1_FAST:
-                if ((d.cols & 255) == 0) pass2_rank1_bulk<BF16, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, ring, a.dev_status);
-                else pass2_rank1_fast<BF16, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut);
+                if ((d.cols & 255) == 0 && d.m_shift == 7) pass2_rank1_bulk<BF16, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, ring, a.dev_status);
+                else pass2_rank1_fast<BF16, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step);
                 break;
-            case K_RANK1_FLAT: pass2_flat<BF16, true, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut); break;
-            case K_BLOCK:      pass2_flat<BF16, false, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut); break;
+            case K_RANK1_FLAT: pass2_flat<BF16, true, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
+            case K_BLOCK:      pass2_flat<BF16, false, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
             default:           pass2_fp32<BF16, EXACT>(d, w, g, local, a.h); break;
         }
     }

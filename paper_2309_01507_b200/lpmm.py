@@ -43,8 +43,8 @@ class Config(C.Structure):
                 ("min_quant_numel", C.c_int64), ("update_math", C.c_int32), ("reserved", C.c_int32)]
 
 
-def default_config(v_mode: int = V_RANK1, min_quant_numel: int = 4096, update_math: int = 0) -> Config:
-    return Config(4, 128, 128, v_mode, min_quant_numel, update_math, 0)
+def default_config(v_mode: int = V_RANK1, min_quant_numel: int = 4096, update_math: int = 0, m_block: int = 128) -> Config:
+    return Config(4, m_block, 128, v_mode, min_quant_numel, update_math, 0)
 
 
 class LpmmError(RuntimeError):

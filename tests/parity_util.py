@@ -39,7 +39,7 @@ class Pair:
             if self.config.v_mode == lpmm.V_BLOCK and want == oracle.RANK1:
                 want = oracle.BLOCK
             assert k == want, (s, k, want)
-            self.ostate.append(oracle.state_init(s.rows, s.cols, k))
+            self.ostate.append(oracle.state_init(s.rows, s.cols, k, m_block=self.config.m_block))
 
     def grads_for(self, step, outlier_p=1e-3, device="cuda"):
         return [workloads.make_grad(s, self.widx, i, step, device=device, dtype=self.grad_dtype, outlier_p=outlier_p)

@@ -62,7 +62,7 @@ def test_bad_configurations_are_rejected_on_the_host():
     assert L.lpmm_state_bytes(None, shapes, 1, C.byref(out)) == lpmm.ERR_INVALID_ARG
     assert L.lpmm_state_bytes(C.byref(cfg), shapes, 0, C.byref(out)) == lpmm.ERR_INVALID_ARG
     assert L.lpmm_state_bytes(C.byref(cfg), shapes, 1, None) == lpmm.ERR_INVALID_ARG
-    for field, value, want in (("bits", 8, lpmm.ERR_UNSUPPORTED), ("m_block", 64, lpmm.ERR_UNSUPPORTED),
+    for field, value, want in (("bits", 8, lpmm.ERR_UNSUPPORTED), ("m_block", 64, lpmm.ERR_UNSUPPORTED), ("v_block", 2048, lpmm.ERR_UNSUPPORTED),
                                ("v_mode", 7, lpmm.ERR_INVALID_ARG), ("min_quant_numel", -1, lpmm.ERR_INVALID_ARG)):
         bad = lpmm.default_config()
         setattr(bad, field, value)

@@ -151,6 +151,20 @@ def test_block_mode_for_matrices():
         pair.compare(tol=1e-6)
 
 
+@pytest.mark.parametrize("grad_dtype", [torch.float32, torch.bfloat16])
+def test_first_moment_block_2048(grad_dtype):
+    # B2048 for m (the block size of the 8-bit optimizers, Sec. 2.2) with rank-1 / B128 v as before.
+    cfg = lpmm.default_config(m_block=2048)
+    specs = [_mat(64, 2048), _mat(24, 4096), _mat(130, 384), _mat(96, 256), _mat(33, 77), _vec(50265), _vec(4097),
+             _vec(2048 * 3, force_quant=True), _mat(40, 1024)]
+    hyper = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
+    pair = Pair(specs, hyper, config=cfg, grad_dtype=grad_dtype, workload_index=11)
+    for t in range(1, 5):
+        pair.step(t, pair.grads_for(t, outlier_p=0.0 if t % 2 == 0 else 1e-3))
+        pair.compare(tol=1e-6)
+    assert pair.ostate[0].m_scale.size == 64     # one scale per 2048 elements
+
+
 def test_transformer_base_three_steps_one_launch_per_pass():
     wl = workloads.transformer_base()
     pair = Pair(wl.tensors, hyper_of(wl), workload_index=wl.index)
