@@ -113,6 +113,14 @@ lpmm_status lpmm_adamw4_step(lpmm_state* st, void* const* d_params, const void* 
                              int32_t grad_dtype, float lr, float beta1, float beta2, float eps,
                              float weight_decay, int64_t step, void* stream);
 
+/* One fused step of Alg. 2 (compressed SGDM) over every tensor of the state: decompress m (B128 or B2048 / DE);
+ * m <- beta m + g ; w <- w - lr m ; new block maxima ; compress m. Only the first-moment part of the state
+ * is used (tensors of <= min_quant_numel elements keep m in fp32); do not mix with lpmm_adamw4_step on one
+ * state. One kernel launch; the parameters follow the same operation order as the algorithm's lines 4-5, so
+ * they are reproducible bit for bit. Arguments as lpmm_adamw4_step; 0 <= beta < 1, lr >= 0. */
+lpmm_status lpmm_sgdm4_step(lpmm_state* st, void* const* d_params, const void* const* d_grads,
+                            int32_t grad_dtype, float lr, float beta, void* stream);
+
 /* The same step for callers whose parameters and gradients live in HOST memory (optimizer
  * offloading): copies every tensor's parameters and gradient into the caller's device staging
  * buffers, runs the step there and copies the updated parameters back. The tensors are processed in

@@ -235,3 +235,14 @@ def adamw4_step(w: np.ndarray, g: np.ndarray, st: TensorState, *, lr, beta1, bet
                                        _p(st.m32), _p(st.v32), C.byref(h))
     if rc != 0:
         raise ValueError("lpmm_oracle_adamw4_step rejected its arguments")
+
+
+def sgdm4_step(w: np.ndarray, g: np.ndarray, st: TensorState, *, lr, beta, true_division: bool = False) -> None:
+    """One compressed SGDM step (Alg. 2) on one tensor; only the first-moment part of `st` is used."""
+    assert w.dtype == np.float32 and w.flags.c_contiguous and w.size == st.numel
+    g = _f32(g)
+    rc = lib().lpmm_oracle_sgdm4_step(_p(w), _p(g), C.c_int64(st.numel), C.c_int(int(st.kind != FP32)),
+                                      C.c_int64(st.m_block), _p(st.m_codes), _p(st.m_scale), _p(st.m32),
+                                      C.c_float(lr), C.c_float(beta), C.c_int(int(true_division)))
+    if rc != 0:
+        raise ValueError("lpmm_oracle_sgdm4_step rejected its arguments")

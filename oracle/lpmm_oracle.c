@@ -350,6 +350,43 @@ int lpmm_oracle_adamw4_step(float* w, const float* g, int64_t rows, int64_t cols
     return 0;
 }
 
+/* ------------------------------------------------------------------ the compressed SGDM step (Alg. 2) */
+
+int lpmm_oracle_sgdm4_step(float* w, const float* g, int64_t numel, int quantized, int64_t m_block,
+                           uint8_t* m_codes, float* m_scale, float* m32, float lr, float beta, int true_division) {
+    if (!w || !g || numel <= 0) return -1;
+    float* m = (float*)malloc(sizeof(float) * (size_t)numel);
+    if (!m) return -1;
+    float Tde[16];
+    lpmm_oracle_de_map(4, 1, 0, Tde);
+    uint8_t* q = NULL;
+    if (quantized) {                                   /* line 3: decompress */
+        q = (uint8_t*)malloc((size_t)numel);
+        if (!q) { free(m); return -1; }
+        lpmm_oracle_unpack4(m_codes, numel, q);
+        lpmm_oracle_dequantize_block(q, numel, m_block, Tde, m_scale, m);
+    } else {
+        memcpy(m, m32, sizeof(float) * (size_t)numel);
+    }
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < numel; ++i) {
+        float a = beta * m[i];
+        float mt = a + g[i];                           /* line 4 */
+        float upd = lr * mt;
+        w[i] = w[i] - upd;                             /* line 5 */
+        m[i] = mt;
+    }
+    if (quantized) {                                   /* line 6: compress */
+        lpmm_oracle_quantize_block(m, numel, m_block, Tde, 16, 0, true_division, m_scale, q);
+        lpmm_oracle_pack4(q, numel, m_codes);
+        free(q);
+    } else {
+        memcpy(m32, m, sizeof(float) * (size_t)numel);
+    }
+    free(m);
+    return 0;
+}
+
 int lpmm_oracle_threads(void) {
 #ifdef _OPENMP
     return omp_get_max_threads();

@@ -121,6 +121,12 @@ void lpmm_oracle_state_init(int64_t rows, int64_t cols, int kind, int64_t m_bloc
                             uint8_t* m_codes, float* m_scale, uint8_t* v_codes, float* v_s0, float* v_s1,
                             float* m32, float* v32);
 
+/* One compressed-SGDM step on one tensor (Alg. 2): m_t = beta * m_{t-1} + g ; w = w - lr * m_t ; compress m_t
+ * (block-wise normalization with block m_block, signed dynamic-exponent map). quantized != 0: m_codes / m_scale
+ * hold the state; else m32 (numel floats). Returns 0, or -1 on a bad argument. */
+int lpmm_oracle_sgdm4_step(float* w, const float* g, int64_t numel, int quantized, int64_t m_block,
+                           uint8_t* m_codes, float* m_scale, float* m32, float lr, float beta, int true_division);
+
 /* Number of OpenMP threads the loops above use (1 when built without OpenMP). */
 int lpmm_oracle_threads(void);
 void lpmm_oracle_set_threads(int n);

@@ -208,3 +208,24 @@ def adamw4_step(w, g, state: dict, *, lr, beta1, beta2, eps, weight_decay, step,
                                                               true_division=true_division)
         state["v_codes"] = pack4(qv)
     return w_new.astype(F32)
+
+
+def sgdm4_step(w, g, state: dict, *, lr, beta, true_division=False):
+    """Alg. 2 (compressed SGDM) on one tensor: m = beta m + g ; w = w - lr m ; compress m (B/DE)."""
+    numel = state["rows"] * state["cols"]
+    w = np.asarray(w, F32).ravel()
+    g = np.asarray(g, F32).ravel()
+    lr, beta = F32(lr), F32(beta)
+    Tde = de_map(4, True)
+    if state["kind"] == "fp32":
+        m = state["m32"]
+    else:
+        m = dequantize_block(unpack4(state["m_codes"], numel), state["m_block"], Tde, state["m_scale"])
+    mt = beta * m + g
+    w_new = w - lr * mt
+    if state["kind"] == "fp32":
+        state["m32"] = mt
+    else:
+        qm, state["m_scale"] = quantize_block(mt, state["m_block"], Tde, true_division=true_division)
+        state["m_codes"] = pack4(qm)
+    return w_new.astype(F32)

@@ -39,7 +39,7 @@ struct TensorLayout {
 
 struct Layout {
     std::vector<TensorLayout> t;
-    size_t descs = 0, params = 0, grads = 0, tiles1 = 0, tiles2 = 0;
+    size_t descs = 0, params = 0, grads = 0, tiles1 = 0, tiles2 = 0, tiles3 = 0;
     size_t rc[2] = {0, 0}, rcp = 0;
     int64_t rc_floats = 0;
     size_t total = 0;
@@ -88,6 +88,7 @@ void compute_layout(const lpmm_config& cfg, const lpmm_shape* shapes, int32_t n,
     L->grads = off;  off = align_up(off + sizeof(void*) * n);
     L->tiles1 = off; off = align_up(off + sizeof(int32_t) * (n + 1));
     L->tiles2 = off; off = align_up(off + sizeof(int32_t) * (n + 1));
+    L->tiles3 = off; off = align_up(off + sizeof(int32_t) * (n + 1));
     int64_t rc = 0;
     for (int32_t i = 0; i < n; ++i) {
         TensorLayout& t = L->t[i];
@@ -140,7 +141,7 @@ struct lpmm_state {
     std::vector<size_t> stage_off;
     int32_t pass2_variant;                 // 0 = register prefetch, 1 = bulk-copy staging
     int32_t sms, occ1, occ2;
-    std::vector<int32_t> tiles1, tiles2;   // host copies of the tile prefix sums
+    std::vector<int32_t> tiles1, tiles2, tiles3;   // host copies of the tile prefix sums (3: element-indexed tiles of every tensor)
     cudaStream_t copy_in, copy_out;        // lazily created by the host-buffer entry point
     std::vector<cudaEvent_t> host_events;
     bool profile;                          // record events around each kernel of a step
@@ -167,7 +168,7 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
     while (tile_elems * 2 <= target && tile_elems < 131072) tile_elems *= 2;
 
     std::vector<TensorDesc> descs(n);
-    std::vector<int32_t> t1(n + 1, 0), t2(n + 1, 0);
+    std::vector<int32_t> t1(n + 1, 0), t2(n + 1, 0), t3(n + 1, 0);
     char* A = st->arena;
     for (int32_t i = 0; i < n; ++i) {
         const TensorLayout& t = st->L.t[i];
@@ -198,12 +199,17 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
             d.tile_rows = (int32_t)tr;
             d.tiles_x = (int32_t)((t.cols + tile_cols - 1) / tile_cols);
             tiles = (int64_t)d.tiles_x * ((t.rows + tr - 1) / tr);
-        } else {
+        }
+        {   // element-indexed tiling: used by the non-tiled kinds in pass 2 and by every tensor in the SGDM step
             int64_t chunks = tile_elems / (kWarps * kWarpElems);
             if (chunks < 1) chunks = 1;
+            if (chunks > 16) chunks = 16;
             d.flat_chunks = (int32_t)chunks;
             const int64_t per_tile = chunks * kWarps * kWarpElems;
-            tiles = (t.numel + per_tile - 1) / per_tile;
+            const int64_t flat_tiles = (t.numel + per_tile - 1) / per_tile;
+            if (t.kind != K_RANK1_FAST) tiles = flat_tiles;
+            if (t3[i] + flat_tiles > 0x7fffffffLL) return LPMM_ERR_UNSUPPORTED;
+            t3[i + 1] = t3[i] + (int32_t)flat_tiles;
         }
         if (t2[i] + tiles > 0x7fffffffLL) return LPMM_ERR_UNSUPPORTED;
         t2[i + 1] = t2[i] + (int32_t)tiles;
@@ -217,6 +223,8 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
     st->sms = sms; st->occ1 = occ1; st->occ2 = occ2;
     st->tiles1 = t1;
     st->tiles2 = t2;
+    st->tiles3 = t3;
+    LPMM_CUDA(cudaMemcpyAsync(A + st->L.tiles3, t3.data(), sizeof(int32_t) * (n + 1), cudaMemcpyHostToDevice, s));
     LPMM_CUDA(cudaMemcpyAsync(A + st->L.descs, descs.data(), sizeof(TensorDesc) * n, cudaMemcpyHostToDevice, s));
     LPMM_CUDA(cudaMemcpyAsync(A + st->L.tiles1, t1.data(), sizeof(int32_t) * (n + 1), cudaMemcpyHostToDevice, s));
     LPMM_CUDA(cudaMemcpyAsync(A + st->L.tiles2, t2.data(), sizeof(int32_t) * (n + 1), cudaMemcpyHostToDevice, s));
@@ -428,6 +436,24 @@ lpmm_status lpmm_adamw4_step(lpmm_state* st, void* const* d_params, const void* 
     if (rc != LPMM_OK) return rc;
     st->phase ^= 1;
     st->last_launches = launches;
+    return LPMM_OK;
+}
+
+lpmm_status lpmm_sgdm4_step(lpmm_state* st, void* const* d_params, const void* const* d_grads,
+                            int32_t grad_dtype, float lr, float beta, void* stream) {
+    lpmm_status rc = check_step_args(st, d_params, d_grads, grad_dtype, lr, beta, 0.0f, 0.0f, 0.0f, 1);
+    if (rc != LPMM_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    rc = set_pointers(st, d_params, d_grads, s);
+    if (rc != LPMM_OK) return rc;
+    StepArgs a = make_args(st, lr, beta, 0.0f, 0.0f, 0.0f, 1);
+    a.h2.neg_step = make_float2(-lr, -lr);
+    a.tile_start = reinterpret_cast<const int32_t*>(st->arena + st->L.tiles3);
+    a.tile_begin = 0;
+    a.tile_end = st->tiles3[st->n];
+    const int32_t cap = st->sms * 3;
+    LPMM_CUDA(launch_sgdm(a, grad_dtype == LPMM_BF16, a.tile_end < cap ? a.tile_end : cap, s));
+    st->last_launches = 1;
     return LPMM_OK;
 }
 

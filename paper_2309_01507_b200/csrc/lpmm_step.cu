@@ -901,6 +901,73 @@ __global__ void __launch_bounds__(kThreads, 3) pass1_kernel(StepArgs a) {
     }
 }
 
+// ---- compressed SGDM (Alg. 2): m = beta m + g ; w = w - lr m ; compress m. One pass, element-indexed -------
+
+template <bool BF16>
+__global__ void __launch_bounds__(kThreads, 3) sgdm_kernel(StepArgs a) {
+    __shared__ __align__(16) unsigned char s_lut[kLutSmemBytes];
+    __shared__ float s_red[2 * kWarps];
+    load_lut_smem(s_lut);
+    __syncthreads();
+    const LaneTables lt = make_lane_tables();
+    const Hyper2& h2 = a.h2;          // beta1 = momentum, neg_step = -lr, one = 1
+    uint32_t red_step = 0;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int tile = a.tile_begin + blockIdx.x; tile < a.tile_end; tile += gridDim.x) {
+        const int t = find_tensor(a.tile_start, a.n_tensors, tile);
+        const TensorDesc d = a.descs[t];
+        float* w = a.params[t];
+        const void* g = a.grads[t];
+        const int local = tile - __ldg(a.tile_start + t);
+        const int64_t m_mask = ((int64_t)1 << d.m_shift) - 1;
+        for (int c = 0; c < d.flat_chunks; ++c) {
+            const int64_t chunk0 = ((int64_t)local * d.flat_chunks + c) * kWarps;
+            const int64_t chunk = chunk0 + warp;
+            const int64_t e = chunk * kWarpElems + lane * kLaneElems;
+            if (chunk0 * kWarpElems >= d.numel) break;                               // uniform over the CTA
+            const bool quant = d.kind != K_FP32;
+            if (!(quant && d.m_shift == 11) && chunk * kWarpElems >= d.numel) break;  // B2048 warps stay for the barrier
+            const bool full = (chunk + 1) * kWarpElems <= d.numel;
+            float wv[8], gv[8], mo[8];
+            uint32_t qm = 0;
+            if (full) { load8_rw(w + e, wv); load8_grad<BF16>(g, e, gv); }
+            else { load8_guard(w, e, d.numel, wv); load8_grad_guard<BF16>(g, e, d.numel, gv); }
+            if (quant) {
+                qm = full ? __ldg(reinterpret_cast<const uint32_t*>(d.m_codes + (e >> 1))) : load_codes_guard(d.m_codes, e, d.numel);
+                const bool group_live = (e & ~m_mask) < d.numel;
+                const float prod = __fmul_rn(lt.de, group_live ? d.m_scale[e >> d.m_shift] : 0.0f);
+#pragma unroll
+                for (int k = 0; k < 8; ++k) mo[k] = __shfl_sync(lt.mask, prod, (int)(qm >> (4 * k)), 16);
+            } else {
+                if (full) load8_rw(d.m32 + e, mo); else load8_guard(d.m32, e, d.numel, mo);
+            }
+            float mt[8];
+#pragma unroll
+            for (int k = 0; k < 8; k += 2) {
+                // fl(fl(beta m) + g) and fl(w + fl(-lr m_t)), each sum written as fma(p, 1, q) (see ema_m2)
+                const float2 m2 = fma2_rn(mul2_rn(h2.beta1, make_float2(mo[k], mo[k + 1])), h2.one, make_float2(gv[k], gv[k + 1]));
+                const float2 w2 = fma2_rn(mul2_rn(h2.neg_step, m2), h2.one, make_float2(wv[k], wv[k + 1]));
+                mt[k] = m2.x; mt[k + 1] = m2.y;
+                wv[k] = w2.x; wv[k + 1] = w2.y;
+            }
+            if (!full) {
+#pragma unroll
+                for (int k = 0; k < 8; ++k) if (e + k >= d.numel) mt[k] = 0.0f;
+            }
+            if (full) store8_f32(w + e, wv); else store8_guard(w, e, d.numel, wv);
+            if (quant) {
+                const float am_new = block_max(absmax8(mt), d.m_shift, lt, s_red, red_step);
+                if (e < d.numel && (threadIdx.x & (d.m_shift == 7 ? 15 : 2047)) == 0) d.m_scale[e >> d.m_shift] = am_new;
+                const uint32_t q_new = quantize8_de(mt, scale_rcp(am_new), s_lut);
+                if (full) *reinterpret_cast<uint32_t*>(d.m_codes + (e >> 1)) = q_new;
+                else store_codes_guard(d.m_codes, e, d.numel, q_new);
+            } else {
+                if (full) store8_f32(d.m32 + e, mt); else store8_guard(d.m32, e, d.numel, mt);
+            }
+        }
+    }
+}
+
 __global__ void rcp_kernel(const float* __restrict__ src, float* __restrict__ dst, int64_t n) {
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
         dst[i] = scale_rcp(src[i]);
@@ -937,6 +1004,13 @@ cudaError_t launch_pass2(const StepArgs& a, bool bf16, bool exact, int grid, cud
         if (exact) pass2_kernel<false, true><<<grid, kThreads, 0, s>>>(a);
         else pass2_kernel<false, false><<<grid, kThreads, 0, s>>>(a);
     }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_sgdm(const StepArgs& a, bool bf16, int grid, cudaStream_t s) {
+    if (a.tile_end <= a.tile_begin) return cudaSuccess;
+    if (bf16) sgdm_kernel<true><<<grid, kThreads, 0, s>>>(a);
+    else sgdm_kernel<false><<<grid, kThreads, 0, s>>>(a);
     return cudaGetLastError();
 }
 

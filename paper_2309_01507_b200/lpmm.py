@@ -28,7 +28,7 @@ KIND_FP32, KIND_BLOCK, KIND_RANK1 = 0, 1, 2
 
 EXPORTS = ("lpmm_state_bytes", "lpmm_state_init", "lpmm_state_attach", "lpmm_adamw4_step",
            "lpmm_adamw4_step_host", "lpmm_stage_bytes", "lpmm_quantize", "lpmm_dequantize",
-           "lpmm_quantize_rank1_noalloc",
+           "lpmm_quantize_rank1_noalloc", "lpmm_sgdm4_step",
            "lpmm_state_view", "lpmm_state_phase", "lpmm_state_last_launches", "lpmm_state_destroy",
            "lpmm_state_profile", "lpmm_state_profile_read", "lpmm_state_device_status",
            "lpmm_status_string", "lpmm_last_cuda_error")
@@ -74,6 +74,7 @@ def lib():
         L.lpmm_adamw4_step.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), i32, f32, f32, f32, f32, f32, i64, vp]
         L.lpmm_adamw4_step_host.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), i32, f32, f32, f32, f32, f32, i64,
                                             vp, vp, C.c_size_t, vp]
+        L.lpmm_sgdm4_step.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), i32, f32, f32, vp]
         L.lpmm_stage_bytes.argtypes = [vp, C.POINTER(C.c_size_t)]
         L.lpmm_quantize.argtypes = [vp, i64, i64, i32, i32, i32, u32, vp, vp, vp, vp]
         L.lpmm_dequantize.argtypes = [vp, vp, vp, i64, i64, i32, i32, i32, vp, vp]
@@ -207,6 +208,14 @@ def adamw4_step(state: State, params, grads, *, lr, beta1, beta2, eps, weight_de
         pp, gp, gd = ptr_cache
     _check(lib().lpmm_adamw4_step(state.handle, pp, gp, gd, lr, beta1, beta2, eps, weight_decay, step,
                                   _stream_ptr(stream)), "lpmm_adamw4_step")
+
+
+def sgdm4_step(state: State, params, grads, *, lr, beta, stream=None) -> None:
+    """lpmm_sgdm4_step: compressed SGDM (Alg. 2) on lists of contiguous CUDA tensors."""
+    if len(params) != state.n or len(grads) != state.n:
+        raise ValueError("params/grads must have one tensor per state entry")
+    _check(lib().lpmm_sgdm4_step(state.handle, _ptr_array(params), _ptr_array(grads), _grad_dtype(grads), lr, beta,
+                                 _stream_ptr(stream)), "lpmm_sgdm4_step")
 
 
 def make_ptr_cache(params, grads):

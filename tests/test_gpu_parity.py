@@ -262,3 +262,28 @@ def test_argument_errors_do_not_launch():
     assert ei.value.status == lpmm.ERR_UNSUPPORTED
     torch.cuda.synchronize()
     assert torch.count_nonzero(p) == 0
+
+
+@pytest.mark.parametrize("grad_dtype,m_block", [(torch.float32, 128), (torch.bfloat16, 128), (torch.float32, 2048)])
+def test_sgdm_step_matches_oracle_bit_for_bit(grad_dtype, m_block):
+    # Alg. 2 (compressed SGDM): the first moment in 4 bits, parameters in the algorithm's own operation order.
+    cfg = lpmm.default_config(m_block=m_block)
+    specs = [_mat(96, 256), _mat(33, 77), _mat(130, 384), _mat(64, 2048), _vec(50265), _vec(4097), _vec(300), _vec(1)]
+    params = [workloads.make_param(s, 12, i, device="cuda") for i, s in enumerate(specs)]
+    state = lpmm.state_init(cfg, specs)
+    w_ref = [p.cpu().numpy().ravel().copy() for p in params]
+    ost = [oracle.state_init(s.rows, s.cols, oracle.FP32 if lpmm.state_view(state, i)["kind"] == lpmm.KIND_FP32 else oracle.BLOCK,
+                             m_block=m_block) for i, s in enumerate(specs)]
+    for t in range(1, 6):
+        grads = [workloads.make_grad(s, 12, i, t, device="cuda", dtype=grad_dtype) for i, s in enumerate(specs)]
+        lpmm.sgdm4_step(state, params, grads, lr=0.01, beta=0.9)
+        torch.cuda.synchronize()
+        for i, s in enumerate(specs):
+            oracle.sgdm4_step(w_ref[i], grads[i].float().cpu().numpy().ravel(), ost[i], lr=0.01, beta=0.9)
+            view = lpmm.state_view(state, i)
+            for name in ("m_codes", "m_scale", "m32"):
+                ref = getattr(ost[i], name)
+                if ref is not None:
+                    assert np.array_equal(view[name].cpu().numpy(), ref), (s.name, name, t)
+            assert np.array_equal(params[i].cpu().numpy().ravel(), w_ref[i]), (s.name, t)
+    assert state.last_launches == 1
