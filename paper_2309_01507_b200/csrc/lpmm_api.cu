@@ -403,7 +403,7 @@ lpmm_status enqueue_range(lpmm_state* st, StepArgs a, int32_t t0, int32_t t1, bo
     a.tile_begin = st->tiles2[t0];
     a.tile_end = st->tiles2[t1];
     const int32_t cap = st->sms * st->occ2, tiles = a.tile_end - a.tile_begin;
-    LPMM_CUDA(launch_pass2(a, bf16, ieee_update, tiles < cap ? tiles : cap, s));
+    LPMM_CUDA(launch_pass2(a, bf16, ieee_update, st->cfg.m_block == 2048 ? 11 : 7, tiles < cap ? tiles : cap, s));
     if (ev) LPMM_CUDA(cudaEventRecord(ev[3], s));
     *launches += 1;
     return LPMM_OK;

@@ -54,7 +54,7 @@ struct StepArgs {
 };
 
 cudaError_t launch_pass1(const StepArgs& a, bool bf16, int grid, cudaStream_t s);
-cudaError_t launch_pass2(const StepArgs& a, bool bf16, bool exact, int grid, cudaStream_t s);
+cudaError_t launch_pass2(const StepArgs& a, bool bf16, bool exact, int m_shift, int grid, cudaStream_t s);
 cudaError_t launch_sgdm(const StepArgs& a, bool bf16, int grid, cudaStream_t s);
 cudaError_t launch_rcp(const float* src, float* dst, int64_t n, cudaStream_t s);
 cudaError_t step_kernel_occupancy(int* pass1_blocks_per_sm, int* pass2_blocks_per_sm);

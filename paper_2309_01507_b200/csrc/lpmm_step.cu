@@ -248,7 +248,7 @@ struct TileView {
 constexpr uint32_t kL2Ahead = 4;   // rows
 __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
-template <bool BF16>
+template <bool BF16, int MSHIFT>
 __device__ __forceinline__ void prefetch_row(const TileView& t, uint32_t k) {
     const uint32_t off = k * t.row_step;
     prefetch_l2(t.w + off);
@@ -259,10 +259,10 @@ __device__ __forceinline__ void prefetch_row(const TileView& t, uint32_t k) {
     }
     prefetch_l2(t.m_codes + (off >> 1));
     prefetch_l2(t.v_codes + (off >> 1));
-    prefetch_l2(t.m_scale + (off >> t.m_shift));
+    prefetch_l2(t.m_scale + (off >> MSHIFT));
 }
 
-template <bool BF16>
+template <bool BF16, int MSHIFT>
 __device__ __forceinline__ void load_row(RowRegs<BF16>& r, const TileView& t, uint32_t k) {
     const uint32_t off = k * t.row_step;
     r.w0 = *reinterpret_cast<const float4*>(t.w + off);
@@ -275,12 +275,12 @@ __device__ __forceinline__ void load_row(RowRegs<BF16>& r, const TileView& t, ui
     }
     r.qm = *reinterpret_cast<const uint32_t*>(t.m_codes + (off >> 1));
     r.qv = *reinterpret_cast<const uint32_t*>(t.v_codes + (off >> 1));
-    r.am = t.m_scale[off >> t.m_shift];
+    r.am = t.m_scale[off >> MSHIFT];
     r.r_old = __ldg(t.r_old + k * t.row_stride);
     r.r_rcp = __ldg(t.r_rcp + k * t.row_stride);
 }
 
-template <bool BF16, bool EXACT>
+template <bool BF16, bool EXACT, int MSHIFT>
 __device__ __forceinline__ void process_row(const RowRegs<BF16>& r, const TileView& t, uint32_t k,
                                             const float (&c_old)[8], const float (&c_rcp)[8], const Hyper& h,
                                             const Hyper2& h2, const LaneTables& lt, const unsigned char* s_lut) {
@@ -295,13 +295,13 @@ __device__ __forceinline__ void process_row(const RowRegs<BF16>& r, const TileVi
     }
     moments_and_update8<EXACT>(wv, gv, r.qm, r.qv, __fmul_rn(lt.de, r.am), vs, h, h2, lt, mt, vt);
     store8_f32(t.w + off, wv);
-    const float am_new = block_max(absmax8(mt), t.m_shift, lt, t.s_red, *t.red_step);
-    if ((threadIdx.x & (t.m_shift == 7 ? 15 : 2047)) == 0) t.m_scale[off >> t.m_shift] = am_new;
+    const float am_new = block_max(absmax8(mt), MSHIFT, lt, t.s_red, *t.red_step);
+    if ((threadIdx.x & (MSHIFT == 7 ? 15 : 2047)) == 0) t.m_scale[off >> MSHIFT] = am_new;
     *reinterpret_cast<uint32_t*>(t.m_codes + (off >> 1)) = quantize8_de(mt, scale_rcp(am_new), s_lut);
     *reinterpret_cast<uint32_t*>(t.v_codes + (off >> 1)) = quantize8_lin(vt, vr, h2);
 }
 
-template <bool BF16, bool EXACT>
+template <bool BF16, bool EXACT, int MSHIFT>
 __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __restrict__ w, const void* __restrict__ g,
                                                  int tile, int phase, const Hyper& h, const Hyper2& h2,
                                                  const LaneTables& lt, const unsigned char* s_lut, float* s_red,
@@ -330,7 +330,7 @@ __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __r
                : static_cast<const void*>(reinterpret_cast<const float*>(g) + e0);
     t.m_codes = d.m_codes + (e0 >> 1);
     t.v_codes = d.v_codes + (e0 >> 1);
-    t.m_scale = d.m_scale + (e0 >> d.m_shift);
+    t.m_scale = d.m_scale + (e0 >> MSHIFT);
     t.r_old = rc_old + row0;
     t.r_rcp = rcp_new + row0;
     t.row_step = (uint32_t)(wy_count * d.cols);
@@ -342,17 +342,17 @@ __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __r
     // Two register sets alternate: while one row is processed the next one is already in flight.
     RowRegs<BF16> ra, rb;
 #pragma unroll
-    for (uint32_t k = 1; k < kL2Ahead; ++k) if (k < nrows) prefetch_row<BF16>(t, k);
-    load_row<BF16>(ra, t, 0);
+    for (uint32_t k = 1; k < kL2Ahead; ++k) if (k < nrows) prefetch_row<BF16, MSHIFT>(t, k);
+    load_row<BF16, MSHIFT>(ra, t, 0);
     for (uint32_t k = 0; k < nrows; k += 2) {
         const bool has_b = k + 1 < nrows;
-        if (k + kL2Ahead < nrows) prefetch_row<BF16>(t, k + kL2Ahead);
-        if (has_b) load_row<BF16>(rb, t, k + 1);
-        process_row<BF16, EXACT>(ra, t, k, c_old, c_rcp, h, h2, lt, s_lut);
+        if (k + kL2Ahead < nrows) prefetch_row<BF16, MSHIFT>(t, k + kL2Ahead);
+        if (has_b) load_row<BF16, MSHIFT>(rb, t, k + 1);
+        process_row<BF16, EXACT, MSHIFT>(ra, t, k, c_old, c_rcp, h, h2, lt, s_lut);
         if (!has_b) break;
-        if (k + 1 + kL2Ahead < nrows) prefetch_row<BF16>(t, k + 1 + kL2Ahead);
-        if (k + 2 < nrows) load_row<BF16>(ra, t, k + 2);
-        process_row<BF16, EXACT>(rb, t, k + 1, c_old, c_rcp, h, h2, lt, s_lut);
+        if (k + 1 + kL2Ahead < nrows) prefetch_row<BF16, MSHIFT>(t, k + 1 + kL2Ahead);
+        if (k + 2 < nrows) load_row<BF16, MSHIFT>(ra, t, k + 2);
+        process_row<BF16, EXACT, MSHIFT>(rb, t, k + 1, c_old, c_rcp, h, h2, lt, s_lut);
     }
 }
 
@@ -531,14 +531,14 @@ __device__ __forceinline__ void pass2_rank1_bulk(const TensorDesc& d, float* __r
 
 // ---- pass 2, flat (element-indexed) tensors: block-wise v, or rank-1 with arbitrary cols ------
 
-template <bool BF16, bool RANK1, bool EXACT>
+template <bool BF16, bool RANK1, bool EXACT, int MSHIFT>
 __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restrict__ w, const void* __restrict__ g,
                                            int tile, int phase, const Hyper& h, const Hyper2& h2, const LaneTables& lt,
                                            const unsigned char* s_lut, float* s_red, uint32_t& red_step) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const float* rc_old = (phase ? d.rc[1] : d.rc[0]);
     const float* rcp_new = d.rcp_new;
-    const int64_t m_mask = ((int64_t)1 << d.m_shift) - 1;
+    const int64_t m_mask = ((int64_t)1 << MSHIFT) - 1;
     for (int c = 0; c < d.flat_chunks; ++c) {
         const int64_t chunk0 = ((int64_t)tile * d.flat_chunks + c) * kWarps;   // the CTA's 8 chunks = 2048 elements
         const int64_t chunk = chunk0 + warp;
@@ -546,7 +546,7 @@ __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restric
         if (chunk0 * kWarpElems >= d.numel) break;          // uniform over the CTA
         // B128: a warp past the end has nothing to do. B2048: it still joins the CTA-wide block maximum
         // (with zeros; its loads and stores are all guarded away).
-        if (d.m_shift == 7 && chunk * kWarpElems >= d.numel) break;
+        if (MSHIFT == 7 && chunk * kWarpElems >= d.numel) break;
         const bool full = (chunk + 1) * kWarpElems <= d.numel;
         float wv[8], gv[8], mt[8], vt[8], vs[8], vr[8];
         uint32_t qm, qv;
@@ -565,7 +565,7 @@ __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restric
         // every lane of a 16-lane group that still holds an element needs the block's scale: the
         // shuffle-based table lookup reads T[q] * scale from the group's other lanes
         const bool group_live = (e & ~m_mask) < d.numel;
-        const float am = group_live ? d.m_scale[e >> d.m_shift] : 0.0f;
+        const float am = group_live ? d.m_scale[e >> MSHIFT] : 0.0f;
         if (RANK1) {
             int64_t i = e / d.cols, j = e - i * d.cols;
 #pragma unroll
@@ -588,7 +588,7 @@ __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restric
 #pragma unroll
             for (int k = 0; k < 8; ++k) if (e + k >= d.numel) { mt[k] = 0.0f; vt[k] = 0.0f; }
         }
-        const float am_new = block_max(absmax8(mt), d.m_shift, lt, s_red, red_step);
+        const float am_new = block_max(absmax8(mt), MSHIFT, lt, s_red, red_step);
         if (!RANK1) {
             const float av_new = half_warp_max(absmax8(vt));
             const float r = scale_rcp(av_new);
@@ -596,7 +596,7 @@ __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restric
             for (int k = 0; k < 8; ++k) vr[k] = r;
             if (lane_live && (lane & 15) == 0) d.v_bscale[e >> 7] = av_new;
         }
-        if (lane_live && (threadIdx.x & (d.m_shift == 7 ? 15 : 2047)) == 0) d.m_scale[e >> d.m_shift] = am_new;
+        if (lane_live && (threadIdx.x & (MSHIFT == 7 ? 15 : 2047)) == 0) d.m_scale[e >> MSHIFT] = am_new;
         const uint32_t qm_new = quantize8_de(mt, scale_rcp(am_new), s_lut);
         const uint32_t qv_new = quantize8_lin(vt, vr, h2);
         if (full) {
@@ -643,7 +643,7 @@ __device__ __forceinline__ void pass2_fp32(const TensorDesc& d, float* __restric
     }
 }
 
-template <bool BF16, bool EXACT>
+template <bool BF16, bool EXACT, int MSHIFT>
 __global__ void __launch_bounds__(kThreads, 2) pass2_kernel(StepArgs a) {
     __shared__ __align__(16) unsigned char s_lut[kLutSmemBytes];
     __shared__ float s_red[2 * kWarps];
@@ -659,15 +659,15 @@ __global__ void __launch_bounds__(kThreads, 2) pass2_kernel(StepArgs a) {
         const void* g = a.grads[t];
         const int local = tile - __ldg(a.tile_start + t);
         switch (d.kind) {
-            case K_RANK1_FAST: pass2_rank1_fast<BF16, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
-            case K_RANK1_FLAT: pass2_flat<BF16, true, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
-            case K_BLOCK:      pass2_flat<BF16, false, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
+            case K_RANK1_FAST: pass2_rank1_fast<BF16, EXACT, MSHIFT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
+            case K_RANK1_FLAT: pass2_flat<BF16, true, EXACT, MSHIFT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
+            case K_BLOCK:      pass2_flat<BF16, false, EXACT, MSHIFT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
             default:           pass2_fp32<BF16, EXACT>(d, w, g, local, a.h); break;
         }
     }
 }
 
-template <bool BF16, bool EXACT>
+template <bool BF16, bool EXACT, int MSHIFT>
 __global__ void __launch_bounds__(kThreads, 2) pass2_bulk_kernel(StepArgs a) {
     extern __shared__ __align__(128) unsigned char s_dyn[];   // [nearest-entry table | warp rings | mbarriers]
     unsigned char* s_lut = s_dyn;
@@ -696,11 +696,11 @@ __global__ void __launch_bounds__(kThreads, 2) pass2_bulk_kernel(StepArgs a) {
         const int local = tile - __ldg(a.tile_start + t);
         switch (d.kind) {
             case K_RANK1_FAST:
-                if ((d.cols & 255) == 0 && d.m_shift == 7) pass2_rank1_bulk<BF16, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, ring, a.dev_status);
-                else pass2_rank1_fast<BF16, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step);
+                if ((d.cols & 255) == 0 && MSHIFT == 7) pass2_rank1_bulk<BF16, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, ring, a.dev_status);
+                else pass2_rank1_fast<BF16, EXACT, MSHIFT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step);
                 break;
-            case K_RANK1_FLAT: pass2_flat<BF16, true, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
-            case K_BLOCK:      pass2_flat<BF16, false, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
+            case K_RANK1_FLAT: pass2_flat<BF16, true, EXACT, MSHIFT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
+            case K_BLOCK:      pass2_flat<BF16, false, EXACT, MSHIFT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
             default:           pass2_fp32<BF16, EXACT>(d, w, g, local, a.h); break;
         }
     }
@@ -982,29 +982,28 @@ cudaError_t launch_pass1(const StepArgs& a, bool bf16, int grid, cudaStream_t s)
     return cudaGetLastError();
 }
 
-template <bool BF16, bool EXACT>
-cudaError_t launch_pass2_bulk_t(const StepArgs& a, int grid, cudaStream_t s) {
-    constexpr int smem = bulk_smem_bytes<BF16>();
-    cudaError_t e = cudaFuncSetAttribute(pass2_bulk_kernel<BF16, EXACT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) return e;
-    pass2_bulk_kernel<BF16, EXACT><<<grid, kThreads, smem, s>>>(a);
+template <bool BF16, bool EXACT, int MSHIFT>
+cudaError_t launch_pass2_t(const StepArgs& a, int grid, cudaStream_t s) {
+    if (a.variant == 1) {
+        constexpr int smem = bulk_smem_bytes<BF16>();
+        cudaError_t e = cudaFuncSetAttribute(pass2_bulk_kernel<BF16, EXACT, MSHIFT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        pass2_bulk_kernel<BF16, EXACT, MSHIFT><<<grid, kThreads, smem, s>>>(a);
+    } else {
+        pass2_kernel<BF16, EXACT, MSHIFT><<<grid, kThreads, 0, s>>>(a);
+    }
     return cudaGetLastError();
 }
 
-cudaError_t launch_pass2(const StepArgs& a, bool bf16, bool exact, int grid, cudaStream_t s) {
+template <bool BF16, bool EXACT>
+cudaError_t launch_pass2_m(const StepArgs& a, int m_shift, int grid, cudaStream_t s) {
+    return m_shift == 11 ? launch_pass2_t<BF16, EXACT, 11>(a, grid, s) : launch_pass2_t<BF16, EXACT, 7>(a, grid, s);
+}
+
+cudaError_t launch_pass2(const StepArgs& a, bool bf16, bool exact, int m_shift, int grid, cudaStream_t s) {
     if (a.tile_end <= a.tile_begin) return cudaSuccess;
-    if (a.variant == 1) {
-        if (bf16) return exact ? launch_pass2_bulk_t<true, true>(a, grid, s) : launch_pass2_bulk_t<true, false>(a, grid, s);
-        return exact ? launch_pass2_bulk_t<false, true>(a, grid, s) : launch_pass2_bulk_t<false, false>(a, grid, s);
-    }
-    if (bf16) {
-        if (exact) pass2_kernel<true, true><<<grid, kThreads, 0, s>>>(a);
-        else pass2_kernel<true, false><<<grid, kThreads, 0, s>>>(a);
-    } else {
-        if (exact) pass2_kernel<false, true><<<grid, kThreads, 0, s>>>(a);
-        else pass2_kernel<false, false><<<grid, kThreads, 0, s>>>(a);
-    }
-    return cudaGetLastError();
+    if (bf16) return exact ? launch_pass2_m<true, true>(a, m_shift, grid, s) : launch_pass2_m<true, false>(a, m_shift, grid, s);
+    return exact ? launch_pass2_m<false, true>(a, m_shift, grid, s) : launch_pass2_m<false, false>(a, m_shift, grid, s);
 }
 
 cudaError_t launch_sgdm(const StepArgs& a, bool bf16, int grid, cudaStream_t s) {
@@ -1025,7 +1024,7 @@ cudaError_t launch_rcp(const float* src, float* dst, int64_t n, cudaStream_t s) 
 cudaError_t step_kernel_occupancy(int* p1, int* p2) {
     cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(p1, pass1_kernel<true>, kThreads, 0);
     if (e != cudaSuccess) return e;
-    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(p2, pass2_kernel<true, false>, kThreads, 0);
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(p2, pass2_kernel<true, false, 7>, kThreads, 0);
 }
 
 }  // namespace lpmm
