@@ -246,3 +246,16 @@ def sgdm4_step(w: np.ndarray, g: np.ndarray, st: TensorState, *, lr, beta, true_
                                       C.c_float(lr), C.c_float(beta), C.c_int(int(true_division)))
     if rc != 0:
         raise ValueError("lpmm_oracle_sgdm4_step rejected its arguments")
+
+
+def adamw4_factor_step(w: np.ndarray, g: np.ndarray, st: TensorState, R: np.ndarray, C_: np.ndarray, *, lr, beta1,
+                       beta2, eps, weight_decay, step: int) -> None:
+    """One step of the factorized-second-moment variant on a matrix; w, the m part of `st`, R and C_ change in place."""
+    assert w.dtype == np.float32 and w.size == st.numel and R.dtype == np.float32 and C_.dtype == np.float32
+    assert R.size == st.rows and C_.size == st.cols
+    g = _f32(g)
+    h = _Hyper(lr, beta1, beta2, eps, weight_decay, step, 0)
+    rc = lib().lpmm_oracle_adamw4_factor_step(_p(w), _p(g), C.c_int64(st.rows), C.c_int64(st.cols), C.c_int64(st.m_block),
+                                              _p(st.m_codes), _p(st.m_scale), _p(R), _p(C_), C.byref(h))
+    if rc != 0:
+        raise ValueError("lpmm_oracle_adamw4_factor_step rejected its arguments")

@@ -350,6 +350,73 @@ int lpmm_oracle_adamw4_step(float* w, const float* g, int64_t rows, int64_t cols
     return 0;
 }
 
+/* ------------------------------------------------------------------ factorized second moment (Sec. 4.3) */
+
+int lpmm_oracle_adamw4_factor_step(float* w, const float* g, int64_t rows, int64_t cols, int64_t m_block,
+                                   uint8_t* m_codes, float* m_scale, float* R, float* C,
+                                   const lpmm_oracle_hyper* h) {
+    if (!w || !g || !h || !R || !C || rows <= 0 || cols <= 0 || h->step < 1) return -1;
+    const int64_t numel = rows * cols;
+    const float beta1 = h->beta1, beta2 = h->beta2;
+    const float omb1 = 1.0f - beta1, omb2 = 1.0f - beta2;
+    const float bc1 = (float)(1.0 - pow((double)beta1, (double)h->step));
+    const float bc2 = (float)(1.0 - pow((double)beta2, (double)h->step));
+    const float decay = 1.0f - h->lr * h->weight_decay;
+    float* m = (float*)malloc(sizeof(float) * (size_t)numel);
+    uint8_t* q = (uint8_t*)malloc((size_t)numel);
+    double* cs = (double*)calloc((size_t)cols, sizeof(double));
+    if (!m || !q || !cs) { free(m); free(q); free(cs); return -1; }
+    float Tde[16];
+    lpmm_oracle_de_map(4, 1, 0, Tde);
+    lpmm_oracle_unpack4(m_codes, numel, q);
+    lpmm_oracle_dequantize_block(q, numel, m_block, Tde, m_scale, m);
+
+    /* row and column sums of the squared gradient, then the statistics' moving averages */
+    for (int64_t i = 0; i < rows; ++i) {
+        double rs = 0.0;
+        for (int64_t j = 0; j < cols; ++j) {
+            float gg = g[i * cols + j] * g[i * cols + j];
+            rs += (double)gg;
+            cs[j] += (double)gg;
+        }
+        float a = beta2 * R[i];
+        float b = omb2 * (float)rs;
+        R[i] = a + b;
+    }
+    double total = 0.0;
+    for (int64_t i = 0; i < rows; ++i) total += (double)R[i];
+    for (int64_t j = 0; j < cols; ++j) {
+        float a = beta2 * C[j];
+        float b = omb2 * (float)cs[j];
+        C[j] = a + b;
+    }
+    const float rS = lpmm_oracle_rcp((float)total);
+
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < rows; ++i) {
+        const float ai = R[i] * rS;
+        for (int64_t j = 0; j < cols; ++j) {
+            const int64_t e = i * cols + j;
+            float gi = g[e];
+            float x = beta1 * m[e];
+            float y = omb1 * gi;
+            float mt = x + y;
+            float vt = ai * C[j];
+            float mhat = mt / bc1;
+            float vhat = vt / bc2;
+            float denom = sqrtf(vhat) + h->eps;
+            float upd = h->lr * (mhat / denom);
+            float wd = w[e] * decay;
+            w[e] = wd - upd;
+            m[e] = mt;
+        }
+    }
+    lpmm_oracle_quantize_block(m, numel, m_block, Tde, 16, 0, h->true_division, m_scale, q);
+    lpmm_oracle_pack4(q, numel, m_codes);
+    free(m); free(q); free(cs);
+    return 0;
+}
+
 /* ------------------------------------------------------------------ the compressed SGDM step (Alg. 2) */
 
 int lpmm_oracle_sgdm4_step(float* w, const float* g, int64_t numel, int quantized, int64_t m_block,

@@ -121,6 +121,18 @@ void lpmm_oracle_state_init(int64_t rows, int64_t cols, int kind, int64_t m_bloc
                             uint8_t* m_codes, float* m_scale, uint8_t* v_codes, float* v_s0, float* v_s1,
                             float* m32, float* v32);
 
+/* One step of the factorized variant ("4-bit Factor", Sec. 4.3 and Sec. 5) on one rows x cols matrix: the first
+ * moment is compressed as in lpmm_oracle_adamw4_step; the second moment is replaced by Adafactor's rank-1
+ * reconstruction from fp32 row and column statistics. The paper gives no formula; the reading is:
+ *   rs_i = sum_j g_ij^2, cs_j = sum_i g_ij^2   (squares in binary32, sums accumulated in binary64, rounded once)
+ *   R <- beta2 R + (1 - beta2) rs ; C <- beta2 C + (1 - beta2) cs            (binary32, R_0 = C_0 = 0)
+ *   v_ij = (R_i * (1 / sum_k R_k)) * C_j    (sum in binary64, rounded once; 0 when the sum is below FLT_MIN)
+ * followed by Eq. 1's bias correction and update with this v (no update clipping, no relative step size).
+ * Parity unpinned beyond the invariants tested in tests/test_oracle_factor.py. Returns 0 or -1. */
+int lpmm_oracle_adamw4_factor_step(float* w, const float* g, int64_t rows, int64_t cols, int64_t m_block,
+                                   uint8_t* m_codes, float* m_scale, float* R, float* C,
+                                   const lpmm_oracle_hyper* h);
+
 /* One compressed-SGDM step on one tensor (Alg. 2): m_t = beta * m_{t-1} + g ; w = w - lr * m_t ; compress m_t
  * (block-wise normalization with block m_block, signed dynamic-exponent map). quantized != 0: m_codes / m_scale
  * hold the state; else m32 (numel floats). Returns 0, or -1 on a bad argument. */

@@ -229,3 +229,35 @@ def sgdm4_step(w, g, state: dict, *, lr, beta, true_division=False):
         qm, state["m_scale"] = quantize_block(mt, state["m_block"], Tde, true_division=true_division)
         state["m_codes"] = pack4(qm)
     return w_new.astype(F32)
+
+
+def adamw4_factor_step(w, g, state: dict, *, lr, beta1, beta2, eps, weight_decay, step):
+    """Factorized second moment (Sec. 4.3, Adafactor's rank-1 reconstruction) with a 4-bit first moment.
+
+    state: {"rows", "cols", "m_block", "m_codes", "m_scale", "R", "C"}; returns the new w (flat float32).
+    """
+    rows, cols = state["rows"], state["cols"]
+    numel = rows * cols
+    w = np.asarray(w, F32).ravel()
+    g = np.asarray(g, F32).reshape(rows, cols)
+    lr, beta1, beta2, eps, wd = F32(lr), F32(beta1), F32(beta2), F32(eps), F32(weight_decay)
+    Tde = de_map(4, True)
+    m = dequantize_block(unpack4(state["m_codes"], numel), state["m_block"], Tde, state["m_scale"])
+    omb1, omb2 = F32(1.0) - beta1, F32(1.0) - beta2
+    bc1 = F32(1.0 - float(beta1) ** step)
+    bc2 = F32(1.0 - float(beta2) ** step)
+    gg = (g * g).astype(np.float64)
+    rs = gg.sum(axis=1).astype(F32)
+    cs = gg.sum(axis=0).astype(F32)
+    R = beta2 * state["R"] + omb2 * rs
+    Cc = beta2 * state["C"] + omb2 * cs
+    total = F32(R.astype(np.float64).sum())
+    rS = rcp(np.array([total], F32))[0]
+    vt = ((R * rS)[:, None] * Cc[None, :]).astype(F32).ravel()
+    mt = beta1 * m + omb1 * g.ravel()
+    upd = lr * ((mt / bc1) / (np.sqrt(vt / bc2) + eps))
+    w_new = w * (F32(1.0) - lr * wd) - upd
+    qm, state["m_scale"] = quantize_block(mt, state["m_block"], Tde)
+    state["m_codes"] = pack4(qm)
+    state["R"], state["C"] = R.astype(F32), Cc.astype(F32)
+    return w_new.astype(F32)
