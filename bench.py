@@ -50,7 +50,8 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--m-block", type=int, default=128, choices=[128, 2048], help="first-moment block size")
-    ap.add_argument("--v-mode", default="rank1", choices=["rank1", "block"], help="second-moment normalizer of matrices")
+    ap.add_argument("--v-mode", default="rank1", choices=["rank1", "block", "factored"],
+                    help="second moment of matrices: rank-1 or block-wise 4-bit, or factorized (fp32 row/column statistics)")
     return ap.parse_args()
 
 
@@ -210,7 +211,8 @@ def run_ours(args):
     hyper = dict(lr=wl.lr, beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps, weight_decay=wl.weight_decay)
     params = [workloads.make_param(t, wl.index, i, device=dev) for i, t in enumerate(wl.tensors)]
     grads = [workloads.make_grad(t, wl.index, i, 1, device=dev, dtype=gdt) for i, t in enumerate(wl.tensors)]
-    cfg = lpmm.default_config(m_block=args.m_block, v_mode=lpmm.V_BLOCK if args.v_mode == "block" else lpmm.V_RANK1)
+    v_mode = {"rank1": lpmm.V_RANK1, "block": lpmm.V_BLOCK, "factored": lpmm.V_FACTORED}[args.v_mode]
+    cfg = lpmm.default_config(m_block=args.m_block, v_mode=v_mode)
     state = lpmm.state_init(cfg, wl.tensors, device=dev)
     cache = lpmm.make_ptr_cache(params, grads)
     n_params = wl.numel
@@ -291,6 +293,9 @@ def run_ours(args):
     p1_ms = prof["pass1_ms"] / max(prof["steps"], 1)
     # block maxima: 8 bytes per block of m (and of v when v is block-wise; then pass 1 has nothing to do)
     pass2_bpp = PASS2_BYTES[wl.grad_dtype] - 8 / 128 + 8 / args.m_block + (8 / 128 if args.v_mode == "block" else 0)
+    pass1_bpp = {"rank1": PASS1_BYTES[wl.grad_dtype], "block": 0.0, "factored": PASS1_BYTES[wl.grad_dtype] - 0.5}[args.v_mode]
+    if args.v_mode == "factored":
+        pass2_bpp -= 1.0      # no second-moment codes are read or written
     alg_bytes = pass2_bpp * n_params
     achieved = alg_bytes / (p2_ms * 1e-3) / 1e9
     traffic_pp = PASS2_TRAFFIC_BYTES_PER_PARAM[wl.grad_dtype]
@@ -299,9 +304,9 @@ def run_ours(args):
                 "traffic": None if traffic_pp is None else traffic_pp * n_params,
                 "algorithmic_bytes_per_launch": alg_bytes, "ms_per_launch": p2_ms,
                 "pass1_ms_per_launch": p1_ms,
-                "pass1_achieved_gbs": PASS1_BYTES[wl.grad_dtype] * n_params / (p1_ms * 1e-3) / 1e9 if p1_ms > 0 else None,
+                "pass1_achieved_gbs": pass1_bpp * n_params / (p1_ms * 1e-3) / 1e9 if p1_ms > 0 else None,
                 "step_algorithmic_gbs": alg_bytes / (ms_step * 1e-3) / 1e9,
-                "step_moved_gbs": (pass2_bpp + (PASS1_BYTES[wl.grad_dtype] if args.v_mode == "rank1" else 0)) * n_params / (ms_step * 1e-3) / 1e9,
+                "step_moved_gbs": (pass2_bpp + pass1_bpp) * n_params / (ms_step * 1e-3) / 1e9,
                 "frac_of_nominal_8tbs": achieved / 8000.0}
 
     cpu = None
@@ -313,7 +318,7 @@ def run_ours(args):
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": wl.name, "tensors": len(wl.tensors), "params_per_gpu": n_params,
-                       "grad_dtype": wl.grad_dtype, "param_dtype": "f32", "m": f"B{args.m_block}/DE 4-bit", "v": ("Rank-1" if args.v_mode == "rank1" else "B128") + "/Linear 4-bit",
+                       "grad_dtype": wl.grad_dtype, "param_dtype": "f32", "m": f"B{args.m_block}/DE 4-bit", "v": {"rank1": "Rank-1/Linear 4-bit", "block": "B128/Linear 4-bit", "factored": "factorized (fp32 row/column statistics)"}[args.v_mode],
                        "l2": f"inputs larger than L2 ({(n_params * (8 + (2 if wl.grad_dtype == 'bf16' else 4) + 1)) / 1e9:.1f} GB touched per step), no flush", "parallelism": f"replicas x{world}, no collective"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu}
     print(json.dumps(line), flush=True)

@@ -42,7 +42,9 @@ typedef int32_t lpmm_status;
 typedef enum { LPMM_F32 = 0, LPMM_BF16 = 1 } lpmm_dtype;
 typedef enum { LPMM_NORM_BLOCK = 0, LPMM_NORM_RANK1 = 1 } lpmm_norm;          /* Sec. 2.2 / Sec. 4.2 */
 typedef enum { LPMM_MAP_DE_SIGNED = 0, LPMM_MAP_LINEAR_NOZERO = 1 } lpmm_map; /* App. D.2 / Sec. 4.1 */
-typedef enum { LPMM_V_RANK1 = 0, LPMM_V_BLOCK = 1 } lpmm_vmode;               /* second-moment normalizer for 2-D tensors */
+/* Second moment of 2-D tensors: 4-bit with rank-1 or block-wise normalization, or not stored at all but
+ * reconstructed from fp32 row / column statistics ("4-bit Factor", Sec. 4.3; 1-D tensors stay quantized). */
+typedef enum { LPMM_V_RANK1 = 0, LPMM_V_BLOCK = 1, LPMM_V_FACTORED = 2 } lpmm_vmode;
 
 /* How Eq. 1's last line (bias correction, sqrt, division) is evaluated. The stored states (codes and
  * scales) are bit-identical in both modes; only the rounding of the updated parameters differs.
@@ -81,6 +83,7 @@ typedef struct lpmm_state lpmm_state; /* opaque host handle */
 #define LPMM_KIND_FP32 0
 #define LPMM_KIND_BLOCK 1
 #define LPMM_KIND_RANK1 2
+#define LPMM_KIND_FACTORED 3 /* LPMM_V_FACTORED: v_scale0 = R (rows), v_scale1 = C (cols), no second-moment codes */
 
 /* Size in bytes of the device arena that holds the states of n tensors (codes, scales, fp32 states
  * of small tensors, the device-side tensor table and the per-step scratch for the rank-1 maxima).
@@ -108,7 +111,11 @@ lpmm_status lpmm_state_attach(const lpmm_config* cfg, const lpmm_shape* shapes, 
  * Both arrays are HOST arrays of n device pointers, each 16-byte aligned. step is t >= 1.
  * Requires 0 <= beta1, beta2 < 1, lr >= 0, eps >= 0, weight_decay >= 0, all finite.
  * Kernels launched: one pass over the rank-1 tensors that reduces the new row/column maxima, one
- * small pass that inverts them, one pass over all tensors that updates and re-quantizes. */
+ * small pass that inverts them, one pass over all tensors that updates and re-quantizes.
+ * LPMM_V_FACTORED (reading of Sec. 4.3, which gives no formula): R <- b2 R + (1-b2) rowsum(g^2), C likewise,
+ * v_ij = R_i C_j / sum(R), then Eq. 1 as usual; the first pass reduces the sums (fp32 atomics, so R and C are
+ * reproducible to rounding only), a fourth small kernel updates R, C and sum(R). Such tensors need
+ * cols % m_block == 0 (else LPMM_ERR_UNSUPPORTED at state creation). */
 lpmm_status lpmm_adamw4_step(lpmm_state* st, void* const* d_params, const void* const* d_grads,
                              int32_t grad_dtype, float lr, float beta1, float beta2, float eps,
                              float weight_decay, int64_t step, void* stream);

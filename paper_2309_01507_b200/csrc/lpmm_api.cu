@@ -45,16 +45,21 @@ struct Layout {
     size_t total = 0;
 };
 
+bool uses_rc(int32_t k) { return k == K_RANK1_FAST || k == K_RANK1_FLAT || k == K_FACT; }
+
 int public_kind(int32_t k) {
     if (k == K_FP32) return LPMM_KIND_FP32;
     if (k == K_BLOCK) return LPMM_KIND_BLOCK;
+    if (k == K_FACT) return LPMM_KIND_FACTORED;
     return LPMM_KIND_RANK1;
 }
+
+int32_t choose_kind(const lpmm_config& cfg, const lpmm_shape& s);
 
 lpmm_status validate_config(const lpmm_config* cfg, const lpmm_shape* shapes, int32_t n) {
     if (!cfg || !shapes || n <= 0) return LPMM_ERR_INVALID_ARG;
     if (cfg->min_quant_numel < 0) return LPMM_ERR_INVALID_ARG;
-    if (cfg->v_mode != LPMM_V_RANK1 && cfg->v_mode != LPMM_V_BLOCK) return LPMM_ERR_INVALID_ARG;
+    if (cfg->v_mode != LPMM_V_RANK1 && cfg->v_mode != LPMM_V_BLOCK && cfg->v_mode != LPMM_V_FACTORED) return LPMM_ERR_INVALID_ARG;
     if (cfg->bits != 4) return LPMM_ERR_UNSUPPORTED;
     if ((cfg->m_block != 128 && cfg->m_block != 2048) || cfg->v_block != 128) return LPMM_ERR_UNSUPPORTED;
     if (cfg->update_math != LPMM_UPDATE_FAST && cfg->update_math != LPMM_UPDATE_IEEE) return LPMM_ERR_INVALID_ARG;
@@ -67,6 +72,8 @@ lpmm_status validate_config(const lpmm_config* cfg, const lpmm_shape* shapes, in
         if (s.rows > (int64_t)1 << 40 || s.cols > (int64_t)1 << 40 || s.rows > ((int64_t)1 << 40) / s.cols)
             return LPMM_ERR_INVALID_ARG;  // numel overflow guard
         if (s.rows + s.cols > (int64_t)1 << 30) return LPMM_ERR_UNSUPPORTED;
+        // the factorized second moment is built for the tiled path only: whole first-moment blocks inside a row
+        if (cfg->v_mode == LPMM_V_FACTORED && choose_kind(*cfg, s) == K_RANK1_FLAT) return LPMM_ERR_UNSUPPORTED;
     }
     return LPMM_OK;
 }
@@ -77,7 +84,8 @@ int32_t choose_kind(const lpmm_config& cfg, const lpmm_shape& s) {
     if (!(s.flags & LPMM_FORCE_QUANT) && numel <= cfg.min_quant_numel) return K_FP32;  // App. C.1
     if (s.ndim == 1 || s.rows == 1 || s.cols == 1 || cfg.v_mode == LPMM_V_BLOCK) return K_BLOCK;  // Sec. 4.2
     // the tiled path needs whole first-moment blocks inside a row (and, for B2048, one block per tile width)
-    return (s.cols % cfg.m_block == 0) ? K_RANK1_FAST : K_RANK1_FLAT;
+    if (s.cols % cfg.m_block != 0) return K_RANK1_FLAT;   // (rejected by validate_config for the factorized mode)
+    return (cfg.v_mode == LPMM_V_FACTORED) ? K_FACT : K_RANK1_FAST;
 }
 
 void compute_layout(const lpmm_config& cfg, const lpmm_shape* shapes, int32_t n, Layout* L) {
@@ -95,7 +103,7 @@ void compute_layout(const lpmm_config& cfg, const lpmm_shape* shapes, int32_t n,
         t = TensorLayout{};
         t.rows = shapes[i].rows; t.cols = shapes[i].cols; t.numel = t.rows * t.cols;
         t.kind = choose_kind(cfg, shapes[i]);
-        if (t.kind == K_RANK1_FAST || t.kind == K_RANK1_FLAT) {
+        if (uses_rc(t.kind)) {
             t.rc_index = rc;
             t.c_off = (int32_t)((t.rows + 3) / 4 * 4);
             rc += t.c_off + (t.cols + 3) / 4 * 4;
@@ -116,7 +124,7 @@ void compute_layout(const lpmm_config& cfg, const lpmm_shape* shapes, int32_t n,
             const size_t nblk = (size_t)((t.numel + 127) / 128);
             const size_t nblk_m = (size_t)((t.numel + cfg.m_block - 1) / cfg.m_block);
             t.m_codes = off; off = align_up(off + code_bytes);
-            t.v_codes = off; off = align_up(off + code_bytes);
+            if (t.kind != K_FACT) { t.v_codes = off; off = align_up(off + code_bytes); }
             t.m_scale = off; off = align_up(off + sizeof(float) * nblk_m);
             if (t.kind == K_BLOCK) { t.v_bscale = off; off = align_up(off + sizeof(float) * nblk); }
         }
@@ -182,16 +190,16 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
             d.v32 = reinterpret_cast<float*>(A + t.v32);
         } else {
             d.m_codes = reinterpret_cast<uint8_t*>(A + t.m_codes);
-            d.v_codes = reinterpret_cast<uint8_t*>(A + t.v_codes);
+            d.v_codes = (t.kind == K_FACT) ? nullptr : reinterpret_cast<uint8_t*>(A + t.v_codes);
             d.m_scale = reinterpret_cast<float*>(A + t.m_scale);
             if (t.kind == K_BLOCK) d.v_bscale = reinterpret_cast<float*>(A + t.v_bscale);
-            if (t.kind == K_RANK1_FAST || t.kind == K_RANK1_FLAT) {
+            if (uses_rc(t.kind)) {
                 d.rc[0] = reinterpret_cast<float*>(A + st->L.rc[0]) + t.rc_index;
                 d.rc[1] = reinterpret_cast<float*>(A + st->L.rc[1]) + t.rc_index;
                 d.rcp_new = reinterpret_cast<float*>(A + st->L.rcp) + t.rc_index;
             }
         }
-        if (t.kind == K_RANK1_FAST) {
+        if (t.kind == K_RANK1_FAST || t.kind == K_FACT) {
             d.wx = (st->cfg.m_block == 2048) ? 8 : (t.cols % 1024 == 0) ? 4 : (t.cols % 512 == 0) ? 2 : 1;
             const int64_t tile_cols = (int64_t)kWarpElems * d.wx;
             int64_t tr = tile_elems / tile_cols;
@@ -207,13 +215,13 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
             d.flat_chunks = (int32_t)chunks;
             const int64_t per_tile = chunks * kWarps * kWarpElems;
             const int64_t flat_tiles = (t.numel + per_tile - 1) / per_tile;
-            if (t.kind != K_RANK1_FAST) tiles = flat_tiles;
+            if (t.kind != K_RANK1_FAST && t.kind != K_FACT) tiles = flat_tiles;
             if (t3[i] + flat_tiles > 0x7fffffffLL) return LPMM_ERR_UNSUPPORTED;
             t3[i + 1] = t3[i] + (int32_t)flat_tiles;
         }
         if (t2[i] + tiles > 0x7fffffffLL) return LPMM_ERR_UNSUPPORTED;
         t2[i + 1] = t2[i] + (int32_t)tiles;
-        const bool rank1 = (t.kind == K_RANK1_FAST || t.kind == K_RANK1_FLAT);
+        const bool rank1 = uses_rc(t.kind);
         t1[i + 1] = t1[i] + (rank1 ? (int32_t)tiles : 0);
     }
     st->total1 = t1[n];
@@ -379,7 +387,7 @@ lpmm_status enqueue_range(lpmm_state* st, StepArgs a, int32_t t0, int32_t t1, bo
         int64_t rc_begin = -1, rc_end = 0;
         for (int32_t i = t0; i < t1; ++i) {
             const TensorLayout& t = st->L.t[i];
-            if (t.kind != K_RANK1_FAST && t.kind != K_RANK1_FLAT) continue;
+            if (!uses_rc(t.kind)) continue;
             if (rc_begin < 0) rc_begin = t.rc_index;
             rc_end = (t.rc_index + t.c_off + (t.cols + 3) / 4 * 4 + 63) / 64 * 64;
         }
@@ -394,6 +402,10 @@ lpmm_status enqueue_range(lpmm_state* st, StepArgs a, int32_t t0, int32_t t1, bo
         if (ev) LPMM_CUDA(cudaEventRecord(ev[1], s));
         LPMM_CUDA(launch_rcp(rc_new, reinterpret_cast<float*>(st->arena + st->L.rcp) + rc_begin, rc_end - rc_begin, s));
         *launches += 2;
+        if (st->cfg.v_mode == LPMM_V_FACTORED) {   // statistics' moving averages and the row factors R_i / sum(R)
+            LPMM_CUDA(launch_factor_finalize(a, t0, t1, s));
+            *launches += 1;
+        }
     } else if (ev) {
         LPMM_CUDA(cudaEventRecord(ev[0], s));
         LPMM_CUDA(cudaEventRecord(ev[1], s));
@@ -403,7 +415,8 @@ lpmm_status enqueue_range(lpmm_state* st, StepArgs a, int32_t t0, int32_t t1, bo
     a.tile_begin = st->tiles2[t0];
     a.tile_end = st->tiles2[t1];
     const int32_t cap = st->sms * st->occ2, tiles = a.tile_end - a.tile_begin;
-    LPMM_CUDA(launch_pass2(a, bf16, ieee_update, st->cfg.m_block == 2048 ? 11 : 7, tiles < cap ? tiles : cap, s));
+    LPMM_CUDA(launch_pass2(a, bf16, ieee_update, st->cfg.m_block == 2048 ? 11 : 7, st->cfg.v_mode == LPMM_V_FACTORED,
+                           tiles < cap ? tiles : cap, s));
     if (ev) LPMM_CUDA(cudaEventRecord(ev[3], s));
     *launches += 1;
     return LPMM_OK;
@@ -594,11 +607,11 @@ lpmm_status lpmm_state_view(const lpmm_state* st, int32_t tensor, int32_t* kind,
     const TensorLayout& t = st->L.t[tensor];
     const char* A = st->arena;
     const bool q = (t.kind != K_FP32);
-    const bool r1 = (t.kind == K_RANK1_FAST || t.kind == K_RANK1_FLAT);
+    const bool r1 = uses_rc(t.kind);
     if (kind) *kind = public_kind(t.kind);
     if (m_codes) *m_codes = q ? reinterpret_cast<const uint8_t*>(A + t.m_codes) : nullptr;
     if (m_scale) *m_scale = q ? reinterpret_cast<const float*>(A + t.m_scale) : nullptr;
-    if (v_codes) *v_codes = q ? reinterpret_cast<const uint8_t*>(A + t.v_codes) : nullptr;
+    if (v_codes) *v_codes = (q && t.kind != K_FACT) ? reinterpret_cast<const uint8_t*>(A + t.v_codes) : nullptr;
     const float* rc = reinterpret_cast<const float*>(A + st->L.rc[st->phase]) + t.rc_index;
     if (v_scale0) *v_scale0 = r1 ? rc : (t.kind == K_BLOCK ? reinterpret_cast<const float*>(A + t.v_bscale) : nullptr);
     if (v_scale1) *v_scale1 = r1 ? rc + t.c_off : nullptr;

@@ -11,7 +11,7 @@ namespace lpmm {
 // Work kinds inside the step kernels. RANK1_FAST needs cols % 128 == 0 (a 128-block then lies inside
 // one row and every row starts on a 16-byte boundary of every operand); other 2-D shapes take the
 // element-indexed RANK1_FLAT path.
-enum : int32_t { K_FP32 = 0, K_BLOCK = 1, K_RANK1_FAST = 2, K_RANK1_FLAT = 3 };
+enum : int32_t { K_FP32 = 0, K_BLOCK = 1, K_RANK1_FAST = 2, K_RANK1_FLAT = 3, K_FACT = 4 };
 
 constexpr int kThreads = 256;          // threads per CTA in the step kernels
 constexpr int kWarps = kThreads / 32;
@@ -24,8 +24,8 @@ struct TensorDesc {
     float* m_scale;     // ceil(numel / m_block) block maxima of |m|
     uint8_t* v_codes;
     float* v_bscale;    // K_BLOCK: ceil(numel/128) block maxima of v
-    float* rc[2];       // K_RANK1_*: two buffers of [r (rows, padded to 4) | c (cols)]
-    float* rcp_new;     // K_RANK1_*: reciprocals of the new r, c (same layout), per-step scratch
+    float* rc[2];       // K_RANK1_*: two buffers of [r (rows, padded to 4) | c (cols)]; K_FACT: [R | C] statistics
+    float* rcp_new;     // K_RANK1_*: reciprocals of the new r, c (same layout), per-step scratch; K_FACT: R_i / sum(R)
     float* m32;         // K_FP32
     float* v32;
     int64_t rows, cols, numel;
@@ -54,7 +54,8 @@ struct StepArgs {
 };
 
 cudaError_t launch_pass1(const StepArgs& a, bool bf16, int grid, cudaStream_t s);
-cudaError_t launch_pass2(const StepArgs& a, bool bf16, bool exact, int m_shift, int grid, cudaStream_t s);
+cudaError_t launch_pass2(const StepArgs& a, bool bf16, bool exact, int m_shift, bool factored, int grid, cudaStream_t s);
+cudaError_t launch_factor_finalize(const StepArgs& a, int t0, int t1, cudaStream_t s);
 cudaError_t launch_sgdm(const StepArgs& a, bool bf16, int grid, cudaStream_t s);
 cudaError_t launch_rcp(const float* src, float* dst, int64_t n, cudaStream_t s);
 cudaError_t step_kernel_occupancy(int* pass1_blocks_per_sm, int* pass2_blocks_per_sm);

@@ -122,7 +122,8 @@ __device__ __forceinline__ LaneTables make_lane_tables() {
 
 // Dequantize (Sec. 2.2), update the moments (Eq. 1) and the parameters for 8 elements, two at a time.
 // m_prod is T_DE[lane & 15] * (old block scale of m); vs[k] the old scale of element k's second moment.
-template <bool EXACT>
+// FACT: the second moment is not dequantized and averaged but given (vs[k] is the reconstructed v_ij itself).
+template <bool EXACT, bool FACT = false>
 __device__ __forceinline__ void moments_and_update8(float (&w)[8], const float (&g)[8], uint32_t qm, uint32_t qv,
                                                     float m_prod, const float (&vs)[8], const Hyper& h,
                                                     const Hyper2& h2, const LaneTables& lt, float (&mt)[8],
@@ -131,12 +132,16 @@ __device__ __forceinline__ void moments_and_update8(float (&w)[8], const float (
     for (int k = 0; k < 8; k += 2) {
         const float2 m = make_float2(__shfl_sync(lt.mask, m_prod, (int)(qm >> (4 * k)), 16),
                                      __shfl_sync(lt.mask, m_prod, (int)(qm >> (4 * k + 4)), 16));
-        const float2 tl = make_float2(__shfl_sync(lt.mask, lt.lin, (int)(qv >> (4 * k)), 16),
-                                      __shfl_sync(lt.mask, lt.lin, (int)(qv >> (4 * k + 4)), 16));
-        const float2 v = mul2_rn(tl, make_float2(vs[k], vs[k + 1]));
         const float2 g2 = make_float2(g[k], g[k + 1]);
         const float2 m2 = ema_m2(m, g2, h2);
-        const float2 v2 = ema_v2(v, g2, h2);
+        float2 v2;
+        if (FACT) {
+            v2 = make_float2(vs[k], vs[k + 1]);
+        } else {
+            const float2 tl = make_float2(__shfl_sync(lt.mask, lt.lin, (int)(qv >> (4 * k)), 16),
+                                          __shfl_sync(lt.mask, lt.lin, (int)(qv >> (4 * k + 4)), 16));
+            v2 = ema_v2(mul2_rn(tl, make_float2(vs[k], vs[k + 1])), g2, h2);
+        }
         mt[k] = m2.x; mt[k + 1] = m2.y;
         vt[k] = v2.x; vt[k + 1] = v2.y;
         if (EXACT) {
@@ -248,7 +253,7 @@ struct TileView {
 constexpr uint32_t kL2Ahead = 4;   // rows
 __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
-template <bool BF16, int MSHIFT>
+template <bool BF16, int MSHIFT, bool FACT>
 __device__ __forceinline__ void prefetch_row(const TileView& t, uint32_t k) {
     const uint32_t off = k * t.row_step;
     prefetch_l2(t.w + off);
@@ -258,11 +263,11 @@ __device__ __forceinline__ void prefetch_row(const TileView& t, uint32_t k) {
         prefetch_l2(reinterpret_cast<const float*>(t.g) + off);
     }
     prefetch_l2(t.m_codes + (off >> 1));
-    prefetch_l2(t.v_codes + (off >> 1));
+    if (!FACT) prefetch_l2(t.v_codes + (off >> 1));
     prefetch_l2(t.m_scale + (off >> MSHIFT));
 }
 
-template <bool BF16, int MSHIFT>
+template <bool BF16, int MSHIFT, bool FACT>
 __device__ __forceinline__ void load_row(RowRegs<BF16>& r, const TileView& t, uint32_t k) {
     const uint32_t off = k * t.row_step;
     r.w0 = *reinterpret_cast<const float4*>(t.w + off);
@@ -274,13 +279,18 @@ __device__ __forceinline__ void load_row(RowRegs<BF16>& r, const TileView& t, ui
         r.g1 = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(t.g) + off + 4));
     }
     r.qm = *reinterpret_cast<const uint32_t*>(t.m_codes + (off >> 1));
-    r.qv = *reinterpret_cast<const uint32_t*>(t.v_codes + (off >> 1));
     r.am = t.m_scale[off >> MSHIFT];
-    r.r_old = __ldg(t.r_old + k * t.row_stride);
-    r.r_rcp = __ldg(t.r_rcp + k * t.row_stride);
+    r.r_rcp = __ldg(t.r_rcp + k * t.row_stride);        // FACT: the row factor R_i / sum(R)
+    if (FACT) {
+        r.qv = 0;
+        r.r_old = 0.0f;
+    } else {
+        r.qv = *reinterpret_cast<const uint32_t*>(t.v_codes + (off >> 1));
+        r.r_old = __ldg(t.r_old + k * t.row_stride);
+    }
 }
 
-template <bool BF16, bool EXACT, int MSHIFT>
+template <bool BF16, bool EXACT, int MSHIFT, bool FACT>
 __device__ __forceinline__ void process_row(const RowRegs<BF16>& r, const TileView& t, uint32_t k,
                                             const float (&c_old)[8], const float (&c_rcp)[8], const Hyper& h,
                                             const Hyper2& h2, const LaneTables& lt, const unsigned char* s_lut) {
@@ -290,18 +300,23 @@ __device__ __forceinline__ void process_row(const RowRegs<BF16>& r, const TileVi
     unpack_grad8<BF16>(r.g0, r.g1, gv);
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-        vs[j] = fminf(r.r_old, c_old[j]);      // Sec. 4.2: scale = min(r_i, c_j)
-        vr[j] = fmaxf(r.r_rcp, c_rcp[j]);      // 1/min(r', c') = max(1/r', 1/c')
+        if (FACT) {
+            vs[j] = __fmul_rn(r.r_rcp, c_rcp[j]);  // Sec. 4.3: v_ij = (R_i / sum R) * C_j
+            vr[j] = 0.0f;
+        } else {
+            vs[j] = fminf(r.r_old, c_old[j]);      // Sec. 4.2: scale = min(r_i, c_j)
+            vr[j] = fmaxf(r.r_rcp, c_rcp[j]);      // 1/min(r', c') = max(1/r', 1/c')
+        }
     }
-    moments_and_update8<EXACT>(wv, gv, r.qm, r.qv, __fmul_rn(lt.de, r.am), vs, h, h2, lt, mt, vt);
+    moments_and_update8<EXACT, FACT>(wv, gv, r.qm, r.qv, __fmul_rn(lt.de, r.am), vs, h, h2, lt, mt, vt);
     store8_f32(t.w + off, wv);
     const float am_new = block_max(absmax8(mt), MSHIFT, lt, t.s_red, *t.red_step);
     if ((threadIdx.x & (MSHIFT == 7 ? 15 : 2047)) == 0) t.m_scale[off >> MSHIFT] = am_new;
     *reinterpret_cast<uint32_t*>(t.m_codes + (off >> 1)) = quantize8_de(mt, scale_rcp(am_new), s_lut);
-    *reinterpret_cast<uint32_t*>(t.v_codes + (off >> 1)) = quantize8_lin(vt, vr, h2);
+    if (!FACT) *reinterpret_cast<uint32_t*>(t.v_codes + (off >> 1)) = quantize8_lin(vt, vr, h2);
 }
 
-template <bool BF16, bool EXACT, int MSHIFT>
+template <bool BF16, bool EXACT, int MSHIFT, bool FACT = false>
 __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __restrict__ w, const void* __restrict__ g,
                                                  int tile, int phase, const Hyper& h, const Hyper2& h2,
                                                  const LaneTables& lt, const unsigned char* s_lut, float* s_red,
@@ -321,15 +336,21 @@ __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __r
     const uint32_t nrows = (uint32_t)((row_end - row0 + wy_count - 1) / wy_count);
 
     float c_old[8], c_rcp[8];
-    load8_f32(rc_old + d.c_off + col0, c_old);
-    load8_f32(rcp_new + d.c_off + col0, c_rcp);
+    if (FACT) {      // the new column statistics C_j sit in the "new" buffer; nothing old is needed
+        load8_f32((phase ? d.rc[0] : d.rc[1]) + d.c_off + col0, c_rcp);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) c_old[j] = 0.0f;
+    } else {
+        load8_f32(rc_old + d.c_off + col0, c_old);
+        load8_f32(rcp_new + d.c_off + col0, c_rcp);
+    }
     const int64_t e0 = row0 * d.cols + col0;
     TileView t;
     t.w = w + e0;
     t.g = BF16 ? static_cast<const void*>(reinterpret_cast<const uint16_t*>(g) + e0)
                : static_cast<const void*>(reinterpret_cast<const float*>(g) + e0);
     t.m_codes = d.m_codes + (e0 >> 1);
-    t.v_codes = d.v_codes + (e0 >> 1);
+    t.v_codes = FACT ? nullptr : d.v_codes + (e0 >> 1);
     t.m_scale = d.m_scale + (e0 >> MSHIFT);
     t.r_old = rc_old + row0;
     t.r_rcp = rcp_new + row0;
@@ -342,17 +363,17 @@ __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __r
     // Two register sets alternate: while one row is processed the next one is already in flight.
     RowRegs<BF16> ra, rb;
 #pragma unroll
-    for (uint32_t k = 1; k < kL2Ahead; ++k) if (k < nrows) prefetch_row<BF16, MSHIFT>(t, k);
-    load_row<BF16, MSHIFT>(ra, t, 0);
+    for (uint32_t k = 1; k < kL2Ahead; ++k) if (k < nrows) prefetch_row<BF16, MSHIFT, FACT>(t, k);
+    load_row<BF16, MSHIFT, FACT>(ra, t, 0);
     for (uint32_t k = 0; k < nrows; k += 2) {
         const bool has_b = k + 1 < nrows;
-        if (k + kL2Ahead < nrows) prefetch_row<BF16, MSHIFT>(t, k + kL2Ahead);
-        if (has_b) load_row<BF16, MSHIFT>(rb, t, k + 1);
-        process_row<BF16, EXACT, MSHIFT>(ra, t, k, c_old, c_rcp, h, h2, lt, s_lut);
+        if (k + kL2Ahead < nrows) prefetch_row<BF16, MSHIFT, FACT>(t, k + kL2Ahead);
+        if (has_b) load_row<BF16, MSHIFT, FACT>(rb, t, k + 1);
+        process_row<BF16, EXACT, MSHIFT, FACT>(ra, t, k, c_old, c_rcp, h, h2, lt, s_lut);
         if (!has_b) break;
-        if (k + 1 + kL2Ahead < nrows) prefetch_row<BF16, MSHIFT>(t, k + 1 + kL2Ahead);
-        if (k + 2 < nrows) load_row<BF16, MSHIFT>(ra, t, k + 2);
-        process_row<BF16, EXACT, MSHIFT>(rb, t, k + 1, c_old, c_rcp, h, h2, lt, s_lut);
+        if (k + 1 + kL2Ahead < nrows) prefetch_row<BF16, MSHIFT, FACT>(t, k + 1 + kL2Ahead);
+        if (k + 2 < nrows) load_row<BF16, MSHIFT, FACT>(ra, t, k + 2);
+        process_row<BF16, EXACT, MSHIFT, FACT>(rb, t, k + 1, c_old, c_rcp, h, h2, lt, s_lut);
     }
 }
 
@@ -643,7 +664,9 @@ __device__ __forceinline__ void pass2_fp32(const TensorDesc& d, float* __restric
     }
 }
 
-template <bool BF16, bool EXACT, int MSHIFT>
+// VF: the state uses the factorized second moment (then no tensor is of the rank-1 tiled kind, and vice versa),
+// so each instantiation carries only one of the two tiled paths.
+template <bool BF16, bool EXACT, int MSHIFT, bool VF>
 __global__ void __launch_bounds__(kThreads, 2) pass2_kernel(StepArgs a) {
     __shared__ __align__(16) unsigned char s_lut[kLutSmemBytes];
     __shared__ float s_red[2 * kWarps];
@@ -659,7 +682,12 @@ __global__ void __launch_bounds__(kThreads, 2) pass2_kernel(StepArgs a) {
         const void* g = a.grads[t];
         const int local = tile - __ldg(a.tile_start + t);
         switch (d.kind) {
-            case K_RANK1_FAST: pass2_rank1_fast<BF16, EXACT, MSHIFT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
+            case K_RANK1_FAST:
+                if (!VF) pass2_rank1_fast<BF16, EXACT, MSHIFT, false>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step);
+                break;
+            case K_FACT:
+                if (VF) pass2_rank1_fast<BF16, EXACT, MSHIFT, true>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step);
+                break;
             case K_RANK1_FLAT: pass2_flat<BF16, true, EXACT, MSHIFT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
             case K_BLOCK:      pass2_flat<BF16, false, EXACT, MSHIFT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
             default:           pass2_fp32<BF16, EXACT>(d, w, g, local, a.h); break;
@@ -858,6 +886,81 @@ __device__ __forceinline__ void pass1_rank1_fast(const TensorDesc& d, const void
     }
 }
 
+// ---- pass 1 of the factorized second moment: row and column sums of g^2 (Sec. 4.3) ---------------------
+//
+// Same tiling as the maxima pass. Sums are accumulated in binary32 (eight squares per lane, a shuffle tree
+// per row, one register per column over the tile's rows) and combined across tiles with atomicAdd, so they
+// are reproducible to rounding only.
+
+template <bool BF16>
+__device__ __forceinline__ void pass1_fact(const TensorDesc& d, const void* __restrict__ g, int tile, int phase,
+                                           float* s_col) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int wx = d.wx, wy_count = kWarps / wx;
+    const int tx = tile % d.tiles_x, ty = tile / d.tiles_x;
+    const int64_t col_w = (int64_t)tx * (kWarpElems * wx) + (warp % wx) * kWarpElems;
+    const int64_t col0 = col_w + lane * kLaneElems;
+    const bool active = col0 < d.cols;                  // cols % 256 == 128: the upper half-warp adds zeros
+    float* sums = (phase ? d.rc[0] : d.rc[1]);          // [row sums | column sums], cleared before the launch
+    const int64_t row0 = (int64_t)ty * d.tile_rows + warp / wx;
+    const int64_t row_end = min((int64_t)(ty + 1) * d.tile_rows, d.rows);
+    float c_sum[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) c_sum[k] = 0.0f;
+    for (int64_t i = row0; i < row_end; i += wy_count) {
+        float gv[8];
+        float rs = 0.0f;
+        if (active) {
+            load8_grad<BF16>(g, i * d.cols + col0, gv);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const float gg = __fmul_rn(gv[k], gv[k]);
+                rs = __fadd_rn(rs, gg);
+                c_sum[k] = __fadd_rn(c_sum[k], gg);
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) rs = __fadd_rn(rs, __shfl_xor_sync(0xffffffffu, rs, o));
+        if (lane == 0) atomicAdd(sums + i, rs);
+    }
+    float* mine = s_col + warp * kWarpElems;
+    __syncwarp();
+#pragma unroll
+    for (int k = 0; k < 8; ++k) mine[lane * kLaneElems + k] = c_sum[k];
+    __syncwarp();
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const int cc = lane + 32 * k;
+        if (col_w + cc < d.cols) atomicAdd(sums + d.c_off + col_w + cc, mine[cc]);
+    }
+}
+
+// One CTA per factorized tensor: turns the sums into the statistics' moving averages R, C (in the "new"
+// buffer), sums R in binary64 in a fixed order and stores the row factors R_i * (1 / sum R).
+__global__ void __launch_bounds__(256) factor_finalize_kernel(StepArgs a, int t0) {
+    const TensorDesc d = a.descs[t0 + blockIdx.x];
+    if (d.kind != K_FACT) return;
+    const float* old = (a.phase ? d.rc[1] : d.rc[0]);
+    float* cur = (a.phase ? d.rc[0] : d.rc[1]);
+    __shared__ double s_part[256];
+    double part = 0.0;
+    for (int64_t i = threadIdx.x; i < d.rows; i += blockDim.x) {
+        const float r = __fadd_rn(__fmul_rn(a.h.beta2, old[i]), __fmul_rn(a.h.omb2, cur[i]));
+        cur[i] = r;
+        part += (double)r;
+    }
+    for (int64_t j = threadIdx.x; j < d.cols; j += blockDim.x)
+        cur[d.c_off + j] = __fadd_rn(__fmul_rn(a.h.beta2, old[d.c_off + j]), __fmul_rn(a.h.omb2, cur[d.c_off + j]));
+    s_part[threadIdx.x] = part;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if ((int)threadIdx.x < o) s_part[threadIdx.x] += s_part[threadIdx.x + o];
+        __syncthreads();
+    }
+    const float r_total = scale_rcp((float)s_part[0]);
+    for (int64_t i = threadIdx.x; i < d.rows; i += blockDim.x) d.rcp_new[i] = __fmul_rn(cur[i], r_total);
+}
+
 template <bool BF16>
 __device__ __forceinline__ void pass1_rank1_flat(const TensorDesc& d, const void* __restrict__ g, int tile, int phase,
                                                  const Hyper& h) {
@@ -897,6 +1000,7 @@ __global__ void __launch_bounds__(kThreads, 3) pass1_kernel(StepArgs a) {
         const void* g = a.grads[t];
         const int local = tile - __ldg(a.tile_start + t);
         if (d.kind == K_RANK1_FAST) pass1_rank1_fast<BF16>(d, g, local, a.phase, h2, lt, s_col);
+        else if (d.kind == K_FACT) pass1_fact<BF16>(d, g, local, a.phase, s_col);
         else pass1_rank1_flat<BF16>(d, g, local, a.phase, a.h);
     }
 }
@@ -983,27 +1087,35 @@ cudaError_t launch_pass1(const StepArgs& a, bool bf16, int grid, cudaStream_t s)
 }
 
 template <bool BF16, bool EXACT, int MSHIFT>
-cudaError_t launch_pass2_t(const StepArgs& a, int grid, cudaStream_t s) {
-    if (a.variant == 1) {
+cudaError_t launch_pass2_t(const StepArgs& a, bool factored, int grid, cudaStream_t s) {
+    if (factored) {
+        pass2_kernel<BF16, EXACT, MSHIFT, true><<<grid, kThreads, 0, s>>>(a);
+    } else if (a.variant == 1) {
         constexpr int smem = bulk_smem_bytes<BF16>();
         cudaError_t e = cudaFuncSetAttribute(pass2_bulk_kernel<BF16, EXACT, MSHIFT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
         pass2_bulk_kernel<BF16, EXACT, MSHIFT><<<grid, kThreads, smem, s>>>(a);
     } else {
-        pass2_kernel<BF16, EXACT, MSHIFT><<<grid, kThreads, 0, s>>>(a);
+        pass2_kernel<BF16, EXACT, MSHIFT, false><<<grid, kThreads, 0, s>>>(a);
     }
     return cudaGetLastError();
 }
 
 template <bool BF16, bool EXACT>
-cudaError_t launch_pass2_m(const StepArgs& a, int m_shift, int grid, cudaStream_t s) {
-    return m_shift == 11 ? launch_pass2_t<BF16, EXACT, 11>(a, grid, s) : launch_pass2_t<BF16, EXACT, 7>(a, grid, s);
+cudaError_t launch_pass2_m(const StepArgs& a, int m_shift, bool factored, int grid, cudaStream_t s) {
+    return m_shift == 11 ? launch_pass2_t<BF16, EXACT, 11>(a, factored, grid, s) : launch_pass2_t<BF16, EXACT, 7>(a, factored, grid, s);
 }
 
-cudaError_t launch_pass2(const StepArgs& a, bool bf16, bool exact, int m_shift, int grid, cudaStream_t s) {
+cudaError_t launch_pass2(const StepArgs& a, bool bf16, bool exact, int m_shift, bool factored, int grid, cudaStream_t s) {
     if (a.tile_end <= a.tile_begin) return cudaSuccess;
-    if (bf16) return exact ? launch_pass2_m<true, true>(a, m_shift, grid, s) : launch_pass2_m<true, false>(a, m_shift, grid, s);
-    return exact ? launch_pass2_m<false, true>(a, m_shift, grid, s) : launch_pass2_m<false, false>(a, m_shift, grid, s);
+    if (bf16) return exact ? launch_pass2_m<true, true>(a, m_shift, factored, grid, s) : launch_pass2_m<true, false>(a, m_shift, factored, grid, s);
+    return exact ? launch_pass2_m<false, true>(a, m_shift, factored, grid, s) : launch_pass2_m<false, false>(a, m_shift, factored, grid, s);
+}
+
+cudaError_t launch_factor_finalize(const StepArgs& a, int t0, int t1, cudaStream_t s) {
+    if (t1 <= t0) return cudaSuccess;
+    factor_finalize_kernel<<<t1 - t0, 256, 0, s>>>(a, t0);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_sgdm(const StepArgs& a, bool bf16, int grid, cudaStream_t s) {
@@ -1024,7 +1136,7 @@ cudaError_t launch_rcp(const float* src, float* dst, int64_t n, cudaStream_t s) 
 cudaError_t step_kernel_occupancy(int* p1, int* p2) {
     cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(p1, pass1_kernel<true>, kThreads, 0);
     if (e != cudaSuccess) return e;
-    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(p2, pass2_kernel<true, false, 7>, kThreads, 0);
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(p2, pass2_kernel<true, false, 7, false>, kThreads, 0);
 }
 
 }  // namespace lpmm

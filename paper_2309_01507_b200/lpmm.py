@@ -20,11 +20,11 @@ NOALLOC_MAX_SCALES = 262144
 F32, BF16 = 0, 1
 NORM_BLOCK, NORM_RANK1 = 0, 1
 MAP_DE_SIGNED, MAP_LINEAR_NOZERO = 0, 1
-V_RANK1, V_BLOCK = 0, 1
+V_RANK1, V_BLOCK, V_FACTORED = 0, 1, 2
 UPDATE_FAST, UPDATE_IEEE = 0, 1
 FORCE_QUANT, FORCE_FP32 = 1, 2
 Q_GIVEN_SCALES = 1
-KIND_FP32, KIND_BLOCK, KIND_RANK1 = 0, 1, 2
+KIND_FP32, KIND_BLOCK, KIND_RANK1, KIND_FACTORED = 0, 1, 2, 3
 
 EXPORTS = ("lpmm_state_bytes", "lpmm_state_init", "lpmm_state_attach", "lpmm_adamw4_step",
            "lpmm_adamw4_step_host", "lpmm_stage_bytes", "lpmm_quantize", "lpmm_dequantize",
@@ -324,7 +324,7 @@ def state_view(state: State, i: int) -> dict:
         "m_codes": view(ptrs[0], (numel + 1) // 2, torch.uint8),
         "m_scale": view(ptrs[1], 4 * nblk_m, torch.float32),
         "v_codes": view(ptrs[2], (numel + 1) // 2, torch.uint8),
-        "v_s0": view(ptrs[3], 4 * (sh.rows if k == KIND_RANK1 else nblk_v), torch.float32),
+        "v_s0": view(ptrs[3], 4 * (sh.rows if k in (KIND_RANK1, KIND_FACTORED) else nblk_v), torch.float32),
         "v_s1": view(ptrs[4], 4 * sh.cols, torch.float32),
         "m32": view(ptrs[5], 4 * numel, torch.float32),
         "v32": view(ptrs[6], 4 * numel, torch.float32),

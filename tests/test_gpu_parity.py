@@ -287,3 +287,54 @@ def test_sgdm_step_matches_oracle_bit_for_bit(grad_dtype, m_block):
                     assert np.array_equal(view[name].cpu().numpy(), ref), (s.name, name, t)
             assert np.array_equal(params[i].cpu().numpy().ravel(), w_ref[i]), (s.name, t)
     assert state.last_launches == 1
+
+
+@pytest.mark.parametrize("grad_dtype", [torch.float32, torch.bfloat16])
+def test_factorized_second_moment_matches_oracle(grad_dtype):
+    # "4-bit Factor": m in 4 bits (bit-exact), v reconstructed from fp32 row/column statistics whose sums the GPU
+    # accumulates in binary32 in another order than the oracle's binary64: R, C within 1e-5, parameters within
+    # 2e-5 * max(|w|, lr) (the update moves with 1/sqrt(v)); 1-D and small tensors behave as in the default mode.
+    cfg = lpmm.default_config(v_mode=lpmm.V_FACTORED)
+    specs = [_mat(96, 256), _mat(40, 1024), _mat(130, 384), _mat(33, 77), _vec(50265), _vec(300), _mat(64, 128)]
+    hyper = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
+    params = [workloads.make_param(s, 13, i, device="cuda") for i, s in enumerate(specs)]
+    state = lpmm.state_init(cfg, specs)
+    kinds = [lpmm.state_view(state, i)["kind"] for i in range(len(specs))]
+    assert kinds == [lpmm.KIND_FACTORED, lpmm.KIND_FACTORED, lpmm.KIND_FACTORED, lpmm.KIND_FP32, lpmm.KIND_BLOCK,
+                     lpmm.KIND_FP32, lpmm.KIND_FACTORED]
+    w_ref = [p.cpu().numpy().ravel().copy() for p in params]
+    ost, Rs, Cs = [], [], []
+    for i, s in enumerate(specs):
+        k = {lpmm.KIND_FACTORED: oracle.RANK1, lpmm.KIND_FP32: oracle.FP32, lpmm.KIND_BLOCK: oracle.BLOCK}[kinds[i]]
+        ost.append(oracle.state_init(s.rows, s.cols, k))
+        Rs.append(np.zeros(s.rows, np.float32)); Cs.append(np.zeros(s.cols, np.float32))
+    for t in range(1, 6):
+        grads = [workloads.make_grad(s, 13, i, t, device="cuda", dtype=grad_dtype) for i, s in enumerate(specs)]
+        lpmm.adamw4_step(state, params, grads, step=t, **hyper)
+        torch.cuda.synchronize()
+        assert lpmm.device_status(state) == 0
+        for i, s in enumerate(specs):
+            g = grads[i].float().cpu().numpy().ravel()
+            view = lpmm.state_view(state, i)
+            if kinds[i] == lpmm.KIND_FACTORED:
+                oracle.adamw4_factor_step(w_ref[i], g, ost[i], Rs[i], Cs[i], step=t, **hyper)
+                assert view["v_codes"] is None
+                np.testing.assert_allclose(view["v_s0"].cpu().numpy(), Rs[i], rtol=1e-5, atol=0)
+                np.testing.assert_allclose(view["v_s1"].cpu().numpy(), Cs[i], rtol=1e-5, atol=0)
+                tol = 2e-5
+            else:
+                oracle.adamw4_step(w_ref[i], g, ost[i], step=t, **hyper)
+                tol = 1e-6
+            for name in ("m_codes", "m_scale", "m32", "v32"):
+                ref = getattr(ost[i], name)
+                if ref is not None:
+                    assert np.array_equal(view[name].cpu().numpy(), ref), (s.name, name, t)
+            w = params[i].cpu().numpy().ravel()
+            err = np.max(np.abs(w - w_ref[i]) / np.maximum(np.abs(w_ref[i]), hyper["lr"]))
+            assert err <= tol, (s.name, t, err)
+            w_ref[i][:] = w
+    assert state.last_launches == 4      # sums pass, reciprocal pass, statistics pass, update pass
+    # a matrix whose rows do not hold whole first-moment blocks is refused in this mode
+    with pytest.raises(lpmm.LpmmError) as ei:
+        lpmm.state_init(cfg, [_mat(257, 129)])
+    assert ei.value.status == lpmm.ERR_UNSUPPORTED
