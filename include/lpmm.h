@@ -19,6 +19,8 @@
  *    in bits 0-3 of byte k and element 2k+1 in bits 4-7; ceil(numel/2) bytes per moment.
  *  - NaN/Inf gradients are not detected; the result is then unspecified (but nothing faults).
  *  - There is no CPU fallback: without a CUDA device every launching call returns LPMM_ERR_CUDA.
+ *  - The device that owns the arena must be the current device of the calling thread. A state handle is not
+ *    thread-safe: use it from one thread at a time.
  */
 #ifndef LPMM_H
 #define LPMM_H

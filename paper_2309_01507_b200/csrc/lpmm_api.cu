@@ -84,7 +84,8 @@ int32_t choose_kind(const lpmm_config& cfg, const lpmm_shape& s) {
     if (!(s.flags & LPMM_FORCE_QUANT) && numel <= cfg.min_quant_numel) return K_FP32;  // App. C.1
     if (s.ndim == 1 || s.rows == 1 || s.cols == 1 || cfg.v_mode == LPMM_V_BLOCK) return K_BLOCK;  // Sec. 4.2
     // the tiled path needs whole first-moment blocks inside a row (and, for B2048, one block per tile width)
-    if (s.cols % cfg.m_block != 0) return K_RANK1_FLAT;   // (rejected by validate_config for the factorized mode)
+    // the tiled path keeps 32-bit element offsets inside a tile: rows of at most 2^24 elements
+    if (s.cols % cfg.m_block != 0 || s.cols > ((int64_t)1 << 24)) return K_RANK1_FLAT;   // (refused in the factorized mode)
     return (cfg.v_mode == LPMM_V_FACTORED) ? K_FACT : K_RANK1_FAST;
 }
 

@@ -976,16 +976,23 @@ __device__ __forceinline__ void pass1_rank1_flat(const TensorDesc& d, const void
         load8_grad_guard<BF16>(g, e, d.numel, gv);
         const uint32_t qv = load_codes_guard(d.v_codes, e, d.numel);
         int64_t i = e / d.cols, j = e - i * d.cols;
+        float run = 0.0f;                      // maximum of the lane's current run of elements in row i
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
             if (e + k < d.numel) {
                 const float s = fminf(__ldg(rc_old + i), __ldg(rc_old + d.c_off + j));
                 const float vt = ema_v(__fmul_rn(lin_value((qv >> (4 * k)) & 15u), s), gv[k], h);
-                atomic_max_nonneg(rc_new + i, vt);
+                run = fmaxf(run, vt);
                 atomic_max_nonneg(rc_new + d.c_off + j, vt);
             }
-            if (++j == d.cols) { j = 0; ++i; }
+            if (++j == d.cols) {               // the row ends inside the lane's elements: publish and start over
+                atomic_max_nonneg(rc_new + i, run);
+                run = 0.0f;
+                j = 0;
+                ++i;
+            }
         }
+        if (i < d.rows) atomic_max_nonneg(rc_new + i, run);
     }
 }
 

@@ -206,16 +206,18 @@ def adamw4_step(state: State, params, grads, *, lr, beta1, beta2, eps, weight_de
         pp, gp, gd = _ptr_array(params), _ptr_array(grads), _grad_dtype(grads)
     else:
         pp, gp, gd = ptr_cache
-    _check(lib().lpmm_adamw4_step(state.handle, pp, gp, gd, lr, beta1, beta2, eps, weight_decay, step,
-                                  _stream_ptr(stream)), "lpmm_adamw4_step")
+    with torch.cuda.device(state.arena.device):
+        _check(lib().lpmm_adamw4_step(state.handle, pp, gp, gd, lr, beta1, beta2, eps, weight_decay, step,
+                                      _stream_ptr(stream)), "lpmm_adamw4_step")
 
 
 def sgdm4_step(state: State, params, grads, *, lr, beta, stream=None) -> None:
     """lpmm_sgdm4_step: compressed SGDM (Alg. 2) on lists of contiguous CUDA tensors."""
     if len(params) != state.n or len(grads) != state.n:
         raise ValueError("params/grads must have one tensor per state entry")
-    _check(lib().lpmm_sgdm4_step(state.handle, _ptr_array(params), _ptr_array(grads), _grad_dtype(grads), lr, beta,
-                                 _stream_ptr(stream)), "lpmm_sgdm4_step")
+    with torch.cuda.device(state.arena.device):
+        _check(lib().lpmm_sgdm4_step(state.handle, _ptr_array(params), _ptr_array(grads), _grad_dtype(grads), lr, beta,
+                                     _stream_ptr(stream)), "lpmm_sgdm4_step")
 
 
 def make_ptr_cache(params, grads):
@@ -252,6 +254,7 @@ def adamw4_step_host(state: State, h_params, h_grads, d_param_stage, d_grad_stag
                      weight_decay, step, stream=None) -> None:
     """lpmm_adamw4_step_host: params/grads are HOST tensors (pinned for asynchronous copies)."""
     gd = _grad_dtype(h_grads)
+    torch.cuda.set_device(state.arena.device)
     _check(lib().lpmm_adamw4_step_host(state.handle, _ptr_array(h_params), _ptr_array(h_grads), gd, lr, beta1,
                                        beta2, eps, weight_decay, step, d_param_stage.data_ptr(),
                                        d_grad_stage.data_ptr(), min(d_param_stage.numel() * d_param_stage.element_size(),
