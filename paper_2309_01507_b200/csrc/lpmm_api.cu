@@ -175,6 +175,10 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
     int64_t target = total_elems / (4LL * sms * occ2);
     int64_t tile_elems = 2048;
     while (tile_elems * 2 <= target && tile_elems < 131072) tile_elems *= 2;
+    if (const char* v = std::getenv("LPMM_TILE_ELEMS")) {   // development switch
+        const long x = std::atol(v);
+        if (x >= 2048 && x <= (1 << 20)) tile_elems = x;
+    }
 
     std::vector<TensorDesc> descs(n);
     std::vector<int32_t> t1(n + 1, 0), t2(n + 1, 0), t3(n + 1, 0);
@@ -289,6 +293,9 @@ lpmm_status make_state(const lpmm_config* cfg, const lpmm_shape* shapes, int32_t
                 e = cudaMemsetAsync(st->arena + t.m_codes + t.numel / 2, 0x07, 1, s);
         }
         if (e != cudaSuccess) rc = cuda_fail(e);
+    } else {   // an attached arena keeps its states; the header block (status word, tile counters) starts clean
+        const cudaError_t e = cudaMemsetAsync(d_arena, 0, kAlign, s);
+        if (e != cudaSuccess) rc = cuda_fail(e);
     }
     if (rc == LPMM_OK) rc = build_tables(st, s);
     if (rc != LPMM_OK) { delete st; return rc; }
@@ -364,6 +371,7 @@ StepArgs make_args(const lpmm_state* st, float lr, float beta1, float beta2, flo
     a.phase = st->phase;
     a.variant = st->pass2_variant;
     a.dev_status = reinterpret_cast<uint32_t*>(st->arena);
+    a.tile_counter = reinterpret_cast<int32_t*>(st->arena + 16);   // header block: [status | .. | counters]
     a.h.lr = lr; a.h.beta1 = beta1; a.h.beta2 = beta2; a.h.eps = eps;
     a.h.omb1 = 1.0f - beta1;
     a.h.omb2 = 1.0f - beta2;

@@ -26,6 +26,33 @@ __device__ __forceinline__ int find_tensor(const int32_t* __restrict__ start, in
     return lo;
 }
 
+// ---- tile hand-out --------------------------------------------------------------------------------
+//
+// The CTAs of a launch take tiles from a counter in the arena header in the order they become free, so an SM
+// that gets less memory bandwidth than its neighbours simply takes fewer tiles (with a fixed stride the whole
+// launch waits for the slowest SM). Thread 0 asks for the next index while the current tile is processed and
+// publishes it through one of two shared words; the CTA that finishes last puts both counters back to zero for
+// the next launch on the stream.
+
+__device__ __forceinline__ int tiles_first(int32_t* ctr, int* s_next) {
+    if (threadIdx.x == 0) s_next[0] = atomicAdd(ctr, 1);
+    __syncthreads();
+    return s_next[0];
+}
+__device__ __forceinline__ int tiles_fetch(int32_t* ctr) { return threadIdx.x == 0 ? atomicAdd(ctr, 1) : 0; }
+__device__ __forceinline__ int tiles_next(int* s_next, int& buf, int fetched) {
+    buf ^= 1;
+    if (threadIdx.x == 0) s_next[buf] = fetched;
+    __syncthreads();
+    return s_next[buf];
+}
+__device__ __forceinline__ void tiles_done(int32_t* ctr) {
+    if (threadIdx.x == 0) {
+        __threadfence();
+        if (atomicAdd(ctr + 1, 1) == (int)gridDim.x - 1) { ctr[0] = 0; ctr[1] = 0; }
+    }
+}
+
 // ---- 8-element loads ------------------------------------------------------------------------
 
 __device__ __forceinline__ void load8_f32(const float* p, float (&x)[8]) {
@@ -675,7 +702,10 @@ __global__ void __launch_bounds__(kThreads, 2) pass2_kernel(StepArgs a) {
     const LaneTables lt = make_lane_tables();
     const Hyper2& h2 = a.h2;
     uint32_t red_step = 0;
-    for (int tile = a.tile_begin + blockIdx.x; tile < a.tile_end; tile += gridDim.x) {
+    __shared__ int s_next[2];
+    int buf = 0;
+    for (int tile = a.tile_begin + tiles_first(a.tile_counter, s_next); tile < a.tile_end;) {
+        const int fetched = tiles_fetch(a.tile_counter);
         const int t = find_tensor(a.tile_start, a.n_tensors, tile);
         const TensorDesc d = a.descs[t];   // by value: the fields stay in registers across the stores below
         float* w = a.params[t];
@@ -692,7 +722,9 @@ __global__ void __launch_bounds__(kThreads, 2) pass2_kernel(StepArgs a) {
             case K_BLOCK:      pass2_flat<BF16, false, EXACT, MSHIFT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
             default:           pass2_fp32<BF16, EXACT>(d, w, g, local, a.h); break;
         }
+        tile = a.tile_begin + tiles_next(s_next, buf, fetched);
     }
+    tiles_done(a.tile_counter);
 }
 
 template <bool BF16, bool EXACT, int MSHIFT>
@@ -716,7 +748,10 @@ __global__ void __launch_bounds__(kThreads, 2) pass2_bulk_kernel(StepArgs a) {
     const LaneTables lt = make_lane_tables();
     const Hyper2& h2 = a.h2;
     uint32_t red_step = 0;
-    for (int tile = a.tile_begin + blockIdx.x; tile < a.tile_end; tile += gridDim.x) {
+    __shared__ int s_next[2];
+    int buf = 0;
+    for (int tile = a.tile_begin + tiles_first(a.tile_counter, s_next); tile < a.tile_end;) {
+        const int fetched = tiles_fetch(a.tile_counter);
         const int t = find_tensor(a.tile_start, a.n_tensors, tile);
         const TensorDesc d = a.descs[t];
         float* w = a.params[t];
@@ -731,7 +766,9 @@ __global__ void __launch_bounds__(kThreads, 2) pass2_bulk_kernel(StepArgs a) {
             case K_BLOCK:      pass2_flat<BF16, false, EXACT, MSHIFT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
             default:           pass2_fp32<BF16, EXACT>(d, w, g, local, a.h); break;
         }
+        tile = a.tile_begin + tiles_next(s_next, buf, fetched);
     }
+    tiles_done(a.tile_counter);
 }
 
 // ---- pass 1: new row / column maxima of v_t for rank-1 tensors -----------------------------------
@@ -1001,7 +1038,10 @@ __global__ void __launch_bounds__(kThreads, 3) pass1_kernel(StepArgs a) {
     __shared__ float s_col[kWarps * kWarpElems];
     const LaneTables lt = make_lane_tables();
     const Hyper2& h2 = a.h2;
-    for (int tile = a.tile_begin + blockIdx.x; tile < a.tile_end; tile += gridDim.x) {
+    __shared__ int s_next[2];
+    int buf = 0;
+    for (int tile = a.tile_begin + tiles_first(a.tile_counter, s_next); tile < a.tile_end;) {
+        const int fetched = tiles_fetch(a.tile_counter);
         const int t = find_tensor(a.tile_start, a.n_tensors, tile);
         const TensorDesc d = a.descs[t];
         const void* g = a.grads[t];
@@ -1009,7 +1049,9 @@ __global__ void __launch_bounds__(kThreads, 3) pass1_kernel(StepArgs a) {
         if (d.kind == K_RANK1_FAST) pass1_rank1_fast<BF16>(d, g, local, a.phase, h2, lt, s_col);
         else if (d.kind == K_FACT) pass1_fact<BF16>(d, g, local, a.phase, s_col);
         else pass1_rank1_flat<BF16>(d, g, local, a.phase, a.h);
+        tile = a.tile_begin + tiles_next(s_next, buf, fetched);
     }
+    tiles_done(a.tile_counter);
 }
 
 // ---- compressed SGDM (Alg. 2): m = beta m + g ; w = w - lr m ; compress m. One pass, element-indexed -------
@@ -1024,7 +1066,10 @@ __global__ void __launch_bounds__(kThreads, 3) sgdm_kernel(StepArgs a) {
     const Hyper2& h2 = a.h2;          // beta1 = momentum, neg_step = -lr, one = 1
     uint32_t red_step = 0;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    for (int tile = a.tile_begin + blockIdx.x; tile < a.tile_end; tile += gridDim.x) {
+    __shared__ int s_next[2];
+    int buf = 0;
+    for (int tile = a.tile_begin + tiles_first(a.tile_counter, s_next); tile < a.tile_end;) {
+        const int fetched = tiles_fetch(a.tile_counter);
         const int t = find_tensor(a.tile_start, a.n_tensors, tile);
         const TensorDesc d = a.descs[t];
         float* w = a.params[t];
@@ -1076,7 +1121,9 @@ __global__ void __launch_bounds__(kThreads, 3) sgdm_kernel(StepArgs a) {
                 if (full) store8_f32(d.m32 + e, mt); else store8_guard(d.m32, e, d.numel, mt);
             }
         }
+        tile = a.tile_begin + tiles_next(s_next, buf, fetched);
     }
+    tiles_done(a.tile_counter);
 }
 
 __global__ void rcp_kernel(const float* __restrict__ src, float* __restrict__ dst, int64_t n) {
