@@ -110,6 +110,7 @@ struct Hyper2 {
     float2 beta1, omb1, beta2, omb2;
     float2 rbc2, eps, neg_step, decay, one;
     float2 c16, cm15, magic;   // 16, -1.5 and 2^23 for the linear quantizer
+    float2 lin_a01, lin_a23, lin_b01, lin_b23;   // see lin_dequant8()
 };
 __host__ __device__ __forceinline__ float2 splat(float x) { return make_float2(x, x); }
 
@@ -151,7 +152,23 @@ __host__ __device__ __forceinline__ Hyper2 make_hyper2(const Hyper& h) {
     p.rbc2 = splat(h.rbc2); p.eps = splat(h.eps); p.neg_step = splat(-h.step_size); p.decay = splat(h.decay);
     p.one = splat(h.one);
     p.c16 = splat(16.0f); p.cm15 = splat(-1.5f); p.magic = splat(8388608.0f);
+    // a_k = 2^-(4k+4), b_k = 2^-4 - 2^(19-4k): (2^23 + q 16^k) a_k + b_k = (q + 1)/16 exactly
+    p.lin_a01 = make_float2(0.0625f, 0.00390625f);
+    p.lin_a23 = make_float2(0.000244140625f, 0.0000152587890625f);
+    p.lin_b01 = make_float2(0.0625f - 524288.0f, 0.0625f - 32768.0f);
+    p.lin_b23 = make_float2(0.0625f - 2048.0f, 0.0625f - 128.0f);
     return p;
+}
+// T_lin(q) = (q + 1)/16 (App. D.2) for the eight codes of one word, without a table: a nibble at bit 4k
+// (k <= 3), OR-ed into the mantissa of 2^23, is the number 2^23 + q 16^k, and one fused multiply-add maps it
+// to (q + 1)/16. Every intermediate and the result are exactly representable, so nothing is rounded.
+// t[i] holds the entries of elements 2i and 2i + 1.
+__device__ __forceinline__ void lin_dequant8(uint32_t q, const Hyper2& h, float2 (&t)[4]) {
+    const uint32_t hi = q >> 16;
+    t[0] = fma2_rn(make_float2(__uint_as_float(kMagicBits | (q & 0xfu)), __uint_as_float(kMagicBits | (q & 0xf0u))), h.lin_a01, h.lin_b01);
+    t[1] = fma2_rn(make_float2(__uint_as_float(kMagicBits | (q & 0xf00u)), __uint_as_float(kMagicBits | (q & 0xf000u))), h.lin_a23, h.lin_b23);
+    t[2] = fma2_rn(make_float2(__uint_as_float(kMagicBits | (hi & 0xfu)), __uint_as_float(kMagicBits | (hi & 0xf0u))), h.lin_a01, h.lin_b01);
+    t[3] = fma2_rn(make_float2(__uint_as_float(kMagicBits | (hi & 0xf00u)), __uint_as_float(kMagicBits | (hi & 0xf000u))), h.lin_a23, h.lin_b23);
 }
 // Both products must be rounded before the sum (Eq. 1 evaluated operation by operation). The assembler
 // was observed to merge a packed multiply with a following packed add into a fused multiply-add even with

@@ -135,7 +135,7 @@ __device__ __forceinline__ float update_param(float w, float mt, float vt, const
 // index is the code (shuffle width 16 takes the source lane modulo 16, so the nibble needs no masking).
 struct LaneTables {
     float de;    // T_DE[lane & 15]
-    float lin;   // (lane & 15 + 1) / 16
+    float lin;   // (lane & 15 + 1) / 16 (the maxima pass looks second-moment codes up with a shuffle)
     unsigned mask;   // the 16 lanes of this lane's group
 };
 __device__ __forceinline__ LaneTables make_lane_tables() {
@@ -155,6 +155,8 @@ __device__ __forceinline__ void moments_and_update8(float (&w)[8], const float (
                                                     float m_prod, const float (&vs)[8], const Hyper& h,
                                                     const Hyper2& h2, const LaneTables& lt, float (&mt)[8],
                                                     float (&vt)[8]) {
+    float2 tlin[4];
+    if (!FACT) lin_dequant8(qv, h2, tlin);
 #pragma unroll
     for (int k = 0; k < 8; k += 2) {
         const float2 m = make_float2(__shfl_sync(lt.mask, m_prod, (int)(qm >> (4 * k)), 16),
@@ -165,9 +167,7 @@ __device__ __forceinline__ void moments_and_update8(float (&w)[8], const float (
         if (FACT) {
             v2 = make_float2(vs[k], vs[k + 1]);
         } else {
-            const float2 tl = make_float2(__shfl_sync(lt.mask, lt.lin, (int)(qv >> (4 * k)), 16),
-                                          __shfl_sync(lt.mask, lt.lin, (int)(qv >> (4 * k + 4)), 16));
-            v2 = ema_v2(mul2_rn(tl, make_float2(vs[k], vs[k + 1])), g2, h2);
+            v2 = ema_v2(mul2_rn(tlin[k >> 1], make_float2(vs[k], vs[k + 1])), g2, h2);
         }
         mt[k] = m2.x; mt[k + 1] = m2.y;
         vt[k] = v2.x; vt[k + 1] = v2.y;
@@ -834,6 +834,8 @@ __device__ __forceinline__ float p1_process_row(const P1Row<BF16>& b, float r_ol
     float rm = 0.0f;
 #pragma unroll
     for (int k = 0; k < 8; k += 2) {
+        // (this pass is bound by the logic/min-max pipe, so the table entry comes from a shuffle here, not from
+        // the arithmetic of lin_dequant8() as in the update pass, which is short of shuffle/shared-memory slots)
         const float2 tl = make_float2(__shfl_sync(0xffffffffu, lt.lin, (int)(b.qv >> (4 * k)), 16),
                                       __shfl_sync(0xffffffffu, lt.lin, (int)(b.qv >> (4 * k + 4)), 16));
         const float2 sc = make_float2(fminf(r_old, c_old[k]), fminf(r_old, c_old[k + 1]));
