@@ -174,7 +174,7 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
     // aim at >= 4 tiles per resident CTA, tiles between 2 Ki and 128 Ki elements (powers of two)
     int64_t target = total_elems / (4LL * sms * occ2);
     int64_t tile_elems = 2048;
-    while (tile_elems * 2 <= target && tile_elems < 131072) tile_elems *= 2;
+    while (tile_elems * 2 <= target && tile_elems < 262144) tile_elems *= 2;
     if (const char* v = std::getenv("LPMM_TILE_ELEMS")) {   // development switch
         const long x = std::atol(v);
         if (x >= 2048 && x <= (1 << 20)) tile_elems = x;
