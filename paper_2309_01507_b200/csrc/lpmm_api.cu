@@ -383,8 +383,19 @@ StepArgs make_args(const lpmm_state* st, float lr, float beta1, float beta2, flo
     a.h.one = 1.0f;
     a.h.step_size = (float)((double)lr / bc1);
     a.h.rbc2 = (float)(1.0 / bc2);
+    const double step_size = (double)lr / bc1;
+    a.h.upd_c1 = step_size > 0.0 ? (float)(-std::sqrt(1.0 / bc2) / step_size) : 0.0f;
+    a.h.upd_e1 = step_size > 0.0 ? (float)(-(double)eps / step_size) : 0.0f;
     a.h2 = make_hyper2(a.h);
     return a;
+}
+
+// The approximate update flushes a denormal v^ before the square root (only safe with a real eps) and divides its
+// constants by the step size (only possible when that is a normal number): otherwise Eq. 1 is evaluated as written.
+bool wants_ieee_update(const lpmm_state* st, const Hyper& h) {
+    if (st->cfg.update_math == LPMM_UPDATE_IEEE) return true;
+    if (h.eps < 1e-30f || h.step_size < 1e-30f) return true;
+    return !(std::isfinite(h.upd_c1) && std::isfinite(h.upd_e1));
 }
 
 // Enqueues the three kernels of one step for tensors [t0, t1). ev (4 events or nullptr) brackets the kernels.
@@ -451,8 +462,7 @@ lpmm_status lpmm_adamw4_step(lpmm_state* st, void* const* d_params, const void* 
             st->prof_events.push_back(ev[k]);
         }
     }
-    // the approximate update flushes a denormal v^ before the square root: only safe with a real eps
-    const bool ieee_update = (st->cfg.update_math == LPMM_UPDATE_IEEE) || eps < 1e-30f;
+    const bool ieee_update = wants_ieee_update(st, a.h);
     int32_t launches = 0;
     rc = enqueue_range(st, a, 0, st->n, grad_dtype == LPMM_BF16, ieee_update, s, st->profile ? ev : nullptr, &launches);
     if (rc != LPMM_OK) return rc;
@@ -532,7 +542,7 @@ lpmm_status lpmm_adamw4_step_host(lpmm_state* st, void* const* h_params, const v
     rc = set_pointers(st, dp.data(), dg.data(), s);
     if (rc != LPMM_OK) return rc;
     const StepArgs a = make_args(st, lr, beta1, beta2, eps, weight_decay, step);
-    const bool ieee_update = (st->cfg.update_math == LPMM_UPDATE_IEEE) || eps < 1e-30f;
+    const bool ieee_update = wants_ieee_update(st, a.h);
 
     LPMM_CUDA(cudaEventRecord(ev_start, s));                       // earlier work on the caller's stream comes first
     LPMM_CUDA(cudaStreamWaitEvent(st->copy_in, ev_start, 0));

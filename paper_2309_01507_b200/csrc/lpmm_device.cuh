@@ -102,13 +102,15 @@ struct Hyper {
     float step_size;   // lr / bc1, evaluated in binary64 and rounded once (fast update)
     float rbc2;        // 1 / bc2, likewise
     float one;         // 1.0f, passed as data (see ema_m2)
+    float upd_c1;      // -sqrt(1 / bc2) / step_size and
+    float upd_e1;      // -eps / step_size (binary64 on the host, rounded once): see adam_update_fast2()
 };
 
 // The same constants as pairs, for the packed two-lane fp32 instructions of sm_100 (mul/add/fma.f32x2:
 // two independent IEEE operations per instruction, so results are bit-identical to the scalar forms).
 struct Hyper2 {
     float2 beta1, omb1, beta2, omb2;
-    float2 rbc2, eps, neg_step, decay, one;
+    float2 rbc2, eps, neg_step, decay, one, upd_c1, upd_e1;
     float2 c16, cm15, magic;   // 16, -1.5 and 2^23 for the linear quantizer
     float2 lin_a01, lin_a23, lin_b01, lin_b23;   // see lin_dequant8()
 };
@@ -150,7 +152,7 @@ __host__ __device__ __forceinline__ Hyper2 make_hyper2(const Hyper& h) {
     Hyper2 p;
     p.beta1 = splat(h.beta1); p.omb1 = splat(h.omb1); p.beta2 = splat(h.beta2); p.omb2 = splat(h.omb2);
     p.rbc2 = splat(h.rbc2); p.eps = splat(h.eps); p.neg_step = splat(-h.step_size); p.decay = splat(h.decay);
-    p.one = splat(h.one);
+    p.one = splat(h.one); p.upd_c1 = splat(h.upd_c1); p.upd_e1 = splat(h.upd_e1);
     p.c16 = splat(16.0f); p.cm15 = splat(-1.5f); p.magic = splat(8388608.0f);
     // a_k = 2^-(4k+4), b_k = 2^-4 - 2^(19-4k): (2^23 + q 16^k) a_k + b_k = (q + 1)/16 exactly
     p.lin_a01 = make_float2(0.0625f, 0.00390625f);
@@ -180,16 +182,18 @@ __device__ __forceinline__ float2 ema_m2(float2 m, float2 g, const Hyper2& h) {
 __device__ __forceinline__ float2 ema_v2(float2 v, float2 g, const Hyper2& h) {
     return fma2_rn(mul2_rn(h.beta2, v), h.one, mul2_rn(h.omb2, mul2_rn(g, g)));
 }
-// adam_update_fast() on a pair (the two approximate special-function calls stay scalar).
+// adam_update_fast() on a pair, with the constants folded on the host so that three packed operations and the
+// two approximate special functions remain:
+//   -step / (sqrt(v_t / bc2) + eps) = 1 / (sqrt(v_t) * c1 + e1),  c1 = -sqrt(1 / bc2) / step,  e1 = -eps / step.
+// The host falls back to adam_update() when step is (almost) zero, where c1 and e1 do not exist.
 __device__ __forceinline__ float2 adam_update_fast2(float2 w, float2 mt, float2 vt, const Hyper2& h) {
-    const float2 vh = mul2_rn(vt, h.rbc2);
     float2 sq, rc;
-    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(sq.x) : "f"(vh.x));
-    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(sq.y) : "f"(vh.y));
-    const float2 den = add2_rn(sq, h.eps);
+    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(sq.x) : "f"(vt.x));
+    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(sq.y) : "f"(vt.y));
+    const float2 den = fma2_rn(sq, h.upd_c1, h.upd_e1);
     asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rc.x) : "f"(den.x));
     asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rc.y) : "f"(den.y));
-    return fma2_rn(w, h.decay, mul2_rn(mul2_rn(mt, h.neg_step), rc));
+    return fma2_rn(w, h.decay, mul2_rn(mt, rc));
 }
 
 // Eq. 1 moment updates; separate roundings, in the order written there.
