@@ -237,6 +237,26 @@ def adamw4_step(w: np.ndarray, g: np.ndarray, st: TensorState, *, lr, beta1, bet
         raise ValueError("lpmm_oracle_adamw4_step rejected its arguments")
 
 
+def adamw4_step_nd(w: np.ndarray, g: np.ndarray, dims, m_block: int, m_codes: np.ndarray, m_scale: np.ndarray,
+                   v_codes: np.ndarray, mu_flat: np.ndarray, *, lr, beta1, beta2, eps, weight_decay, step: int,
+                   true_division: bool = False) -> None:
+    """One compressed AdamW step on a tensor of any rank with the general rank-1 normalization of Alg. 4;
+    w, the codes, m_scale and mu_flat (per-axis maxima, concatenated) are updated in place."""
+    dims = np.asarray(dims, np.int64)
+    numel = int(np.prod(dims))
+    assert w.dtype == np.float32 and w.flags.c_contiguous and w.size == numel
+    assert m_codes.dtype == np.uint8 and v_codes.dtype == np.uint8 and m_codes.size == (numel + 1) // 2 == v_codes.size
+    assert m_scale.dtype == np.float32 and m_scale.size == (numel + m_block - 1) // m_block
+    assert mu_flat.dtype == np.float32 and mu_flat.size == int(dims.sum())
+    g = _f32(g)
+    assert g.size == numel
+    h = _Hyper(lr, beta1, beta2, eps, weight_decay, step, int(true_division))
+    rc = lib().lpmm_oracle_adamw4_step_nd(_p(w), _p(g), C.c_int(len(dims)), _p(dims), C.c_int64(m_block), _p(m_codes),
+                                          _p(m_scale), _p(v_codes), _p(mu_flat), C.byref(h))
+    if rc != 0:
+        raise ValueError("lpmm_oracle_adamw4_step_nd rejected its arguments")
+
+
 def sgdm4_step(w: np.ndarray, g: np.ndarray, st: TensorState, *, lr, beta, true_division: bool = False) -> None:
     """One compressed SGDM step (Alg. 2) on one tensor; only the first-moment part of `st` is used."""
     assert w.dtype == np.float32 and w.flags.c_contiguous and w.size == st.numel

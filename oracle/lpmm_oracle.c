@@ -350,6 +350,67 @@ int lpmm_oracle_adamw4_step(float* w, const float* g, int64_t rows, int64_t cols
     return 0;
 }
 
+/* ------------------------------------------------------------------ Alg. 3 on a tensor of any rank (Alg. 4) */
+
+int lpmm_oracle_adamw4_step_nd(float* w, const float* g, int ndim, const int64_t* dims, int64_t m_block,
+                               uint8_t* m_codes, float* m_scale, uint8_t* v_codes, float* mu_flat,
+                               const lpmm_oracle_hyper* h) {
+    if (!w || !g || !h || !dims || ndim < 1 || ndim > 16 || h->step < 1) return -1;
+    int64_t numel = 1;
+    for (int r = 0; r < ndim; ++r) { if (dims[r] <= 0) return -1; numel *= dims[r]; }
+    const float beta1 = h->beta1, beta2 = h->beta2;
+    const float omb1 = 1.0f - beta1, omb2 = 1.0f - beta2;
+    const float bc1 = (float)(1.0 - pow((double)beta1, (double)h->step));
+    const float bc2 = (float)(1.0 - pow((double)beta2, (double)h->step));
+    const float decay = 1.0f - h->lr * h->weight_decay;
+    float* m = (float*)malloc(sizeof(float) * (size_t)numel);
+    float* v = (float*)malloc(sizeof(float) * (size_t)numel);
+    float* M = (float*)malloc(sizeof(float) * (size_t)numel);
+    uint8_t* q = (uint8_t*)malloc((size_t)numel);
+    if (!m || !v || !M || !q) { free(m); free(v); free(M); free(q); return -1; }
+    float Tde[16], Tlin[16];
+    lpmm_oracle_de_map(4, 1, 0, Tde);
+    lpmm_oracle_linear_map(4, Tlin);
+
+    /* decompress: m block-wise; v with the scale field M_i = min_r mu_r[Phi(i)_r] of the stored statistics */
+    lpmm_oracle_unpack4(m_codes, numel, q);
+    lpmm_oracle_dequantize_block(q, numel, m_block, Tde, m_scale, m);
+    lpmm_oracle_unpack4(v_codes, numel, q);
+    lpmm_oracle_rank1_scale_field(ndim, dims, mu_flat, M);
+    for (int64_t i = 0; i < numel; ++i) v[i] = Tlin[q[i]] * M[i];
+
+    /* Eq. 1 with the decoupled decay, operation by operation as in lpmm_oracle_adamw4_step */
+    for (int64_t i = 0; i < numel; ++i) {
+        float gi = g[i];
+        float a = beta1 * m[i];
+        float b = omb1 * gi;
+        float mt = a + b;
+        float gg = gi * gi;
+        float c = beta2 * v[i];
+        float d = omb2 * gg;
+        float vt = c + d;
+        float mhat = mt / bc1;
+        float vhat = vt / bc2;
+        float denom = sqrtf(vhat) + h->eps;
+        float ratio = mhat / denom;
+        float upd = h->lr * ratio;
+        float wd = w[i] * decay;
+        w[i] = wd - upd;
+        m[i] = mt;
+        v[i] = vt;
+    }
+
+    /* compress: new per-axis maxima (Alg. 4, first loop), their scale field (second loop), nearest codes */
+    lpmm_oracle_quantize_block(m, numel, m_block, Tde, 16, 0, h->true_division, m_scale, q);
+    lpmm_oracle_pack4(q, numel, m_codes);
+    lpmm_oracle_rank1_stats(v, ndim, dims, mu_flat);
+    lpmm_oracle_rank1_scale_field(ndim, dims, mu_flat, M);
+    lpmm_oracle_map_codes(v, M, numel, Tlin, 16, h->true_division, q);
+    lpmm_oracle_pack4(q, numel, v_codes);
+    free(m); free(v); free(M); free(q);
+    return 0;
+}
+
 /* ------------------------------------------------------------------ factorized second moment (Sec. 4.3) */
 
 int lpmm_oracle_adamw4_factor_step(float* w, const float* g, int64_t rows, int64_t cols, int64_t m_block,

@@ -115,6 +115,15 @@ int lpmm_oracle_adamw4_step(float* w, const float* g, int64_t rows, int64_t cols
                             float* m32, float* v32,
                             const lpmm_oracle_hyper* h);
 
+/* The same step on a tensor of any rank p >= 1 (row-major dims[0..p-1]) whose second moment uses rank-1
+ * normalization in the general form of Alg. 4: mu_flat holds the per-axis maxima mu_1 (dims[0] values), mu_2, ...
+ * of the stored second moment; the scale of element i is M_i = min_r mu_r[Phi(i)_r] and n_i = v_i * rcp(M_i).
+ * The first moment is compressed block-wise over the flattened tensor. With p = 2 this is the RANK1 case of
+ * lpmm_oracle_adamw4_step (mu_1 = r, mu_2 = c). Returns 0, or -1 on a bad argument. */
+int lpmm_oracle_adamw4_step_nd(float* w, const float* g, int ndim, const int64_t* dims, int64_t m_block,
+                               uint8_t* m_codes, float* m_scale, uint8_t* v_codes, float* mu_flat,
+                               const lpmm_oracle_hyper* h);
+
 /* Initial compressed state s_0 = 0 (Alg. 1): m codes all "the entry 0" of the signed DE table,
  * v codes 0, every scale 0. */
 void lpmm_oracle_state_init(int64_t rows, int64_t cols, int kind, int64_t m_block, int64_t v_block,

@@ -210,6 +210,34 @@ def adamw4_step(w, g, state: dict, *, lr, beta1, beta2, eps, weight_decay, step,
     return w_new.astype(F32)
 
 
+def adamw4_step_nd(w, g, state: dict, *, lr, beta1, beta2, eps, weight_decay, step):
+    """Alg. 3 on a tensor of any rank with Alg. 4's normalization for the second moment.
+
+    state: {"dims", "m_block", "m_codes", "m_scale", "v_codes", "mu": [per-axis maxima]}; returns the new w (flat).
+    """
+    dims = tuple(int(d) for d in state["dims"])
+    numel = int(np.prod(dims))
+    w = np.asarray(w, F32).ravel()
+    g = np.asarray(g, F32).ravel()
+    lr, beta1, beta2, eps, wd = F32(lr), F32(beta1), F32(beta2), F32(eps), F32(weight_decay)
+    Tde, Tlin = de_map(4, True), linear_map(4)
+    m = dequantize_block(unpack4(state["m_codes"], numel), state["m_block"], Tde, state["m_scale"])
+    v = (Tlin[unpack4(state["v_codes"], numel)] * rank1_scale_field(dims, state["mu"]).ravel()).astype(F32)
+    omb1, omb2 = F32(1.0) - beta1, F32(1.0) - beta2
+    bc1 = F32(1.0 - float(beta1) ** step)
+    bc2 = F32(1.0 - float(beta2) ** step)
+    mt = beta1 * m + omb1 * g
+    vt = beta2 * v + omb2 * (g * g)
+    upd = lr * ((mt / bc1) / (np.sqrt(vt / bc2) + eps))
+    w_new = w * (F32(1.0) - lr * wd) - upd
+    qm, state["m_scale"] = quantize_block(mt, state["m_block"], Tde)
+    state["m_codes"] = pack4(qm)
+    state["mu"] = rank1_stats(vt.reshape(dims))
+    M = rank1_scale_field(dims, state["mu"]).ravel()
+    state["v_codes"] = pack4(nearest(Tlin, vt * rcp(M)))
+    return w_new.astype(F32)
+
+
 def sgdm4_step(w, g, state: dict, *, lr, beta, true_division=False):
     """Alg. 2 (compressed SGDM) on one tensor: m = beta m + g ; w = w - lr m ; compress m (B/DE)."""
     numel = state["rows"] * state["cols"]
