@@ -62,10 +62,15 @@ typedef enum { LPMM_UPDATE_FAST = 0, LPMM_UPDATE_IEEE = 1 } lpmm_update_math;
 /* lpmm_quantize flags */
 #define LPMM_Q_GIVEN_SCALES 1u /* use the scales already in d_scale0/d_scale1 instead of recomputing them */
 
+#define LPMM_MAX_NDIM 4
 typedef struct {
-    int64_t rows, cols; /* ndim 1: rows = numel, cols = 1; ndim 2: rows x cols, row-major */
-    int32_t ndim;       /* 1 or 2 */
+    int64_t rows, cols; /* ndim 1: rows = numel, cols = 1; ndim 2: rows x cols, row-major;
+                           ndim >= 3: rows = product of the leading extents, cols = the last extent */
+    int32_t ndim;       /* 1 .. LPMM_MAX_NDIM */
     uint32_t flags;
+    int64_t dims[LPMM_MAX_NDIM]; /* ndim >= 3: the extents, row-major (read only then; rows and cols must agree
+                                    with them). Such tensors use the general rank-1 normalization of Alg. 4 (App. G):
+                                    one vector of maxima per axis, scale of an element = the minimum over its axes. */
 } lpmm_shape;
 
 typedef struct {
@@ -197,6 +202,12 @@ lpmm_status lpmm_state_view(const lpmm_state* st, int32_t tensor, int32_t* kind,
                             const uint8_t** m_codes, const float** m_scale,
                             const uint8_t** v_codes, const float** v_scale0, const float** v_scale1,
                             const float** m32, const float** v32);
+
+/* Statistics of one axis of a tensor with rank-1 normalization (Alg. 4: mu_r, one maximum per index of axis r):
+ * *mu receives a device pointer into the arena, *extent the axis' length. axis counts the tensor's own axes
+ * (a matrix has axis 0 = r, axis 1 = c). The pointer is valid until the next step (the buffers alternate).
+ * LPMM_ERR_INVALID_ARG for tensors of another kind or an axis out of range. */
+lpmm_status lpmm_state_view_axis(const lpmm_state* st, int32_t tensor, int32_t axis, const float** mu, int64_t* extent);
 
 /* Reads the device-side error word of the state (synchronizes `stream`). 0 = no error; 1 = a bounded wait
  * for an asynchronous shared-memory copy inside a step kernel expired (the affected warp stopped early, so

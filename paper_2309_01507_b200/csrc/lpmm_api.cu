@@ -35,6 +35,9 @@ struct TensorLayout {
     size_t m_codes, m_scale, v_codes, v_bscale, m32, v32;  // byte offsets into the arena (0 = unused)
     int64_t rc_index;   // float index of this tensor's [r | c] inside each rank-1 scale buffer
     int32_t c_off;
+    int32_t n_outer = 1;            // leading axes (Alg. 4 in general form: ndim - 1)
+    int32_t outer_dim[3] = {0, 0, 0};
+    int32_t outer_off[3] = {0, 0, 0};
 };
 
 struct Layout {
@@ -66,12 +69,30 @@ lpmm_status validate_config(const lpmm_config* cfg, const lpmm_shape* shapes, in
     for (int32_t i = 0; i < n; ++i) {
         const lpmm_shape& s = shapes[i];
         if (s.rows <= 0 || s.cols <= 0) return LPMM_ERR_INVALID_ARG;
-        if (s.ndim != 1 && s.ndim != 2) return (s.ndim >= 3) ? LPMM_ERR_UNSUPPORTED : LPMM_ERR_INVALID_ARG;
+        if (s.ndim < 1) return LPMM_ERR_INVALID_ARG;
+        if (s.ndim > LPMM_MAX_NDIM) return LPMM_ERR_UNSUPPORTED;
         if (s.ndim == 1 && s.cols != 1) return LPMM_ERR_INVALID_ARG;
+        if (s.ndim >= 3) {   // rows, cols restate dims
+            int64_t lead = 1;
+            for (int32_t a = 0; a < s.ndim; ++a) {
+                if (s.dims[a] <= 0 || s.dims[a] > (int64_t)1 << 30) return LPMM_ERR_INVALID_ARG;
+                if (a + 1 < s.ndim) {
+                    if (lead > ((int64_t)1 << 40) / s.dims[a]) return LPMM_ERR_INVALID_ARG;
+                    lead *= s.dims[a];
+                }
+            }
+            if (lead != s.rows || s.dims[s.ndim - 1] != s.cols) return LPMM_ERR_INVALID_ARG;
+            if (cfg->v_mode == LPMM_V_FACTORED) return LPMM_ERR_UNSUPPORTED;   // Sec. 4.3 factorizes matrices
+        }
         if ((s.flags & LPMM_FORCE_QUANT) && (s.flags & LPMM_FORCE_FP32)) return LPMM_ERR_INVALID_ARG;
         if (s.rows > (int64_t)1 << 40 || s.cols > (int64_t)1 << 40 || s.rows > ((int64_t)1 << 40) / s.cols)
             return LPMM_ERR_INVALID_ARG;  // numel overflow guard
         if (s.rows + s.cols > (int64_t)1 << 30) return LPMM_ERR_UNSUPPORTED;
+        if (s.ndim >= 3) {
+            int64_t stats = 0;
+            for (int32_t a = 0; a < s.ndim; ++a) stats += s.dims[a] + 3;
+            if (stats > (int64_t)1 << 30) return LPMM_ERR_UNSUPPORTED;
+        }
         // the factorized second moment is built for the tiled path only: whole first-moment blocks inside a row
         if (cfg->v_mode == LPMM_V_FACTORED && choose_kind(*cfg, s) == K_RANK1_FLAT) return LPMM_ERR_UNSUPPORTED;
     }
@@ -85,6 +106,7 @@ int32_t choose_kind(const lpmm_config& cfg, const lpmm_shape& s) {
     if (s.ndim == 1 || s.rows == 1 || s.cols == 1 || cfg.v_mode == LPMM_V_BLOCK) return K_BLOCK;  // Sec. 4.2
     // the tiled path needs whole first-moment blocks inside a row (and, for B2048, one block per tile width)
     // the tiled path keeps 32-bit element offsets inside a tile: rows of at most 2^24 elements
+    if (s.ndim >= 3) return K_RANK1_FLAT;     // Alg. 4 with more than two axes: element-indexed path
     if (s.cols % cfg.m_block != 0 || s.cols > ((int64_t)1 << 24)) return K_RANK1_FLAT;   // (refused in the factorized mode)
     return (cfg.v_mode == LPMM_V_FACTORED) ? K_FACT : K_RANK1_FAST;
 }
@@ -106,7 +128,20 @@ void compute_layout(const lpmm_config& cfg, const lpmm_shape* shapes, int32_t n,
         t.kind = choose_kind(cfg, shapes[i]);
         if (uses_rc(t.kind)) {
             t.rc_index = rc;
-            t.c_off = (int32_t)((t.rows + 3) / 4 * 4);
+            if (shapes[i].ndim >= 3) {   // one vector of statistics per axis, each padded to 4 floats
+                t.n_outer = shapes[i].ndim - 1;
+                int64_t o = 0;
+                for (int32_t a = 0; a < t.n_outer; ++a) {
+                    t.outer_dim[a] = (int32_t)shapes[i].dims[a];
+                    t.outer_off[a] = (int32_t)o;
+                    o += (shapes[i].dims[a] + 3) / 4 * 4;
+                }
+                t.c_off = (int32_t)o;
+            } else {
+                t.n_outer = 1;
+                t.outer_dim[0] = (int32_t)t.rows;
+                t.c_off = (int32_t)((t.rows + 3) / 4 * 4);
+            }
             rc += t.c_off + (t.cols + 3) / 4 * 4;
             rc = (rc + 63) / 64 * 64;  // 256-byte granules so r and c always start 16-byte aligned
         }
@@ -188,6 +223,8 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
         TensorDesc& d = descs[i];
         std::memset(&d, 0, sizeof(d));
         d.rows = t.rows; d.cols = t.cols; d.numel = t.numel; d.kind = t.kind; d.c_off = t.c_off;
+        d.n_outer = t.n_outer;
+        for (int a = 0; a < 3; ++a) { d.outer_dim[a] = t.outer_dim[a]; d.outer_off[a] = t.outer_off[a]; }
         d.m_shift = (st->cfg.m_block == 2048) ? 11 : 7;
         int64_t tiles = 0;
         if (t.kind == K_FP32) {
@@ -636,6 +673,16 @@ lpmm_status lpmm_state_view(const lpmm_state* st, int32_t tensor, int32_t* kind,
     if (v_scale1) *v_scale1 = r1 ? rc + t.c_off : nullptr;
     if (m32) *m32 = q ? nullptr : reinterpret_cast<const float*>(A + t.m32);
     if (v32) *v32 = q ? nullptr : reinterpret_cast<const float*>(A + t.v32);
+    return LPMM_OK;
+}
+
+lpmm_status lpmm_state_view_axis(const lpmm_state* st, int32_t tensor, int32_t axis, const float** mu, int64_t* extent) {
+    if (!st || tensor < 0 || tensor >= st->n || !mu || !extent) return LPMM_ERR_INVALID_ARG;
+    const TensorLayout& t = st->L.t[tensor];
+    if (!uses_rc(t.kind) || axis < 0 || axis > t.n_outer) return LPMM_ERR_INVALID_ARG;
+    const float* rc = reinterpret_cast<const float*>(st->arena + st->L.rc[st->phase]) + t.rc_index;
+    if (axis < t.n_outer) { *mu = rc + t.outer_off[axis]; *extent = t.outer_dim[axis]; }
+    else { *mu = rc + t.c_off; *extent = t.cols; }
     return LPMM_OK;
 }
 

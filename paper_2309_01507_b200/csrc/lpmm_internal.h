@@ -36,7 +36,12 @@ struct TensorDesc {
     int32_t tile_rows;  // K_RANK1_FAST: rows per tile
     int32_t flat_chunks;  // other kinds: 256-element chunks per warp per tile
     int32_t m_shift;    // log2 of the first-moment block size: 7 (B128) or 11 (B2048)
-    int32_t pad;
+    // K_RANK1_FLAT, general form of Alg. 4: the tensor is [outer_dim[0] x .. x outer_dim[n_outer-1]] x cols,
+    // rows = the product of the leading extents. The statistics of leading axis a start at float outer_off[a]
+    // of rc[] / rcp_new (axis 0 at 0), those of the last axis at c_off. A matrix has n_outer = 1.
+    int32_t n_outer;
+    int32_t outer_dim[3];
+    int32_t outer_off[3];
 };
 
 struct StepArgs {

@@ -577,6 +577,36 @@ __device__ __forceinline__ void pass2_rank1_bulk(const TensorDesc& d, float* __r
     }
 }
 
+// ---- rank-1 normalization in the general form of Alg. 4 (element-indexed paths) --------------------
+//
+// The leading axes of the tensor are flattened into "rows". For row i the contribution of the leading axes to
+// an element's scale is the minimum of their statistics at the row's multi-index (for the reciprocals of the
+// new statistics: the maximum). A matrix has one leading axis and this is a single load.
+
+template <bool MAX>
+__device__ __forceinline__ float outer_stat(const TensorDesc& d, const float* __restrict__ base, int64_t i) {
+    if (d.n_outer == 1) return __ldg(base + i);
+    int64_t rem = i;
+    float s = MAX ? 0.0f : 3.402823466e38f;
+    for (int a = d.n_outer - 1; a >= 0; --a) {          // the last leading axis varies fastest
+        const int64_t q = rem / d.outer_dim[a];
+        const float x = __ldg(base + d.outer_off[a] + (rem - q * d.outer_dim[a]));
+        s = MAX ? fmaxf(s, x) : fminf(s, x);
+        rem = q;
+    }
+    return s;
+}
+// Publishes the maximum of a run of elements of row i to every leading axis.
+__device__ __forceinline__ void outer_publish(const TensorDesc& d, float* base, int64_t i, float x) {
+    if (d.n_outer == 1) { atomic_max_nonneg(base + i, x); return; }
+    int64_t rem = i;
+    for (int a = d.n_outer - 1; a >= 0; --a) {
+        const int64_t q = rem / d.outer_dim[a];
+        atomic_max_nonneg(base + d.outer_off[a] + (rem - q * d.outer_dim[a]), x);
+        rem = q;
+    }
+}
+
 // ---- pass 2, flat (element-indexed) tensors: block-wise v, or rank-1 with arbitrary cols ------
 
 template <bool BF16, bool RANK1, bool EXACT, int MSHIFT>
@@ -616,15 +646,22 @@ __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restric
         const float am = group_live ? d.m_scale[e >> MSHIFT] : 0.0f;
         if (RANK1) {
             int64_t i = e / d.cols, j = e - i * d.cols;
+            float so = 0.0f, ro = 0.0f;          // leading axes' share of the old scale / the new reciprocal, row i
+            bool fresh = true;
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
                 if (e + k < d.numel) {
-                    vs[k] = fminf(__ldg(rc_old + i), __ldg(rc_old + d.c_off + j));
-                    vr[k] = fmaxf(__ldg(rcp_new + i), __ldg(rcp_new + d.c_off + j));
+                    if (fresh) {
+                        so = outer_stat<false>(d, rc_old, i);
+                        ro = outer_stat<true>(d, rcp_new, i);
+                        fresh = false;
+                    }
+                    vs[k] = fminf(so, __ldg(rc_old + d.c_off + j));
+                    vr[k] = fmaxf(ro, __ldg(rcp_new + d.c_off + j));
                 } else {
                     vs[k] = 0.0f; vr[k] = 0.0f;
                 }
-                if (++j == d.cols) { j = 0; ++i; }
+                if (++j == d.cols) { j = 0; ++i; fresh = true; }
             }
         } else {
             const float av = lane_live ? d.v_bscale[e >> 7] : 0.0f;
@@ -1016,22 +1053,26 @@ __device__ __forceinline__ void pass1_rank1_flat(const TensorDesc& d, const void
         const uint32_t qv = load_codes_guard(d.v_codes, e, d.numel);
         int64_t i = e / d.cols, j = e - i * d.cols;
         float run = 0.0f;                      // maximum of the lane's current run of elements in row i
+        float so = 0.0f;                       // leading axes' share of the old scale in row i
+        bool fresh = true;
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
             if (e + k < d.numel) {
-                const float s = fminf(__ldg(rc_old + i), __ldg(rc_old + d.c_off + j));
+                if (fresh) { so = outer_stat<false>(d, rc_old, i); fresh = false; }
+                const float s = fminf(so, __ldg(rc_old + d.c_off + j));
                 const float vt = ema_v(__fmul_rn(lin_value((qv >> (4 * k)) & 15u), s), gv[k], h);
                 run = fmaxf(run, vt);
                 atomic_max_nonneg(rc_new + d.c_off + j, vt);
             }
             if (++j == d.cols) {               // the row ends inside the lane's elements: publish and start over
-                atomic_max_nonneg(rc_new + i, run);
+                outer_publish(d, rc_new, i, run);
                 run = 0.0f;
                 j = 0;
                 ++i;
+                fresh = true;
             }
         }
-        if (i < d.rows) atomic_max_nonneg(rc_new + i, run);
+        if (i < d.rows) outer_publish(d, rc_new, i, run);
     }
 }
 

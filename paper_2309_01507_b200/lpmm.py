@@ -29,13 +29,27 @@ KIND_FP32, KIND_BLOCK, KIND_RANK1, KIND_FACTORED = 0, 1, 2, 3
 EXPORTS = ("lpmm_state_bytes", "lpmm_state_init", "lpmm_state_attach", "lpmm_adamw4_step",
            "lpmm_adamw4_step_host", "lpmm_stage_bytes", "lpmm_quantize", "lpmm_dequantize",
            "lpmm_quantize_rank1_noalloc", "lpmm_sgdm4_step",
-           "lpmm_state_view", "lpmm_state_phase", "lpmm_state_last_launches", "lpmm_state_destroy",
+           "lpmm_state_view", "lpmm_state_view_axis", "lpmm_state_phase", "lpmm_state_last_launches", "lpmm_state_destroy",
            "lpmm_state_profile", "lpmm_state_profile_read", "lpmm_state_device_status",
            "lpmm_status_string", "lpmm_last_cuda_error")
 
 
+MAX_NDIM = 4
+
+
 class Shape(C.Structure):
-    _fields_ = [("rows", C.c_int64), ("cols", C.c_int64), ("ndim", C.c_int32), ("flags", C.c_uint32)]
+    _fields_ = [("rows", C.c_int64), ("cols", C.c_int64), ("ndim", C.c_int32), ("flags", C.c_uint32),
+                ("dims", C.c_int64 * MAX_NDIM)]
+
+
+def nd_shape(dims, flags: int = 0) -> Shape:
+    """Shape of a tensor with three or more axes (row-major extents): rows is the product of the leading ones."""
+    dims = [int(d) for d in dims]
+    rows = 1
+    for d in dims[:-1]:
+        rows *= d
+    arr = (C.c_int64 * MAX_NDIM)(*(dims + [0] * (MAX_NDIM - len(dims)))) if len(dims) <= MAX_NDIM else (C.c_int64 * MAX_NDIM)()
+    return Shape(rows, dims[-1], len(dims), flags, arr)
 
 
 class Config(C.Structure):
@@ -80,6 +94,7 @@ def lib():
         L.lpmm_dequantize.argtypes = [vp, vp, vp, i64, i64, i32, i32, i32, vp, vp]
         L.lpmm_quantize_rank1_noalloc.argtypes = [vp, i64, i64, vp, vp, vp, vp]
         L.lpmm_state_view.argtypes = [vp, i32, C.POINTER(i32)] + [C.POINTER(vp)] * 7
+        L.lpmm_state_view_axis.argtypes = [vp, i32, i32, C.POINTER(vp), C.POINTER(i64)]
         L.lpmm_state_profile.argtypes = [vp, i32]
         L.lpmm_state_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_double),
                                               C.POINTER(i32)]
@@ -120,7 +135,11 @@ def make_shapes(shapes) -> C.Array:
             items.append(Shape(rows, cols, ndim, flags))
         else:
             flags = FORCE_QUANT if getattr(s, "force_quant", False) else 0
-            items.append(Shape(s.rows, s.cols, s.ndim, flags))
+            dims = getattr(s, "dims", None)
+            if dims is not None and len(dims) >= 3:
+                items.append(nd_shape(dims, flags))
+            else:
+                items.append(Shape(s.rows, s.cols, s.ndim, flags))
     return (Shape * len(items))(*items)
 
 
@@ -327,8 +346,19 @@ def state_view(state: State, i: int) -> dict:
         "m_codes": view(ptrs[0], (numel + 1) // 2, torch.uint8),
         "m_scale": view(ptrs[1], 4 * nblk_m, torch.float32),
         "v_codes": view(ptrs[2], (numel + 1) // 2, torch.uint8),
-        "v_s0": view(ptrs[3], 4 * (sh.rows if k in (KIND_RANK1, KIND_FACTORED) else nblk_v), torch.float32),
+        # rank-1: the first axis' maxima (a matrix: r; three or more axes: see state_view_axis for the others)
+        "v_s0": view(ptrs[3], 4 * ((sh.dims[0] if sh.ndim >= 3 else sh.rows) if k in (KIND_RANK1, KIND_FACTORED) else nblk_v),
+                     torch.float32),
         "v_s1": view(ptrs[4], 4 * sh.cols, torch.float32),
         "m32": view(ptrs[5], 4 * numel, torch.float32),
         "v32": view(ptrs[6], 4 * numel, torch.float32),
     }
+
+
+def state_view_axis(state: State, tensor: int, axis: int) -> torch.Tensor:
+    """Per-axis maxima of a rank-1 tensor's second moment (Alg. 4), as a view into the arena."""
+    p = C.c_void_p()
+    n = C.c_int64()
+    _check(lib().lpmm_state_view_axis(state.handle, tensor, axis, C.byref(p), C.byref(n)), "lpmm_state_view_axis")
+    off = p.value - state.arena.data_ptr()
+    return state.arena[off:off + 4 * n.value].view(torch.float32)

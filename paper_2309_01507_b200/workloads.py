@@ -23,10 +23,11 @@ class TensorSpec:
     name: str
     rows: int
     cols: int
-    ndim: int                # 1 or 2 (ndim 1: rows = numel, cols = 1)
+    ndim: int                # 1 or 2 (ndim 1: rows = numel, cols = 1); with `dims`: their number
     init: str = "normal"     # "normal" N(0, 0.02^2), "ones", "zeros"
     force_quant: bool = False
     sparse_rows: float = 0.0  # fraction of gradient rows zeroed each step (token-sparse embeddings)
+    dims: tuple | None = None  # three or more axes (e.g. a convolution weight): rows = product of the leading extents
 
     @property
     def numel(self) -> int:
@@ -34,6 +35,8 @@ class TensorSpec:
 
     @property
     def shape(self):
+        if self.dims is not None:
+            return tuple(self.dims)
         return (self.rows,) if self.ndim == 1 else (self.rows, self.cols)
 
 
@@ -172,7 +175,7 @@ def make_grad(spec: TensorSpec, workload_index: int, tensor_index: int, step: in
     a = torch.exp(torch.randn(rows, 1, generator=fixed, dtype=torch.float32, device=device))
     g = torch.randn(rows, cols, generator=fresh, dtype=torch.float32, device=device)
     g *= a
-    if spec.ndim == 2:
+    if spec.ndim >= 2:
         b = torch.exp(torch.randn(1, cols, generator=fixed, dtype=torch.float32, device=device))
         g *= b
     if outlier_p > 0:

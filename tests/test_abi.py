@@ -67,10 +67,21 @@ def test_bad_configurations_are_rejected_on_the_host():
         bad = lpmm.default_config()
         setattr(bad, field, value)
         assert L.lpmm_state_bytes(C.byref(bad), shapes, 1, C.byref(out)) == want
-    for shp, want in (((0, 4, 2, 0), lpmm.ERR_INVALID_ARG), ((4, 4, 3, 0), lpmm.ERR_UNSUPPORTED),
+    for shp, want in (((0, 4, 2, 0), lpmm.ERR_INVALID_ARG), ((4, 4, 3, 0), lpmm.ERR_INVALID_ARG),   # ndim 3 without extents
+                      ((4, 4, 5, 0), lpmm.ERR_UNSUPPORTED),
                       ((4, 4, 1, 0), lpmm.ERR_INVALID_ARG), ((4, 4, 2, 3), lpmm.ERR_INVALID_ARG),
                       ((1 << 39, 1 << 39, 2, 0), lpmm.ERR_INVALID_ARG)):
         assert L.lpmm_state_bytes(C.byref(cfg), lpmm.make_shapes([shp]), 1, C.byref(out)) == want
+    # three and four axes (Alg. 4 in general form): extents must restate rows and cols
+    nd = lpmm.nd_shape((6, 10, 200))
+    assert L.lpmm_state_bytes(C.byref(cfg), lpmm.make_shapes([nd]), 1, C.byref(out)) == lpmm.OK
+    assert out.value >= 2 * (12000 // 2) + 4 * (12000 // 128) + 3 * 4 * (6 + 10 + 200)
+    bad = lpmm.nd_shape((6, 10, 200))
+    bad.rows = 61
+    assert L.lpmm_state_bytes(C.byref(cfg), lpmm.make_shapes([bad]), 1, C.byref(out)) == lpmm.ERR_INVALID_ARG
+    fact = lpmm.default_config(v_mode=lpmm.V_FACTORED)
+    assert L.lpmm_state_bytes(C.byref(fact), lpmm.make_shapes([nd]), 1, C.byref(out)) == lpmm.ERR_UNSUPPORTED
+    assert L.lpmm_state_view_axis(None, 0, 0, None, None) == lpmm.ERR_INVALID_ARG
     h = C.c_void_p()
     assert L.lpmm_state_init(C.byref(cfg), shapes, 1, None, 1 << 20, C.byref(h), None) == lpmm.ERR_INVALID_ARG
     assert L.lpmm_state_init(C.byref(cfg), shapes, 1, 0x1010, 1 << 20, C.byref(h), None) == lpmm.ERR_ALIGNMENT

@@ -338,3 +338,53 @@ def test_factorized_second_moment_matches_oracle(grad_dtype):
     with pytest.raises(lpmm.LpmmError) as ei:
         lpmm.state_init(cfg, [_mat(257, 129)])
     assert ei.value.status == lpmm.ERR_UNSUPPORTED
+
+
+def _nd(*dims):
+    rows = int(np.prod(dims[:-1]))
+    return workloads.TensorSpec("t" + "x".join(map(str, dims)), rows, dims[-1], len(dims), dims=tuple(dims))
+
+
+@pytest.mark.parametrize("grad_dtype,update_math", [(torch.float32, lpmm.UPDATE_IEEE), (torch.bfloat16, lpmm.UPDATE_FAST)])
+def test_tensors_with_three_and_four_axes_match_oracle(grad_dtype, update_math):
+    # Alg. 4 in its general form: one vector of maxima per axis, scale = minimum over the element's axes.
+    # Codes, block scales and every axis' statistics bit-exact; parameters bit-exact with IEEE update math,
+    # within 1e-6 * max(|w|, lr) with the approximate one. A matrix rides along to cover mixed lists.
+    cfg = lpmm.default_config(update_math=update_math)
+    specs = [_nd(6, 10, 200), _nd(3, 5, 7, 64), _nd(16, 33, 9), _mat(96, 256), _nd(2, 4099, 3), _nd(1, 40, 128)]
+    hyper = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
+    params = [workloads.make_param(s, 14, i, device="cuda") for i, s in enumerate(specs)]
+    state = lpmm.state_init(cfg, specs)
+    assert all(lpmm.state_view(state, i)["kind"] == lpmm.KIND_RANK1 for i in range(len(specs)))
+    w_ref = [p.cpu().numpy().ravel().copy() for p in params]
+    ref = []
+    for s in specs:
+        dims = s.shape
+        ref.append(dict(m_codes=np.full((s.numel + 1) // 2, 0x77, np.uint8), m_scale=np.zeros((s.numel + 127) // 128, np.float32),
+                        v_codes=np.zeros((s.numel + 1) // 2, np.uint8), mu=np.zeros(int(sum(dims)), np.float32)))
+        if s.numel % 2:
+            ref[-1]["m_codes"][-1] = 0x07
+    for t in range(1, 5):
+        grads = [workloads.make_grad(s, 14, i, t, device="cuda", dtype=grad_dtype) for i, s in enumerate(specs)]
+        lpmm.adamw4_step(state, params, grads, step=t, **hyper)
+        torch.cuda.synchronize()
+        assert lpmm.device_status(state) == 0
+        for i, s in enumerate(specs):
+            r = ref[i]
+            oracle.adamw4_step_nd(w_ref[i], grads[i].float().cpu().numpy().ravel(), s.shape, 128, r["m_codes"], r["m_scale"],
+                                  r["v_codes"], r["mu"], step=t, **hyper)
+            view = lpmm.state_view(state, i)
+            for name in ("m_codes", "m_scale", "v_codes"):
+                assert np.array_equal(view[name].cpu().numpy(), r[name]), (s.name, name, t)
+            mu = np.concatenate([lpmm.state_view_axis(state, i, a).cpu().numpy() for a in range(len(s.shape))])
+            assert np.array_equal(mu, r["mu"]), (s.name, "mu", t)
+            w = params[i].cpu().numpy().ravel()
+            if update_math == lpmm.UPDATE_IEEE:
+                assert np.array_equal(w, w_ref[i]), (s.name, t)
+            else:
+                err = np.max(np.abs(w - w_ref[i]) / np.maximum(np.abs(w_ref[i]), hyper["lr"]))
+                assert err <= 1e-6, (s.name, t, err)
+                w_ref[i][:] = w
+    with pytest.raises(lpmm.LpmmError) as ei:      # five axes: not supported
+        lpmm.state_init(cfg, [_nd(2, 2, 2, 2, 300)])
+    assert ei.value.status == lpmm.ERR_UNSUPPORTED
