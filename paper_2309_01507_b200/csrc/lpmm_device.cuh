@@ -248,4 +248,12 @@ __device__ __forceinline__ void atomic_max_nonneg(float* addr, float v) {
     atomicMax(reinterpret_cast<unsigned int*>(addr), __float_as_uint(v));
 }
 
+// The same with a look first: a value that does not exceed what the slot already holds needs no atomic at all.
+// The slot only ever grows within a pass, so a stale read can cost a redundant atomic but never lose a maximum;
+// the read bypasses L1 to see other SMs' updates early. Over a stream of values the number of atomics per slot
+// drops from the number of elements to roughly the number of running maxima.
+__device__ __forceinline__ void atomic_max_nonneg_filtered(float* addr, float v) {
+    if (v > __ldcg(addr)) atomicMax(reinterpret_cast<unsigned int*>(addr), __float_as_uint(v));
+}
+
 }  // namespace lpmm

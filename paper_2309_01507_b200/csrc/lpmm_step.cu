@@ -583,14 +583,26 @@ __device__ __forceinline__ void pass2_rank1_bulk(const TensorDesc& d, float* __r
 // an element's scale is the minimum of their statistics at the row's multi-index (for the reciprocals of the
 // new statistics: the maximum). A matrix has one leading axis and this is a single load.
 
+// Row and column of flat element e of a rows x cols tensor (one 32-bit division when the indices allow it).
+__device__ __forceinline__ void split_index(const TensorDesc& d, int64_t e, int64_t& i, int64_t& j) {
+    if (d.numel <= 0xffffffffLL) {
+        const uint32_t q = (uint32_t)e / (uint32_t)d.cols;
+        i = q;
+        j = (uint32_t)e - q * (uint32_t)d.cols;
+    } else {
+        i = e / d.cols;
+        j = e - i * d.cols;
+    }
+}
+
 template <bool MAX>
 __device__ __forceinline__ float outer_stat(const TensorDesc& d, const float* __restrict__ base, int64_t i) {
     if (d.n_outer == 1) return __ldg(base + i);
-    int64_t rem = i;
+    uint32_t rem = (uint32_t)i;                          // rows <= 2^30 (checked on the host)
     float s = MAX ? 0.0f : 3.402823466e38f;
     for (int a = d.n_outer - 1; a >= 0; --a) {          // the last leading axis varies fastest
-        const int64_t q = rem / d.outer_dim[a];
-        const float x = __ldg(base + d.outer_off[a] + (rem - q * d.outer_dim[a]));
+        const uint32_t q = rem / (uint32_t)d.outer_dim[a];
+        const float x = __ldg(base + d.outer_off[a] + (rem - q * (uint32_t)d.outer_dim[a]));
         s = MAX ? fmaxf(s, x) : fminf(s, x);
         rem = q;
     }
@@ -598,11 +610,11 @@ __device__ __forceinline__ float outer_stat(const TensorDesc& d, const float* __
 }
 // Publishes the maximum of a run of elements of row i to every leading axis.
 __device__ __forceinline__ void outer_publish(const TensorDesc& d, float* base, int64_t i, float x) {
-    if (d.n_outer == 1) { atomic_max_nonneg(base + i, x); return; }
-    int64_t rem = i;
+    if (d.n_outer == 1) { atomic_max_nonneg_filtered(base + i, x); return; }
+    uint32_t rem = (uint32_t)i;
     for (int a = d.n_outer - 1; a >= 0; --a) {
-        const int64_t q = rem / d.outer_dim[a];
-        atomic_max_nonneg(base + d.outer_off[a] + (rem - q * d.outer_dim[a]), x);
+        const uint32_t q = rem / (uint32_t)d.outer_dim[a];
+        atomic_max_nonneg_filtered(base + d.outer_off[a] + (rem - q * (uint32_t)d.outer_dim[a]), x);
         rem = q;
     }
 }
@@ -645,7 +657,8 @@ __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restric
         const bool group_live = (e & ~m_mask) < d.numel;
         const float am = group_live ? d.m_scale[e >> MSHIFT] : 0.0f;
         if (RANK1) {
-            int64_t i = e / d.cols, j = e - i * d.cols;
+            int64_t i, j;
+            split_index(d, e, i, j);
             float so = 0.0f, ro = 0.0f;          // leading axes' share of the old scale / the new reciprocal, row i
             bool fresh = true;
 #pragma unroll
@@ -1051,7 +1064,8 @@ __device__ __forceinline__ void pass1_rank1_flat(const TensorDesc& d, const void
         float gv[8];
         load8_grad_guard<BF16>(g, e, d.numel, gv);
         const uint32_t qv = load_codes_guard(d.v_codes, e, d.numel);
-        int64_t i = e / d.cols, j = e - i * d.cols;
+        int64_t i, j;
+        split_index(d, e, i, j);
         float run = 0.0f;                      // maximum of the lane's current run of elements in row i
         float so = 0.0f;                       // leading axes' share of the old scale in row i
         bool fresh = true;
@@ -1062,7 +1076,7 @@ __device__ __forceinline__ void pass1_rank1_flat(const TensorDesc& d, const void
                 const float s = fminf(so, __ldg(rc_old + d.c_off + j));
                 const float vt = ema_v(__fmul_rn(lin_value((qv >> (4 * k)) & 15u), s), gv[k], h);
                 run = fmaxf(run, vt);
-                atomic_max_nonneg(rc_new + d.c_off + j, vt);
+                atomic_max_nonneg_filtered(rc_new + d.c_off + j, vt);
             }
             if (++j == d.cols) {               // the row ends inside the lane's elements: publish and start over
                 outer_publish(d, rc_new, i, run);
