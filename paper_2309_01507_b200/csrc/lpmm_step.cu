@@ -273,6 +273,8 @@ struct TileView {
     int m_shift;           // log2 of the first-moment block size
     float* s_red;          // CTA scratch for B2048 block maxima
     uint32_t* red_step;    // running count of CTA-wide reductions
+    const char* pf_base;   // this lane's share of the row prefetch: one cache line of one of the arrays
+    uint32_t pf_step;      // bytes between two of the warp's rows in that array (0: this lane prefetches nothing)
 };
 
 // Asks L2 to fetch this lane's share of row k ahead of time (no register is tied up): the later
@@ -280,18 +282,43 @@ struct TileView {
 constexpr uint32_t kL2Ahead = 4;   // rows
 __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
+// One instruction per row for the whole warp: the 256 elements a warp owns in a row are 8 lines of parameters,
+// 4 (bf16) or 8 (fp32) lines of gradient, one line of each code array and one of block scales, and each of the
+// first lanes asks for one of those lines.
 template <bool BF16, int MSHIFT, bool FACT>
 __device__ __forceinline__ void prefetch_row(const TileView& t, uint32_t k) {
-    const uint32_t off = k * t.row_step;
-    prefetch_l2(t.w + off);
-    if (BF16) {
-        prefetch_l2(reinterpret_cast<const uint16_t*>(t.g) + off);
-    } else {
-        prefetch_l2(reinterpret_cast<const float*>(t.g) + off);
+    if (t.pf_step != 0) prefetch_l2(t.pf_base + (size_t)k * t.pf_step);
+}
+// Assigns the lane its line (warp_* point at the warp's first element of row 0; row_step in elements).
+// `valid` = how many of the warp's 256 columns exist (128 in a tensor's last warp column when cols % 256 == 128):
+// no lane asks for a line past the end of the row.
+template <bool BF16, int MSHIFT, bool FACT>
+__device__ __forceinline__ void prefetch_roles(TileView& t, int lane, int valid, const float* warp_w, const void* warp_g,
+                                               const uint8_t* warp_mq, const uint8_t* warp_vq, const float* warp_ms) {
+    constexpr int kGLines = BF16 ? 4 : 8;
+    constexpr int kGLineElems = BF16 ? 64 : 32;
+    t.pf_base = nullptr;
+    t.pf_step = 0;
+    if (lane < 8) {
+        if (lane * 32 < valid) {
+            t.pf_base = reinterpret_cast<const char*>(warp_w) + lane * 128;
+            t.pf_step = t.row_step * 4u;
+        }
+    } else if (lane < 8 + kGLines) {
+        if ((lane - 8) * kGLineElems < valid) {
+            t.pf_base = reinterpret_cast<const char*>(warp_g) + (lane - 8) * 128;
+            t.pf_step = t.row_step * (BF16 ? 2u : 4u);
+        }
+    } else if (lane == 8 + kGLines) {
+        t.pf_base = reinterpret_cast<const char*>(warp_mq);
+        t.pf_step = t.row_step / 2u;
+    } else if (lane == 9 + kGLines && !FACT) {
+        t.pf_base = reinterpret_cast<const char*>(warp_vq);
+        t.pf_step = t.row_step / 2u;
+    } else if (lane == 10 + kGLines) {
+        t.pf_base = reinterpret_cast<const char*>(warp_ms);
+        t.pf_step = (t.row_step >> MSHIFT) * 4u;
     }
-    prefetch_l2(t.m_codes + (off >> 1));
-    if (!FACT) prefetch_l2(t.v_codes + (off >> 1));
-    prefetch_l2(t.m_scale + (off >> MSHIFT));
 }
 
 template <bool BF16, int MSHIFT, bool FACT>
@@ -386,6 +413,14 @@ __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __r
     t.m_shift = d.m_shift;
     t.s_red = s_red;
     t.red_step = &red_step;
+    {
+        const int64_t ew = e0 - lane * kLaneElems;       // the warp's first element of its first row
+        const int64_t left = d.cols - (col0 - lane * kLaneElems);
+        prefetch_roles<BF16, MSHIFT, FACT>(t, lane, left < kWarpElems ? (int)left : kWarpElems, w + ew,
+                                           BF16 ? static_cast<const void*>(reinterpret_cast<const uint16_t*>(g) + ew)
+                                                : static_cast<const void*>(reinterpret_cast<const float*>(g) + ew),
+                                           d.m_codes + (ew >> 1), FACT ? nullptr : d.v_codes + (ew >> 1), d.m_scale + (ew >> MSHIFT));
+    }
 
     // Two register sets alternate: while one row is processed the next one is already in flight.
     RowRegs<BF16> ra, rb;
@@ -600,11 +635,14 @@ __device__ __forceinline__ float outer_stat(const TensorDesc& d, const float* __
     if (d.n_outer == 1) return __ldg(base + i);
     uint32_t rem = (uint32_t)i;                          // rows <= 2^30 (checked on the host)
     float s = MAX ? 0.0f : 3.402823466e38f;
-    for (int a = d.n_outer - 1; a >= 0; --a) {          // the last leading axis varies fastest
-        const uint32_t q = rem / (uint32_t)d.outer_dim[a];
-        const float x = __ldg(base + d.outer_off[a] + (rem - q * (uint32_t)d.outer_dim[a]));
-        s = MAX ? fmaxf(s, x) : fminf(s, x);
-        rem = q;
+#pragma unroll
+    for (int a = 2; a >= 0; --a) {                       // the last leading axis varies fastest; constant indices keep
+        if (a < d.n_outer) {                             // the descriptor in registers
+            const uint32_t q = rem / (uint32_t)d.outer_dim[a];
+            const float x = __ldg(base + d.outer_off[a] + (rem - q * (uint32_t)d.outer_dim[a]));
+            s = MAX ? fmaxf(s, x) : fminf(s, x);
+            rem = q;
+        }
     }
     return s;
 }
@@ -612,10 +650,13 @@ __device__ __forceinline__ float outer_stat(const TensorDesc& d, const float* __
 __device__ __forceinline__ void outer_publish(const TensorDesc& d, float* base, int64_t i, float x) {
     if (d.n_outer == 1) { atomic_max_nonneg_filtered(base + i, x); return; }
     uint32_t rem = (uint32_t)i;
-    for (int a = d.n_outer - 1; a >= 0; --a) {
-        const uint32_t q = rem / (uint32_t)d.outer_dim[a];
-        atomic_max_nonneg_filtered(base + d.outer_off[a] + (rem - q * (uint32_t)d.outer_dim[a]), x);
-        rem = q;
+#pragma unroll
+    for (int a = 2; a >= 0; --a) {
+        if (a < d.n_outer) {
+            const uint32_t q = rem / (uint32_t)d.outer_dim[a];
+            atomic_max_nonneg_filtered(base + d.outer_off[a] + (rem - q * (uint32_t)d.outer_dim[a]), x);
+            rem = q;
+        }
     }
 }
 
@@ -836,6 +877,9 @@ struct P1View {
     const void* g;             // at the lane's first element of the tile (row i0, the lane's 8 columns)
     const uint8_t* v_codes;    // likewise
     uint32_t row_step;         // elements between two rows this warp handles
+    const char* pf_base;       // this lane's share of the prefetch of a group of rows: one line of one array in one row
+    uint32_t pf_step;          // bytes between two of the warp's rows in that array (0: nothing to prefetch)
+    uint32_t pf_row;           // which row of the group
 };
 
 template <bool BF16>
@@ -850,12 +894,35 @@ __device__ __forceinline__ void load_p1_row(P1Row<BF16>& b, const P1View& t, uin
     b.qv = __ldg(reinterpret_cast<const uint32_t*>(t.v_codes + (off >> 1)));
 }
 
+// L2 prefetch of a group of rows with one instruction for the whole warp: a row of the warp is 4 (bf16) or 8
+// (fp32) lines of gradient and one line of codes, so 4 (2) rows fit the 32 lanes.
+template <bool BF16> struct P1Pf {
+    static constexpr int kGLines = BF16 ? 4 : 8;
+    static constexpr int kLines = kGLines + 1;
+    static constexpr int kRows = BF16 ? 4 : 2;          // rows per instruction
+};
 template <bool BF16>
-__device__ __forceinline__ void prefetch_p1_row(const P1View& t, uint32_t k) {
-    const uint32_t off = k * t.row_step;
-    if (BF16) prefetch_l2(reinterpret_cast<const uint16_t*>(t.g) + off);
-    else prefetch_l2(reinterpret_cast<const float*>(t.g) + off);
-    prefetch_l2(t.v_codes + (off >> 1));
+__device__ __forceinline__ void p1_prefetch_roles(P1View& t, int lane, int valid, const void* warp_g, const uint8_t* warp_vq) {
+    const int u = lane / P1Pf<BF16>::kLines, item = lane - u * P1Pf<BF16>::kLines;
+    t.pf_base = nullptr;
+    t.pf_step = 0;
+    t.pf_row = (uint32_t)u;
+    if (u >= P1Pf<BF16>::kRows) return;
+    if (item < P1Pf<BF16>::kGLines) {
+        if (item * (BF16 ? 64 : 32) < valid) {
+            t.pf_base = reinterpret_cast<const char*>(warp_g) + item * 128;
+            t.pf_step = t.row_step * (BF16 ? 2u : 4u);
+        }
+    } else {
+        t.pf_base = reinterpret_cast<const char*>(warp_vq);
+        t.pf_step = t.row_step / 2u;
+    }
+}
+// Rows k .. k + kRows - 1 (those below nrows).
+template <bool BF16>
+__device__ __forceinline__ void prefetch_p1_group(const P1View& t, uint32_t k, uint32_t nrows) {
+    const uint32_t row = k + t.pf_row;
+    if (t.pf_step != 0 && row < nrows) prefetch_l2(t.pf_base + (size_t)row * t.pf_step);
 }
 
 // Maxima of four per-lane values over the warp with 6 shuffles: afterwards the lanes with
@@ -927,8 +994,16 @@ __device__ __forceinline__ void pass1_rank1_fast(const TensorDesc& d, const void
     t.v_codes = d.v_codes + (e0 >> 1);
     t.row_step = (uint32_t)(wy_count * d.cols);
 
+    {
+        const int64_t ew = row0 * d.cols + col_w;          // the warp's first element of its first row
+        const int64_t left = d.cols - col_w;
+        p1_prefetch_roles<BF16>(t, lane, left < kWarpElems ? (int)left : kWarpElems,
+                                BF16 ? static_cast<const void*>(reinterpret_cast<const uint16_t*>(g) + ew)
+                                     : static_cast<const void*>(reinterpret_cast<const float*>(g) + ew),
+                                d.v_codes + (ew >> 1));
+    }
 #pragma unroll
-    for (uint32_t k = 1; k < kP1L2Ahead; ++k) if (k < nrows) prefetch_p1_row<BF16>(t, k);
+    for (uint32_t k = 0; k < kP1L2Ahead; k += P1Pf<BF16>::kRows) prefetch_p1_group<BF16>(t, k, nrows);
     // Lane j keeps the old row scale of the warp's row number base + j (32 rows per refill); a row's scale is
     // then read with one shuffle instead of a load.
     float r_vec = 0.0f;
@@ -940,8 +1015,7 @@ __device__ __forceinline__ void pass1_rank1_fast(const TensorDesc& d, const void
             r_vec = __ldg(rc_old + row0 + (int64_t)kk * wy_count);
         }
 #pragma unroll
-        for (uint32_t u = 0; u < 4; ++u)
-            if (k + kP1L2Ahead + u < nrows) prefetch_p1_row<BF16>(t, k + kP1L2Ahead + u);
+        for (uint32_t u = 0; u < 4; u += P1Pf<BF16>::kRows) prefetch_p1_group<BF16>(t, k + kP1L2Ahead + u, nrows);
         float r_max[4] = {0.0f, 0.0f, 0.0f, 0.0f};
         if (k + 1 < nrows) load_p1_row<BF16>(rb, t, k + 1);
         r_max[0] = p1_process_row<BF16>(ra, __shfl_sync(0xffffffffu, r_vec, k & 31), c_old, c_max, h2, lt);
