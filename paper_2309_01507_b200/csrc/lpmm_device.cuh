@@ -66,14 +66,14 @@ __device__ __forceinline__ uint32_t lin_nearest_magic(float n) {
     return __float_as_uint(__fadd_ru(y, 8388608.0f));
 }
 
-// Shared-memory image of the nearest-entry table, directly indexed by the top 12 bits of n: 2048 eight-byte
-// entries for n >= 0 followed by 2048 for n < 0, so that no clamping is needed and every bit pattern (NaN
+// Shared-memory image of the nearest-entry table, directly indexed by the top 11 bits of n: 1024 eight-byte
+// entries for n >= 0 followed by 1024 for n < 0, so that no clamping is needed and every bit pattern (NaN
 // and infinities included) stays inside the table.
-constexpr int kLutSmemBytes = 2 * 2048 * 8;
+constexpr int kLutSmemBytes = 2 * 1024 * 8;
 
 __device__ __forceinline__ void load_lut_smem(unsigned char* smem) {
-    for (uint32_t i = threadIdx.x; i < 4096u; i += blockDim.x) {
-        const uint32_t key = i & 2047u, neg = i >> 11;
+    for (uint32_t i = threadIdx.x; i < 2048u; i += blockDim.x) {
+        const uint32_t key = i & 1023u, neg = i >> 10;
         uint2 e;
         if (key < kDeLutFirstKey) e = make_uint2(0x7f7fffffu, 7u);
         else if (key >= kDeLutFirstKey + kDeLutBins) e = make_uint2(0x7f7fffffu, neg ? 0u : 15u);
@@ -84,7 +84,7 @@ __device__ __forceinline__ void load_lut_smem(unsigned char* smem) {
 
 // Table-driven equivalent of de_nearest(): one lookup, one comparison, one add.
 __device__ __forceinline__ uint32_t de_nearest_lut(float n, const unsigned char* smem) {
-    const uint2 e = *reinterpret_cast<const uint2*>(smem + ((__float_as_uint(n) >> 17) & 0x7ff8u));
+    const uint2 e = *reinterpret_cast<const uint2*>(smem + ((__float_as_uint(n) >> 18) & 0x3ff8u));
     return e.y + (n > __uint_as_float(e.x) ? 1u : 0u);
 }
 
