@@ -167,10 +167,16 @@ __host__ __device__ __forceinline__ Hyper2 make_hyper2(const Hyper& h) {
 // t[i] holds the entries of elements 2i and 2i + 1.
 __device__ __forceinline__ void lin_dequant8(uint32_t q, const Hyper2& h, float2 (&t)[4]) {
     const uint32_t hi = q >> 16;
-    t[0] = fma2_rn(make_float2(__uint_as_float(kMagicBits | (q & 0xfu)), __uint_as_float(kMagicBits | (q & 0xf0u))), h.lin_a01, h.lin_b01);
-    t[1] = fma2_rn(make_float2(__uint_as_float(kMagicBits | (q & 0xf00u)), __uint_as_float(kMagicBits | (q & 0xf000u))), h.lin_a23, h.lin_b23);
-    t[2] = fma2_rn(make_float2(__uint_as_float(kMagicBits | (hi & 0xfu)), __uint_as_float(kMagicBits | (hi & 0xf0u))), h.lin_a01, h.lin_b01);
-    t[3] = fma2_rn(make_float2(__uint_as_float(kMagicBits | (hi & 0xf00u)), __uint_as_float(kMagicBits | (hi & 0xf000u))), h.lin_a23, h.lin_b23);
+    const uint32_t magic = __float_as_uint(h.magic.x);     // 2^23: its mantissa field is empty
+    uint32_t f[8];
+#define LPMM_NIB(dst, src, m) asm("lop3.b32 %0, %1, " #m ", %2, 0xEA;" : "=r"(dst) : "r"(src), "r"(magic))
+    LPMM_NIB(f[0], q, 0xf);   LPMM_NIB(f[1], q, 0xf0);   LPMM_NIB(f[2], q, 0xf00);   LPMM_NIB(f[3], q, 0xf000);
+    LPMM_NIB(f[4], hi, 0xf);  LPMM_NIB(f[5], hi, 0xf0);  LPMM_NIB(f[6], hi, 0xf00);  LPMM_NIB(f[7], hi, 0xf000);
+#undef LPMM_NIB
+    t[0] = fma2_rn(make_float2(__uint_as_float(f[0]), __uint_as_float(f[1])), h.lin_a01, h.lin_b01);
+    t[1] = fma2_rn(make_float2(__uint_as_float(f[2]), __uint_as_float(f[3])), h.lin_a23, h.lin_b23);
+    t[2] = fma2_rn(make_float2(__uint_as_float(f[4]), __uint_as_float(f[5])), h.lin_a01, h.lin_b01);
+    t[3] = fma2_rn(make_float2(__uint_as_float(f[6]), __uint_as_float(f[7])), h.lin_a23, h.lin_b23);
 }
 // Both products must be rounded before the sum (Eq. 1 evaluated operation by operation). The assembler
 // was observed to merge a packed multiply with a following packed add into a fused multiply-add even with
