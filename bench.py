@@ -35,8 +35,8 @@ PASS2_BYTES = {"bf16": 12.0625, "f32": 14.0625}
 PASS1_BYTES = {"bf16": 2.5, "f32": 4.5}
 # DRAM traffic of the update/re-quantize pass measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum)
 # per parameter, from the capture of the 464.5 M-parameter LLaMA slice summarised in
-# profiles/pass2_llama_7b_1l.txt (3.2706 GB read + 2.2839 GB written); traffic scales with the parameter count.
-PASS2_TRAFFIC_BYTES_PER_PARAM = {"bf16": 11.957, "f32": None}
+# profiles/pass2_llama_7b_1l.txt (3.3009 GB read + 2.2857 GB written); traffic scales with the parameter count.
+PASS2_TRAFFIC_BYTES_PER_PARAM = {"bf16": 12.026, "f32": None}
 
 
 def parse_args():
