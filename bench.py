@@ -299,7 +299,8 @@ def run_ours(args):
         pass2_bpp -= 1.0      # no second-moment codes are read or written
     alg_bytes = pass2_bpp * n_params
     achieved = alg_bytes / (p2_ms * 1e-3) / 1e9
-    traffic_pp = PASS2_TRAFFIC_BYTES_PER_PARAM[wl.grad_dtype]
+    # the captures cover the default quantizers only
+    traffic_pp = PASS2_TRAFFIC_BYTES_PER_PARAM[wl.grad_dtype] if (args.v_mode == "rank1" and args.m_block == 128) else None
     roofline = {"bound": "hbm", "kernel": "pass2_kernel (update + re-quantize)", "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                 "traffic": None if traffic_pp is None else traffic_pp * n_params,
