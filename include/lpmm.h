@@ -20,7 +20,9 @@
  *  - NaN/Inf gradients are not detected; the result is then unspecified (but nothing faults).
  *  - There is no CPU fallback: without a CUDA device every launching call returns LPMM_ERR_CUDA.
  *  - The device that owns the arena must be the current device of the calling thread. A state handle is not
- *    thread-safe: use it from one thread at a time.
+ *    thread-safe: use it from one thread at a time. Steps on one state must also be ordered on the device (the
+ *    same stream, or streams ordered by events): the kernels of a step share work counters in the arena header
+ *    that each launch leaves at zero for the next one.
  */
 #ifndef LPMM_H
 #define LPMM_H
