@@ -129,6 +129,16 @@ lpmm_status lpmm_adamw4_step(lpmm_state* st, void* const* d_params, const void* 
                              int32_t grad_dtype, float lr, float beta1, float beta2, float eps,
                              float weight_decay, int64_t step, void* stream);
 
+/* The same step, which also writes a bfloat16 copy (round to nearest even) of every updated parameter, for training
+ * set-ups that keep fp32 master parameters here and run the model on a bf16 copy (+2 bytes per parameter of traffic;
+ * the paper's method has no such output: its states and fp32 parameters are updated exactly as by lpmm_adamw4_step).
+ *   d_params_bf16[i] : device pointer to numel bfloat16 values of tensor i (written), 16-byte aligned; a HOST array
+ *                      of n device pointers like d_params.
+ * Not available with LPMM_V_FACTORED (LPMM_ERR_UNSUPPORTED). */
+lpmm_status lpmm_adamw4_step_bf16w(lpmm_state* st, void* const* d_params, void* const* d_params_bf16,
+                                   const void* const* d_grads, int32_t grad_dtype, float lr, float beta1, float beta2,
+                                   float eps, float weight_decay, int64_t step, void* stream);
+
 /* One fused step of Alg. 2 (compressed SGDM) over every tensor of the state: decompress m (B128 or B2048 / DE);
  * m <- beta m + g ; w <- w - lr m ; new block maxima ; compress m. Only the first-moment part of the state
  * is used (tensors of <= min_quant_numel elements keep m in fp32); do not mix with lpmm_adamw4_step on one

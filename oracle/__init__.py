@@ -175,6 +175,13 @@ def bf16_bits_to_f32(bits) -> np.ndarray:
     return out.reshape(bits.shape)
 
 
+def f32_to_bf16_bits(x) -> np.ndarray:
+    x = _f32(x)
+    out = np.zeros(x.size, np.uint16)
+    lib().lpmm_oracle_f32_to_bf16(_p(x), C.c_int64(x.size), _p(out))
+    return out.reshape(x.shape)
+
+
 def kind_of(rows: int, cols: int, ndim: int, min_quant_numel: int = 4096, force: int = 0) -> int:
     return int(lib().lpmm_oracle_kind(rows, cols, ndim, min_quant_numel, force))
 

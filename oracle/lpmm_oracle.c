@@ -350,6 +350,19 @@ int lpmm_oracle_adamw4_step(float* w, const float* g, int64_t rows, int64_t cols
     return 0;
 }
 
+/* binary32 -> bfloat16 bit pattern, round to nearest, ties to even (IEEE 754 roundTiesToEven on the 16 dropped
+ * bits); a NaN becomes the canonical 0x7fff. */
+void lpmm_oracle_f32_to_bf16(const float* in, int64_t numel, uint16_t* out) {
+    for (int64_t i = 0; i < numel; ++i) {
+        uint32_t u;
+        memcpy(&u, &in[i], 4);
+        if ((u & 0x7fffffffu) > 0x7f800000u) { out[i] = 0x7fffu; continue; }
+        uint32_t keep = u >> 16, rest = u & 0xffffu;
+        if (rest > 0x8000u || (rest == 0x8000u && (keep & 1u))) keep += 1u;   /* may carry into the exponent: that is the rounding to the next binade or to infinity */
+        out[i] = (uint16_t)keep;
+    }
+}
+
 /* ------------------------------------------------------------------ Alg. 3 on a tensor of any rank (Alg. 4) */
 
 int lpmm_oracle_adamw4_step_nd(float* w, const float* g, int ndim, const int64_t* dims, int64_t m_block,

@@ -87,6 +87,10 @@ void lpmm_oracle_unpack4(const uint8_t* packed, int64_t numel, uint8_t* codes);
 /* bfloat16 bit pattern -> binary32 (exact). */
 void lpmm_oracle_bf16_to_f32(const uint16_t* in, int64_t numel, float* out);
 
+/* binary32 -> bfloat16 bit pattern: round to nearest, ties to even; NaN -> 0x7fff. (Not part of the paper's method:
+ * checks the optional bfloat16 copy of the parameters that the CUDA library can write.) */
+void lpmm_oracle_f32_to_bf16(const float* in, int64_t numel, uint16_t* out);
+
 /* Hyper-parameters of Eq. 1 plus decoupled weight decay. */
 typedef struct {
     float lr, beta1, beta2, eps, weight_decay;

@@ -42,7 +42,7 @@ struct TensorLayout {
 
 struct Layout {
     std::vector<TensorLayout> t;
-    size_t descs = 0, params = 0, grads = 0, tiles1 = 0, tiles2 = 0, tiles3 = 0;
+    size_t descs = 0, params = 0, params16 = 0, grads = 0, tiles1 = 0, tiles2 = 0, tiles3 = 0;
     size_t rc[2] = {0, 0}, rcp = 0;
     int64_t rc_floats = 0;
     size_t total = 0;
@@ -116,6 +116,7 @@ void compute_layout(const lpmm_config& cfg, const lpmm_shape* shapes, int32_t n,
     size_t off = kAlign;  // header block
     L->descs = off;  off = align_up(off + sizeof(TensorDesc) * n);
     L->params = off; off = align_up(off + sizeof(void*) * n);
+    L->params16 = off; off = align_up(off + sizeof(void*) * n);
     L->grads = off;  off = align_up(off + sizeof(void*) * n);
     L->tiles1 = off; off = align_up(off + sizeof(int32_t) * (n + 1));
     L->tiles2 = off; off = align_up(off + sizeof(int32_t) * (n + 1));
@@ -181,6 +182,7 @@ struct lpmm_state {
     int32_t last_launches;
     bool ptrs_valid;
     std::vector<void*> params, grads;  // what the device-side pointer arrays currently hold
+    std::vector<void*> params16;       // likewise for the optional bfloat16 copies (empty until first used)
     size_t stage_bytes;
     std::vector<size_t> stage_off;
     int32_t pass2_variant;                 // 0 = register prefetch, 1 = bulk-copy staging
@@ -403,6 +405,7 @@ StepArgs make_args(const lpmm_state* st, float lr, float beta1, float beta2, flo
     StepArgs a;
     a.descs = reinterpret_cast<const TensorDesc*>(st->arena + st->L.descs);
     a.params = reinterpret_cast<float* const*>(st->arena + st->L.params);
+    a.params_bf16 = nullptr;
     a.grads = reinterpret_cast<const void* const*>(st->arena + st->L.grads);
     a.n_tensors = st->n;
     a.phase = st->phase;
@@ -479,19 +482,39 @@ lpmm_status enqueue_range(lpmm_state* st, StepArgs a, int32_t t0, int32_t t1, bo
     return LPMM_OK;
 }
 
-}  // namespace
+// Makes the device-side array of bfloat16-copy pointers hold d_params16 (uploads only on change).
+lpmm_status set_pointers16(lpmm_state* st, void* const* d_params16, cudaStream_t s) {
+    const int32_t n = st->n;
+    bool changed = st->params16.empty();
+    if (changed) st->params16.assign(n, nullptr);
+    for (int32_t i = 0; i < n; ++i) {
+        if (!d_params16[i]) return LPMM_ERR_INVALID_ARG;
+        if (!aligned16(d_params16[i])) return LPMM_ERR_ALIGNMENT;
+        if (d_params16[i] != st->params16[i]) changed = true;
+    }
+    if (changed) {
+        for (int32_t i = 0; i < n; ++i) st->params16[i] = d_params16[i];
+        const cudaError_t e = cudaMemcpyAsync(st->arena + st->L.params16, st->params16.data(), sizeof(void*) * n, cudaMemcpyHostToDevice, s);
+        if (e != cudaSuccess) { st->params16.clear(); return cuda_fail(e); }
+    }
+    return LPMM_OK;
+}
 
-extern "C" {
-
-lpmm_status lpmm_adamw4_step(lpmm_state* st, void* const* d_params, const void* const* d_grads,
+lpmm_status adamw4_step_impl(lpmm_state* st, void* const* d_params, void* const* d_params16, const void* const* d_grads,
                              int32_t grad_dtype, float lr, float beta1, float beta2, float eps,
                              float weight_decay, int64_t step, void* stream) {
     lpmm_status rc = check_step_args(st, d_params, d_grads, grad_dtype, lr, beta1, beta2, eps, weight_decay, step);
     if (rc != LPMM_OK) return rc;
+    if (d_params16 && st->cfg.v_mode == LPMM_V_FACTORED) return LPMM_ERR_UNSUPPORTED;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     rc = set_pointers(st, d_params, d_grads, s);
     if (rc != LPMM_OK) return rc;
-    const StepArgs a = make_args(st, lr, beta1, beta2, eps, weight_decay, step);
+    if (d_params16) {
+        rc = set_pointers16(st, d_params16, s);
+        if (rc != LPMM_OK) return rc;
+    }
+    StepArgs a = make_args(st, lr, beta1, beta2, eps, weight_decay, step);
+    if (d_params16) a.params_bf16 = reinterpret_cast<uint16_t* const*>(st->arena + st->L.params16);
     cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
     if (st->profile) {
         for (int k = 0; k < 4; ++k) {
@@ -506,6 +529,23 @@ lpmm_status lpmm_adamw4_step(lpmm_state* st, void* const* d_params, const void* 
     st->phase ^= 1;
     st->last_launches = launches;
     return LPMM_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+lpmm_status lpmm_adamw4_step(lpmm_state* st, void* const* d_params, const void* const* d_grads,
+                             int32_t grad_dtype, float lr, float beta1, float beta2, float eps,
+                             float weight_decay, int64_t step, void* stream) {
+    return adamw4_step_impl(st, d_params, nullptr, d_grads, grad_dtype, lr, beta1, beta2, eps, weight_decay, step, stream);
+}
+
+lpmm_status lpmm_adamw4_step_bf16w(lpmm_state* st, void* const* d_params, void* const* d_params_bf16,
+                                   const void* const* d_grads, int32_t grad_dtype, float lr, float beta1, float beta2,
+                                   float eps, float weight_decay, int64_t step, void* stream) {
+    if (!d_params_bf16) return LPMM_ERR_INVALID_ARG;
+    return adamw4_step_impl(st, d_params, d_params_bf16, d_grads, grad_dtype, lr, beta1, beta2, eps, weight_decay, step, stream);
 }
 
 lpmm_status lpmm_sgdm4_step(lpmm_state* st, void* const* d_params, const void* const* d_grads,

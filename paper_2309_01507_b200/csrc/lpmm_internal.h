@@ -47,6 +47,7 @@ struct TensorDesc {
 struct StepArgs {
     const TensorDesc* descs;
     float* const* params;        // n device pointers, fp32
+    uint16_t* const* params_bf16;  // n device pointers to bfloat16 copies of the parameters, or nullptr (no copy)
     const void* const* grads;    // n device pointers
     const int32_t* tile_start;   // n + 1 prefix sums of tiles (pass-specific)
     int32_t n_tensors;

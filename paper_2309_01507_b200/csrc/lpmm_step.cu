@@ -69,6 +69,24 @@ __device__ __forceinline__ void store8_f32(float* p, const float (&x)[8]) {
     *reinterpret_cast<float4*>(p) = make_float4(x[0], x[1], x[2], x[3]);
     *(reinterpret_cast<float4*>(p) + 1) = make_float4(x[4], x[5], x[6], x[7]);
 }
+// Eight parameters as bfloat16 (round to nearest even), one 16-byte store.
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+__device__ __forceinline__ void store8_bf16(uint16_t* p, const float (&x)[8]) {
+    *reinterpret_cast<uint4*>(p) = make_uint4(pack_bf16x2(x[0], x[1]), pack_bf16x2(x[2], x[3]),
+                                              pack_bf16x2(x[4], x[5]), pack_bf16x2(x[6], x[7]));
+}
+__device__ __forceinline__ void store8_bf16_guard(uint16_t* p, int64_t e, int64_t numel, const float (&x)[8]) {
+#pragma unroll
+    for (int k = 0; k < 8; k += 2) {
+        const uint32_t pr = pack_bf16x2(x[k], x[k + 1]);
+        if (e + k < numel) p[e + k] = (uint16_t)(pr & 0xffffu);
+        if (e + k + 1 < numel) p[e + k + 1] = (uint16_t)(pr >> 16);
+    }
+}
 __device__ __forceinline__ void load8_bf16(const uint16_t* p, float (&x)[8]) {
     uint4 r = __ldg(reinterpret_cast<const uint4*>(p));
     x[0] = bf16_lo(r.x); x[1] = bf16_hi(r.x); x[2] = bf16_lo(r.y); x[3] = bf16_hi(r.y);
@@ -262,6 +280,7 @@ struct RowRegs {           // one lane's share of one row: raw, still packed
 // Per-lane view of a tile: base pointers at the lane's first element and 32-bit offsets from there.
 struct TileView {
     float* w;
+    uint16_t* w16;         // optional bfloat16 copy of the parameters (same indexing as w), or nullptr
     const void* g;
     uint8_t* m_codes;
     uint8_t* v_codes;
@@ -344,7 +363,7 @@ __device__ __forceinline__ void load_row(RowRegs<BF16>& r, const TileView& t, ui
     }
 }
 
-template <bool BF16, bool EXACT, int MSHIFT, bool FACT>
+template <bool BF16, bool EXACT, int MSHIFT, bool FACT, bool WB>
 __device__ __forceinline__ void process_row(const RowRegs<BF16>& r, const TileView& t, uint32_t k,
                                             const float (&c_old)[8], const float (&c_rcp)[8], const Hyper& h,
                                             const Hyper2& h2, const LaneTables& lt, const unsigned char* s_lut) {
@@ -364,14 +383,16 @@ __device__ __forceinline__ void process_row(const RowRegs<BF16>& r, const TileVi
     }
     moments_and_update8<EXACT, FACT>(wv, gv, r.qm, r.qv, __fmul_rn(lt.de, r.am), vs, h, h2, lt, mt, vt);
     store8_f32(t.w + off, wv);
+    if (WB) store8_bf16(t.w16 + off, wv);
     const float am_new = block_max(absmax8(mt), MSHIFT, lt, t.s_red, *t.red_step);
     if ((threadIdx.x & (MSHIFT == 7 ? 15 : 2047)) == 0) t.m_scale[off >> MSHIFT] = am_new;
     *reinterpret_cast<uint32_t*>(t.m_codes + (off >> 1)) = quantize8_de(mt, scale_rcp(am_new), s_lut);
     if (!FACT) *reinterpret_cast<uint32_t*>(t.v_codes + (off >> 1)) = quantize8_lin(vt, vr, h2);
 }
 
-template <bool BF16, bool EXACT, int MSHIFT, bool FACT = false>
-__device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __restrict__ w, const void* __restrict__ g,
+template <bool BF16, bool EXACT, int MSHIFT, bool FACT = false, bool WB = false>
+__device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __restrict__ w, uint16_t* __restrict__ w16,
+                                                 const void* __restrict__ g,
                                                  int tile, int phase, const Hyper& h, const Hyper2& h2,
                                                  const LaneTables& lt, const unsigned char* s_lut, float* s_red,
                                                  uint32_t& red_step) {
@@ -401,6 +422,7 @@ __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __r
     const int64_t e0 = row0 * d.cols + col0;
     TileView t;
     t.w = w + e0;
+    t.w16 = WB ? w16 + e0 : nullptr;
     t.g = BF16 ? static_cast<const void*>(reinterpret_cast<const uint16_t*>(g) + e0)
                : static_cast<const void*>(reinterpret_cast<const float*>(g) + e0);
     t.m_codes = d.m_codes + (e0 >> 1);
@@ -431,11 +453,11 @@ __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __r
         const bool has_b = k + 1 < nrows;
         if (k + kL2Ahead < nrows) prefetch_row<BF16, MSHIFT, FACT>(t, k + kL2Ahead);
         if (has_b) load_row<BF16, MSHIFT, FACT>(rb, t, k + 1);
-        process_row<BF16, EXACT, MSHIFT, FACT>(ra, t, k, c_old, c_rcp, h, h2, lt, s_lut);
+        process_row<BF16, EXACT, MSHIFT, FACT, WB>(ra, t, k, c_old, c_rcp, h, h2, lt, s_lut);
         if (!has_b) break;
         if (k + 1 + kL2Ahead < nrows) prefetch_row<BF16, MSHIFT, FACT>(t, k + 1 + kL2Ahead);
         if (k + 2 < nrows) load_row<BF16, MSHIFT, FACT>(ra, t, k + 2);
-        process_row<BF16, EXACT, MSHIFT, FACT>(rb, t, k + 1, c_old, c_rcp, h, h2, lt, s_lut);
+        process_row<BF16, EXACT, MSHIFT, FACT, WB>(rb, t, k + 1, c_old, c_rcp, h, h2, lt, s_lut);
     }
 }
 
@@ -662,8 +684,9 @@ __device__ __forceinline__ void outer_publish(const TensorDesc& d, float* base, 
 
 // ---- pass 2, flat (element-indexed) tensors: block-wise v, or rank-1 with arbitrary cols ------
 
-template <bool BF16, bool RANK1, bool EXACT, int MSHIFT>
-__device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restrict__ w, const void* __restrict__ g,
+template <bool BF16, bool RANK1, bool EXACT, int MSHIFT, bool WB = false>
+__device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restrict__ w, uint16_t* __restrict__ w16,
+                                           const void* __restrict__ g,
                                            int tile, int phase, const Hyper& h, const Hyper2& h2, const LaneTables& lt,
                                            const unsigned char* s_lut, float* s_red, uint32_t& red_step) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -738,6 +761,9 @@ __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restric
         if (lane_live && (threadIdx.x & (MSHIFT == 7 ? 15 : 2047)) == 0) d.m_scale[e >> MSHIFT] = am_new;
         const uint32_t qm_new = quantize8_de(mt, scale_rcp(am_new), s_lut);
         const uint32_t qv_new = quantize8_lin(vt, vr, h2);
+        if (WB) {
+            if (full) store8_bf16(w16 + e, wv); else store8_bf16_guard(w16, e, d.numel, wv);
+        }
         if (full) {
             store8_f32(w + e, wv);
             *reinterpret_cast<uint32_t*>(d.m_codes + (e >> 1)) = qm_new;
@@ -752,9 +778,9 @@ __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restric
 
 // ---- pass 2, small tensors with fp32 states (App. C.1) ------------------------------------------
 
-template <bool BF16, bool EXACT>
-__device__ __forceinline__ void pass2_fp32(const TensorDesc& d, float* __restrict__ w, const void* __restrict__ g,
-                                           int tile, const Hyper& h) {
+template <bool BF16, bool EXACT, bool WB = false>
+__device__ __forceinline__ void pass2_fp32(const TensorDesc& d, float* __restrict__ w, uint16_t* __restrict__ w16,
+                                           const void* __restrict__ g, int tile, const Hyper& h) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int c = 0; c < d.flat_chunks; ++c) {
         const int64_t chunk = ((int64_t)tile * d.flat_chunks + c) * kWarps + warp;
@@ -774,6 +800,9 @@ __device__ __forceinline__ void pass2_fp32(const TensorDesc& d, float* __restric
             v[k] = ema_v(v[k], gv[k], h);
             wv[k] = update_param<EXACT>(wv[k], m[k], v[k], h);
         }
+        if (WB) {
+            if (full) store8_bf16(w16 + e, wv); else store8_bf16_guard(w16, e, d.numel, wv);
+        }
         if (full) {
             store8_f32(w + e, wv); store8_f32(d.m32 + e, m); store8_f32(d.v32 + e, v);
         } else {
@@ -784,7 +813,8 @@ __device__ __forceinline__ void pass2_fp32(const TensorDesc& d, float* __restric
 
 // VF: the state uses the factorized second moment (then no tensor is of the rank-1 tiled kind, and vice versa),
 // so each instantiation carries only one of the two tiled paths.
-template <bool BF16, bool EXACT, int MSHIFT, bool VF>
+// WB: a bfloat16 copy of every updated parameter is written as well (a.params_bf16).
+template <bool BF16, bool EXACT, int MSHIFT, bool VF, bool WB>
 __global__ void __launch_bounds__(kThreads, 2) pass2_kernel(StepArgs a) {
     __shared__ __align__(16) unsigned char s_lut[kLutSmemBytes];
     __shared__ float s_red[2 * kWarps];
@@ -800,18 +830,19 @@ __global__ void __launch_bounds__(kThreads, 2) pass2_kernel(StepArgs a) {
         const int t = find_tensor(a.tile_start, a.n_tensors, tile);
         const TensorDesc d = a.descs[t];   // by value: the fields stay in registers across the stores below
         float* w = a.params[t];
+        uint16_t* w16 = WB ? a.params_bf16[t] : nullptr;
         const void* g = a.grads[t];
         const int local = tile - __ldg(a.tile_start + t);
         switch (d.kind) {
             case K_RANK1_FAST:
-                if (!VF) pass2_rank1_fast<BF16, EXACT, MSHIFT, false>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step);
+                if (!VF) pass2_rank1_fast<BF16, EXACT, MSHIFT, false, WB>(d, w, w16, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step);
                 break;
             case K_FACT:
-                if (VF) pass2_rank1_fast<BF16, EXACT, MSHIFT, true>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step);
+                if (VF) pass2_rank1_fast<BF16, EXACT, MSHIFT, true, WB>(d, w, w16, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step);
                 break;
-            case K_RANK1_FLAT: pass2_flat<BF16, true, EXACT, MSHIFT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
-            case K_BLOCK:      pass2_flat<BF16, false, EXACT, MSHIFT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
-            default:           pass2_fp32<BF16, EXACT>(d, w, g, local, a.h); break;
+            case K_RANK1_FLAT: pass2_flat<BF16, true, EXACT, MSHIFT, WB>(d, w, w16, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
+            case K_BLOCK:      pass2_flat<BF16, false, EXACT, MSHIFT, WB>(d, w, w16, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
+            default:           pass2_fp32<BF16, EXACT, WB>(d, w, w16, g, local, a.h); break;
         }
         tile = a.tile_begin + tiles_next(s_next, buf, fetched);
     }
@@ -851,11 +882,11 @@ __global__ void __launch_bounds__(kThreads, 2) pass2_bulk_kernel(StepArgs a) {
         switch (d.kind) {
             case K_RANK1_FAST:
                 if ((d.cols & 255) == 0 && MSHIFT == 7) pass2_rank1_bulk<BF16, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, ring, a.dev_status);
-                else pass2_rank1_fast<BF16, EXACT, MSHIFT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step);
+                else pass2_rank1_fast<BF16, EXACT, MSHIFT>(d, w, nullptr, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step);
                 break;
-            case K_RANK1_FLAT: pass2_flat<BF16, true, EXACT, MSHIFT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
-            case K_BLOCK:      pass2_flat<BF16, false, EXACT, MSHIFT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
-            default:           pass2_fp32<BF16, EXACT>(d, w, g, local, a.h); break;
+            case K_RANK1_FLAT: pass2_flat<BF16, true, EXACT, MSHIFT>(d, w, nullptr, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
+            case K_BLOCK:      pass2_flat<BF16, false, EXACT, MSHIFT>(d, w, nullptr, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
+            default:           pass2_fp32<BF16, EXACT>(d, w, nullptr, g, local, a.h); break;
         }
         tile = a.tile_begin + tiles_next(s_next, buf, fetched);
     }
@@ -1274,14 +1305,16 @@ cudaError_t launch_pass1(const StepArgs& a, bool bf16, int grid, cudaStream_t s)
 template <bool BF16, bool EXACT, int MSHIFT>
 cudaError_t launch_pass2_t(const StepArgs& a, bool factored, int grid, cudaStream_t s) {
     if (factored) {
-        pass2_kernel<BF16, EXACT, MSHIFT, true><<<grid, kThreads, 0, s>>>(a);
+        pass2_kernel<BF16, EXACT, MSHIFT, true, false><<<grid, kThreads, 0, s>>>(a);
+    } else if (a.params_bf16 != nullptr) {
+        pass2_kernel<BF16, EXACT, MSHIFT, false, true><<<grid, kThreads, 0, s>>>(a);
     } else if (a.variant == 1) {
         constexpr int smem = bulk_smem_bytes<BF16>();
         cudaError_t e = cudaFuncSetAttribute(pass2_bulk_kernel<BF16, EXACT, MSHIFT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
         pass2_bulk_kernel<BF16, EXACT, MSHIFT><<<grid, kThreads, smem, s>>>(a);
     } else {
-        pass2_kernel<BF16, EXACT, MSHIFT, false><<<grid, kThreads, 0, s>>>(a);
+        pass2_kernel<BF16, EXACT, MSHIFT, false, false><<<grid, kThreads, 0, s>>>(a);
     }
     return cudaGetLastError();
 }
@@ -1321,7 +1354,7 @@ cudaError_t launch_rcp(const float* src, float* dst, int64_t n, cudaStream_t s) 
 cudaError_t step_kernel_occupancy(int* p1, int* p2) {
     cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(p1, pass1_kernel<true>, kThreads, 0);
     if (e != cudaSuccess) return e;
-    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(p2, pass2_kernel<true, false, 7, false>, kThreads, 0);
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(p2, pass2_kernel<true, false, 7, false, false>, kThreads, 0);
 }
 
 }  // namespace lpmm

@@ -26,7 +26,7 @@ FORCE_QUANT, FORCE_FP32 = 1, 2
 Q_GIVEN_SCALES = 1
 KIND_FP32, KIND_BLOCK, KIND_RANK1, KIND_FACTORED = 0, 1, 2, 3
 
-EXPORTS = ("lpmm_state_bytes", "lpmm_state_init", "lpmm_state_attach", "lpmm_adamw4_step",
+EXPORTS = ("lpmm_state_bytes", "lpmm_state_init", "lpmm_state_attach", "lpmm_adamw4_step", "lpmm_adamw4_step_bf16w",
            "lpmm_adamw4_step_host", "lpmm_stage_bytes", "lpmm_quantize", "lpmm_dequantize",
            "lpmm_quantize_rank1_noalloc", "lpmm_sgdm4_step",
            "lpmm_state_view", "lpmm_state_view_axis", "lpmm_state_phase", "lpmm_state_last_launches", "lpmm_state_destroy",
@@ -86,6 +86,7 @@ def lib():
         L.lpmm_state_init.argtypes = [C.POINTER(Config), C.POINTER(Shape), i32, vp, C.c_size_t, C.POINTER(vp), vp]
         L.lpmm_state_attach.argtypes = [C.POINTER(Config), C.POINTER(Shape), i32, vp, C.c_size_t, i32, C.POINTER(vp), vp]
         L.lpmm_adamw4_step.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), i32, f32, f32, f32, f32, f32, i64, vp]
+        L.lpmm_adamw4_step_bf16w.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), i32, f32, f32, f32, f32, f32, i64, vp]
         L.lpmm_adamw4_step_host.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), i32, f32, f32, f32, f32, f32, i64,
                                             vp, vp, C.c_size_t, vp]
         L.lpmm_sgdm4_step.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), i32, f32, f32, vp]
@@ -211,8 +212,10 @@ def _grad_dtype(grads) -> int:
 
 
 def adamw4_step(state: State, params, grads, *, lr, beta1, beta2, eps, weight_decay, step, stream=None,
-                ptr_cache=None) -> None:
-    """lpmm_adamw4_step: params (fp32, updated in place) and grads are lists of contiguous CUDA tensors."""
+                ptr_cache=None, params_bf16=None) -> None:
+    """lpmm_adamw4_step: params (fp32, updated in place) and grads are lists of contiguous CUDA tensors.
+    params_bf16 (optional list of bfloat16 tensors of the same sizes) receives a rounded copy of the new parameters
+    (lpmm_adamw4_step_bf16w)."""
     if len(params) != state.n or len(grads) != state.n:
         raise ValueError("params/grads must have one tensor per state entry")
     if ptr_cache is None:
@@ -226,6 +229,15 @@ def adamw4_step(state: State, params, grads, *, lr, beta1, beta2, eps, weight_de
     else:
         pp, gp, gd = ptr_cache
     with torch.cuda.device(state.arena.device):
+        if params_bf16 is not None:
+            if len(params_bf16) != state.n:
+                raise ValueError("params_bf16 must have one tensor per state entry")
+            for p, c in zip(params, params_bf16):
+                if c.dtype != torch.bfloat16 or not c.is_contiguous() or not c.is_cuda or c.numel() != p.numel():
+                    raise ValueError("bfloat16 copies must be contiguous CUDA tensors of the parameters' sizes")
+            _check(lib().lpmm_adamw4_step_bf16w(state.handle, pp, _ptr_array(params_bf16), gp, gd, lr, beta1, beta2, eps,
+                                                weight_decay, step, _stream_ptr(stream)), "lpmm_adamw4_step_bf16w")
+            return
         _check(lib().lpmm_adamw4_step(state.handle, pp, gp, gd, lr, beta1, beta2, eps, weight_decay, step,
                                       _stream_ptr(stream)), "lpmm_adamw4_step")
 

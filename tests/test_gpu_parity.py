@@ -388,3 +388,38 @@ def test_tensors_with_three_and_four_axes_match_oracle(grad_dtype, update_math):
     with pytest.raises(lpmm.LpmmError) as ei:      # five axes: not supported
         lpmm.state_init(cfg, [_nd(2, 2, 2, 2, 300)])
     assert ei.value.status == lpmm.ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("grad_dtype,m_block", [(torch.bfloat16, 128), (torch.float32, 2048)])
+def test_bf16_copy_of_the_parameters(grad_dtype, m_block):
+    # lpmm_adamw4_step_bf16w: states and fp32 parameters exactly as the plain step leaves them, plus a bfloat16 copy
+    # that is the nearest-even rounding of the new fp32 parameters, on every kind of tensor and on ragged tails.
+    cfg = lpmm.default_config(m_block=m_block)
+    specs = [_mat(96, 256), _mat(64, 2048), _mat(130, 384), _mat(33, 77), _mat(257, 129), _vec(50265), _vec(4097), _vec(300), _vec(1),
+             _nd(6, 10, 200)]
+    hyper = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
+    pa = [workloads.make_param(s, 15, i, device="cuda") for i, s in enumerate(specs)]
+    pb = [p.clone() for p in pa]
+    copies = [torch.full((s.numel,), -7.0, dtype=torch.bfloat16, device="cuda") for s in specs]
+    sa, sb = lpmm.state_init(cfg, specs), lpmm.state_init(cfg, specs)
+    for t in range(1, 4):
+        grads = [workloads.make_grad(s, 15, i, t, device="cuda", dtype=grad_dtype) for i, s in enumerate(specs)]
+        lpmm.adamw4_step(sa, pa, grads, step=t, **hyper)
+        lpmm.adamw4_step(sb, pb, grads, step=t, params_bf16=copies, **hyper)
+        torch.cuda.synchronize()
+        assert lpmm.device_status(sb) == 0
+        for i, s in enumerate(specs):
+            assert torch.equal(pa[i], pb[i]), (s.name, t)
+            va, vb = lpmm.state_view(sa, i), lpmm.state_view(sb, i)
+            for name in ("m_codes", "m_scale", "v_codes", "m32", "v32"):
+                if va[name] is not None:
+                    assert torch.equal(va[name], vb[name]), (s.name, name, t)
+            want = oracle.f32_to_bf16_bits(pb[i].cpu().numpy().ravel())
+            got = copies[i].view(torch.int16).cpu().numpy().view(np.uint16)
+            assert np.array_equal(got, want), (s.name, t)
+    assert sb.last_launches == 3
+    # refused with the factorized second moment, and with a missing pointer array
+    sf = lpmm.state_init(lpmm.default_config(v_mode=lpmm.V_FACTORED), [_mat(96, 256)])
+    with pytest.raises(lpmm.LpmmError) as ei:
+        lpmm.adamw4_step(sf, [pa[0]], [grads[0]], step=1, params_bf16=[copies[0]], **hyper)
+    assert ei.value.status == lpmm.ERR_UNSUPPORTED

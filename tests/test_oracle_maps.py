@@ -145,3 +145,21 @@ def test_reciprocal_rule():
     assert oracle.rcp(3.0) == float(np.float32(1.0) / np.float32(3.0))
     s = np.array([0.0, tiny / 2, tiny, 3.0, 1e30], np.float32)
     assert np.array_equal(onp.rcp(s), np.array([oracle.rcp(float(x)) for x in s], np.float32))
+
+
+def test_bf16_rounding_is_nearest_even():
+    # worked cases: exact values, ties to even in both directions, just off a tie, binade and infinity carries, zeros
+    cases = [(0x3F800000, 0x3F80), (0x3F808000, 0x3F80), (0x3F818000, 0x3F82), (0x3F808001, 0x3F81), (0x3F807FFF, 0x3F80),
+             (0x3FFF8000, 0x4000), (0x7F7FFFFF, 0x7F80), (0x7F800000, 0x7F80), (0x80000000, 0x8000), (0x00000000, 0x0000),
+             (0x00008000, 0x0000), (0x00018000, 0x0002), (0xBF818000, 0xBF82), (0x7FC00001, 0x7FFF), (0xFF800001, 0x7FFF)]
+    x = np.array([c[0] for c in cases], np.uint32).view(np.float32)
+    assert list(oracle.f32_to_bf16_bits(x)) == [c[1] for c in cases]
+    # a library routine on random data (finite values of every magnitude)
+    import torch
+    rng = np.random.default_rng(0)
+    r = (rng.standard_normal(200000) * np.exp(rng.uniform(-80, 80, 200000))).astype(np.float32)
+    want = torch.from_numpy(r).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(oracle.f32_to_bf16_bits(r), want)
+    # and it inverts the exact widening
+    back = oracle.bf16_bits_to_f32(want)
+    assert np.array_equal(oracle.f32_to_bf16_bits(back), want)
