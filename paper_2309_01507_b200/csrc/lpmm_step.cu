@@ -449,7 +449,16 @@ __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __r
 #pragma unroll
     for (uint32_t k = 1; k < kL2Ahead; ++k) if (k < nrows) prefetch_row<BF16, MSHIFT, FACT>(t, k);
     load_row<BF16, MSHIFT, FACT>(ra, t, 0);
-    for (uint32_t k = 0; k < nrows; k += 2) {
+    uint32_t k = 0;
+    for (; k + 1 + kL2Ahead < nrows; k += 2) {        // every row touched below exists: no guards
+        prefetch_row<BF16, MSHIFT, FACT>(t, k + kL2Ahead);
+        load_row<BF16, MSHIFT, FACT>(rb, t, k + 1);
+        process_row<BF16, EXACT, MSHIFT, FACT, WB>(ra, t, k, c_old, c_rcp, h, h2, lt, s_lut);
+        prefetch_row<BF16, MSHIFT, FACT>(t, k + 1 + kL2Ahead);
+        load_row<BF16, MSHIFT, FACT>(ra, t, k + 2);
+        process_row<BF16, EXACT, MSHIFT, FACT, WB>(rb, t, k + 1, c_old, c_rcp, h, h2, lt, s_lut);
+    }
+    for (; k < nrows; k += 2) {                       // the last rows of the tile
         const bool has_b = k + 1 < nrows;
         if (k + kL2Ahead < nrows) prefetch_row<BF16, MSHIFT, FACT>(t, k + kL2Ahead);
         if (has_b) load_row<BF16, MSHIFT, FACT>(rb, t, k + 1);
