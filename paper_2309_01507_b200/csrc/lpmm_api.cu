@@ -208,8 +208,10 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
     const int32_t n = st->n;
     int64_t total_elems = 0;
     for (int32_t i = 0; i < n; ++i) total_elems += st->L.t[i].numel;
-    // aim at >= 4 tiles per resident CTA, tiles between 2 Ki and 128 Ki elements (powers of two)
-    int64_t target = total_elems / (4LL * sms * occ2);
+    // aim at >= 6 tiles per resident CTA of the update pass (tiles are handed out on demand, the tail is what is
+    // balanced), tiles between 2 Ki and 256 Ki elements (powers of two). Measured optima: 32 Ki for 60-70 M
+    // parameters, 64-128 Ki for 355 M, 256 Ki for 6.7 G.
+    int64_t target = total_elems / (6LL * sms * occ2);
     int64_t tile_elems = 2048;
     while (tile_elems * 2 <= target && tile_elems < 262144) tile_elems *= 2;
     if (const char* v = std::getenv("LPMM_TILE_ELEMS")) {   // development switch
