@@ -450,7 +450,8 @@ __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __r
     for (uint32_t k = 1; k < kL2Ahead; ++k) if (k < nrows) prefetch_row<BF16, MSHIFT, FACT>(t, k);
     load_row<BF16, MSHIFT, FACT>(ra, t, 0);
     uint32_t k = 0;
-    for (; k + 1 + kL2Ahead < nrows; k += 2) {        // every row touched below exists: no guards
+    // (B2048 rows end in a CTA-wide barrier, where the longer straight-line body only costs registers: guarded loop only)
+    for (; MSHIFT == 7 && k + 1 + kL2Ahead < nrows; k += 2) {        // every row touched below exists: no guards
         prefetch_row<BF16, MSHIFT, FACT>(t, k + kL2Ahead);
         load_row<BF16, MSHIFT, FACT>(rb, t, k + 1);
         process_row<BF16, EXACT, MSHIFT, FACT, WB>(ra, t, k, c_old, c_rcp, h, h2, lt, s_lut);
