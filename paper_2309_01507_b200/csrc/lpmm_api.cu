@@ -183,6 +183,7 @@ struct lpmm_state {
     bool ptrs_valid;
     std::vector<void*> params, grads;  // what the device-side pointer arrays currently hold
     std::vector<void*> params16;       // likewise for the optional bfloat16 copies (empty until first used)
+    bool params_a32 = false, grads_a32 = false;   // all current parameter / gradient pointers are 32-byte aligned
     size_t stage_bytes;
     std::vector<size_t> stage_off;
     int32_t pass2_variant;                 // 0 = register prefetch, 1 = bulk-copy staging
@@ -394,7 +395,13 @@ lpmm_status set_pointers(lpmm_state* st, void* const* d_params, const void* cons
         if (d_params[i] != st->params[i] || d_grads[i] != st->grads[i]) changed = true;
     }
     if (changed) {
-        for (int32_t i = 0; i < n; ++i) { st->params[i] = d_params[i]; st->grads[i] = const_cast<void*>(d_grads[i]); }
+        bool pa = true, ga = true;
+        for (int32_t i = 0; i < n; ++i) {
+            st->params[i] = d_params[i]; st->grads[i] = const_cast<void*>(d_grads[i]);
+            pa = pa && (reinterpret_cast<uintptr_t>(d_params[i]) & 31u) == 0;
+            ga = ga && (reinterpret_cast<uintptr_t>(d_grads[i]) & 31u) == 0;
+        }
+        st->params_a32 = pa; st->grads_a32 = ga;
         st->ptrs_valid = false;
         LPMM_CUDA(cudaMemcpyAsync(st->arena + st->L.params, st->params.data(), sizeof(void*) * n, cudaMemcpyHostToDevice, s));
         LPMM_CUDA(cudaMemcpyAsync(st->arena + st->L.grads, st->grads.data(), sizeof(void*) * n, cudaMemcpyHostToDevice, s));
@@ -412,6 +419,7 @@ StepArgs make_args(const lpmm_state* st, float lr, float beta1, float beta2, flo
     a.n_tensors = st->n;
     a.phase = st->phase;
     a.variant = st->pass2_variant;
+    a.aligned32 = 0;   // set by the callers that know the gradient type
     a.dev_status = reinterpret_cast<uint32_t*>(st->arena);
     a.tile_counter = reinterpret_cast<int32_t*>(st->arena + 16);   // header block: [status | .. | counters]
     a.h.lr = lr; a.h.beta1 = beta1; a.h.beta2 = beta2; a.h.eps = eps;
@@ -443,6 +451,7 @@ bool wants_ieee_update(const lpmm_state* st, const Hyper& h) {
 // Enqueues the three kernels of one step for tensors [t0, t1). ev (4 events or nullptr) brackets the kernels.
 lpmm_status enqueue_range(lpmm_state* st, StepArgs a, int32_t t0, int32_t t1, bool bf16, bool ieee_update,
                           cudaStream_t s, cudaEvent_t* ev, int32_t* launches) {
+    a.aligned32 = (st->params_a32 && (bf16 || st->grads_a32)) ? 1 : 0;
     const int32_t p1_begin = st->tiles1[t0], p1_end = st->tiles1[t1];
     if (p1_end > p1_begin) {
         // the rank-1 scale region of these tensors is one contiguous range of the scale buffers

@@ -54,6 +54,7 @@ struct StepArgs {
     int32_t tile_begin, tile_end;  // this launch covers tiles [tile_begin, tile_end) of the prefix table
     int32_t phase;               // rc[phase] holds the current r, c; rc[1 - phase] receives the new ones
     int32_t variant;             // pass 2: 0 = rows prefetched into registers, 1 = rows staged by bulk copies
+    int32_t aligned32;           // every parameter (and fp32 gradient) pointer is 32-byte aligned: 256-bit accesses
     uint32_t* dev_status;        // device error word in the arena header (0 = ok)
     int32_t* tile_counter;       // two words in the arena header: next tile of this launch, finished CTAs (both 0 between launches)
     Hyper h;

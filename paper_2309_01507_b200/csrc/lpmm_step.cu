@@ -267,6 +267,21 @@ __device__ __forceinline__ void unpack_grad8(const uint4& g0, const uint4& g1, f
     }
 }
 
+// 256-bit global accesses (sm_100): a lane's 8 fp32 values in one instruction instead of two. The address must be
+// 32-byte aligned; callers check the tensor's base pointer once per tile and fall back to two 128-bit accesses.
+__device__ __forceinline__ void load8_f32_256(const float* p, float4& a, float4& b) {
+    asm volatile("ld.global.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=f"(a.x), "=f"(a.y), "=f"(a.z), "=f"(a.w), "=f"(b.x), "=f"(b.y), "=f"(b.z), "=f"(b.w) : "l"(p));
+}
+__device__ __forceinline__ void load8_u32_256_nc(const void* p, uint4& a, uint4& b) {
+    asm volatile("ld.global.nc.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w), "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w) : "l"(p));
+}
+__device__ __forceinline__ void store8_f32_256(float* p, const float (&x)[8]) {
+    asm volatile("st.global.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 :: "l"(p), "f"(x[0]), "f"(x[1]), "f"(x[2]), "f"(x[3]), "f"(x[4]), "f"(x[5]), "f"(x[6]), "f"(x[7]) : "memory");
+}
+
 // ---- pass 2, rank-1 tensors with cols % 128 == 0 ---------------------------------------------------
 
 template <bool BF16>
@@ -340,13 +355,20 @@ __device__ __forceinline__ void prefetch_roles(TileView& t, int lane, int valid,
     }
 }
 
-template <bool BF16, int MSHIFT, bool FACT>
+// A32: the parameter rows (and fp32 gradient rows) of this tensor are 32-byte aligned.
+template <bool BF16, int MSHIFT, bool FACT, bool A32>
 __device__ __forceinline__ void load_row(RowRegs<BF16>& r, const TileView& t, uint32_t k) {
     const uint32_t off = k * t.row_step;
-    r.w0 = *reinterpret_cast<const float4*>(t.w + off);
-    r.w1 = *reinterpret_cast<const float4*>(t.w + off + 4);
+    if (A32) {
+        load8_f32_256(t.w + off, r.w0, r.w1);
+    } else {
+        r.w0 = *reinterpret_cast<const float4*>(t.w + off);
+        r.w1 = *reinterpret_cast<const float4*>(t.w + off + 4);
+    }
     if (BF16) {
         r.g0 = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(t.g) + off));
+    } else if (A32) {
+        load8_u32_256_nc(reinterpret_cast<const float*>(t.g) + off, r.g0, r.g1);
     } else {
         r.g0 = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(t.g) + off));
         r.g1 = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(t.g) + off + 4));
@@ -363,7 +385,7 @@ __device__ __forceinline__ void load_row(RowRegs<BF16>& r, const TileView& t, ui
     }
 }
 
-template <bool BF16, bool EXACT, int MSHIFT, bool FACT, bool WB>
+template <bool BF16, bool EXACT, int MSHIFT, bool FACT, bool WB, bool A32>
 __device__ __forceinline__ void process_row(const RowRegs<BF16>& r, const TileView& t, uint32_t k,
                                             const float (&c_old)[8], const float (&c_rcp)[8], const Hyper& h,
                                             const Hyper2& h2, const LaneTables& lt, const unsigned char* s_lut) {
@@ -382,7 +404,7 @@ __device__ __forceinline__ void process_row(const RowRegs<BF16>& r, const TileVi
         }
     }
     moments_and_update8<EXACT, FACT>(wv, gv, r.qm, r.qv, __fmul_rn(lt.de, r.am), vs, h, h2, lt, mt, vt);
-    store8_f32(t.w + off, wv);
+    if (A32) store8_f32_256(t.w + off, wv); else store8_f32(t.w + off, wv);
     if (WB) store8_bf16(t.w16 + off, wv);
     const float am_new = block_max(absmax8(mt), MSHIFT, lt, t.s_red, *t.red_step);
     if ((threadIdx.x & (MSHIFT == 7 ? 15 : 2047)) == 0) t.m_scale[off >> MSHIFT] = am_new;
@@ -390,7 +412,7 @@ __device__ __forceinline__ void process_row(const RowRegs<BF16>& r, const TileVi
     if (!FACT) *reinterpret_cast<uint32_t*>(t.v_codes + (off >> 1)) = quantize8_lin(vt, vr, h2);
 }
 
-template <bool BF16, bool EXACT, int MSHIFT, bool FACT = false, bool WB = false>
+template <bool BF16, bool EXACT, int MSHIFT, bool FACT = false, bool WB = false, bool A32 = false>
 __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __restrict__ w, uint16_t* __restrict__ w16,
                                                  const void* __restrict__ g,
                                                  int tile, int phase, const Hyper& h, const Hyper2& h2,
@@ -448,26 +470,26 @@ __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __r
     RowRegs<BF16> ra, rb;
 #pragma unroll
     for (uint32_t k = 1; k < kL2Ahead; ++k) if (k < nrows) prefetch_row<BF16, MSHIFT, FACT>(t, k);
-    load_row<BF16, MSHIFT, FACT>(ra, t, 0);
+    load_row<BF16, MSHIFT, FACT, A32>(ra, t, 0);
     uint32_t k = 0;
     // (B2048 rows end in a CTA-wide barrier, where the longer straight-line body only costs registers: guarded loop only)
     for (; MSHIFT == 7 && k + 1 + kL2Ahead < nrows; k += 2) {        // every row touched below exists: no guards
         prefetch_row<BF16, MSHIFT, FACT>(t, k + kL2Ahead);
-        load_row<BF16, MSHIFT, FACT>(rb, t, k + 1);
-        process_row<BF16, EXACT, MSHIFT, FACT, WB>(ra, t, k, c_old, c_rcp, h, h2, lt, s_lut);
+        load_row<BF16, MSHIFT, FACT, A32>(rb, t, k + 1);
+        process_row<BF16, EXACT, MSHIFT, FACT, WB, A32>(ra, t, k, c_old, c_rcp, h, h2, lt, s_lut);
         prefetch_row<BF16, MSHIFT, FACT>(t, k + 1 + kL2Ahead);
-        load_row<BF16, MSHIFT, FACT>(ra, t, k + 2);
-        process_row<BF16, EXACT, MSHIFT, FACT, WB>(rb, t, k + 1, c_old, c_rcp, h, h2, lt, s_lut);
+        load_row<BF16, MSHIFT, FACT, A32>(ra, t, k + 2);
+        process_row<BF16, EXACT, MSHIFT, FACT, WB, A32>(rb, t, k + 1, c_old, c_rcp, h, h2, lt, s_lut);
     }
     for (; k < nrows; k += 2) {                       // the last rows of the tile
         const bool has_b = k + 1 < nrows;
         if (k + kL2Ahead < nrows) prefetch_row<BF16, MSHIFT, FACT>(t, k + kL2Ahead);
-        if (has_b) load_row<BF16, MSHIFT, FACT>(rb, t, k + 1);
-        process_row<BF16, EXACT, MSHIFT, FACT, WB>(ra, t, k, c_old, c_rcp, h, h2, lt, s_lut);
+        if (has_b) load_row<BF16, MSHIFT, FACT, A32>(rb, t, k + 1);
+        process_row<BF16, EXACT, MSHIFT, FACT, WB, A32>(ra, t, k, c_old, c_rcp, h, h2, lt, s_lut);
         if (!has_b) break;
         if (k + 1 + kL2Ahead < nrows) prefetch_row<BF16, MSHIFT, FACT>(t, k + 1 + kL2Ahead);
-        if (k + 2 < nrows) load_row<BF16, MSHIFT, FACT>(ra, t, k + 2);
-        process_row<BF16, EXACT, MSHIFT, FACT, WB>(rb, t, k + 1, c_old, c_rcp, h, h2, lt, s_lut);
+        if (k + 2 < nrows) load_row<BF16, MSHIFT, FACT, A32>(ra, t, k + 2);
+        process_row<BF16, EXACT, MSHIFT, FACT, WB, A32>(rb, t, k + 1, c_old, c_rcp, h, h2, lt, s_lut);
     }
 }
 
@@ -824,7 +846,9 @@ __device__ __forceinline__ void pass2_fp32(const TensorDesc& d, float* __restric
 // VF: the state uses the factorized second moment (then no tensor is of the rank-1 tiled kind, and vice versa),
 // so each instantiation carries only one of the two tiled paths.
 // WB: a bfloat16 copy of every updated parameter is written as well (a.params_bf16).
-template <bool BF16, bool EXACT, int MSHIFT, bool VF, bool WB>
+// A32: every parameter pointer (and, with fp32 gradients, every gradient pointer) of the step is 32-byte aligned,
+// checked on the host: the tiled path then moves a lane's 8 values with one 256-bit access.
+template <bool BF16, bool EXACT, int MSHIFT, bool VF, bool WB, bool A32>
 __global__ void __launch_bounds__(kThreads, 2) pass2_kernel(StepArgs a) {
     __shared__ __align__(16) unsigned char s_lut[kLutSmemBytes];
     __shared__ float s_red[2 * kWarps];
@@ -845,7 +869,7 @@ __global__ void __launch_bounds__(kThreads, 2) pass2_kernel(StepArgs a) {
         const int local = tile - __ldg(a.tile_start + t);
         switch (d.kind) {
             case K_RANK1_FAST:
-                if (!VF) pass2_rank1_fast<BF16, EXACT, MSHIFT, false, WB>(d, w, w16, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step);
+                if (!VF) pass2_rank1_fast<BF16, EXACT, MSHIFT, false, WB, A32>(d, w, w16, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step);
                 break;
             case K_FACT:
                 if (VF) pass2_rank1_fast<BF16, EXACT, MSHIFT, true, WB>(d, w, w16, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step);
@@ -1315,16 +1339,19 @@ cudaError_t launch_pass1(const StepArgs& a, bool bf16, int grid, cudaStream_t s)
 template <bool BF16, bool EXACT, int MSHIFT>
 cudaError_t launch_pass2_t(const StepArgs& a, bool factored, int grid, cudaStream_t s) {
     if (factored) {
-        pass2_kernel<BF16, EXACT, MSHIFT, true, false><<<grid, kThreads, 0, s>>>(a);
+        pass2_kernel<BF16, EXACT, MSHIFT, true, false, false><<<grid, kThreads, 0, s>>>(a);
     } else if (a.params_bf16 != nullptr) {
-        pass2_kernel<BF16, EXACT, MSHIFT, false, true><<<grid, kThreads, 0, s>>>(a);
+        if (a.aligned32) pass2_kernel<BF16, EXACT, MSHIFT, false, true, true><<<grid, kThreads, 0, s>>>(a);
+        else pass2_kernel<BF16, EXACT, MSHIFT, false, true, false><<<grid, kThreads, 0, s>>>(a);
     } else if (a.variant == 1) {
         constexpr int smem = bulk_smem_bytes<BF16>();
         cudaError_t e = cudaFuncSetAttribute(pass2_bulk_kernel<BF16, EXACT, MSHIFT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
         pass2_bulk_kernel<BF16, EXACT, MSHIFT><<<grid, kThreads, smem, s>>>(a);
+    } else if (a.aligned32) {
+        pass2_kernel<BF16, EXACT, MSHIFT, false, false, true><<<grid, kThreads, 0, s>>>(a);
     } else {
-        pass2_kernel<BF16, EXACT, MSHIFT, false, false><<<grid, kThreads, 0, s>>>(a);
+        pass2_kernel<BF16, EXACT, MSHIFT, false, false, false><<<grid, kThreads, 0, s>>>(a);
     }
     return cudaGetLastError();
 }
@@ -1364,7 +1391,7 @@ cudaError_t launch_rcp(const float* src, float* dst, int64_t n, cudaStream_t s) 
 cudaError_t step_kernel_occupancy(int* p1, int* p2) {
     cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(p1, pass1_kernel<true>, kThreads, 0);
     if (e != cudaSuccess) return e;
-    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(p2, pass2_kernel<true, false, 7, false, false>, kThreads, 0);
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(p2, pass2_kernel<true, false, 7, false, false, true>, kThreads, 0);
 }
 
 }  // namespace lpmm

@@ -423,3 +423,35 @@ def test_bf16_copy_of_the_parameters(grad_dtype, m_block):
     with pytest.raises(lpmm.LpmmError) as ei:
         lpmm.adamw4_step(sf, [pa[0]], [grads[0]], step=1, params_bf16=[copies[0]], **hyper)
     assert ei.value.status == lpmm.ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("grad_dtype", [torch.bfloat16, torch.float32])
+def test_pointers_aligned_to_16_but_not_32_bytes_give_the_same_result(grad_dtype):
+    # The tiled update pass moves a lane's eight fp32 values with one 256-bit access when every pointer is 32-byte
+    # aligned and with two 128-bit accesses otherwise; both must leave identical parameters and states.
+    cfg = lpmm.default_config()
+    specs = [_mat(96, 256), _mat(64, 1024), _mat(130, 384), _vec(5000)]
+    hyper = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
+    pa = [workloads.make_param(s, 16, i, device="cuda") for i, s in enumerate(specs)]
+    store = [torch.empty(s.numel + 16, device="cuda") for s in specs]           # fp32: 4 elements = 16 bytes
+    pb = [b[4:4 + s.numel] for b, s in zip(store, specs)]
+    for a, b in zip(pa, pb):
+        b.copy_(a.ravel())
+        assert a.data_ptr() % 32 == 0 and b.data_ptr() % 32 == 16
+    sa, sb = lpmm.state_init(cfg, specs), lpmm.state_init(cfg, specs)
+    for t in range(1, 4):
+        grads = [workloads.make_grad(s, 16, i, t, device="cuda", dtype=grad_dtype) for i, s in enumerate(specs)]
+        per = 16 // grads[0].element_size()
+        gstore = [torch.empty(s.numel + 2 * per, device="cuda", dtype=grad_dtype) for s in specs]
+        gb = [b[per:per + s.numel] for b, s in zip(gstore, specs)]
+        for g, b in zip(grads, gb):
+            b.copy_(g.ravel())
+        lpmm.adamw4_step(sa, pa, grads, step=t, **hyper)
+        lpmm.adamw4_step(sb, pb, gb, step=t, **hyper)
+        torch.cuda.synchronize()
+        for i, s in enumerate(specs):
+            assert torch.equal(pa[i].ravel(), pb[i]), (s.name, t)
+            va, vb = lpmm.state_view(sa, i), lpmm.state_view(sb, i)
+            for name in ("m_codes", "m_scale", "v_codes", "v_s0", "v_s1"):
+                if va[name] is not None:
+                    assert torch.equal(va[name], vb[name]), (s.name, name, t)
