@@ -282,6 +282,32 @@ __device__ __forceinline__ void store8_f32_256(float* p, const float (&x)[8]) {
                  :: "l"(p), "f"(x[0]), "f"(x[1]), "f"(x[2]), "f"(x[3]), "f"(x[4]), "f"(x[5]), "f"(x[6]), "f"(x[7]) : "memory");
 }
 
+template <bool A32>
+__device__ __forceinline__ void load8_rw_a(const float* p, float (&x)[8]) {
+    if (A32) {
+        float4 a, b;
+        load8_f32_256(p, a, b);
+        x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+    } else {
+        load8_rw(p, x);
+    }
+}
+template <bool A32>
+__device__ __forceinline__ void store8_f32_a(float* p, const float (&x)[8]) {
+    if (A32) store8_f32_256(p, x); else store8_f32(p, x);
+}
+template <bool BF16, bool A32>
+__device__ __forceinline__ void load8_grad_a(const void* g, int64_t e, float (&x)[8]) {
+    if (!BF16 && A32) {
+        uint4 a, b;
+        load8_u32_256_nc(reinterpret_cast<const float*>(g) + e, a, b);
+        x[0] = __uint_as_float(a.x); x[1] = __uint_as_float(a.y); x[2] = __uint_as_float(a.z); x[3] = __uint_as_float(a.w);
+        x[4] = __uint_as_float(b.x); x[5] = __uint_as_float(b.y); x[6] = __uint_as_float(b.z); x[7] = __uint_as_float(b.w);
+    } else {
+        load8_grad<BF16>(g, e, x);
+    }
+}
+
 // ---- pass 2, rank-1 tensors with cols % 128 == 0 ---------------------------------------------------
 
 template <bool BF16>
@@ -716,7 +742,7 @@ __device__ __forceinline__ void outer_publish(const TensorDesc& d, float* base, 
 
 // ---- pass 2, flat (element-indexed) tensors: block-wise v, or rank-1 with arbitrary cols ------
 
-template <bool BF16, bool RANK1, bool EXACT, int MSHIFT, bool WB = false>
+template <bool BF16, bool RANK1, bool EXACT, int MSHIFT, bool WB = false, bool A32 = false>
 __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restrict__ w, uint16_t* __restrict__ w16,
                                            const void* __restrict__ g,
                                            int tile, int phase, const Hyper& h, const Hyper2& h2, const LaneTables& lt,
@@ -737,8 +763,8 @@ __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restric
         float wv[8], gv[8], mt[8], vt[8], vs[8], vr[8];
         uint32_t qm, qv;
         if (full) {
-            load8_rw(w + e, wv);
-            load8_grad<BF16>(g, e, gv);
+            load8_rw_a<A32>(w + e, wv);
+            load8_grad_a<BF16, A32>(g, e, gv);
             qm = __ldg(reinterpret_cast<const uint32_t*>(d.m_codes + (e >> 1)));
             qv = __ldg(reinterpret_cast<const uint32_t*>(d.v_codes + (e >> 1)));
         } else {
@@ -797,7 +823,7 @@ __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restric
             if (full) store8_bf16(w16 + e, wv); else store8_bf16_guard(w16, e, d.numel, wv);
         }
         if (full) {
-            store8_f32(w + e, wv);
+            store8_f32_a<A32>(w + e, wv);
             *reinterpret_cast<uint32_t*>(d.m_codes + (e >> 1)) = qm_new;
             *reinterpret_cast<uint32_t*>(d.v_codes + (e >> 1)) = qv_new;
         } else {
@@ -810,7 +836,7 @@ __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restric
 
 // ---- pass 2, small tensors with fp32 states (App. C.1) ------------------------------------------
 
-template <bool BF16, bool EXACT, bool WB = false>
+template <bool BF16, bool EXACT, bool WB = false, bool A32 = false>
 __device__ __forceinline__ void pass2_fp32(const TensorDesc& d, float* __restrict__ w, uint16_t* __restrict__ w16,
                                            const void* __restrict__ g, int tile, const Hyper& h) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -821,7 +847,8 @@ __device__ __forceinline__ void pass2_fp32(const TensorDesc& d, float* __restric
         const bool full = (chunk + 1) * kWarpElems <= d.numel;
         float wv[8], gv[8], m[8], v[8];
         if (full) {
-            load8_rw(w + e, wv); load8_grad<BF16>(g, e, gv); load8_rw(d.m32 + e, m); load8_rw(d.v32 + e, v);
+            // (the fp32 states live in the arena at 256-byte aligned offsets: always 32-byte aligned here)
+            load8_rw_a<A32>(w + e, wv); load8_grad_a<BF16, A32>(g, e, gv); load8_rw_a<true>(d.m32 + e, m); load8_rw_a<true>(d.v32 + e, v);
         } else {
             load8_guard(w, e, d.numel, wv); load8_grad_guard<BF16>(g, e, d.numel, gv);
             load8_guard(d.m32, e, d.numel, m); load8_guard(d.v32, e, d.numel, v);
@@ -836,7 +863,7 @@ __device__ __forceinline__ void pass2_fp32(const TensorDesc& d, float* __restric
             if (full) store8_bf16(w16 + e, wv); else store8_bf16_guard(w16, e, d.numel, wv);
         }
         if (full) {
-            store8_f32(w + e, wv); store8_f32(d.m32 + e, m); store8_f32(d.v32 + e, v);
+            store8_f32_a<A32>(w + e, wv); store8_f32_a<true>(d.m32 + e, m); store8_f32_a<true>(d.v32 + e, v);
         } else {
             store8_guard(w, e, d.numel, wv); store8_guard(d.m32, e, d.numel, m); store8_guard(d.v32, e, d.numel, v);
         }
@@ -874,9 +901,9 @@ __global__ void __launch_bounds__(kThreads, 2) pass2_kernel(StepArgs a) {
             case K_FACT:
                 if (VF) pass2_rank1_fast<BF16, EXACT, MSHIFT, true, WB>(d, w, w16, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step);
                 break;
-            case K_RANK1_FLAT: pass2_flat<BF16, true, EXACT, MSHIFT, WB>(d, w, w16, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
-            case K_BLOCK:      pass2_flat<BF16, false, EXACT, MSHIFT, WB>(d, w, w16, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
-            default:           pass2_fp32<BF16, EXACT, WB>(d, w, w16, g, local, a.h); break;
+            case K_RANK1_FLAT: pass2_flat<BF16, true, EXACT, MSHIFT, WB, A32>(d, w, w16, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
+            case K_BLOCK:      pass2_flat<BF16, false, EXACT, MSHIFT, WB, A32>(d, w, w16, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
+            default:           pass2_fp32<BF16, EXACT, WB, A32>(d, w, w16, g, local, a.h); break;
         }
         tile = a.tile_begin + tiles_next(s_next, buf, fetched);
     }
