@@ -250,7 +250,8 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
             d.wx = (st->cfg.m_block == 2048) ? 8 : (t.cols % 1024 == 0) ? 4 : (t.cols % 512 == 0) ? 2 : 1;
             const int64_t tile_cols = (int64_t)kWarpElems * d.wx;
             int64_t tr = tile_elems / tile_cols;
-            if (tr < kWarps / d.wx) tr = kWarps / d.wx;
+            // at least four rows per warp: the maxima pass works in trips of four rows (shorter tiles repeat rows)
+            if (tr < 4 * (kWarps / d.wx)) tr = 4 * (kWarps / d.wx);
             d.tile_rows = (int32_t)tr;
             d.tiles_x = (int32_t)((t.cols + tile_cols - 1) / tile_cols);
             tiles = (int64_t)d.tiles_x * ((t.rows + tr - 1) / tr);

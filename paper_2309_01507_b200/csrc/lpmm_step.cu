@@ -1056,6 +1056,33 @@ __device__ __forceinline__ float p1_process_row(const P1Row<BF16>& b, float r_ol
     return rm;
 }
 
+// Two rows at once: the column maxima take one three-input maximum per column for both rows.
+template <bool BF16>
+__device__ __forceinline__ void p1_process_2rows(const P1Row<BF16>& a, const P1Row<BF16>& b, float ra_old, float rb_old,
+                                                 const float (&c_old)[8], float (&c_max)[8], const Hyper2& h2,
+                                                 const LaneTables& lt, float& rm_a, float& rm_b) {
+    float ga[8], gb[8];
+    unpack_grad8<BF16>(a.g0, a.g1, ga);
+    unpack_grad8<BF16>(b.g0, b.g1, gb);
+    rm_a = 0.0f;
+    rm_b = 0.0f;
+#pragma unroll
+    for (int k = 0; k < 8; k += 2) {
+        const float2 ta = make_float2(__shfl_sync(0xffffffffu, lt.lin, (int)(a.qv >> (4 * k)), 16),
+                                      __shfl_sync(0xffffffffu, lt.lin, (int)(a.qv >> (4 * k + 4)), 16));
+        const float2 tb = make_float2(__shfl_sync(0xffffffffu, lt.lin, (int)(b.qv >> (4 * k)), 16),
+                                      __shfl_sync(0xffffffffu, lt.lin, (int)(b.qv >> (4 * k + 4)), 16));
+        const float2 sa = make_float2(fminf(ra_old, c_old[k]), fminf(ra_old, c_old[k + 1]));
+        const float2 sb = make_float2(fminf(rb_old, c_old[k]), fminf(rb_old, c_old[k + 1]));
+        const float2 va = ema_v2(mul2_rn(ta, sa), make_float2(ga[k], ga[k + 1]), h2);
+        const float2 vb = ema_v2(mul2_rn(tb, sb), make_float2(gb[k], gb[k + 1]), h2);
+        rm_a = fmaxf(rm_a, fmaxf(va.x, va.y));
+        rm_b = fmaxf(rm_b, fmaxf(vb.x, vb.y));
+        c_max[k] = fmaxf(c_max[k], fmaxf(va.x, vb.x));
+        c_max[k + 1] = fmaxf(c_max[k + 1], fmaxf(va.y, vb.y));
+    }
+}
+
 constexpr uint32_t kP1L2Ahead = 8;  // rows the L2 prefetch hints run ahead
 
 template <bool BF16>
@@ -1099,33 +1126,34 @@ __device__ __forceinline__ void pass1_rank1_fast(const TensorDesc& d, const void
     // Lane j keeps the old row scale of the warp's row number base + j (32 rows per refill); a row's scale is
     // then read with one shuffle instead of a load.
     float r_vec = 0.0f;
-    P1Row<BF16> ra, rb;                               // two register sets alternate: the next row is always in flight
-    load_p1_row<BF16>(ra, t, 0);
+    // Four register sets: the rows of a trip were loaded during the previous trip (four rows of loads in flight per
+    // lane). Maxima are idempotent, so row numbers are clamped to the tile's last row instead of guarded: a trip
+    // past the end re-reads that row and contributes the same values again, and the loop body has no branches.
+    P1Row<BF16> s0, s1, s2, s3;
+    const uint32_t last = nrows - 1;
+    load_p1_row<BF16>(s0, t, 0);
+    load_p1_row<BF16>(s1, t, min(1u, last));
+    load_p1_row<BF16>(s2, t, min(2u, last));
+    load_p1_row<BF16>(s3, t, min(3u, last));
     for (uint32_t k = 0; k < nrows; k += 4) {         // four rows per trip so that their maxima reduce together
         if ((k & 31) == 0) {
-            const uint32_t kk = min(k + lane, nrows - 1);
+            const uint32_t kk = min(k + lane, last);
             r_vec = __ldg(rc_old + row0 + (int64_t)kk * wy_count);
         }
 #pragma unroll
         for (uint32_t u = 0; u < 4; u += P1Pf<BF16>::kRows) prefetch_p1_group<BF16>(t, k + kP1L2Ahead + u, nrows);
-        float r_max[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-        if (k + 1 < nrows) load_p1_row<BF16>(rb, t, k + 1);
-        r_max[0] = p1_process_row<BF16>(ra, __shfl_sync(0xffffffffu, r_vec, k & 31), c_old, c_max, h2, lt);
-        if (k + 1 < nrows) {
-            if (k + 2 < nrows) load_p1_row<BF16>(ra, t, k + 2);
-            r_max[1] = p1_process_row<BF16>(rb, __shfl_sync(0xffffffffu, r_vec, (k + 1) & 31), c_old, c_max, h2, lt);
-        }
-        if (k + 2 < nrows) {
-            if (k + 3 < nrows) load_p1_row<BF16>(rb, t, k + 3);
-            r_max[2] = p1_process_row<BF16>(ra, __shfl_sync(0xffffffffu, r_vec, (k + 2) & 31), c_old, c_max, h2, lt);
-        }
-        if (k + 3 < nrows) {
-            if (k + 4 < nrows) load_p1_row<BF16>(ra, t, k + 4);
-            r_max[3] = p1_process_row<BF16>(rb, __shfl_sync(0xffffffffu, r_vec, (k + 3) & 31), c_old, c_max, h2, lt);
-        }
+        float r_max[4];
+        p1_process_2rows<BF16>(s0, s1, __shfl_sync(0xffffffffu, r_vec, k & 31), __shfl_sync(0xffffffffu, r_vec, (k + 1) & 31),
+                               c_old, c_max, h2, lt, r_max[0], r_max[1]);
+        load_p1_row<BF16>(s0, t, min(k + 4, last));
+        load_p1_row<BF16>(s1, t, min(k + 5, last));
+        p1_process_2rows<BF16>(s2, s3, __shfl_sync(0xffffffffu, r_vec, (k + 2) & 31), __shfl_sync(0xffffffffu, r_vec, (k + 3) & 31),
+                               c_old, c_max, h2, lt, r_max[2], r_max[3]);
+        load_p1_row<BF16>(s2, t, min(k + 6, last));
+        load_p1_row<BF16>(s3, t, min(k + 7, last));
         const float rm = warp_max4(r_max, lane);
-        const uint32_t kr = k + ((lane >> 4) & 1) * 2 + ((lane >> 3) & 1);   // the row whose maximum this lane holds
-        if ((lane & 7) == 0 && kr < nrows) atomic_max_nonneg(rc_new + row0 + (int64_t)kr * wy_count, rm);
+        const uint32_t kr = min(k + ((lane >> 4) & 1) * 2 + ((lane >> 3) & 1), last);   // the row whose maximum this lane holds
+        if ((lane & 7) == 0) atomic_max_nonneg(rc_new + row0 + (int64_t)kr * wy_count, rm);
     }
     // Column maxima: transpose through this warp's slice of shared memory so that consecutive lanes hold
     // consecutive columns, then one atomic per column. Only the warp itself touches its slice.
@@ -1257,7 +1285,7 @@ __device__ __forceinline__ void pass1_rank1_flat(const TensorDesc& d, const void
 }
 
 template <bool BF16>
-__global__ void __launch_bounds__(kThreads, 3) pass1_kernel(StepArgs a) {
+__global__ void __launch_bounds__(kThreads, 2) pass1_kernel(StepArgs a) {
     __shared__ float s_col[kWarps * kWarpElems];
     const LaneTables lt = make_lane_tables();
     const Hyper2& h2 = a.h2;
