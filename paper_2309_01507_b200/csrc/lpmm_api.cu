@@ -188,6 +188,7 @@ struct lpmm_state {
     std::vector<size_t> stage_off;
     int32_t pass2_variant;                 // 0 = register prefetch, 1 = bulk-copy staging
     int32_t sms, occ1, occ2;
+    int32_t p1_ctas;                       // which instantiation of the maxima pass (2 or 3 CTAs per SM)
     std::vector<int32_t> tiles1, tiles2, tiles3;   // host copies of the tile prefix sums (3: element-indexed tiles of every tensor)
     cudaStream_t copy_in, copy_out;        // lazily created by the host-buffer entry point
     std::vector<cudaEvent_t> host_events;
@@ -203,7 +204,16 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
     int dev = 0, sms = 0, occ1 = 1, occ2 = 1;
     LPMM_CUDA(cudaGetDevice(&dev));
     LPMM_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    LPMM_CUDA(step_kernel_occupancy(&occ1, &occ2));
+    {   // the tiled maxima path wants two CTAs per SM, the other pass-1 paths three: go by the elements of each
+        int64_t tiled = 0, other = 0;
+        for (int32_t i = 0; i < st->n; ++i) {
+            const TensorLayout& t = st->L.t[i];
+            if (t.kind == K_RANK1_FAST) tiled += t.numel;
+            else if (t.kind == K_RANK1_FLAT || t.kind == K_FACT) other += t.numel;
+        }
+        st->p1_ctas = tiled >= other ? 2 : 3;
+    }
+    LPMM_CUDA(step_kernel_occupancy(st->p1_ctas, &occ1, &occ2));
     if (occ1 < 1) occ1 = 1;
     if (occ2 < 1) occ2 = 1;
     const int32_t n = st->n;
@@ -470,7 +480,7 @@ lpmm_status enqueue_range(lpmm_state* st, StepArgs a, int32_t t0, int32_t t1, bo
         a.tile_begin = p1_begin;
         a.tile_end = p1_end;
         const int32_t cap = st->sms * st->occ1, tiles = p1_end - p1_begin;
-        LPMM_CUDA(launch_pass1(a, bf16, tiles < cap ? tiles : cap, s));
+        LPMM_CUDA(launch_pass1(a, bf16, st->p1_ctas, tiles < cap ? tiles : cap, s));
         if (ev) LPMM_CUDA(cudaEventRecord(ev[1], s));
         LPMM_CUDA(launch_rcp(rc_new, reinterpret_cast<float*>(st->arena + st->L.rcp) + rc_begin, rc_end - rc_begin, s));
         *launches += 2;

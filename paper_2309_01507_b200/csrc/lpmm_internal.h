@@ -61,12 +61,12 @@ struct StepArgs {
     Hyper2 h2;                   // the same constants as pairs (kernel-parameter space: usable as operands)
 };
 
-cudaError_t launch_pass1(const StepArgs& a, bool bf16, int grid, cudaStream_t s);
+cudaError_t launch_pass1(const StepArgs& a, bool bf16, int ctas_per_sm, int grid, cudaStream_t s);
 cudaError_t launch_pass2(const StepArgs& a, bool bf16, bool exact, int m_shift, bool factored, int grid, cudaStream_t s);
 cudaError_t launch_factor_finalize(const StepArgs& a, int t0, int t1, cudaStream_t s);
 cudaError_t launch_sgdm(const StepArgs& a, bool bf16, int grid, cudaStream_t s);
 cudaError_t launch_rcp(const float* src, float* dst, int64_t n, cudaStream_t s);
-cudaError_t step_kernel_occupancy(int* pass1_blocks_per_sm, int* pass2_blocks_per_sm);
+cudaError_t step_kernel_occupancy(int pass1_ctas_per_sm, int* pass1_blocks_per_sm, int* pass2_blocks_per_sm);
 
 cudaError_t launch_quantize(const float* x, int64_t rows, int64_t cols, int norm, int map, int block,
                             bool given, uint8_t* codes, float* s0, float* s1, cudaStream_t s);

@@ -1284,8 +1284,11 @@ __device__ __forceinline__ void pass1_rank1_flat(const TensorDesc& d, const void
     }
 }
 
-template <bool BF16>
-__global__ void __launch_bounds__(kThreads, 2) pass1_kernel(StepArgs a) {
+// MINB: CTAs per SM the kernel is compiled for. The tiled maxima path keeps four rows of loads in registers and
+// runs best at two (128 registers); the element-indexed and the sum-of-squares paths hold little state and want
+// three. The host picks the instantiation by which kind holds most of a state's elements.
+template <bool BF16, int MINB>
+__global__ void __launch_bounds__(kThreads, MINB) pass1_kernel(StepArgs a) {
     __shared__ float s_col[kWarps * kWarpElems];
     const LaneTables lt = make_lane_tables();
     const Hyper2& h2 = a.h2;
@@ -1384,10 +1387,15 @@ __global__ void rcp_kernel(const float* __restrict__ src, float* __restrict__ ds
 
 }  // namespace
 
-cudaError_t launch_pass1(const StepArgs& a, bool bf16, int grid, cudaStream_t s) {
+cudaError_t launch_pass1(const StepArgs& a, bool bf16, int ctas_per_sm, int grid, cudaStream_t s) {
     if (a.tile_end <= a.tile_begin) return cudaSuccess;
-    if (bf16) pass1_kernel<true><<<grid, kThreads, 0, s>>>(a);
-    else pass1_kernel<false><<<grid, kThreads, 0, s>>>(a);
+    if (ctas_per_sm == 2) {
+        if (bf16) pass1_kernel<true, 2><<<grid, kThreads, 0, s>>>(a);
+        else pass1_kernel<false, 2><<<grid, kThreads, 0, s>>>(a);
+    } else {
+        if (bf16) pass1_kernel<true, 3><<<grid, kThreads, 0, s>>>(a);
+        else pass1_kernel<false, 3><<<grid, kThreads, 0, s>>>(a);
+    }
     return cudaGetLastError();
 }
 
@@ -1443,8 +1451,9 @@ cudaError_t launch_rcp(const float* src, float* dst, int64_t n, cudaStream_t s) 
     return cudaGetLastError();
 }
 
-cudaError_t step_kernel_occupancy(int* p1, int* p2) {
-    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(p1, pass1_kernel<true>, kThreads, 0);
+cudaError_t step_kernel_occupancy(int pass1_ctas_per_sm, int* p1, int* p2) {
+    cudaError_t e = pass1_ctas_per_sm == 2 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(p1, pass1_kernel<true, 2>, kThreads, 0)
+                                           : cudaOccupancyMaxActiveBlocksPerMultiprocessor(p1, pass1_kernel<true, 3>, kThreads, 0);
     if (e != cudaSuccess) return e;
     return cudaOccupancyMaxActiveBlocksPerMultiprocessor(p2, pass2_kernel<true, false, 7, false, false, true>, kThreads, 0);
 }
