@@ -35,9 +35,9 @@ PASS2_BYTES = {"bf16": 12.0625, "f32": 14.0625}
 PASS1_BYTES = {"bf16": 2.5, "f32": 4.5}
 # DRAM traffic of the update/re-quantize pass measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum)
 # per parameter, from the capture of the 464.5 M-parameter LLaMA slice summarised in
-# profiles/pass2_llama_7b_1l.txt (3.3049 GB read + 2.2844 GB written); traffic scales with the parameter count.
-# fp32 gradients: capture of the RoBERTa-large list (355.4 M params, 3.2834 GB read + 1.7464 GB written), same file.
-PASS2_TRAFFIC_BYTES_PER_PARAM = {"bf16": 12.032, "f32": 14.152}
+# profiles/pass2_llama_7b_1l.txt (3.2950 GB read + 2.2835 GB written); traffic scales with the parameter count.
+# fp32 gradients: capture of the RoBERTa-large list (355.4 M params, 3.2749 GB read + 1.7452 GB written), same file.
+PASS2_TRAFFIC_BYTES_PER_PARAM = {"bf16": 12.009, "f32": 14.125}
 
 
 def parse_args():
