@@ -229,6 +229,18 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
         const long x = std::atol(v);
         if (x >= 2048 && x <= (1 << 20)) tile_elems = x;
     }
+    // The maxima pass gets its own, taller tiles (same width): every tile ends with a flush of its column maxima and
+    // starts with an empty load pipeline, so it gains up to 1 Mi elements (3.92 -> 3.72 ms on the 6.7 G list) where
+    // the update pass is best at 256 Ki.
+    int64_t tile_elems1 = tile_elems;
+    {
+        const int64_t target1 = total_elems / (6LL * sms * occ1);
+        while (tile_elems1 * 2 <= target1 && tile_elems1 < (1 << 20)) tile_elems1 *= 2;
+        if (const char* v = std::getenv("LPMM_TILE_ELEMS1")) {   // development switch
+            const long x = std::atol(v);
+            if (x >= tile_elems && x <= (1 << 22)) tile_elems1 = x;
+        }
+    }
 
     std::vector<TensorDesc> descs(n);
     std::vector<int32_t> t1(n + 1, 0), t2(n + 1, 0), t3(n + 1, 0);
@@ -241,7 +253,7 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
         d.n_outer = t.n_outer;
         for (int a = 0; a < 3; ++a) { d.outer_dim[a] = t.outer_dim[a]; d.outer_off[a] = t.outer_off[a]; }
         d.m_shift = (st->cfg.m_block == 2048) ? 11 : 7;
-        int64_t tiles = 0;
+        int64_t tiles = 0, tiles_p1 = 0;
         if (t.kind == K_FP32) {
             d.m32 = reinterpret_cast<float*>(A + t.m32);
             d.v32 = reinterpret_cast<float*>(A + t.v32);
@@ -265,6 +277,10 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
             d.tile_rows = (int32_t)tr;
             d.tiles_x = (int32_t)((t.cols + tile_cols - 1) / tile_cols);
             tiles = (int64_t)d.tiles_x * ((t.rows + tr - 1) / tr);
+            int64_t tr1 = tile_elems1 / tile_cols;
+            if (tr1 < tr) tr1 = tr;
+            d.tile_rows1 = (int32_t)tr1;
+            tiles_p1 = (int64_t)d.tiles_x * ((t.rows + tr1 - 1) / tr1);
         }
         {   // element-indexed tiling: used by the non-tiled kinds in pass 2 and by every tensor in the SGDM step
             int64_t chunks = tile_elems / (kWarps * kWarpElems);
@@ -280,7 +296,8 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
         if (t2[i] + tiles > 0x7fffffffLL) return LPMM_ERR_UNSUPPORTED;
         t2[i + 1] = t2[i] + (int32_t)tiles;
         const bool rank1 = uses_rc(t.kind);
-        t1[i + 1] = t1[i] + (rank1 ? (int32_t)tiles : 0);
+        const bool tiled = (t.kind == K_RANK1_FAST || t.kind == K_FACT);
+        t1[i + 1] = t1[i] + (rank1 ? (int32_t)(tiled ? tiles_p1 : tiles) : 0);
     }
     st->total1 = t1[n];
     st->total2 = t2[n];

@@ -33,7 +33,7 @@ struct TensorDesc {
     int32_t c_off;      // float offset of c inside rc[] and rcp_new
     int32_t wx;         // K_RANK1_FAST: warps across a tile (1, 2 or 4); tile is 256*wx columns wide
     int32_t tiles_x;    // K_RANK1_FAST: column tiles
-    int32_t tile_rows;  // K_RANK1_FAST: rows per tile
+    int32_t tile_rows;  // K_RANK1_FAST: rows per tile of the update pass
     int32_t flat_chunks;  // other kinds: 256-element chunks per warp per tile
     int32_t m_shift;    // log2 of the first-moment block size: 7 (B128) or 11 (B2048)
     // K_RANK1_FLAT, general form of Alg. 4: the tensor is [outer_dim[0] x .. x outer_dim[n_outer-1]] x cols,
@@ -42,6 +42,7 @@ struct TensorDesc {
     int32_t n_outer;
     int32_t outer_dim[3];
     int32_t outer_off[3];
+    int32_t tile_rows1; // K_RANK1_FAST: rows per tile of the maxima pass (at least tile_rows; same tile width)
 };
 
 struct StepArgs {

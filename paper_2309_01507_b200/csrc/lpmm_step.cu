@@ -1097,8 +1097,8 @@ __device__ __forceinline__ void pass1_rank1_fast(const TensorDesc& d, const void
     if (col0 >= d.cols) col0 -= 128;
     const float* rc_old = (phase ? d.rc[1] : d.rc[0]);
     float* rc_new = (phase ? d.rc[0] : d.rc[1]);
-    const int64_t row0 = (int64_t)ty * d.tile_rows + warp / wx;
-    const int64_t row_end = min((int64_t)(ty + 1) * d.tile_rows, d.rows);
+    const int64_t row0 = (int64_t)ty * d.tile_rows1 + warp / wx;
+    const int64_t row_end = min((int64_t)(ty + 1) * d.tile_rows1, d.rows);
     if (row0 >= row_end) return;                      // uniform over the warp
     const uint32_t nrows = (uint32_t)((row_end - row0 + wy_count - 1) / wy_count);
 
@@ -1185,8 +1185,8 @@ __device__ __forceinline__ void pass1_fact(const TensorDesc& d, const void* __re
     const int64_t col0 = col_w + lane * kLaneElems;
     const bool active = col0 < d.cols;                  // cols % 256 == 128: the upper half-warp adds zeros
     float* sums = (phase ? d.rc[0] : d.rc[1]);          // [row sums | column sums], cleared before the launch
-    const int64_t row0 = (int64_t)ty * d.tile_rows + warp / wx;
-    const int64_t row_end = min((int64_t)(ty + 1) * d.tile_rows, d.rows);
+    const int64_t row0 = (int64_t)ty * d.tile_rows1 + warp / wx;
+    const int64_t row_end = min((int64_t)(ty + 1) * d.tile_rows1, d.rows);
     float c_sum[8];
 #pragma unroll
     for (int k = 0; k < 8; ++k) c_sum[k] = 0.0f;
