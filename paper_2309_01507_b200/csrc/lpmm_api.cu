@@ -52,7 +52,7 @@ bool uses_rc(int32_t k) { return k == K_RANK1_FAST || k == K_RANK1_FLAT || k == 
 
 int public_kind(int32_t k) {
     if (k == K_FP32) return LPMM_KIND_FP32;
-    if (k == K_BLOCK) return LPMM_KIND_BLOCK;
+    if (k == K_BLOCK || k == K_BLOCK_TILED) return LPMM_KIND_BLOCK;
     if (k == K_FACT) return LPMM_KIND_FACTORED;
     return LPMM_KIND_RANK1;
 }
@@ -103,7 +103,11 @@ int32_t choose_kind(const lpmm_config& cfg, const lpmm_shape& s) {
     const int64_t numel = s.rows * s.cols;
     if (s.flags & LPMM_FORCE_FP32) return K_FP32;
     if (!(s.flags & LPMM_FORCE_QUANT) && numel <= cfg.min_quant_numel) return K_FP32;  // App. C.1
-    if (s.ndim == 1 || s.rows == 1 || s.cols == 1 || cfg.v_mode == LPMM_V_BLOCK) return K_BLOCK;  // Sec. 4.2
+    if (s.ndim == 1 || s.rows == 1 || s.cols == 1) return K_BLOCK;  // Sec. 4.2
+    if (cfg.v_mode == LPMM_V_BLOCK) {   // block-wise second moment on a matrix: tiled when whole blocks lie inside a row
+        const bool tiled = s.ndim == 2 && s.cols % 128 == 0 && s.cols % cfg.m_block == 0 && s.cols <= ((int64_t)1 << 24);
+        return tiled ? K_BLOCK_TILED : K_BLOCK;
+    }
     // the tiled path needs whole first-moment blocks inside a row (and, for B2048, one block per tile width)
     // the tiled path keeps 32-bit element offsets inside a tile: rows of at most 2^24 elements
     if (s.ndim >= 3) return K_RANK1_FLAT;     // Alg. 4 with more than two axes: element-indexed path
@@ -163,7 +167,7 @@ void compute_layout(const lpmm_config& cfg, const lpmm_shape* shapes, int32_t n,
             t.m_codes = off; off = align_up(off + code_bytes);
             if (t.kind != K_FACT) { t.v_codes = off; off = align_up(off + code_bytes); }
             t.m_scale = off; off = align_up(off + sizeof(float) * nblk_m);
-            if (t.kind == K_BLOCK) { t.v_bscale = off; off = align_up(off + sizeof(float) * nblk); }
+            if (t.kind == K_BLOCK || t.kind == K_BLOCK_TILED) { t.v_bscale = off; off = align_up(off + sizeof(float) * nblk); }
         }
     }
     L->total = off;
@@ -261,14 +265,14 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
             d.m_codes = reinterpret_cast<uint8_t*>(A + t.m_codes);
             d.v_codes = (t.kind == K_FACT) ? nullptr : reinterpret_cast<uint8_t*>(A + t.v_codes);
             d.m_scale = reinterpret_cast<float*>(A + t.m_scale);
-            if (t.kind == K_BLOCK) d.v_bscale = reinterpret_cast<float*>(A + t.v_bscale);
+            if (t.kind == K_BLOCK || t.kind == K_BLOCK_TILED) d.v_bscale = reinterpret_cast<float*>(A + t.v_bscale);
             if (uses_rc(t.kind)) {
                 d.rc[0] = reinterpret_cast<float*>(A + st->L.rc[0]) + t.rc_index;
                 d.rc[1] = reinterpret_cast<float*>(A + st->L.rc[1]) + t.rc_index;
                 d.rcp_new = reinterpret_cast<float*>(A + st->L.rcp) + t.rc_index;
             }
         }
-        if (t.kind == K_RANK1_FAST || t.kind == K_FACT) {
+        if (t.kind == K_RANK1_FAST || t.kind == K_FACT || t.kind == K_BLOCK_TILED) {
             d.wx = (st->cfg.m_block == 2048) ? 8 : (t.cols % 1024 == 0) ? 4 : (t.cols % 512 == 0) ? 2 : 1;
             const int64_t tile_cols = (int64_t)kWarpElems * d.wx;
             int64_t tr = tile_elems / tile_cols;
@@ -289,7 +293,7 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
             d.flat_chunks = (int32_t)chunks;
             const int64_t per_tile = chunks * kWarps * kWarpElems;
             const int64_t flat_tiles = (t.numel + per_tile - 1) / per_tile;
-            if (t.kind != K_RANK1_FAST && t.kind != K_FACT) tiles = flat_tiles;
+            if (t.kind != K_RANK1_FAST && t.kind != K_FACT && t.kind != K_BLOCK_TILED) tiles = flat_tiles;
             if (t3[i] + flat_tiles > 0x7fffffffLL) return LPMM_ERR_UNSUPPORTED;
             t3[i + 1] = t3[i] + (int32_t)flat_tiles;
         }
@@ -514,7 +518,8 @@ lpmm_status enqueue_range(lpmm_state* st, StepArgs a, int32_t t0, int32_t t1, bo
     a.tile_begin = st->tiles2[t0];
     a.tile_end = st->tiles2[t1];
     const int32_t cap = st->sms * st->occ2, tiles = a.tile_end - a.tile_begin;
-    LPMM_CUDA(launch_pass2(a, bf16, ieee_update, st->cfg.m_block == 2048 ? 11 : 7, st->cfg.v_mode == LPMM_V_FACTORED,
+    LPMM_CUDA(launch_pass2(a, bf16, ieee_update, st->cfg.m_block == 2048 ? 11 : 7,
+                           st->cfg.v_mode == LPMM_V_FACTORED ? 1 : (st->cfg.v_mode == LPMM_V_BLOCK ? 2 : 0),
                            tiles < cap ? tiles : cap, s));
     if (ev) LPMM_CUDA(cudaEventRecord(ev[3], s));
     *launches += 1;
@@ -544,7 +549,7 @@ lpmm_status adamw4_step_impl(lpmm_state* st, void* const* d_params, void* const*
                              float weight_decay, int64_t step, void* stream) {
     lpmm_status rc = check_step_args(st, d_params, d_grads, grad_dtype, lr, beta1, beta2, eps, weight_decay, step);
     if (rc != LPMM_OK) return rc;
-    if (d_params16 && st->cfg.v_mode == LPMM_V_FACTORED) return LPMM_ERR_UNSUPPORTED;
+    if (d_params16 && st->cfg.v_mode != LPMM_V_RANK1) return LPMM_ERR_UNSUPPORTED;   // the copy rides on the default kernels
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     rc = set_pointers(st, d_params, d_grads, s);
     if (rc != LPMM_OK) return rc;
@@ -748,7 +753,7 @@ lpmm_status lpmm_state_view(const lpmm_state* st, int32_t tensor, int32_t* kind,
     if (m_scale) *m_scale = q ? reinterpret_cast<const float*>(A + t.m_scale) : nullptr;
     if (v_codes) *v_codes = (q && t.kind != K_FACT) ? reinterpret_cast<const uint8_t*>(A + t.v_codes) : nullptr;
     const float* rc = reinterpret_cast<const float*>(A + st->L.rc[st->phase]) + t.rc_index;
-    if (v_scale0) *v_scale0 = r1 ? rc : (t.kind == K_BLOCK ? reinterpret_cast<const float*>(A + t.v_bscale) : nullptr);
+    if (v_scale0) *v_scale0 = r1 ? rc : ((t.kind == K_BLOCK || t.kind == K_BLOCK_TILED) ? reinterpret_cast<const float*>(A + t.v_bscale) : nullptr);
     if (v_scale1) *v_scale1 = r1 ? rc + t.c_off : nullptr;
     if (m32) *m32 = q ? nullptr : reinterpret_cast<const float*>(A + t.m32);
     if (v32) *v32 = q ? nullptr : reinterpret_cast<const float*>(A + t.v32);

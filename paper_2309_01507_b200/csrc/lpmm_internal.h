@@ -10,8 +10,9 @@ namespace lpmm {
 
 // Work kinds inside the step kernels. RANK1_FAST needs cols % 128 == 0 (a 128-block then lies inside
 // one row and every row starts on a 16-byte boundary of every operand); other 2-D shapes take the
-// element-indexed RANK1_FLAT path.
-enum : int32_t { K_FP32 = 0, K_BLOCK = 1, K_RANK1_FAST = 2, K_RANK1_FLAT = 3, K_FACT = 4 };
+// element-indexed RANK1_FLAT path. BLOCK_TILED: a matrix with a block-wise second moment (LPMM_V_BLOCK) and
+// cols % 128 == 0 on the tiled path; BLOCK: every other block-wise tensor, element-indexed.
+enum : int32_t { K_FP32 = 0, K_BLOCK = 1, K_RANK1_FAST = 2, K_RANK1_FLAT = 3, K_FACT = 4, K_BLOCK_TILED = 5 };
 
 constexpr int kThreads = 256;          // threads per CTA in the step kernels
 constexpr int kWarps = kThreads / 32;
@@ -63,7 +64,7 @@ struct StepArgs {
 };
 
 cudaError_t launch_pass1(const StepArgs& a, bool bf16, int ctas_per_sm, int grid, cudaStream_t s);
-cudaError_t launch_pass2(const StepArgs& a, bool bf16, bool exact, int m_shift, bool factored, int grid, cudaStream_t s);
+cudaError_t launch_pass2(const StepArgs& a, bool bf16, bool exact, int m_shift, int v_kind, int grid, cudaStream_t s);
 cudaError_t launch_factor_finalize(const StepArgs& a, int t0, int t1, cudaStream_t s);
 cudaError_t launch_sgdm(const StepArgs& a, bool bf16, int grid, cudaStream_t s);
 cudaError_t launch_rcp(const float* src, float* dst, int64_t n, cudaStream_t s);

@@ -326,6 +326,7 @@ struct TileView {
     uint8_t* m_codes;
     uint8_t* v_codes;
     float* m_scale;
+    float* v_bscale;       // VM == 2: block maxima of the second moment (same indexing as m_scale with B128)
     const float* r_old;
     const float* r_rcp;
     uint32_t row_step;     // elements between two rows this warp handles
@@ -345,16 +346,17 @@ __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefe
 // One instruction per row for the whole warp: the 256 elements a warp owns in a row are 8 lines of parameters,
 // 4 (bf16) or 8 (fp32) lines of gradient, one line of each code array and one of block scales, and each of the
 // first lanes asks for one of those lines.
-template <bool BF16, int MSHIFT, bool FACT>
+template <bool BF16, int MSHIFT, int VM>
 __device__ __forceinline__ void prefetch_row(const TileView& t, uint32_t k) {
     if (t.pf_step != 0) prefetch_l2(t.pf_base + (size_t)k * t.pf_step);
 }
 // Assigns the lane its line (warp_* point at the warp's first element of row 0; row_step in elements).
 // `valid` = how many of the warp's 256 columns exist (128 in a tensor's last warp column when cols % 256 == 128):
 // no lane asks for a line past the end of the row.
-template <bool BF16, int MSHIFT, bool FACT>
+template <bool BF16, int MSHIFT, int VM>
 __device__ __forceinline__ void prefetch_roles(TileView& t, int lane, int valid, const float* warp_w, const void* warp_g,
-                                               const uint8_t* warp_mq, const uint8_t* warp_vq, const float* warp_ms) {
+                                               const uint8_t* warp_mq, const uint8_t* warp_vq, const float* warp_ms,
+                                               const float* warp_vs) {
     constexpr int kGLines = BF16 ? 4 : 8;
     constexpr int kGLineElems = BF16 ? 64 : 32;
     t.pf_base = nullptr;
@@ -372,17 +374,20 @@ __device__ __forceinline__ void prefetch_roles(TileView& t, int lane, int valid,
     } else if (lane == 8 + kGLines) {
         t.pf_base = reinterpret_cast<const char*>(warp_mq);
         t.pf_step = t.row_step / 2u;
-    } else if (lane == 9 + kGLines && !FACT) {
+    } else if (lane == 9 + kGLines && VM != 1) {
         t.pf_base = reinterpret_cast<const char*>(warp_vq);
         t.pf_step = t.row_step / 2u;
     } else if (lane == 10 + kGLines) {
         t.pf_base = reinterpret_cast<const char*>(warp_ms);
         t.pf_step = (t.row_step >> MSHIFT) * 4u;
+    } else if (lane == 11 + kGLines && VM == 2) {
+        t.pf_base = reinterpret_cast<const char*>(warp_vs);
+        t.pf_step = (t.row_step >> 7) * 4u;
     }
 }
 
 // A32: the parameter rows (and fp32 gradient rows) of this tensor are 32-byte aligned.
-template <bool BF16, int MSHIFT, bool FACT, bool A32>
+template <bool BF16, int MSHIFT, int VM, bool A32>
 __device__ __forceinline__ void load_row(RowRegs<BF16>& r, const TileView& t, uint32_t k) {
     const uint32_t off = k * t.row_step;
     if (A32) {
@@ -401,8 +406,14 @@ __device__ __forceinline__ void load_row(RowRegs<BF16>& r, const TileView& t, ui
     }
     r.qm = *reinterpret_cast<const uint32_t*>(t.m_codes + (off >> 1));
     r.am = t.m_scale[off >> MSHIFT];
-    r.r_rcp = __ldg(t.r_rcp + k * t.row_stride);        // FACT: the row factor R_i / sum(R)
-    if (FACT) {
+    if (VM == 2) {                                        // block-wise second moment: r_old carries the block's scale
+        r.qv = *reinterpret_cast<const uint32_t*>(t.v_codes + (off >> 1));
+        r.r_old = t.v_bscale[off >> 7];
+        r.r_rcp = 0.0f;
+        return;
+    }
+    r.r_rcp = __ldg(t.r_rcp + k * t.row_stride);        // VM == 1: the row factor R_i / sum(R)
+    if (VM == 1) {
         r.qv = 0;
         r.r_old = 0.0f;
     } else {
@@ -411,7 +422,7 @@ __device__ __forceinline__ void load_row(RowRegs<BF16>& r, const TileView& t, ui
     }
 }
 
-template <bool BF16, bool EXACT, int MSHIFT, bool FACT, bool WB, bool A32>
+template <bool BF16, bool EXACT, int MSHIFT, int VM, bool WB, bool A32>
 __device__ __forceinline__ void process_row(const RowRegs<BF16>& r, const TileView& t, uint32_t k,
                                             const float (&c_old)[8], const float (&c_rcp)[8], const Hyper& h,
                                             const Hyper2& h2, const LaneTables& lt, const unsigned char* s_lut) {
@@ -421,24 +432,35 @@ __device__ __forceinline__ void process_row(const RowRegs<BF16>& r, const TileVi
     unpack_grad8<BF16>(r.g0, r.g1, gv);
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-        if (FACT) {
+        if (VM == 1) {
             vs[j] = __fmul_rn(r.r_rcp, c_rcp[j]);  // Sec. 4.3: v_ij = (R_i / sum R) * C_j
+            vr[j] = 0.0f;
+        } else if (VM == 2) {
+            vs[j] = r.r_old;                       // Sec. 2.2: the block's maximum
             vr[j] = 0.0f;
         } else {
             vs[j] = fminf(r.r_old, c_old[j]);      // Sec. 4.2: scale = min(r_i, c_j)
             vr[j] = fmaxf(r.r_rcp, c_rcp[j]);      // 1/min(r', c') = max(1/r', 1/c')
         }
     }
-    moments_and_update8<EXACT, FACT>(wv, gv, r.qm, r.qv, __fmul_rn(lt.de, r.am), vs, h, h2, lt, mt, vt);
+    moments_and_update8<EXACT, VM == 1>(wv, gv, r.qm, r.qv, __fmul_rn(lt.de, r.am), vs, h, h2, lt, mt, vt);
     if (A32) store8_f32_256(t.w + off, wv); else store8_f32(t.w + off, wv);
     if (WB) store8_bf16(t.w16 + off, wv);
     const float am_new = block_max(absmax8(mt), MSHIFT, lt, t.s_red, *t.red_step);
     if ((threadIdx.x & (MSHIFT == 7 ? 15 : 2047)) == 0) t.m_scale[off >> MSHIFT] = am_new;
     *reinterpret_cast<uint32_t*>(t.m_codes + (off >> 1)) = quantize8_de(mt, scale_rcp(am_new), s_lut);
-    if (!FACT) *reinterpret_cast<uint32_t*>(t.v_codes + (off >> 1)) = quantize8_lin(vt, vr, h2);
+    if (VM == 2) {       // new block maximum of v_t (non-negative), its reciprocal for all eight elements
+        const float av_new = group_max(absmax8(vt), lt.mask);
+        if ((threadIdx.x & 15) == 0) t.v_bscale[off >> 7] = av_new;
+        const float rv = scale_rcp(av_new);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) vr[j] = rv;
+    }
+    if (VM != 1) *reinterpret_cast<uint32_t*>(t.v_codes + (off >> 1)) = quantize8_lin(vt, vr, h2);
 }
 
-template <bool BF16, bool EXACT, int MSHIFT, bool FACT = false, bool WB = false, bool A32 = false>
+// VM: how the second moment is kept: 0 rank-1 codes (Sec. 4.2), 1 factorized statistics (Sec. 4.3), 2 block-wise codes.
+template <bool BF16, bool EXACT, int MSHIFT, int VM = 0, bool WB = false, bool A32 = false>
 __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __restrict__ w, uint16_t* __restrict__ w16,
                                                  const void* __restrict__ g,
                                                  int tile, int phase, const Hyper& h, const Hyper2& h2,
@@ -459,7 +481,10 @@ __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __r
     const uint32_t nrows = (uint32_t)((row_end - row0 + wy_count - 1) / wy_count);
 
     float c_old[8], c_rcp[8];
-    if (FACT) {      // the new column statistics C_j sit in the "new" buffer; nothing old is needed
+    if (VM == 2) {   // no row / column statistics at all
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { c_old[j] = 0.0f; c_rcp[j] = 0.0f; }
+    } else if (VM == 1) {      // the new column statistics C_j sit in the "new" buffer; nothing old is needed
         load8_f32((phase ? d.rc[0] : d.rc[1]) + d.c_off + col0, c_rcp);
 #pragma unroll
         for (int j = 0; j < 8; ++j) c_old[j] = 0.0f;
@@ -474,7 +499,8 @@ __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __r
     t.g = BF16 ? static_cast<const void*>(reinterpret_cast<const uint16_t*>(g) + e0)
                : static_cast<const void*>(reinterpret_cast<const float*>(g) + e0);
     t.m_codes = d.m_codes + (e0 >> 1);
-    t.v_codes = FACT ? nullptr : d.v_codes + (e0 >> 1);
+    t.v_codes = VM == 1 ? nullptr : d.v_codes + (e0 >> 1);
+    t.v_bscale = VM == 2 ? d.v_bscale + (e0 >> 7) : nullptr;
     t.m_scale = d.m_scale + (e0 >> MSHIFT);
     t.r_old = rc_old + row0;
     t.r_rcp = rcp_new + row0;
@@ -486,36 +512,37 @@ __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __r
     {
         const int64_t ew = e0 - lane * kLaneElems;       // the warp's first element of its first row
         const int64_t left = d.cols - (col0 - lane * kLaneElems);
-        prefetch_roles<BF16, MSHIFT, FACT>(t, lane, left < kWarpElems ? (int)left : kWarpElems, w + ew,
+        prefetch_roles<BF16, MSHIFT, VM>(t, lane, left < kWarpElems ? (int)left : kWarpElems, w + ew,
                                            BF16 ? static_cast<const void*>(reinterpret_cast<const uint16_t*>(g) + ew)
                                                 : static_cast<const void*>(reinterpret_cast<const float*>(g) + ew),
-                                           d.m_codes + (ew >> 1), FACT ? nullptr : d.v_codes + (ew >> 1), d.m_scale + (ew >> MSHIFT));
+                                           d.m_codes + (ew >> 1), VM == 1 ? nullptr : d.v_codes + (ew >> 1), d.m_scale + (ew >> MSHIFT),
+                                           VM == 2 ? d.v_bscale + (ew >> 7) : nullptr);
     }
 
     // Two register sets alternate: while one row is processed the next one is already in flight.
     RowRegs<BF16> ra, rb;
 #pragma unroll
-    for (uint32_t k = 1; k < kL2Ahead; ++k) if (k < nrows) prefetch_row<BF16, MSHIFT, FACT>(t, k);
-    load_row<BF16, MSHIFT, FACT, A32>(ra, t, 0);
+    for (uint32_t k = 1; k < kL2Ahead; ++k) if (k < nrows) prefetch_row<BF16, MSHIFT, VM>(t, k);
+    load_row<BF16, MSHIFT, VM, A32>(ra, t, 0);
     uint32_t k = 0;
     // (B2048 rows end in a CTA-wide barrier, where the longer straight-line body only costs registers: guarded loop only)
     for (; MSHIFT == 7 && k + 1 + kL2Ahead < nrows; k += 2) {        // every row touched below exists: no guards
-        prefetch_row<BF16, MSHIFT, FACT>(t, k + kL2Ahead);
-        load_row<BF16, MSHIFT, FACT, A32>(rb, t, k + 1);
-        process_row<BF16, EXACT, MSHIFT, FACT, WB, A32>(ra, t, k, c_old, c_rcp, h, h2, lt, s_lut);
-        prefetch_row<BF16, MSHIFT, FACT>(t, k + 1 + kL2Ahead);
-        load_row<BF16, MSHIFT, FACT, A32>(ra, t, k + 2);
-        process_row<BF16, EXACT, MSHIFT, FACT, WB, A32>(rb, t, k + 1, c_old, c_rcp, h, h2, lt, s_lut);
+        prefetch_row<BF16, MSHIFT, VM>(t, k + kL2Ahead);
+        load_row<BF16, MSHIFT, VM, A32>(rb, t, k + 1);
+        process_row<BF16, EXACT, MSHIFT, VM, WB, A32>(ra, t, k, c_old, c_rcp, h, h2, lt, s_lut);
+        prefetch_row<BF16, MSHIFT, VM>(t, k + 1 + kL2Ahead);
+        load_row<BF16, MSHIFT, VM, A32>(ra, t, k + 2);
+        process_row<BF16, EXACT, MSHIFT, VM, WB, A32>(rb, t, k + 1, c_old, c_rcp, h, h2, lt, s_lut);
     }
     for (; k < nrows; k += 2) {                       // the last rows of the tile
         const bool has_b = k + 1 < nrows;
-        if (k + kL2Ahead < nrows) prefetch_row<BF16, MSHIFT, FACT>(t, k + kL2Ahead);
-        if (has_b) load_row<BF16, MSHIFT, FACT, A32>(rb, t, k + 1);
-        process_row<BF16, EXACT, MSHIFT, FACT, WB, A32>(ra, t, k, c_old, c_rcp, h, h2, lt, s_lut);
+        if (k + kL2Ahead < nrows) prefetch_row<BF16, MSHIFT, VM>(t, k + kL2Ahead);
+        if (has_b) load_row<BF16, MSHIFT, VM, A32>(rb, t, k + 1);
+        process_row<BF16, EXACT, MSHIFT, VM, WB, A32>(ra, t, k, c_old, c_rcp, h, h2, lt, s_lut);
         if (!has_b) break;
-        if (k + 1 + kL2Ahead < nrows) prefetch_row<BF16, MSHIFT, FACT>(t, k + 1 + kL2Ahead);
-        if (k + 2 < nrows) load_row<BF16, MSHIFT, FACT, A32>(ra, t, k + 2);
-        process_row<BF16, EXACT, MSHIFT, FACT, WB, A32>(rb, t, k + 1, c_old, c_rcp, h, h2, lt, s_lut);
+        if (k + 1 + kL2Ahead < nrows) prefetch_row<BF16, MSHIFT, VM>(t, k + 1 + kL2Ahead);
+        if (k + 2 < nrows) load_row<BF16, MSHIFT, VM, A32>(ra, t, k + 2);
+        process_row<BF16, EXACT, MSHIFT, VM, WB, A32>(rb, t, k + 1, c_old, c_rcp, h, h2, lt, s_lut);
     }
 }
 
@@ -870,12 +897,12 @@ __device__ __forceinline__ void pass2_fp32(const TensorDesc& d, float* __restric
     }
 }
 
-// VF: the state uses the factorized second moment (then no tensor is of the rank-1 tiled kind, and vice versa),
-// so each instantiation carries only one of the two tiled paths.
+// VF: how the state keeps the second moment of its tiled tensors: 0 rank-1 codes, 1 factorized, 2 block-wise codes.
+// A state has tiled tensors of one of these kinds only, so each instantiation carries only one tiled path.
 // WB: a bfloat16 copy of every updated parameter is written as well (a.params_bf16).
 // A32: every parameter pointer (and, with fp32 gradients, every gradient pointer) of the step is 32-byte aligned,
 // checked on the host: the tiled path then moves a lane's 8 values with one 256-bit access.
-template <bool BF16, bool EXACT, int MSHIFT, bool VF, bool WB, bool A32>
+template <bool BF16, bool EXACT, int MSHIFT, int VF, bool WB, bool A32>
 __global__ void __launch_bounds__(kThreads, 2) pass2_kernel(StepArgs a) {
     __shared__ __align__(16) unsigned char s_lut[kLutSmemBytes];
     __shared__ float s_red[2 * kWarps];
@@ -896,10 +923,13 @@ __global__ void __launch_bounds__(kThreads, 2) pass2_kernel(StepArgs a) {
         const int local = tile - __ldg(a.tile_start + t);
         switch (d.kind) {
             case K_RANK1_FAST:
-                if (!VF) pass2_rank1_fast<BF16, EXACT, MSHIFT, false, WB, A32>(d, w, w16, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step);
+                if (VF == 0) pass2_rank1_fast<BF16, EXACT, MSHIFT, 0, WB, A32>(d, w, w16, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step);
                 break;
             case K_FACT:
-                if (VF) pass2_rank1_fast<BF16, EXACT, MSHIFT, true, WB>(d, w, w16, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step);
+                if (VF == 1) pass2_rank1_fast<BF16, EXACT, MSHIFT, 1, WB>(d, w, w16, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step);
+                break;
+            case K_BLOCK_TILED:
+                if (VF == 2) pass2_rank1_fast<BF16, EXACT, MSHIFT, 2, WB, A32>(d, w, w16, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step);
                 break;
             case K_RANK1_FLAT: pass2_flat<BF16, true, EXACT, MSHIFT, WB, A32>(d, w, w16, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
             case K_BLOCK:      pass2_flat<BF16, false, EXACT, MSHIFT, WB, A32>(d, w, w16, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
@@ -1400,34 +1430,38 @@ cudaError_t launch_pass1(const StepArgs& a, bool bf16, int ctas_per_sm, int grid
 }
 
 template <bool BF16, bool EXACT, int MSHIFT>
-cudaError_t launch_pass2_t(const StepArgs& a, bool factored, int grid, cudaStream_t s) {
-    if (factored) {
-        pass2_kernel<BF16, EXACT, MSHIFT, true, false, false><<<grid, kThreads, 0, s>>>(a);
+cudaError_t launch_pass2_t(const StepArgs& a, int v_kind, int grid, cudaStream_t s) {
+    if (v_kind == 1) {
+        pass2_kernel<BF16, EXACT, MSHIFT, 1, false, false><<<grid, kThreads, 0, s>>>(a);
+    } else if (v_kind == 2) {
+        if (a.aligned32) pass2_kernel<BF16, EXACT, MSHIFT, 2, false, true><<<grid, kThreads, 0, s>>>(a);
+        else pass2_kernel<BF16, EXACT, MSHIFT, 2, false, false><<<grid, kThreads, 0, s>>>(a);
     } else if (a.params_bf16 != nullptr) {
-        if (a.aligned32) pass2_kernel<BF16, EXACT, MSHIFT, false, true, true><<<grid, kThreads, 0, s>>>(a);
-        else pass2_kernel<BF16, EXACT, MSHIFT, false, true, false><<<grid, kThreads, 0, s>>>(a);
+        if (a.aligned32) pass2_kernel<BF16, EXACT, MSHIFT, 0, true, true><<<grid, kThreads, 0, s>>>(a);
+        else pass2_kernel<BF16, EXACT, MSHIFT, 0, true, false><<<grid, kThreads, 0, s>>>(a);
     } else if (a.variant == 1) {
         constexpr int smem = bulk_smem_bytes<BF16>();
         cudaError_t e = cudaFuncSetAttribute(pass2_bulk_kernel<BF16, EXACT, MSHIFT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
         pass2_bulk_kernel<BF16, EXACT, MSHIFT><<<grid, kThreads, smem, s>>>(a);
     } else if (a.aligned32) {
-        pass2_kernel<BF16, EXACT, MSHIFT, false, false, true><<<grid, kThreads, 0, s>>>(a);
+        pass2_kernel<BF16, EXACT, MSHIFT, 0, false, true><<<grid, kThreads, 0, s>>>(a);
     } else {
-        pass2_kernel<BF16, EXACT, MSHIFT, false, false, false><<<grid, kThreads, 0, s>>>(a);
+        pass2_kernel<BF16, EXACT, MSHIFT, 0, false, false><<<grid, kThreads, 0, s>>>(a);
     }
     return cudaGetLastError();
 }
 
 template <bool BF16, bool EXACT>
-cudaError_t launch_pass2_m(const StepArgs& a, int m_shift, bool factored, int grid, cudaStream_t s) {
-    return m_shift == 11 ? launch_pass2_t<BF16, EXACT, 11>(a, factored, grid, s) : launch_pass2_t<BF16, EXACT, 7>(a, factored, grid, s);
+cudaError_t launch_pass2_m(const StepArgs& a, int m_shift, int v_kind, int grid, cudaStream_t s) {
+    return m_shift == 11 ? launch_pass2_t<BF16, EXACT, 11>(a, v_kind, grid, s) : launch_pass2_t<BF16, EXACT, 7>(a, v_kind, grid, s);
 }
 
-cudaError_t launch_pass2(const StepArgs& a, bool bf16, bool exact, int m_shift, bool factored, int grid, cudaStream_t s) {
+// v_kind: 0 rank-1 second moments, 1 factorized, 2 block-wise (which tiled path the state's matrices take).
+cudaError_t launch_pass2(const StepArgs& a, bool bf16, bool exact, int m_shift, int v_kind, int grid, cudaStream_t s) {
     if (a.tile_end <= a.tile_begin) return cudaSuccess;
-    if (bf16) return exact ? launch_pass2_m<true, true>(a, m_shift, factored, grid, s) : launch_pass2_m<true, false>(a, m_shift, factored, grid, s);
-    return exact ? launch_pass2_m<false, true>(a, m_shift, factored, grid, s) : launch_pass2_m<false, false>(a, m_shift, factored, grid, s);
+    if (bf16) return exact ? launch_pass2_m<true, true>(a, m_shift, v_kind, grid, s) : launch_pass2_m<true, false>(a, m_shift, v_kind, grid, s);
+    return exact ? launch_pass2_m<false, true>(a, m_shift, v_kind, grid, s) : launch_pass2_m<false, false>(a, m_shift, v_kind, grid, s);
 }
 
 cudaError_t launch_factor_finalize(const StepArgs& a, int t0, int t1, cudaStream_t s) {
@@ -1455,7 +1489,7 @@ cudaError_t step_kernel_occupancy(int pass1_ctas_per_sm, int* p1, int* p2) {
     cudaError_t e = pass1_ctas_per_sm == 2 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(p1, pass1_kernel<true, 2>, kThreads, 0)
                                            : cudaOccupancyMaxActiveBlocksPerMultiprocessor(p1, pass1_kernel<true, 3>, kThreads, 0);
     if (e != cudaSuccess) return e;
-    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(p2, pass2_kernel<true, false, 7, false, false, true>, kThreads, 0);
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(p2, pass2_kernel<true, false, 7, 0, false, true>, kThreads, 0);
 }
 
 }  // namespace lpmm
