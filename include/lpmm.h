@@ -3,8 +3,8 @@
  *
  * Implements the hot path of "Memory Efficient Optimizers with 4-bit States" (arXiv 2309.01507):
  * Alg. 3 (compressed Adam) with Eq. 1, decoupled weight decay, the first moment kept as
- * B128/DE (Sec. 3, App. D.2) and the second moment as Rank-1/Linear (Sec. 4.1, 4.2), B128/Linear
- * for one-dimensional tensors (Sec. 4.2) and fp32 states for tensors of <= 4096 elements (App. C.1).
+ * B128/DE (Sec. 3, App. E.2) and the second moment as Rank-1/Linear (Sec. 4.1, 4.2), B128/Linear
+ * for one-dimensional tensors (Sec. 4.2) and fp32 states for tensors of <= 4096 elements (App. D.1).
  *
  * Conventions
  *  - Pointers named d_* are DEVICE pointers, h_* are HOST pointers; everything else is host memory.
@@ -45,7 +45,7 @@ typedef int32_t lpmm_status;
 
 typedef enum { LPMM_F32 = 0, LPMM_BF16 = 1 } lpmm_dtype;
 typedef enum { LPMM_NORM_BLOCK = 0, LPMM_NORM_RANK1 = 1 } lpmm_norm;          /* Sec. 2.2 / Sec. 4.2 */
-typedef enum { LPMM_MAP_DE_SIGNED = 0, LPMM_MAP_LINEAR_NOZERO = 1 } lpmm_map; /* App. D.2 / Sec. 4.1 */
+typedef enum { LPMM_MAP_DE_SIGNED = 0, LPMM_MAP_LINEAR_NOZERO = 1 } lpmm_map; /* App. E.2 / Sec. 4.1 */
 /* Second moment of 2-D tensors: 4-bit with rank-1 or block-wise normalization, or not stored at all but
  * reconstructed from fp32 row / column statistics ("4-bit Factor", Sec. 4.3; 1-D tensors stay quantized). */
 typedef enum { LPMM_V_RANK1 = 0, LPMM_V_BLOCK = 1, LPMM_V_FACTORED = 2 } lpmm_vmode;
@@ -80,14 +80,14 @@ typedef struct {
     int32_t m_block;         /* first-moment block size B: 128 (Sec. 3) or 2048 (the 8-bit optimizer's size, Sec. 2.2) */
     int32_t v_block;         /* second-moment block size for 1-D tensors and LPMM_V_BLOCK (Sec. 4.2: 128) */
     int32_t v_mode;          /* lpmm_vmode */
-    int64_t min_quant_numel; /* tensors with numel <= this keep fp32 states (App. C.1: 4096) */
+    int64_t min_quant_numel; /* tensors with numel <= this keep fp32 states (App. D.1: 4096) */
     int32_t update_math;     /* lpmm_update_math: arithmetic of the parameter update only */
     int32_t reserved;        /* 0 */
 } lpmm_config;
 
 typedef struct lpmm_state lpmm_state; /* opaque host handle */
 
-/* State kind chosen per tensor (App. C.1 size rule; Sec. 4.2: a tensor that is 1-D, or has an
+/* State kind chosen per tensor (App. D.1 size rule; Sec. 4.2: a tensor that is 1-D, or has an
  * extent of 1, uses block-wise normalization for v). */
 #define LPMM_KIND_FP32 0
 #define LPMM_KIND_BLOCK 1

@@ -19,7 +19,7 @@
 /* ------------------------------------------------------------------ quantization mappings */
 
 int lpmm_oracle_linear_map(int bits, float* T) {
-    /* App. D.2: the 2^b + 1 evenly spaced points of [0, 1] with the first (zero) dropped. */
+    /* App. E.2: the 2^b + 1 evenly spaced points of [0, 1] with the first (zero) dropped. */
     int n = 1 << bits;
     for (int i = 0; i < n; ++i) T[i] = (float)((double)(i + 1) / (double)n);
     return n;
@@ -234,7 +234,7 @@ void lpmm_oracle_bf16_to_f32(const uint16_t* in, int64_t numel, float* out) {
 int lpmm_oracle_kind(int64_t rows, int64_t cols, int ndim, int64_t min_quant_numel, int force) {
     int64_t numel = rows * cols;
     if (force == 2) return LPMM_ORACLE_FP32;
-    if (force != 1 && numel <= min_quant_numel) return LPMM_ORACLE_FP32; /* App. C.1: size <= 4096 */
+    if (force != 1 && numel <= min_quant_numel) return LPMM_ORACLE_FP32; /* App. D.1: size <= 4096 */
     if (ndim <= 1 || rows == 1 || cols == 1) return LPMM_ORACLE_BLOCK;   /* Sec. 4.2: 1-D uses B128 */
     return LPMM_ORACLE_RANK1;
 }

@@ -24,10 +24,10 @@
 extern "C" {
 #endif
 
-/* Sec. 2.2 "Mapping" and App. D.2 "Linear mapping": T(i) = (i+1)/2^b, i = 0 .. 2^b-1. Returns 2^b. */
+/* Sec. 2.2 "Mapping" and App. E.2 "Linear mapping": T(i) = (i+1)/2^b, i = 0 .. 2^b-1. Returns 2^b. */
 int lpmm_oracle_linear_map(int bits, float* T);
 
-/* App. D.2 "Dynamic exponent mapping". Builds the table from the bit patterns:
+/* App. E.2 "Dynamic exponent mapping". Builds the table from the bit patterns:
  * unsigned  b = E + 1 + F : E leading zeros, indicator bit, F fraction bits,
  *           value 10^-E * fraction_F[k]; corner cases 0...0 -> 0 and 0...01 -> 1;
  * signed    b = 1 + E + 1 + F : first bit is the sign; corner cases 00..0 -> 0, 10..0 -> +1
@@ -36,7 +36,7 @@ int lpmm_oracle_linear_map(int bits, float* T);
  * increasingly; T(i) is its i-th entry. Returns the number of entries. */
 int lpmm_oracle_de_map(int bits, int is_signed, int drop_zero, float* T);
 
-/* App. D.2: fraction_F[k] = (p_k + p_{k+1})/2 with p_j = 0.9 j / 2^F + 0.1, as a double. */
+/* App. E.2: fraction_F[k] = (p_k + p_{k+1})/2 with p_j = 0.9 j / 2^F + 0.1, as a double. */
 double lpmm_oracle_de_fraction(int F, int k);
 
 /* Sec. 2.2 "Mapping": argmin_i |n - T(i)| in exact arithmetic on the binary32 values
@@ -98,7 +98,7 @@ typedef struct {
     int32_t true_division; /* 0: multiply by reciprocal scale (contract); 1: divide by the scale */
 } lpmm_oracle_hyper;
 
-/* State kinds chosen by the rule of App. C.1 and Sec. 4.2. */
+/* State kinds chosen by the rule of App. D.1 and Sec. 4.2. */
 enum { LPMM_ORACLE_FP32 = 0, LPMM_ORACLE_BLOCK = 1, LPMM_ORACLE_RANK1 = 2 };
 
 /* numel <= min_quant_numel (and not forced) -> FP32; one-dimensional or any extent 1 -> BLOCK;

@@ -18,12 +18,12 @@ FLT_MIN = np.finfo(np.float32).tiny  # smallest normal binary32
 # ----------------------------------------------------------------------------- mappings
 
 def linear_map(bits: int = 4) -> np.ndarray:
-    """App. D.2: T(i) = (i+1)/2^b; zero is excluded (Sec. 4.1)."""
+    """App. E.2: T(i) = (i+1)/2^b; zero is excluded (Sec. 4.1)."""
     return np.array([Fraction(i + 1, 2 ** bits) for i in range(2 ** bits)], dtype=np.float64).astype(F32)
 
 
 def de_fraction(F: int, k: int) -> Fraction:
-    """App. D.2: midpoint of the k-th of 2^F equal cells of [0.1, 1]."""
+    """App. E.2: midpoint of the k-th of 2^F equal cells of [0.1, 1]."""
     p = lambda j: Fraction(9, 10) * Fraction(j, 2 ** F) + Fraction(1, 10)
     return (p(k) + p(k + 1)) / 2
 
@@ -36,7 +36,7 @@ def _de_value(bitstring: str) -> Fraction:
 
 
 def de_map(bits: int = 4, signed: bool = True, drop_zero: bool = False) -> np.ndarray:
-    """App. D.2: dynamic-exponent table from the bit patterns, sorted increasingly."""
+    """App. E.2: dynamic-exponent table from the bit patterns, sorted increasingly."""
     vals = []
     for p in range(2 ** bits):
         s = format(p, f"0{bits}b")

@@ -42,7 +42,7 @@ struct TensorLayout {
 
 struct Layout {
     std::vector<TensorLayout> t;
-    size_t descs = 0, params = 0, params16 = 0, grads = 0, tiles1 = 0, tiles2 = 0, tiles3 = 0;
+    size_t descs = 0, params = 0, params16 = 0, grads = 0, tiles1 = 0, tiles2 = 0, tiles3 = 0, tiles4 = 0;
     size_t rc[2] = {0, 0}, rcp = 0;
     int64_t rc_floats = 0;
     size_t total = 0;
@@ -58,6 +58,7 @@ int public_kind(int32_t k) {
 }
 
 int32_t choose_kind(const lpmm_config& cfg, const lpmm_shape& s);
+int64_t folded_cols(const lpmm_config& cfg, int64_t numel);
 
 lpmm_status validate_config(const lpmm_config* cfg, const lpmm_shape* shapes, int32_t n) {
     if (!cfg || !shapes || n <= 0) return LPMM_ERR_INVALID_ARG;
@@ -99,11 +100,23 @@ lpmm_status validate_config(const lpmm_config* cfg, const lpmm_shape* shapes, in
     return LPMM_OK;
 }
 
+// A long 1-D tensor (a flattened parameter group, say) is block-wise in both moments, and its blocks do not care
+// how the elements are folded into rows: folded into rows of `cols` elements it can take the tiled update path.
+// Returns that row length, or 0 when the tensor stays on the element-indexed path.
+int64_t folded_cols(const lpmm_config& cfg, int64_t numel) {
+    if (numel < 65536) return 0;
+    if (cfg.m_block == 2048) return (numel % 2048 == 0) ? 2048 : 0;
+    for (int64_t c = 1024; c >= 128; c /= 2)
+        if (numel % c == 0) return c;
+    return 0;
+}
+
 int32_t choose_kind(const lpmm_config& cfg, const lpmm_shape& s) {
     const int64_t numel = s.rows * s.cols;
     if (s.flags & LPMM_FORCE_FP32) return K_FP32;
-    if (!(s.flags & LPMM_FORCE_QUANT) && numel <= cfg.min_quant_numel) return K_FP32;  // App. C.1
-    if (s.ndim == 1 || s.rows == 1 || s.cols == 1) return K_BLOCK;  // Sec. 4.2
+    if (!(s.flags & LPMM_FORCE_QUANT) && numel <= cfg.min_quant_numel) return K_FP32;  // App. D.1
+    if (s.ndim == 1 || s.rows == 1 || s.cols == 1)   // Sec. 4.2
+        return (cfg.v_mode != LPMM_V_FACTORED && folded_cols(cfg, numel) > 0) ? K_BLOCK_TILED : K_BLOCK;
     if (cfg.v_mode == LPMM_V_BLOCK) {   // block-wise second moment on a matrix: tiled when whole blocks lie inside a row
         const bool tiled = s.ndim == 2 && s.cols % 128 == 0 && s.cols % cfg.m_block == 0 && s.cols <= ((int64_t)1 << 24);
         return tiled ? K_BLOCK_TILED : K_BLOCK;
@@ -125,12 +138,17 @@ void compute_layout(const lpmm_config& cfg, const lpmm_shape* shapes, int32_t n,
     L->tiles1 = off; off = align_up(off + sizeof(int32_t) * (n + 1));
     L->tiles2 = off; off = align_up(off + sizeof(int32_t) * (n + 1));
     L->tiles3 = off; off = align_up(off + sizeof(int32_t) * (n + 1));
+    L->tiles4 = off; off = align_up(off + sizeof(int32_t) * (n + 1));
     int64_t rc = 0;
     for (int32_t i = 0; i < n; ++i) {
         TensorLayout& t = L->t[i];
         t = TensorLayout{};
         t.rows = shapes[i].rows; t.cols = shapes[i].cols; t.numel = t.rows * t.cols;
         t.kind = choose_kind(cfg, shapes[i]);
+        if (t.kind == K_BLOCK_TILED && (shapes[i].ndim == 1 || t.rows == 1 || t.cols == 1)) {   // folded, see folded_cols()
+            t.cols = folded_cols(cfg, t.numel);
+            t.rows = t.numel / t.cols;
+        }
         if (uses_rc(t.kind)) {
             t.rc_index = rc;
             if (shapes[i].ndim >= 3) {   // one vector of statistics per axis, each padded to 4 floats
@@ -183,6 +201,7 @@ struct lpmm_state {
     size_t arena_bytes;
     int32_t phase;
     int32_t grid1, grid2, total1, total2;
+    std::vector<int32_t> tiles4;           // prefix sums of the folded 1-D tensors' tiles (their own update launch)
     int32_t last_launches;
     bool ptrs_valid;
     std::vector<void*> params, grads;  // what the device-side pointer arrays currently hold
@@ -247,7 +266,10 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
     }
 
     std::vector<TensorDesc> descs(n);
-    std::vector<int32_t> t1(n + 1, 0), t2(n + 1, 0), t3(n + 1, 0);
+    std::vector<int32_t> t1(n + 1, 0), t2(n + 1, 0), t3(n + 1, 0), t4(n + 1, 0);
+    // In a state whose matrices are not block-wise, folded 1-D tensors leave the main update launch (0 tiles there)
+    // and get one of their own with the block-wise kernel (table 4).
+    const bool own_launch = st->cfg.v_mode != LPMM_V_BLOCK;
     char* A = st->arena;
     for (int32_t i = 0; i < n; ++i) {
         const TensorLayout& t = st->L.t[i];
@@ -298,7 +320,9 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
             t3[i + 1] = t3[i] + (int32_t)flat_tiles;
         }
         if (t2[i] + tiles > 0x7fffffffLL) return LPMM_ERR_UNSUPPORTED;
-        t2[i + 1] = t2[i] + (int32_t)tiles;
+        const bool moved = own_launch && t.kind == K_BLOCK_TILED;
+        t2[i + 1] = t2[i] + (moved ? 0 : (int32_t)tiles);
+        t4[i + 1] = t4[i] + (moved ? (int32_t)tiles : 0);
         const bool rank1 = uses_rc(t.kind);
         const bool tiled = (t.kind == K_RANK1_FAST || t.kind == K_FACT);
         t1[i + 1] = t1[i] + (rank1 ? (int32_t)(tiled ? tiles_p1 : tiles) : 0);
@@ -311,6 +335,8 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
     st->tiles1 = t1;
     st->tiles2 = t2;
     st->tiles3 = t3;
+    st->tiles4 = t4;
+    LPMM_CUDA(cudaMemcpyAsync(A + st->L.tiles4, t4.data(), sizeof(int32_t) * (n + 1), cudaMemcpyHostToDevice, s));
     LPMM_CUDA(cudaMemcpyAsync(A + st->L.tiles3, t3.data(), sizeof(int32_t) * (n + 1), cudaMemcpyHostToDevice, s));
     LPMM_CUDA(cudaMemcpyAsync(A + st->L.descs, descs.data(), sizeof(TensorDesc) * n, cudaMemcpyHostToDevice, s));
     LPMM_CUDA(cudaMemcpyAsync(A + st->L.tiles1, t1.data(), sizeof(int32_t) * (n + 1), cudaMemcpyHostToDevice, s));
@@ -521,8 +547,17 @@ lpmm_status enqueue_range(lpmm_state* st, StepArgs a, int32_t t0, int32_t t1, bo
     LPMM_CUDA(launch_pass2(a, bf16, ieee_update, st->cfg.m_block == 2048 ? 11 : 7,
                            st->cfg.v_mode == LPMM_V_FACTORED ? 1 : (st->cfg.v_mode == LPMM_V_BLOCK ? 2 : 0),
                            tiles < cap ? tiles : cap, s));
-    if (ev) LPMM_CUDA(cudaEventRecord(ev[3], s));
     *launches += 1;
+    if (st->tiles4[t1] > st->tiles4[t0]) {   // folded 1-D tensors of a state that is not block-wise
+        a.tile_start = reinterpret_cast<const int32_t*>(st->arena + st->L.tiles4);
+        a.tile_begin = st->tiles4[t0];
+        a.tile_end = st->tiles4[t1];
+        const int32_t tiles4 = a.tile_end - a.tile_begin;
+        a.params_bf16 = nullptr;   // (refused above together with such tensors)
+        LPMM_CUDA(launch_pass2(a, bf16, ieee_update, st->cfg.m_block == 2048 ? 11 : 7, 2, tiles4 < cap ? tiles4 : cap, s));
+        *launches += 1;
+    }
+    if (ev) LPMM_CUDA(cudaEventRecord(ev[3], s));
     return LPMM_OK;
 }
 
@@ -549,7 +584,7 @@ lpmm_status adamw4_step_impl(lpmm_state* st, void* const* d_params, void* const*
                              float weight_decay, int64_t step, void* stream) {
     lpmm_status rc = check_step_args(st, d_params, d_grads, grad_dtype, lr, beta1, beta2, eps, weight_decay, step);
     if (rc != LPMM_OK) return rc;
-    if (d_params16 && st->cfg.v_mode != LPMM_V_RANK1) return LPMM_ERR_UNSUPPORTED;   // the copy rides on the default kernels
+    if (d_params16 && (st->cfg.v_mode != LPMM_V_RANK1 || st->tiles4[st->n] > 0)) return LPMM_ERR_UNSUPPORTED;   // the copy rides on the default kernels
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     rc = set_pointers(st, d_params, d_grads, s);
     if (rc != LPMM_OK) return rc;

@@ -13,7 +13,7 @@ namespace lpmm {
 
 constexpr float kFltMin = 1.17549435e-38f;  // smallest normal binary32
 
-// Signed 4-bit dynamic-exponent table (App. D.2 with b = 1 + E + 1 + F = 4), sorted increasingly:
+// Signed 4-bit dynamic-exponent table (App. E.2 with b = 1 + E + 1 + F = 4), sorted increasingly:
 // +-{0.2125, 0.4375, 0.6625, 0.8875}, +-{0.0325, 0.0775}, +-0.0055, 0 and +1 (no -1).
 __device__ __constant__ float kDeTable[16] = {
     -0.8875f, -0.6625f, -0.4375f, -0.2125f, -0.0775f, -0.0325f, -0.0055f, 0.0f,
@@ -161,7 +161,7 @@ __host__ __device__ __forceinline__ Hyper2 make_hyper2(const Hyper& h) {
     p.lin_b23 = make_float2(0.0625f - 2048.0f, 0.0625f - 128.0f);
     return p;
 }
-// T_lin(q) = (q + 1)/16 (App. D.2) for the eight codes of one word, without a table: a nibble at bit 4k
+// T_lin(q) = (q + 1)/16 (App. E.2) for the eight codes of one word, without a table: a nibble at bit 4k
 // (k <= 3), OR-ed into the mantissa of 2^23, is the number 2^23 + q 16^k, and one fused multiply-add maps it
 // to (q + 1)/16. Every intermediate and the result are exactly representable, so nothing is rounded.
 // t[i] holds the entries of elements 2i and 2i + 1.

@@ -861,7 +861,7 @@ __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restric
     }
 }
 
-// ---- pass 2, small tensors with fp32 states (App. C.1) ------------------------------------------
+// ---- pass 2, small tensors with fp32 states (App. D.1) ------------------------------------------
 
 template <bool BF16, bool EXACT, bool WB = false, bool A32 = false>
 __device__ __forceinline__ void pass2_fp32(const TensorDesc& d, float* __restrict__ w, uint16_t* __restrict__ w16,
@@ -928,7 +928,8 @@ __global__ void __launch_bounds__(kThreads, 2) pass2_kernel(StepArgs a) {
             case K_FACT:
                 if (VF == 1) pass2_rank1_fast<BF16, EXACT, MSHIFT, 1, WB>(d, w, w16, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step);
                 break;
-            case K_BLOCK_TILED:
+            case K_BLOCK_TILED:   // matrices of a block-wise state; long 1-D tensors folded into rows (in states of another
+                                  // kind these get a launch of their own, so that the default kernels stay lean)
                 if (VF == 2) pass2_rank1_fast<BF16, EXACT, MSHIFT, 2, WB, A32>(d, w, w16, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step);
                 break;
             case K_RANK1_FLAT: pass2_flat<BF16, true, EXACT, MSHIFT, WB, A32>(d, w, w16, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;

@@ -455,3 +455,23 @@ def test_pointers_aligned_to_16_but_not_32_bytes_give_the_same_result(grad_dtype
             for name in ("m_codes", "m_scale", "v_codes", "v_s0", "v_s1"):
                 if va[name] is not None:
                     assert torch.equal(va[name], vb[name]), (s.name, name, t)
+
+
+@pytest.mark.parametrize("grad_dtype,m_block,v_mode", [(torch.bfloat16, 128, lpmm.V_RANK1), (torch.float32, 128, lpmm.V_BLOCK),
+                                                       (torch.float32, 2048, lpmm.V_RANK1)])
+def test_long_one_dimensional_tensors_folded_into_rows(grad_dtype, m_block, v_mode):
+    # 1-D tensors of at least 65536 elements whose length is a multiple of 128 (2048 with B2048) are folded into rows
+    # and take the tiled update path (in a state that is not block-wise: in a launch of their own); block-wise
+    # quantization does not see the folding, so codes and scales must equal the oracle's 1-D result bit for bit.
+    cfg = lpmm.default_config(m_block=m_block, v_mode=v_mode)
+    specs = [_vec(196608), _vec(70016 if m_block == 128 else 67584), _vec(65536 + 2048 * 5), _mat(96, 256), _vec(66000), _vec(300)]
+    hyper = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
+    pair = Pair(specs, hyper, grad_dtype=grad_dtype, config=cfg, workload_index=17)
+    for t in range(1, 5):
+        grads = pair.grads_for(t, outlier_p=0.0 if t % 2 == 0 else 1e-3)
+        if t == 3:
+            grads[0][:70000] = 0
+        pair.step(t, grads)
+        pair.compare(tol=1e-6)
+    want = 4 if v_mode == lpmm.V_RANK1 else 1     # maxima + reciprocal + update (+ the folded tensors' own update launch)
+    assert pair.state.last_launches == want

@@ -1,7 +1,7 @@
 """Pins of the oracle's quantization mappings and nearest-entry rule (CPU only).
 
 Each test ties the oracle to something other than itself: constants the paper prints, tables
-worked by hand from App. D.2, exact rational arithmetic, or brute force.
+worked by hand from App. E.2, exact rational arithmetic, or brute force.
 """
 from fractions import Fraction
 
