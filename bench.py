@@ -292,15 +292,17 @@ def run_ours(args):
     peak, peak_kind = measured_peak()
     p2_ms = prof["pass2_ms"] / max(prof["steps"], 1)
     p1_ms = prof["pass1_ms"] / max(prof["steps"], 1)
-    # block maxima: 8 bytes per block of m (and of v when v is block-wise; then pass 1 has nothing to do)
-    pass2_bpp = PASS2_BYTES[wl.grad_dtype] - 8 / 128 + 8 / args.m_block + (8 / 128 if args.v_mode == "block" else 0)
-    pass1_bpp = {"rank1": PASS1_BYTES[wl.grad_dtype], "block": 0.0, "factored": PASS1_BYTES[wl.grad_dtype] - 0.5}[args.v_mode]
-    if args.v_mode == "factored":
+    # block maxima: 8 bytes per block of m (and of v when v is block-wise; then pass 1 has nothing to do).
+    # A list of 1-D tensors only (flattened parameters) is block-wise whatever the mode (Sec. 4.2).
+    v_kind = "block" if all(t.ndim == 1 for t in wl.tensors) else args.v_mode
+    pass2_bpp = PASS2_BYTES[wl.grad_dtype] - 8 / 128 + 8 / args.m_block + (8 / 128 if v_kind == "block" else 0)
+    pass1_bpp = {"rank1": PASS1_BYTES[wl.grad_dtype], "block": 0.0, "factored": PASS1_BYTES[wl.grad_dtype] - 0.5}[v_kind]
+    if v_kind == "factored":
         pass2_bpp -= 1.0      # no second-moment codes are read or written
     alg_bytes = pass2_bpp * n_params
     achieved = alg_bytes / (p2_ms * 1e-3) / 1e9
     # the captures cover the default quantizers only
-    traffic_pp = PASS2_TRAFFIC_BYTES_PER_PARAM[wl.grad_dtype] if (args.v_mode == "rank1" and args.m_block == 128) else None
+    traffic_pp = PASS2_TRAFFIC_BYTES_PER_PARAM[wl.grad_dtype] if (v_kind == "rank1" and args.m_block == 128) else None
     roofline = {"bound": "hbm", "kernel": "pass2_kernel (update + re-quantize)", "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                 "traffic": None if traffic_pp is None else traffic_pp * n_params,
@@ -320,7 +322,7 @@ def run_ours(args):
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": wl.name, "tensors": len(wl.tensors), "params_per_gpu": n_params,
-                       "grad_dtype": wl.grad_dtype, "param_dtype": "f32", "m": f"B{args.m_block}/DE 4-bit", "v": {"rank1": "Rank-1/Linear 4-bit", "block": "B128/Linear 4-bit", "factored": "factorized (fp32 row/column statistics)"}[args.v_mode],
+                       "grad_dtype": wl.grad_dtype, "param_dtype": "f32", "m": f"B{args.m_block}/DE 4-bit", "v": {"rank1": "Rank-1/Linear 4-bit", "block": "B128/Linear 4-bit", "factored": "factorized (fp32 row/column statistics)"}[v_kind],
                        "l2": f"inputs larger than L2 ({(n_params * (8 + (2 if wl.grad_dtype == 'bf16' else 4) + 1)) / 1e9:.1f} GB touched per step), no flush", "parallelism": f"replicas x{world}, no collective"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu}
     print(json.dumps(line), flush=True)

@@ -128,6 +128,16 @@ def llama_7b(layers: int = 32, vocab: int = 32000) -> Workload:
     return Workload(name, 3, tuple(ts), lr=2e-5, weight_decay=0.0, grad_dtype="bf16", steps=20)
 
 
+def llama_7b_flat() -> Workload:
+    """The LLaMA-7B parameters packed into 1-D arrays, one per decoder layer plus embedding and head, as a
+    sharded-data-parallel wrapper flattens them (App. D.2 "LLaMA": all parameters one-dimensional, hence block-wise
+    normalization for both moments); bf16 gradients."""
+    d, ff, vocab = 4096, 11008, 32000
+    per_layer = 4 * d * d + 3 * d * ff + 2 * d
+    ts = [_vec("embed", vocab * d)] + [_vec(f"l{i}", per_layer) for i in range(32)] + [_vec("head", vocab * d + d)]
+    return Workload("llama_7b_flat", 5, tuple(ts), lr=2e-5, weight_decay=0.0, grad_dtype="bf16", steps=20)
+
+
 def square_8192() -> Workload:
     """One 8192x8192 matrix for the quantizer/normalizer sweep."""
     return Workload("square_8192", 4, (_mat("weight", 8192, 8192),), lr=1e-3, steps=10)
@@ -139,6 +149,7 @@ WORKLOADS = {
     "roberta_large": roberta_large,
     "llama_7b": llama_7b,
     "square_8192": square_8192,
+    "llama_7b_flat": llama_7b_flat,
     # reduced LLaMA list (embedding, head and a few decoder layers) for profiler captures and quick checks
     "llama_7b_1l": lambda: llama_7b(layers=1),
     "llama_7b_4l": lambda: llama_7b(layers=4),
