@@ -805,7 +805,20 @@ __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restric
         // shuffle-based table lookup reads T[q] * scale from the group's other lanes
         const bool group_live = (e & ~m_mask) < d.numel;
         const float am = group_live ? d.m_scale[e >> MSHIFT] : 0.0f;
-        if (RANK1) {
+        if (RANK1 && full && (d.cols & 7) == 0) {
+            // cols % 8 == 0: the lane's eight elements lie in one row, their column statistics are two 16-byte loads
+            int64_t i, j;
+            split_index(d, e, i, j);
+            const float so = outer_stat<false>(d, rc_old, i), ro = outer_stat<true>(d, rcp_new, i);
+            float co[8], cr[8];
+            load8_f32(rc_old + d.c_off + j, co);
+            load8_f32(rcp_new + d.c_off + j, cr);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                vs[k] = fminf(so, co[k]);
+                vr[k] = fmaxf(ro, cr[k]);
+            }
+        } else if (RANK1) {
             int64_t i, j;
             split_index(d, e, i, j);
             float so = 0.0f, ro = 0.0f;          // leading axes' share of the old scale / the new reciprocal, row i
