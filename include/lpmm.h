@@ -121,7 +121,9 @@ lpmm_status lpmm_state_attach(const lpmm_config* cfg, const lpmm_shape* shapes, 
  * framework allocations are, the update pass uses 256-bit accesses and is ~6 % faster). step is t >= 1.
  * Requires 0 <= beta1, beta2 < 1, lr >= 0, eps >= 0, weight_decay >= 0, all finite.
  * Kernels launched: one pass over the rank-1 tensors that reduces the new row/column maxima, one
- * small pass that inverts them, one pass over all tensors that updates and re-quantizes.
+ * small pass that inverts them, one pass over all tensors that updates and re-quantizes; one more update
+ * launch when the state holds 1-D tensors of 65536 elements or more whose length is a multiple of 128 (they are
+ * folded into rows and updated by the block-wise form of the tiled kernel) and its matrices are not block-wise.
  * LPMM_V_FACTORED (reading of Sec. 4.3, which gives no formula): R <- b2 R + (1-b2) rowsum(g^2), C likewise,
  * v_ij = R_i C_j / sum(R), then Eq. 1 as usual; the first pass reduces the sums (fp32 atomics, so R and C are
  * reproducible to rounding only), a fourth small kernel updates R, C and sum(R). Such tensors need
@@ -135,7 +137,7 @@ lpmm_status lpmm_adamw4_step(lpmm_state* st, void* const* d_params, const void* 
  * the paper's method has no such output: its states and fp32 parameters are updated exactly as by lpmm_adamw4_step).
  *   d_params_bf16[i] : device pointer to numel bfloat16 values of tensor i (written), 16-byte aligned; a HOST array
  *                      of n device pointers like d_params.
- * Not available with LPMM_V_FACTORED (LPMM_ERR_UNSUPPORTED). */
+ * Only with LPMM_V_RANK1 and without folded 1-D tensors (see lpmm_adamw4_step); LPMM_ERR_UNSUPPORTED otherwise. */
 lpmm_status lpmm_adamw4_step_bf16w(lpmm_state* st, void* const* d_params, void* const* d_params_bf16,
                                    const void* const* d_grads, int32_t grad_dtype, float lr, float beta1, float beta2,
                                    float eps, float weight_decay, int64_t step, void* stream);
