@@ -137,7 +137,7 @@ lpmm_status lpmm_adamw4_step(lpmm_state* st, void* const* d_params, const void* 
  * the paper's method has no such output: its states and fp32 parameters are updated exactly as by lpmm_adamw4_step).
  *   d_params_bf16[i] : device pointer to numel bfloat16 values of tensor i (written), 16-byte aligned; a HOST array
  *                      of n device pointers like d_params.
- * Only with LPMM_V_RANK1 and without folded 1-D tensors (see lpmm_adamw4_step); LPMM_ERR_UNSUPPORTED otherwise. */
+ * Not available with LPMM_V_FACTORED (LPMM_ERR_UNSUPPORTED). */
 lpmm_status lpmm_adamw4_step_bf16w(lpmm_state* st, void* const* d_params, void* const* d_params_bf16,
                                    const void* const* d_grads, int32_t grad_dtype, float lr, float beta1, float beta2,
                                    float eps, float weight_decay, int64_t step, void* stream);

@@ -553,7 +553,6 @@ lpmm_status enqueue_range(lpmm_state* st, StepArgs a, int32_t t0, int32_t t1, bo
         a.tile_begin = st->tiles4[t0];
         a.tile_end = st->tiles4[t1];
         const int32_t tiles4 = a.tile_end - a.tile_begin;
-        a.params_bf16 = nullptr;   // (refused above together with such tensors)
         LPMM_CUDA(launch_pass2(a, bf16, ieee_update, st->cfg.m_block == 2048 ? 11 : 7, 2, tiles4 < cap ? tiles4 : cap, s));
         *launches += 1;
     }
@@ -584,7 +583,7 @@ lpmm_status adamw4_step_impl(lpmm_state* st, void* const* d_params, void* const*
                              float weight_decay, int64_t step, void* stream) {
     lpmm_status rc = check_step_args(st, d_params, d_grads, grad_dtype, lr, beta1, beta2, eps, weight_decay, step);
     if (rc != LPMM_OK) return rc;
-    if (d_params16 && (st->cfg.v_mode != LPMM_V_RANK1 || st->tiles4[st->n] > 0)) return LPMM_ERR_UNSUPPORTED;   // the copy rides on the default kernels
+    if (d_params16 && st->cfg.v_mode == LPMM_V_FACTORED) return LPMM_ERR_UNSUPPORTED;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     rc = set_pointers(st, d_params, d_grads, s);
     if (rc != LPMM_OK) return rc;

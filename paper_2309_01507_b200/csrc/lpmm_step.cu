@@ -1448,8 +1448,13 @@ cudaError_t launch_pass2_t(const StepArgs& a, int v_kind, int grid, cudaStream_t
     if (v_kind == 1) {
         pass2_kernel<BF16, EXACT, MSHIFT, 1, false, false><<<grid, kThreads, 0, s>>>(a);
     } else if (v_kind == 2) {
-        if (a.aligned32) pass2_kernel<BF16, EXACT, MSHIFT, 2, false, true><<<grid, kThreads, 0, s>>>(a);
-        else pass2_kernel<BF16, EXACT, MSHIFT, 2, false, false><<<grid, kThreads, 0, s>>>(a);
+        if (a.params_bf16 != nullptr) {
+            if (a.aligned32) pass2_kernel<BF16, EXACT, MSHIFT, 2, true, true><<<grid, kThreads, 0, s>>>(a);
+            else pass2_kernel<BF16, EXACT, MSHIFT, 2, true, false><<<grid, kThreads, 0, s>>>(a);
+        } else {
+            if (a.aligned32) pass2_kernel<BF16, EXACT, MSHIFT, 2, false, true><<<grid, kThreads, 0, s>>>(a);
+            else pass2_kernel<BF16, EXACT, MSHIFT, 2, false, false><<<grid, kThreads, 0, s>>>(a);
+        }
     } else if (a.params_bf16 != nullptr) {
         if (a.aligned32) pass2_kernel<BF16, EXACT, MSHIFT, 0, true, true><<<grid, kThreads, 0, s>>>(a);
         else pass2_kernel<BF16, EXACT, MSHIFT, 0, true, false><<<grid, kThreads, 0, s>>>(a);
