@@ -10,9 +10,11 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "liblpmm.so")
-SOURCES = ["lpmm_api.cu", "lpmm_step.cu", "lpmm_quant.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "-fmad=false", "-Xcompiler", "-fPIC", "-shared", "-cudart", "static"]
+              "-fmad=false", "-Xcompiler", "-fPIC"]
+# (source, extra flags, object name): the step kernels are compiled as four parts side by side
+UNITS = [("lpmm_api.cu", [], "api.o"), ("lpmm_quant.cu", [], "quant.o")] + \
+        [("lpmm_step.cu", [f"-DLPMM_STEP_PART={p}"], f"step{p}.o") for p in range(4)]
 
 
 def _newest_source() -> float:
@@ -25,9 +27,18 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _newest_source():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    cmd = [nvcc, *NVCC_FLAGS, *(["-Xptxas", "-v"] if verbose else []), "-o", LIB,
-           *[os.path.join(CSRC, s) for s in SOURCES]]
-    subprocess.run(cmd, check=True, cwd=CSRC)
+    objdir = os.path.join(HERE, "build")
+    os.makedirs(objdir, exist_ok=True)
+    procs = []
+    for src, extra, obj in UNITS:
+        cmd = [nvcc, *NVCC_FLAGS, *extra, *(["-Xptxas", "-v"] if verbose else []), "-c", "-o", os.path.join(objdir, obj),
+               os.path.join(CSRC, src)]
+        procs.append((cmd, subprocess.Popen(cmd, cwd=CSRC)))
+    for cmd, p in procs:
+        if p.wait() != 0:
+            raise subprocess.CalledProcessError(p.returncode, cmd)
+    subprocess.run([nvcc, "-shared", "-cudart", "static", "-o", LIB, *[os.path.join(objdir, o) for _, _, o in UNITS]],
+                   check=True, cwd=CSRC)
     return LIB
 
 

@@ -65,6 +65,10 @@ struct StepArgs {
 
 cudaError_t launch_pass1(const StepArgs& a, bool bf16, int ctas_per_sm, int grid, cudaStream_t s);
 cudaError_t launch_pass2(const StepArgs& a, bool bf16, bool exact, int m_shift, int v_kind, int grid, cudaStream_t s);
+cudaError_t launch_pass2_bf16_fast(const StepArgs& a, int m_shift, int v_kind, int grid, cudaStream_t s);
+cudaError_t launch_pass2_bf16_ieee(const StepArgs& a, int m_shift, int v_kind, int grid, cudaStream_t s);
+cudaError_t launch_pass2_f32_fast(const StepArgs& a, int m_shift, int v_kind, int grid, cudaStream_t s);
+cudaError_t launch_pass2_f32_ieee(const StepArgs& a, int m_shift, int v_kind, int grid, cudaStream_t s);
 cudaError_t launch_factor_finalize(const StepArgs& a, int t0, int t1, cudaStream_t s);
 cudaError_t launch_sgdm(const StepArgs& a, bool bf16, int grid, cudaStream_t s);
 cudaError_t launch_rcp(const float* src, float* dst, int64_t n, cudaStream_t s);

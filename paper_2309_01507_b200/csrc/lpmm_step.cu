@@ -13,6 +13,14 @@
 // of fp32) gradient and one 32-bit word of each moment's codes; 16 lanes own one 128-element block.
 #include "lpmm_internal.h"
 
+// The update pass has 80 instantiations; to build in parallel this file can be compiled four times with
+// -DLPMM_STEP_PART=0..3, each part holding the update-pass launchers of one (gradient type, update math) pair and
+// part 0 the remaining launchers as well. Without the macro one translation unit holds everything.
+#ifndef LPMM_STEP_PART
+#define LPMM_STEP_ALL 1
+#define LPMM_STEP_PART 0
+#endif
+
 namespace lpmm {
 
 namespace {
@@ -1262,6 +1270,7 @@ __device__ __forceinline__ void pass1_fact(const TensorDesc& d, const void* __re
     }
 }
 
+#if LPMM_STEP_PART == 0   // non-template kernels live in one part only
 // One CTA per factorized tensor: turns the sums into the statistics' moving averages R, C (in the "new"
 // buffer), sums R in binary64 in a fixed order and stores the row factors R_i * (1 / sum R).
 __global__ void __launch_bounds__(256) factor_finalize_kernel(StepArgs a, int t0) {
@@ -1287,6 +1296,7 @@ __global__ void __launch_bounds__(256) factor_finalize_kernel(StepArgs a, int t0
     const float r_total = scale_rcp((float)s_part[0]);
     for (int64_t i = threadIdx.x; i < d.rows; i += blockDim.x) d.rcp_new[i] = __fmul_rn(cur[i], r_total);
 }
+#endif
 
 template <bool BF16>
 __device__ __forceinline__ void pass1_rank1_flat(const TensorDesc& d, const void* __restrict__ g, int tile, int phase,
@@ -1424,13 +1434,16 @@ __global__ void __launch_bounds__(kThreads, 3) sgdm_kernel(StepArgs a) {
     tiles_done(a.tile_counter);
 }
 
+#if LPMM_STEP_PART == 0
 __global__ void rcp_kernel(const float* __restrict__ src, float* __restrict__ dst, int64_t n) {
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
         dst[i] = scale_rcp(src[i]);
 }
+#endif
 
 }  // namespace
 
+#if LPMM_STEP_PART == 0
 cudaError_t launch_pass1(const StepArgs& a, bool bf16, int ctas_per_sm, int grid, cudaStream_t s) {
     if (a.tile_end <= a.tile_begin) return cudaSuccess;
     if (ctas_per_sm == 2) {
@@ -1442,6 +1455,8 @@ cudaError_t launch_pass1(const StepArgs& a, bool bf16, int ctas_per_sm, int grid
     }
     return cudaGetLastError();
 }
+
+#endif
 
 template <bool BF16, bool EXACT, int MSHIFT>
 cudaError_t launch_pass2_t(const StepArgs& a, int v_kind, int grid, cudaStream_t s) {
@@ -1476,11 +1491,26 @@ cudaError_t launch_pass2_m(const StepArgs& a, int m_shift, int v_kind, int grid,
     return m_shift == 11 ? launch_pass2_t<BF16, EXACT, 11>(a, v_kind, grid, s) : launch_pass2_t<BF16, EXACT, 7>(a, v_kind, grid, s);
 }
 
+// One launcher per (gradient type, update math) pair, each in its own part of the build.
+#if defined(LPMM_STEP_ALL) || LPMM_STEP_PART == 0
+cudaError_t launch_pass2_bf16_fast(const StepArgs& a, int m_shift, int v_kind, int grid, cudaStream_t s) { return launch_pass2_m<true, false>(a, m_shift, v_kind, grid, s); }
+#endif
+#if defined(LPMM_STEP_ALL) || LPMM_STEP_PART == 1
+cudaError_t launch_pass2_bf16_ieee(const StepArgs& a, int m_shift, int v_kind, int grid, cudaStream_t s) { return launch_pass2_m<true, true>(a, m_shift, v_kind, grid, s); }
+#endif
+#if defined(LPMM_STEP_ALL) || LPMM_STEP_PART == 2
+cudaError_t launch_pass2_f32_fast(const StepArgs& a, int m_shift, int v_kind, int grid, cudaStream_t s) { return launch_pass2_m<false, false>(a, m_shift, v_kind, grid, s); }
+#endif
+#if defined(LPMM_STEP_ALL) || LPMM_STEP_PART == 3
+cudaError_t launch_pass2_f32_ieee(const StepArgs& a, int m_shift, int v_kind, int grid, cudaStream_t s) { return launch_pass2_m<false, true>(a, m_shift, v_kind, grid, s); }
+#endif
+
+#if LPMM_STEP_PART == 0
 // v_kind: 0 rank-1 second moments, 1 factorized, 2 block-wise (which tiled path the state's matrices take).
 cudaError_t launch_pass2(const StepArgs& a, bool bf16, bool exact, int m_shift, int v_kind, int grid, cudaStream_t s) {
     if (a.tile_end <= a.tile_begin) return cudaSuccess;
-    if (bf16) return exact ? launch_pass2_m<true, true>(a, m_shift, v_kind, grid, s) : launch_pass2_m<true, false>(a, m_shift, v_kind, grid, s);
-    return exact ? launch_pass2_m<false, true>(a, m_shift, v_kind, grid, s) : launch_pass2_m<false, false>(a, m_shift, v_kind, grid, s);
+    if (bf16) return exact ? launch_pass2_bf16_ieee(a, m_shift, v_kind, grid, s) : launch_pass2_bf16_fast(a, m_shift, v_kind, grid, s);
+    return exact ? launch_pass2_f32_ieee(a, m_shift, v_kind, grid, s) : launch_pass2_f32_fast(a, m_shift, v_kind, grid, s);
 }
 
 cudaError_t launch_factor_finalize(const StepArgs& a, int t0, int t1, cudaStream_t s) {
@@ -1510,5 +1540,7 @@ cudaError_t step_kernel_occupancy(int pass1_ctas_per_sm, int* p1, int* p2) {
     if (e != cudaSuccess) return e;
     return cudaOccupancyMaxActiveBlocksPerMultiprocessor(p2, pass2_kernel<true, false, 7, 0, false, true>, kThreads, 0);
 }
+
+#endif  // LPMM_STEP_PART == 0
 
 }  // namespace lpmm
