@@ -11,7 +11,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "liblpmm.so")
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "-fmad=false", "-Xcompiler", "-fPIC"]
+              "-fmad=false", "-Xcompiler", "-fPIC", "-Xfatbin", "-compress-all"]
 # (source, extra flags, object name): the step kernels are compiled as four parts side by side
 UNITS = [("lpmm_api.cu", [], "api.o"), ("lpmm_quant.cu", [], "quant.o")] + \
         [("lpmm_step.cu", [f"-DLPMM_STEP_PART={p}"], f"step{p}.o") for p in range(4)]
