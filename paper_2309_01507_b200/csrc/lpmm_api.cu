@@ -635,6 +635,7 @@ lpmm_status lpmm_sgdm4_step(lpmm_state* st, void* const* d_params, const void* c
     if (rc != LPMM_OK) return rc;
     StepArgs a = make_args(st, lr, beta, 0.0f, 0.0f, 0.0f, 1);
     a.h2.neg_step = make_float2(-lr, -lr);
+    a.aligned32 = (st->params_a32 && (grad_dtype == LPMM_BF16 || st->grads_a32)) ? 1 : 0;
     a.tile_start = reinterpret_cast<const int32_t*>(st->arena + st->L.tiles3);
     a.tile_begin = 0;
     a.tile_end = st->tiles3[st->n];

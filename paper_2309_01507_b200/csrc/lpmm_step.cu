@@ -1364,7 +1364,27 @@ __global__ void __launch_bounds__(kThreads, MINB) pass1_kernel(StepArgs a) {
 
 // ---- compressed SGDM (Alg. 2): m = beta m + g ; w = w - lr m ; compress m. One pass, element-indexed -------
 
-template <bool BF16>
+// One full chunk of a B128 tensor: the lane's eight elements, already loaded.
+template <bool A32>
+__device__ __forceinline__ void sgdm_chunk(float* w, uint8_t* mq, float* ms, float (&wv)[8], const float (&gv)[8], uint32_t qm,
+                                           float prod, const Hyper2& h2, const LaneTables& lt, const unsigned char* s_lut) {
+    float mt[8];
+#pragma unroll
+    for (int k = 0; k < 8; k += 2) {
+        const float2 mo = make_float2(__shfl_sync(lt.mask, prod, (int)(qm >> (4 * k)), 16),
+                                      __shfl_sync(lt.mask, prod, (int)(qm >> (4 * k + 4)), 16));
+        const float2 m2 = fma2_rn(mul2_rn(h2.beta1, mo), h2.one, make_float2(gv[k], gv[k + 1]));
+        const float2 w2 = fma2_rn(mul2_rn(h2.neg_step, m2), h2.one, make_float2(wv[k], wv[k + 1]));
+        mt[k] = m2.x; mt[k + 1] = m2.y;
+        wv[k] = w2.x; wv[k + 1] = w2.y;
+    }
+    store8_f32_a<A32>(w, wv);
+    const float am_new = group_max(absmax8(mt), lt.mask);
+    if ((threadIdx.x & 15) == 0) *ms = am_new;
+    *reinterpret_cast<uint32_t*>(mq) = quantize8_de(mt, scale_rcp(am_new), s_lut);
+}
+
+template <bool BF16, bool A32>
 __global__ void __launch_bounds__(kThreads, 3) sgdm_kernel(StepArgs a) {
     __shared__ __align__(16) unsigned char s_lut[kLutSmemBytes];
     __shared__ float s_red[2 * kWarps];
@@ -1384,7 +1404,26 @@ __global__ void __launch_bounds__(kThreads, 3) sgdm_kernel(StepArgs a) {
         const void* g = a.grads[t];
         const int local = tile - __ldg(a.tile_start + t);
         const int64_t m_mask = ((int64_t)1 << d.m_shift) - 1;
-        for (int c = 0; c < d.flat_chunks; ++c) {
+        int c_first = 0;
+        // A tile that lies wholly inside a B128 tensor takes its chunks two at a time: both chunks' loads are in flight
+        // before either is processed, and nothing needs a guard.
+        if (d.kind != K_FP32 && d.m_shift == 7 && ((int64_t)(local + 1) * d.flat_chunks) * kWarps * kWarpElems <= d.numel) {
+            for (; c_first + 1 < d.flat_chunks; c_first += 2) {
+                const int64_t e0 = (((int64_t)local * d.flat_chunks + c_first) * kWarps + warp) * kWarpElems + lane * kLaneElems;
+                const int64_t e1 = e0 + (int64_t)kWarps * kWarpElems;
+                float w0[8], w1[8], g0[8], g1[8];
+                load8_rw_a<A32>(w + e0, w0);
+                load8_rw_a<A32>(w + e1, w1);
+                load8_grad_a<BF16, A32>(g, e0, g0);
+                load8_grad_a<BF16, A32>(g, e1, g1);
+                const uint32_t q0 = *reinterpret_cast<const uint32_t*>(d.m_codes + (e0 >> 1));
+                const uint32_t q1 = *reinterpret_cast<const uint32_t*>(d.m_codes + (e1 >> 1));
+                const float p0 = __fmul_rn(lt.de, d.m_scale[e0 >> 7]), p1 = __fmul_rn(lt.de, d.m_scale[e1 >> 7]);
+                sgdm_chunk<A32>(w + e0, d.m_codes + (e0 >> 1), d.m_scale + (e0 >> 7), w0, g0, q0, p0, h2, lt, s_lut);
+                sgdm_chunk<A32>(w + e1, d.m_codes + (e1 >> 1), d.m_scale + (e1 >> 7), w1, g1, q1, p1, h2, lt, s_lut);
+            }
+        }
+        for (int c = c_first; c < d.flat_chunks; ++c) {
             const int64_t chunk0 = ((int64_t)local * d.flat_chunks + c) * kWarps;
             const int64_t chunk = chunk0 + warp;
             const int64_t e = chunk * kWarpElems + lane * kLaneElems;
@@ -1521,8 +1560,13 @@ cudaError_t launch_factor_finalize(const StepArgs& a, int t0, int t1, cudaStream
 
 cudaError_t launch_sgdm(const StepArgs& a, bool bf16, int grid, cudaStream_t s) {
     if (a.tile_end <= a.tile_begin) return cudaSuccess;
-    if (bf16) sgdm_kernel<true><<<grid, kThreads, 0, s>>>(a);
-    else sgdm_kernel<false><<<grid, kThreads, 0, s>>>(a);
+    if (a.aligned32) {
+        if (bf16) sgdm_kernel<true, true><<<grid, kThreads, 0, s>>>(a);
+        else sgdm_kernel<false, true><<<grid, kThreads, 0, s>>>(a);
+    } else {
+        if (bf16) sgdm_kernel<true, false><<<grid, kThreads, 0, s>>>(a);
+        else sgdm_kernel<false, false><<<grid, kThreads, 0, s>>>(a);
+    }
     return cudaGetLastError();
 }
 
