@@ -47,6 +47,8 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama_7b")
+    ap.add_argument("--optimizer", choices=["adamw", "sgdm"], default="adamw",
+                    help="sgdm: the compressed SGDM step (Alg. 2) instead of the AdamW step; no end-to-end leg")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -219,10 +221,18 @@ def run_ours(args):
     n_params = wl.numel
     torch.cuda.synchronize()
 
+    sgdm = args.optimizer == "sgdm"
+
+    def one_step(t):
+        if sgdm:
+            lpmm.sgdm4_step(state, params, grads, lr=wl.lr, beta=wl.beta1)
+        else:
+            lpmm.adamw4_step(state, params, grads, step=t, ptr_cache=cache, **hyper)
+
     step = 0
     for _ in range(max(args.warmup, 3)):
         step += 1
-        lpmm.adamw4_step(state, params, grads, step=step, ptr_cache=cache, **hyper)
+        one_step(step)
     torch.cuda.synchronize()
     dist.barrier()
 
@@ -234,7 +244,7 @@ def run_ours(args):
     ev0.record()
     for _ in range(args.steps):
         step += 1
-        lpmm.adamw4_step(state, params, grads, step=step, ptr_cache=cache, **hyper)
+        one_step(step)
     ev1.record()
     torch.cuda.synchronize()
     t_wall1 = time.time()
@@ -249,7 +259,7 @@ def run_ours(args):
 
     # ---- end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
     e2e = None
-    if not args.no_e2e and args.e2e_steps > 0:
+    if not args.no_e2e and args.e2e_steps > 0 and not sgdm:
         gsz = 2 if wl.grad_dtype == "bf16" else 4
         nstage = lpmm.stage_bytes(state)
         d_pstage = torch.empty(nstage, dtype=torch.uint8, device=dev)
@@ -292,6 +302,8 @@ def run_ours(args):
     peak, peak_kind = measured_peak()
     p2_ms = prof["pass2_ms"] / max(prof["steps"], 1)
     p1_ms = prof["pass1_ms"] / max(prof["steps"], 1)
+    if sgdm:      # one kernel per step: its duration is the step time
+        p2_ms, p1_ms = ms_step, 0.0
     # block maxima: 8 bytes per block of m (and of v when v is block-wise; then pass 1 has nothing to do).
     # A list of 1-D tensors only (flattened parameters) is block-wise whatever the mode (Sec. 4.2).
     v_kind = "block" if all(t.ndim == 1 for t in wl.tensors) else args.v_mode
@@ -299,11 +311,14 @@ def run_ours(args):
     pass1_bpp = {"rank1": PASS1_BYTES[wl.grad_dtype], "block": 0.0, "factored": PASS1_BYTES[wl.grad_dtype] - 0.5}[v_kind]
     if v_kind == "factored":
         pass2_bpp -= 1.0      # no second-moment codes are read or written
+    if sgdm:                  # w 4+4, g, first-moment codes 1, block maxima
+        pass2_bpp = 8.0 + (2.0 if wl.grad_dtype == "bf16" else 4.0) + 1.0 + 8 / args.m_block
+        pass1_bpp = 0.0
     alg_bytes = pass2_bpp * n_params
     achieved = alg_bytes / (p2_ms * 1e-3) / 1e9
     # the captures cover the default quantizers only
-    traffic_pp = PASS2_TRAFFIC_BYTES_PER_PARAM[wl.grad_dtype] if (v_kind == "rank1" and args.m_block == 128) else None
-    roofline = {"bound": "hbm", "kernel": "pass2_kernel (update + re-quantize)", "achieved": achieved, "peak": peak,
+    traffic_pp = PASS2_TRAFFIC_BYTES_PER_PARAM[wl.grad_dtype] if (v_kind == "rank1" and args.m_block == 128 and not sgdm) else None
+    roofline = {"bound": "hbm", "kernel": "sgdm_kernel" if sgdm else "pass2_kernel (update + re-quantize)", "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                 "traffic": None if traffic_pp is None else traffic_pp * n_params,
                 "algorithmic_bytes_per_launch": alg_bytes, "ms_per_launch": p2_ms,
@@ -322,7 +337,7 @@ def run_ours(args):
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": wl.name, "tensors": len(wl.tensors), "params_per_gpu": n_params,
-                       "grad_dtype": wl.grad_dtype, "param_dtype": "f32", "m": f"B{args.m_block}/DE 4-bit", "v": {"rank1": "Rank-1/Linear 4-bit", "block": "B128/Linear 4-bit", "factored": "factorized (fp32 row/column statistics)"}[v_kind],
+                       "grad_dtype": wl.grad_dtype, "param_dtype": "f32", "m": f"B{args.m_block}/DE 4-bit", "v": {"rank1": "Rank-1/Linear 4-bit", "block": "B128/Linear 4-bit", "factored": "factorized (fp32 row/column statistics)"}[v_kind] if not sgdm else "none (compressed SGDM, Alg. 2)",
                        "l2": f"inputs larger than L2 ({(n_params * (8 + (2 if wl.grad_dtype == 'bf16' else 4) + 1)) / 1e9:.1f} GB touched per step), no flush", "parallelism": f"replicas x{world}, no collective"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu}
     print(json.dumps(line), flush=True)
