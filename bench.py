@@ -55,6 +55,14 @@ def parse_args():
     ap.add_argument("--m-block", type=int, default=128, choices=[128, 2048], help="first-moment block size")
     ap.add_argument("--v-mode", default="rank1", choices=["rank1", "block", "factored"],
                     help="second moment of matrices: rank-1 or block-wise 4-bit, or factorized (fp32 row/column statistics)")
+    ap.add_argument("--schedule", default="auto", choices=["auto", "two_pass", "fused"],
+                    help="order of the maxima and update work inside a step (lpmm_schedule)")
+    ap.add_argument("--tile-elems", type=int, default=0)
+    ap.add_argument("--tile-elems-maxima", type=int, default=0)
+    ap.add_argument("--l2-keep-mb", type=int, default=0)
+    ap.add_argument("--lead-melems", type=int, default=0)
+    ap.add_argument("--gap-items", type=int, default=0)
+    ap.add_argument("--no-l2-hints", action="store_true")
     return ap.parse_args()
 
 
@@ -215,7 +223,10 @@ def run_ours(args):
     params = [workloads.make_param(t, wl.index, i, device=dev) for i, t in enumerate(wl.tensors)]
     grads = [workloads.make_grad(t, wl.index, i, 1, device=dev, dtype=gdt) for i, t in enumerate(wl.tensors)]
     v_mode = {"rank1": lpmm.V_RANK1, "block": lpmm.V_BLOCK, "factored": lpmm.V_FACTORED}[args.v_mode]
-    cfg = lpmm.default_config(m_block=args.m_block, v_mode=v_mode)
+    schedule = {"auto": lpmm.SCHEDULE_AUTO, "two_pass": lpmm.SCHEDULE_TWO_PASS, "fused": lpmm.SCHEDULE_FUSED}[args.schedule]
+    cfg = lpmm.default_config(m_block=args.m_block, v_mode=v_mode, schedule=schedule, tile_elems=args.tile_elems,
+                              tile_elems_maxima=args.tile_elems_maxima, l2_keep_mbytes=args.l2_keep_mb,
+                              lead_melems=args.lead_melems, gap_items=args.gap_items, no_l2_hints=int(args.no_l2_hints))
     state = lpmm.state_init(cfg, wl.tensors, device=dev)
     cache = lpmm.make_ptr_cache(params, grads)
     n_params = wl.numel
@@ -237,6 +248,8 @@ def run_ours(args):
     dist.barrier()
 
     sampler = ClockSampler(local_rank) if rank == 0 else None
+    if state.schedule == lpmm.SCHEDULE_FUSED:
+        lpmm.wait_stats(state)          # clear what the warm-up left
     lpmm.profile(state, True)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
@@ -251,6 +264,7 @@ def run_ours(args):
     dist.barrier()
     clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
     prof = lpmm.profile_read(state)
+    waits = lpmm.wait_stats(state) if state.schedule == lpmm.SCHEDULE_FUSED else None
     lpmm.profile(state, False)
     launches = state.last_launches * args.steps
     ms_total = dist.max_over_ranks(ev0.elapsed_time(ev1), device=dev)
@@ -339,7 +353,7 @@ def run_ours(args):
             "config": {"workload": wl.name, "tensors": len(wl.tensors), "params_per_gpu": n_params,
                        "grad_dtype": wl.grad_dtype, "param_dtype": "f32", "m": f"B{args.m_block}/DE 4-bit", "v": {"rank1": "Rank-1/Linear 4-bit", "block": "B128/Linear 4-bit", "factored": "factorized (fp32 row/column statistics)"}[v_kind] if not sgdm else "none (compressed SGDM, Alg. 2)",
                        "l2": f"inputs larger than L2 ({(n_params * (8 + (2 if wl.grad_dtype == 'bf16' else 4) + 1)) / 1e9:.1f} GB touched per step), no flush", "parallelism": f"replicas x{world}, no collective"},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu}
+            "clocks": clocks, "waits": waits, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu}
     print(json.dumps(line), flush=True)
     dist.shutdown()
 

@@ -57,6 +57,19 @@ typedef enum { LPMM_V_RANK1 = 0, LPMM_V_BLOCK = 1, LPMM_V_FACTORED = 2 } lpmm_vm
  *   IEEE: every division and the square root correctly rounded, in the order Eq. 1 writes them. */
 typedef enum { LPMM_UPDATE_FAST = 0, LPMM_UPDATE_IEEE = 1 } lpmm_update_math;
 
+/* Order of the work inside one step (Sec. 4.2: the row and column maxima of the NEW second moment depend on the whole
+ * tensor, so every rank-1 tensor is read twice: once to reduce r', c' and once to update and re-quantize).
+ *   TWO_PASS: the maxima pass over all tensors, then the update pass over all tensors (three launches). The second read
+ *             of the gradient and the second-moment codes comes from DRAM.
+ *   FUSED:    one launch whose work list interleaves the maxima tiles of a tensor closely before its update tiles, with
+ *             L2 eviction priorities on every access, so that the second read is served by L2 where the tensor (or its
+ *             tail) fits. Needs the default quantizers (LPMM_V_RANK1, m_block 128); other states and
+ *             lpmm_adamw4_step_bf16w / lpmm_adamw4_step_host run TWO_PASS. CTAs wait for one another through
+ *             counters in the arena; every wait is bounded (see lpmm_state_device_status).
+ *   AUTO:     FUSED where it applies, else TWO_PASS.
+ * The stored states and the parameters are bit-identical under both schedules. */
+typedef enum { LPMM_SCHEDULE_AUTO = 0, LPMM_SCHEDULE_TWO_PASS = 1, LPMM_SCHEDULE_FUSED = 2 } lpmm_schedule;
+
 /* lpmm_shape.flags */
 #define LPMM_FORCE_QUANT 1u /* quantize even if numel <= min_quant_numel */
 #define LPMM_FORCE_FP32 2u  /* keep fp32 states whatever the size */
@@ -82,7 +95,15 @@ typedef struct {
     int32_t v_mode;          /* lpmm_vmode */
     int64_t min_quant_numel; /* tensors with numel <= this keep fp32 states (App. D.1: 4096) */
     int32_t update_math;     /* lpmm_update_math: arithmetic of the parameter update only */
-    int32_t reserved;        /* 0 */
+    int32_t schedule;        /* lpmm_schedule: how the two passes over a rank-1 tensor are ordered on the GPU */
+    /* Tuning of the schedules; 0 everywhere = the library's choice. None of them changes any result. */
+    int32_t tile_elems;        /* elements per tile of the update pass (a power of two, 2048 .. 4 Mi) */
+    int32_t tile_elems_maxima; /* elements per tile of the maxima pass (likewise; at least tile_elems) */
+    int32_t l2_keep_mbytes;    /* fused: MiB of gradient + second-moment codes at the end of a tensor's maxima pass that
+                                  are loaded "evict last" so that the update pass finds them in L2 */
+    int32_t lead_melems;       /* fused: Mi elements of ready update work the maxima pass stays ahead of the update pass */
+    int32_t gap_items;         /* fused: work items between a tensor's last maxima tile and its first update tile */
+    int32_t no_l2_hints;       /* fused: 1 = plain accesses without eviction priorities (to measure what the hints buy) */
 } lpmm_config;
 
 typedef struct lpmm_state lpmm_state; /* opaque host handle */
@@ -108,7 +129,14 @@ lpmm_status lpmm_state_init(const lpmm_config* cfg, const lpmm_shape* shapes, in
 
 /* Re-creates a handle over an arena that already holds states (checkpoint restore): the arena bytes
  * are a copy of an arena previously produced with the same cfg/shapes, `phase` is the value
- * lpmm_state_phase() returned when that copy was taken. Only the tensor table is rewritten. */
+ * lpmm_state_phase() returned when that copy was taken. The arena starts with a header (magic word, layout
+ * version, total size, a hash of cfg's quantizer fields and of the shapes); if it does not match what cfg/shapes
+ * describe - another library version, another parameter list, not an arena at all - the call changes nothing and
+ * returns LPMM_ERR_INVALID_ARG. Otherwise only the tensor table, the work list and the per-step scratch are
+ * rewritten. The schedule and tuning fields of cfg may differ from the original's: the states occupy the same
+ * offsets under every schedule (the fused schedule's work list lies behind them), so a copy of the first
+ * lpmm_state_bytes(original cfg) bytes restored into an arena of lpmm_state_bytes(cfg) bytes is enough.
+ * Synchronizes `stream`. */
 lpmm_status lpmm_state_attach(const lpmm_config* cfg, const lpmm_shape* shapes, int32_t n,
                               void* d_arena, size_t arena_bytes, int32_t phase, lpmm_state** out, void* stream);
 
@@ -224,16 +252,33 @@ lpmm_status lpmm_state_view(const lpmm_state* st, int32_t tensor, int32_t* kind,
  * LPMM_ERR_INVALID_ARG for tensors of another kind or an axis out of range. */
 lpmm_status lpmm_state_view_axis(const lpmm_state* st, int32_t tensor, int32_t axis, const float** mu, int64_t* extent);
 
-/* Reads the device-side error word of the state (synchronizes `stream`). 0 = no error; 1 = a bounded wait
- * for an asynchronous shared-memory copy inside a step kernel expired (the affected warp stopped early, so
- * the states written by that step are incomplete). Kernels never trap or spin without limit. */
+/* Reads the device-side error word of the state (synchronizes `stream`). 0 = no error; 2 = a CTA of the fused
+ * schedule waited for another tile's result longer than the limit (about two seconds) and stopped taking work: the
+ * states written by that step are incomplete and the arena must be re-initialised or restored from a checkpoint.
+ * Kernels never trap or spin without limit. */
 lpmm_status lpmm_state_device_status(lpmm_state* st, int32_t* status, void* stream);
 
-/* 0 or 1: which of the two rank-1 scale buffers is current. Save it with a copy of the arena. */
+/* Self-test of the bounded wait the fused schedule relies on: launches two CTAs that wait (with a limit of a few
+ * milliseconds) for a counter in the arena header that nothing ever advances. *ctas_gave_up receives how many of them
+ * ran out of patience (2), *status_word what they left in the device status word (2). The word and the counters are
+ * put back to zero afterwards, so the state stays usable. Synchronizes `stream`. */
+lpmm_status lpmm_state_selftest_wait(lpmm_state* st, int32_t* ctas_gave_up, int32_t* status_word, void* stream);
+
+/* Fused schedule: how many waits of an update tile for its tensor's maxima tiles did not succeed at the first look
+ * since the last call, and how many nanoseconds they took in all (summed over CTAs). Reads and clears the two
+ * counters; synchronizes `stream`. A tuning aid for lead_melems / gap_items. */
+lpmm_status lpmm_state_wait_stats(lpmm_state* st, int64_t* waits, int64_t* wait_ns, void* stream);
+
+/* LPMM_SCHEDULE_TWO_PASS or LPMM_SCHEDULE_FUSED: what lpmm_adamw4_step runs on this state. */
+int32_t lpmm_state_schedule(const lpmm_state* st);
+
+/* 0, 1 or 2: which of the three rank-1 scale buffers is current (they rotate: current, new, being cleared for the
+ * step after). Save it with a copy of the arena. */
 int32_t lpmm_state_phase(const lpmm_state* st);
 
 /* Optional per-kernel timing. While enabled, every lpmm_adamw4_step records CUDA events on its stream
- * around its three kernels (host-side event objects only; no device memory). */
+ * around its kernels (host-side event objects only, created by this call, none by a step; at most 256 steps are
+ * recorded between two reads). Under the fused schedule the whole launch is reported as the update pass. */
 lpmm_status lpmm_state_profile(lpmm_state* st, int32_t enable);
 
 /* Waits for the recorded steps to finish, returns the summed durations in milliseconds of the rank-1
@@ -241,8 +286,9 @@ lpmm_status lpmm_state_profile(lpmm_state* st, int32_t enable);
  * clears the record. Any output pointer may be NULL. */
 lpmm_status lpmm_state_profile_read(lpmm_state* st, double* pass1_ms, double* rcp_ms, double* pass2_ms, int32_t* steps);
 
-/* Number of kernels the last lpmm_adamw4_step on this state launched (3 when a rank-1 tensor is present,
- * else 1; one additional memset node clears the new row/column maxima). */
+/* Number of kernels the last lpmm_adamw4_step on this state launched. Two-pass schedule: 3 when a rank-1 tensor is
+ * present, else 1, and one additional memset node clears the new row/column maxima. Fused schedule: 1 (no memset
+ * node: a tensor's last update tile clears the buffer that receives the next step's maxima). */
 int32_t lpmm_state_last_launches(const lpmm_state* st);
 
 /* Frees the host handle only; the arena stays the caller's. NULL is allowed. */

@@ -1,7 +1,7 @@
 // Host side of the C ABI declared in include/lpmm.h: argument validation, arena layout, the
 // device-side tensor table and the launch sequence of one step. No device memory is allocated here.
 #include <cmath>
-#include <cstdlib>
+#include <cstddef>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -43,10 +43,40 @@ struct TensorLayout {
 struct Layout {
     std::vector<TensorLayout> t;
     size_t descs = 0, params = 0, params16 = 0, grads = 0, tiles1 = 0, tiles2 = 0, tiles3 = 0, tiles4 = 0;
-    size_t rc[2] = {0, 0}, rcp = 0;
+    size_t tsync = 0, work = 0;       // fused schedule: per-tensor progress counters, work list
+    int64_t work_items = 0;           // capacity of the work list
+    size_t rc[3] = {0, 0, 0}, rcp = 0;
     int64_t rc_floats = 0;
     size_t total = 0;
+    size_t states_end = 0;            // end of the schedule-independent part (the work list comes after it)
+    uint64_t shape_hash = 0;          // of everything the layout depends on (checked by lpmm_state_attach)
 };
+
+// The first 256 bytes of the arena: device status word, the tile counters of a launch, and a description of the
+// layout that lpmm_state_attach compares with what the caller claims the arena holds.
+constexpr uint32_t kArenaMagic = 0x4d4d504cu;    // "LPMM"
+constexpr uint32_t kArenaLayoutVersion = 2u;     // bump whenever offsets or the meaning of a region change
+struct ArenaHeader {
+    uint32_t status;          // byte 0: device status word (0 = ok)
+    uint32_t pad0[3];
+    int32_t tile_counter[2];  // byte 16: next tile of the running launch, finished CTAs
+    uint32_t pad1[2];
+    uint32_t magic;           // byte 32
+    uint32_t version;
+    uint64_t total_bytes;
+    uint64_t shape_hash;
+    int32_t n_tensors;
+    int32_t m_block;
+    int32_t v_mode;
+    int32_t pad2;
+    uint64_t pad3[7];
+    unsigned long long wait_stats[2];   // byte 128: fused schedule, {waits that had to poll, their summed nanoseconds}
+};
+static_assert(sizeof(ArenaHeader) <= 256, "header block");
+
+// Resident CTAs of the step kernels on a B200 (148 SMs x 2): the device-independent figure the tile sizes are planned
+// with, so that lpmm_state_bytes can size the work list without a device.
+constexpr int kPlanResidentCtas = 296;
 
 bool uses_rc(int32_t k) { return k == K_RANK1_FAST || k == K_RANK1_FLAT || k == K_FACT; }
 
@@ -59,6 +89,7 @@ int public_kind(int32_t k) {
 
 int32_t choose_kind(const lpmm_config& cfg, const lpmm_shape& s);
 int64_t folded_cols(const lpmm_config& cfg, int64_t numel);
+bool fused_eligible(const lpmm_config& cfg);
 
 lpmm_status validate_config(const lpmm_config* cfg, const lpmm_shape* shapes, int32_t n) {
     if (!cfg || !shapes || n <= 0) return LPMM_ERR_INVALID_ARG;
@@ -67,6 +98,13 @@ lpmm_status validate_config(const lpmm_config* cfg, const lpmm_shape* shapes, in
     if (cfg->bits != 4) return LPMM_ERR_UNSUPPORTED;
     if ((cfg->m_block != 128 && cfg->m_block != 2048) || cfg->v_block != 128) return LPMM_ERR_UNSUPPORTED;
     if (cfg->update_math != LPMM_UPDATE_FAST && cfg->update_math != LPMM_UPDATE_IEEE) return LPMM_ERR_INVALID_ARG;
+    if (cfg->schedule != LPMM_SCHEDULE_AUTO && cfg->schedule != LPMM_SCHEDULE_TWO_PASS && cfg->schedule != LPMM_SCHEDULE_FUSED)
+        return LPMM_ERR_INVALID_ARG;
+    if (cfg->schedule == LPMM_SCHEDULE_FUSED && !fused_eligible(*cfg)) return LPMM_ERR_UNSUPPORTED;
+    for (int32_t te : {cfg->tile_elems, cfg->tile_elems_maxima})
+        if (te != 0 && (te < 2048 || te > (1 << 22) || (te & (te - 1)) != 0)) return LPMM_ERR_INVALID_ARG;
+    if (cfg->l2_keep_mbytes < 0 || cfg->lead_melems < 0 || cfg->gap_items < 0) return LPMM_ERR_INVALID_ARG;
+    if (cfg->no_l2_hints != 0 && cfg->no_l2_hints != 1) return LPMM_ERR_INVALID_ARG;
     for (int32_t i = 0; i < n; ++i) {
         const lpmm_shape& s = shapes[i];
         if (s.rows <= 0 || s.cols <= 0) return LPMM_ERR_INVALID_ARG;
@@ -128,8 +166,97 @@ int32_t choose_kind(const lpmm_config& cfg, const lpmm_shape& s) {
     return (cfg.v_mode == LPMM_V_FACTORED) ? K_FACT : K_RANK1_FAST;
 }
 
+// Which schedule a state runs: the fused one needs the default quantizers (rank-1 second moments, B128 first moments).
+bool fused_eligible(const lpmm_config& cfg) { return cfg.v_mode == LPMM_V_RANK1 && cfg.m_block == 128; }
+// AUTO goes by measurement (B200): the fused launch wins where the step is bound by launch overhead (a few million
+// parameters: one launch instead of three and a memset); on larger lists its short tiles cost more than its L2 hits save.
+constexpr int64_t kAutoFusedMaxElems = (int64_t)8 << 20;
+bool wants_fused(const lpmm_config& cfg, int64_t total_elems) {
+    if (!fused_eligible(cfg)) return false;
+    if (cfg.schedule == LPMM_SCHEDULE_FUSED) return true;
+    return cfg.schedule == LPMM_SCHEDULE_AUTO && total_elems <= kAutoFusedMaxElems;
+}
+
+struct TileSizes { int64_t update, maxima; };
+
+// Elements per tile of the update pass and of the maxima pass (powers of two). Tiles are handed out on demand, so the
+// aim is >= 6 tiles per resident CTA (the tail is what is balanced). Two-pass schedule, measured optima of the update
+// pass: 32 Ki for 60-70 M parameters, 64-128 Ki for 355 M, 256 Ki for 6.7 G; the maxima pass gains from taller tiles
+// (each tile ends with a flush of its column maxima and starts with an empty load pipeline), up to 1 Mi. The fused
+// schedule wants short tiles: an update tile can only start when the tensor's last maxima tile has finished.
+TileSizes choose_tile_sizes(const lpmm_config& cfg, int64_t total_elems, bool fused) {
+    const int64_t cap2 = fused ? 32768 : 262144, cap1 = fused ? 65536 : (1 << 20);
+    const int64_t hard2 = fused ? 262144 : ((int64_t)1 << 22);   // fused: an update tile has at most 1024 rows of 256 columns
+    const int64_t target = total_elems / (6LL * kPlanResidentCtas);
+    TileSizes ts;
+    ts.update = 2048;
+    while (ts.update * 2 <= target && ts.update < cap2) ts.update *= 2;
+    if (cfg.tile_elems > 0) ts.update = cfg.tile_elems < hard2 ? cfg.tile_elems : hard2;
+    ts.maxima = ts.update;
+    while (ts.maxima * 2 <= target && ts.maxima < cap1) ts.maxima *= 2;
+    if (fused && ts.maxima < cap1 && ts.maxima * 2 <= 2 * target) ts.maxima *= 2;
+    if (cfg.tile_elems_maxima > 0) ts.maxima = cfg.tile_elems_maxima;
+    if (ts.maxima < ts.update) ts.maxima = ts.update;
+    return ts;
+}
+
+struct TilePlan {
+    int32_t wx = 0, tiles_x = 0, tile_rows = 0, tile_rows1 = 0, flat_chunks = 1;
+    int64_t tiles_update = 0;   // tiles of the update pass (tiled or element-indexed, by kind)
+    int64_t tiles_maxima = 0;   // tiles of the maxima pass (rank-1 kinds and the factorized kind; else 0)
+    int64_t tiles_flat = 0;     // element-indexed tiles (what the SGDM step uses for every tensor)
+};
+
+TilePlan plan_tensor(const lpmm_config& cfg, const TensorLayout& t, const TileSizes& ts) {
+    TilePlan p;
+    const bool tiled = t.kind == K_RANK1_FAST || t.kind == K_FACT || t.kind == K_BLOCK_TILED;
+    if (tiled) {
+        p.wx = (cfg.m_block == 2048) ? 8 : (t.cols % 1024 == 0) ? 4 : (t.cols % 512 == 0) ? 2 : 1;
+        const int64_t tile_cols = (int64_t)kWarpElems * p.wx;
+        int64_t tr = ts.update / tile_cols;
+        // at least four rows per warp: the maxima pass works in trips of four rows (shorter tiles repeat rows)
+        if (tr < 4 * (kWarps / p.wx)) tr = 4 * (kWarps / p.wx);
+        p.tile_rows = (int32_t)tr;
+        p.tiles_x = (int32_t)((t.cols + tile_cols - 1) / tile_cols);
+        p.tiles_update = (int64_t)p.tiles_x * ((t.rows + tr - 1) / tr);
+        int64_t tr1 = ts.maxima / tile_cols;
+        if (tr1 < tr) tr1 = tr;
+        p.tile_rows1 = (int32_t)tr1;
+        if (t.kind != K_BLOCK_TILED) p.tiles_maxima = (int64_t)p.tiles_x * ((t.rows + tr1 - 1) / tr1);
+    }
+    int64_t chunks = ts.update / (kWarps * kWarpElems);
+    if (chunks < 1) chunks = 1;
+    if (chunks > 16) chunks = 16;
+    p.flat_chunks = (int32_t)chunks;
+    const int64_t per_tile = chunks * kWarps * kWarpElems;
+    p.tiles_flat = (t.numel + per_tile - 1) / per_tile;
+    if (!tiled) {
+        p.tiles_update = p.tiles_flat;
+        if (t.kind == K_RANK1_FLAT) p.tiles_maxima = p.tiles_flat;
+    }
+    return p;
+}
+
+uint64_t fnv1a(uint64_t h, const void* data, size_t bytes) {
+    const unsigned char* p = static_cast<const unsigned char*>(data);
+    for (size_t i = 0; i < bytes; ++i) { h ^= p[i]; h *= 1099511628211ull; }
+    return h;
+}
+
 void compute_layout(const lpmm_config& cfg, const lpmm_shape* shapes, int32_t n, Layout* L) {
     L->t.resize(n);
+    {
+        uint64_t h = 1469598103934665603ull;
+        const int64_t c[5] = {cfg.bits, cfg.m_block, cfg.v_block, cfg.v_mode, cfg.min_quant_numel};
+        h = fnv1a(h, c, sizeof(c));
+        for (int32_t i = 0; i < n; ++i) {
+            const lpmm_shape& s = shapes[i];
+            const int64_t v[4] = {s.rows, s.cols, s.ndim, (int64_t)s.flags};
+            h = fnv1a(h, v, sizeof(v));
+            if (s.ndim >= 3) h = fnv1a(h, s.dims, sizeof(int64_t) * s.ndim);
+        }
+        L->shape_hash = h;
+    }
     size_t off = kAlign;  // header block
     L->descs = off;  off = align_up(off + sizeof(TensorDesc) * n);
     L->params = off; off = align_up(off + sizeof(void*) * n);
@@ -139,6 +266,7 @@ void compute_layout(const lpmm_config& cfg, const lpmm_shape* shapes, int32_t n,
     L->tiles2 = off; off = align_up(off + sizeof(int32_t) * (n + 1));
     L->tiles3 = off; off = align_up(off + sizeof(int32_t) * (n + 1));
     L->tiles4 = off; off = align_up(off + sizeof(int32_t) * (n + 1));
+    L->tsync = off;  off = align_up(off + sizeof(TensorSync) * n);
     int64_t rc = 0;
     for (int32_t i = 0; i < n; ++i) {
         TensorLayout& t = L->t[i];
@@ -172,6 +300,7 @@ void compute_layout(const lpmm_config& cfg, const lpmm_shape* shapes, int32_t n,
     L->rc_floats = rc;
     L->rc[0] = off; off = align_up(off + sizeof(float) * rc);
     L->rc[1] = off; off = align_up(off + sizeof(float) * rc);
+    L->rc[2] = off; off = align_up(off + sizeof(float) * rc);
     L->rcp = off;   off = align_up(off + sizeof(float) * rc);
     for (int32_t i = 0; i < n; ++i) {
         TensorLayout& t = L->t[i];
@@ -187,6 +316,19 @@ void compute_layout(const lpmm_config& cfg, const lpmm_shape* shapes, int32_t n,
             t.m_scale = off; off = align_up(off + sizeof(float) * nblk_m);
             if (t.kind == K_BLOCK || t.kind == K_BLOCK_TILED) { t.v_bscale = off; off = align_up(off + sizeof(float) * nblk); }
         }
+    }
+    L->states_end = off;   // everything a checkpoint must keep lies below this offset
+    int64_t total_elems = 0;
+    for (int32_t i = 0; i < n; ++i) total_elems += L->t[i].numel;
+    if (wants_fused(cfg, total_elems)) {   // the work list: one item per tile of either pass
+        const TileSizes ts = choose_tile_sizes(cfg, total_elems, true);
+        int64_t items = 0;
+        for (int32_t i = 0; i < n; ++i) {
+            const TilePlan p = plan_tensor(cfg, L->t[i], ts);
+            items += p.tiles_update + p.tiles_maxima;
+        }
+        L->work_items = items;
+        L->work = off; off = align_up(off + sizeof(uint2) * (size_t)items);
     }
     L->total = off;
 }
@@ -209,17 +351,87 @@ struct lpmm_state {
     bool params_a32 = false, grads_a32 = false;   // all current parameter / gradient pointers are 32-byte aligned
     size_t stage_bytes;
     std::vector<size_t> stage_off;
-    int32_t pass2_variant;                 // 0 = register prefetch, 1 = bulk-copy staging
+    bool fused = false;                    // the state runs the fused schedule (one launch per step)
+    int32_t work_total = 0;                // items of the work list
+    bool new_rc_clean = false;             // the scale buffer that receives the next step's maxima is known to be zero
+    uint32_t epoch = 0;                    // fused launches made on this state (the per-tensor counters count along)
     int32_t sms, occ1, occ2;
     int32_t p1_ctas;                       // which instantiation of the maxima pass (2 or 3 CTAs per SM)
     std::vector<int32_t> tiles1, tiles2, tiles3;   // host copies of the tile prefix sums (3: element-indexed tiles of every tensor)
     cudaStream_t copy_in, copy_out;        // lazily created by the host-buffer entry point
     std::vector<cudaEvent_t> host_events;
     bool profile;                          // record events around each kernel of a step
-    std::vector<cudaEvent_t> prof_events;  // 4 per recorded step: start, after pass 1, after rcp, after pass 2
+    std::vector<cudaEvent_t> prof_events;  // ring of 4 per recorded step: start, after pass 1, after rcp, after pass 2
+    size_t prof_used = 0;                  // events of the ring in use since the last read
 };
 
 namespace {
+
+constexpr size_t kProfRingSteps = 256;     // steps that can be recorded between two reads
+
+// The work list of the fused schedule, built by a small simulation of the hand-out. Two streams are merged: the
+// maxima tiles of the rank-1 tensors in table order, and the update tiles of the same tensors in the same order (inside
+// a tensor: last rows first - the maxima pass read them last, so they are the likeliest to be in L2).
+//   - An update tile may only be listed once its tensor's maxima tiles are all listed, and then at least `gap` items
+//     later, so that the maxima tiles still running when it is handed out have time to finish (else the CTA waits).
+//   - The maxima stream runs ahead until `lead` elements of update work are ready, and no further: what it has read
+//     should still be in L2 when the update pass comes for it. While both streams have something to list they alternate.
+//   - A maxima tile is flagged "keep" when it lies in the last `keep` bytes (gradient + codes) of its tensor's maxima
+//     pass: only what can still be in L2 when the update pass arrives asks for it.
+// The update tiles of everything else (fp32 and block-wise tensors: no dependencies) come last.
+void build_work_list(const lpmm_state* st, const std::vector<TilePlan>& plans, std::vector<uint2>* work) {
+    const lpmm_config& cfg = st->cfg;
+    const int32_t n = st->n;
+    std::vector<int32_t> rank1;
+    for (int32_t i = 0; i < n; ++i)
+        if (plans[i].tiles_maxima > 0) rank1.push_back(i);
+    const int64_t keep_bytes = (cfg.l2_keep_mbytes > 0 ? (int64_t)cfg.l2_keep_mbytes : 48) << 20;
+    const int64_t lead_elems = (cfg.lead_melems > 0 ? (int64_t)cfg.lead_melems : 10) << 20;
+    const int64_t gap = cfg.gap_items > 0 ? cfg.gap_items : kPlanResidentCtas / 2;
+    work->clear();
+    auto tile_elems1 = [&](int32_t t) {
+        const TilePlan& p = plans[t];
+        return (p.wx > 0) ? (int64_t)p.tile_rows1 * kWarpElems * p.wx : (int64_t)p.flat_chunks * kWarps * kWarpElems;
+    };
+    size_t k1 = 0, k2 = 0;             // tensors (positions in rank1) the two streams are at
+    int64_t i1 = 0, i2 = 0;            // next tile inside them
+    int64_t ready = 0;                 // elements of update work whose maxima tiles are all listed
+    std::vector<int64_t> complete_at(rank1.size(), -1);   // list position of a tensor's last maxima tile
+    bool turn_update = true;
+    while (k1 < rank1.size() || k2 < rank1.size()) {
+        const bool have1 = k1 < rank1.size();
+        const bool want1 = have1 && ready < lead_elems;
+        bool can2 = k2 < rank1.size() && complete_at[k2] >= 0;
+        if (can2 && i2 == 0 && (int64_t)work->size() - complete_at[k2] < gap && have1) can2 = false;   // too early (unless nothing else is left)
+        bool emit_update;
+        if (want1 && can2) { emit_update = turn_update; turn_update = !turn_update; }
+        else if (want1) emit_update = false;
+        else if (can2) emit_update = true;
+        else emit_update = !have1;     // neither wanted nor allowed: run the maxima stream further ahead if it has anything
+        if (emit_update) {
+            const int32_t t = rank1[k2];
+            const int64_t n2 = plans[t].tiles_update;
+            work->push_back(make_uint2((uint32_t)t | kWorkUpdate, (uint32_t)(n2 - 1 - i2)));
+            ready -= st->L.t[t].numel / n2;
+            if (++i2 == n2) { ++k2; i2 = 0; }
+        } else {
+            const int32_t t = rank1[k1];
+            const int64_t n1 = plans[t].tiles_maxima;
+            // bytes of gradient (counted at 2 per element) and codes from this tile to the end of the tensor's pass
+            const int64_t after = (n1 - i1) * tile_elems1(t) * 5 / 2;
+            work->push_back(make_uint2((uint32_t)t | (after <= keep_bytes ? kWorkKeep : 0u), (uint32_t)i1));
+            if (++i1 == n1) {
+                complete_at[k1] = (int64_t)work->size() - 1;
+                ready += st->L.t[t].numel;
+                ++k1; i1 = 0;
+            }
+        }
+    }
+    for (int32_t i = 0; i < n; ++i) {
+        if (plans[i].tiles_maxima > 0 || st->L.t[i].kind == K_BLOCK_TILED) continue;
+        for (int64_t j = 0; j < plans[i].tiles_update; ++j) work->push_back(make_uint2((uint32_t)i | kWorkUpdate, (uint32_t)j));
+    }
+}
 
 // Fills descriptors and tile tables, and uploads them. Tile sizes adapt to the amount of work so that
 // small parameter sets still spread over the whole GPU.
@@ -242,30 +454,11 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
     const int32_t n = st->n;
     int64_t total_elems = 0;
     for (int32_t i = 0; i < n; ++i) total_elems += st->L.t[i].numel;
-    // aim at >= 6 tiles per resident CTA of the update pass (tiles are handed out on demand, the tail is what is
-    // balanced), tiles between 2 Ki and 256 Ki elements (powers of two). Measured optima: 32 Ki for 60-70 M
-    // parameters, 64-128 Ki for 355 M, 256 Ki for 6.7 G.
-    int64_t target = total_elems / (6LL * sms * occ2);
-    int64_t tile_elems = 2048;
-    while (tile_elems * 2 <= target && tile_elems < 262144) tile_elems *= 2;
-    if (const char* v = std::getenv("LPMM_TILE_ELEMS")) {   // development switch
-        const long x = std::atol(v);
-        if (x >= 2048 && x <= (1 << 20)) tile_elems = x;
-    }
-    // The maxima pass gets its own, taller tiles (same width): every tile ends with a flush of its column maxima and
-    // starts with an empty load pipeline, so it gains up to 1 Mi elements (3.92 -> 3.72 ms on the 6.7 G list) where
-    // the update pass is best at 256 Ki.
-    int64_t tile_elems1 = tile_elems;
-    {
-        const int64_t target1 = total_elems / (6LL * sms * occ1);
-        while (tile_elems1 * 2 <= target1 && tile_elems1 < (1 << 20)) tile_elems1 *= 2;
-        if (const char* v = std::getenv("LPMM_TILE_ELEMS1")) {   // development switch
-            const long x = std::atol(v);
-            if (x >= tile_elems && x <= (1 << 22)) tile_elems1 = x;
-        }
-    }
+    st->fused = wants_fused(st->cfg, total_elems) && st->L.work_items > 0 && st->L.work_items <= 0x7fffffffLL;
+    const TileSizes ts = choose_tile_sizes(st->cfg, total_elems, st->fused);
 
     std::vector<TensorDesc> descs(n);
+    std::vector<TilePlan> plans(n);
     std::vector<int32_t> t1(n + 1, 0), t2(n + 1, 0), t3(n + 1, 0), t4(n + 1, 0);
     // In a state whose matrices are not block-wise, folded 1-D tensors leave the main update launch (0 tiles there)
     // and get one of their own with the block-wise kernel (table 4).
@@ -279,7 +472,6 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
         d.n_outer = t.n_outer;
         for (int a = 0; a < 3; ++a) { d.outer_dim[a] = t.outer_dim[a]; d.outer_off[a] = t.outer_off[a]; }
         d.m_shift = (st->cfg.m_block == 2048) ? 11 : 7;
-        int64_t tiles = 0, tiles_p1 = 0;
         if (t.kind == K_FP32) {
             d.m32 = reinterpret_cast<float*>(A + t.m32);
             d.v32 = reinterpret_cast<float*>(A + t.v32);
@@ -291,41 +483,26 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
             if (uses_rc(t.kind)) {
                 d.rc[0] = reinterpret_cast<float*>(A + st->L.rc[0]) + t.rc_index;
                 d.rc[1] = reinterpret_cast<float*>(A + st->L.rc[1]) + t.rc_index;
+                d.rc[2] = reinterpret_cast<float*>(A + st->L.rc[2]) + t.rc_index;
                 d.rcp_new = reinterpret_cast<float*>(A + st->L.rcp) + t.rc_index;
+                d.rc_floats = (int32_t)(t.c_off + (t.cols + 3) / 4 * 4);
             }
         }
-        if (t.kind == K_RANK1_FAST || t.kind == K_FACT || t.kind == K_BLOCK_TILED) {
-            d.wx = (st->cfg.m_block == 2048) ? 8 : (t.cols % 1024 == 0) ? 4 : (t.cols % 512 == 0) ? 2 : 1;
-            const int64_t tile_cols = (int64_t)kWarpElems * d.wx;
-            int64_t tr = tile_elems / tile_cols;
-            // at least four rows per warp: the maxima pass works in trips of four rows (shorter tiles repeat rows)
-            if (tr < 4 * (kWarps / d.wx)) tr = 4 * (kWarps / d.wx);
-            d.tile_rows = (int32_t)tr;
-            d.tiles_x = (int32_t)((t.cols + tile_cols - 1) / tile_cols);
-            tiles = (int64_t)d.tiles_x * ((t.rows + tr - 1) / tr);
-            int64_t tr1 = tile_elems1 / tile_cols;
-            if (tr1 < tr) tr1 = tr;
-            d.tile_rows1 = (int32_t)tr1;
-            tiles_p1 = (int64_t)d.tiles_x * ((t.rows + tr1 - 1) / tr1);
-        }
-        {   // element-indexed tiling: used by the non-tiled kinds in pass 2 and by every tensor in the SGDM step
-            int64_t chunks = tile_elems / (kWarps * kWarpElems);
-            if (chunks < 1) chunks = 1;
-            if (chunks > 16) chunks = 16;
-            d.flat_chunks = (int32_t)chunks;
-            const int64_t per_tile = chunks * kWarps * kWarpElems;
-            const int64_t flat_tiles = (t.numel + per_tile - 1) / per_tile;
-            if (t.kind != K_RANK1_FAST && t.kind != K_FACT && t.kind != K_BLOCK_TILED) tiles = flat_tiles;
-            if (t3[i] + flat_tiles > 0x7fffffffLL) return LPMM_ERR_UNSUPPORTED;
-            t3[i + 1] = t3[i] + (int32_t)flat_tiles;
-        }
-        if (t2[i] + tiles > 0x7fffffffLL) return LPMM_ERR_UNSUPPORTED;
+        const TilePlan p = plan_tensor(st->cfg, t, ts);
+        plans[i] = p;
+        d.wx = p.wx; d.tiles_x = p.tiles_x; d.tile_rows = p.tile_rows; d.tile_rows1 = p.tile_rows1;
+        d.flat_chunks = p.flat_chunks;
+        if (p.tiles_update > 0x7fffffffLL || p.tiles_maxima > 0x7fffffffLL || p.tiles_flat > 0x7fffffffLL) return LPMM_ERR_UNSUPPORTED;
+        d.tiles1 = (int32_t)p.tiles_maxima;
+        d.tiles2 = (int32_t)p.tiles_update;
+        if (t3[i] + p.tiles_flat > 0x7fffffffLL) return LPMM_ERR_UNSUPPORTED;
+        t3[i + 1] = t3[i] + (int32_t)p.tiles_flat;
+        if (t2[i] + p.tiles_update > 0x7fffffffLL) return LPMM_ERR_UNSUPPORTED;
         const bool moved = own_launch && t.kind == K_BLOCK_TILED;
-        t2[i + 1] = t2[i] + (moved ? 0 : (int32_t)tiles);
-        t4[i + 1] = t4[i] + (moved ? (int32_t)tiles : 0);
-        const bool rank1 = uses_rc(t.kind);
-        const bool tiled = (t.kind == K_RANK1_FAST || t.kind == K_FACT);
-        t1[i + 1] = t1[i] + (rank1 ? (int32_t)(tiled ? tiles_p1 : tiles) : 0);
+        t2[i + 1] = t2[i] + (moved ? 0 : (int32_t)p.tiles_update);
+        t4[i + 1] = t4[i] + (moved ? (int32_t)p.tiles_update : 0);
+        if (t1[i] + p.tiles_maxima > 0x7fffffffLL) return LPMM_ERR_UNSUPPORTED;
+        t1[i + 1] = t1[i] + (int32_t)p.tiles_maxima;
     }
     st->total1 = t1[n];
     st->total2 = t2[n];
@@ -336,6 +513,14 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
     st->tiles2 = t2;
     st->tiles3 = t3;
     st->tiles4 = t4;
+    if (st->fused) {
+        std::vector<uint2> work;
+        build_work_list(st, plans, &work);
+        if ((int64_t)work.size() > st->L.work_items) return LPMM_ERR_ARENA_TOO_SMALL;   // cannot happen: same plan as the layout
+        st->work_total = (int32_t)work.size();
+        LPMM_CUDA(cudaMemcpyAsync(A + st->L.work, work.data(), sizeof(uint2) * work.size(), cudaMemcpyHostToDevice, s));
+        LPMM_CUDA(cudaStreamSynchronize(s));   // `work` is about to go out of scope
+    }
     LPMM_CUDA(cudaMemcpyAsync(A + st->L.tiles4, t4.data(), sizeof(int32_t) * (n + 1), cudaMemcpyHostToDevice, s));
     LPMM_CUDA(cudaMemcpyAsync(A + st->L.tiles3, t3.data(), sizeof(int32_t) * (n + 1), cudaMemcpyHostToDevice, s));
     LPMM_CUDA(cudaMemcpyAsync(A + st->L.descs, descs.data(), sizeof(TensorDesc) * n, cudaMemcpyHostToDevice, s));
@@ -353,7 +538,7 @@ lpmm_status make_state(const lpmm_config* cfg, const lpmm_shape* shapes, int32_t
     if (v != LPMM_OK) return v;
     if (!d_arena) return LPMM_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(d_arena) % kAlign != 0) return LPMM_ERR_ALIGNMENT;
-    if (phase != 0 && phase != 1) return LPMM_ERR_INVALID_ARG;
+    if (phase < 0 || phase > 2) return LPMM_ERR_INVALID_ARG;
     lpmm_state* st = new (std::nothrow) lpmm_state();
     if (!st) return LPMM_ERR_INVALID_ARG;
     st->cfg = *cfg;
@@ -367,10 +552,6 @@ lpmm_status make_state(const lpmm_config* cfg, const lpmm_shape* shapes, int32_t
     st->profile = false;
     st->copy_in = nullptr;
     st->copy_out = nullptr;
-    {
-        const char* v = std::getenv("LPMM_PASS2_VARIANT");   // development switch
-        st->pass2_variant = (v && v[0] == '1') ? 1 : 0;
-    }
     st->ptrs_valid = false;
     st->params.assign(n, nullptr);
     st->grads.assign(n, nullptr);
@@ -393,10 +574,43 @@ lpmm_status make_state(const lpmm_config* cfg, const lpmm_shape* shapes, int32_t
                 e = cudaMemsetAsync(st->arena + t.m_codes + t.numel / 2, 0x07, 1, s);
         }
         if (e != cudaSuccess) rc = cuda_fail(e);
-    } else {   // an attached arena keeps its states; the header block (status word, tile counters) starts clean
-        const cudaError_t e = cudaMemsetAsync(d_arena, 0, kAlign, s);
+    } else {
+        // An attached arena must describe itself as what the caller says it is ...
+        ArenaHeader hd;
+        cudaError_t e = cudaMemcpyAsync(&hd, d_arena, sizeof(hd), cudaMemcpyDeviceToHost, s);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+        if (e != cudaSuccess) {
+            rc = cuda_fail(e);
+        } else if (hd.magic != kArenaMagic || hd.version != kArenaLayoutVersion || hd.total_bytes != st->L.states_end ||
+                   hd.shape_hash != st->L.shape_hash || hd.n_tensors != n || hd.m_block != cfg->m_block ||
+                   hd.v_mode != cfg->v_mode) {
+            rc = LPMM_ERR_INVALID_ARG;
+        } else {
+            // ... and keeps its states; the status word, the tile counters, the progress counters and the scale buffer
+            // that receives the next step's maxima start clean.
+            e = cudaMemsetAsync(d_arena, 0, 32, s);
+            if (e == cudaSuccess) e = cudaMemsetAsync(st->arena + offsetof(ArenaHeader, wait_stats), 0, 16, s);
+            if (e == cudaSuccess) e = cudaMemsetAsync(st->arena + st->L.tsync, 0, sizeof(TensorSync) * n, s);
+            for (int k = 1; k <= 2 && e == cudaSuccess && st->L.rc_floats > 0; ++k)
+                e = cudaMemsetAsync(st->arena + st->L.rc[(phase + k) % 3], 0, sizeof(float) * (size_t)st->L.rc_floats, s);
+            if (e != cudaSuccess) rc = cuda_fail(e);
+        }
+    }
+    if (rc == LPMM_OK && fresh) {
+        ArenaHeader hd;
+        std::memset(&hd, 0, sizeof(hd));
+        hd.magic = kArenaMagic; hd.version = kArenaLayoutVersion; hd.total_bytes = st->L.states_end;
+        hd.shape_hash = st->L.shape_hash; hd.n_tensors = n; hd.m_block = cfg->m_block; hd.v_mode = cfg->v_mode;
+        const cudaError_t e = cudaMemcpyAsync(d_arena, &hd, sizeof(hd), cudaMemcpyHostToDevice, s);   // pageable: staged before return
         if (e != cudaSuccess) rc = cuda_fail(e);
     }
+    st->new_rc_clean = true;
+#ifdef LPMM_EXP_SETASIDE
+    if (rc == LPMM_OK) {   // experiment: an L2 set-aside for "evict last" lines
+        const cudaError_t e = cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, (size_t)LPMM_EXP_SETASIDE << 20);
+        if (e != cudaSuccess) rc = cuda_fail(e);
+    }
+#endif
     if (rc == LPMM_OK) rc = build_tables(st, s);
     if (rc != LPMM_OK) { delete st; return rc; }
     *out = st;
@@ -404,6 +618,10 @@ lpmm_status make_state(const lpmm_config* cfg, const lpmm_shape* shapes, int32_t
 }
 
 bool finite_nonneg(float x) { return std::isfinite(x) && x >= 0.0f; }
+
+// Polls of a device-side wait before it gives up (each poll is an L2 round trip plus a short sleep: about two
+// seconds in all, far beyond any legitimate wait, which is bounded by the duration of one tile).
+constexpr uint32_t kSpinLimit = 1u << 22;
 
 }  // namespace
 
@@ -475,8 +693,15 @@ StepArgs make_args(const lpmm_state* st, float lr, float beta1, float beta2, flo
     a.params_bf16 = nullptr;
     a.grads = reinterpret_cast<const void* const*>(st->arena + st->L.grads);
     a.n_tensors = st->n;
-    a.phase = st->phase;
-    a.variant = st->pass2_variant;
+    a.sel.old_i = st->phase;
+    a.sel.new_i = (st->phase + 1) % 3;
+    a.sel.zero_i = (st->phase + 2) % 3;
+    a.epoch = 0;
+    a.l2_hints = st->cfg.no_l2_hints ? 0 : 1;
+    a.wait_stats = reinterpret_cast<unsigned long long*>(st->arena + offsetof(ArenaHeader, wait_stats));
+    a.work = reinterpret_cast<const uint2*>(st->arena + st->L.work);
+    a.tsync = reinterpret_cast<TensorSync*>(st->arena + st->L.tsync);
+    a.spin_limit = kSpinLimit;
     a.aligned32 = 0;   // set by the callers that know the gradient type
     a.dev_status = reinterpret_cast<uint32_t*>(st->arena);
     a.tile_counter = reinterpret_cast<int32_t*>(st->arena + 16);   // header block: [status | .. | counters]
@@ -520,7 +745,7 @@ lpmm_status enqueue_range(lpmm_state* st, StepArgs a, int32_t t0, int32_t t1, bo
             if (rc_begin < 0) rc_begin = t.rc_index;
             rc_end = (t.rc_index + t.c_off + (t.cols + 3) / 4 * 4 + 63) / 64 * 64;
         }
-        float* rc_new = reinterpret_cast<float*>(st->arena + st->L.rc[st->phase ^ 1]) + rc_begin;
+        float* rc_new = reinterpret_cast<float*>(st->arena + st->L.rc[(st->phase + 1) % 3]) + rc_begin;
         LPMM_CUDA(cudaMemsetAsync(rc_new, 0, sizeof(float) * (size_t)(rc_end - rc_begin), s));
         if (ev) LPMM_CUDA(cudaEventRecord(ev[0], s));
         a.tile_start = reinterpret_cast<const int32_t*>(st->arena + st->L.tiles1);
@@ -593,18 +818,42 @@ lpmm_status adamw4_step_impl(lpmm_state* st, void* const* d_params, void* const*
     }
     StepArgs a = make_args(st, lr, beta1, beta2, eps, weight_decay, step);
     if (d_params16) a.params_bf16 = reinterpret_cast<uint16_t* const*>(st->arena + st->L.params16);
-    cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
-    if (st->profile) {
-        for (int k = 0; k < 4; ++k) {
-            LPMM_CUDA(cudaEventCreate(&ev[k]));
-            st->prof_events.push_back(ev[k]);
-        }
+    // Per-kernel timing: the next four events of the ring made by lpmm_state_profile (a full ring records nothing more).
+    cudaEvent_t* ev = nullptr;
+    if (st->profile && st->prof_used + 4 <= st->prof_events.size()) {
+        ev = &st->prof_events[st->prof_used];
+        st->prof_used += 4;
     }
     const bool ieee_update = wants_ieee_update(st, a.h);
+    const bool bf16 = grad_dtype == LPMM_BF16;
     int32_t launches = 0;
-    rc = enqueue_range(st, a, 0, st->n, grad_dtype == LPMM_BF16, ieee_update, s, st->profile ? ev : nullptr, &launches);
-    if (rc != LPMM_OK) return rc;
-    st->phase ^= 1;
+    if (st->fused && !d_params16) {
+        // One launch over the work list: maxima tiles and update tiles of every tensor, ordered by counters in the arena.
+        if (!st->new_rc_clean && st->L.rc_floats > 0)
+            LPMM_CUDA(cudaMemsetAsync(st->arena + st->L.rc[(st->phase + 1) % 3], 0, sizeof(float) * (size_t)st->L.rc_floats, s));
+        a.aligned32 = (st->params_a32 && (bf16 || st->grads_a32)) ? 1 : 0;
+        a.tile_begin = 0;
+        a.tile_end = st->work_total;
+        a.tile_start = nullptr;
+        a.epoch = ++st->epoch;
+        if (ev) { LPMM_CUDA(cudaEventRecord(ev[0], s)); LPMM_CUDA(cudaEventRecord(ev[1], s)); LPMM_CUDA(cudaEventRecord(ev[2], s)); }
+        const int32_t cap = st->sms * st->occ2;
+        LPMM_CUDA(launch_fused(a, bf16, ieee_update, st->work_total < cap ? st->work_total : cap, s));
+        launches = 1;
+        if (st->tiles4[st->n] > 0) {   // folded 1-D tensors: the block-wise form of the tiled update kernel
+            a.tile_start = reinterpret_cast<const int32_t*>(st->arena + st->L.tiles4);
+            a.tile_end = st->tiles4[st->n];
+            LPMM_CUDA(launch_pass2(a, bf16, ieee_update, 7, 2, a.tile_end < cap ? a.tile_end : cap, s));
+            launches += 1;
+        }
+        if (ev) LPMM_CUDA(cudaEventRecord(ev[3], s));
+        st->new_rc_clean = true;       // the maxima tiles have cleared the buffer the next step reduces into
+    } else {
+        rc = enqueue_range(st, a, 0, st->n, bf16, ieee_update, s, ev, &launches);
+        if (rc != LPMM_OK) return rc;
+        st->new_rc_clean = false;
+    }
+    st->phase = (st->phase + 1) % 3;
     st->last_launches = launches;
     return LPMM_OK;
 }
@@ -722,7 +971,8 @@ lpmm_status lpmm_adamw4_step_host(lpmm_state* st, void* const* h_params, const v
     }
     LPMM_CUDA(cudaEventRecord(ev_end, st->copy_out));
     LPMM_CUDA(cudaStreamWaitEvent(s, ev_end, 0));                  // the caller's stream ends after the last copy-out
-    st->phase ^= 1;
+    st->new_rc_clean = false;
+    st->phase = (st->phase + 1) % 3;
     st->last_launches = launches;
     return LPMM_OK;
 }
@@ -807,6 +1057,13 @@ lpmm_status lpmm_state_view_axis(const lpmm_state* st, int32_t tensor, int32_t a
 
 lpmm_status lpmm_state_profile(lpmm_state* st, int32_t enable) {
     if (!st) return LPMM_ERR_INVALID_ARG;
+    if (enable) {   // the events are made here, once, so that a recorded step creates nothing
+        while (st->prof_events.size() < 4 * kProfRingSteps) {
+            cudaEvent_t e;
+            LPMM_CUDA(cudaEventCreate(&e));
+            st->prof_events.push_back(e);
+        }
+    }
     st->profile = (enable != 0);
     return LPMM_OK;
 }
@@ -814,7 +1071,7 @@ lpmm_status lpmm_state_profile(lpmm_state* st, int32_t enable) {
 lpmm_status lpmm_state_profile_read(lpmm_state* st, double* pass1_ms, double* rcp_ms, double* pass2_ms, int32_t* steps) {
     if (!st) return LPMM_ERR_INVALID_ARG;
     double t[3] = {0.0, 0.0, 0.0};
-    const size_t n = st->prof_events.size() / 4;
+    const size_t n = st->prof_used / 4;
     lpmm_status rc = LPMM_OK;
     for (size_t i = 0; i < n && rc == LPMM_OK; ++i) {
         cudaEvent_t* e = &st->prof_events[4 * i];
@@ -826,8 +1083,7 @@ lpmm_status lpmm_state_profile_read(lpmm_state* st, double* pass1_ms, double* rc
         }
         if (err != cudaSuccess) rc = cuda_fail(err);
     }
-    for (cudaEvent_t e : st->prof_events) cudaEventDestroy(e);
-    st->prof_events.clear();
+    st->prof_used = 0;
     if (pass1_ms) *pass1_ms = t[0];
     if (rcp_ms) *rcp_ms = t[1];
     if (pass2_ms) *pass2_ms = t[2];
@@ -845,7 +1101,39 @@ lpmm_status lpmm_state_device_status(lpmm_state* st, int32_t* status, void* stre
     return LPMM_OK;
 }
 
+lpmm_status lpmm_state_selftest_wait(lpmm_state* st, int32_t* ctas_gave_up, int32_t* status_word, void* stream) {
+    if (!st || !ctas_gave_up || !status_word) return LPMM_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    ArenaHeader* hd = reinterpret_cast<ArenaHeader*>(st->arena);
+    // pad1[0] counts the CTAs that gave up; pad1[1] is the flag they wait on, which nothing ever sets
+    LPMM_CUDA(cudaMemsetAsync(hd->pad1, 0, sizeof(hd->pad1), s));
+    LPMM_CUDA(launch_wait_selftest(&hd->pad1[1], 1u, 2000u, &hd->status,
+                                   reinterpret_cast<int32_t*>(&hd->pad1[0]), s));
+    uint32_t words[8] = {0};
+    LPMM_CUDA(cudaMemcpyAsync(words, st->arena, sizeof(words), cudaMemcpyDeviceToHost, s));
+    LPMM_CUDA(cudaStreamSynchronize(s));
+    *status_word = (int32_t)words[0];
+    *ctas_gave_up = (int32_t)words[6];
+    LPMM_CUDA(cudaMemsetAsync(st->arena, 0, 32, s));     // the state stays usable: status word and counters back to zero
+    return LPMM_OK;
+}
+
+lpmm_status lpmm_state_wait_stats(lpmm_state* st, int64_t* waits, int64_t* wait_ns, void* stream) {
+    if (!st || !waits || !wait_ns) return LPMM_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    unsigned long long w[2] = {0, 0};
+    char* p = st->arena + offsetof(ArenaHeader, wait_stats);
+    LPMM_CUDA(cudaMemcpyAsync(w, p, sizeof(w), cudaMemcpyDeviceToHost, s));
+    LPMM_CUDA(cudaStreamSynchronize(s));
+    LPMM_CUDA(cudaMemsetAsync(p, 0, sizeof(w), s));
+    *waits = (int64_t)w[0];
+    *wait_ns = (int64_t)w[1];
+    return LPMM_OK;
+}
+
 int32_t lpmm_state_phase(const lpmm_state* st) { return st ? st->phase : -1; }
+
+int32_t lpmm_state_schedule(const lpmm_state* st) { return st ? (st->fused ? LPMM_SCHEDULE_FUSED : LPMM_SCHEDULE_TWO_PASS) : -1; }
 
 int32_t lpmm_state_last_launches(const lpmm_state* st) { return st ? st->last_launches : 0; }
 

@@ -25,7 +25,8 @@ struct TensorDesc {
     float* m_scale;     // ceil(numel / m_block) block maxima of |m|
     uint8_t* v_codes;
     float* v_bscale;    // K_BLOCK: ceil(numel/128) block maxima of v
-    float* rc[2];       // K_RANK1_*: two buffers of [r (rows, padded to 4) | c (cols)]; K_FACT: [R | C] statistics
+    float* rc[3];       // K_RANK1_*: three buffers of [r (rows, padded to 4) | c (cols)] that rotate from step to step
+                        // (current, new, being cleared for the step after); K_FACT: [R | C] statistics
     float* rcp_new;     // K_RANK1_*: reciprocals of the new r, c (same layout), per-step scratch; K_FACT: R_i / sum(R)
     float* m32;         // K_FP32
     float* v32;
@@ -44,7 +45,30 @@ struct TensorDesc {
     int32_t outer_dim[3];
     int32_t outer_off[3];
     int32_t tile_rows1; // K_RANK1_FAST: rows per tile of the maxima pass (at least tile_rows; same tile width)
+    int32_t tiles1;     // rank-1 kinds: tiles of the maxima pass
+    int32_t tiles2;     // tiles of the update pass
+    int32_t rc_floats;  // rank-1 kinds: floats of this tensor's share of rc[] / rcp_new (c_off + cols rounded up to 4)
 };
+
+// Fused schedule: progress of one tensor. The counter is never reset: launch number e (1, 2, ...) of a state waits for
+// e * tiles1, modulo 2^32.
+struct TensorSync {
+    uint32_t maxima_done;  // finished tiles of the maxima pass, summed over all launches
+    uint32_t ready;        // element-indexed tensors: the last launch whose new reciprocals are in place
+};
+
+// Which of a tensor's three scale buffers is which in this step.
+struct RcSel {
+    int32_t old_i;    // current r, c (read)
+    int32_t new_i;    // receives the new r', c' (all zero when the step starts)
+    int32_t zero_i;   // fused schedule: cleared during this step, becomes new_i of the next one
+};
+
+// Fused schedule: one item of the work list = one tile. x = tensor index | flags, y = tile number inside the
+// tensor's pass (the maxima pass and the update pass have tilings of their own).
+constexpr uint32_t kWorkTensorMask = 0x0fffffffu;
+constexpr uint32_t kWorkUpdate = 0x40000000u;   // a tile of the update pass (else: of the maxima pass)
+constexpr uint32_t kWorkKeep = 0x80000000u;     // maxima pass: load this tile so that it stays in L2 for the update pass
 
 struct StepArgs {
     const TensorDesc* descs;
@@ -54,8 +78,13 @@ struct StepArgs {
     const int32_t* tile_start;   // n + 1 prefix sums of tiles (pass-specific)
     int32_t n_tensors;
     int32_t tile_begin, tile_end;  // this launch covers tiles [tile_begin, tile_end) of the prefix table
-    int32_t phase;               // rc[phase] holds the current r, c; rc[1 - phase] receives the new ones
-    int32_t variant;             // pass 2: 0 = rows prefetched into registers, 1 = rows staged by bulk copies
+    RcSel sel;                   // roles of the three scale buffers in this step
+    const uint2* work;           // fused schedule: the work list
+    TensorSync* tsync;           // fused schedule: per-tensor progress counters
+    uint32_t spin_limit;         // fused schedule: polls before a wait gives up
+    uint32_t epoch;              // fused schedule: number of this launch on the state (1, 2, ...)
+    int32_t l2_hints;            // fused schedule: 1 = accesses carry L2 eviction priorities
+    unsigned long long* wait_stats;   // fused schedule: {waits that had to poll, their summed nanoseconds}, or nullptr
     int32_t aligned32;           // every parameter (and fp32 gradient) pointer is 32-byte aligned: 256-bit accesses
     uint32_t* dev_status;        // device error word in the arena header (0 = ok)
     int32_t* tile_counter;       // two words in the arena header: next tile of this launch, finished CTAs (both 0 between launches)
@@ -69,6 +98,13 @@ cudaError_t launch_pass2_bf16_fast(const StepArgs& a, int m_shift, int v_kind, i
 cudaError_t launch_pass2_bf16_ieee(const StepArgs& a, int m_shift, int v_kind, int grid, cudaStream_t s);
 cudaError_t launch_pass2_f32_fast(const StepArgs& a, int m_shift, int v_kind, int grid, cudaStream_t s);
 cudaError_t launch_pass2_f32_ieee(const StepArgs& a, int m_shift, int v_kind, int grid, cudaStream_t s);
+cudaError_t launch_fused(const StepArgs& a, bool bf16, bool exact, int grid, cudaStream_t s);
+cudaError_t launch_fused_bf16_fast(const StepArgs& a, int grid, cudaStream_t s);
+cudaError_t launch_fused_bf16_ieee(const StepArgs& a, int grid, cudaStream_t s);
+cudaError_t launch_fused_f32_fast(const StepArgs& a, int grid, cudaStream_t s);
+cudaError_t launch_fused_f32_ieee(const StepArgs& a, int grid, cudaStream_t s);
+cudaError_t launch_wait_selftest(const uint32_t* flag, uint32_t want, uint32_t limit, uint32_t* dev_status, int32_t* gave_up,
+                                 cudaStream_t s);
 cudaError_t launch_factor_finalize(const StepArgs& a, int t0, int t1, cudaStream_t s);
 cudaError_t launch_sgdm(const StepArgs& a, bool bf16, int grid, cudaStream_t s);
 cudaError_t launch_rcp(const float* src, float* dst, int64_t n, cudaStream_t s);

@@ -34,6 +34,9 @@ __device__ __forceinline__ int find_tensor(const int32_t* __restrict__ start, in
     return lo;
 }
 
+// One of the three rank-1 scale buffers of a tensor (selected without indexing the by-value descriptor dynamically).
+__device__ __forceinline__ float* rc_pick(const TensorDesc& d, int i) { return i == 0 ? d.rc[0] : (i == 1 ? d.rc[1] : d.rc[2]); }
+
 // ---- tile hand-out --------------------------------------------------------------------------------
 //
 // The CTAs of a launch take tiles from a counter in the arena header in the order they become free, so an SM
@@ -290,6 +293,70 @@ __device__ __forceinline__ void store8_f32_256(float* p, const float (&x)[8]) {
                  :: "l"(p), "f"(x[0]), "f"(x[1]), "f"(x[2]), "f"(x[3]), "f"(x[4]), "f"(x[5]), "f"(x[6]), "f"(x[7]) : "memory");
 }
 
+// ---- L2 residency hints (fused schedule) --------------------------------------------------------------
+//
+// In the fused schedule the maxima pass and the update pass of a tensor run close together and the update pass
+// should find the gradient and the second-moment codes still in L2. Accesses therefore carry a cache policy:
+// the maxima pass reads them "evict last" (for the part of a tensor that is meant to stay), the update pass reads
+// and writes everything "evict first" (each line is dead once it has been used), so that the streaming operands
+// (parameters, first-moment codes) are the first victims and do not push the kept lines out.
+struct L2Policies {
+    uint64_t first, last, normal;
+};
+__device__ __forceinline__ L2Policies make_l2_policies() {
+    L2Policies p;
+    asm("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p.first));
+    asm("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p.last));
+    asm("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p.normal));
+    return p;
+}
+__device__ __forceinline__ void load8_f32_256_h(const float* p, float4& a, float4& b, uint64_t pol) {
+    asm volatile("ld.global.L2::cache_hint.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8], %9;"
+                 : "=f"(a.x), "=f"(a.y), "=f"(a.z), "=f"(a.w), "=f"(b.x), "=f"(b.y), "=f"(b.z), "=f"(b.w) : "l"(p), "l"(pol));
+}
+__device__ __forceinline__ float4 load4_f32_h(const float* p, uint64_t pol) {
+    float4 a;
+    asm volatile("ld.global.L2::cache_hint.v4.f32 {%0,%1,%2,%3}, [%4], %5;"
+                 : "=f"(a.x), "=f"(a.y), "=f"(a.z), "=f"(a.w) : "l"(p), "l"(pol));
+    return a;
+}
+__device__ __forceinline__ void load8_u32_256_nc_h(const void* p, uint4& a, uint4& b, uint64_t pol) {
+    asm volatile("ld.global.nc.L2::cache_hint.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8], %9;"
+                 : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w), "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w) : "l"(p), "l"(pol));
+}
+__device__ __forceinline__ uint4 load4_u32_nc_h(const void* p, uint64_t pol) {
+    uint4 a;
+    asm volatile("ld.global.nc.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
+                 : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w) : "l"(p), "l"(pol));
+    return a;
+}
+__device__ __forceinline__ uint32_t load1_u32_h(const void* p, uint64_t pol) {
+    uint32_t a;
+    asm volatile("ld.global.L2::cache_hint.u32 %0, [%1], %2;" : "=r"(a) : "l"(p), "l"(pol));
+    return a;
+}
+__device__ __forceinline__ uint32_t load1_u32_nc_h(const void* p, uint64_t pol) {
+    uint32_t a;
+    asm volatile("ld.global.nc.L2::cache_hint.u32 %0, [%1], %2;" : "=r"(a) : "l"(p), "l"(pol));
+    return a;
+}
+__device__ __forceinline__ void store8_f32_256_h(float* p, const float (&x)[8], uint64_t pol) {
+    asm volatile("st.global.L2::cache_hint.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8}, %9;"
+                 :: "l"(p), "f"(x[0]), "f"(x[1]), "f"(x[2]), "f"(x[3]), "f"(x[4]), "f"(x[5]), "f"(x[6]), "f"(x[7]), "l"(pol) : "memory");
+}
+__device__ __forceinline__ void store4_f32_h(float* p, float a, float b, float c, float d, uint64_t pol) {
+    asm volatile("st.global.L2::cache_hint.v4.f32 [%0], {%1,%2,%3,%4}, %5;"
+                 :: "l"(p), "f"(a), "f"(b), "f"(c), "f"(d), "l"(pol) : "memory");
+}
+__device__ __forceinline__ void store1_u32_h(void* p, uint32_t v, uint64_t pol) {
+    asm volatile("st.global.L2::cache_hint.u32 [%0], %1, %2;" :: "l"(p), "r"(v), "l"(pol) : "memory");
+}
+__device__ __forceinline__ void load8_f32_cg(const float* p, float (&x)[8]) {   // data written earlier in the same launch
+    float4 a = __ldcg(reinterpret_cast<const float4*>(p));
+    float4 b = __ldcg(reinterpret_cast<const float4*>(p) + 1);
+    x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+}
+
 template <bool A32>
 __device__ __forceinline__ void load8_rw_a(const float* p, float (&x)[8]) {
     if (A32) {
@@ -344,7 +411,19 @@ struct TileView {
     uint32_t* red_step;    // running count of CTA-wide reductions
     const char* pf_base;   // this lane's share of the row prefetch: one cache line of one of the arrays
     uint32_t pf_step;      // bytes between two of the warp's rows in that array (0: this lane prefetches nothing)
+    uint32_t pf_bytes;     // fused schedule: size of this lane's bulk prefetch request (0: a plain one-line prefetch)
+    uint64_t pol;          // fused schedule: cache policy of every access of the update pass (evict first)
+    const float* s_rows;   // fused schedule: shared memory, the tile's old row maxima [kFusedTileRows] followed by the
+                           // reciprocals of its new ones, starting at this warp's first row
 };
+
+// Fused schedule: most rows an update tile may have (its row scalars are staged in shared memory).
+constexpr int kFusedTileRows = 1024;
+#ifdef LPMM_EXP_PLAIN_P2
+constexpr bool kHintedUpdate = false;   // experiment: the fused update pass with plain accesses
+#else
+constexpr bool kHintedUpdate = true;
+#endif
 
 // Asks L2 to fetch this lane's share of row k ahead of time (no register is tied up): the later
 // loads then find their data in L2 instead of waiting for DRAM.
@@ -354,9 +433,41 @@ __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefe
 // One instruction per row for the whole warp: the 256 elements a warp owns in a row are 8 lines of parameters,
 // 4 (bf16) or 8 (fp32) lines of gradient, one line of each code array and one of block scales, and each of the
 // first lanes asks for one of those lines.
-template <bool BF16, int MSHIFT, int VM>
+// Fused schedule: the same as one bulk request per array with the streaming policy, so that the lines arrive in L2
+// already marked as first victims (a plain prefetch would bring them in with normal priority). pf_bytes = the size of
+// this lane's request (0: this lane asks with a plain one-line prefetch, or for nothing).
+__device__ __forceinline__ void prefetch_l2_bulk(const void* p, uint32_t bytes, uint64_t pol) {
+    asm volatile("cp.async.bulk.prefetch.L2.global.L2::cache_hint [%0], %1, %2;" ::"l"(p), "r"(bytes), "l"(pol) : "memory");
+}
+template <bool BF16, int MSHIFT, int VM, bool FU = false>
 __device__ __forceinline__ void prefetch_row(const TileView& t, uint32_t k) {
+    if (FU) {
+        if (t.pf_bytes != 0) prefetch_l2_bulk(t.pf_base + (size_t)k * t.pf_step, t.pf_bytes, t.pol);
+        else if (t.pf_step != 0) prefetch_l2(t.pf_base + (size_t)k * t.pf_step);
+        return;
+    }
     if (t.pf_step != 0) prefetch_l2(t.pf_base + (size_t)k * t.pf_step);
+}
+// Fused schedule: lane 0 asks for the warp's parameters of a row, lane 1 for its first-moment codes (bulk requests),
+// lane 2 for the line with its block maxima. The gradient and the second-moment codes are expected in L2 already.
+template <int MSHIFT>
+__device__ __forceinline__ void prefetch_roles_fused(TileView& t, int lane, int valid, const float* warp_w, const uint8_t* warp_mq,
+                                                     const float* warp_ms) {
+    t.pf_base = nullptr;
+    t.pf_step = 0;
+    t.pf_bytes = 0;
+    if (lane == 0) {
+        t.pf_base = reinterpret_cast<const char*>(warp_w);
+        t.pf_step = t.row_step * 4u;
+        t.pf_bytes = (uint32_t)valid * 4u;
+    } else if (lane == 1) {
+        t.pf_base = reinterpret_cast<const char*>(warp_mq);
+        t.pf_step = t.row_step / 2u;
+        t.pf_bytes = (uint32_t)valid / 2u;
+    } else if (lane == 2) {
+        t.pf_base = reinterpret_cast<const char*>(warp_ms);
+        t.pf_step = (t.row_step >> MSHIFT) * 4u;
+    }
 }
 // Assigns the lane its line (warp_* point at the warp's first element of row 0; row_step in elements).
 // `valid` = how many of the warp's 256 columns exist (128 in a tensor's last warp column when cols % 256 == 128):
@@ -395,9 +506,32 @@ __device__ __forceinline__ void prefetch_roles(TileView& t, int lane, int valid,
 }
 
 // A32: the parameter rows (and fp32 gradient rows) of this tensor are 32-byte aligned.
-template <bool BF16, int MSHIFT, int VM, bool A32>
+template <bool BF16, int MSHIFT, int VM, bool A32, bool FU = false>
 __device__ __forceinline__ void load_row(RowRegs<BF16>& r, const TileView& t, uint32_t k) {
     const uint32_t off = k * t.row_step;
+    if (FU && kHintedUpdate) {   // fused schedule (rank-1, B128 only): every access carries the streaming policy; r', c' reciprocals were
+                // written earlier in this launch and are read past L1
+        if (A32) {
+            load8_f32_256_h(t.w + off, r.w0, r.w1, t.pol);
+        } else {
+            r.w0 = load4_f32_h(t.w + off, t.pol);
+            r.w1 = load4_f32_h(t.w + off + 4, t.pol);
+        }
+        if (BF16) {
+            r.g0 = load4_u32_nc_h(reinterpret_cast<const uint16_t*>(t.g) + off, t.pol);
+        } else if (A32) {
+            load8_u32_256_nc_h(reinterpret_cast<const float*>(t.g) + off, r.g0, r.g1, t.pol);
+        } else {
+            r.g0 = load4_u32_nc_h(reinterpret_cast<const float*>(t.g) + off, t.pol);
+            r.g1 = load4_u32_nc_h(reinterpret_cast<const float*>(t.g) + off + 4, t.pol);
+        }
+        r.qm = load1_u32_h(t.m_codes + (off >> 1), t.pol);
+        r.am = __uint_as_float(load1_u32_h(t.m_scale + (off >> MSHIFT), t.pol));
+        r.qv = load1_u32_h(t.v_codes + (off >> 1), t.pol);
+        r.r_old = t.s_rows[k * t.row_stride];
+        r.r_rcp = t.s_rows[kFusedTileRows + k * t.row_stride];
+        return;
+    }
     if (A32) {
         load8_f32_256(t.w + off, r.w0, r.w1);
     } else {
@@ -420,6 +554,12 @@ __device__ __forceinline__ void load_row(RowRegs<BF16>& r, const TileView& t, ui
         r.r_rcp = 0.0f;
         return;
     }
+    if (FU) {
+        r.qv = *reinterpret_cast<const uint32_t*>(t.v_codes + (off >> 1));
+        r.r_old = t.s_rows[k * t.row_stride];
+        r.r_rcp = t.s_rows[kFusedTileRows + k * t.row_stride];
+        return;
+    }
     r.r_rcp = __ldg(t.r_rcp + k * t.row_stride);        // VM == 1: the row factor R_i / sum(R)
     if (VM == 1) {
         r.qv = 0;
@@ -430,7 +570,7 @@ __device__ __forceinline__ void load_row(RowRegs<BF16>& r, const TileView& t, ui
     }
 }
 
-template <bool BF16, bool EXACT, int MSHIFT, int VM, bool WB, bool A32>
+template <bool BF16, bool EXACT, int MSHIFT, int VM, bool WB, bool A32, bool FU = false>
 __device__ __forceinline__ void process_row(const RowRegs<BF16>& r, const TileView& t, uint32_t k,
                                             const float (&c_old)[8], const float (&c_rcp)[8], const Hyper& h,
                                             const Hyper2& h2, const LaneTables& lt, const unsigned char* s_lut) {
@@ -452,6 +592,19 @@ __device__ __forceinline__ void process_row(const RowRegs<BF16>& r, const TileVi
         }
     }
     moments_and_update8<EXACT, VM == 1>(wv, gv, r.qm, r.qv, __fmul_rn(lt.de, r.am), vs, h, h2, lt, mt, vt);
+    if (FU && kHintedUpdate) {
+        if (A32) {
+            store8_f32_256_h(t.w + off, wv, t.pol);
+        } else {
+            store4_f32_h(t.w + off, wv[0], wv[1], wv[2], wv[3], t.pol);
+            store4_f32_h(t.w + off + 4, wv[4], wv[5], wv[6], wv[7], t.pol);
+        }
+        const float am_f = group_max(absmax8(mt), lt.mask);
+        if ((threadIdx.x & 15) == 0) store1_u32_h(t.m_scale + (off >> 7), __float_as_uint(am_f), t.pol);
+        store1_u32_h(t.m_codes + (off >> 1), quantize8_de(mt, scale_rcp(am_f), s_lut), t.pol);
+        store1_u32_h(t.v_codes + (off >> 1), quantize8_lin(vt, vr, h2), t.pol);
+        return;
+    }
     if (A32) store8_f32_256(t.w + off, wv); else store8_f32(t.w + off, wv);
     if (WB) store8_bf16(t.w16 + off, wv);
     const float am_new = block_max(absmax8(mt), MSHIFT, lt, t.s_red, *t.red_step);
@@ -468,20 +621,33 @@ __device__ __forceinline__ void process_row(const RowRegs<BF16>& r, const TileVi
 }
 
 // VM: how the second moment is kept: 0 rank-1 codes (Sec. 4.2), 1 factorized statistics (Sec. 4.3), 2 block-wise codes.
-template <bool BF16, bool EXACT, int MSHIFT, int VM = 0, bool WB = false, bool A32 = false>
+template <bool BF16, bool EXACT, int MSHIFT, int VM = 0, bool WB = false, bool A32 = false, bool FU = false>
 __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __restrict__ w, uint16_t* __restrict__ w16,
                                                  const void* __restrict__ g,
-                                                 int tile, int phase, const Hyper& h, const Hyper2& h2,
+                                                 int tile, RcSel sel, const Hyper& h, const Hyper2& h2,
                                                  const LaneTables& lt, const unsigned char* s_lut, float* s_red,
-                                                 uint32_t& red_step) {
+                                                 uint32_t& red_step, uint64_t pol = 0, float* s_rows = nullptr) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int wx = d.wx, wy_count = kWarps / wx;
     const int tx = tile % d.tiles_x, ty = tile / d.tiles_x;
+    if (FU) {
+        // The tile's row scalars go to shared memory first (before any warp leaves): the old row maxima, and the
+        // reciprocals of the new ones, which the maxima pass reduced earlier in this launch (read past L1).
+        const int64_t r0 = (int64_t)ty * d.tile_rows;
+        const int nr = (int)min((int64_t)d.tile_rows, d.rows - r0);
+        const float* ro = rc_pick(d, sel.old_i) + r0;
+        const float* rn = rc_pick(d, sel.new_i) + r0;
+        for (int i = threadIdx.x; i < nr; i += kThreads) {
+            s_rows[i] = __ldg(ro + i);
+            s_rows[kFusedTileRows + i] = scale_rcp(__ldcg(rn + i));
+        }
+        __syncthreads();
+    }
     const int64_t col0 = (int64_t)tx * (kWarpElems * wx) + (warp % wx) * kWarpElems + lane * kLaneElems;
     // cols % 128 == 0: a whole 16-lane group (one block) is in or out together. With B2048 the tile is one
     // block wide (wx = 8, cols % 2048 == 0), every warp is inside and all of them run the same rows.
     if (col0 >= d.cols) return;
-    const float* rc_old = (phase ? d.rc[1] : d.rc[0]);
+    const float* rc_old = rc_pick(d, sel.old_i);
     const float* rcp_new = d.rcp_new;
     const int64_t row0 = (int64_t)ty * d.tile_rows + warp / wx;
     const int64_t row_end = min((int64_t)(ty + 1) * d.tile_rows, d.rows);
@@ -493,15 +659,22 @@ __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __r
 #pragma unroll
         for (int j = 0; j < 8; ++j) { c_old[j] = 0.0f; c_rcp[j] = 0.0f; }
     } else if (VM == 1) {      // the new column statistics C_j sit in the "new" buffer; nothing old is needed
-        load8_f32((phase ? d.rc[0] : d.rc[1]) + d.c_off + col0, c_rcp);
+        load8_f32(rc_pick(d, sel.new_i) + d.c_off + col0, c_rcp);
 #pragma unroll
         for (int j = 0; j < 8; ++j) c_old[j] = 0.0f;
     } else {
         load8_f32(rc_old + d.c_off + col0, c_old);
-        load8_f32(rcp_new + d.c_off + col0, c_rcp);
+        if (FU) {   // the new column maxima c' were reduced earlier in this launch: read past L1, invert here
+            load8_f32_cg(rc_pick(d, sel.new_i) + d.c_off + col0, c_rcp);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) c_rcp[j] = scale_rcp(c_rcp[j]);
+        } else {
+            load8_f32(rcp_new + d.c_off + col0, c_rcp);
+        }
     }
     const int64_t e0 = row0 * d.cols + col0;
     TileView t;
+    t.pol = pol;
     t.w = w + e0;
     t.w16 = WB ? w16 + e0 : nullptr;
     t.g = BF16 ? static_cast<const void*>(reinterpret_cast<const uint16_t*>(g) + e0)
@@ -512,6 +685,7 @@ __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __r
     t.m_scale = d.m_scale + (e0 >> MSHIFT);
     t.r_old = rc_old + row0;
     t.r_rcp = rcp_new + row0;
+    t.s_rows = FU ? s_rows + warp / wx : nullptr;
     t.row_step = (uint32_t)(wy_count * d.cols);
     t.row_stride = (uint32_t)wy_count;
     t.m_shift = d.m_shift;
@@ -520,6 +694,9 @@ __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __r
     {
         const int64_t ew = e0 - lane * kLaneElems;       // the warp's first element of its first row
         const int64_t left = d.cols - (col0 - lane * kLaneElems);
+        if (FU) prefetch_roles_fused<MSHIFT>(t, lane, left < kWarpElems ? (int)left : kWarpElems, w + ew, d.m_codes + (ew >> 1),
+                                             d.m_scale + (ew >> MSHIFT));
+        else
         prefetch_roles<BF16, MSHIFT, VM>(t, lane, left < kWarpElems ? (int)left : kWarpElems, w + ew,
                                            BF16 ? static_cast<const void*>(reinterpret_cast<const uint16_t*>(g) + ew)
                                                 : static_cast<const void*>(reinterpret_cast<const float*>(g) + ew),
@@ -530,200 +707,27 @@ __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __r
     // Two register sets alternate: while one row is processed the next one is already in flight.
     RowRegs<BF16> ra, rb;
 #pragma unroll
-    for (uint32_t k = 1; k < kL2Ahead; ++k) if (k < nrows) prefetch_row<BF16, MSHIFT, VM>(t, k);
-    load_row<BF16, MSHIFT, VM, A32>(ra, t, 0);
+    for (uint32_t k = 1; k < kL2Ahead; ++k) if (k < nrows) prefetch_row<BF16, MSHIFT, VM, FU>(t, k);
+    load_row<BF16, MSHIFT, VM, A32, FU>(ra, t, 0);
     uint32_t k = 0;
     // (B2048 rows end in a CTA-wide barrier, where the longer straight-line body only costs registers: guarded loop only)
     for (; MSHIFT == 7 && k + 1 + kL2Ahead < nrows; k += 2) {        // every row touched below exists: no guards
-        prefetch_row<BF16, MSHIFT, VM>(t, k + kL2Ahead);
-        load_row<BF16, MSHIFT, VM, A32>(rb, t, k + 1);
-        process_row<BF16, EXACT, MSHIFT, VM, WB, A32>(ra, t, k, c_old, c_rcp, h, h2, lt, s_lut);
-        prefetch_row<BF16, MSHIFT, VM>(t, k + 1 + kL2Ahead);
-        load_row<BF16, MSHIFT, VM, A32>(ra, t, k + 2);
-        process_row<BF16, EXACT, MSHIFT, VM, WB, A32>(rb, t, k + 1, c_old, c_rcp, h, h2, lt, s_lut);
+        prefetch_row<BF16, MSHIFT, VM, FU>(t, k + kL2Ahead);
+        load_row<BF16, MSHIFT, VM, A32, FU>(rb, t, k + 1);
+        process_row<BF16, EXACT, MSHIFT, VM, WB, A32, FU>(ra, t, k, c_old, c_rcp, h, h2, lt, s_lut);
+        prefetch_row<BF16, MSHIFT, VM, FU>(t, k + 1 + kL2Ahead);
+        load_row<BF16, MSHIFT, VM, A32, FU>(ra, t, k + 2);
+        process_row<BF16, EXACT, MSHIFT, VM, WB, A32, FU>(rb, t, k + 1, c_old, c_rcp, h, h2, lt, s_lut);
     }
     for (; k < nrows; k += 2) {                       // the last rows of the tile
         const bool has_b = k + 1 < nrows;
-        if (k + kL2Ahead < nrows) prefetch_row<BF16, MSHIFT, VM>(t, k + kL2Ahead);
-        if (has_b) load_row<BF16, MSHIFT, VM, A32>(rb, t, k + 1);
-        process_row<BF16, EXACT, MSHIFT, VM, WB, A32>(ra, t, k, c_old, c_rcp, h, h2, lt, s_lut);
+        if (k + kL2Ahead < nrows) prefetch_row<BF16, MSHIFT, VM, FU>(t, k + kL2Ahead);
+        if (has_b) load_row<BF16, MSHIFT, VM, A32, FU>(rb, t, k + 1);
+        process_row<BF16, EXACT, MSHIFT, VM, WB, A32, FU>(ra, t, k, c_old, c_rcp, h, h2, lt, s_lut);
         if (!has_b) break;
-        if (k + 1 + kL2Ahead < nrows) prefetch_row<BF16, MSHIFT, VM>(t, k + 1 + kL2Ahead);
-        if (k + 2 < nrows) load_row<BF16, MSHIFT, VM, A32>(ra, t, k + 2);
-        process_row<BF16, EXACT, MSHIFT, VM, WB, A32>(rb, t, k + 1, c_old, c_rcp, h, h2, lt, s_lut);
-    }
-}
-
-// ---- pass 2, rank-1 tensors, rows staged by bulk asynchronous copies ---------------------------------
-//
-// Each warp owns a small ring in shared memory. One lane asks the copy engine (cp.async.bulk, completion
-// counted on an mbarrier) for the warp's 256-element segment of the next rows: parameters, gradient and
-// both code words. The data of several rows is then in flight without holding registers or issue slots,
-// and the lanes read their 8 elements back with plain shared-memory loads. Nothing is shared between
-// warps, so there is no block-wide barrier; a warp reuses a slot right after its own lanes have read it.
-// Every wait is bounded: if a copy never completes, the warp records an error word and stops.
-
-constexpr int kBulkStages = 4;
-constexpr uint32_t kSpinLimit = 1u << 18;   // polls of a (self-suspending) try_wait before giving up
-constexpr uint32_t kStatusCopyTimeout = 1u;
-
-template <bool BF16>
-struct WarpStage {                                   // byte offsets inside one stage of one warp
-    static constexpr int kW = 0;                                    // 256 floats
-    static constexpr int kG = 1024;                                 // 256 bf16 / 256 floats
-    static constexpr int kQm = kG + (BF16 ? 512 : 1024);            // 128 bytes of codes
-    static constexpr int kQv = kQm + 128;
-    static constexpr int kBytes = kQv + 128;
-};
-template <bool BF16>
-constexpr int bulk_smem_bytes() {
-    return kLutSmemBytes + kWarps * kBulkStages * WarpStage<BF16>::kBytes + kWarps * kBulkStages * 8;
-}
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-// Bounded wait for the given phase parity of an mbarrier; false if it never completed.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    for (uint32_t it = 0; it < kSpinLimit; ++it) {
-        uint32_t done;
-        asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
-                     : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-        if (done) return true;
-    }
-    return false;
-}
-
-struct WarpRing {
-    unsigned char* data;     // kBulkStages stages of this warp
-    uint32_t bars;           // shared address of this warp's kBulkStages mbarriers
-    uint32_t slot;           // stage that receives / delivers the next row
-    uint32_t phases;         // bit s = parity to wait for on stage s
-    bool dead;               // a wait timed out: this warp does no further work
-};
-
-// Warp-uniform description of the warp's rows in one tile (addresses at the warp's first column).
-struct BulkView {
-    const float* w;
-    const void* g;
-    const uint8_t* m_codes;
-    const uint8_t* v_codes;
-    uint32_t row_step;
-};
-
-template <bool BF16>
-__device__ __forceinline__ void bulk_issue_row(const WarpRing& r, uint32_t slot, const BulkView& t, uint32_t k) {
-    // called by one lane
-    const uint32_t off = k * t.row_step;
-    const uint32_t bar = r.bars + slot * 8;
-    const uint32_t dst = smem_u32(r.data + slot * WarpStage<BF16>::kBytes);
-    mbar_expect_tx(bar, WarpStage<BF16>::kBytes);
-    bulk_load(dst + WarpStage<BF16>::kW, t.w + off, 1024, bar);
-    if (BF16) bulk_load(dst + WarpStage<BF16>::kG, reinterpret_cast<const uint16_t*>(t.g) + off, 512, bar);
-    else bulk_load(dst + WarpStage<BF16>::kG, reinterpret_cast<const float*>(t.g) + off, 1024, bar);
-    bulk_load(dst + WarpStage<BF16>::kQm, t.m_codes + (off >> 1), 128, bar);
-    bulk_load(dst + WarpStage<BF16>::kQv, t.v_codes + (off >> 1), 128, bar);
-}
-
-template <bool BF16, bool EXACT>
-__device__ __forceinline__ void pass2_rank1_bulk(const TensorDesc& d, float* __restrict__ w, const void* __restrict__ g,
-                                                 int tile, int phase, const Hyper& h, const Hyper2& h2,
-                                                 const LaneTables& lt, const unsigned char* s_lut, WarpRing& ring,
-                                                 uint32_t* dev_status) {
-    if (ring.dead) return;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int wx = d.wx, wy_count = kWarps / wx;
-    const int tx = tile % d.tiles_x, ty = tile / d.tiles_x;
-    const int64_t col_w = (int64_t)tx * (kWarpElems * wx) + (warp % wx) * kWarpElems;   // cols % 256 == 0 here
-    const int64_t col0 = col_w + lane * kLaneElems;
-    const float* rc_old = (phase ? d.rc[1] : d.rc[0]);
-    const float* rcp_new = d.rcp_new;
-    const int64_t row0 = (int64_t)ty * d.tile_rows + warp / wx;
-    const int64_t row_end = min((int64_t)(ty + 1) * d.tile_rows, d.rows);
-    if (row0 >= row_end) return;                       // uniform over the warp
-    const uint32_t nrows = (uint32_t)((row_end - row0 + wy_count - 1) / wy_count);
-    const int64_t e_w = row0 * d.cols + col_w;         // warp's first element
-    BulkView t;
-    t.w = w + e_w;
-    t.g = BF16 ? static_cast<const void*>(reinterpret_cast<const uint16_t*>(g) + e_w)
-               : static_cast<const void*>(reinterpret_cast<const float*>(g) + e_w);
-    t.m_codes = d.m_codes + (e_w >> 1);
-    t.v_codes = d.v_codes + (e_w >> 1);
-    t.row_step = (uint32_t)(wy_count * d.cols);
-
-    if (lane == 0) {                                   // fill the ring
-        for (uint32_t k = 0; k < (uint32_t)kBulkStages && k < nrows; ++k)
-            bulk_issue_row<BF16>(ring, (ring.slot + k) % kBulkStages, t, k);
-    }
-    float c_old[8], c_rcp[8];
-    load8_f32(rc_old + d.c_off + col0, c_old);
-    load8_f32(rcp_new + d.c_off + col0, c_rcp);
-    // Per-row scalars: lane j (mod 16) keeps the values of the warp's row number base + j, 16 rows per refill;
-    // lanes 0-15 hold the first block's old scale of m, lanes 16-31 the second block's.
-    float* w_lane = w + e_w + lane * kLaneElems;
-    uint8_t* mq_lane = d.m_codes + ((e_w + lane * kLaneElems) >> 1);
-    uint8_t* vq_lane = d.v_codes + ((e_w + lane * kLaneElems) >> 1);
-    float* ms_warp = d.m_scale + (e_w >> 7);
-    float am_vec = 0.0f, ro_vec = 0.0f, rr_vec = 0.0f;
-    for (uint32_t k = 0; k < nrows; ++k) {
-        if ((k & 15) == 0) {
-            const uint32_t kk = min(k + (lane & 15), nrows - 1);
-            am_vec = ms_warp[(size_t)((kk * t.row_step) >> 7) + (lane >> 4)];
-            ro_vec = __ldg(rc_old + row0 + (int64_t)kk * wy_count);
-            rr_vec = __ldg(rcp_new + row0 + (int64_t)kk * wy_count);
-        }
-        const uint32_t slot = ring.slot;
-        if (!mbar_wait(ring.bars + slot * 8, (ring.phases >> slot) & 1u)) {
-            if (lane == 0) atomicExch(dev_status, kStatusCopyTimeout);
-            ring.dead = true;
-            return;
-        }
-        ring.phases ^= 1u << slot;
-        const unsigned char* st = ring.data + slot * WarpStage<BF16>::kBytes;
-        const float4 w0 = *reinterpret_cast<const float4*>(st + WarpStage<BF16>::kW + lane * 32);
-        const float4 w1 = *reinterpret_cast<const float4*>(st + WarpStage<BF16>::kW + lane * 32 + 16);
-        uint4 g0, g1 = make_uint4(0, 0, 0, 0);
-        if (BF16) {
-            g0 = *reinterpret_cast<const uint4*>(st + WarpStage<BF16>::kG + lane * 16);
-        } else {
-            g0 = *reinterpret_cast<const uint4*>(st + WarpStage<BF16>::kG + lane * 32);
-            g1 = *reinterpret_cast<const uint4*>(st + WarpStage<BF16>::kG + lane * 32 + 16);
-        }
-        const uint32_t qm = *reinterpret_cast<const uint32_t*>(st + WarpStage<BF16>::kQm + lane * 4);
-        const uint32_t qv = *reinterpret_cast<const uint32_t*>(st + WarpStage<BF16>::kQv + lane * 4);
-        __syncwarp();                                  // every lane has read the slot
-        if (lane == 0 && k + kBulkStages < nrows) {
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            bulk_issue_row<BF16>(ring, slot, t, k + kBulkStages);
-        }
-        ring.slot = (slot + 1 == (uint32_t)kBulkStages) ? 0u : slot + 1;
-
-        const float am = __shfl_sync(0xffffffffu, am_vec, (lane & 16) | (k & 15));
-        const float r_old = __shfl_sync(0xffffffffu, ro_vec, k & 15);
-        const float r_rcp = __shfl_sync(0xffffffffu, rr_vec, k & 15);
-        float wv[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
-        float gv[8], mt[8], vt[8], vs[8], vr[8];
-        unpack_grad8<BF16>(g0, g1, gv);
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            vs[j] = fminf(r_old, c_old[j]);
-            vr[j] = fmaxf(r_rcp, c_rcp[j]);
-        }
-        moments_and_update8<EXACT>(wv, gv, qm, qv, __fmul_rn(lt.de, am), vs, h, h2, lt, mt, vt);
-        const uint32_t off = k * t.row_step;
-        store8_f32(w_lane + off, wv);
-        const float am_new = group_max(absmax8(mt), lt.mask);
-        if ((lane & 15) == 0) ms_warp[(size_t)(off >> 7) + (lane >> 4)] = am_new;
-        *reinterpret_cast<uint32_t*>(mq_lane + (off >> 1)) = quantize8_de(mt, scale_rcp(am_new), s_lut);
-        *reinterpret_cast<uint32_t*>(vq_lane + (off >> 1)) = quantize8_lin(vt, vr, h2);
+        if (k + 1 + kL2Ahead < nrows) prefetch_row<BF16, MSHIFT, VM, FU>(t, k + 1 + kL2Ahead);
+        if (k + 2 < nrows) load_row<BF16, MSHIFT, VM, A32, FU>(ra, t, k + 2);
+        process_row<BF16, EXACT, MSHIFT, VM, WB, A32, FU>(rb, t, k + 1, c_old, c_rcp, h, h2, lt, s_lut);
     }
 }
 
@@ -745,16 +749,18 @@ __device__ __forceinline__ void split_index(const TensorDesc& d, int64_t e, int6
     }
 }
 
-template <bool MAX>
+// CG: the statistics were written earlier in the same launch (fused schedule): read them past L1.
+template <bool MAX, bool CG = false>
 __device__ __forceinline__ float outer_stat(const TensorDesc& d, const float* __restrict__ base, int64_t i) {
-    if (d.n_outer == 1) return __ldg(base + i);
+    if (d.n_outer == 1) return CG ? __ldcg(base + i) : __ldg(base + i);
     uint32_t rem = (uint32_t)i;                          // rows <= 2^30 (checked on the host)
     float s = MAX ? 0.0f : 3.402823466e38f;
 #pragma unroll
     for (int a = 2; a >= 0; --a) {                       // the last leading axis varies fastest; constant indices keep
         if (a < d.n_outer) {                             // the descriptor in registers
             const uint32_t q = rem / (uint32_t)d.outer_dim[a];
-            const float x = __ldg(base + d.outer_off[a] + (rem - q * (uint32_t)d.outer_dim[a]));
+            const float* px = base + d.outer_off[a] + (rem - q * (uint32_t)d.outer_dim[a]);
+            const float x = CG ? __ldcg(px) : __ldg(px);
             s = MAX ? fmaxf(s, x) : fminf(s, x);
             rem = q;
         }
@@ -777,13 +783,13 @@ __device__ __forceinline__ void outer_publish(const TensorDesc& d, float* base, 
 
 // ---- pass 2, flat (element-indexed) tensors: block-wise v, or rank-1 with arbitrary cols ------
 
-template <bool BF16, bool RANK1, bool EXACT, int MSHIFT, bool WB = false, bool A32 = false>
+template <bool BF16, bool RANK1, bool EXACT, int MSHIFT, bool WB = false, bool A32 = false, bool FU = false>
 __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restrict__ w, uint16_t* __restrict__ w16,
                                            const void* __restrict__ g,
-                                           int tile, int phase, const Hyper& h, const Hyper2& h2, const LaneTables& lt,
+                                           int tile, RcSel sel, const Hyper& h, const Hyper2& h2, const LaneTables& lt,
                                            const unsigned char* s_lut, float* s_red, uint32_t& red_step) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const float* rc_old = (phase ? d.rc[1] : d.rc[0]);
+    const float* rc_old = rc_pick(d, sel.old_i);
     const float* rcp_new = d.rcp_new;
     const int64_t m_mask = ((int64_t)1 << MSHIFT) - 1;
     for (int c = 0; c < d.flat_chunks; ++c) {
@@ -817,10 +823,11 @@ __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restric
             // cols % 8 == 0: the lane's eight elements lie in one row, their column statistics are two 16-byte loads
             int64_t i, j;
             split_index(d, e, i, j);
-            const float so = outer_stat<false>(d, rc_old, i), ro = outer_stat<true>(d, rcp_new, i);
+            const float so = outer_stat<false>(d, rc_old, i), ro = outer_stat<true, FU>(d, rcp_new, i);
             float co[8], cr[8];
             load8_f32(rc_old + d.c_off + j, co);
-            load8_f32(rcp_new + d.c_off + j, cr);
+            if (FU) load8_f32_cg(rcp_new + d.c_off + j, cr);
+            else load8_f32(rcp_new + d.c_off + j, cr);
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
                 vs[k] = fminf(so, co[k]);
@@ -836,11 +843,11 @@ __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restric
                 if (e + k < d.numel) {
                     if (fresh) {
                         so = outer_stat<false>(d, rc_old, i);
-                        ro = outer_stat<true>(d, rcp_new, i);
+                        ro = outer_stat<true, FU>(d, rcp_new, i);
                         fresh = false;
                     }
                     vs[k] = fminf(so, __ldg(rc_old + d.c_off + j));
-                    vr[k] = fmaxf(ro, __ldg(rcp_new + d.c_off + j));
+                    vr[k] = fmaxf(ro, FU ? __ldcg(rcp_new + d.c_off + j) : __ldg(rcp_new + d.c_off + j));
                 } else {
                     vs[k] = 0.0f; vr[k] = 0.0f;
                 }
@@ -944,62 +951,18 @@ __global__ void __launch_bounds__(kThreads, 2) pass2_kernel(StepArgs a) {
         const int local = tile - __ldg(a.tile_start + t);
         switch (d.kind) {
             case K_RANK1_FAST:
-                if (VF == 0) pass2_rank1_fast<BF16, EXACT, MSHIFT, 0, WB, A32>(d, w, w16, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step);
+                if (VF == 0) pass2_rank1_fast<BF16, EXACT, MSHIFT, 0, WB, A32>(d, w, w16, g, local, a.sel, a.h, h2, lt, s_lut, s_red, red_step);
                 break;
             case K_FACT:
-                if (VF == 1) pass2_rank1_fast<BF16, EXACT, MSHIFT, 1, WB>(d, w, w16, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step);
+                if (VF == 1) pass2_rank1_fast<BF16, EXACT, MSHIFT, 1, WB>(d, w, w16, g, local, a.sel, a.h, h2, lt, s_lut, s_red, red_step);
                 break;
             case K_BLOCK_TILED:   // matrices of a block-wise state; long 1-D tensors folded into rows (in states of another
                                   // kind these get a launch of their own, so that the default kernels stay lean)
-                if (VF == 2) pass2_rank1_fast<BF16, EXACT, MSHIFT, 2, WB, A32>(d, w, w16, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step);
+                if (VF == 2) pass2_rank1_fast<BF16, EXACT, MSHIFT, 2, WB, A32>(d, w, w16, g, local, a.sel, a.h, h2, lt, s_lut, s_red, red_step);
                 break;
-            case K_RANK1_FLAT: pass2_flat<BF16, true, EXACT, MSHIFT, WB, A32>(d, w, w16, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
-            case K_BLOCK:      pass2_flat<BF16, false, EXACT, MSHIFT, WB, A32>(d, w, w16, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
+            case K_RANK1_FLAT: pass2_flat<BF16, true, EXACT, MSHIFT, WB, A32>(d, w, w16, g, local, a.sel, a.h, h2, lt, s_lut, s_red, red_step); break;
+            case K_BLOCK:      pass2_flat<BF16, false, EXACT, MSHIFT, WB, A32>(d, w, w16, g, local, a.sel, a.h, h2, lt, s_lut, s_red, red_step); break;
             default:           pass2_fp32<BF16, EXACT, WB, A32>(d, w, w16, g, local, a.h); break;
-        }
-        tile = a.tile_begin + tiles_next(s_next, buf, fetched);
-    }
-    tiles_done(a.tile_counter);
-}
-
-template <bool BF16, bool EXACT, int MSHIFT>
-__global__ void __launch_bounds__(kThreads, 2) pass2_bulk_kernel(StepArgs a) {
-    extern __shared__ __align__(128) unsigned char s_dyn[];   // [nearest-entry table | warp rings | mbarriers]
-    unsigned char* s_lut = s_dyn;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    __shared__ float s_red[2 * kWarps];
-    WarpRing ring;
-    ring.data = s_dyn + kLutSmemBytes + warp * kBulkStages * WarpStage<BF16>::kBytes;
-    ring.bars = smem_u32(s_dyn + kLutSmemBytes + kWarps * kBulkStages * WarpStage<BF16>::kBytes) + warp * kBulkStages * 8;
-    ring.slot = 0;
-    ring.phases = 0;
-    ring.dead = false;
-    if (lane == 0) {
-        for (int s = 0; s < kBulkStages; ++s) mbar_init(ring.bars + s * 8, 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    load_lut_smem(s_lut);
-    __syncthreads();
-    const LaneTables lt = make_lane_tables();
-    const Hyper2& h2 = a.h2;
-    uint32_t red_step = 0;
-    __shared__ int s_next[2];
-    int buf = 0;
-    for (int tile = a.tile_begin + tiles_first(a.tile_counter, s_next); tile < a.tile_end;) {
-        const int fetched = tiles_fetch(a.tile_counter);
-        const int t = find_tensor(a.tile_start, a.n_tensors, tile);
-        const TensorDesc d = a.descs[t];
-        float* w = a.params[t];
-        const void* g = a.grads[t];
-        const int local = tile - __ldg(a.tile_start + t);
-        switch (d.kind) {
-            case K_RANK1_FAST:
-                if ((d.cols & 255) == 0 && MSHIFT == 7) pass2_rank1_bulk<BF16, EXACT>(d, w, g, local, a.phase, a.h, h2, lt, s_lut, ring, a.dev_status);
-                else pass2_rank1_fast<BF16, EXACT, MSHIFT>(d, w, nullptr, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step);
-                break;
-            case K_RANK1_FLAT: pass2_flat<BF16, true, EXACT, MSHIFT>(d, w, nullptr, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
-            case K_BLOCK:      pass2_flat<BF16, false, EXACT, MSHIFT>(d, w, nullptr, g, local, a.phase, a.h, h2, lt, s_lut, s_red, red_step); break;
-            default:           pass2_fp32<BF16, EXACT>(d, w, nullptr, g, local, a.h); break;
         }
         tile = a.tile_begin + tiles_next(s_next, buf, fetched);
     }
@@ -1024,11 +987,23 @@ struct P1View {
     const char* pf_base;       // this lane's share of the prefetch of a group of rows: one line of one array in one row
     uint32_t pf_step;          // bytes between two of the warp's rows in that array (0: nothing to prefetch)
     uint32_t pf_row;           // which row of the group
+    uint64_t pol;              // fused schedule: cache policy of the loads (evict last where the tile is meant to stay in L2)
+    bool keep;                 // fused schedule: whether the prefetch hints ask for evict-last lines
 };
 
-template <bool BF16>
+template <bool BF16, bool FU = false>
 __device__ __forceinline__ void load_p1_row(P1Row<BF16>& b, const P1View& t, uint32_t k) {
     const uint32_t off = k * t.row_step;
+    if (FU) {
+        if (BF16) {
+            b.g0 = load4_u32_nc_h(reinterpret_cast<const uint16_t*>(t.g) + off, t.pol);
+        } else {
+            b.g0 = load4_u32_nc_h(reinterpret_cast<const float*>(t.g) + off, t.pol);
+            b.g1 = load4_u32_nc_h(reinterpret_cast<const float*>(t.g) + off + 4, t.pol);
+        }
+        b.qv = load1_u32_nc_h(t.v_codes + (off >> 1), t.pol);
+        return;
+    }
     if (BF16) {
         b.g0 = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(t.g) + off));
     } else {
@@ -1063,10 +1038,14 @@ __device__ __forceinline__ void p1_prefetch_roles(P1View& t, int lane, int valid
     }
 }
 // Rows k .. k + kRows - 1 (those below nrows).
-template <bool BF16>
+__device__ __forceinline__ void prefetch_l2_keep(const void* p) { asm volatile("prefetch.global.L2::evict_last [%0];" ::"l"(p)); }
+template <bool BF16, bool FU = false>
 __device__ __forceinline__ void prefetch_p1_group(const P1View& t, uint32_t k, uint32_t nrows) {
     const uint32_t row = k + t.pf_row;
-    if (t.pf_step != 0 && row < nrows) prefetch_l2(t.pf_base + (size_t)row * t.pf_step);
+    if (t.pf_step != 0 && row < nrows) {
+        if (FU && t.keep) prefetch_l2_keep(t.pf_base + (size_t)row * t.pf_step);
+        else prefetch_l2(t.pf_base + (size_t)row * t.pf_step);
+    }
 }
 
 // Maxima of four per-lane values over the warp with 6 shuffles: afterwards the lanes with
@@ -1137,9 +1116,10 @@ __device__ __forceinline__ void p1_process_2rows(const P1Row<BF16>& a, const P1R
 
 constexpr uint32_t kP1L2Ahead = 8;  // rows the L2 prefetch hints run ahead
 
-template <bool BF16>
-__device__ __forceinline__ void pass1_rank1_fast(const TensorDesc& d, const void* __restrict__ g, int tile, int phase,
-                                                 const Hyper2& h2, const LaneTables& lt, float* s_col) {
+template <bool BF16, bool FU = false>
+__device__ __forceinline__ void pass1_rank1_fast(const TensorDesc& d, const void* __restrict__ g, int tile, RcSel sel,
+                                                 const Hyper2& h2, const LaneTables& lt, float* s_col, uint64_t pol = 0,
+                                                 bool keep = false) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int wx = d.wx, wy_count = kWarps / wx;
     const int tx = tile % d.tiles_x, ty = tile / d.tiles_x;
@@ -1147,8 +1127,8 @@ __device__ __forceinline__ void pass1_rank1_fast(const TensorDesc& d, const void
     int64_t col0 = col_w + lane * kLaneElems;
     // Maxima are idempotent: when cols % 256 == 128 the upper half-warp repeats the lower one's columns.
     if (col0 >= d.cols) col0 -= 128;
-    const float* rc_old = (phase ? d.rc[1] : d.rc[0]);
-    float* rc_new = (phase ? d.rc[0] : d.rc[1]);
+    const float* rc_old = rc_pick(d, sel.old_i);
+    float* rc_new = rc_pick(d, sel.new_i);
     const int64_t row0 = (int64_t)ty * d.tile_rows1 + warp / wx;
     const int64_t row_end = min((int64_t)(ty + 1) * d.tile_rows1, d.rows);
     if (row0 >= row_end) return;                      // uniform over the warp
@@ -1160,6 +1140,8 @@ __device__ __forceinline__ void pass1_rank1_fast(const TensorDesc& d, const void
     load8_f32(rc_old + d.c_off + col0, c_old);
     const int64_t e0 = row0 * d.cols + col0;
     P1View t;
+    t.pol = pol;
+    t.keep = keep;
     t.g = BF16 ? static_cast<const void*>(reinterpret_cast<const uint16_t*>(g) + e0)
                : static_cast<const void*>(reinterpret_cast<const float*>(g) + e0);
     t.v_codes = d.v_codes + (e0 >> 1);
@@ -1174,7 +1156,7 @@ __device__ __forceinline__ void pass1_rank1_fast(const TensorDesc& d, const void
                                 d.v_codes + (ew >> 1));
     }
 #pragma unroll
-    for (uint32_t k = 0; k < kP1L2Ahead; k += P1Pf<BF16>::kRows) prefetch_p1_group<BF16>(t, k, nrows);
+    for (uint32_t k = 0; k < kP1L2Ahead; k += P1Pf<BF16>::kRows) prefetch_p1_group<BF16, FU>(t, k, nrows);
     // Lane j keeps the old row scale of the warp's row number base + j (32 rows per refill); a row's scale is
     // then read with one shuffle instead of a load.
     float r_vec = 0.0f;
@@ -1183,26 +1165,26 @@ __device__ __forceinline__ void pass1_rank1_fast(const TensorDesc& d, const void
     // past the end re-reads that row and contributes the same values again, and the loop body has no branches.
     P1Row<BF16> s0, s1, s2, s3;
     const uint32_t last = nrows - 1;
-    load_p1_row<BF16>(s0, t, 0);
-    load_p1_row<BF16>(s1, t, min(1u, last));
-    load_p1_row<BF16>(s2, t, min(2u, last));
-    load_p1_row<BF16>(s3, t, min(3u, last));
+    load_p1_row<BF16, FU>(s0, t, 0);
+    load_p1_row<BF16, FU>(s1, t, min(1u, last));
+    load_p1_row<BF16, FU>(s2, t, min(2u, last));
+    load_p1_row<BF16, FU>(s3, t, min(3u, last));
     for (uint32_t k = 0; k < nrows; k += 4) {         // four rows per trip so that their maxima reduce together
         if ((k & 31) == 0) {
             const uint32_t kk = min(k + lane, last);
             r_vec = __ldg(rc_old + row0 + (int64_t)kk * wy_count);
         }
 #pragma unroll
-        for (uint32_t u = 0; u < 4; u += P1Pf<BF16>::kRows) prefetch_p1_group<BF16>(t, k + kP1L2Ahead + u, nrows);
+        for (uint32_t u = 0; u < 4; u += P1Pf<BF16>::kRows) prefetch_p1_group<BF16, FU>(t, k + kP1L2Ahead + u, nrows);
         float r_max[4];
         p1_process_2rows<BF16>(s0, s1, __shfl_sync(0xffffffffu, r_vec, k & 31), __shfl_sync(0xffffffffu, r_vec, (k + 1) & 31),
                                c_old, c_max, h2, lt, r_max[0], r_max[1]);
-        load_p1_row<BF16>(s0, t, min(k + 4, last));
-        load_p1_row<BF16>(s1, t, min(k + 5, last));
+        load_p1_row<BF16, FU>(s0, t, min(k + 4, last));
+        load_p1_row<BF16, FU>(s1, t, min(k + 5, last));
         p1_process_2rows<BF16>(s2, s3, __shfl_sync(0xffffffffu, r_vec, (k + 2) & 31), __shfl_sync(0xffffffffu, r_vec, (k + 3) & 31),
                                c_old, c_max, h2, lt, r_max[2], r_max[3]);
-        load_p1_row<BF16>(s2, t, min(k + 6, last));
-        load_p1_row<BF16>(s3, t, min(k + 7, last));
+        load_p1_row<BF16, FU>(s2, t, min(k + 6, last));
+        load_p1_row<BF16, FU>(s3, t, min(k + 7, last));
         const float rm = warp_max4(r_max, lane);
         const uint32_t kr = min(k + ((lane >> 4) & 1) * 2 + ((lane >> 3) & 1), last);   // the row whose maximum this lane holds
         if ((lane & 7) == 0) atomic_max_nonneg(rc_new + row0 + (int64_t)kr * wy_count, rm);
@@ -1228,7 +1210,7 @@ __device__ __forceinline__ void pass1_rank1_fast(const TensorDesc& d, const void
 // are reproducible to rounding only.
 
 template <bool BF16>
-__device__ __forceinline__ void pass1_fact(const TensorDesc& d, const void* __restrict__ g, int tile, int phase,
+__device__ __forceinline__ void pass1_fact(const TensorDesc& d, const void* __restrict__ g, int tile, RcSel sel,
                                            float* s_col) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int wx = d.wx, wy_count = kWarps / wx;
@@ -1236,7 +1218,7 @@ __device__ __forceinline__ void pass1_fact(const TensorDesc& d, const void* __re
     const int64_t col_w = (int64_t)tx * (kWarpElems * wx) + (warp % wx) * kWarpElems;
     const int64_t col0 = col_w + lane * kLaneElems;
     const bool active = col0 < d.cols;                  // cols % 256 == 128: the upper half-warp adds zeros
-    float* sums = (phase ? d.rc[0] : d.rc[1]);          // [row sums | column sums], cleared before the launch
+    float* sums = rc_pick(d, sel.new_i);          // [row sums | column sums], cleared before the launch
     const int64_t row0 = (int64_t)ty * d.tile_rows1 + warp / wx;
     const int64_t row_end = min((int64_t)(ty + 1) * d.tile_rows1, d.rows);
     float c_sum[8];
@@ -1276,8 +1258,8 @@ __device__ __forceinline__ void pass1_fact(const TensorDesc& d, const void* __re
 __global__ void __launch_bounds__(256) factor_finalize_kernel(StepArgs a, int t0) {
     const TensorDesc d = a.descs[t0 + blockIdx.x];
     if (d.kind != K_FACT) return;
-    const float* old = (a.phase ? d.rc[1] : d.rc[0]);
-    float* cur = (a.phase ? d.rc[0] : d.rc[1]);
+    const float* old = rc_pick(d, a.sel.old_i);
+    float* cur = rc_pick(d, a.sel.new_i);
     __shared__ double s_part[256];
     double part = 0.0;
     for (int64_t i = threadIdx.x; i < d.rows; i += blockDim.x) {
@@ -1299,11 +1281,11 @@ __global__ void __launch_bounds__(256) factor_finalize_kernel(StepArgs a, int t0
 #endif
 
 template <bool BF16>
-__device__ __forceinline__ void pass1_rank1_flat(const TensorDesc& d, const void* __restrict__ g, int tile, int phase,
+__device__ __forceinline__ void pass1_rank1_flat(const TensorDesc& d, const void* __restrict__ g, int tile, RcSel sel,
                                                  const Hyper& h) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const float* rc_old = (phase ? d.rc[1] : d.rc[0]);
-    float* rc_new = (phase ? d.rc[0] : d.rc[1]);
+    const float* rc_old = rc_pick(d, sel.old_i);
+    float* rc_new = rc_pick(d, sel.new_i);
     for (int c = 0; c < d.flat_chunks; ++c) {
         const int64_t chunk = ((int64_t)tile * d.flat_chunks + c) * kWarps + warp;
         const int64_t e = chunk * kWarpElems + lane * kLaneElems;
@@ -1354,13 +1336,166 @@ __global__ void __launch_bounds__(kThreads, MINB) pass1_kernel(StepArgs a) {
         const TensorDesc d = a.descs[t];
         const void* g = a.grads[t];
         const int local = tile - __ldg(a.tile_start + t);
-        if (d.kind == K_RANK1_FAST) pass1_rank1_fast<BF16>(d, g, local, a.phase, h2, lt, s_col);
-        else if (d.kind == K_FACT) pass1_fact<BF16>(d, g, local, a.phase, s_col);
-        else pass1_rank1_flat<BF16>(d, g, local, a.phase, a.h);
+        if (d.kind == K_RANK1_FAST) pass1_rank1_fast<BF16>(d, g, local, a.sel, h2, lt, s_col);
+        else if (d.kind == K_FACT) pass1_fact<BF16>(d, g, local, a.sel, s_col);
+        else pass1_rank1_flat<BF16>(d, g, local, a.sel, a.h);
         tile = a.tile_begin + tiles_next(s_next, buf, fetched);
     }
     tiles_done(a.tile_counter);
 }
+
+// ---- the fused schedule: both passes of every tensor in one launch --------------------------------------
+//
+// The launch walks an explicit work list (built on the host) whose items are tiles of the maxima pass and tiles of
+// the update pass. The update tiles of a rank-1 tensor come after all of its maxima tiles in the list, close
+// enough that the gradient and the second-moment codes read by the maxima pass are still in L2 when the update
+// pass reads them again (the loads carry eviction priorities, see L2Policies), and the list interleaves the next
+// tensor's maxima tiles with the current tensor's update tiles.
+//
+// Dependencies are counted per tensor in the arena (TensorSync). Items are handed out in list order, so whatever an
+// update tile waits for was handed out earlier to a CTA that is already running and never waits itself: the oldest
+// unfinished item always makes progress, whether or not all CTAs of the grid are resident. Every wait is bounded:
+// when it runs out the CTA records kStatusWaitTimeout in the device status word and stops taking work.
+
+constexpr uint32_t kStatusWaitTimeout = 2u;
+
+// Polls until the counter has reached `target` (compared modulo 2^32: the counters are never reset, a tensor's
+// target grows by its tile count with every launch). False when the limit ran out or another CTA has already reported
+// an error. A wait that did not succeed at the first look adds its duration to the statistics words.
+__device__ __forceinline__ bool wait_count(const uint32_t* counter, uint32_t target, uint32_t limit, const uint32_t* dev_status,
+                                           unsigned long long* stats) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
+    if ((int32_t)(v - target) >= 0) return true;
+    unsigned long long t0;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+    bool ok = false;
+    for (uint32_t it = 0; it < limit; ++it) {
+        __nanosleep(it < 64u ? 50u : 500u);
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
+        if ((int32_t)(v - target) >= 0) { ok = true; break; }
+        if ((it & 63u) == 63u && *reinterpret_cast<const volatile uint32_t*>(dev_status) != 0u) break;
+    }
+    if (stats) {
+        unsigned long long t1;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
+        atomicAdd(stats, 1ull);
+        atomicAdd(stats + 1, t1 - t0);
+    }
+    return ok;
+}
+
+template <bool BF16, bool EXACT, bool A32>
+__global__ void __launch_bounds__(kThreads, 2) step_fused_kernel(StepArgs a) {
+    __shared__ __align__(16) unsigned char s_lut[kLutSmemBytes];
+    __shared__ float s_col[kWarps * kWarpElems];
+    __shared__ float s_red[2 * kWarps];
+    __shared__ float s_rows[2 * kFusedTileRows];
+    __shared__ int s_next[2];
+    __shared__ int s_flag;
+    load_lut_smem(s_lut);
+    __syncthreads();
+    const LaneTables lt = make_lane_tables();
+    const Hyper2& h2 = a.h2;
+    uint32_t red_step = 0;
+    int buf = 0;
+    int ready_tensor = -1;     // the last tensor this CTA has seen complete its maxima pass (uniform over the CTA)
+    for (int tile = a.tile_begin + tiles_first(a.tile_counter, s_next); tile < a.tile_end;) {
+        const int fetched = tiles_fetch(a.tile_counter);
+        const uint2 item = __ldg(a.work + tile);
+        const int t = (int)(item.x & kWorkTensorMask);
+        const bool update = (item.x & kWorkUpdate) != 0, keep = (item.x & kWorkKeep) != 0;
+        const int local = (int)item.y;
+        const TensorDesc d = a.descs[t];
+        const void* g = a.grads[t];
+        TensorSync* sy = a.tsync + t;
+        const bool rank1 = d.kind == K_RANK1_FAST || d.kind == K_RANK1_FLAT;
+        if (!update) {
+            {   // this tile's share of clearing the buffer that will receive the NEXT step's maxima (nothing reads or
+                // writes it during this step)
+                float4* z = reinterpret_cast<float4*>(rc_pick(d, a.sel.zero_i));
+                const int n4 = d.rc_floats >> 2;
+                const int z0 = (int)((int64_t)n4 * local / d.tiles1), z1 = (int)((int64_t)n4 * (local + 1) / d.tiles1);
+                for (int i = z0 + (int)threadIdx.x; i < z1; i += kThreads) z[i] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            }
+            if (d.kind == K_RANK1_FAST) {
+                const L2Policies pol = make_l2_policies();
+                pass1_rank1_fast<BF16, true>(d, g, local, a.sel, h2, lt, s_col, (keep && a.l2_hints) ? pol.last : pol.normal, keep && a.l2_hints);
+                // Count the tile. The barrier orders every thread's atomic maxima before thread 0's fence, which is
+                // cumulative; nobody waits for the counter's old value.
+                __syncthreads();
+                if (threadIdx.x == 0) {
+                    __threadfence();
+                    atomicAdd(&sy->maxima_done, 1u);
+                }
+            } else {
+                // Element-indexed tensors (odd shapes, three or four axes): their update path reads the reciprocals of
+                // the new statistics from memory, so the CTA that finishes the tensor's last maxima tile inverts them
+                // and only then announces the tensor (`ready` takes the launch number).
+                pass1_rank1_flat<BF16>(d, g, local, a.sel, a.h);
+                __syncthreads();
+                if (threadIdx.x == 0) {
+                    __threadfence();
+                    s_flag = (atomicAdd(&sy->maxima_done, 1u) + 1u == a.epoch * (uint32_t)d.tiles1);
+                }
+                __syncthreads();
+                if (s_flag) {
+                    __threadfence();
+                    const float4* src = reinterpret_cast<const float4*>(rc_pick(d, a.sel.new_i));
+                    float4* dst = reinterpret_cast<float4*>(d.rcp_new);
+                    for (int i = threadIdx.x; i < (d.rc_floats >> 2); i += kThreads) {
+                        const float4 v = __ldcg(src + i);
+                        dst[i] = make_float4(scale_rcp(v.x), scale_rcp(v.y), scale_rcp(v.z), scale_rcp(v.w));
+                    }
+                    __threadfence();
+                    __syncthreads();
+                    if (threadIdx.x == 0) asm volatile("st.release.gpu.global.u32 [%0], %1;" :: "l"(&sy->ready), "r"(a.epoch) : "memory");
+                }
+            }
+        } else {
+            if (rank1 && t != ready_tensor) {
+                if (threadIdx.x == 0) {
+                    const bool ok = d.kind == K_RANK1_FAST
+                        ? wait_count(&sy->maxima_done, a.epoch * (uint32_t)d.tiles1, a.spin_limit, a.dev_status, a.wait_stats)
+                        : wait_count(&sy->ready, a.epoch, a.spin_limit, a.dev_status, a.wait_stats);
+                    if (!ok) atomicCAS(a.dev_status, 0u, kStatusWaitTimeout);
+                    s_flag = ok;
+                }
+                __syncthreads();
+                if (!s_flag) break;                // uniform over the CTA; the states of this step are incomplete
+                ready_tensor = t;
+            }
+            float* w = a.params[t];
+            switch (d.kind) {
+                case K_RANK1_FAST: {
+                    const L2Policies pol = make_l2_policies();
+                    pass2_rank1_fast<BF16, EXACT, 7, 0, false, A32, true>(d, w, nullptr, g, local, a.sel, a.h, h2, lt, s_lut, s_red, red_step,
+                                                                           a.l2_hints ? pol.first : pol.normal, s_rows);
+                    break;
+                }
+                case K_RANK1_FLAT: pass2_flat<BF16, true, EXACT, 7, false, A32, true>(d, w, nullptr, g, local, a.sel, a.h, h2, lt, s_lut, s_red, red_step); break;
+                case K_BLOCK:      pass2_flat<BF16, false, EXACT, 7, false, A32>(d, w, nullptr, g, local, a.sel, a.h, h2, lt, s_lut, s_red, red_step); break;
+                case K_FP32:       pass2_fp32<BF16, EXACT, false, A32>(d, w, nullptr, g, local, a.h); break;
+                default: break;                    // (tiled block-wise tensors have a launch of their own)
+            }
+        }
+        tile = a.tile_begin + tiles_next(s_next, buf, fetched);
+    }
+    tiles_done(a.tile_counter);
+}
+
+#if LPMM_STEP_PART == 0
+// Two CTAs wait for a count that nothing will ever reach (test hook for the bounded wait): each gives up after
+// `limit` polls, records the timeout in the status word and returns.
+__global__ void wait_selftest_kernel(const uint32_t* flag, uint32_t want, uint32_t limit, uint32_t* dev_status, int32_t* gave_up) {
+    if (threadIdx.x == 0) {
+        if (!wait_count(flag, want, limit, dev_status, nullptr)) {
+            atomicCAS(dev_status, 0u, kStatusWaitTimeout);
+            atomicAdd(gave_up, 1);
+        }
+    }
+}
+#endif
 
 // ---- compressed SGDM (Alg. 2): m = beta m + g ; w = w - lr m ; compress m. One pass, element-indexed -------
 
@@ -1512,11 +1647,6 @@ cudaError_t launch_pass2_t(const StepArgs& a, int v_kind, int grid, cudaStream_t
     } else if (a.params_bf16 != nullptr) {
         if (a.aligned32) pass2_kernel<BF16, EXACT, MSHIFT, 0, true, true><<<grid, kThreads, 0, s>>>(a);
         else pass2_kernel<BF16, EXACT, MSHIFT, 0, true, false><<<grid, kThreads, 0, s>>>(a);
-    } else if (a.variant == 1) {
-        constexpr int smem = bulk_smem_bytes<BF16>();
-        cudaError_t e = cudaFuncSetAttribute(pass2_bulk_kernel<BF16, EXACT, MSHIFT>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        if (e != cudaSuccess) return e;
-        pass2_bulk_kernel<BF16, EXACT, MSHIFT><<<grid, kThreads, smem, s>>>(a);
     } else if (a.aligned32) {
         pass2_kernel<BF16, EXACT, MSHIFT, 0, false, true><<<grid, kThreads, 0, s>>>(a);
     } else {
@@ -1530,18 +1660,29 @@ cudaError_t launch_pass2_m(const StepArgs& a, int m_shift, int v_kind, int grid,
     return m_shift == 11 ? launch_pass2_t<BF16, EXACT, 11>(a, v_kind, grid, s) : launch_pass2_t<BF16, EXACT, 7>(a, v_kind, grid, s);
 }
 
+template <bool BF16, bool EXACT>
+cudaError_t launch_fused_t(const StepArgs& a, int grid, cudaStream_t s) {
+    if (a.aligned32) step_fused_kernel<BF16, EXACT, true><<<grid, kThreads, 0, s>>>(a);
+    else step_fused_kernel<BF16, EXACT, false><<<grid, kThreads, 0, s>>>(a);
+    return cudaGetLastError();
+}
+
 // One launcher per (gradient type, update math) pair, each in its own part of the build.
 #if defined(LPMM_STEP_ALL) || LPMM_STEP_PART == 0
 cudaError_t launch_pass2_bf16_fast(const StepArgs& a, int m_shift, int v_kind, int grid, cudaStream_t s) { return launch_pass2_m<true, false>(a, m_shift, v_kind, grid, s); }
+cudaError_t launch_fused_bf16_fast(const StepArgs& a, int grid, cudaStream_t s) { return launch_fused_t<true, false>(a, grid, s); }
 #endif
 #if defined(LPMM_STEP_ALL) || LPMM_STEP_PART == 1
 cudaError_t launch_pass2_bf16_ieee(const StepArgs& a, int m_shift, int v_kind, int grid, cudaStream_t s) { return launch_pass2_m<true, true>(a, m_shift, v_kind, grid, s); }
+cudaError_t launch_fused_bf16_ieee(const StepArgs& a, int grid, cudaStream_t s) { return launch_fused_t<true, true>(a, grid, s); }
 #endif
 #if defined(LPMM_STEP_ALL) || LPMM_STEP_PART == 2
 cudaError_t launch_pass2_f32_fast(const StepArgs& a, int m_shift, int v_kind, int grid, cudaStream_t s) { return launch_pass2_m<false, false>(a, m_shift, v_kind, grid, s); }
+cudaError_t launch_fused_f32_fast(const StepArgs& a, int grid, cudaStream_t s) { return launch_fused_t<false, false>(a, grid, s); }
 #endif
 #if defined(LPMM_STEP_ALL) || LPMM_STEP_PART == 3
 cudaError_t launch_pass2_f32_ieee(const StepArgs& a, int m_shift, int v_kind, int grid, cudaStream_t s) { return launch_pass2_m<false, true>(a, m_shift, v_kind, grid, s); }
+cudaError_t launch_fused_f32_ieee(const StepArgs& a, int grid, cudaStream_t s) { return launch_fused_t<false, true>(a, grid, s); }
 #endif
 
 #if LPMM_STEP_PART == 0
@@ -1550,6 +1691,19 @@ cudaError_t launch_pass2(const StepArgs& a, bool bf16, bool exact, int m_shift, 
     if (a.tile_end <= a.tile_begin) return cudaSuccess;
     if (bf16) return exact ? launch_pass2_bf16_ieee(a, m_shift, v_kind, grid, s) : launch_pass2_bf16_fast(a, m_shift, v_kind, grid, s);
     return exact ? launch_pass2_f32_ieee(a, m_shift, v_kind, grid, s) : launch_pass2_f32_fast(a, m_shift, v_kind, grid, s);
+}
+
+// The fused schedule (rank-1 states with B128 first moments): one launch over the work list [tile_begin, tile_end).
+cudaError_t launch_fused(const StepArgs& a, bool bf16, bool exact, int grid, cudaStream_t s) {
+    if (a.tile_end <= a.tile_begin) return cudaSuccess;
+    if (bf16) return exact ? launch_fused_bf16_ieee(a, grid, s) : launch_fused_bf16_fast(a, grid, s);
+    return exact ? launch_fused_f32_ieee(a, grid, s) : launch_fused_f32_fast(a, grid, s);
+}
+
+cudaError_t launch_wait_selftest(const uint32_t* flag, uint32_t want, uint32_t limit, uint32_t* dev_status, int32_t* gave_up,
+                                 cudaStream_t s) {
+    wait_selftest_kernel<<<2, 32, 0, s>>>(flag, want, limit, dev_status, gave_up);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_factor_finalize(const StepArgs& a, int t0, int t1, cudaStream_t s) {

@@ -22,6 +22,7 @@ NORM_BLOCK, NORM_RANK1 = 0, 1
 MAP_DE_SIGNED, MAP_LINEAR_NOZERO = 0, 1
 V_RANK1, V_BLOCK, V_FACTORED = 0, 1, 2
 UPDATE_FAST, UPDATE_IEEE = 0, 1
+SCHEDULE_AUTO, SCHEDULE_TWO_PASS, SCHEDULE_FUSED = 0, 1, 2
 FORCE_QUANT, FORCE_FP32 = 1, 2
 Q_GIVEN_SCALES = 1
 KIND_FP32, KIND_BLOCK, KIND_RANK1, KIND_FACTORED = 0, 1, 2, 3
@@ -30,7 +31,8 @@ EXPORTS = ("lpmm_state_bytes", "lpmm_state_init", "lpmm_state_attach", "lpmm_ada
            "lpmm_adamw4_step_host", "lpmm_stage_bytes", "lpmm_quantize", "lpmm_dequantize",
            "lpmm_quantize_rank1_noalloc", "lpmm_sgdm4_step",
            "lpmm_state_view", "lpmm_state_view_axis", "lpmm_state_phase", "lpmm_state_last_launches", "lpmm_state_destroy",
-           "lpmm_state_profile", "lpmm_state_profile_read", "lpmm_state_device_status",
+           "lpmm_state_profile", "lpmm_state_profile_read", "lpmm_state_device_status", "lpmm_state_selftest_wait",
+           "lpmm_state_schedule", "lpmm_state_wait_stats",
            "lpmm_status_string", "lpmm_last_cuda_error")
 
 
@@ -54,11 +56,16 @@ def nd_shape(dims, flags: int = 0) -> Shape:
 
 class Config(C.Structure):
     _fields_ = [("bits", C.c_int32), ("m_block", C.c_int32), ("v_block", C.c_int32), ("v_mode", C.c_int32),
-                ("min_quant_numel", C.c_int64), ("update_math", C.c_int32), ("reserved", C.c_int32)]
+                ("min_quant_numel", C.c_int64), ("update_math", C.c_int32), ("schedule", C.c_int32),
+                ("tile_elems", C.c_int32), ("tile_elems_maxima", C.c_int32), ("l2_keep_mbytes", C.c_int32),
+                ("lead_melems", C.c_int32), ("gap_items", C.c_int32), ("no_l2_hints", C.c_int32)]
 
 
-def default_config(v_mode: int = V_RANK1, min_quant_numel: int = 4096, update_math: int = 0, m_block: int = 128) -> Config:
-    return Config(4, m_block, 128, v_mode, min_quant_numel, update_math, 0)
+def default_config(v_mode: int = V_RANK1, min_quant_numel: int = 4096, update_math: int = 0, m_block: int = 128,
+                   schedule: int = 0, tile_elems: int = 0, tile_elems_maxima: int = 0, l2_keep_mbytes: int = 0,
+                   lead_melems: int = 0, gap_items: int = 0, no_l2_hints: int = 0) -> Config:
+    return Config(4, m_block, 128, v_mode, min_quant_numel, update_math, schedule, tile_elems, tile_elems_maxima,
+                  l2_keep_mbytes, lead_melems, gap_items, no_l2_hints)
 
 
 class LpmmError(RuntimeError):
@@ -100,6 +107,9 @@ def lib():
         L.lpmm_state_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_double),
                                               C.POINTER(i32)]
         L.lpmm_state_device_status.argtypes = [vp, C.POINTER(i32), vp]
+        L.lpmm_state_selftest_wait.argtypes = [vp, C.POINTER(i32), C.POINTER(i32), vp]
+        L.lpmm_state_schedule.argtypes = [vp]
+        L.lpmm_state_wait_stats.argtypes = [vp, C.POINTER(i64), C.POINTER(i64), vp]
         L.lpmm_state_phase.argtypes = [vp]
         L.lpmm_state_last_launches.argtypes = [vp]
         L.lpmm_state_destroy.argtypes = [vp]
@@ -174,6 +184,10 @@ class State:
     @property
     def last_launches(self) -> int:
         return lib().lpmm_state_last_launches(self.handle)
+
+    @property
+    def schedule(self) -> int:
+        return lib().lpmm_state_schedule(self.handle)
 
 
 def state_init(config: Config, shapes, device="cuda", stream=None) -> State:
@@ -273,6 +287,23 @@ def device_status(state: State, stream=None) -> int:
     out = C.c_int32()
     _check(lib().lpmm_state_device_status(state.handle, C.byref(out), _stream_ptr(stream)), "lpmm_state_device_status")
     return out.value
+
+
+def selftest_wait(state: State, stream=None):
+    """lpmm_state_selftest_wait: (CTAs that gave up, status word they left)."""
+    n, w = C.c_int32(), C.c_int32()
+    with torch.cuda.device(state.arena.device):
+        _check(lib().lpmm_state_selftest_wait(state.handle, C.byref(n), C.byref(w), _stream_ptr(stream)),
+               "lpmm_state_selftest_wait")
+    return n.value, w.value
+
+
+def wait_stats(state: State, stream=None):
+    """lpmm_state_wait_stats: (waits that had to poll, their summed nanoseconds) since the last call."""
+    n, ns = C.c_int64(), C.c_int64()
+    with torch.cuda.device(state.arena.device):
+        _check(lib().lpmm_state_wait_stats(state.handle, C.byref(n), C.byref(ns), _stream_ptr(stream)), "lpmm_state_wait_stats")
+    return n.value, ns.value
 
 
 def stage_bytes(state: State) -> int:

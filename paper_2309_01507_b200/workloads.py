@@ -153,6 +153,8 @@ WORKLOADS = {
     # reduced LLaMA list (embedding, head and a few decoder layers) for profiler captures and quick checks
     "llama_7b_1l": lambda: llama_7b(layers=1),
     "llama_7b_4l": lambda: llama_7b(layers=4),
+    # four decoder layers with a token table of 1024 rows: 0.82 G parameters, the matrices of the decoder alone
+    "llama_7b_4l_1kv": lambda: llama_7b(layers=4, vocab=1024),
 }
 
 

@@ -22,10 +22,13 @@ def param_tol(w_ref: np.ndarray, lr: float, tol: float) -> np.ndarray:
 class Pair:
     """The same tensors held by the CUDA library (device) and by the oracle (host)."""
 
-    def __init__(self, specs, hyper, *, config=None, device="cuda", grad_dtype=torch.float32, workload_index=9):
+    def __init__(self, specs, hyper, *, config=None, device="cuda", grad_dtype=torch.float32, workload_index=9,
+                 schedule=None):
         self.specs = list(specs)
         self.hyper = dict(hyper)
         self.config = config or lpmm.default_config()
+        if schedule is not None:
+            self.config.schedule = schedule
         self.grad_dtype = grad_dtype
         self.widx = workload_index
         self.params = [workloads.make_param(s, self.widx, i, device=device) for i, s in enumerate(self.specs)]

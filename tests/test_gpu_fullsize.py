@@ -12,7 +12,8 @@ from parity_util import ORACLE_KIND, hyper_of
 pytestmark = pytest.mark.gpu
 
 
-def test_llama_7b_full_size_sampled_tensors():
+@pytest.mark.parametrize("schedule", [lpmm.SCHEDULE_AUTO, lpmm.SCHEDULE_FUSED], ids=["auto", "fused"])
+def test_llama_7b_full_size_sampled_tensors(schedule):
     free, _ = torch.cuda.mem_get_info()
     if free < 60 * 2 ** 30:
         pytest.skip("needs about 50 GB of free device memory")
@@ -20,7 +21,7 @@ def test_llama_7b_full_size_sampled_tensors():
     hyper = hyper_of(wl)
     dev = "cuda"
     params = [workloads.make_param(t, wl.index, i, device=dev) for i, t in enumerate(wl.tensors)]
-    state = lpmm.state_init(lpmm.default_config(), wl.tensors, device=dev)
+    state = lpmm.state_init(lpmm.default_config(schedule=schedule), wl.tensors, device=dev)
     names = {t.name: i for i, t in enumerate(wl.tensors)}
     sample = [names[n] for n in ("embed", "l0.q", "l17.gate", "l31.down", "l5.norm1", "lm_head")]
     w_ref = {i: params[i].detach().cpu().numpy().ravel().copy() for i in sample}
@@ -37,7 +38,7 @@ def test_llama_7b_full_size_sampled_tensors():
         for i in sample:
             oracle.adamw4_step(w_ref[i], grads[i].float().cpu().numpy().ravel(), ostate[i], step=step, **hyper)
         del grads
-    assert state.last_launches == 3
+    assert state.last_launches == (1 if schedule == lpmm.SCHEDULE_FUSED else 3)
     for i in sample:
         t = wl.tensors[i]
         view = lpmm.state_view(state, i)

@@ -18,6 +18,14 @@ pytestmark = pytest.mark.gpu
 TDE = oracle.de_map(4, True)
 TLIN = oracle.linear_map(4)
 
+# Both orders of the work inside a step (maxima pass and update pass as separate launches, or one fused launch whose
+# tiles wait for one another) must give the same bits: the tests of the default quantizers run under each.
+SCHEDULES = pytest.mark.parametrize("schedule", [lpmm.SCHEDULE_TWO_PASS, lpmm.SCHEDULE_FUSED], ids=["two_pass", "fused"])
+
+
+def _launches(schedule, two_pass):
+    return 1 if schedule == lpmm.SCHEDULE_FUSED else two_pass
+
 
 def _mat(r, c, **kw):
     return TensorSpec(f"m{r}x{c}", r, c, 2, **kw)
@@ -99,10 +107,13 @@ def test_rank1_quantizer_matches_oracle(rows, cols):
 
 # ------------------------------------------------------------------ the fused step
 
+@SCHEDULES
 @pytest.mark.parametrize("update_math", [lpmm.UPDATE_FAST, lpmm.UPDATE_IEEE])
-def test_single_matrix_config_ten_steps(update_math):
+def test_single_matrix_config_ten_steps(update_math, schedule):
     wl = workloads.single_matrix()
-    pair = Pair(wl.tensors, hyper_of(wl), workload_index=wl.index, config=lpmm.default_config(update_math=update_math))
+    pair = Pair(wl.tensors, hyper_of(wl), workload_index=wl.index, config=lpmm.default_config(update_math=update_math),
+                schedule=schedule)
+    assert pair.state.schedule == schedule
     kinds = [lpmm.state_view(pair.state, i)["kind"] for i in range(2)]
     assert kinds == [lpmm.KIND_RANK1, lpmm.KIND_BLOCK]          # bias forced onto the quantized 1-D path
     seen_v, seen_m = set(), set()
@@ -113,18 +124,20 @@ def test_single_matrix_config_ten_steps(update_math):
         seen_m |= set(np.unique(oracle.unpack4(pair.ostate[0].m_codes, 1024 * 4096)).tolist())
         seen_v |= set(np.unique(oracle.unpack4(pair.ostate[0].v_codes, 1024 * 4096)).tolist())
     assert seen_m == set(range(16)) and seen_v == set(range(16))
-    assert pair.state.last_launches == 3
+    assert pair.state.last_launches == _launches(schedule, 3)
 
 
 @pytest.mark.parametrize("grad_dtype,update_math", [(torch.float32, lpmm.UPDATE_FAST), (torch.bfloat16, lpmm.UPDATE_FAST),
                                                     (torch.float32, lpmm.UPDATE_IEEE)])
-def test_shape_zoo_multi_tensor(grad_dtype, update_math):
+@SCHEDULES
+def test_shape_zoo_multi_tensor(grad_dtype, update_math, schedule):
     specs = [_mat(96, 256), _mat(33, 77), _mat(5, 1000), _mat(130, 384), _mat(64, 1024), _mat(8, 2048),
              _mat(1, 8192), _mat(8192, 1), _mat(300, 640), _mat(257, 129), _mat(70, 128),
              _vec(50265), _vec(4097), _vec(4096), _vec(4096, force_quant=True), _vec(1), _vec(300),
              _mat(16, 16), _mat(64, 64), _mat(65, 64), _vec(12345)]
     hyper = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
-    pair = Pair(specs, hyper, grad_dtype=grad_dtype, workload_index=7, config=lpmm.default_config(update_math=update_math))
+    pair = Pair(specs, hyper, grad_dtype=grad_dtype, workload_index=7, config=lpmm.default_config(update_math=update_math),
+                schedule=schedule)
     for t in range(1, 6):
         grads = pair.grads_for(t, outlier_p=0.0 if t % 2 == 0 else 1e-3)
         if t == 3:
@@ -165,24 +178,26 @@ def test_first_moment_block_2048(grad_dtype):
     assert pair.ostate[0].m_scale.size == 64     # one scale per 2048 elements
 
 
-def test_transformer_base_three_steps_one_launch_per_pass():
+@SCHEDULES
+def test_transformer_base_three_steps_one_launch_per_pass(schedule):
     wl = workloads.transformer_base()
-    pair = Pair(wl.tensors, hyper_of(wl), workload_index=wl.index)
+    pair = Pair(wl.tensors, hyper_of(wl), workload_index=wl.index, schedule=schedule)
     kinds = [lpmm.state_view(pair.state, i)["kind"] for i in range(len(wl.tensors))]
     assert kinds.count(lpmm.KIND_RANK1) == 61 and kinds.count(lpmm.KIND_FP32) == 120
     for t in range(1, 4):
         pair.step(t, pair.grads_for(t))
         pair.compare(tol=1e-6)
-    assert pair.state.last_launches == 3        # pass 1 + reciprocal + pass 2 cover all 181 tensors
+    assert pair.state.last_launches == _launches(schedule, 3)   # two-pass: maxima + reciprocal + update cover all 181 tensors
 
 
-def test_sparse_token_rows_and_lm_head_bias():
+@SCHEDULES
+def test_sparse_token_rows_and_lm_head_bias(schedule):
     # RoBERTa-shaped slice: token-sparse embedding gradients (90% of rows zero) and the odd-length 50265 bias.
     specs = [TensorSpec("emb.word", 50265, 1024, 2, sparse_rows=0.9), TensorSpec("emb.pos", 514, 1024, 2),
              TensorSpec("emb.type", 1, 1024, 2), _vec(1024), TensorSpec("fc1", 4096, 1024, 2),
              TensorSpec("head.bias", 50265, 1, 1)]
     hyper = dict(lr=1e-5, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
-    pair = Pair(specs, hyper, workload_index=2)
+    pair = Pair(specs, hyper, workload_index=2, schedule=schedule)
     for t in range(1, 4):
         pair.step(t, pair.grads_for(t))
         pair.compare(tol=1e-6)
@@ -190,10 +205,11 @@ def test_sparse_token_rows_and_lm_head_bias():
     assert np.sum(r == 0) > 0.5 * r.size * 0.9 ** 3      # rows never touched keep scale 0 and dequantize to 0
 
 
-def test_trajectory_100_steps():
+@SCHEDULES
+def test_trajectory_100_steps(schedule):
     specs = [_mat(256, 1024), _vec(8192)]
     hyper = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
-    pair = Pair(specs, hyper, workload_index=5)
+    pair = Pair(specs, hyper, workload_index=5, schedule=schedule)
     for t in range(1, 101):
         pair.step(t, pair.grads_for(t))
         if t % 25 == 0 or t < 3:
@@ -201,27 +217,78 @@ def test_trajectory_100_steps():
     pair.compare(tol=1e-4, share_params=False)
 
 
-def test_checkpoint_attach_resumes_bit_exactly():
-    specs = [_mat(128, 512), _vec(5000), _vec(100)]
+@pytest.mark.parametrize("sched_a,sched_b", [(lpmm.SCHEDULE_TWO_PASS, lpmm.SCHEDULE_TWO_PASS), (lpmm.SCHEDULE_FUSED, lpmm.SCHEDULE_FUSED),
+                                             (lpmm.SCHEDULE_TWO_PASS, lpmm.SCHEDULE_FUSED), (lpmm.SCHEDULE_FUSED, lpmm.SCHEDULE_TWO_PASS)])
+def test_checkpoint_attach_resumes_bit_exactly(sched_a, sched_b):
+    # 50 steps, save, 50 more; against: restore the copy (into a state that may run the other schedule) and 50 steps.
+    specs = [_mat(128, 512), _mat(130, 384), _vec(5000), _vec(100)]
     hyper = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
-    a = Pair(specs, hyper, workload_index=6)
-    for t in range(1, 4):
-        a.step(t, a.grads_for(t))
-    arena_copy = a.state.arena.clone()
+    a = Pair(specs, hyper, workload_index=6, schedule=sched_a)
+    for t in range(1, 51):
+        lpmm.adamw4_step(a.state, a.params, a.grads_for(t), step=t, **hyper)
+    saved = a.state.arena.clone()
     phase = a.state.phase
     params_copy = [p.clone() for p in a.params]
-    for t in range(4, 7):
-        a.step(t, a.grads_for(t))
-    resumed = lpmm.state_attach(a.config, specs, arena_copy, phase)
-    for t in range(4, 7):
+    for t in range(51, 101):
+        lpmm.adamw4_step(a.state, a.params, a.grads_for(t), step=t, **hyper)
+    cfg_b = lpmm.default_config(schedule=sched_b)
+    arena_b = torch.zeros(lpmm.state_bytes(cfg_b, specs), dtype=torch.uint8, device="cuda")
+    k = min(saved.numel(), arena_b.numel())
+    arena_b[:k] = saved[:k]
+    resumed = lpmm.state_attach(cfg_b, specs, arena_b, phase)
+    assert resumed.schedule == sched_b
+    for t in range(51, 101):
         lpmm.adamw4_step(resumed, params_copy, a.grads_for(t), step=t, **hyper)
     torch.cuda.synchronize()
+    assert lpmm.device_status(a.state) == 0 and lpmm.device_status(resumed) == 0
     for i in range(len(specs)):
         va, vb = lpmm.state_view(a.state, i), lpmm.state_view(resumed, i)
         for k in ("m_codes", "m_scale", "v_codes", "v_s0", "v_s1", "m32", "v32"):
             if va[k] is not None:
                 assert torch.equal(va[k], vb[k]), (i, k)
         assert torch.equal(a.params[i], params_copy[i])
+
+
+def test_attach_refuses_an_arena_that_is_something_else():
+    specs = [_mat(128, 512), _vec(5000)]
+    cfg = lpmm.default_config()
+    st = lpmm.state_init(cfg, specs)
+    torch.cuda.synchronize()
+    good = st.arena.clone()
+    assert lpmm.state_attach(cfg, specs, good.clone(), 0).n == 2
+    cases = {
+        "not an arena": torch.zeros_like(good),
+        "other shapes": (good.clone(), [_mat(128, 512), _vec(5001)]),
+        "other block size": (good.clone(), specs, lpmm.default_config(m_block=2048)),
+    }
+    for name, case in cases.items():
+        arena, shp, c = (case, specs, cfg) if torch.is_tensor(case) else (case + (cfg,))[:3]
+        big = torch.zeros(max(arena.numel(), lpmm.state_bytes(c, shp)), dtype=torch.uint8, device="cuda")
+        big[:arena.numel()] = arena
+        with pytest.raises(lpmm.LpmmError) as ei:
+            lpmm.state_attach(c, shp, big, 0)
+        assert ei.value.status == lpmm.ERR_INVALID_ARG, name
+    bad_version = good.clone()
+    bad_version[36] += 1                 # the layout-version word of the header
+    with pytest.raises(lpmm.LpmmError) as ei:
+        lpmm.state_attach(cfg, specs, bad_version, 0)
+    assert ei.value.status == lpmm.ERR_INVALID_ARG
+    with pytest.raises(lpmm.LpmmError) as ei:
+        lpmm.state_attach(cfg, specs, good.clone(), 3)       # phases are 0, 1, 2
+    assert ei.value.status == lpmm.ERR_INVALID_ARG
+
+
+def test_bounded_wait_gives_up_and_reports():
+    # The fused schedule's CTAs wait for one another with a limit; here two CTAs wait for a counter nothing advances.
+    st = lpmm.state_init(lpmm.default_config(schedule=lpmm.SCHEDULE_FUSED), [_mat(128, 512)])
+    gave_up, word = lpmm.selftest_wait(st)
+    assert gave_up == 2 and word == 2
+    assert lpmm.device_status(st) == 0          # the self-test cleans up after itself
+    p = torch.zeros(128, 512, device="cuda")
+    g = torch.ones(128, 512, device="cuda")
+    lpmm.adamw4_step(st, [p], [g], step=1, lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0)
+    torch.cuda.synchronize()
+    assert lpmm.device_status(st) == 0 and torch.all(p < 0)
 
 
 def test_host_buffer_step_matches_device_step():
@@ -345,12 +412,13 @@ def _nd(*dims):
     return workloads.TensorSpec("t" + "x".join(map(str, dims)), rows, dims[-1], len(dims), dims=tuple(dims))
 
 
+@SCHEDULES
 @pytest.mark.parametrize("grad_dtype,update_math", [(torch.float32, lpmm.UPDATE_IEEE), (torch.bfloat16, lpmm.UPDATE_FAST)])
-def test_tensors_with_three_and_four_axes_match_oracle(grad_dtype, update_math):
+def test_tensors_with_three_and_four_axes_match_oracle(grad_dtype, update_math, schedule):
     # Alg. 4 in its general form: one vector of maxima per axis, scale = minimum over the element's axes.
     # Codes, block scales and every axis' statistics bit-exact; parameters bit-exact with IEEE update math,
     # within 1e-6 * max(|w|, lr) with the approximate one. A matrix rides along to cover mixed lists.
-    cfg = lpmm.default_config(update_math=update_math)
+    cfg = lpmm.default_config(update_math=update_math, schedule=schedule)
     specs = [_nd(6, 10, 200), _nd(3, 5, 7, 64), _nd(16, 33, 9), _mat(96, 256), _nd(2, 4099, 3), _nd(1, 40, 128)]
     hyper = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
     params = [workloads.make_param(s, 14, i, device="cuda") for i, s in enumerate(specs)]
@@ -417,7 +485,7 @@ def test_bf16_copy_of_the_parameters(grad_dtype, m_block):
             want = oracle.f32_to_bf16_bits(pb[i].cpu().numpy().ravel())
             got = copies[i].view(torch.int16).cpu().numpy().view(np.uint16)
             assert np.array_equal(got, want), (s.name, t)
-    assert sb.last_launches == 4
+    assert sb.last_launches == 4     # (the bfloat16 copy always runs the two-pass schedule)
     # refused with the factorized second moment, and with a missing pointer array
     sf = lpmm.state_init(lpmm.default_config(v_mode=lpmm.V_FACTORED), [_mat(96, 256)])
     with pytest.raises(lpmm.LpmmError) as ei:
@@ -425,11 +493,12 @@ def test_bf16_copy_of_the_parameters(grad_dtype, m_block):
     assert ei.value.status == lpmm.ERR_UNSUPPORTED
 
 
+@SCHEDULES
 @pytest.mark.parametrize("grad_dtype", [torch.bfloat16, torch.float32])
-def test_pointers_aligned_to_16_but_not_32_bytes_give_the_same_result(grad_dtype):
+def test_pointers_aligned_to_16_but_not_32_bytes_give_the_same_result(grad_dtype, schedule):
     # The tiled update pass moves a lane's eight fp32 values with one 256-bit access when every pointer is 32-byte
     # aligned and with two 128-bit accesses otherwise; both must leave identical parameters and states.
-    cfg = lpmm.default_config()
+    cfg = lpmm.default_config(schedule=schedule)
     specs = [_mat(96, 256), _mat(64, 1024), _mat(130, 384), _vec(5000)]
     hyper = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
     pa = [workloads.make_param(s, 16, i, device="cuda") for i, s in enumerate(specs)]
@@ -473,5 +542,7 @@ def test_long_one_dimensional_tensors_folded_into_rows(grad_dtype, m_block, v_mo
             grads[0][:70000] = 0
         pair.step(t, grads)
         pair.compare(tol=1e-6)
-    want = 4 if v_mode == lpmm.V_RANK1 else 1     # maxima + reciprocal + update (+ the folded tensors' own update launch)
+    # two-pass: maxima + reciprocal + update (+ the folded tensors' own update launch); this small list of the default
+    # quantizers runs the fused schedule: one launch + the folded tensors' own
+    want = {(128, lpmm.V_RANK1): 2, (2048, lpmm.V_RANK1): 4}.get((m_block, v_mode), 1)
     assert pair.state.last_launches == want
