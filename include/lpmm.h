@@ -222,7 +222,9 @@ lpmm_status lpmm_quantize(const float* d_x, int64_t rows, int64_t cols, int32_t 
  *    and returns LPMM_ERR_TOO_LARGE. The array costs LPMM_NOALLOC_MAX_SCALES * 4 bytes (1 MiB) of device
  *    memory on every GPU that loads the library, from load until the process exits.
  *  - The first call on each device looks up the array's device address (a host-side query, no allocation).
- *    Make that first call before starting any stream capture on that device.
+ *    Make that first call before starting any stream capture on that device. The address is remembered per
+ *    device for the life of the process and does not survive cudaDeviceReset(): do not call this function
+ *    again after a reset of a device it has already been used on.
  *  - All calls on a device share the one array and it keeps whatever the last call left there. Nothing
  *    in it needs to start at zero (each call overwrites the part it uses before reading it; the outputs
  *    d_scale0 / d_scale1 are cleared by the call itself). Two calls that overlap on the GPU - different

@@ -349,8 +349,22 @@ def quantize(x: torch.Tensor, norm: int, map_: int, block: int = 128, scales=Non
 
 
 def quantize_rank1_noalloc(x: torch.Tensor, codes: torch.Tensor, r: torch.Tensor, c: torch.Tensor, stream=None) -> None:
-    """lpmm_quantize_rank1_noalloc: the caller supplies the input and all three outputs; nothing is allocated."""
+    """lpmm_quantize_rank1_noalloc: the caller supplies the input and all three outputs; nothing is allocated.
+
+    The C entry point only sees raw pointers, so the buffers are checked here: x a contiguous 2-D fp32 CUDA tensor,
+    codes uint8 with at least ceil(rows*cols/2) bytes, r and c contiguous fp32 with at least rows / cols elements, all
+    on x's device. Anything else raises ValueError before the library is called."""
+    if x.dim() != 2 or x.dtype != torch.float32 or not x.is_cuda or not x.is_contiguous():
+        raise ValueError("x must be a contiguous 2-D fp32 CUDA tensor")
     rows, cols = x.shape
+    if rows <= 0 or cols <= 0:
+        raise ValueError("x must not be empty")
+    for name, t, dtype, need in (("codes", codes, torch.uint8, (rows * cols + 1) // 2), ("r", r, torch.float32, rows),
+                                 ("c", c, torch.float32, cols)):
+        if t.dtype != dtype or not t.is_cuda or not t.is_contiguous() or t.device != x.device:
+            raise ValueError(f"{name} must be a contiguous {dtype} CUDA tensor on x's device")
+        if t.numel() < need:
+            raise ValueError(f"{name} holds {t.numel()} elements, {need} are needed")
     with torch.cuda.device(x.device):
         _check(lib().lpmm_quantize_rank1_noalloc(x.data_ptr(), rows, cols, codes.data_ptr(), r.data_ptr(),
                                                  c.data_ptr(), _stream_ptr(stream)), "lpmm_quantize_rank1_noalloc")

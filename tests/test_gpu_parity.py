@@ -11,7 +11,7 @@ import torch
 import oracle
 from paper_2309_01507_b200 import lpmm, workloads
 from paper_2309_01507_b200.workloads import TensorSpec
-from parity_util import Pair, hyper_of
+from parity_util import ORACLE_KIND, Pair, hyper_of
 
 pytestmark = pytest.mark.gpu
 
@@ -105,6 +105,75 @@ def test_rank1_quantizer_matches_oracle(rows, cols):
     assert torch.equal(r, r2) and torch.equal(c, c2) and torch.equal(codes, codes2)
 
 
+def _hot_path_probe():
+    """Gradients that put the step's own quantizers (the table-driven signed search and the round-up linear rule) on,
+    just below and just above every decision threshold: with beta1 = beta2 = 0, Eq. 1 gives m_t = g and v_t = g*g."""
+    pts = []
+    for a, b in zip(TDE[:-1], TDE[1:]):                      # first moment: g itself around each midpoint
+        p = np.float32((float(a) + float(b)) / 2)
+        for _ in range(6):
+            p = np.nextafter(p, np.float32(-np.inf), dtype=np.float32)
+        for _ in range(13):
+            pts.append(float(p))
+            p = np.nextafter(p, np.float32(np.inf), dtype=np.float32)
+    for a, b in zip(TLIN[:-1], TLIN[1:]):                    # second moment: g around the square root of each midpoint
+        p = np.float32(np.sqrt((float(a) + float(b)) / 2))
+        for _ in range(8):
+            p = np.nextafter(p, np.float32(-np.inf), dtype=np.float32)
+        for _ in range(17):
+            pts.append(float(p))
+            pts.append(-float(p))
+            p = np.nextafter(p, np.float32(np.inf), dtype=np.float32)
+    pts += [float(t) for t in TDE] + [0.0, -0.0, 1e-30, -1e-30, 1e-45, 0.99999994, -0.99999994]
+    rng = np.random.default_rng(1)
+    pts += list(rng.uniform(-1.0, 1.0, 2000))
+    return np.array(pts, dtype=np.float32)
+
+
+@pytest.mark.parametrize("layout", ["vector", "long_vector", "matrix"])
+@pytest.mark.parametrize("step_kind", ["adamw_two_pass", "adamw_fused", "sgdm"])
+def test_step_quantizers_at_every_threshold(layout, step_kind):
+    # One 1.0 per 128-block (and per row and column of the matrix) makes every scale exactly 1, so n = m_t and n = v_t.
+    x = _hot_path_probe()
+    per = 127
+    nblk = -(-x.size // per)
+    if layout == "long_vector":
+        nblk = max(nblk, 65536 // 128)                      # long enough to be folded onto the tiled path
+    g = np.zeros((nblk, 128), np.float32)
+    g[:, 0] = 1.0
+    flat = np.resize(x, nblk * per)
+    g[:, 1:] = flat.reshape(nblk, per)
+    if layout == "matrix":
+        g[0, :] = 1.0                                       # every column maximum is 1 as well
+        spec = _mat(nblk, 128, force_quant=True)
+    else:
+        spec = _vec(nblk * 128, force_quant=True)
+    gt = torch.from_numpy(g.reshape(spec.shape)).cuda()
+    w = torch.zeros(spec.shape, device="cuda")
+    sched = lpmm.SCHEDULE_FUSED if step_kind == "adamw_fused" else lpmm.SCHEDULE_TWO_PASS
+    st = lpmm.state_init(lpmm.default_config(schedule=sched), [spec])
+    kind = ORACLE_KIND[lpmm.state_view(st, 0)["kind"]]
+    ost = oracle.state_init(spec.rows, spec.cols, kind)
+    w_ref = np.zeros(spec.numel, np.float32)
+    if step_kind == "sgdm":
+        lpmm.sgdm4_step(st, [w], [gt], lr=0.0, beta=0.0)
+        oracle.sgdm4_step(w_ref, g.ravel(), ost, lr=0.0, beta=0.0)
+        names = ("m_codes", "m_scale")
+    else:
+        hyper = dict(lr=0.0, beta1=0.0, beta2=0.0, eps=1e-8, weight_decay=0.0)
+        lpmm.adamw4_step(st, [w], [gt], step=1, **hyper)
+        oracle.adamw4_step(w_ref, g.ravel(), ost, step=1, **hyper)
+        names = ("m_codes", "m_scale", "v_codes", "v_s0", "v_s1")
+    torch.cuda.synchronize()
+    view = lpmm.state_view(st, 0)
+    assert np.all(ost.m_scale == 1.0)
+    for name in names:
+        ref = getattr(ost, name)
+        if ref is not None:
+            assert np.array_equal(view[name].cpu().numpy(), ref), name
+    assert len(np.unique(oracle.unpack4(ost.m_codes, spec.numel))) == 16
+
+
 # ------------------------------------------------------------------ the fused step
 
 @SCHEDULES
@@ -153,15 +222,21 @@ def test_shape_zoo_multi_tensor(grad_dtype, update_math, schedule):
         pair.compare(tol=1e-6)
 
 
-def test_block_mode_for_matrices():
-    cfg = lpmm.default_config(v_mode=lpmm.V_BLOCK)
-    specs = [_mat(96, 256), _mat(133, 77), _mat(512, 1024)]
+@pytest.mark.parametrize("m_block,grad_dtype", [(128, torch.float32), (128, torch.bfloat16), (2048, torch.bfloat16),
+                                                (2048, torch.float32)])
+def test_block_mode_for_matrices(m_block, grad_dtype):
+    # Block-wise second moments on matrices (the B128/Linear rows of the ablation, Tab. 1), with both first-moment block
+    # sizes and both gradient types: matrices whose rows hold whole blocks ride the tiled kernel, the others the
+    # element-indexed one.
+    cfg = lpmm.default_config(v_mode=lpmm.V_BLOCK, m_block=m_block)
+    specs = [_mat(96, 256), _mat(133, 77), _mat(512, 1024), _mat(24, 4096), _mat(64, 2048), _vec(70016)]
     hyper = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0)
-    pair = Pair(specs, hyper, config=cfg, workload_index=8)
-    assert all(lpmm.state_view(pair.state, i)["kind"] == lpmm.KIND_BLOCK for i in range(3))
+    pair = Pair(specs, hyper, config=cfg, workload_index=8, grad_dtype=grad_dtype)
+    assert all(lpmm.state_view(pair.state, i)["kind"] == lpmm.KIND_BLOCK for i in range(len(specs)))
     for t in range(1, 4):
-        pair.step(t, pair.grads_for(t))
+        pair.step(t, pair.grads_for(t, outlier_p=0.0 if t == 2 else 1e-3))
         pair.compare(tol=1e-6)
+    assert pair.state.last_launches == 1
 
 
 @pytest.mark.parametrize("grad_dtype", [torch.float32, torch.bfloat16])
@@ -356,13 +431,15 @@ def test_sgdm_step_matches_oracle_bit_for_bit(grad_dtype, m_block):
     assert state.last_launches == 1
 
 
-@pytest.mark.parametrize("grad_dtype", [torch.float32, torch.bfloat16])
-def test_factorized_second_moment_matches_oracle(grad_dtype):
+@pytest.mark.parametrize("grad_dtype,m_block", [(torch.float32, 128), (torch.bfloat16, 128), (torch.bfloat16, 2048)])
+def test_factorized_second_moment_matches_oracle(grad_dtype, m_block):
     # "4-bit Factor": m in 4 bits (bit-exact), v reconstructed from fp32 row/column statistics whose sums the GPU
     # accumulates in binary32 in another order than the oracle's binary64: R, C within 1e-5, parameters within
     # 2e-5 * max(|w|, lr) (the update moves with 1/sqrt(v)); 1-D and small tensors behave as in the default mode.
-    cfg = lpmm.default_config(v_mode=lpmm.V_FACTORED)
+    cfg = lpmm.default_config(v_mode=lpmm.V_FACTORED, m_block=m_block)
     specs = [_mat(96, 256), _mat(40, 1024), _mat(130, 384), _mat(33, 77), _vec(50265), _vec(300), _mat(64, 128)]
+    if m_block == 2048:      # rows must hold whole first-moment blocks
+        specs = [_mat(24, 4096), _mat(40, 2048), _mat(7, 6144), _mat(33, 77), _vec(50265), _vec(300), _mat(64, 2048)]
     hyper = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
     params = [workloads.make_param(s, 13, i, device="cuda") for i, s in enumerate(specs)]
     state = lpmm.state_init(cfg, specs)
@@ -373,7 +450,7 @@ def test_factorized_second_moment_matches_oracle(grad_dtype):
     ost, Rs, Cs = [], [], []
     for i, s in enumerate(specs):
         k = {lpmm.KIND_FACTORED: oracle.RANK1, lpmm.KIND_FP32: oracle.FP32, lpmm.KIND_BLOCK: oracle.BLOCK}[kinds[i]]
-        ost.append(oracle.state_init(s.rows, s.cols, k))
+        ost.append(oracle.state_init(s.rows, s.cols, k, m_block=m_block))
         Rs.append(np.zeros(s.rows, np.float32)); Cs.append(np.zeros(s.cols, np.float32))
     for t in range(1, 6):
         grads = [workloads.make_grad(s, 13, i, t, device="cuda", dtype=grad_dtype) for i, s in enumerate(specs)]
