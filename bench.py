@@ -38,6 +38,10 @@ PASS1_BYTES = {"bf16": 2.5, "f32": 4.5}
 # profiles/pass2_llama_7b_1l.txt (3.2950 GB read + 2.2835 GB written); traffic scales with the parameter count.
 # fp32 gradients: capture of the RoBERTa-large list (355.4 M params, 3.2749 GB read + 1.7452 GB written), same file.
 PASS2_TRAFFIC_BYTES_PER_PARAM = {"bf16": 12.009, "f32": 14.125}
+# DRAM traffic of the whole step per parameter by schedule (ncu, same metrics): two-pass = the update pass above plus
+# the maxima pass (2.503 B/param, profiles/pass1_llama_7b_1l.txt); fused = one launch, from the capture of the
+# four-decoder-layer LLaMA slice summarised in profiles/step_fused_llama_7b_4l.txt.
+STEP_TRAFFIC_BYTES_PER_PARAM = {"two_pass": {"bf16": 14.512}, "fused": {"bf16": None}}
 
 
 def parse_args():
@@ -141,48 +145,68 @@ class ClockSampler:
 
 # ----------------------------------------------------------------------------- oracle legs
 
-def oracle_sample(wl):
-    """The bounded sample of the workload the CPU oracle is timed on: its largest repeated group of
-    matrices (one attention block of the LLaMA list), or the whole list when that is small."""
-    mats = [(i, t) for i, t in enumerate(wl.tensors) if t.ndim == 2 and t.numel > 4096]
+def oracle_sample(wl, small: bool = False, budget: int = 350_000_000):
+    """The bounded sample of the workload the CPU oracle is timed on. Lists of up to 80 M parameters: all of it. The
+    LLaMA list: the token embedding plus every tensor of one decoder layer (333 M parameters); other large lists: their
+    first tensors up to about 350 M parameters. A smaller `budget` (parameters per step) drops tensors from the end of
+    that sample. small=True: the first large matrix only (for the single-thread leg)."""
+    items = list(enumerate(wl.tensors))
+    if small:
+        mats = [(i, t) for i, t in items if t.ndim >= 2 and t.numel >= 1 << 20] or items
+        i, t = mats[1] if len(mats) > 1 else mats[0]
+        return [(i, t)], f"one tensor ({t.name}, {t.rows}x{t.cols})"
     if wl.numel <= 80_000_000:
-        return list(enumerate(wl.tensors)), "whole workload"
+        return items, "whole workload"
+    if wl.name.startswith("llama_7b") and not wl.name.endswith("flat"):
+        cand = [(i, t) for i, t in items if t.name.startswith("l0.")] + [(i, t) for i, t in items if t.name == "embed"]
+        if sum(t.numel for _, t in cand) <= budget:
+            return cand, "every tensor of one decoder layer + the token embedding"
+        label = "tensors of one decoder layer"
+    else:
+        cand, label = items, "tensors of the list"
     picked, total = [], 0
-    for i, t in mats[1:]:
-        if total + t.numel > 70_000_000:
+    for i, t in cand:
+        if total + t.numel > budget and picked:
             break
         picked.append((i, t))
         total += t.numel
-    return picked, f"{len(picked)} matrices of one layer ({', '.join(f'{t.rows}x{t.cols}' for _, t in picked)})"
+    return picked, f"the first {len(picked)} {label} ({', '.join(sorted({f'{t.rows}x{t.cols}' for _, t in picked if t.numel > 4096}))})"
 
 
-def time_oracle(wl, steps: int, warmup: int):
+def time_oracle(wl, steps: int, warmup: int, threads: int | None = None, small: bool = False, budget: int = 350_000_000):
     """Runs the oracle as it stands on the sample; returns (Gparams/s, threads, description, ms/step)."""
     import numpy as np
     import torch
     import oracle
     from paper_2309_01507_b200 import workloads
-    sample, desc = oracle_sample(wl)
+    sample, desc = oracle_sample(wl, small, budget)
     hyper = dict(lr=wl.lr, beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps, weight_decay=wl.weight_decay)
     gdt = torch.bfloat16 if wl.grad_dtype == "bf16" else torch.float32
-    ws, gs, sts = [], [], []
-    for i, t in sample:
-        ws.append(workloads.make_param(t, wl.index, i).numpy().ravel().copy())
-        gs.append(workloads.make_grad(t, wl.index, i, 1, dtype=gdt).float().numpy().ravel())
-        sts.append(oracle.state_init(t.rows, t.cols, oracle.kind_of(t.rows, t.cols, t.ndim, 4096, int(t.force_quant))))
-    n = sum(t.numel for _, t in sample)
-    step = 0
-    for _ in range(warmup):
-        step += 1
-        for w, g, st in zip(ws, gs, sts):
-            oracle.adamw4_step(w, g, st, step=step, **hyper)
-    t0 = time.perf_counter()
-    for _ in range(steps):
-        step += 1
-        for w, g, st in zip(ws, gs, sts):
-            oracle.adamw4_step(w, g, st, step=step, **hyper)
-    dt = time.perf_counter() - t0
-    return n * steps / dt / 1e9, oracle.threads(), f"{desc}, {n / 1e6:.1f} M params per step, {steps} step(s)", dt / steps * 1e3
+    all_threads = oracle.threads()
+    if threads is not None:
+        oracle.set_threads(threads)
+    try:
+        ws, gs, sts = [], [], []
+        for i, t in sample:
+            ws.append(workloads.make_param(t, wl.index, i).numpy().ravel().copy())
+            gs.append(workloads.make_grad(t, wl.index, i, 1, dtype=gdt).float().numpy().ravel())
+            sts.append(oracle.state_init(t.rows, t.cols, oracle.kind_of(t.rows, t.cols, t.ndim, 4096, int(t.force_quant))))
+        n = sum(t.numel for _, t in sample)
+        step = 0
+        for _ in range(warmup):
+            step += 1
+            for w, g, st in zip(ws, gs, sts):
+                oracle.adamw4_step(w, g, st, step=step, **hyper)
+        t0 = time.perf_counter()
+        for _ in range(steps):
+            step += 1
+            for w, g, st in zip(ws, gs, sts):
+                oracle.adamw4_step(w, g, st, step=step, **hyper)
+        dt = time.perf_counter() - t0
+        used = oracle.threads()
+    finally:
+        oracle.set_threads(all_threads)
+    return n * steps / dt / 1e9, used, f"{desc}, {n / 1e6:.1f} M params per step, {steps} step(s)", dt / steps * 1e3
 
 
 def run_reference(args):
@@ -191,9 +215,12 @@ def run_reference(args):
     if rank != 0:
         return
     wl = workloads.WORKLOADS[args.workload]()
-    value, threads, desc, ms = time_oracle(wl, max(args.steps, 1), args.warmup)
+    # about two minutes of oracle time in all at the ~0.06 Gparams/s it reaches on 16 cores: the sample shrinks with K + W
+    steps, warmup = max(args.steps, 1), max(args.warmup, 0)
+    budget = int(min(350e6, 0.06e9 * 120 / (steps + warmup)))
+    value, threads, desc, ms = time_oracle(wl, steps, warmup, budget=budget)
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "steps": steps, "warmup": warmup, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": wl.name, "sample": desc, "grad_dtype": wl.grad_dtype},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
@@ -314,9 +341,10 @@ def run_ours(args):
         return
 
     peak, peak_kind = measured_peak()
+    fused = state.schedule == lpmm.SCHEDULE_FUSED and not sgdm
     p2_ms = prof["pass2_ms"] / max(prof["steps"], 1)
     p1_ms = prof["pass1_ms"] / max(prof["steps"], 1)
-    if sgdm:      # one kernel per step: its duration is the step time
+    if sgdm or fused:      # one kernel per step: its duration is the step time
         p2_ms, p1_ms = ms_step, 0.0
     # block maxima: 8 bytes per block of m (and of v when v is block-wise; then pass 1 has nothing to do).
     # A list of 1-D tensors only (flattened parameters) is block-wise whatever the mode (Sec. 4.2).
@@ -328,24 +356,48 @@ def run_ours(args):
     if sgdm:                  # w 4+4, g, first-moment codes 1, block maxima
         pass2_bpp = 8.0 + (2.0 if wl.grad_dtype == "bf16" else 4.0) + 1.0 + 8 / args.m_block
         pass1_bpp = 0.0
-    alg_bytes = pass2_bpp * n_params
-    achieved = alg_bytes / (p2_ms * 1e-3) / 1e9
-    # the captures cover the default quantizers only
-    traffic_pp = PASS2_TRAFFIC_BYTES_PER_PARAM[wl.grad_dtype] if (v_kind == "rank1" and args.m_block == 128 and not sgdm) else None
-    roofline = {"bound": "hbm", "kernel": "sgdm_kernel" if sgdm else "pass2_kernel (update + re-quantize)", "achieved": achieved, "peak": peak,
-                "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+    # The step as a whole. "Algorithmic" = what the method's two reads of every rank-1 tensor amount to (the maxima
+    # pass re-reads the gradient and the second-moment codes): pass1_bpp + pass2_bpp per parameter. The single-pass
+    # figure (each operand once) is printed beside it.
+    step_bytes = (pass1_bpp + pass2_bpp) * n_params
+    single_bytes = pass2_bpp * n_params
+    step_gbs = step_bytes / (ms_step * 1e-3) / 1e9
+    single_gbs = single_bytes / (ms_step * 1e-3) / 1e9
+    default_quant = v_kind == "rank1" and args.m_block == 128 and not sgdm
+    traffic_pp = None
+    if default_quant:         # the captures cover the default quantizers only
+        traffic_pp = STEP_TRAFFIC_BYTES_PER_PARAM["fused" if fused else "two_pass"].get(wl.grad_dtype)
+    kernels = {}
+    if not (sgdm or fused):
+        p2_gbs = single_bytes / (p2_ms * 1e-3) / 1e9
+        kernels["pass2_kernel (update + re-quantize)"] = {
+            "ms_per_launch": p2_ms, "algorithmic_bytes_per_launch": single_bytes, "achieved": p2_gbs, "frac": p2_gbs / peak,
+            "frac_of_nominal_8tbs": p2_gbs / 8000.0,
+            "traffic": None if not default_quant else PASS2_TRAFFIC_BYTES_PER_PARAM[wl.grad_dtype] * n_params}
+        if p1_ms > 0:
+            p1_gbs = pass1_bpp * n_params / (p1_ms * 1e-3) / 1e9
+            kernels["pass1_kernel (row/column maxima)"] = {
+                "ms_per_launch": p1_ms, "algorithmic_bytes_per_launch": pass1_bpp * n_params, "achieved": p1_gbs,
+                "frac": p1_gbs / peak, "frac_of_nominal_8tbs": p1_gbs / 8000.0}
+    sm_mhz = (clocks or {}).get("sm_mhz")
+    roofline = {"bound": "hbm",
+                "kernel": "sgdm_kernel" if sgdm else ("step_fused_kernel (one launch per step)" if fused else
+                                                      "whole step: pass1_kernel + rcp_kernel + pass2_kernel"),
+                "achieved": step_gbs, "peak": peak, "unit": "GB/s", "frac": step_gbs / peak, "peak_kind": f"of {peak_kind}",
+                "frac_of_nominal_8tbs": step_gbs / 8000.0,
                 "traffic": None if traffic_pp is None else traffic_pp * n_params,
-                "algorithmic_bytes_per_launch": alg_bytes, "ms_per_launch": p2_ms,
-                "pass1_ms_per_launch": p1_ms,
-                "pass1_achieved_gbs": pass1_bpp * n_params / (p1_ms * 1e-3) / 1e9 if p1_ms > 0 else None,
-                "step_algorithmic_gbs": alg_bytes / (ms_step * 1e-3) / 1e9,
-                "step_moved_gbs": (pass2_bpp + pass1_bpp) * n_params / (ms_step * 1e-3) / 1e9,
-                "frac_of_nominal_8tbs": achieved / 8000.0}
+                "algorithmic_bytes_per_step": step_bytes, "bytes_per_param": pass1_bpp + pass2_bpp,
+                "single_pass": {"bytes_per_param": pass2_bpp, "achieved": single_gbs, "frac": single_gbs / peak,
+                                "frac_of_nominal_8tbs": single_gbs / 8000.0},
+                "ms_per_step": ms_step, "ms_x_sm_ghz": None if not sm_mhz else ms_step * sm_mhz / 1000.0,
+                "kernels": kernels}
 
     cpu = None
     if not args.no_cpu_baseline and world == 1:
-        v, threads, desc, _ = time_oracle(wl, 2, 1)
-        cpu = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}
+        v, threads, desc, _ = time_oracle(wl, 1, 1)
+        v1, t1, desc1, _ = time_oracle(wl, 1, 1, threads=1, small=True)
+        cpu = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc,
+               "single_thread": {"value": v1, "unit": UNIT, "cores": t1, "sample": desc1}}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
