@@ -59,7 +59,7 @@ def parse_args():
     ap.add_argument("--m-block", type=int, default=128, choices=[128, 2048], help="first-moment block size")
     ap.add_argument("--v-mode", default="rank1", choices=["rank1", "block", "factored"],
                     help="second moment of matrices: rank-1 or block-wise 4-bit, or factorized (fp32 row/column statistics)")
-    ap.add_argument("--schedule", default="auto", choices=["auto", "two_pass", "fused"],
+    ap.add_argument("--schedule", default="auto", choices=["auto", "two_pass", "fused", "overlap"],
                     help="order of the maxima and update work inside a step (lpmm_schedule)")
     ap.add_argument("--tile-elems", type=int, default=0)
     ap.add_argument("--tile-elems-maxima", type=int, default=0)
@@ -67,6 +67,7 @@ def parse_args():
     ap.add_argument("--lead-melems", type=int, default=0)
     ap.add_argument("--gap-items", type=int, default=0)
     ap.add_argument("--no-l2-hints", action="store_true")
+    ap.add_argument("--overlap-groups", type=int, default=0)
     return ap.parse_args()
 
 
@@ -250,10 +251,11 @@ def run_ours(args):
     params = [workloads.make_param(t, wl.index, i, device=dev) for i, t in enumerate(wl.tensors)]
     grads = [workloads.make_grad(t, wl.index, i, 1, device=dev, dtype=gdt) for i, t in enumerate(wl.tensors)]
     v_mode = {"rank1": lpmm.V_RANK1, "block": lpmm.V_BLOCK, "factored": lpmm.V_FACTORED}[args.v_mode]
-    schedule = {"auto": lpmm.SCHEDULE_AUTO, "two_pass": lpmm.SCHEDULE_TWO_PASS, "fused": lpmm.SCHEDULE_FUSED}[args.schedule]
+    schedule = {"auto": lpmm.SCHEDULE_AUTO, "two_pass": lpmm.SCHEDULE_TWO_PASS, "fused": lpmm.SCHEDULE_FUSED,
+                "overlap": lpmm.SCHEDULE_OVERLAP}[args.schedule]
     cfg = lpmm.default_config(m_block=args.m_block, v_mode=v_mode, schedule=schedule, tile_elems=args.tile_elems,
                               tile_elems_maxima=args.tile_elems_maxima, l2_keep_mbytes=args.l2_keep_mb,
-                              lead_melems=args.lead_melems, gap_items=args.gap_items, no_l2_hints=int(args.no_l2_hints))
+                              lead_melems=args.lead_melems, gap_items=args.gap_items, no_l2_hints=int(args.no_l2_hints), overlap_groups=args.overlap_groups)
     state = lpmm.state_init(cfg, wl.tensors, device=dev)
     cache = lpmm.make_ptr_cache(params, grads)
     n_params = wl.numel

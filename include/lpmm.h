@@ -68,7 +68,7 @@ typedef enum { LPMM_UPDATE_FAST = 0, LPMM_UPDATE_IEEE = 1 } lpmm_update_math;
  *             counters in the arena; every wait is bounded (see lpmm_state_device_status).
  *   AUTO:     FUSED where it applies, else TWO_PASS.
  * The stored states and the parameters are bit-identical under both schedules. */
-typedef enum { LPMM_SCHEDULE_AUTO = 0, LPMM_SCHEDULE_TWO_PASS = 1, LPMM_SCHEDULE_FUSED = 2 } lpmm_schedule;
+typedef enum { LPMM_SCHEDULE_AUTO = 0, LPMM_SCHEDULE_TWO_PASS = 1, LPMM_SCHEDULE_FUSED = 2, LPMM_SCHEDULE_OVERLAP = 3 } lpmm_schedule;
 
 /* lpmm_shape.flags */
 #define LPMM_FORCE_QUANT 1u /* quantize even if numel <= min_quant_numel */
@@ -104,6 +104,7 @@ typedef struct {
     int32_t lead_melems;       /* fused: Mi elements of ready update work the maxima pass stays ahead of the update pass */
     int32_t gap_items;         /* fused: work items between a tensor's last maxima tile and its first update tile */
     int32_t no_l2_hints;       /* fused: 1 = plain accesses without eviction priorities (to measure what the hints buy) */
+    int32_t overlap_groups;    /* overlap: number of tensor groups (0 = 8) */
 } lpmm_config;
 
 typedef struct lpmm_state lpmm_state; /* opaque host handle */

@@ -71,6 +71,7 @@ struct ArenaHeader {
     int32_t pad2;
     uint64_t pad3[7];
     unsigned long long wait_stats[2];   // byte 128: fused schedule, {waits that had to poll, their summed nanoseconds}
+    int32_t tile_counter_aux[2];        // byte 144: the same pair as tile_counter for a launch that runs beside another one
 };
 static_assert(sizeof(ArenaHeader) <= 256, "header block");
 
@@ -98,8 +99,10 @@ lpmm_status validate_config(const lpmm_config* cfg, const lpmm_shape* shapes, in
     if (cfg->bits != 4) return LPMM_ERR_UNSUPPORTED;
     if ((cfg->m_block != 128 && cfg->m_block != 2048) || cfg->v_block != 128) return LPMM_ERR_UNSUPPORTED;
     if (cfg->update_math != LPMM_UPDATE_FAST && cfg->update_math != LPMM_UPDATE_IEEE) return LPMM_ERR_INVALID_ARG;
-    if (cfg->schedule != LPMM_SCHEDULE_AUTO && cfg->schedule != LPMM_SCHEDULE_TWO_PASS && cfg->schedule != LPMM_SCHEDULE_FUSED)
+    if (cfg->schedule != LPMM_SCHEDULE_AUTO && cfg->schedule != LPMM_SCHEDULE_TWO_PASS && cfg->schedule != LPMM_SCHEDULE_FUSED &&
+        cfg->schedule != LPMM_SCHEDULE_OVERLAP)
         return LPMM_ERR_INVALID_ARG;
+    if (cfg->overlap_groups < 0 || cfg->overlap_groups > 4096) return LPMM_ERR_INVALID_ARG;
     if (cfg->schedule == LPMM_SCHEDULE_FUSED && !fused_eligible(*cfg)) return LPMM_ERR_UNSUPPORTED;
     for (int32_t te : {cfg->tile_elems, cfg->tile_elems_maxima})
         if (te != 0 && (te < 2048 || te > (1 << 22) || (te & (te - 1)) != 0)) return LPMM_ERR_INVALID_ARG;
@@ -168,9 +171,10 @@ int32_t choose_kind(const lpmm_config& cfg, const lpmm_shape& s) {
 
 // Which schedule a state runs: the fused one needs the default quantizers (rank-1 second moments, B128 first moments).
 bool fused_eligible(const lpmm_config& cfg) { return cfg.v_mode == LPMM_V_RANK1 && cfg.m_block == 128; }
-// AUTO goes by measurement (B200): the fused launch wins where the step is bound by launch overhead (a few million
-// parameters: one launch instead of three and a memset); on larger lists its short tiles cost more than its L2 hits save.
-constexpr int64_t kAutoFusedMaxElems = (int64_t)8 << 20;
+// AUTO goes by measurement (B200): the fused launch wins where launch overhead and the gaps between the three kernels
+// matter (1024x4096 + bias: 44 vs 51 us; the 181-tensor Transformer-base list, 60.5 M: 0.228 vs 0.254 ms); from one
+// 8192x8192 matrix (64 Mi) upwards the two-pass schedule is ahead (0.250 vs 0.258 ms; LLaMA-7B list 17.2 vs 18.3 ms).
+constexpr int64_t kAutoFusedMaxElems = (int64_t)63 << 20;
 bool wants_fused(const lpmm_config& cfg, int64_t total_elems) {
     if (!fused_eligible(cfg)) return false;
     if (cfg.schedule == LPMM_SCHEDULE_FUSED) return true;
@@ -183,9 +187,10 @@ struct TileSizes { int64_t update, maxima; };
 // aim is >= 6 tiles per resident CTA (the tail is what is balanced). Two-pass schedule, measured optima of the update
 // pass: 32 Ki for 60-70 M parameters, 64-128 Ki for 355 M, 256 Ki for 6.7 G; the maxima pass gains from taller tiles
 // (each tile ends with a flush of its column maxima and starts with an empty load pipeline), up to 1 Mi. The fused
-// schedule wants short tiles: an update tile can only start when the tensor's last maxima tile has finished.
+// schedule wants shorter tiles (an update tile can only start when the tensor's last maxima tile has finished), but
+// every tile costs about 2 us of start-up: 128 Ki / 256 Ki measured best on the 6.7 G list.
 TileSizes choose_tile_sizes(const lpmm_config& cfg, int64_t total_elems, bool fused) {
-    const int64_t cap2 = fused ? 32768 : 262144, cap1 = fused ? 65536 : (1 << 20);
+    const int64_t cap2 = fused ? 131072 : 262144, cap1 = fused ? 262144 : (1 << 20);
     const int64_t hard2 = fused ? 262144 : ((int64_t)1 << 22);   // fused: an update tile has at most 1024 rows of 256 columns
     const int64_t target = total_elems / (6LL * kPlanResidentCtas);
     TileSizes ts;
@@ -358,6 +363,9 @@ struct lpmm_state {
     int32_t sms, occ1, occ2;
     int32_t p1_ctas;                       // which instantiation of the maxima pass (2 or 3 CTAs per SM)
     std::vector<int32_t> tiles1, tiles2, tiles3;   // host copies of the tile prefix sums (3: element-indexed tiles of every tensor)
+    cudaStream_t aux = nullptr;            // overlapped schedule: the stream of the maxima passes (lazily created)
+    std::vector<cudaEvent_t> ov_events;    // overlapped schedule: per group {maxima done, update done}, then the fork event
+    std::vector<int32_t> group_cut;        // overlapped schedule: first tensor of every group, then n
     cudaStream_t copy_in, copy_out;        // lazily created by the host-buffer entry point
     std::vector<cudaEvent_t> host_events;
     bool profile;                          // record events around each kernel of a step
@@ -386,8 +394,8 @@ void build_work_list(const lpmm_state* st, const std::vector<TilePlan>& plans, s
     for (int32_t i = 0; i < n; ++i)
         if (plans[i].tiles_maxima > 0) rank1.push_back(i);
     const int64_t keep_bytes = (cfg.l2_keep_mbytes > 0 ? (int64_t)cfg.l2_keep_mbytes : 48) << 20;
-    const int64_t lead_elems = (cfg.lead_melems > 0 ? (int64_t)cfg.lead_melems : 10) << 20;
-    const int64_t gap = cfg.gap_items > 0 ? cfg.gap_items : kPlanResidentCtas / 2;
+    const int64_t lead_elems = (cfg.lead_melems > 0 ? (int64_t)cfg.lead_melems : 30) << 20;
+    const int64_t gap = cfg.gap_items > 0 ? cfg.gap_items : 2 * kPlanResidentCtas;
     work->clear();
     auto tile_elems1 = [&](int32_t t) {
         const TilePlan& p = plans[t];
@@ -513,6 +521,18 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
     st->tiles2 = t2;
     st->tiles3 = t3;
     st->tiles4 = t4;
+    {   // overlapped schedule: consecutive groups of about equal size, each with at least one maxima tile
+        int32_t groups = st->cfg.overlap_groups > 0 ? st->cfg.overlap_groups : 8;
+        st->group_cut.assign(1, 0);
+        const int64_t per_group = total_elems / groups + 1;
+        int64_t acc = 0;
+        for (int32_t i = 0; i < n; ++i) {
+            acc += st->L.t[i].numel;
+            if (acc >= per_group && i + 1 < n && t1[i + 1] > t1[st->group_cut.back()]) { st->group_cut.push_back(i + 1); acc = 0; }
+        }
+        if (t1[n] == t1[st->group_cut.back()] && st->group_cut.size() > 1) st->group_cut.pop_back();   // no maxima work in the tail
+        st->group_cut.push_back(n);
+    }
     if (st->fused) {
         std::vector<uint2> work;
         build_work_list(st, plans, &work);
@@ -605,12 +625,6 @@ lpmm_status make_state(const lpmm_config* cfg, const lpmm_shape* shapes, int32_t
         if (e != cudaSuccess) rc = cuda_fail(e);
     }
     st->new_rc_clean = true;
-#ifdef LPMM_EXP_SETASIDE
-    if (rc == LPMM_OK) {   // experiment: an L2 set-aside for "evict last" lines
-        const cudaError_t e = cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, (size_t)LPMM_EXP_SETASIDE << 20);
-        if (e != cudaSuccess) rc = cuda_fail(e);
-    }
-#endif
     if (rc == LPMM_OK) rc = build_tables(st, s);
     if (rc != LPMM_OK) { delete st; return rc; }
     *out = st;
@@ -731,40 +745,48 @@ bool wants_ieee_update(const lpmm_state* st, const Hyper& h) {
     return !(std::isfinite(h.upd_c1) && std::isfinite(h.upd_e1));
 }
 
-// Enqueues the three kernels of one step for tensors [t0, t1). ev (4 events or nullptr) brackets the kernels.
-lpmm_status enqueue_range(lpmm_state* st, StepArgs a, int32_t t0, int32_t t1, bool bf16, bool ieee_update,
-                          cudaStream_t s, cudaEvent_t* ev, int32_t* launches) {
+// Enqueues the maxima pass of tensors [t0, t1) and what follows it (clearing of the new r, c before; their
+// reciprocals, or the factorized statistics, after). grid_cap: most CTAs to launch. aux: the launch may run beside
+// another step kernel and uses the second pair of tile counters. ev (2 events or nullptr) brackets the maxima kernel.
+lpmm_status enqueue_maxima(lpmm_state* st, StepArgs a, int32_t t0, int32_t t1, bool bf16, int32_t grid_cap, bool aux,
+                           cudaStream_t s, cudaEvent_t* ev, int32_t* launches) {
     a.aligned32 = (st->params_a32 && (bf16 || st->grads_a32)) ? 1 : 0;
+    if (aux) a.tile_counter = reinterpret_cast<int32_t*>(st->arena + offsetof(ArenaHeader, tile_counter_aux));
     const int32_t p1_begin = st->tiles1[t0], p1_end = st->tiles1[t1];
-    if (p1_end > p1_begin) {
-        // the rank-1 scale region of these tensors is one contiguous range of the scale buffers
-        int64_t rc_begin = -1, rc_end = 0;
-        for (int32_t i = t0; i < t1; ++i) {
-            const TensorLayout& t = st->L.t[i];
-            if (!uses_rc(t.kind)) continue;
-            if (rc_begin < 0) rc_begin = t.rc_index;
-            rc_end = (t.rc_index + t.c_off + (t.cols + 3) / 4 * 4 + 63) / 64 * 64;
-        }
-        float* rc_new = reinterpret_cast<float*>(st->arena + st->L.rc[(st->phase + 1) % 3]) + rc_begin;
-        LPMM_CUDA(cudaMemsetAsync(rc_new, 0, sizeof(float) * (size_t)(rc_end - rc_begin), s));
-        if (ev) LPMM_CUDA(cudaEventRecord(ev[0], s));
-        a.tile_start = reinterpret_cast<const int32_t*>(st->arena + st->L.tiles1);
-        a.tile_begin = p1_begin;
-        a.tile_end = p1_end;
-        const int32_t cap = st->sms * st->occ1, tiles = p1_end - p1_begin;
-        LPMM_CUDA(launch_pass1(a, bf16, st->p1_ctas, tiles < cap ? tiles : cap, s));
-        if (ev) LPMM_CUDA(cudaEventRecord(ev[1], s));
-        LPMM_CUDA(launch_rcp(rc_new, reinterpret_cast<float*>(st->arena + st->L.rcp) + rc_begin, rc_end - rc_begin, s));
-        *launches += 2;
-        if (st->cfg.v_mode == LPMM_V_FACTORED) {   // statistics' moving averages and the row factors R_i / sum(R)
-            LPMM_CUDA(launch_factor_finalize(a, t0, t1, s));
-            *launches += 1;
-        }
-    } else if (ev) {
-        LPMM_CUDA(cudaEventRecord(ev[0], s));
-        LPMM_CUDA(cudaEventRecord(ev[1], s));
+    if (p1_end <= p1_begin) {
+        if (ev) { LPMM_CUDA(cudaEventRecord(ev[0], s)); LPMM_CUDA(cudaEventRecord(ev[1], s)); }
+        return LPMM_OK;
     }
-    if (ev) LPMM_CUDA(cudaEventRecord(ev[2], s));
+    // the rank-1 scale region of these tensors is one contiguous range of the scale buffers
+    int64_t rc_begin = -1, rc_end = 0;
+    for (int32_t i = t0; i < t1; ++i) {
+        const TensorLayout& t = st->L.t[i];
+        if (!uses_rc(t.kind)) continue;
+        if (rc_begin < 0) rc_begin = t.rc_index;
+        rc_end = (t.rc_index + t.c_off + (t.cols + 3) / 4 * 4 + 63) / 64 * 64;
+    }
+    float* rc_new = reinterpret_cast<float*>(st->arena + st->L.rc[(st->phase + 1) % 3]) + rc_begin;
+    LPMM_CUDA(cudaMemsetAsync(rc_new, 0, sizeof(float) * (size_t)(rc_end - rc_begin), s));
+    if (ev) LPMM_CUDA(cudaEventRecord(ev[0], s));
+    a.tile_start = reinterpret_cast<const int32_t*>(st->arena + st->L.tiles1);
+    a.tile_begin = p1_begin;
+    a.tile_end = p1_end;
+    const int32_t tiles = p1_end - p1_begin;
+    LPMM_CUDA(launch_pass1(a, bf16, st->p1_ctas, tiles < grid_cap ? tiles : grid_cap, s));
+    if (ev) LPMM_CUDA(cudaEventRecord(ev[1], s));
+    LPMM_CUDA(launch_rcp(rc_new, reinterpret_cast<float*>(st->arena + st->L.rcp) + rc_begin, rc_end - rc_begin, s));
+    *launches += 2;
+    if (st->cfg.v_mode == LPMM_V_FACTORED) {   // statistics' moving averages and the row factors R_i / sum(R)
+        LPMM_CUDA(launch_factor_finalize(a, t0, t1, s));
+        *launches += 1;
+    }
+    return LPMM_OK;
+}
+
+// Enqueues the update pass of tensors [t0, t1) (and the folded 1-D tensors' own launch).
+lpmm_status enqueue_update(lpmm_state* st, StepArgs a, int32_t t0, int32_t t1, bool bf16, bool ieee_update,
+                           cudaStream_t s, int32_t* launches) {
+    a.aligned32 = (st->params_a32 && (bf16 || st->grads_a32)) ? 1 : 0;
     a.tile_start = reinterpret_cast<const int32_t*>(st->arena + st->L.tiles2);
     a.tile_begin = st->tiles2[t0];
     a.tile_end = st->tiles2[t1];
@@ -772,7 +794,7 @@ lpmm_status enqueue_range(lpmm_state* st, StepArgs a, int32_t t0, int32_t t1, bo
     LPMM_CUDA(launch_pass2(a, bf16, ieee_update, st->cfg.m_block == 2048 ? 11 : 7,
                            st->cfg.v_mode == LPMM_V_FACTORED ? 1 : (st->cfg.v_mode == LPMM_V_BLOCK ? 2 : 0),
                            tiles < cap ? tiles : cap, s));
-    *launches += 1;
+    if (tiles > 0) *launches += 1;
     if (st->tiles4[t1] > st->tiles4[t0]) {   // folded 1-D tensors of a state that is not block-wise
         a.tile_start = reinterpret_cast<const int32_t*>(st->arena + st->L.tiles4);
         a.tile_begin = st->tiles4[t0];
@@ -781,8 +803,57 @@ lpmm_status enqueue_range(lpmm_state* st, StepArgs a, int32_t t0, int32_t t1, bo
         LPMM_CUDA(launch_pass2(a, bf16, ieee_update, st->cfg.m_block == 2048 ? 11 : 7, 2, tiles4 < cap ? tiles4 : cap, s));
         *launches += 1;
     }
+    return LPMM_OK;
+}
+
+// Enqueues the kernels of one step for tensors [t0, t1) one after the other. ev (4 events or nullptr) brackets them.
+lpmm_status enqueue_range(lpmm_state* st, StepArgs a, int32_t t0, int32_t t1, bool bf16, bool ieee_update,
+                          cudaStream_t s, cudaEvent_t* ev, int32_t* launches) {
+    lpmm_status rc = enqueue_maxima(st, a, t0, t1, bf16, st->sms * st->occ1, false, s, ev, launches);
+    if (rc != LPMM_OK) return rc;
+    if (ev) LPMM_CUDA(cudaEventRecord(ev[2], s));
+    rc = enqueue_update(st, a, t0, t1, bf16, ieee_update, s, launches);
+    if (rc != LPMM_OK) return rc;
     if (ev) LPMM_CUDA(cudaEventRecord(ev[3], s));
     return LPMM_OK;
+}
+
+// The overlapped two-pass schedule: the tensor list is cut into groups; the maxima pass of group k + 1 runs on a second
+// stream beside the update pass of group k (the two kernels share every SM, one CTA each: the maxima pass is bound by
+// instruction issue, the update pass by DRAM). Nothing waits on the device; the order is kept by events:
+//   aux:  maxima(0) | maxima(1) after update(-)... each maxima(k+1) starts when update(k-1) has finished
+//   main: update(k) after maxima(k)
+lpmm_status enqueue_overlapped(lpmm_state* st, const StepArgs& a, bool bf16, bool ieee_update, cudaStream_t s, int32_t* launches) {
+    const int32_t n = st->n;
+    if (!st->aux) LPMM_CUDA(cudaStreamCreateWithFlags(&st->aux, cudaStreamNonBlocking));
+    const std::vector<int32_t>& cut = st->group_cut;
+    const size_t groups = cut.size() - 1;
+    while (st->ov_events.size() < 2 * groups + 1) {
+        cudaEvent_t e;
+        LPMM_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+        st->ov_events.push_back(e);
+    }
+    cudaEvent_t ev_fork = st->ov_events[2 * groups];
+    LPMM_CUDA(cudaEventRecord(ev_fork, s));              // earlier work on the caller's stream comes first
+    LPMM_CUDA(cudaStreamWaitEvent(st->aux, ev_fork, 0));
+    lpmm_status rc = enqueue_maxima(st, a, cut[0], cut[1], bf16, st->sms * st->occ1, true, st->aux, nullptr, launches);
+    if (rc != LPMM_OK) return rc;
+    LPMM_CUDA(cudaEventRecord(st->ov_events[0], st->aux));
+    for (size_t k = 0; k < groups; ++k) {
+        cudaEvent_t ev_m = st->ov_events[2 * k], ev_u = st->ov_events[2 * k + 1];
+        if (k + 1 < groups) {    // the next group's maxima pass: beside this group's update pass, one CTA per SM
+            if (k > 0) LPMM_CUDA(cudaStreamWaitEvent(st->aux, st->ov_events[2 * (k - 1) + 1], 0));
+            rc = enqueue_maxima(st, a, cut[k + 1], cut[k + 2], bf16, st->sms, true, st->aux, nullptr, launches);
+            if (rc != LPMM_OK) return rc;
+            LPMM_CUDA(cudaEventRecord(st->ov_events[2 * (k + 1)], st->aux));
+        }
+        LPMM_CUDA(cudaStreamWaitEvent(s, ev_m, 0));
+        rc = enqueue_update(st, a, cut[k], cut[k + 1], bf16, ieee_update, s, launches);
+        if (rc != LPMM_OK) return rc;
+        LPMM_CUDA(cudaEventRecord(ev_u, s));
+    }
+    (void)n;
+    return LPMM_OK;   // the caller's stream ends after the last update; the second stream has nothing left in flight
 }
 
 // Makes the device-side array of bfloat16-copy pointers hold d_params16 (uploads only on change).
@@ -848,6 +919,12 @@ lpmm_status adamw4_step_impl(lpmm_state* st, void* const* d_params, void* const*
         }
         if (ev) LPMM_CUDA(cudaEventRecord(ev[3], s));
         st->new_rc_clean = true;       // the maxima tiles have cleared the buffer the next step reduces into
+    } else if (st->cfg.schedule == LPMM_SCHEDULE_OVERLAP && st->group_cut.size() > 2) {
+        if (ev) { LPMM_CUDA(cudaEventRecord(ev[0], s)); LPMM_CUDA(cudaEventRecord(ev[1], s)); LPMM_CUDA(cudaEventRecord(ev[2], s)); }
+        rc = enqueue_overlapped(st, a, bf16, ieee_update, s, &launches);
+        if (rc != LPMM_OK) return rc;
+        if (ev) LPMM_CUDA(cudaEventRecord(ev[3], s));
+        st->new_rc_clean = false;
     } else {
         rc = enqueue_range(st, a, 0, st->n, bf16, ieee_update, s, ev, &launches);
         if (rc != LPMM_OK) return rc;
@@ -1133,7 +1210,11 @@ lpmm_status lpmm_state_wait_stats(lpmm_state* st, int64_t* waits, int64_t* wait_
 
 int32_t lpmm_state_phase(const lpmm_state* st) { return st ? st->phase : -1; }
 
-int32_t lpmm_state_schedule(const lpmm_state* st) { return st ? (st->fused ? LPMM_SCHEDULE_FUSED : LPMM_SCHEDULE_TWO_PASS) : -1; }
+int32_t lpmm_state_schedule(const lpmm_state* st) {
+    if (!st) return -1;
+    if (st->fused) return LPMM_SCHEDULE_FUSED;
+    return (st->cfg.schedule == LPMM_SCHEDULE_OVERLAP && st->group_cut.size() > 2) ? LPMM_SCHEDULE_OVERLAP : LPMM_SCHEDULE_TWO_PASS;
+}
 
 int32_t lpmm_state_last_launches(const lpmm_state* st) { return st ? st->last_launches : 0; }
 
@@ -1141,6 +1222,8 @@ void lpmm_state_destroy(lpmm_state* st) {
     if (!st) return;
     for (cudaEvent_t e : st->prof_events) cudaEventDestroy(e);
     for (cudaEvent_t e : st->host_events) cudaEventDestroy(e);
+    for (cudaEvent_t e : st->ov_events) cudaEventDestroy(e);
+    if (st->aux) cudaStreamDestroy(st->aux);
     if (st->copy_in) cudaStreamDestroy(st->copy_in);
     if (st->copy_out) cudaStreamDestroy(st->copy_out);
     delete st;

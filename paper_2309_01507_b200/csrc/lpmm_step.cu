@@ -296,33 +296,17 @@ __device__ __forceinline__ void store8_f32_256(float* p, const float (&x)[8]) {
 // ---- L2 residency hints (fused schedule) --------------------------------------------------------------
 //
 // In the fused schedule the maxima pass and the update pass of a tensor run close together and the update pass
-// should find the gradient and the second-moment codes still in L2. Accesses therefore carry a cache policy:
-// the maxima pass reads them "evict last" (for the part of a tensor that is meant to stay), the update pass reads
-// and writes everything "evict first" (each line is dead once it has been used), so that the streaming operands
-// (parameters, first-moment codes) are the first victims and do not push the kept lines out.
+// should find the gradient and the second-moment codes still in L2. The maxima pass therefore reads the part of a
+// tensor that is meant to stay with the "evict last" priority. (Marking the update pass's accesses "evict first" as
+// well was measured and dropped: the hinted forms of its loads and stores cost more than the few extra hits saved.)
 struct L2Policies {
-    uint64_t first, last, normal;
+    uint64_t last, normal;
 };
 __device__ __forceinline__ L2Policies make_l2_policies() {
     L2Policies p;
-    asm("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p.first));
     asm("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p.last));
     asm("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p.normal));
     return p;
-}
-__device__ __forceinline__ void load8_f32_256_h(const float* p, float4& a, float4& b, uint64_t pol) {
-    asm volatile("ld.global.L2::cache_hint.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8], %9;"
-                 : "=f"(a.x), "=f"(a.y), "=f"(a.z), "=f"(a.w), "=f"(b.x), "=f"(b.y), "=f"(b.z), "=f"(b.w) : "l"(p), "l"(pol));
-}
-__device__ __forceinline__ float4 load4_f32_h(const float* p, uint64_t pol) {
-    float4 a;
-    asm volatile("ld.global.L2::cache_hint.v4.f32 {%0,%1,%2,%3}, [%4], %5;"
-                 : "=f"(a.x), "=f"(a.y), "=f"(a.z), "=f"(a.w) : "l"(p), "l"(pol));
-    return a;
-}
-__device__ __forceinline__ void load8_u32_256_nc_h(const void* p, uint4& a, uint4& b, uint64_t pol) {
-    asm volatile("ld.global.nc.L2::cache_hint.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8], %9;"
-                 : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w), "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w) : "l"(p), "l"(pol));
 }
 __device__ __forceinline__ uint4 load4_u32_nc_h(const void* p, uint64_t pol) {
     uint4 a;
@@ -330,26 +314,10 @@ __device__ __forceinline__ uint4 load4_u32_nc_h(const void* p, uint64_t pol) {
                  : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w) : "l"(p), "l"(pol));
     return a;
 }
-__device__ __forceinline__ uint32_t load1_u32_h(const void* p, uint64_t pol) {
-    uint32_t a;
-    asm volatile("ld.global.L2::cache_hint.u32 %0, [%1], %2;" : "=r"(a) : "l"(p), "l"(pol));
-    return a;
-}
 __device__ __forceinline__ uint32_t load1_u32_nc_h(const void* p, uint64_t pol) {
     uint32_t a;
     asm volatile("ld.global.nc.L2::cache_hint.u32 %0, [%1], %2;" : "=r"(a) : "l"(p), "l"(pol));
     return a;
-}
-__device__ __forceinline__ void store8_f32_256_h(float* p, const float (&x)[8], uint64_t pol) {
-    asm volatile("st.global.L2::cache_hint.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8}, %9;"
-                 :: "l"(p), "f"(x[0]), "f"(x[1]), "f"(x[2]), "f"(x[3]), "f"(x[4]), "f"(x[5]), "f"(x[6]), "f"(x[7]), "l"(pol) : "memory");
-}
-__device__ __forceinline__ void store4_f32_h(float* p, float a, float b, float c, float d, uint64_t pol) {
-    asm volatile("st.global.L2::cache_hint.v4.f32 [%0], {%1,%2,%3,%4}, %5;"
-                 :: "l"(p), "f"(a), "f"(b), "f"(c), "f"(d), "l"(pol) : "memory");
-}
-__device__ __forceinline__ void store1_u32_h(void* p, uint32_t v, uint64_t pol) {
-    asm volatile("st.global.L2::cache_hint.u32 [%0], %1, %2;" :: "l"(p), "r"(v), "l"(pol) : "memory");
 }
 __device__ __forceinline__ void load8_f32_cg(const float* p, float (&x)[8]) {   // data written earlier in the same launch
     float4 a = __ldcg(reinterpret_cast<const float4*>(p));
@@ -411,20 +379,12 @@ struct TileView {
     uint32_t* red_step;    // running count of CTA-wide reductions
     const char* pf_base;   // this lane's share of the row prefetch: one cache line of one of the arrays
     uint32_t pf_step;      // bytes between two of the warp's rows in that array (0: this lane prefetches nothing)
-    uint32_t pf_bytes;     // fused schedule: size of this lane's bulk prefetch request (0: a plain one-line prefetch)
-    uint64_t pol;          // fused schedule: cache policy of every access of the update pass (evict first)
     const float* s_rows;   // fused schedule: shared memory, the tile's old row maxima [kFusedTileRows] followed by the
                            // reciprocals of its new ones, starting at this warp's first row
 };
 
 // Fused schedule: most rows an update tile may have (its row scalars are staged in shared memory).
 constexpr int kFusedTileRows = 1024;
-#ifdef LPMM_EXP_PLAIN_P2
-constexpr bool kHintedUpdate = false;   // experiment: the fused update pass with plain accesses
-#else
-constexpr bool kHintedUpdate = true;
-#endif
-
 // Asks L2 to fetch this lane's share of row k ahead of time (no register is tied up): the later
 // loads then find their data in L2 instead of waiting for DRAM.
 constexpr uint32_t kL2Ahead = 4;   // rows
@@ -433,41 +393,9 @@ __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefe
 // One instruction per row for the whole warp: the 256 elements a warp owns in a row are 8 lines of parameters,
 // 4 (bf16) or 8 (fp32) lines of gradient, one line of each code array and one of block scales, and each of the
 // first lanes asks for one of those lines.
-// Fused schedule: the same as one bulk request per array with the streaming policy, so that the lines arrive in L2
-// already marked as first victims (a plain prefetch would bring them in with normal priority). pf_bytes = the size of
-// this lane's request (0: this lane asks with a plain one-line prefetch, or for nothing).
-__device__ __forceinline__ void prefetch_l2_bulk(const void* p, uint32_t bytes, uint64_t pol) {
-    asm volatile("cp.async.bulk.prefetch.L2.global.L2::cache_hint [%0], %1, %2;" ::"l"(p), "r"(bytes), "l"(pol) : "memory");
-}
 template <bool BF16, int MSHIFT, int VM, bool FU = false>
 __device__ __forceinline__ void prefetch_row(const TileView& t, uint32_t k) {
-    if (FU) {
-        if (t.pf_bytes != 0) prefetch_l2_bulk(t.pf_base + (size_t)k * t.pf_step, t.pf_bytes, t.pol);
-        else if (t.pf_step != 0) prefetch_l2(t.pf_base + (size_t)k * t.pf_step);
-        return;
-    }
     if (t.pf_step != 0) prefetch_l2(t.pf_base + (size_t)k * t.pf_step);
-}
-// Fused schedule: lane 0 asks for the warp's parameters of a row, lane 1 for its first-moment codes (bulk requests),
-// lane 2 for the line with its block maxima. The gradient and the second-moment codes are expected in L2 already.
-template <int MSHIFT>
-__device__ __forceinline__ void prefetch_roles_fused(TileView& t, int lane, int valid, const float* warp_w, const uint8_t* warp_mq,
-                                                     const float* warp_ms) {
-    t.pf_base = nullptr;
-    t.pf_step = 0;
-    t.pf_bytes = 0;
-    if (lane == 0) {
-        t.pf_base = reinterpret_cast<const char*>(warp_w);
-        t.pf_step = t.row_step * 4u;
-        t.pf_bytes = (uint32_t)valid * 4u;
-    } else if (lane == 1) {
-        t.pf_base = reinterpret_cast<const char*>(warp_mq);
-        t.pf_step = t.row_step / 2u;
-        t.pf_bytes = (uint32_t)valid / 2u;
-    } else if (lane == 2) {
-        t.pf_base = reinterpret_cast<const char*>(warp_ms);
-        t.pf_step = (t.row_step >> MSHIFT) * 4u;
-    }
 }
 // Assigns the lane its line (warp_* point at the warp's first element of row 0; row_step in elements).
 // `valid` = how many of the warp's 256 columns exist (128 in a tensor's last warp column when cols % 256 == 128):
@@ -509,29 +437,6 @@ __device__ __forceinline__ void prefetch_roles(TileView& t, int lane, int valid,
 template <bool BF16, int MSHIFT, int VM, bool A32, bool FU = false>
 __device__ __forceinline__ void load_row(RowRegs<BF16>& r, const TileView& t, uint32_t k) {
     const uint32_t off = k * t.row_step;
-    if (FU && kHintedUpdate) {   // fused schedule (rank-1, B128 only): every access carries the streaming policy; r', c' reciprocals were
-                // written earlier in this launch and are read past L1
-        if (A32) {
-            load8_f32_256_h(t.w + off, r.w0, r.w1, t.pol);
-        } else {
-            r.w0 = load4_f32_h(t.w + off, t.pol);
-            r.w1 = load4_f32_h(t.w + off + 4, t.pol);
-        }
-        if (BF16) {
-            r.g0 = load4_u32_nc_h(reinterpret_cast<const uint16_t*>(t.g) + off, t.pol);
-        } else if (A32) {
-            load8_u32_256_nc_h(reinterpret_cast<const float*>(t.g) + off, r.g0, r.g1, t.pol);
-        } else {
-            r.g0 = load4_u32_nc_h(reinterpret_cast<const float*>(t.g) + off, t.pol);
-            r.g1 = load4_u32_nc_h(reinterpret_cast<const float*>(t.g) + off + 4, t.pol);
-        }
-        r.qm = load1_u32_h(t.m_codes + (off >> 1), t.pol);
-        r.am = __uint_as_float(load1_u32_h(t.m_scale + (off >> MSHIFT), t.pol));
-        r.qv = load1_u32_h(t.v_codes + (off >> 1), t.pol);
-        r.r_old = t.s_rows[k * t.row_stride];
-        r.r_rcp = t.s_rows[kFusedTileRows + k * t.row_stride];
-        return;
-    }
     if (A32) {
         load8_f32_256(t.w + off, r.w0, r.w1);
     } else {
@@ -592,19 +497,6 @@ __device__ __forceinline__ void process_row(const RowRegs<BF16>& r, const TileVi
         }
     }
     moments_and_update8<EXACT, VM == 1>(wv, gv, r.qm, r.qv, __fmul_rn(lt.de, r.am), vs, h, h2, lt, mt, vt);
-    if (FU && kHintedUpdate) {
-        if (A32) {
-            store8_f32_256_h(t.w + off, wv, t.pol);
-        } else {
-            store4_f32_h(t.w + off, wv[0], wv[1], wv[2], wv[3], t.pol);
-            store4_f32_h(t.w + off + 4, wv[4], wv[5], wv[6], wv[7], t.pol);
-        }
-        const float am_f = group_max(absmax8(mt), lt.mask);
-        if ((threadIdx.x & 15) == 0) store1_u32_h(t.m_scale + (off >> 7), __float_as_uint(am_f), t.pol);
-        store1_u32_h(t.m_codes + (off >> 1), quantize8_de(mt, scale_rcp(am_f), s_lut), t.pol);
-        store1_u32_h(t.v_codes + (off >> 1), quantize8_lin(vt, vr, h2), t.pol);
-        return;
-    }
     if (A32) store8_f32_256(t.w + off, wv); else store8_f32(t.w + off, wv);
     if (WB) store8_bf16(t.w16 + off, wv);
     const float am_new = block_max(absmax8(mt), MSHIFT, lt, t.s_red, *t.red_step);
@@ -626,7 +518,7 @@ __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __r
                                                  const void* __restrict__ g,
                                                  int tile, RcSel sel, const Hyper& h, const Hyper2& h2,
                                                  const LaneTables& lt, const unsigned char* s_lut, float* s_red,
-                                                 uint32_t& red_step, uint64_t pol = 0, float* s_rows = nullptr) {
+                                                 uint32_t& red_step, float* s_rows = nullptr) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int wx = d.wx, wy_count = kWarps / wx;
     const int tx = tile % d.tiles_x, ty = tile / d.tiles_x;
@@ -674,7 +566,6 @@ __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __r
     }
     const int64_t e0 = row0 * d.cols + col0;
     TileView t;
-    t.pol = pol;
     t.w = w + e0;
     t.w16 = WB ? w16 + e0 : nullptr;
     t.g = BF16 ? static_cast<const void*>(reinterpret_cast<const uint16_t*>(g) + e0)
@@ -694,9 +585,6 @@ __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __r
     {
         const int64_t ew = e0 - lane * kLaneElems;       // the warp's first element of its first row
         const int64_t left = d.cols - (col0 - lane * kLaneElems);
-        if (FU) prefetch_roles_fused<MSHIFT>(t, lane, left < kWarpElems ? (int)left : kWarpElems, w + ew, d.m_codes + (ew >> 1),
-                                             d.m_scale + (ew >> MSHIFT));
-        else
         prefetch_roles<BF16, MSHIFT, VM>(t, lane, left < kWarpElems ? (int)left : kWarpElems, w + ew,
                                            BF16 ? static_cast<const void*>(reinterpret_cast<const uint16_t*>(g) + ew)
                                                 : static_cast<const void*>(reinterpret_cast<const float*>(g) + ew),
@@ -1467,12 +1355,9 @@ __global__ void __launch_bounds__(kThreads, 2) step_fused_kernel(StepArgs a) {
             }
             float* w = a.params[t];
             switch (d.kind) {
-                case K_RANK1_FAST: {
-                    const L2Policies pol = make_l2_policies();
-                    pass2_rank1_fast<BF16, EXACT, 7, 0, false, A32, true>(d, w, nullptr, g, local, a.sel, a.h, h2, lt, s_lut, s_red, red_step,
-                                                                           a.l2_hints ? pol.first : pol.normal, s_rows);
+                case K_RANK1_FAST:
+                    pass2_rank1_fast<BF16, EXACT, 7, 0, false, A32, true>(d, w, nullptr, g, local, a.sel, a.h, h2, lt, s_lut, s_red, red_step, s_rows);
                     break;
-                }
                 case K_RANK1_FLAT: pass2_flat<BF16, true, EXACT, 7, false, A32, true>(d, w, nullptr, g, local, a.sel, a.h, h2, lt, s_lut, s_red, red_step); break;
                 case K_BLOCK:      pass2_flat<BF16, false, EXACT, 7, false, A32>(d, w, nullptr, g, local, a.sel, a.h, h2, lt, s_lut, s_red, red_step); break;
                 case K_FP32:       pass2_fp32<BF16, EXACT, false, A32>(d, w, nullptr, g, local, a.h); break;

@@ -22,7 +22,7 @@ NORM_BLOCK, NORM_RANK1 = 0, 1
 MAP_DE_SIGNED, MAP_LINEAR_NOZERO = 0, 1
 V_RANK1, V_BLOCK, V_FACTORED = 0, 1, 2
 UPDATE_FAST, UPDATE_IEEE = 0, 1
-SCHEDULE_AUTO, SCHEDULE_TWO_PASS, SCHEDULE_FUSED = 0, 1, 2
+SCHEDULE_AUTO, SCHEDULE_TWO_PASS, SCHEDULE_FUSED, SCHEDULE_OVERLAP = 0, 1, 2, 3
 FORCE_QUANT, FORCE_FP32 = 1, 2
 Q_GIVEN_SCALES = 1
 KIND_FP32, KIND_BLOCK, KIND_RANK1, KIND_FACTORED = 0, 1, 2, 3
@@ -58,14 +58,14 @@ class Config(C.Structure):
     _fields_ = [("bits", C.c_int32), ("m_block", C.c_int32), ("v_block", C.c_int32), ("v_mode", C.c_int32),
                 ("min_quant_numel", C.c_int64), ("update_math", C.c_int32), ("schedule", C.c_int32),
                 ("tile_elems", C.c_int32), ("tile_elems_maxima", C.c_int32), ("l2_keep_mbytes", C.c_int32),
-                ("lead_melems", C.c_int32), ("gap_items", C.c_int32), ("no_l2_hints", C.c_int32)]
+                ("lead_melems", C.c_int32), ("gap_items", C.c_int32), ("no_l2_hints", C.c_int32), ("overlap_groups", C.c_int32)]
 
 
 def default_config(v_mode: int = V_RANK1, min_quant_numel: int = 4096, update_math: int = 0, m_block: int = 128,
                    schedule: int = 0, tile_elems: int = 0, tile_elems_maxima: int = 0, l2_keep_mbytes: int = 0,
-                   lead_melems: int = 0, gap_items: int = 0, no_l2_hints: int = 0) -> Config:
+                   lead_melems: int = 0, gap_items: int = 0, no_l2_hints: int = 0, overlap_groups: int = 0) -> Config:
     return Config(4, m_block, 128, v_mode, min_quant_numel, update_math, schedule, tile_elems, tile_elems_maxima,
-                  l2_keep_mbytes, lead_melems, gap_items, no_l2_hints)
+                  l2_keep_mbytes, lead_melems, gap_items, no_l2_hints, overlap_groups)
 
 
 class LpmmError(RuntimeError):
