@@ -29,6 +29,8 @@ class Pair:
         self.config = config or lpmm.default_config()
         if schedule is not None:
             self.config.schedule = schedule
+            if schedule == lpmm.SCHEDULE_OVERLAP:
+                self.config.overlap_groups = 3
         self.grad_dtype = grad_dtype
         self.widx = workload_index
         self.params = [workloads.make_param(s, self.widx, i, device=device) for i, s in enumerate(self.specs)]

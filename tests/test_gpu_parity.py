@@ -23,6 +23,11 @@ TLIN = oracle.linear_map(4)
 SCHEDULES = pytest.mark.parametrize("schedule", [lpmm.SCHEDULE_TWO_PASS, lpmm.SCHEDULE_FUSED], ids=["two_pass", "fused"])
 
 
+# ... and, on lists with several rank-1 tensors, the overlapped form of the two-pass schedule (two streams, three groups).
+SCHEDULES3 = pytest.mark.parametrize("schedule", [lpmm.SCHEDULE_TWO_PASS, lpmm.SCHEDULE_FUSED, lpmm.SCHEDULE_OVERLAP],
+                                     ids=["two_pass", "fused", "overlap"])
+
+
 def _launches(schedule, two_pass):
     return 1 if schedule == lpmm.SCHEDULE_FUSED else two_pass
 
@@ -198,7 +203,7 @@ def test_single_matrix_config_ten_steps(update_math, schedule):
 
 @pytest.mark.parametrize("grad_dtype,update_math", [(torch.float32, lpmm.UPDATE_FAST), (torch.bfloat16, lpmm.UPDATE_FAST),
                                                     (torch.float32, lpmm.UPDATE_IEEE)])
-@SCHEDULES
+@SCHEDULES3
 def test_shape_zoo_multi_tensor(grad_dtype, update_math, schedule):
     specs = [_mat(96, 256), _mat(33, 77), _mat(5, 1000), _mat(130, 384), _mat(64, 1024), _mat(8, 2048),
              _mat(1, 8192), _mat(8192, 1), _mat(300, 640), _mat(257, 129), _mat(70, 128),
@@ -220,6 +225,7 @@ def test_shape_zoo_multi_tensor(grad_dtype, update_math, schedule):
             grads[12].mul_(1e-18)
         pair.step(t, grads)
         pair.compare(tol=1e-6)
+    assert pair.state.schedule == schedule
 
 
 @pytest.mark.parametrize("m_block,grad_dtype", [(128, torch.float32), (128, torch.bfloat16), (2048, torch.bfloat16),
@@ -253,7 +259,7 @@ def test_first_moment_block_2048(grad_dtype):
     assert pair.ostate[0].m_scale.size == 64     # one scale per 2048 elements
 
 
-@SCHEDULES
+@SCHEDULES3
 def test_transformer_base_three_steps_one_launch_per_pass(schedule):
     wl = workloads.transformer_base()
     pair = Pair(wl.tensors, hyper_of(wl), workload_index=wl.index, schedule=schedule)
@@ -262,7 +268,8 @@ def test_transformer_base_three_steps_one_launch_per_pass(schedule):
     for t in range(1, 4):
         pair.step(t, pair.grads_for(t))
         pair.compare(tol=1e-6)
-    assert pair.state.last_launches == _launches(schedule, 3)   # two-pass: maxima + reciprocal + update cover all 181 tensors
+    # two-pass: maxima + reciprocal + update cover all 181 tensors; overlapped: the same three per group of tensors
+    assert pair.state.last_launches == {lpmm.SCHEDULE_TWO_PASS: 3, lpmm.SCHEDULE_FUSED: 1, lpmm.SCHEDULE_OVERLAP: 9}[schedule]
 
 
 @SCHEDULES
