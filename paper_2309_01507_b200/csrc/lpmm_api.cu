@@ -38,11 +38,13 @@ struct TensorLayout {
     int32_t n_outer = 1;            // leading axes (Alg. 4 in general form: ndim - 1)
     int32_t outer_dim[3] = {0, 0, 0};
     int32_t outer_off[3] = {0, 0, 0};
+    size_t fact_rowpart = 0, fact_colpart = 0, fact_blockpart = 0;   // K_FACT: scratch for the partial sums of g^2
+    int32_t fact_nstrips = 0, fact_tiles_y = 0;
 };
 
 struct Layout {
     std::vector<TensorLayout> t;
-    size_t descs = 0, params = 0, params16 = 0, grads = 0, tiles1 = 0, tiles2 = 0, tiles3 = 0, tiles4 = 0;
+    size_t descs = 0, params = 0, params16 = 0, grads = 0, tiles1 = 0, tiles2 = 0, tiles3 = 0, tiles4 = 0, tiles5 = 0;
     size_t tsync = 0, work = 0;       // fused schedule: per-tensor progress counters, work list
     int64_t work_items = 0;           // capacity of the work list
     size_t rc[3] = {0, 0, 0}, rcp = 0;
@@ -271,6 +273,7 @@ void compute_layout(const lpmm_config& cfg, const lpmm_shape* shapes, int32_t n,
     L->tiles2 = off; off = align_up(off + sizeof(int32_t) * (n + 1));
     L->tiles3 = off; off = align_up(off + sizeof(int32_t) * (n + 1));
     L->tiles4 = off; off = align_up(off + sizeof(int32_t) * (n + 1));
+    L->tiles5 = off; off = align_up(off + sizeof(int32_t) * (n + 1));
     L->tsync = off;  off = align_up(off + sizeof(TensorSync) * n);
     int64_t rc = 0;
     for (int32_t i = 0; i < n; ++i) {
@@ -307,6 +310,8 @@ void compute_layout(const lpmm_config& cfg, const lpmm_shape* shapes, int32_t n,
     L->rc[1] = off; off = align_up(off + sizeof(float) * rc);
     L->rc[2] = off; off = align_up(off + sizeof(float) * rc);
     L->rcp = off;   off = align_up(off + sizeof(float) * rc);
+    int64_t total_elems = 0;
+    for (int32_t i = 0; i < n; ++i) total_elems += L->t[i].numel;
     for (int32_t i = 0; i < n; ++i) {
         TensorLayout& t = L->t[i];
         if (t.kind == K_FP32) {
@@ -322,9 +327,20 @@ void compute_layout(const lpmm_config& cfg, const lpmm_shape* shapes, int32_t n,
             if (t.kind == K_BLOCK || t.kind == K_BLOCK_TILED) { t.v_bscale = off; off = align_up(off + sizeof(float) * nblk); }
         }
     }
+    if (cfg.v_mode == LPMM_V_FACTORED) {   // scratch of the sums pass (same tile plan as build_tables)
+        const TileSizes ts = choose_tile_sizes(cfg, total_elems, false);
+        for (int32_t i = 0; i < n; ++i) {
+            TensorLayout& t = L->t[i];
+            if (t.kind != K_FACT) continue;
+            const TilePlan p = plan_tensor(cfg, t, ts);
+            t.fact_nstrips = (int32_t)((t.cols + kWarpElems - 1) / kWarpElems);
+            t.fact_tiles_y = (int32_t)((t.rows + p.tile_rows1 - 1) / p.tile_rows1);
+            t.fact_rowpart = off; off = align_up(off + sizeof(float) * (size_t)t.rows * t.fact_nstrips);
+            t.fact_colpart = off; off = align_up(off + sizeof(float) * (size_t)t.fact_tiles_y * t.cols);
+            t.fact_blockpart = off; off = align_up(off + sizeof(double) * (size_t)((t.c_off + (t.cols + 3) / 4 * 4 + 31) / 32));
+        }
+    }
     L->states_end = off;   // everything a checkpoint must keep lies below this offset
-    int64_t total_elems = 0;
-    for (int32_t i = 0; i < n; ++i) total_elems += L->t[i].numel;
     if (wants_fused(cfg, total_elems)) {   // the work list: one item per tile of either pass
         const TileSizes ts = choose_tile_sizes(cfg, total_elems, true);
         int64_t items = 0;
@@ -362,6 +378,7 @@ struct lpmm_state {
     uint32_t epoch = 0;                    // fused launches made on this state (the per-tensor counters count along)
     int32_t sms, occ1, occ2;
     int32_t p1_ctas;                       // which instantiation of the maxima pass (2 or 3 CTAs per SM)
+    std::vector<int32_t> tiles5;           // prefix sums of the factorized tensors' 32-statistic chunks (finalize kernel)
     std::vector<int32_t> tiles1, tiles2, tiles3;   // host copies of the tile prefix sums (3: element-indexed tiles of every tensor)
     cudaStream_t aux = nullptr;            // overlapped schedule: the stream of the maxima passes (lazily created)
     std::vector<cudaEvent_t> ov_events;    // overlapped schedule: per group {maxima done, update done}, then the fork event
@@ -467,7 +484,7 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
 
     std::vector<TensorDesc> descs(n);
     std::vector<TilePlan> plans(n);
-    std::vector<int32_t> t1(n + 1, 0), t2(n + 1, 0), t3(n + 1, 0), t4(n + 1, 0);
+    std::vector<int32_t> t1(n + 1, 0), t2(n + 1, 0), t3(n + 1, 0), t4(n + 1, 0), t5(n + 1, 0);
     // In a state whose matrices are not block-wise, folded 1-D tensors leave the main update launch (0 tiles there)
     // and get one of their own with the block-wise kernel (table 4).
     const bool own_launch = st->cfg.v_mode != LPMM_V_BLOCK;
@@ -495,6 +512,13 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
                 d.rcp_new = reinterpret_cast<float*>(A + st->L.rcp) + t.rc_index;
                 d.rc_floats = (int32_t)(t.c_off + (t.cols + 3) / 4 * 4);
             }
+            if (t.kind == K_FACT) {
+                d.fact_rowpart = reinterpret_cast<float*>(A + t.fact_rowpart);
+                d.fact_colpart = reinterpret_cast<float*>(A + t.fact_colpart);
+                d.fact_blockpart = reinterpret_cast<double*>(A + t.fact_blockpart);
+                d.fact_nstrips = t.fact_nstrips;
+                d.fact_tiles_y = t.fact_tiles_y;
+            }
         }
         const TilePlan p = plan_tensor(st->cfg, t, ts);
         plans[i] = p;
@@ -511,6 +535,8 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
         t4[i + 1] = t4[i] + (moved ? (int32_t)p.tiles_update : 0);
         if (t1[i] + p.tiles_maxima > 0x7fffffffLL) return LPMM_ERR_UNSUPPORTED;
         t1[i + 1] = t1[i] + (int32_t)p.tiles_maxima;
+        t5[i + 1] = t5[i] + (t.kind == K_FACT ? (d.rc_floats + 31) / 32 : 0);
+        if (t.kind == K_FACT && (int64_t)d.tile_rows1 * d.fact_tiles_y < t.rows) return LPMM_ERR_UNSUPPORTED;   // (layout and plan disagree)
     }
     st->total1 = t1[n];
     st->total2 = t2[n];
@@ -521,6 +547,8 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
     st->tiles2 = t2;
     st->tiles3 = t3;
     st->tiles4 = t4;
+    st->tiles5 = t5;
+    LPMM_CUDA(cudaMemcpyAsync(A + st->L.tiles5, t5.data(), sizeof(int32_t) * (n + 1), cudaMemcpyHostToDevice, s));
     {   // overlapped schedule: consecutive groups of about equal size, each with at least one maxima tile
         int32_t groups = st->cfg.overlap_groups > 0 ? st->cfg.overlap_groups : 8;
         st->group_cut.assign(1, 0);
@@ -766,7 +794,8 @@ lpmm_status enqueue_maxima(lpmm_state* st, StepArgs a, int32_t t0, int32_t t1, b
         rc_end = (t.rc_index + t.c_off + (t.cols + 3) / 4 * 4 + 63) / 64 * 64;
     }
     float* rc_new = reinterpret_cast<float*>(st->arena + st->L.rc[(st->phase + 1) % 3]) + rc_begin;
-    LPMM_CUDA(cudaMemsetAsync(rc_new, 0, sizeof(float) * (size_t)(rc_end - rc_begin), s));
+    const bool factored = st->cfg.v_mode == LPMM_V_FACTORED;    // (its sums are written, not accumulated: nothing to clear)
+    if (!factored) LPMM_CUDA(cudaMemsetAsync(rc_new, 0, sizeof(float) * (size_t)(rc_end - rc_begin), s));
     if (ev) LPMM_CUDA(cudaEventRecord(ev[0], s));
     a.tile_start = reinterpret_cast<const int32_t*>(st->arena + st->L.tiles1);
     a.tile_begin = p1_begin;
@@ -774,11 +803,15 @@ lpmm_status enqueue_maxima(lpmm_state* st, StepArgs a, int32_t t0, int32_t t1, b
     const int32_t tiles = p1_end - p1_begin;
     LPMM_CUDA(launch_pass1(a, bf16, st->p1_ctas, tiles < grid_cap ? tiles : grid_cap, s));
     if (ev) LPMM_CUDA(cudaEventRecord(ev[1], s));
-    LPMM_CUDA(launch_rcp(rc_new, reinterpret_cast<float*>(st->arena + st->L.rcp) + rc_begin, rc_end - rc_begin, s));
-    *launches += 2;
-    if (st->cfg.v_mode == LPMM_V_FACTORED) {   // statistics' moving averages and the row factors R_i / sum(R)
-        LPMM_CUDA(launch_factor_finalize(a, t0, t1, s));
-        *launches += 1;
+    if (factored) {   // partial sums -> statistics' moving averages, sum(R), row factors R_i / sum(R): one small kernel
+        a.tile_start = reinterpret_cast<const int32_t*>(st->arena + st->L.tiles5);
+        a.tile_begin = st->tiles5[t0];
+        a.tile_end = st->tiles5[t1];
+        LPMM_CUDA(launch_factor_finalize(a, s));
+        *launches += 2;
+    } else {
+        LPMM_CUDA(launch_rcp(rc_new, reinterpret_cast<float*>(st->arena + st->L.rcp) + rc_begin, rc_end - rc_begin, s));
+        *launches += 2;
     }
     return LPMM_OK;
 }

@@ -48,6 +48,12 @@ struct TensorDesc {
     int32_t tiles1;     // rank-1 kinds: tiles of the maxima pass
     int32_t tiles2;     // tiles of the update pass
     int32_t rc_floats;  // rank-1 kinds: floats of this tensor's share of rc[] / rcp_new (c_off + cols rounded up to 4)
+    // K_FACT: partial sums of g^2 written by the sums pass and added up in a fixed order by the finalize kernels
+    float* fact_rowpart;    // rows x fact_nstrips: one partial per row and 256-column strip
+    float* fact_colpart;    // fact_tiles_y x cols: one partial per column and tile row-block of the sums pass
+    double* fact_blockpart; // ceil(rc_floats / 32): each finalize CTA's share of sum(R)
+    int32_t fact_nstrips;
+    int32_t fact_tiles_y;
 };
 
 // Fused schedule: progress of one tensor. The counter is never reset: launch number e (1, 2, ...) of a state waits for
@@ -105,7 +111,7 @@ cudaError_t launch_fused_f32_fast(const StepArgs& a, int grid, cudaStream_t s);
 cudaError_t launch_fused_f32_ieee(const StepArgs& a, int grid, cudaStream_t s);
 cudaError_t launch_wait_selftest(const uint32_t* flag, uint32_t want, uint32_t limit, uint32_t* dev_status, int32_t* gave_up,
                                  cudaStream_t s);
-cudaError_t launch_factor_finalize(const StepArgs& a, int t0, int t1, cudaStream_t s);
+cudaError_t launch_factor_finalize(const StepArgs& a, cudaStream_t s);
 cudaError_t launch_sgdm(const StepArgs& a, bool bf16, int grid, cudaStream_t s);
 cudaError_t launch_rcp(const float* src, float* dst, int64_t n, cudaStream_t s);
 cudaError_t step_kernel_occupancy(int pass1_ctas_per_sm, int* pass1_blocks_per_sm, int* pass2_blocks_per_sm);

@@ -1093,78 +1093,169 @@ __device__ __forceinline__ void pass1_rank1_fast(const TensorDesc& d, const void
 
 // ---- pass 1 of the factorized second moment: row and column sums of g^2 (Sec. 4.3) ---------------------
 //
-// Same tiling as the maxima pass. Sums are accumulated in binary32 (eight squares per lane, a shuffle tree
-// per row, one register per column over the tile's rows) and combined across tiles with atomicAdd, so they
-// are reproducible to rounding only.
+// Same tiling as the maxima pass. Nothing is accumulated with atomics: every tile writes partial sums to a scratch
+// region of the arena and two small kernels add them up in a fixed order, so R and C are reproducible bit for bit
+// from run to run (and from GPU to GPU).
+//   row i:    one partial per 256-column strip (a lane adds its eight squares in order, then a shuffle tree over the
+//             warp), rowpart[i * nstrips + strip];
+//   column j: one partial per tile row-block: every warp adds its rows in increasing order with a compensated
+//             (Kahan) sum, so that the rounding error does not grow with the tile's height; the warps that share a
+//             column strip are combined in warp order through shared memory, colpart[ty * cols + j].
+// All arithmetic is binary32; the finalize kernels add the partials in binary64.
+
+__device__ __forceinline__ void kahan_add(float& s, float& c, float x) {
+    const float y = __fsub_rn(x, c);
+    const float t = __fadd_rn(s, y);
+    c = __fsub_rn(__fsub_rn(t, s), y);
+    s = t;
+}
 
 template <bool BF16>
-__device__ __forceinline__ void pass1_fact(const TensorDesc& d, const void* __restrict__ g, int tile, RcSel sel,
-                                           float* s_col) {
+__device__ __forceinline__ void pass1_fact(const TensorDesc& d, const void* __restrict__ g, int tile, float* s_col) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int wx = d.wx, wy_count = kWarps / wx;
     const int tx = tile % d.tiles_x, ty = tile / d.tiles_x;
     const int64_t col_w = (int64_t)tx * (kWarpElems * wx) + (warp % wx) * kWarpElems;
     const int64_t col0 = col_w + lane * kLaneElems;
     const bool active = col0 < d.cols;                  // cols % 256 == 128: the upper half-warp adds zeros
-    float* sums = rc_pick(d, sel.new_i);          // [row sums | column sums], cleared before the launch
+    const bool strip_exists = col_w < d.cols;
+    const int64_t strip = col_w / kWarpElems;
     const int64_t row0 = (int64_t)ty * d.tile_rows1 + warp / wx;
     const int64_t row_end = min((int64_t)(ty + 1) * d.tile_rows1, d.rows);
-    float c_sum[8];
+    float c_sum[8], c_cmp[8];
 #pragma unroll
-    for (int k = 0; k < 8; ++k) c_sum[k] = 0.0f;
-    for (int64_t i = row0; i < row_end; i += wy_count) {
-        float gv[8];
-        float rs = 0.0f;
-        if (active) {
-            load8_grad<BF16>(g, i * d.cols + col0, gv);
+    for (int k = 0; k < 8; ++k) { c_sum[k] = 0.0f; c_cmp[k] = 0.0f; }
+    for (int64_t i = row0; i < row_end; i += 4 * wy_count) {     // four rows of loads in flight
+        float gv[4][8];
 #pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                const float gg = __fmul_rn(gv[k], gv[k]);
-                rs = __fadd_rn(rs, gg);
-                c_sum[k] = __fadd_rn(c_sum[k], gg);
+        for (int u = 0; u < 4; ++u) {
+            const int64_t r = i + (int64_t)u * wy_count;
+            if (active && r < row_end) {
+                load8_grad<BF16>(g, r * d.cols + col0, gv[u]);
+            } else {
+#pragma unroll
+                for (int k = 0; k < 8; ++k) gv[u][k] = 0.0f;
             }
         }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) rs = __fadd_rn(rs, __shfl_xor_sync(0xffffffffu, rs, o));
-        if (lane == 0) atomicAdd(sums + i, rs);
+        for (int u = 0; u < 4; ++u) {
+            const int64_t r = i + (int64_t)u * wy_count;
+            float rs = 0.0f;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const float gg = __fmul_rn(gv[u][k], gv[u][k]);
+                rs = __fadd_rn(rs, gg);
+                kahan_add(c_sum[k], c_cmp[k], gg);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) rs = __fadd_rn(rs, __shfl_xor_sync(0xffffffffu, rs, o));
+            if (lane == 0 && strip_exists && r < row_end) d.fact_rowpart[r * d.fact_nstrips + strip] = rs;
+        }
     }
     float* mine = s_col + warp * kWarpElems;
-    __syncwarp();
 #pragma unroll
     for (int k = 0; k < 8; ++k) mine[lane * kLaneElems + k] = c_sum[k];
-    __syncwarp();
+    __syncthreads();
+    if (warp < wx) {                                    // the first warp of every column strip adds the strip's warps in order
 #pragma unroll
-    for (int k = 0; k < 8; ++k) {
-        const int cc = lane + 32 * k;
-        if (col_w + cc < d.cols) atomicAdd(sums + d.c_off + col_w + cc, mine[cc]);
+        for (int k = 0; k < 8; ++k) {
+            const int cc = lane + 32 * k;
+            float t = 0.0f;
+            for (int wy = 0; wy < wy_count; ++wy) t = __fadd_rn(t, s_col[(wy * wx + warp) * kWarpElems + cc]);
+            if (col_w + cc < d.cols) d.fact_colpart[(int64_t)ty * d.cols + col_w + cc] = t;
+        }
     }
+    // (the tile loop's barrier comes before anybody writes s_col again)
 }
 
 #if LPMM_STEP_PART == 0   // non-template kernels live in one part only
-// One CTA per factorized tensor: turns the sums into the statistics' moving averages R, C (in the "new"
-// buffer), sums R in binary64 in a fixed order and stores the row factors R_i * (1 / sum R).
-__global__ void __launch_bounds__(256) factor_finalize_kernel(StepArgs a, int t0) {
-    const TensorDesc d = a.descs[t0 + blockIdx.x];
-    if (d.kind != K_FACT) return;
+// Finalize: one CTA per 32 consecutive statistics of one factorized tensor ([R | C] index space), eight warps per
+// statistic: warp w adds the w-th eighth of the statistic's partial sums in order, the eighths are added in warp order
+// (binary64), the moving average is applied (R <- b2 R + (1 - b2) sum, reading of Sec. 4.3) and the CTA's share of
+// sum(R) goes to fact_blockpart[chunk]. The CTA that finishes a tensor's last chunk (a counter, no waiting) then adds
+// the shares in a fixed tree and stores the row factors R_i / sum(R). Every order is fixed, whichever CTA comes last.
+constexpr int kFactChunk = 32;
+
+__global__ void __launch_bounds__(256) factor_finalize_kernel(StepArgs a) {
+    const int chunk_g = a.tile_begin + blockIdx.x;
+    const int t = find_tensor(a.tile_start, a.n_tensors, chunk_g);
+    const TensorDesc d = a.descs[t];
+    const int chunk = chunk_g - __ldg(a.tile_start + t);
+    const int n_chunks = __ldg(a.tile_start + t + 1) - __ldg(a.tile_start + t);
     const float* old = rc_pick(d, a.sel.old_i);
     float* cur = rc_pick(d, a.sel.new_i);
-    __shared__ double s_part[256];
-    double part = 0.0;
-    for (int64_t i = threadIdx.x; i < d.rows; i += blockDim.x) {
-        const float r = __fadd_rn(__fmul_rn(a.h.beta2, old[i]), __fmul_rn(a.h.omb2, cur[i]));
-        cur[i] = r;
-        part += (double)r;
+    const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t idx = (int64_t)chunk * kFactChunk + lane;
+    const bool is_row = idx < d.rows, is_col = idx >= d.c_off && idx < d.c_off + d.cols;
+    __shared__ double s_part[8][32];
+    __shared__ double s_tree[256];
+    __shared__ int s_last;
+    // (binary64 additions are scarce on this part: an eighth is added in binary32 with a compensated sum, which is as
+    // good as exact for a few hundred terms, and only the eighths and what follows are added in binary64)
+    float part = 0.0f, comp = 0.0f;
+    if (is_row) {
+        const float* p = d.fact_rowpart + idx * d.fact_nstrips;
+        const int n = d.fact_nstrips, lo = n * w / 8, hi = n * (w + 1) / 8;
+        for (int k = lo; k < hi; ++k) kahan_add(part, comp, p[k]);
+    } else if (is_col) {
+        const float* p = d.fact_colpart + (idx - d.c_off);
+        const int n = d.fact_tiles_y, lo = n * w / 8, hi = n * (w + 1) / 8;
+        int k = lo;
+        for (; k + 4 <= hi; k += 4) {                              // four loads in flight, added in order
+            const float x0 = p[(int64_t)k * d.cols], x1 = p[(int64_t)(k + 1) * d.cols];
+            const float x2 = p[(int64_t)(k + 2) * d.cols], x3 = p[(int64_t)(k + 3) * d.cols];
+            kahan_add(part, comp, x0); kahan_add(part, comp, x1); kahan_add(part, comp, x2); kahan_add(part, comp, x3);
+        }
+        for (; k < hi; ++k) kahan_add(part, comp, p[(int64_t)k * d.cols]);
     }
-    for (int64_t j = threadIdx.x; j < d.cols; j += blockDim.x)
-        cur[d.c_off + j] = __fadd_rn(__fmul_rn(a.h.beta2, old[d.c_off + j]), __fmul_rn(a.h.omb2, cur[d.c_off + j]));
-    s_part[threadIdx.x] = part;
+    s_part[w][lane] = (double)part - (double)comp;
+    __syncthreads();
+    if (w == 0) {
+        double sum = 0.0;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) sum += s_part[k][lane];
+        double r_share = 0.0;
+        if (is_row || is_col) {
+            const float v = __fadd_rn(__fmul_rn(a.h.beta2, old[idx]), __fmul_rn(a.h.omb2, (float)sum));
+            cur[idx] = v;
+            if (is_row) r_share = (double)v;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) r_share += __shfl_xor_sync(0xffffffffu, r_share, o);
+        if (lane == 0) {
+            d.fact_blockpart[chunk] = r_share;
+            __threadfence();
+            s_last = (atomicAdd(&a.tsync[t].maxima_done, 1u) == (uint32_t)(n_chunks - 1));
+        }
+    }
+    __syncthreads();
+    if (!s_last) return;
+    // the tensor's last chunk: every statistic and every share is in place
+    __threadfence();
+    if (threadIdx.x == 0) a.tsync[t].maxima_done = 0u;
+    const int row_chunks = (int)((d.rows + kFactChunk - 1) / kFactChunk);
+    double mine = 0.0;
+    for (int c = threadIdx.x; c < row_chunks; c += 256) mine += __ldcg(d.fact_blockpart + c);
+    s_tree[threadIdx.x] = mine;
     __syncthreads();
     for (int o = 128; o > 0; o >>= 1) {
-        if ((int)threadIdx.x < o) s_part[threadIdx.x] += s_part[threadIdx.x + o];
+        if ((int)threadIdx.x < o) s_tree[threadIdx.x] += s_tree[threadIdx.x + o];
         __syncthreads();
     }
-    const float r_total = scale_rcp((float)s_part[0]);
-    for (int64_t i = threadIdx.x; i < d.rows; i += blockDim.x) d.rcp_new[i] = __fmul_rn(cur[i], r_total);
+    const float r_total = scale_rcp((float)s_tree[0]);
+    for (int64_t i0 = 0; i0 < d.rows; i0 += 8 * 256) {           // eight loads in flight per thread, then eight stores
+        float v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int64_t i = i0 + u * 256 + threadIdx.x;
+            v[u] = i < d.rows ? __ldcg(cur + i) : 0.0f;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int64_t i = i0 + u * 256 + threadIdx.x;
+            if (i < d.rows) d.rcp_new[i] = __fmul_rn(v[u], r_total);
+        }
+    }
 }
 #endif
 
@@ -1225,7 +1316,7 @@ __global__ void __launch_bounds__(kThreads, MINB) pass1_kernel(StepArgs a) {
         const void* g = a.grads[t];
         const int local = tile - __ldg(a.tile_start + t);
         if (d.kind == K_RANK1_FAST) pass1_rank1_fast<BF16>(d, g, local, a.sel, h2, lt, s_col);
-        else if (d.kind == K_FACT) pass1_fact<BF16>(d, g, local, a.sel, s_col);
+        else if (d.kind == K_FACT) pass1_fact<BF16>(d, g, local, s_col);
         else pass1_rank1_flat<BF16>(d, g, local, a.sel, a.h);
         tile = a.tile_begin + tiles_next(s_next, buf, fetched);
     }
@@ -1591,9 +1682,10 @@ cudaError_t launch_wait_selftest(const uint32_t* flag, uint32_t want, uint32_t l
     return cudaGetLastError();
 }
 
-cudaError_t launch_factor_finalize(const StepArgs& a, int t0, int t1, cudaStream_t s) {
-    if (t1 <= t0) return cudaSuccess;
-    factor_finalize_kernel<<<t1 - t0, 256, 0, s>>>(a, t0);
+// a.tile_start / tile_begin / tile_end: the table of 32-statistic chunks of the factorized tensors.
+cudaError_t launch_factor_finalize(const StepArgs& a, cudaStream_t s) {
+    if (a.tile_end <= a.tile_begin) return cudaSuccess;
+    factor_finalize_kernel<<<a.tile_end - a.tile_begin, 256, 0, s>>>(a);
     return cudaGetLastError();
 }
 
