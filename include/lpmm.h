@@ -66,8 +66,10 @@ typedef enum { LPMM_UPDATE_FAST = 0, LPMM_UPDATE_IEEE = 1 } lpmm_update_math;
  *             tail) fits. Needs the default quantizers (LPMM_V_RANK1, m_block 128); other states and
  *             lpmm_adamw4_step_bf16w / lpmm_adamw4_step_host run TWO_PASS. CTAs wait for one another through
  *             counters in the arena; every wait is bounded (see lpmm_state_device_status).
- *   AUTO:     FUSED where it applies, else TWO_PASS.
+ *   AUTO:     by measurement: FUSED for eligible states of fewer than 63 Mi elements, else TWO_PASS.
  * The stored states and the parameters are bit-identical under both schedules. */
+/*   OVERLAP:  TWO_PASS on groups of tensors, with the maxima pass of group k + 1 launched on a second stream (owned by the
+ *             handle) beside the update pass of group k; ordered by events, no device-side waiting. */
 typedef enum { LPMM_SCHEDULE_AUTO = 0, LPMM_SCHEDULE_TWO_PASS = 1, LPMM_SCHEDULE_FUSED = 2, LPMM_SCHEDULE_OVERLAP = 3 } lpmm_schedule;
 
 /* lpmm_shape.flags */
@@ -272,7 +274,22 @@ lpmm_status lpmm_state_selftest_wait(lpmm_state* st, int32_t* ctas_gave_up, int3
  * counters; synchronizes `stream`. A tuning aid for lead_melems / gap_items. */
 lpmm_status lpmm_state_wait_stats(lpmm_state* st, int64_t* waits, int64_t* wait_ns, void* stream);
 
-/* LPMM_SCHEDULE_TWO_PASS or LPMM_SCHEDULE_FUSED: what lpmm_adamw4_step runs on this state. */
+/* The checking build. The library can be compiled with -DLPMM_DEBUG (paper_2309_01507_b200/build.py builds it as
+ * liblpmm_debug.so beside the normal one); it stands in for a memory checker where none can be run:
+ *   - every sub-buffer of the arena is followed by a 256-byte guard zone filled with a pattern (so lpmm_state_bytes is
+ *     larger and arenas of the two builds cannot be attached to one another), and
+ *   - the step kernels check, per tile, that the first and last element they are about to touch lie inside the tensor;
+ *     a failed check puts 0x100 + its number into the device status word (lpmm_state_device_status) and the tile is
+ *     skipped - nothing traps.
+ * lpmm_build_is_checking() tells the two builds apart. lpmm_state_check_guards() counts the guard bytes that no longer
+ * hold the pattern (*zones receives the number of guard zones); lpmm_state_selftest_check() runs one check that fails on
+ * purpose and returns the status word it produced (0x17f), then clears it. Both return LPMM_ERR_UNSUPPORTED in the
+ * normal build and synchronize `stream`. */
+int32_t lpmm_build_is_checking(void);
+lpmm_status lpmm_state_check_guards(lpmm_state* st, int64_t* zones, int64_t* damaged, void* stream);
+lpmm_status lpmm_state_selftest_check(lpmm_state* st, int32_t* status_word, void* stream);
+
+/* LPMM_SCHEDULE_TWO_PASS, LPMM_SCHEDULE_FUSED or LPMM_SCHEDULE_OVERLAP: what lpmm_adamw4_step runs on this state. */
 int32_t lpmm_state_schedule(const lpmm_state* st);
 
 /* 0, 1 or 2: which of the three rank-1 scale buffers is current (they rotate: current, new, being cleared for the

@@ -52,12 +52,17 @@ struct Layout {
     size_t total = 0;
     size_t states_end = 0;            // end of the schedule-independent part (the work list comes after it)
     uint64_t shape_hash = 0;          // of everything the layout depends on (checked by lpmm_state_attach)
+    std::vector<size_t> guards;       // checking build: offsets of the 256-byte guard zones
 };
 
 // The first 256 bytes of the arena: device status word, the tile counters of a launch, and a description of the
 // layout that lpmm_state_attach compares with what the caller claims the arena holds.
 constexpr uint32_t kArenaMagic = 0x4d4d504cu;    // "LPMM"
+#ifdef LPMM_DEBUG
+constexpr uint32_t kArenaLayoutVersion = 0x80000002u;   // the checking build's arenas carry guard zones: another layout
+#else
 constexpr uint32_t kArenaLayoutVersion = 2u;     // bump whenever offsets or the meaning of a region change
+#endif
 struct ArenaHeader {
     uint32_t status;          // byte 0: device status word (0 = ok)
     uint32_t pad0[3];
@@ -244,6 +249,21 @@ TilePlan plan_tensor(const lpmm_config& cfg, const TensorLayout& t, const TileSi
     return p;
 }
 
+// End of a sub-buffer that stops at byte `end`: the next 256-byte boundary. The checking build (-DLPMM_DEBUG) puts a
+// guard zone of 256 bytes behind every sub-buffer, filled with a pattern at initialisation and never written by any
+// kernel: lpmm_state_check_guards() finds a stray write that crossed a sub-buffer's end.
+#ifdef LPMM_DEBUG
+constexpr bool kGuards = true;
+#else
+constexpr bool kGuards = false;
+#endif
+constexpr unsigned char kGuardByte = 0xC5;
+size_t region_end(Layout* L, size_t end) {
+    size_t e = align_up(end);
+    if (kGuards) { L->guards.push_back(e); e += kAlign; }
+    return e;
+}
+
 uint64_t fnv1a(uint64_t h, const void* data, size_t bytes) {
     const unsigned char* p = static_cast<const unsigned char*>(data);
     for (size_t i = 0; i < bytes; ++i) { h ^= p[i]; h *= 1099511628211ull; }
@@ -252,6 +272,7 @@ uint64_t fnv1a(uint64_t h, const void* data, size_t bytes) {
 
 void compute_layout(const lpmm_config& cfg, const lpmm_shape* shapes, int32_t n, Layout* L) {
     L->t.resize(n);
+    L->guards.clear();
     {
         uint64_t h = 1469598103934665603ull;
         const int64_t c[5] = {cfg.bits, cfg.m_block, cfg.v_block, cfg.v_mode, cfg.min_quant_numel};
@@ -265,16 +286,16 @@ void compute_layout(const lpmm_config& cfg, const lpmm_shape* shapes, int32_t n,
         L->shape_hash = h;
     }
     size_t off = kAlign;  // header block
-    L->descs = off;  off = align_up(off + sizeof(TensorDesc) * n);
-    L->params = off; off = align_up(off + sizeof(void*) * n);
-    L->params16 = off; off = align_up(off + sizeof(void*) * n);
-    L->grads = off;  off = align_up(off + sizeof(void*) * n);
-    L->tiles1 = off; off = align_up(off + sizeof(int32_t) * (n + 1));
-    L->tiles2 = off; off = align_up(off + sizeof(int32_t) * (n + 1));
-    L->tiles3 = off; off = align_up(off + sizeof(int32_t) * (n + 1));
-    L->tiles4 = off; off = align_up(off + sizeof(int32_t) * (n + 1));
-    L->tiles5 = off; off = align_up(off + sizeof(int32_t) * (n + 1));
-    L->tsync = off;  off = align_up(off + sizeof(TensorSync) * n);
+    L->descs = off;  off = region_end(L, off + sizeof(TensorDesc) * n);
+    L->params = off; off = region_end(L, off + sizeof(void*) * n);
+    L->params16 = off; off = region_end(L, off + sizeof(void*) * n);
+    L->grads = off;  off = region_end(L, off + sizeof(void*) * n);
+    L->tiles1 = off; off = region_end(L, off + sizeof(int32_t) * (n + 1));
+    L->tiles2 = off; off = region_end(L, off + sizeof(int32_t) * (n + 1));
+    L->tiles3 = off; off = region_end(L, off + sizeof(int32_t) * (n + 1));
+    L->tiles4 = off; off = region_end(L, off + sizeof(int32_t) * (n + 1));
+    L->tiles5 = off; off = region_end(L, off + sizeof(int32_t) * (n + 1));
+    L->tsync = off;  off = region_end(L, off + sizeof(TensorSync) * n);
     int64_t rc = 0;
     for (int32_t i = 0; i < n; ++i) {
         TensorLayout& t = L->t[i];
@@ -306,25 +327,25 @@ void compute_layout(const lpmm_config& cfg, const lpmm_shape* shapes, int32_t n,
         }
     }
     L->rc_floats = rc;
-    L->rc[0] = off; off = align_up(off + sizeof(float) * rc);
-    L->rc[1] = off; off = align_up(off + sizeof(float) * rc);
-    L->rc[2] = off; off = align_up(off + sizeof(float) * rc);
-    L->rcp = off;   off = align_up(off + sizeof(float) * rc);
+    L->rc[0] = off; off = region_end(L, off + sizeof(float) * rc);
+    L->rc[1] = off; off = region_end(L, off + sizeof(float) * rc);
+    L->rc[2] = off; off = region_end(L, off + sizeof(float) * rc);
+    L->rcp = off;   off = region_end(L, off + sizeof(float) * rc);
     int64_t total_elems = 0;
     for (int32_t i = 0; i < n; ++i) total_elems += L->t[i].numel;
     for (int32_t i = 0; i < n; ++i) {
         TensorLayout& t = L->t[i];
         if (t.kind == K_FP32) {
-            t.m32 = off; off = align_up(off + sizeof(float) * t.numel);
-            t.v32 = off; off = align_up(off + sizeof(float) * t.numel);
+            t.m32 = off; off = region_end(L, off + sizeof(float) * t.numel);
+            t.v32 = off; off = region_end(L, off + sizeof(float) * t.numel);
         } else {
             const size_t code_bytes = (size_t)((t.numel + 1) / 2);
             const size_t nblk = (size_t)((t.numel + 127) / 128);
             const size_t nblk_m = (size_t)((t.numel + cfg.m_block - 1) / cfg.m_block);
-            t.m_codes = off; off = align_up(off + code_bytes);
-            if (t.kind != K_FACT) { t.v_codes = off; off = align_up(off + code_bytes); }
-            t.m_scale = off; off = align_up(off + sizeof(float) * nblk_m);
-            if (t.kind == K_BLOCK || t.kind == K_BLOCK_TILED) { t.v_bscale = off; off = align_up(off + sizeof(float) * nblk); }
+            t.m_codes = off; off = region_end(L, off + code_bytes);
+            if (t.kind != K_FACT) { t.v_codes = off; off = region_end(L, off + code_bytes); }
+            t.m_scale = off; off = region_end(L, off + sizeof(float) * nblk_m);
+            if (t.kind == K_BLOCK || t.kind == K_BLOCK_TILED) { t.v_bscale = off; off = region_end(L, off + sizeof(float) * nblk); }
         }
     }
     if (cfg.v_mode == LPMM_V_FACTORED) {   // scratch of the sums pass (same tile plan as build_tables)
@@ -335,9 +356,9 @@ void compute_layout(const lpmm_config& cfg, const lpmm_shape* shapes, int32_t n,
             const TilePlan p = plan_tensor(cfg, t, ts);
             t.fact_nstrips = (int32_t)((t.cols + kWarpElems - 1) / kWarpElems);
             t.fact_tiles_y = (int32_t)((t.rows + p.tile_rows1 - 1) / p.tile_rows1);
-            t.fact_rowpart = off; off = align_up(off + sizeof(float) * (size_t)t.rows * t.fact_nstrips);
-            t.fact_colpart = off; off = align_up(off + sizeof(float) * (size_t)t.fact_tiles_y * t.cols);
-            t.fact_blockpart = off; off = align_up(off + sizeof(double) * (size_t)((t.c_off + (t.cols + 3) / 4 * 4 + 31) / 32));
+            t.fact_rowpart = off; off = region_end(L, off + sizeof(float) * (size_t)t.rows * t.fact_nstrips);
+            t.fact_colpart = off; off = region_end(L, off + sizeof(float) * (size_t)t.fact_tiles_y * t.cols);
+            t.fact_blockpart = off; off = region_end(L, off + sizeof(double) * (size_t)((t.c_off + (t.cols + 3) / 4 * 4 + 31) / 32));
         }
     }
     L->states_end = off;   // everything a checkpoint must keep lies below this offset
@@ -349,7 +370,7 @@ void compute_layout(const lpmm_config& cfg, const lpmm_shape* shapes, int32_t n,
             items += p.tiles_update + p.tiles_maxima;
         }
         L->work_items = items;
-        L->work = off; off = align_up(off + sizeof(uint2) * (size_t)items);
+        L->work = off; off = region_end(L, off + sizeof(uint2) * (size_t)items);
     }
     L->total = off;
 }
@@ -497,6 +518,7 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
         d.n_outer = t.n_outer;
         for (int a = 0; a < 3; ++a) { d.outer_dim[a] = t.outer_dim[a]; d.outer_off[a] = t.outer_off[a]; }
         d.m_shift = (st->cfg.m_block == 2048) ? 11 : 7;
+        d.dbg_status = reinterpret_cast<uint32_t*>(A);
         if (t.kind == K_FP32) {
             d.m32 = reinterpret_cast<float*>(A + t.m32);
             d.v32 = reinterpret_cast<float*>(A + t.v32);
@@ -621,6 +643,8 @@ lpmm_status make_state(const lpmm_config* cfg, const lpmm_shape* shapes, int32_t
             if (e == cudaSuccess && (t.numel & 1))
                 e = cudaMemsetAsync(st->arena + t.m_codes + t.numel / 2, 0x07, 1, s);
         }
+        for (size_t k = 0; k < st->L.guards.size() && e == cudaSuccess; ++k)
+            e = cudaMemsetAsync(st->arena + st->L.guards[k], kGuardByte, kAlign, s);
         if (e != cudaSuccess) rc = cuda_fail(e);
     } else {
         // An attached arena must describe itself as what the caller says it is ...
@@ -1238,6 +1262,38 @@ lpmm_status lpmm_state_wait_stats(lpmm_state* st, int64_t* waits, int64_t* wait_
     LPMM_CUDA(cudaMemsetAsync(p, 0, sizeof(w), s));
     *waits = (int64_t)w[0];
     *wait_ns = (int64_t)w[1];
+    return LPMM_OK;
+}
+
+lpmm_status lpmm_state_check_guards(lpmm_state* st, int64_t* zones, int64_t* damaged, void* stream) {
+    if (!st || !zones || !damaged) return LPMM_ERR_INVALID_ARG;
+    if (!kGuards) return LPMM_ERR_UNSUPPORTED;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    ArenaHeader* hd = reinterpret_cast<ArenaHeader*>(st->arena);
+    LPMM_CUDA(cudaMemsetAsync(hd->pad1, 0, sizeof(hd->pad1), s));
+    for (size_t k = 0; k < st->L.guards.size(); ++k)
+        LPMM_CUDA(launch_guard_check(reinterpret_cast<const unsigned char*>(st->arena + st->L.guards[k]), (int)kAlign, kGuardByte, &hd->pad1[0], s));
+    uint32_t bad = 0;
+    LPMM_CUDA(cudaMemcpyAsync(&bad, &hd->pad1[0], sizeof(bad), cudaMemcpyDeviceToHost, s));
+    LPMM_CUDA(cudaStreamSynchronize(s));
+    LPMM_CUDA(cudaMemsetAsync(hd->pad1, 0, sizeof(hd->pad1), s));
+    *zones = (int64_t)st->L.guards.size();
+    *damaged = (int64_t)bad;
+    return LPMM_OK;
+}
+
+int32_t lpmm_build_is_checking(void) { return kGuards ? 1 : 0; }
+
+lpmm_status lpmm_state_selftest_check(lpmm_state* st, int32_t* status_word, void* stream) {
+    if (!st || !status_word) return LPMM_ERR_INVALID_ARG;
+    if (!kGuards) return LPMM_ERR_UNSUPPORTED;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    uint32_t word = 0;
+    LPMM_CUDA(launch_check_selftest(reinterpret_cast<uint32_t*>(st->arena), s));
+    LPMM_CUDA(cudaMemcpyAsync(&word, st->arena, sizeof(word), cudaMemcpyDeviceToHost, s));
+    LPMM_CUDA(cudaStreamSynchronize(s));
+    LPMM_CUDA(cudaMemsetAsync(st->arena, 0, 4, s));
+    *status_word = (int32_t)word;
     return LPMM_OK;
 }
 

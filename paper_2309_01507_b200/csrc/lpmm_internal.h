@@ -54,7 +54,19 @@ struct TensorDesc {
     double* fact_blockpart; // ceil(rc_floats / 32): each finalize CTA's share of sum(R)
     int32_t fact_nstrips;
     int32_t fact_tiles_y;
+    uint32_t* dbg_status;   // the arena's device status word (written by the checking build's index checks)
 };
+
+// Index checks of the checking build (-DLPMM_DEBUG): a failed check records its code in the device status word (the
+// first failure wins) and evaluates to false, on which the tile functions return without touching memory. Nothing
+// traps. In the normal build the macro is the constant true.
+constexpr uint32_t kStatusCheckBase = 0x100u;   // status words >= this: a failed index check, low byte = which one
+#ifdef LPMM_DEBUG
+#define LPMM_DBG_OK(desc, cond, code) \
+    ((cond) ? true : (atomicCAS((desc).dbg_status, 0u, kStatusCheckBase + (uint32_t)(code)), false))
+#else
+#define LPMM_DBG_OK(desc, cond, code) (true)
+#endif
 
 // Fused schedule: progress of one tensor. The counter is never reset: launch number e (1, 2, ...) of a state waits for
 // e * tiles1, modulo 2^32.
@@ -111,6 +123,8 @@ cudaError_t launch_fused_f32_fast(const StepArgs& a, int grid, cudaStream_t s);
 cudaError_t launch_fused_f32_ieee(const StepArgs& a, int grid, cudaStream_t s);
 cudaError_t launch_wait_selftest(const uint32_t* flag, uint32_t want, uint32_t limit, uint32_t* dev_status, int32_t* gave_up,
                                  cudaStream_t s);
+cudaError_t launch_check_selftest(uint32_t* dev_status, cudaStream_t s);
+cudaError_t launch_guard_check(const unsigned char* zone, int bytes, unsigned char want, uint32_t* damaged, cudaStream_t s);
 cudaError_t launch_factor_finalize(const StepArgs& a, cudaStream_t s);
 cudaError_t launch_sgdm(const StepArgs& a, bool bf16, int grid, cudaStream_t s);
 cudaError_t launch_rcp(const float* src, float* dst, int64_t n, cudaStream_t s);

@@ -545,6 +545,10 @@ __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __r
     const int64_t row_end = min((int64_t)(ty + 1) * d.tile_rows, d.rows);
     if (row0 >= row_end) return;
     const uint32_t nrows = (uint32_t)((row_end - row0 + wy_count - 1) / wy_count);
+    // checking build: the lane's first and last accesses of this tile lie inside the tensor (B2048 tiles end rows in a
+    // CTA-wide barrier, so there the failure is recorded and the tile goes on)
+    if (!LPMM_DBG_OK(d, tile >= 0 && tile < d.tiles2 && col0 + kLaneElems <= d.cols && row0 + (int64_t)(nrows - 1) * wy_count < d.rows &&
+                        (row0 + (int64_t)(nrows - 1) * wy_count) * d.cols + col0 + kLaneElems <= d.numel, 1) && MSHIFT == 7) return;
 
     float c_old[8], c_rcp[8];
     if (VM == 2) {   // no row / column statistics at all
@@ -680,6 +684,8 @@ __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restric
     const float* rc_old = rc_pick(d, sel.old_i);
     const float* rcp_new = d.rcp_new;
     const int64_t m_mask = ((int64_t)1 << MSHIFT) - 1;
+    // checking build: the tile starts inside the tensor (B2048: recorded only, the CTA-wide barrier needs every warp)
+    if (!LPMM_DBG_OK(d, tile >= 0 && (int64_t)tile * d.flat_chunks * kWarps * kWarpElems < d.numel, 3) && MSHIFT == 7) return;
     for (int c = 0; c < d.flat_chunks; ++c) {
         const int64_t chunk0 = ((int64_t)tile * d.flat_chunks + c) * kWarps;   // the CTA's 8 chunks = 2048 elements
         const int64_t chunk = chunk0 + warp;
@@ -783,6 +789,7 @@ template <bool BF16, bool EXACT, bool WB = false, bool A32 = false>
 __device__ __forceinline__ void pass2_fp32(const TensorDesc& d, float* __restrict__ w, uint16_t* __restrict__ w16,
                                            const void* __restrict__ g, int tile, const Hyper& h) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (!LPMM_DBG_OK(d, tile >= 0 && (int64_t)tile * d.flat_chunks * kWarps * kWarpElems < d.numel && d.m32 != nullptr && d.v32 != nullptr, 4)) return;
     for (int c = 0; c < d.flat_chunks; ++c) {
         const int64_t chunk = ((int64_t)tile * d.flat_chunks + c) * kWarps + warp;
         const int64_t e = chunk * kWarpElems + lane * kLaneElems;
@@ -1021,6 +1028,8 @@ __device__ __forceinline__ void pass1_rank1_fast(const TensorDesc& d, const void
     const int64_t row_end = min((int64_t)(ty + 1) * d.tile_rows1, d.rows);
     if (row0 >= row_end) return;                      // uniform over the warp
     const uint32_t nrows = (uint32_t)((row_end - row0 + wy_count - 1) / wy_count);
+    if (!LPMM_DBG_OK(d, tile >= 0 && tile < d.tiles1 && col0 >= 0 && col0 + kLaneElems <= d.cols &&
+                        row0 + (int64_t)(nrows - 1) * wy_count < d.rows, 2)) return;
 
     float c_old[8], c_max[8];
 #pragma unroll
@@ -1385,6 +1394,12 @@ __global__ void __launch_bounds__(kThreads, 2) step_fused_kernel(StepArgs a) {
         const int t = (int)(item.x & kWorkTensorMask);
         const bool update = (item.x & kWorkUpdate) != 0, keep = (item.x & kWorkKeep) != 0;
         const int local = (int)item.y;
+        if (t >= a.n_tensors) {            // (never: the host built the list; the checking build says so before stopping)
+#ifdef LPMM_DEBUG
+            atomicCAS(a.dev_status, 0u, kStatusCheckBase + 6u);
+#endif
+            break;
+        }
         const TensorDesc d = a.descs[t];
         const void* g = a.grads[t];
         TensorSync* sy = a.tsync + t;
@@ -1674,6 +1689,27 @@ cudaError_t launch_fused(const StepArgs& a, bool bf16, bool exact, int grid, cud
     if (a.tile_end <= a.tile_begin) return cudaSuccess;
     if (bf16) return exact ? launch_fused_bf16_ieee(a, grid, s) : launch_fused_bf16_fast(a, grid, s);
     return exact ? launch_fused_f32_ieee(a, grid, s) : launch_fused_f32_fast(a, grid, s);
+}
+
+// Checking build: counts the bytes of one guard zone that no longer hold the pattern.
+__global__ void guard_check_kernel(const unsigned char* zone, int bytes, unsigned char want, uint32_t* damaged) {
+    for (int i = threadIdx.x; i < bytes; i += blockDim.x)
+        if (zone[i] != want) atomicAdd(damaged, 1u);
+}
+cudaError_t launch_guard_check(const unsigned char* zone, int bytes, unsigned char want, uint32_t* damaged, cudaStream_t s) {
+    guard_check_kernel<<<1, 256, 0, s>>>(zone, bytes, want, damaged);
+    return cudaGetLastError();
+}
+// A check that fails on purpose (host-requested): shows that a failed index check reaches the status word.
+__global__ void check_selftest_kernel(uint32_t* dev_status) {
+    TensorDesc d;
+    d.dbg_status = dev_status;
+    d.numel = 0;
+    if (!LPMM_DBG_OK(d, d.numel > 0, 0x7f)) return;
+}
+cudaError_t launch_check_selftest(uint32_t* dev_status, cudaStream_t s) {
+    check_selftest_kernel<<<1, 1, 0, s>>>(dev_status);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_wait_selftest(const uint32_t* flag, uint32_t want, uint32_t limit, uint32_t* dev_status, int32_t* gave_up,

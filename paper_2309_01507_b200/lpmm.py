@@ -32,7 +32,8 @@ EXPORTS = ("lpmm_state_bytes", "lpmm_state_init", "lpmm_state_attach", "lpmm_ada
            "lpmm_quantize_rank1_noalloc", "lpmm_sgdm4_step",
            "lpmm_state_view", "lpmm_state_view_axis", "lpmm_state_phase", "lpmm_state_last_launches", "lpmm_state_destroy",
            "lpmm_state_profile", "lpmm_state_profile_read", "lpmm_state_device_status", "lpmm_state_selftest_wait",
-           "lpmm_state_schedule", "lpmm_state_wait_stats",
+           "lpmm_state_schedule", "lpmm_state_wait_stats", "lpmm_build_is_checking", "lpmm_state_check_guards",
+           "lpmm_state_selftest_check",
            "lpmm_status_string", "lpmm_last_cuda_error")
 
 
@@ -80,6 +81,14 @@ class LpmmError(RuntimeError):
 _lib = None
 
 
+def use_library(path: str) -> None:
+    """Binds this module to another build of the library (e.g. the checking build liblpmm_debug.so). Call it before
+    anything else in the process: states made by one build must not be handed to another."""
+    global _lib, LIB_PATH
+    LIB_PATH = path
+    _lib = None
+
+
 def lib():
     """Loads liblpmm.so; fails loudly if it has not been built (python -m paper_2309_01507_b200.build)."""
     global _lib
@@ -110,6 +119,9 @@ def lib():
         L.lpmm_state_selftest_wait.argtypes = [vp, C.POINTER(i32), C.POINTER(i32), vp]
         L.lpmm_state_schedule.argtypes = [vp]
         L.lpmm_state_wait_stats.argtypes = [vp, C.POINTER(i64), C.POINTER(i64), vp]
+        L.lpmm_build_is_checking.argtypes = []
+        L.lpmm_state_check_guards.argtypes = [vp, C.POINTER(i64), C.POINTER(i64), vp]
+        L.lpmm_state_selftest_check.argtypes = [vp, C.POINTER(i32), vp]
         L.lpmm_state_phase.argtypes = [vp]
         L.lpmm_state_last_launches.argtypes = [vp]
         L.lpmm_state_destroy.argtypes = [vp]
@@ -304,6 +316,22 @@ def wait_stats(state: State, stream=None):
     with torch.cuda.device(state.arena.device):
         _check(lib().lpmm_state_wait_stats(state.handle, C.byref(n), C.byref(ns), _stream_ptr(stream)), "lpmm_state_wait_stats")
     return n.value, ns.value
+
+
+def check_guards(state: State, stream=None):
+    """lpmm_state_check_guards (checking build only): (guard zones, damaged bytes)."""
+    z, b = C.c_int64(), C.c_int64()
+    with torch.cuda.device(state.arena.device):
+        _check(lib().lpmm_state_check_guards(state.handle, C.byref(z), C.byref(b), _stream_ptr(stream)), "lpmm_state_check_guards")
+    return z.value, b.value
+
+
+def selftest_check(state: State, stream=None) -> int:
+    """lpmm_state_selftest_check (checking build only): the status word a failing index check leaves."""
+    w = C.c_int32()
+    with torch.cuda.device(state.arena.device):
+        _check(lib().lpmm_state_selftest_check(state.handle, C.byref(w), _stream_ptr(stream)), "lpmm_state_selftest_check")
+    return w.value
 
 
 def stage_bytes(state: State) -> int:
