@@ -38,13 +38,21 @@ struct TensorLayout {
     int32_t n_outer = 1;            // leading axes (Alg. 4 in general form: ndim - 1)
     int32_t outer_dim[3] = {0, 0, 0};
     int32_t outer_off[3] = {0, 0, 0};
+    int32_t rc_len = 0;             // floats of this tensor's share of every rank-1 scale buffer (all axes, padded)
+    int32_t nd = 0;                 // three or four axes: their number, extents and offsets inside the tensor's share
+    int32_t nd_dim[4] = {0, 0, 0, 0};
+    int32_t nd_off[4] = {0, 0, 0, 0};
+    bool p1_tiled = false;          // K_RANK1_FLAT matrix whose maxima pass runs on the tiled kernel (cols % 8 == 0)
+    int32_t nd_split = 0;           // > 0: composite tensor on the tiled path, axes [0, nd_split) are its rows
+    size_t exp_old = 0, exp_new = 0, exp_rcp = 0;   // composite: per-step expanded statistics (arena offsets)
+    int32_t exp_len = 0;
     size_t fact_rowpart = 0, fact_colpart = 0, fact_blockpart = 0;   // K_FACT: scratch for the partial sums of g^2
     int32_t fact_nstrips = 0, fact_tiles_y = 0;
 };
 
 struct Layout {
     std::vector<TensorLayout> t;
-    size_t descs = 0, params = 0, params16 = 0, grads = 0, tiles1 = 0, tiles2 = 0, tiles3 = 0, tiles4 = 0, tiles5 = 0;
+    size_t descs = 0, params = 0, params16 = 0, grads = 0, tiles1 = 0, tiles2 = 0, tiles3 = 0, tiles4 = 0, tiles5 = 0, tiles6 = 0, tiles7 = 0;
     size_t tsync = 0, work = 0;       // fused schedule: per-tensor progress counters, work list
     int64_t work_items = 0;           // capacity of the work list
     size_t rc[3] = {0, 0, 0}, rcp = 0;
@@ -222,7 +230,7 @@ struct TilePlan {
 TilePlan plan_tensor(const lpmm_config& cfg, const TensorLayout& t, const TileSizes& ts) {
     TilePlan p;
     const bool tiled = t.kind == K_RANK1_FAST || t.kind == K_FACT || t.kind == K_BLOCK_TILED;
-    if (tiled) {
+    if (tiled || t.p1_tiled) {
         p.wx = (cfg.m_block == 2048) ? 8 : (t.cols % 1024 == 0) ? 4 : (t.cols % 512 == 0) ? 2 : 1;
         const int64_t tile_cols = (int64_t)kWarpElems * p.wx;
         int64_t tr = ts.update / tile_cols;
@@ -235,6 +243,7 @@ TilePlan plan_tensor(const lpmm_config& cfg, const TensorLayout& t, const TileSi
         if (tr1 < tr) tr1 = tr;
         p.tile_rows1 = (int32_t)tr1;
         if (t.kind != K_BLOCK_TILED) p.tiles_maxima = (int64_t)p.tiles_x * ((t.rows + tr1 - 1) / tr1);
+        if (!tiled) p.tiles_update = 0;   // (set below: the update pass of such a tensor is element-indexed)
     }
     int64_t chunks = ts.update / (kWarps * kWarpElems);
     if (chunks < 1) chunks = 1;
@@ -244,7 +253,7 @@ TilePlan plan_tensor(const lpmm_config& cfg, const TensorLayout& t, const TileSi
     p.tiles_flat = (t.numel + per_tile - 1) / per_tile;
     if (!tiled) {
         p.tiles_update = p.tiles_flat;
-        if (t.kind == K_RANK1_FLAT) p.tiles_maxima = p.tiles_flat;
+        if (t.kind == K_RANK1_FLAT && !t.p1_tiled) p.tiles_maxima = p.tiles_flat;
     }
     return p;
 }
@@ -295,6 +304,8 @@ void compute_layout(const lpmm_config& cfg, const lpmm_shape* shapes, int32_t n,
     L->tiles3 = off; off = region_end(L, off + sizeof(int32_t) * (n + 1));
     L->tiles4 = off; off = region_end(L, off + sizeof(int32_t) * (n + 1));
     L->tiles5 = off; off = region_end(L, off + sizeof(int32_t) * (n + 1));
+    L->tiles6 = off; off = region_end(L, off + sizeof(int32_t) * (n + 1));
+    L->tiles7 = off; off = region_end(L, off + sizeof(int32_t) * (n + 1));
     L->tsync = off;  off = region_end(L, off + sizeof(TensorSync) * n);
     int64_t rc = 0;
     for (int32_t i = 0; i < n; ++i) {
@@ -317,12 +328,20 @@ void compute_layout(const lpmm_config& cfg, const lpmm_shape* shapes, int32_t n,
                     o += (shapes[i].dims[a] + 3) / 4 * 4;
                 }
                 t.c_off = (int32_t)o;
+                t.nd = shapes[i].ndim;
+                for (int32_t a = 0; a < t.nd; ++a) {
+                    t.nd_dim[a] = (int32_t)shapes[i].dims[a];
+                    t.nd_off[a] = a + 1 < t.nd ? t.outer_off[a] : t.c_off;
+                }
             } else {
                 t.n_outer = 1;
                 t.outer_dim[0] = (int32_t)t.rows;
                 t.c_off = (int32_t)((t.rows + 3) / 4 * 4);
             }
-            rc += t.c_off + (t.cols + 3) / 4 * 4;
+            t.rc_len = (int32_t)(t.c_off + (t.cols + 3) / 4 * 4);
+            t.p1_tiled = t.kind == K_RANK1_FLAT && shapes[i].ndim == 2 && t.cols % 8 == 0 && t.cols >= 128 &&
+                         t.cols <= ((int64_t)1 << 24);
+            rc += t.rc_len;
             rc = (rc + 63) / 64 * 64;  // 256-byte granules so r and c always start 16-byte aligned
         }
     }
@@ -333,6 +352,34 @@ void compute_layout(const lpmm_config& cfg, const lpmm_shape* shapes, int32_t n,
     L->rcp = off;   off = region_end(L, off + sizeof(float) * rc);
     int64_t total_elems = 0;
     for (int32_t i = 0; i < n; ++i) total_elems += L->t[i].numel;
+    // Tensors with three or four axes whose trailing axes multiply to whole first-moment blocks go to the tiled path as
+    // "composite" matrices (leading axes = rows, trailing axes = columns) with per-step expanded statistics. (Not under
+    // the fused schedule, whose element-indexed tiles handle them.)
+    if (!wants_fused(cfg, total_elems)) {
+        for (int32_t i = 0; i < n; ++i) {
+            TensorLayout& t = L->t[i];
+            if (t.kind != K_RANK1_FLAT || t.nd < 3) continue;
+            int32_t best = 0;
+            int64_t best_cols = 0;
+            for (int32_t sp = t.nd - 1; sp >= 1; --sp) {
+                int64_t c = 1;
+                for (int32_t a = sp; a < t.nd; ++a) c *= t.nd_dim[a];
+                if (c % 128 != 0 || c % cfg.m_block != 0 || c > ((int64_t)1 << 24)) continue;
+                if (best == 0 || (best_cols < 1024 && c > best_cols)) { best = sp; best_cols = c; }   // the narrowest one that fills a tile
+            }
+            if (best == 0) continue;
+            t.kind = K_RANK1_FAST;
+            t.nd_split = best;
+            t.cols = best_cols;
+            t.rows = t.numel / best_cols;
+            t.n_outer = 1;
+            t.c_off = (int32_t)((t.rows + 3) / 4 * 4);
+            t.exp_len = (int32_t)(t.c_off + (t.cols + 3) / 4 * 4);
+            t.exp_old = off; off = region_end(L, off + sizeof(float) * (size_t)t.exp_len);
+            t.exp_new = off; off = region_end(L, off + sizeof(float) * (size_t)t.exp_len);
+            t.exp_rcp = off; off = region_end(L, off + sizeof(float) * (size_t)t.exp_len);
+        }
+    }
     for (int32_t i = 0; i < n; ++i) {
         TensorLayout& t = L->t[i];
         if (t.kind == K_FP32) {
@@ -358,7 +405,7 @@ void compute_layout(const lpmm_config& cfg, const lpmm_shape* shapes, int32_t n,
             t.fact_tiles_y = (int32_t)((t.rows + p.tile_rows1 - 1) / p.tile_rows1);
             t.fact_rowpart = off; off = region_end(L, off + sizeof(float) * (size_t)t.rows * t.fact_nstrips);
             t.fact_colpart = off; off = region_end(L, off + sizeof(float) * (size_t)t.fact_tiles_y * t.cols);
-            t.fact_blockpart = off; off = region_end(L, off + sizeof(double) * (size_t)((t.c_off + (t.cols + 3) / 4 * 4 + 31) / 32));
+            t.fact_blockpart = off; off = region_end(L, off + sizeof(double) * (size_t)((t.rc_len + 31) / 32));
         }
     }
     L->states_end = off;   // everything a checkpoint must keep lies below this offset
@@ -399,6 +446,8 @@ struct lpmm_state {
     uint32_t epoch = 0;                    // fused launches made on this state (the per-tensor counters count along)
     int32_t sms, occ1, occ2;
     int32_t p1_ctas;                       // which instantiation of the maxima pass (2 or 3 CTAs per SM)
+    std::vector<int32_t> tiles7;           // prefix sums of the update tiles of the tensors that are not on the tiled path
+    std::vector<int32_t> tiles6;           // prefix sums of the composite tensors' 256-entry chunks of expanded statistics
     std::vector<int32_t> tiles5;           // prefix sums of the factorized tensors' 32-statistic chunks (finalize kernel)
     std::vector<int32_t> tiles1, tiles2, tiles3;   // host copies of the tile prefix sums (3: element-indexed tiles of every tensor)
     cudaStream_t aux = nullptr;            // overlapped schedule: the stream of the maxima passes (lazily created)
@@ -505,7 +554,7 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
 
     std::vector<TensorDesc> descs(n);
     std::vector<TilePlan> plans(n);
-    std::vector<int32_t> t1(n + 1, 0), t2(n + 1, 0), t3(n + 1, 0), t4(n + 1, 0), t5(n + 1, 0);
+    std::vector<int32_t> t1(n + 1, 0), t2(n + 1, 0), t3(n + 1, 0), t4(n + 1, 0), t5(n + 1, 0), t6(n + 1, 0), t7(n + 1, 0);
     // In a state whose matrices are not block-wise, folded 1-D tensors leave the main update launch (0 tiles there)
     // and get one of their own with the block-wise kernel (table 4).
     const bool own_launch = st->cfg.v_mode != LPMM_V_BLOCK;
@@ -519,6 +568,7 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
         for (int a = 0; a < 3; ++a) { d.outer_dim[a] = t.outer_dim[a]; d.outer_off[a] = t.outer_off[a]; }
         d.m_shift = (st->cfg.m_block == 2048) ? 11 : 7;
         d.dbg_status = reinterpret_cast<uint32_t*>(A);
+        d.p1_tiled = t.p1_tiled ? 1 : 0;
         if (t.kind == K_FP32) {
             d.m32 = reinterpret_cast<float*>(A + t.m32);
             d.v32 = reinterpret_cast<float*>(A + t.v32);
@@ -532,7 +582,15 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
                 d.rc[1] = reinterpret_cast<float*>(A + st->L.rc[1]) + t.rc_index;
                 d.rc[2] = reinterpret_cast<float*>(A + st->L.rc[2]) + t.rc_index;
                 d.rcp_new = reinterpret_cast<float*>(A + st->L.rcp) + t.rc_index;
-                d.rc_floats = (int32_t)(t.c_off + (t.cols + 3) / 4 * 4);
+                d.rc_floats = t.rc_len;
+            }
+            if (t.nd_split > 0) {
+                d.exp_old = reinterpret_cast<float*>(A + t.exp_old);
+                d.exp_new = reinterpret_cast<float*>(A + t.exp_new);
+                d.rcp_new = reinterpret_cast<float*>(A + t.exp_rcp);
+                d.exp_len = t.exp_len;
+                d.nd = t.nd; d.nd_split = t.nd_split;
+                for (int a = 0; a < 4; ++a) { d.nd_dim[a] = t.nd_dim[a]; d.nd_off[a] = t.nd_off[a]; }
             }
             if (t.kind == K_FACT) {
                 d.fact_rowpart = reinterpret_cast<float*>(A + t.fact_rowpart);
@@ -553,11 +611,14 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
         t3[i + 1] = t3[i] + (int32_t)p.tiles_flat;
         if (t2[i] + p.tiles_update > 0x7fffffffLL) return LPMM_ERR_UNSUPPORTED;
         const bool moved = own_launch && t.kind == K_BLOCK_TILED;
-        t2[i + 1] = t2[i] + (moved ? 0 : (int32_t)p.tiles_update);
+        const bool on_tiled_path = t.kind == K_RANK1_FAST || t.kind == K_FACT || t.kind == K_BLOCK_TILED;
+        t2[i + 1] = t2[i] + ((moved || !on_tiled_path) ? 0 : (int32_t)p.tiles_update);
+        t7[i + 1] = t7[i] + (on_tiled_path ? 0 : (int32_t)p.tiles_update);
         t4[i + 1] = t4[i] + (moved ? (int32_t)p.tiles_update : 0);
         if (t1[i] + p.tiles_maxima > 0x7fffffffLL) return LPMM_ERR_UNSUPPORTED;
         t1[i + 1] = t1[i] + (int32_t)p.tiles_maxima;
         t5[i + 1] = t5[i] + (t.kind == K_FACT ? (d.rc_floats + 31) / 32 : 0);
+        t6[i + 1] = t6[i] + (t.nd_split > 0 ? (t.exp_len + 255) / 256 : 0);
         if (t.kind == K_FACT && (int64_t)d.tile_rows1 * d.fact_tiles_y < t.rows) return LPMM_ERR_UNSUPPORTED;   // (layout and plan disagree)
     }
     st->total1 = t1[n];
@@ -570,6 +631,10 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
     st->tiles3 = t3;
     st->tiles4 = t4;
     st->tiles5 = t5;
+    st->tiles6 = t6;
+    st->tiles7 = t7;
+    LPMM_CUDA(cudaMemcpyAsync(A + st->L.tiles7, t7.data(), sizeof(int32_t) * (n + 1), cudaMemcpyHostToDevice, s));
+    LPMM_CUDA(cudaMemcpyAsync(A + st->L.tiles6, t6.data(), sizeof(int32_t) * (n + 1), cudaMemcpyHostToDevice, s));
     LPMM_CUDA(cudaMemcpyAsync(A + st->L.tiles5, t5.data(), sizeof(int32_t) * (n + 1), cudaMemcpyHostToDevice, s));
     {   // overlapped schedule: consecutive groups of about equal size, each with at least one maxima tile
         int32_t groups = st->cfg.overlap_groups > 0 ? st->cfg.overlap_groups : 8;
@@ -815,11 +880,20 @@ lpmm_status enqueue_maxima(lpmm_state* st, StepArgs a, int32_t t0, int32_t t1, b
         const TensorLayout& t = st->L.t[i];
         if (!uses_rc(t.kind)) continue;
         if (rc_begin < 0) rc_begin = t.rc_index;
-        rc_end = (t.rc_index + t.c_off + (t.cols + 3) / 4 * 4 + 63) / 64 * 64;
+        rc_end = (t.rc_index + t.rc_len + 63) / 64 * 64;
     }
     float* rc_new = reinterpret_cast<float*>(st->arena + st->L.rc[(st->phase + 1) % 3]) + rc_begin;
     const bool factored = st->cfg.v_mode == LPMM_V_FACTORED;    // (its sums are written, not accumulated: nothing to clear)
     if (!factored) LPMM_CUDA(cudaMemsetAsync(rc_new, 0, sizeof(float) * (size_t)(rc_end - rc_begin), s));
+    const bool composite = st->tiles6[t1] > st->tiles6[t0];
+    StepArgs nd_args = a;
+    if (composite) {   // expanded current statistics of the composite tensors; their expanded accumulators start at zero
+        nd_args.tile_start = reinterpret_cast<const int32_t*>(st->arena + st->L.tiles6);
+        nd_args.tile_begin = st->tiles6[t0];
+        nd_args.tile_end = st->tiles6[t1];
+        LPMM_CUDA(launch_nd_stats(nd_args, 0, s));
+        *launches += 1;
+    }
     if (ev) LPMM_CUDA(cudaEventRecord(ev[0], s));
     a.tile_start = reinterpret_cast<const int32_t*>(st->arena + st->L.tiles1);
     a.tile_begin = p1_begin;
@@ -836,6 +910,11 @@ lpmm_status enqueue_maxima(lpmm_state* st, StepArgs a, int32_t t0, int32_t t1, b
     } else {
         LPMM_CUDA(launch_rcp(rc_new, reinterpret_cast<float*>(st->arena + st->L.rcp) + rc_begin, rc_end - rc_begin, s));
         *launches += 2;
+        if (composite) {   // row / column maxima -> per-axis maxima (Alg. 4), then their expanded reciprocals
+            LPMM_CUDA(launch_nd_stats(nd_args, 1, s));
+            LPMM_CUDA(launch_nd_stats(nd_args, 2, s));
+            *launches += 2;
+        }
     }
     return LPMM_OK;
 }
@@ -852,6 +931,14 @@ lpmm_status enqueue_update(lpmm_state* st, StepArgs a, int32_t t0, int32_t t1, b
                            st->cfg.v_mode == LPMM_V_FACTORED ? 1 : (st->cfg.v_mode == LPMM_V_BLOCK ? 2 : 0),
                            tiles < cap ? tiles : cap, s));
     if (tiles > 0) *launches += 1;
+    if (st->tiles7[t1] > st->tiles7[t0]) {   // the tensors that are not on the tiled path: a kernel (and launch) of their own
+        a.tile_start = reinterpret_cast<const int32_t*>(st->arena + st->L.tiles7);
+        a.tile_begin = st->tiles7[t0];
+        a.tile_end = st->tiles7[t1];
+        const int32_t tiles7 = a.tile_end - a.tile_begin;
+        LPMM_CUDA(launch_pass2(a, bf16, ieee_update, st->cfg.m_block == 2048 ? 11 : 7, 3, tiles7 < cap ? tiles7 : cap, s));
+        *launches += 1;
+    }
     if (st->tiles4[t1] > st->tiles4[t0]) {   // folded 1-D tensors of a state that is not block-wise
         a.tile_start = reinterpret_cast<const int32_t*>(st->arena + st->L.tiles4);
         a.tile_begin = st->tiles4[t0];
@@ -1173,7 +1260,7 @@ lpmm_status lpmm_state_view(const lpmm_state* st, int32_t tensor, int32_t* kind,
     if (v_codes) *v_codes = (q && t.kind != K_FACT) ? reinterpret_cast<const uint8_t*>(A + t.v_codes) : nullptr;
     const float* rc = reinterpret_cast<const float*>(A + st->L.rc[st->phase]) + t.rc_index;
     if (v_scale0) *v_scale0 = r1 ? rc : ((t.kind == K_BLOCK || t.kind == K_BLOCK_TILED) ? reinterpret_cast<const float*>(A + t.v_bscale) : nullptr);
-    if (v_scale1) *v_scale1 = r1 ? rc + t.c_off : nullptr;
+    if (v_scale1) *v_scale1 = r1 ? rc + (t.nd >= 3 ? t.nd_off[t.nd - 1] : t.c_off) : nullptr;
     if (m32) *m32 = q ? nullptr : reinterpret_cast<const float*>(A + t.m32);
     if (v32) *v32 = q ? nullptr : reinterpret_cast<const float*>(A + t.v32);
     return LPMM_OK;
@@ -1182,9 +1269,10 @@ lpmm_status lpmm_state_view(const lpmm_state* st, int32_t tensor, int32_t* kind,
 lpmm_status lpmm_state_view_axis(const lpmm_state* st, int32_t tensor, int32_t axis, const float** mu, int64_t* extent) {
     if (!st || tensor < 0 || tensor >= st->n || !mu || !extent) return LPMM_ERR_INVALID_ARG;
     const TensorLayout& t = st->L.t[tensor];
-    if (!uses_rc(t.kind) || axis < 0 || axis > t.n_outer) return LPMM_ERR_INVALID_ARG;
+    if (!uses_rc(t.kind) || axis < 0 || axis >= (t.nd >= 3 ? t.nd : 2)) return LPMM_ERR_INVALID_ARG;
     const float* rc = reinterpret_cast<const float*>(st->arena + st->L.rc[st->phase]) + t.rc_index;
-    if (axis < t.n_outer) { *mu = rc + t.outer_off[axis]; *extent = t.outer_dim[axis]; }
+    if (t.nd >= 3) { *mu = rc + t.nd_off[axis]; *extent = t.nd_dim[axis]; }
+    else if (axis == 0) { *mu = rc; *extent = t.rows; }
     else { *mu = rc + t.c_off; *extent = t.cols; }
     return LPMM_OK;
 }

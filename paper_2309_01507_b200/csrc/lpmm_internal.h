@@ -55,6 +55,19 @@ struct TensorDesc {
     int32_t fact_nstrips;
     int32_t fact_tiles_y;
     uint32_t* dbg_status;   // the arena's device status word (written by the checking build's index checks)
+    // K_RANK1_FAST for a tensor with three or four axes ("composite", Alg. 4): the leading nd_split axes are flattened
+    // into rows, the others into columns (rows, cols, c_off above describe that matrix). The persistent statistics stay one
+    // vector per axis (axis a at float nd_off[a] of rc[]); every step they are expanded into per-row / per-column vectors
+    // (minimum over the axes of a side) which the tiled kernels read and reduce into exactly like a matrix's r and c:
+    //   exp_old [rows padded to 4 | cols]   current scales, exp_new: maxima of this step, rcp_new: their reciprocals.
+    float* exp_old;         // nullptr: not a composite tensor
+    float* exp_new;
+    int32_t exp_len;        // floats of each expanded vector
+    int32_t nd, nd_split;
+    int32_t p1_tiled;       // K_RANK1_FLAT matrix with cols % 8 == 0: its maxima pass runs on the tiled kernel (ragged last
+                            // column group clamped onto valid columns: maxima are idempotent)
+    int32_t nd_dim[4];
+    int32_t nd_off[4];
 };
 
 // Index checks of the checking build (-DLPMM_DEBUG): a failed check records its code in the device status word (the
@@ -124,6 +137,9 @@ cudaError_t launch_fused_f32_ieee(const StepArgs& a, int grid, cudaStream_t s);
 cudaError_t launch_wait_selftest(const uint32_t* flag, uint32_t want, uint32_t limit, uint32_t* dev_status, int32_t* gave_up,
                                  cudaStream_t s);
 cudaError_t launch_check_selftest(uint32_t* dev_status, cudaStream_t s);
+// mode 0: expand the current per-axis statistics and clear exp_new; 1: fold exp_new into the new per-axis statistics
+// (atomic maxima into the cleared buffer); 2: expanded reciprocals of the new statistics. a.tile_*: the chunk table.
+cudaError_t launch_nd_stats(const StepArgs& a, int mode, cudaStream_t s);
 cudaError_t launch_guard_check(const unsigned char* zone, int bytes, unsigned char want, uint32_t* damaged, cudaStream_t s);
 cudaError_t launch_factor_finalize(const StepArgs& a, cudaStream_t s);
 cudaError_t launch_sgdm(const StepArgs& a, bool bf16, int grid, cudaStream_t s);

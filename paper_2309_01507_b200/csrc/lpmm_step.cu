@@ -37,6 +37,10 @@ __device__ __forceinline__ int find_tensor(const int32_t* __restrict__ start, in
 // One of the three rank-1 scale buffers of a tensor (selected without indexing the by-value descriptor dynamically).
 __device__ __forceinline__ float* rc_pick(const TensorDesc& d, int i) { return i == 0 ? d.rc[0] : (i == 1 ? d.rc[1] : d.rc[2]); }
 
+// The row / column scale vectors a tiled kernel works with: a matrix's own r, c, or a composite tensor's expanded ones.
+__device__ __forceinline__ float* stats_old(const TensorDesc& d, RcSel sel) { return d.exp_old ? d.exp_old : rc_pick(d, sel.old_i); }
+__device__ __forceinline__ float* stats_new(const TensorDesc& d, RcSel sel) { return d.exp_old ? d.exp_new : rc_pick(d, sel.new_i); }
+
 // ---- tile hand-out --------------------------------------------------------------------------------
 //
 // The CTAs of a launch take tiles from a counter in the arena header in the order they become free, so an SM
@@ -539,7 +543,7 @@ __device__ __forceinline__ void pass2_rank1_fast(const TensorDesc& d, float* __r
     // cols % 128 == 0: a whole 16-lane group (one block) is in or out together. With B2048 the tile is one
     // block wide (wx = 8, cols % 2048 == 0), every warp is inside and all of them run the same rows.
     if (col0 >= d.cols) return;
-    const float* rc_old = rc_pick(d, sel.old_i);
+    const float* rc_old = stats_old(d, sel);
     const float* rcp_new = d.rcp_new;
     const int64_t row0 = (int64_t)ty * d.tile_rows + warp / wx;
     const int64_t row_end = min((int64_t)(ty + 1) * d.tile_rows, d.rows);
@@ -675,6 +679,96 @@ __device__ __forceinline__ void outer_publish(const TensorDesc& d, float* base, 
 
 // ---- pass 2, flat (element-indexed) tensors: block-wise v, or rank-1 with arbitrary cols ------
 
+// Interior tiles of a matrix whose rows hold a whole number of lanes (cols % 8 == 0, cols >= 2048) but not of
+// first-moment blocks: the flat 128-aligned walk of pass2_flat() with everything that walk recomputes per chunk taken
+// out of the loop. 32-bit offsets from the tile's first element; the (row, column) of a lane's elements is divided out
+// once per tile and then stepped (a chunk step of 2048 elements wraps a row at most once); the streaming operands of
+// the next chunk are loaded before the current one is processed (two alternating register sets), the row and column
+// statistics - which come from L1 - when they are needed.
+template <bool BF16>
+struct FlatRegs {
+    float4 w0, w1;
+    uint4 g0, g1;          // bf16: g0 only
+    uint32_t qm, qv;
+    float am;
+};
+template <bool BF16, bool A32>
+__device__ __forceinline__ void flat_load(FlatRegs<BF16>& r, const float* w, const void* g, const uint8_t* mq, const uint8_t* vq,
+                                          const float* ms, uint32_t off) {
+    if (A32) {
+        load8_f32_256(w + off, r.w0, r.w1);
+    } else {
+        r.w0 = *reinterpret_cast<const float4*>(w + off);
+        r.w1 = *reinterpret_cast<const float4*>(w + off + 4);
+    }
+    if (BF16) {
+        r.g0 = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(g) + off));
+    } else if (A32) {
+        load8_u32_256_nc(reinterpret_cast<const float*>(g) + off, r.g0, r.g1);
+    } else {
+        r.g0 = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(g) + off));
+        r.g1 = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(g) + off + 4));
+    }
+    r.qm = *reinterpret_cast<const uint32_t*>(mq + (off >> 1));
+    r.qv = *reinterpret_cast<const uint32_t*>(vq + (off >> 1));
+    r.am = ms[off >> 7];
+}
+template <bool BF16, bool EXACT, bool WB, bool A32, bool FU>
+__device__ __forceinline__ void pass2_flat_interior(const TensorDesc& d, float* __restrict__ w, uint16_t* __restrict__ w16,
+                                                    const void* __restrict__ g, int tile, RcSel sel, const Hyper& h,
+                                                    const Hyper2& h2, const LaneTables& lt, const unsigned char* s_lut) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t base = (int64_t)tile * d.flat_chunks * (kWarps * kWarpElems);
+    const float* rc_old = rc_pick(d, sel.old_i);
+    const float* rcp_new = d.rcp_new;
+    float* wb = w + base;
+    uint16_t* w16b = WB ? w16 + base : nullptr;
+    const void* gb = BF16 ? static_cast<const void*>(reinterpret_cast<const uint16_t*>(g) + base)
+                          : static_cast<const void*>(reinterpret_cast<const float*>(g) + base);
+    uint8_t* mq = d.m_codes + (base >> 1);
+    uint8_t* vq = d.v_codes + (base >> 1);
+    float* ms = d.m_scale + (base >> 7);
+    uint32_t off = (uint32_t)(warp * kWarpElems + lane * kLaneElems);
+    int64_t i64, j64;
+    split_index(d, base + off, i64, j64);
+    uint32_t i = (uint32_t)i64, j = (uint32_t)j64;
+    const uint32_t cols = (uint32_t)d.cols;
+    constexpr uint32_t kStep = kWarps * kWarpElems;
+    FlatRegs<BF16> ra, rb;
+    flat_load<BF16, A32>(ra, wb, gb, mq, vq, ms, off);
+    const int n = d.flat_chunks;
+    for (int c = 0; c < n; ++c) {
+        FlatRegs<BF16>& cur = (c & 1) ? rb : ra;
+        FlatRegs<BF16>& nxt = (c & 1) ? ra : rb;
+        if (c + 1 < n) flat_load<BF16, A32>(nxt, wb, gb, mq, vq, ms, off + kStep);
+        float wv[8] = {cur.w0.x, cur.w0.y, cur.w0.z, cur.w0.w, cur.w1.x, cur.w1.y, cur.w1.z, cur.w1.w};
+        float gv[8], mt[8], vt[8], vs[8], vr[8], co[8], cr[8];
+        unpack_grad8<BF16>(cur.g0, cur.g1, gv);
+        const float so = __ldg(rc_old + i);
+        const float ro = FU ? __ldcg(rcp_new + i) : __ldg(rcp_new + i);
+        load8_f32(rc_old + d.c_off + j, co);
+        if (FU) load8_f32_cg(rcp_new + d.c_off + j, cr);
+        else load8_f32(rcp_new + d.c_off + j, cr);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            vs[k] = fminf(so, co[k]);
+            vr[k] = fmaxf(ro, cr[k]);
+        }
+        moments_and_update8<EXACT>(wv, gv, cur.qm, cur.qv, __fmul_rn(lt.de, cur.am), vs, h, h2, lt, mt, vt);
+        store8_f32_a<A32>(wb + off, wv);
+        if (WB) store8_bf16(w16b + off, wv);
+        const float am_new = group_max(absmax8(mt), lt.mask);
+        if ((lane & 15) == 0) ms[off >> 7] = am_new;
+        *reinterpret_cast<uint32_t*>(mq + (off >> 1)) = quantize8_de(mt, scale_rcp(am_new), s_lut);
+        *reinterpret_cast<uint32_t*>(vq + (off >> 1)) = quantize8_lin(vt, vr, h2);
+        off += kStep;
+        j += kStep;
+        if (j >= cols) { j -= cols; ++i; }
+    }
+}
+
+// (FU: called from the fused kernel, which reads the new reciprocals past L1 and, to keep its register allocation,
+// does without the interior loop.)
 template <bool BF16, bool RANK1, bool EXACT, int MSHIFT, bool WB = false, bool A32 = false, bool FU = false>
 __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restrict__ w, uint16_t* __restrict__ w16,
                                            const void* __restrict__ g,
@@ -686,6 +780,11 @@ __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restric
     const int64_t m_mask = ((int64_t)1 << MSHIFT) - 1;
     // checking build: the tile starts inside the tensor (B2048: recorded only, the CTA-wide barrier needs every warp)
     if (!LPMM_DBG_OK(d, tile >= 0 && (int64_t)tile * d.flat_chunks * kWarps * kWarpElems < d.numel, 3) && MSHIFT == 7) return;
+    if (!FU && RANK1 && MSHIFT == 7 && d.n_outer == 1 && (d.cols & 7) == 0 && d.cols >= kWarps * kWarpElems &&
+        (int64_t)(tile + 1) * d.flat_chunks * (kWarps * kWarpElems) <= d.numel) {   // uniform over the CTA
+        pass2_flat_interior<BF16, EXACT, WB, A32, FU>(d, w, w16, g, tile, sel, h, h2, lt, s_lut);
+        return;
+    }
     for (int c = 0; c < d.flat_chunks; ++c) {
         const int64_t chunk0 = ((int64_t)tile * d.flat_chunks + c) * kWarps;   // the CTA's 8 chunks = 2048 elements
         const int64_t chunk = chunk0 + warp;
@@ -695,6 +794,20 @@ __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restric
         // (with zeros; its loads and stores are all guarded away).
         if (MSHIFT == 7 && chunk * kWarpElems >= d.numel) break;
         const bool full = (chunk + 1) * kWarpElems <= d.numel;
+        if (c + 2 < d.flat_chunks) {
+            // L2 hint for the warp's chunk after next (one line per lane: 8 of parameters, 4 or 8 of gradient, one of
+            // each code array), so that its loads find their data in L2
+            const int64_t en = (chunk + 2 * kWarps) * kWarpElems;
+            if (en + kWarpElems <= d.numel) {
+                constexpr int kG = BF16 ? 4 : 8;
+                const char* p = nullptr;
+                if (lane < 8) p = reinterpret_cast<const char*>(w + en) + lane * 128;
+                else if (lane < 8 + kG) p = reinterpret_cast<const char*>(g) + en * (BF16 ? 2 : 4) + (lane - 8) * 128;
+                else if (lane == 8 + kG) p = reinterpret_cast<const char*>(d.m_codes) + (en >> 1);
+                else if (lane == 9 + kG) p = reinterpret_cast<const char*>(d.v_codes) + (en >> 1);
+                if (p) prefetch_l2(p);
+            }
+        }
         float wv[8], gv[8], mt[8], vt[8], vs[8], vr[8];
         uint32_t qm, qv;
         if (full) {
@@ -825,7 +938,11 @@ __device__ __forceinline__ void pass2_fp32(const TensorDesc& d, float* __restric
 // WB: a bfloat16 copy of every updated parameter is written as well (a.params_bf16).
 // A32: every parameter pointer (and, with fp32 gradients, every gradient pointer) of the step is 32-byte aligned,
 // checked on the host: the tiled path then moves a lane's 8 values with one 256-bit access.
-template <bool BF16, bool EXACT, int MSHIFT, int VF, bool WB, bool A32>
+// MISC: false = the tensors on the tiled path; true = all the others (element-indexed: odd shapes, ragged 1-D tensors;
+// fp32 states of small tensors). They are two kernels (two launches per step) so that the register allocation of the
+// tiled path - where nearly all parameters of a real model are - is not shared with paths it never runs: with both in
+// one kernel the update pass of the LLaMA-7B list took 13.9-14.0 ms instead of 13.3-13.4.
+template <bool BF16, bool EXACT, int MSHIFT, int VF, bool WB, bool A32, bool MISC = false>
 __global__ void __launch_bounds__(kThreads, 2) pass2_kernel(StepArgs a) {
     __shared__ __align__(16) unsigned char s_lut[kLutSmemBytes];
     __shared__ float s_red[2 * kWarps];
@@ -844,20 +961,27 @@ __global__ void __launch_bounds__(kThreads, 2) pass2_kernel(StepArgs a) {
         uint16_t* w16 = WB ? a.params_bf16[t] : nullptr;
         const void* g = a.grads[t];
         const int local = tile - __ldg(a.tile_start + t);
-        switch (d.kind) {
-            case K_RANK1_FAST:
-                if (VF == 0) pass2_rank1_fast<BF16, EXACT, MSHIFT, 0, WB, A32>(d, w, w16, g, local, a.sel, a.h, h2, lt, s_lut, s_red, red_step);
-                break;
-            case K_FACT:
-                if (VF == 1) pass2_rank1_fast<BF16, EXACT, MSHIFT, 1, WB>(d, w, w16, g, local, a.sel, a.h, h2, lt, s_lut, s_red, red_step);
-                break;
-            case K_BLOCK_TILED:   // matrices of a block-wise state; long 1-D tensors folded into rows (in states of another
-                                  // kind these get a launch of their own, so that the default kernels stay lean)
-                if (VF == 2) pass2_rank1_fast<BF16, EXACT, MSHIFT, 2, WB, A32>(d, w, w16, g, local, a.sel, a.h, h2, lt, s_lut, s_red, red_step);
-                break;
-            case K_RANK1_FLAT: pass2_flat<BF16, true, EXACT, MSHIFT, WB, A32>(d, w, w16, g, local, a.sel, a.h, h2, lt, s_lut, s_red, red_step); break;
-            case K_BLOCK:      pass2_flat<BF16, false, EXACT, MSHIFT, WB, A32>(d, w, w16, g, local, a.sel, a.h, h2, lt, s_lut, s_red, red_step); break;
-            default:           pass2_fp32<BF16, EXACT, WB, A32>(d, w, w16, g, local, a.h); break;
+        if (MISC) {
+            switch (d.kind) {
+                case K_RANK1_FLAT: pass2_flat<BF16, true, EXACT, MSHIFT, WB, A32>(d, w, w16, g, local, a.sel, a.h, h2, lt, s_lut, s_red, red_step); break;
+                case K_BLOCK:      pass2_flat<BF16, false, EXACT, MSHIFT, WB, A32>(d, w, w16, g, local, a.sel, a.h, h2, lt, s_lut, s_red, red_step); break;
+                case K_FP32:       pass2_fp32<BF16, EXACT, WB, A32>(d, w, w16, g, local, a.h); break;
+                default: break;
+            }
+        } else {
+            switch (d.kind) {
+                case K_RANK1_FAST:
+                    if (VF == 0) pass2_rank1_fast<BF16, EXACT, MSHIFT, 0, WB, A32>(d, w, w16, g, local, a.sel, a.h, h2, lt, s_lut, s_red, red_step);
+                    break;
+                case K_FACT:
+                    if (VF == 1) pass2_rank1_fast<BF16, EXACT, MSHIFT, 1, WB>(d, w, w16, g, local, a.sel, a.h, h2, lt, s_lut, s_red, red_step);
+                    break;
+                case K_BLOCK_TILED:   // matrices of a block-wise state; long 1-D tensors folded into rows (in states of another
+                                      // kind these get a launch of their own, so that the default kernels stay lean)
+                    if (VF == 2) pass2_rank1_fast<BF16, EXACT, MSHIFT, 2, WB, A32>(d, w, w16, g, local, a.sel, a.h, h2, lt, s_lut, s_red, red_step);
+                    break;
+                default: break;
+            }
         }
         tile = a.tile_begin + tiles_next(s_next, buf, fetched);
     }
@@ -1020,10 +1144,10 @@ __device__ __forceinline__ void pass1_rank1_fast(const TensorDesc& d, const void
     const int tx = tile % d.tiles_x, ty = tile / d.tiles_x;
     const int64_t col_w = (int64_t)tx * (kWarpElems * wx) + (warp % wx) * kWarpElems;   // first column of this warp
     int64_t col0 = col_w + lane * kLaneElems;
-    // Maxima are idempotent: when cols % 256 == 128 the upper half-warp repeats the lower one's columns.
-    if (col0 >= d.cols) col0 -= 128;
-    const float* rc_old = rc_pick(d, sel.old_i);
-    float* rc_new = rc_pick(d, sel.new_i);
+    // Maxima are idempotent: lanes beyond the last column (cols % 256 != 0) repeat its last eight columns.
+    if (col0 >= d.cols) col0 = d.cols - kLaneElems;
+    const float* rc_old = stats_old(d, sel);
+    float* rc_new = stats_new(d, sel);
     const int64_t row0 = (int64_t)ty * d.tile_rows1 + warp / wx;
     const int64_t row_end = min((int64_t)(ty + 1) * d.tile_rows1, d.rows);
     if (row0 >= row_end) return;                      // uniform over the warp
@@ -1324,7 +1448,7 @@ __global__ void __launch_bounds__(kThreads, MINB) pass1_kernel(StepArgs a) {
         const TensorDesc d = a.descs[t];
         const void* g = a.grads[t];
         const int local = tile - __ldg(a.tile_start + t);
-        if (d.kind == K_RANK1_FAST) pass1_rank1_fast<BF16>(d, g, local, a.sel, h2, lt, s_col);
+        if (d.kind == K_RANK1_FAST || d.p1_tiled) pass1_rank1_fast<BF16>(d, g, local, a.sel, h2, lt, s_col);
         else if (d.kind == K_FACT) pass1_fact<BF16>(d, g, local, s_col);
         else pass1_rank1_flat<BF16>(d, g, local, a.sel, a.h);
         tile = a.tile_begin + tiles_next(s_next, buf, fetched);
@@ -1412,9 +1536,13 @@ __global__ void __launch_bounds__(kThreads, 2) step_fused_kernel(StepArgs a) {
                 const int z0 = (int)((int64_t)n4 * local / d.tiles1), z1 = (int)((int64_t)n4 * (local + 1) / d.tiles1);
                 for (int i = z0 + (int)threadIdx.x; i < z1; i += kThreads) z[i] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
             }
-            if (d.kind == K_RANK1_FAST) {
+            if (d.kind == K_RANK1_FAST || d.p1_tiled) {
                 const L2Policies pol = make_l2_policies();
                 pass1_rank1_fast<BF16, true>(d, g, local, a.sel, h2, lt, s_col, (keep && a.l2_hints) ? pol.last : pol.normal, keep && a.l2_hints);
+            } else {
+                pass1_rank1_flat<BF16>(d, g, local, a.sel, a.h);
+            }
+            if (d.kind == K_RANK1_FAST) {
                 // Count the tile. The barrier orders every thread's atomic maxima before thread 0's fence, which is
                 // cumulative; nobody waits for the counter's old value.
                 __syncthreads();
@@ -1426,7 +1554,6 @@ __global__ void __launch_bounds__(kThreads, 2) step_fused_kernel(StepArgs a) {
                 // Element-indexed tensors (odd shapes, three or four axes): their update path reads the reciprocals of
                 // the new statistics from memory, so the CTA that finishes the tensor's last maxima tile inverts them
                 // and only then announces the tensor (`ready` takes the launch number).
-                pass1_rank1_flat<BF16>(d, g, local, a.sel, a.h);
                 __syncthreads();
                 if (threadIdx.x == 0) {
                     __threadfence();
@@ -1625,7 +1752,15 @@ cudaError_t launch_pass1(const StepArgs& a, bool bf16, int ctas_per_sm, int grid
 
 template <bool BF16, bool EXACT, int MSHIFT>
 cudaError_t launch_pass2_t(const StepArgs& a, int v_kind, int grid, cudaStream_t s) {
-    if (v_kind == 1) {
+    if (v_kind == 3) {   // the tensors that are not on the tiled path
+        if (a.params_bf16 != nullptr) {
+            if (a.aligned32) pass2_kernel<BF16, EXACT, MSHIFT, 0, true, true, true><<<grid, kThreads, 0, s>>>(a);
+            else pass2_kernel<BF16, EXACT, MSHIFT, 0, true, false, true><<<grid, kThreads, 0, s>>>(a);
+        } else {
+            if (a.aligned32) pass2_kernel<BF16, EXACT, MSHIFT, 0, false, true, true><<<grid, kThreads, 0, s>>>(a);
+            else pass2_kernel<BF16, EXACT, MSHIFT, 0, false, false, true><<<grid, kThreads, 0, s>>>(a);
+        }
+    } else if (v_kind == 1) {
         pass2_kernel<BF16, EXACT, MSHIFT, 1, false, false><<<grid, kThreads, 0, s>>>(a);
     } else if (v_kind == 2) {
         if (a.params_bf16 != nullptr) {
@@ -1677,7 +1812,8 @@ cudaError_t launch_fused_f32_ieee(const StepArgs& a, int grid, cudaStream_t s) {
 #endif
 
 #if LPMM_STEP_PART == 0
-// v_kind: 0 rank-1 second moments, 1 factorized, 2 block-wise (which tiled path the state's matrices take).
+// v_kind: 0 rank-1 second moments, 1 factorized, 2 block-wise (which tiled path the state's matrices take);
+// 3: the kernel of the tensors that are not on the tiled path.
 cudaError_t launch_pass2(const StepArgs& a, bool bf16, bool exact, int m_shift, int v_kind, int grid, cudaStream_t s) {
     if (a.tile_end <= a.tile_begin) return cudaSuccess;
     if (bf16) return exact ? launch_pass2_bf16_ieee(a, m_shift, v_kind, grid, s) : launch_pass2_bf16_fast(a, m_shift, v_kind, grid, s);
@@ -1689,6 +1825,61 @@ cudaError_t launch_fused(const StepArgs& a, bool bf16, bool exact, int grid, cud
     if (a.tile_end <= a.tile_begin) return cudaSuccess;
     if (bf16) return exact ? launch_fused_bf16_ieee(a, grid, s) : launch_fused_bf16_fast(a, grid, s);
     return exact ? launch_fused_f32_ieee(a, grid, s) : launch_fused_f32_fast(a, grid, s);
+}
+
+// ---- composite tensors (three or four axes on the tiled path): expanded statistics -------------------------
+//
+// One thread per entry of a composite tensor's expanded vector [rows padded to 4 | cols]; one CTA per 256 entries.
+// The side's axes are walked from the last (fastest) to the first; `digit` is the entry's index along the axis.
+template <typename F>
+__device__ __forceinline__ void nd_for_axes(const TensorDesc& d, int a0, int a1, uint32_t idx, F f) {
+    uint32_t rem = idx;
+#pragma unroll
+    for (int a = 3; a >= 0; --a) {
+        if (a >= a0 && a < a1) {
+            const uint32_t q = rem / (uint32_t)d.nd_dim[a];
+            f(d.nd_off[a] + (int)(rem - q * (uint32_t)d.nd_dim[a]));
+            rem = q;
+        }
+    }
+}
+__global__ void __launch_bounds__(256) nd_stats_kernel(StepArgs a, int mode) {
+    const int chunk_g = a.tile_begin + blockIdx.x;
+    const int t = find_tensor(a.tile_start, a.n_tensors, chunk_g);
+    const TensorDesc d = a.descs[t];
+    const int e = (chunk_g - __ldg(a.tile_start + t)) * 256 + (int)threadIdx.x;
+    if (e >= d.exp_len) return;
+    const bool is_row = e < d.rows, is_col = e >= d.c_off && e < d.c_off + d.cols;
+    const int a0 = is_row ? 0 : d.nd_split, a1 = is_row ? d.nd_split : d.nd;
+    const uint32_t idx = (uint32_t)(is_row ? e : e - d.c_off);
+    if (mode == 0) {
+        float s = 0.0f;
+        if (is_row || is_col) {
+            const float* old = rc_pick(d, a.sel.old_i);
+            s = 3.402823466e38f;
+            nd_for_axes(d, a0, a1, idx, [&](int off) { s = fminf(s, old[off]); });
+        }
+        d.exp_old[e] = s;
+        d.exp_new[e] = 0.0f;
+    } else if (mode == 1) {
+        if (is_row || is_col) {
+            const float v = d.exp_new[e];
+            float* cur = rc_pick(d, a.sel.new_i);
+            nd_for_axes(d, a0, a1, idx, [&](int off) { atomic_max_nonneg_filtered(cur + off, v); });
+        }
+    } else {
+        float r = 0.0f;
+        if (is_row || is_col) {
+            const float* cur = rc_pick(d, a.sel.new_i);
+            nd_for_axes(d, a0, a1, idx, [&](int off) { r = fmaxf(r, scale_rcp(cur[off])); });
+        }
+        d.rcp_new[e] = r;
+    }
+}
+cudaError_t launch_nd_stats(const StepArgs& a, int mode, cudaStream_t s) {
+    if (a.tile_end <= a.tile_begin) return cudaSuccess;
+    nd_stats_kernel<<<a.tile_end - a.tile_begin, 256, 0, s>>>(a, mode);
+    return cudaGetLastError();
 }
 
 // Checking build: counts the bytes of one guard zone that no longer hold the pattern.

@@ -198,7 +198,7 @@ def test_single_matrix_config_ten_steps(update_math, schedule):
         seen_m |= set(np.unique(oracle.unpack4(pair.ostate[0].m_codes, 1024 * 4096)).tolist())
         seen_v |= set(np.unique(oracle.unpack4(pair.ostate[0].v_codes, 1024 * 4096)).tolist())
     assert seen_m == set(range(16)) and seen_v == set(range(16))
-    assert pair.state.last_launches == _launches(schedule, 3)
+    assert pair.state.last_launches == _launches(schedule, 4)     # two-pass: maxima, reciprocals, tiled update, the bias' own update kernel
 
 
 @pytest.mark.parametrize("grad_dtype,update_math", [(torch.float32, lpmm.UPDATE_FAST), (torch.bfloat16, lpmm.UPDATE_FAST),
@@ -242,7 +242,7 @@ def test_block_mode_for_matrices(m_block, grad_dtype):
     for t in range(1, 4):
         pair.step(t, pair.grads_for(t, outlier_p=0.0 if t == 2 else 1e-3))
         pair.compare(tol=1e-6)
-    assert pair.state.last_launches == 1
+    assert pair.state.last_launches == 2     # no maxima pass at all: the tiled update kernel and the element-indexed one
 
 
 @pytest.mark.parametrize("grad_dtype", [torch.float32, torch.bfloat16])
@@ -268,8 +268,9 @@ def test_transformer_base_three_steps_one_launch_per_pass(schedule):
     for t in range(1, 4):
         pair.step(t, pair.grads_for(t))
         pair.compare(tol=1e-6)
-    # two-pass: maxima + reciprocal + update cover all 181 tensors; overlapped: the same three per group of tensors
-    assert pair.state.last_launches == {lpmm.SCHEDULE_TWO_PASS: 3, lpmm.SCHEDULE_FUSED: 1, lpmm.SCHEDULE_OVERLAP: 9}[schedule]
+    # two-pass: maxima + reciprocals + tiled update + the update kernel of the small fp32 tensors cover all 181 tensors;
+    # overlapped: the same four per group of tensors
+    assert pair.state.last_launches == {lpmm.SCHEDULE_TWO_PASS: 4, lpmm.SCHEDULE_FUSED: 1, lpmm.SCHEDULE_OVERLAP: 12}[schedule]
 
 
 @SCHEDULES
@@ -489,7 +490,7 @@ def test_factorized_second_moment_matches_oracle(grad_dtype, m_block):
             err = np.max(np.abs(w - w_ref[i]) / scale)
             assert err <= tol, (s.name, t, err)
             w_ref[i][:] = w
-    assert state.last_launches == 3      # sums pass, finalize kernel, update pass
+    assert state.last_launches == 4      # sums pass, finalize kernel, tiled update, element-indexed / fp32 update
     # a matrix whose rows do not hold whole first-moment blocks is refused in this mode
     with pytest.raises(lpmm.LpmmError) as ei:
         lpmm.state_init(cfg, [_mat(257, 129)])
@@ -544,7 +545,11 @@ def test_tensors_with_three_and_four_axes_match_oracle(grad_dtype, update_math, 
     # Codes, block scales and every axis' statistics bit-exact; parameters bit-exact with IEEE update math,
     # within 1e-6 * max(|w|, lr) with the approximate one. A matrix rides along to cover mixed lists.
     cfg = lpmm.default_config(update_math=update_math, schedule=schedule)
-    specs = [_nd(6, 10, 200), _nd(3, 5, 7, 64), _nd(16, 33, 9), _mat(96, 256), _nd(2, 4099, 3), _nd(1, 40, 128)]
+    # (under the two-pass schedule the tensors whose trailing axes multiply to whole 128-blocks - the last five - run on
+    # the tiled kernels as composite matrices with expanded statistics; the others, and all of them under the fused
+    # schedule, on the element-indexed ones)
+    specs = [_nd(6, 10, 200), _nd(3, 5, 7, 64), _nd(16, 33, 9), _mat(96, 256), _nd(2, 4099, 3), _nd(1, 40, 128),
+             _nd(4, 6, 256), _nd(3, 4, 8, 128), _nd(5, 3, 384), _nd(37, 128, 3, 3)]
     hyper = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
     params = [workloads.make_param(s, 14, i, device="cuda") for i, s in enumerate(specs)]
     state = lpmm.state_init(cfg, specs)
@@ -610,7 +615,9 @@ def test_bf16_copy_of_the_parameters(grad_dtype, m_block):
             want = oracle.f32_to_bf16_bits(pb[i].cpu().numpy().ravel())
             got = copies[i].view(torch.int16).cpu().numpy().view(np.uint16)
             assert np.array_equal(got, want), (s.name, t)
-    assert sb.last_launches == 4     # (the bfloat16 copy always runs the two-pass schedule)
+    # (the bfloat16 copy always runs the two-pass schedule: maxima, reciprocals, tiled update, element-indexed update, and
+    # the folded tensor's own update launch)
+    assert sb.last_launches == 5
     # refused with the factorized second moment, and with a missing pointer array
     sf = lpmm.state_init(lpmm.default_config(v_mode=lpmm.V_FACTORED), [_mat(96, 256)])
     with pytest.raises(lpmm.LpmmError) as ei:
@@ -669,5 +676,5 @@ def test_long_one_dimensional_tensors_folded_into_rows(grad_dtype, m_block, v_mo
         pair.compare(tol=1e-6)
     # two-pass: maxima + reciprocal + update (+ the folded tensors' own update launch); this small list of the default
     # quantizers runs the fused schedule: one launch + the folded tensors' own
-    want = {(128, lpmm.V_RANK1): 2, (2048, lpmm.V_RANK1): 4}.get((m_block, v_mode), 1)
+    want = {(128, lpmm.V_RANK1): 2, (2048, lpmm.V_RANK1): 4}.get((m_block, v_mode), 2)
     assert pair.state.last_launches == want
