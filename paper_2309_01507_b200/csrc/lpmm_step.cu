@@ -679,10 +679,10 @@ __device__ __forceinline__ void outer_publish(const TensorDesc& d, float* base, 
 
 // ---- pass 2, flat (element-indexed) tensors: block-wise v, or rank-1 with arbitrary cols ------
 
-// Interior tiles of a matrix whose rows hold a whole number of lanes (cols % 8 == 0, cols >= 2048) but not of
+// Interior tiles of a matrix whose rows hold a whole number of lanes (cols % 8 == 0, cols >= 256) but not of
 // first-moment blocks: the flat 128-aligned walk of pass2_flat() with everything that walk recomputes per chunk taken
 // out of the loop. 32-bit offsets from the tile's first element; the (row, column) of a lane's elements is divided out
-// once per tile and then stepped (a chunk step of 2048 elements wraps a row at most once); the streaming operands of
+// once per tile and then stepped (a chunk step of 2048 elements passes at most eight row ends); the streaming operands of
 // the next chunk are loaded before the current one is processed (two alternating register sets), the row and column
 // statistics - which come from L1 - when they are needed.
 template <bool BF16>
@@ -763,7 +763,7 @@ __device__ __forceinline__ void pass2_flat_interior(const TensorDesc& d, float* 
         *reinterpret_cast<uint32_t*>(vq + (off >> 1)) = quantize8_lin(vt, vr, h2);
         off += kStep;
         j += kStep;
-        if (j >= cols) { j -= cols; ++i; }
+        while (j >= cols) { j -= cols; ++i; }     // cols >= 256: at most eight rows per chunk step
     }
 }
 
@@ -780,7 +780,7 @@ __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restric
     const int64_t m_mask = ((int64_t)1 << MSHIFT) - 1;
     // checking build: the tile starts inside the tensor (B2048: recorded only, the CTA-wide barrier needs every warp)
     if (!LPMM_DBG_OK(d, tile >= 0 && (int64_t)tile * d.flat_chunks * kWarps * kWarpElems < d.numel, 3) && MSHIFT == 7) return;
-    if (!FU && RANK1 && MSHIFT == 7 && d.n_outer == 1 && (d.cols & 7) == 0 && d.cols >= kWarps * kWarpElems &&
+    if (!FU && RANK1 && MSHIFT == 7 && d.n_outer == 1 && (d.cols & 7) == 0 && d.cols >= kWarpElems &&
         (int64_t)(tile + 1) * d.flat_chunks * (kWarps * kWarpElems) <= d.numel) {   // uniform over the CTA
         pass2_flat_interior<BF16, EXACT, WB, A32, FU>(d, w, w16, g, tile, sel, h, h2, lt, s_lut);
         return;

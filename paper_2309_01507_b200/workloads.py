@@ -143,6 +143,17 @@ def square_8192() -> Workload:
     return Workload("square_8192", 4, (_mat("weight", 8192, 8192),), lr=1e-3, steps=10)
 
 
+def odd_shape(*dims) -> Workload:
+    """One tensor of an awkward shape (rows that are not whole 128-blocks, or three / four axes such as a convolution
+    weight), bf16 gradients: for timing the paths beside the tiled one."""
+    rows = 1
+    for d in dims[:-1]:
+        rows *= d
+    name = "x".join(str(d) for d in dims)
+    spec = TensorSpec(name, rows, dims[-1], len(dims), dims=tuple(dims) if len(dims) >= 3 else None)
+    return Workload("odd_" + name, 6, (spec,), lr=1e-3, grad_dtype="bf16", steps=10)
+
+
 WORKLOADS = {
     "single_matrix": single_matrix,
     "transformer_base": transformer_base,
@@ -155,6 +166,12 @@ WORKLOADS = {
     "llama_7b_4l": lambda: llama_7b(layers=4),
     # four decoder layers with a token table of 1024 rows: 0.82 G parameters, the matrices of the decoder alone
     "llama_7b_4l_1kv": lambda: llama_7b(layers=4, vocab=1024),
+    "odd_8192x8200": lambda: odd_shape(8192, 8200),
+    "odd_65536x1000": lambda: odd_shape(65536, 1000),
+    "odd_8200x8193": lambda: odd_shape(8200, 8193),
+    "odd_64x128x8192": lambda: odd_shape(64, 128, 8192),
+    "odd_2048x2048x4x4": lambda: odd_shape(2048, 2048, 4, 4),
+    "odd_4096x4096x3": lambda: odd_shape(4096, 4096, 3),
 }
 
 

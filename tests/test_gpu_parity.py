@@ -208,7 +208,7 @@ def test_shape_zoo_multi_tensor(grad_dtype, update_math, schedule):
     specs = [_mat(96, 256), _mat(33, 77), _mat(5, 1000), _mat(130, 384), _mat(64, 1024), _mat(8, 2048),
              _mat(1, 8192), _mat(8192, 1), _mat(300, 640), _mat(257, 129), _mat(70, 128),
              _vec(50265), _vec(4097), _vec(4096), _vec(4096, force_quant=True), _vec(1), _vec(300),
-             _mat(16, 16), _mat(64, 64), _mat(65, 64), _vec(12345)]
+             _mat(16, 16), _mat(64, 64), _mat(65, 64), _vec(12345), _mat(77, 1992), _mat(260, 264)]
     hyper = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
     pair = Pair(specs, hyper, grad_dtype=grad_dtype, workload_index=7, config=lpmm.default_config(update_math=update_math),
                 schedule=schedule)
