@@ -196,7 +196,7 @@ bool wants_fused(const lpmm_config& cfg, int64_t total_elems) {
     return cfg.schedule == LPMM_SCHEDULE_AUTO && total_elems <= kAutoFusedMaxElems;
 }
 
-struct TileSizes { int64_t update, maxima; };
+struct TileSizes { int64_t update, maxima, flat; };   // flat: the element-indexed tensors' tiles (a launch of their own)
 
 // Elements per tile of the update pass and of the maxima pass (powers of two). Tiles are handed out on demand, so the
 // aim is >= 6 tiles per resident CTA (the tail is what is balanced). Two-pass schedule, measured optima of the update
@@ -204,7 +204,7 @@ struct TileSizes { int64_t update, maxima; };
 // (each tile ends with a flush of its column maxima and starts with an empty load pipeline), up to 1 Mi. The fused
 // schedule wants shorter tiles (an update tile can only start when the tensor's last maxima tile has finished), but
 // every tile costs about 2 us of start-up: 128 Ki / 256 Ki measured best on the 6.7 G list.
-TileSizes choose_tile_sizes(const lpmm_config& cfg, int64_t total_elems, bool fused) {
+TileSizes choose_tile_sizes(const lpmm_config& cfg, int64_t total_elems, int64_t flat_elems, bool fused) {
     const int64_t cap2 = fused ? 131072 : 262144, cap1 = fused ? 262144 : (1 << 20);
     const int64_t hard2 = fused ? 262144 : ((int64_t)1 << 22);   // fused: an update tile has at most 1024 rows of 256 columns
     const int64_t target = total_elems / (6LL * kPlanResidentCtas);
@@ -217,6 +217,11 @@ TileSizes choose_tile_sizes(const lpmm_config& cfg, int64_t total_elems, bool fu
     if (fused && ts.maxima < cap1 && ts.maxima * 2 <= 2 * target) ts.maxima *= 2;
     if (cfg.tile_elems_maxima > 0) ts.maxima = cfg.tile_elems_maxima;
     if (ts.maxima < ts.update) ts.maxima = ts.update;
+    // the element-indexed tensors are sized by their own total: their kernel is a separate launch, and a few long tiles
+    // would leave most of the GPU idle behind a chain of dependent chunks
+    const int64_t target_flat = (fused ? total_elems : flat_elems) / (6LL * kPlanResidentCtas);
+    ts.flat = 2048;
+    while (ts.flat * 2 <= target_flat && ts.flat < ts.update) ts.flat *= 2;
     return ts;
 }
 
@@ -245,7 +250,7 @@ TilePlan plan_tensor(const lpmm_config& cfg, const TensorLayout& t, const TileSi
         if (t.kind != K_BLOCK_TILED) p.tiles_maxima = (int64_t)p.tiles_x * ((t.rows + tr1 - 1) / tr1);
         if (!tiled) p.tiles_update = 0;   // (set below: the update pass of such a tensor is element-indexed)
     }
-    int64_t chunks = ts.update / (kWarps * kWarpElems);
+    int64_t chunks = (tiled || t.kind == K_FP32 ? ts.update : ts.flat) / (kWarps * kWarpElems);
     if (chunks < 1) chunks = 1;
     if (chunks > 16) chunks = 16;
     p.flat_chunks = (int32_t)chunks;
@@ -350,7 +355,7 @@ void compute_layout(const lpmm_config& cfg, const lpmm_shape* shapes, int32_t n,
     L->rc[1] = off; off = region_end(L, off + sizeof(float) * rc);
     L->rc[2] = off; off = region_end(L, off + sizeof(float) * rc);
     L->rcp = off;   off = region_end(L, off + sizeof(float) * rc);
-    int64_t total_elems = 0;
+    int64_t total_elems = 0, flat_elems = 0;
     for (int32_t i = 0; i < n; ++i) total_elems += L->t[i].numel;
     // Tensors with three or four axes whose trailing axes multiply to whole first-moment blocks go to the tiled path as
     // "composite" matrices (leading axes = rows, trailing axes = columns) with per-step expanded statistics. (Not under
@@ -380,6 +385,8 @@ void compute_layout(const lpmm_config& cfg, const lpmm_shape* shapes, int32_t n,
             t.exp_rcp = off; off = region_end(L, off + sizeof(float) * (size_t)t.exp_len);
         }
     }
+    for (int32_t i = 0; i < n; ++i)
+        if (L->t[i].kind == K_RANK1_FLAT || L->t[i].kind == K_BLOCK) flat_elems += L->t[i].numel;
     for (int32_t i = 0; i < n; ++i) {
         TensorLayout& t = L->t[i];
         if (t.kind == K_FP32) {
@@ -396,7 +403,7 @@ void compute_layout(const lpmm_config& cfg, const lpmm_shape* shapes, int32_t n,
         }
     }
     if (cfg.v_mode == LPMM_V_FACTORED) {   // scratch of the sums pass (same tile plan as build_tables)
-        const TileSizes ts = choose_tile_sizes(cfg, total_elems, false);
+        const TileSizes ts = choose_tile_sizes(cfg, total_elems, flat_elems, false);
         for (int32_t i = 0; i < n; ++i) {
             TensorLayout& t = L->t[i];
             if (t.kind != K_FACT) continue;
@@ -410,7 +417,7 @@ void compute_layout(const lpmm_config& cfg, const lpmm_shape* shapes, int32_t n,
     }
     L->states_end = off;   // everything a checkpoint must keep lies below this offset
     if (wants_fused(cfg, total_elems)) {   // the work list: one item per tile of either pass
-        const TileSizes ts = choose_tile_sizes(cfg, total_elems, true);
+        const TileSizes ts = choose_tile_sizes(cfg, total_elems, flat_elems, true);
         int64_t items = 0;
         for (int32_t i = 0; i < n; ++i) {
             const TilePlan p = plan_tensor(cfg, L->t[i], ts);
@@ -446,7 +453,7 @@ struct lpmm_state {
     uint32_t epoch = 0;                    // fused launches made on this state (the per-tensor counters count along)
     int32_t sms, occ1, occ2;
     int32_t p1_ctas;                       // which instantiation of the maxima pass (2 or 3 CTAs per SM)
-    std::vector<int32_t> tiles7;           // prefix sums of the update tiles of the tensors that are not on the tiled path
+    std::vector<int32_t> tiles7;           // prefix sums of the update tiles of the element-indexed tensors
     std::vector<int32_t> tiles6;           // prefix sums of the composite tensors' 256-entry chunks of expanded statistics
     std::vector<int32_t> tiles5;           // prefix sums of the factorized tensors' 32-statistic chunks (finalize kernel)
     std::vector<int32_t> tiles1, tiles2, tiles3;   // host copies of the tile prefix sums (3: element-indexed tiles of every tensor)
@@ -550,7 +557,12 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
     int64_t total_elems = 0;
     for (int32_t i = 0; i < n; ++i) total_elems += st->L.t[i].numel;
     st->fused = wants_fused(st->cfg, total_elems) && st->L.work_items > 0 && st->L.work_items <= 0x7fffffffLL;
-    const TileSizes ts = choose_tile_sizes(st->cfg, total_elems, st->fused);
+    int64_t flat_elems = 0;
+    for (int32_t i = 0; i < n; ++i) {
+        const int32_t k = st->L.t[i].kind;
+        if (k == K_RANK1_FLAT || k == K_BLOCK) flat_elems += st->L.t[i].numel;
+    }
+    const TileSizes ts = choose_tile_sizes(st->cfg, total_elems, flat_elems, st->fused);
 
     std::vector<TensorDesc> descs(n);
     std::vector<TilePlan> plans(n);
@@ -611,7 +623,7 @@ lpmm_status build_tables(lpmm_state* st, cudaStream_t s) {
         t3[i + 1] = t3[i] + (int32_t)p.tiles_flat;
         if (t2[i] + p.tiles_update > 0x7fffffffLL) return LPMM_ERR_UNSUPPORTED;
         const bool moved = own_launch && t.kind == K_BLOCK_TILED;
-        const bool on_tiled_path = t.kind == K_RANK1_FAST || t.kind == K_FACT || t.kind == K_BLOCK_TILED;
+        const bool on_tiled_path = t.kind == K_RANK1_FAST || t.kind == K_FACT || t.kind == K_BLOCK_TILED || t.kind == K_FP32;
         t2[i + 1] = t2[i] + ((moved || !on_tiled_path) ? 0 : (int32_t)p.tiles_update);
         t7[i + 1] = t7[i] + (on_tiled_path ? 0 : (int32_t)p.tiles_update);
         t4[i + 1] = t4[i] + (moved ? (int32_t)p.tiles_update : 0);
@@ -931,7 +943,7 @@ lpmm_status enqueue_update(lpmm_state* st, StepArgs a, int32_t t0, int32_t t1, b
                            st->cfg.v_mode == LPMM_V_FACTORED ? 1 : (st->cfg.v_mode == LPMM_V_BLOCK ? 2 : 0),
                            tiles < cap ? tiles : cap, s));
     if (tiles > 0) *launches += 1;
-    if (st->tiles7[t1] > st->tiles7[t0]) {   // the tensors that are not on the tiled path: a kernel (and launch) of their own
+    if (st->tiles7[t1] > st->tiles7[t0]) {   // the element-indexed tensors: a kernel (and launch) of their own
         a.tile_start = reinterpret_cast<const int32_t*>(st->arena + st->L.tiles7);
         a.tile_begin = st->tiles7[t0];
         a.tile_end = st->tiles7[t1];

@@ -938,10 +938,11 @@ __device__ __forceinline__ void pass2_fp32(const TensorDesc& d, float* __restric
 // WB: a bfloat16 copy of every updated parameter is written as well (a.params_bf16).
 // A32: every parameter pointer (and, with fp32 gradients, every gradient pointer) of the step is 32-byte aligned,
 // checked on the host: the tiled path then moves a lane's 8 values with one 256-bit access.
-// MISC: false = the tensors on the tiled path; true = all the others (element-indexed: odd shapes, ragged 1-D tensors;
-// fp32 states of small tensors). They are two kernels (two launches per step) so that the register allocation of the
-// tiled path - where nearly all parameters of a real model are - is not shared with paths it never runs: with both in
-// one kernel the update pass of the LLaMA-7B list took 13.9-14.0 ms instead of 13.3-13.4.
+// MISC: false = the tensors on the tiled path and the small tensors with fp32 states; true = the element-indexed ones
+// (odd shapes, ragged or short 1-D tensors). They are two kernels (two launches per step when a state has both) so that
+// the register allocation of the tiled path - where nearly all parameters of a real model are - is not shared with
+// the element-indexed paths: with both in one kernel the update pass of the LLaMA-7B list took 13.9-14.0 ms instead
+// of 13.3-13.4.
 template <bool BF16, bool EXACT, int MSHIFT, int VF, bool WB, bool A32, bool MISC = false>
 __global__ void __launch_bounds__(kThreads, 2) pass2_kernel(StepArgs a) {
     __shared__ __align__(16) unsigned char s_lut[kLutSmemBytes];
@@ -965,7 +966,6 @@ __global__ void __launch_bounds__(kThreads, 2) pass2_kernel(StepArgs a) {
             switch (d.kind) {
                 case K_RANK1_FLAT: pass2_flat<BF16, true, EXACT, MSHIFT, WB, A32>(d, w, w16, g, local, a.sel, a.h, h2, lt, s_lut, s_red, red_step); break;
                 case K_BLOCK:      pass2_flat<BF16, false, EXACT, MSHIFT, WB, A32>(d, w, w16, g, local, a.sel, a.h, h2, lt, s_lut, s_red, red_step); break;
-                case K_FP32:       pass2_fp32<BF16, EXACT, WB, A32>(d, w, w16, g, local, a.h); break;
                 default: break;
             }
         } else {
@@ -979,6 +979,9 @@ __global__ void __launch_bounds__(kThreads, 2) pass2_kernel(StepArgs a) {
                 case K_BLOCK_TILED:   // matrices of a block-wise state; long 1-D tensors folded into rows (in states of another
                                       // kind these get a launch of their own, so that the default kernels stay lean)
                     if (VF == 2) pass2_rank1_fast<BF16, EXACT, MSHIFT, 2, WB, A32>(d, w, w16, g, local, a.sel, a.h, h2, lt, s_lut, s_red, red_step);
+                    break;
+                case K_FP32:      // small tensors with fp32 states ride along (a short, register-light path)
+                    pass2_fp32<BF16, EXACT, WB, A32>(d, w, w16, g, local, a.h);
                     break;
                 default: break;
             }
