@@ -97,6 +97,39 @@ def test_bad_configurations_are_rejected_on_the_host():
     L.lpmm_state_destroy(None)
 
 
+def test_schedule_and_tuning_fields_are_validated_and_sized_on_the_host():
+    L = lpmm.lib()
+    out = C.c_size_t()
+    shapes = lpmm.make_shapes([(1024, 4096, 2, 0), (4096, 1, 1, 1)])
+    for field, value, want in (("schedule", 9, lpmm.ERR_INVALID_ARG), ("tile_elems", 3000, lpmm.ERR_INVALID_ARG),
+                               ("tile_elems", 1024, lpmm.ERR_INVALID_ARG), ("tile_elems_maxima", 1 << 23, lpmm.ERR_INVALID_ARG),
+                               ("l2_keep_mbytes", -1, lpmm.ERR_INVALID_ARG), ("lead_melems", -1, lpmm.ERR_INVALID_ARG),
+                               ("gap_items", -5, lpmm.ERR_INVALID_ARG), ("no_l2_hints", 2, lpmm.ERR_INVALID_ARG),
+                               ("overlap_groups", -1, lpmm.ERR_INVALID_ARG)):
+        bad = lpmm.default_config()
+        setattr(bad, field, value)
+        assert L.lpmm_state_bytes(C.byref(bad), shapes, 2, C.byref(out)) == want, field
+    # the fused schedule needs the default quantizers
+    for kw in (dict(v_mode=lpmm.V_BLOCK), dict(v_mode=lpmm.V_FACTORED), dict(m_block=2048)):
+        cfg = lpmm.default_config(schedule=lpmm.SCHEDULE_FUSED, **kw)
+        assert L.lpmm_state_bytes(C.byref(cfg), shapes, 2, C.byref(out)) == lpmm.ERR_UNSUPPORTED
+    # its work list lies behind the states: a fused arena is a two-pass arena plus 8 bytes per tile
+    two = lpmm.state_bytes(lpmm.default_config(schedule=lpmm.SCHEDULE_TWO_PASS), shapes)
+    fused = lpmm.state_bytes(lpmm.default_config(schedule=lpmm.SCHEDULE_FUSED), shapes)
+    auto = lpmm.state_bytes(lpmm.default_config(), shapes)
+    assert two < fused <= two + 8 * 2 * (1024 * 4096 // 2048 + 8) + 512 and auto == fused      # 4.2 M elements: AUTO = fused
+    big = workloads.llama_7b().tensors
+    assert lpmm.state_bytes(lpmm.default_config(), big) == lpmm.state_bytes(lpmm.default_config(schedule=lpmm.SCHEDULE_TWO_PASS), big)
+    # smaller tiles, longer list
+    assert lpmm.state_bytes(lpmm.default_config(schedule=lpmm.SCHEDULE_FUSED, tile_elems=32768, tile_elems_maxima=65536), big) > \
+        lpmm.state_bytes(lpmm.default_config(schedule=lpmm.SCHEDULE_FUSED), big)
+    assert L.lpmm_state_selftest_wait(None, None, None, None) == lpmm.ERR_INVALID_ARG
+    assert L.lpmm_state_wait_stats(None, None, None, None) == lpmm.ERR_INVALID_ARG
+    assert L.lpmm_state_check_guards(None, None, None, None) == lpmm.ERR_INVALID_ARG
+    assert L.lpmm_build_is_checking() == 0
+    assert L.lpmm_state_schedule(None) == -1
+
+
 def test_workload_shapes_match_the_named_architectures():
     assert len(workloads.transformer_base().tensors) == 181
     assert len(workloads.roberta_large().tensors) == 394
