@@ -332,6 +332,39 @@ def test_checkpoint_attach_resumes_bit_exactly(sched_a, sched_b):
         assert torch.equal(a.params[i], params_copy[i])
 
 
+def test_fused_state_interleaved_with_two_pass_steps():
+    # A state on the fused schedule also serves the entry points that always run two-pass (the bfloat16 copy, the
+    # host-buffer step); the two kinds of step hand the rotating statistics buffers and their "cleared" status to each
+    # other. Every step is checked against the oracle.
+    specs = [_mat(128, 512), _mat(130, 384), _mat(33, 77), _mat(5, 1000), _vec(5000), _vec(100)]
+    hyper = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
+    pair = Pair(specs, hyper, workload_index=19, schedule=lpmm.SCHEDULE_FUSED)
+    copies = [torch.empty(s.numel, dtype=torch.bfloat16, device="cuda") for s in specs]
+    nbytes = lpmm.stage_bytes(pair.state)
+    dp = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    dg = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    for t in range(1, 10):
+        grads = pair.grads_for(t)
+        if t in (3, 4, 8):          # two-pass with the bfloat16 copy
+            lpmm.adamw4_step(pair.state, pair.params, grads, step=t, params_bf16=copies, **hyper)
+            launches = pair.state.last_launches
+            assert launches > 1
+        elif t == 6:                # two-pass through host buffers
+            h_params = [p.detach().cpu().pin_memory() for p in pair.params]
+            h_grads = [g.cpu().pin_memory() for g in grads]
+            lpmm.adamw4_step_host(pair.state, h_params, h_grads, dp, dg, step=t, **hyper)
+            torch.cuda.synchronize()
+            for p, h in zip(pair.params, h_params):
+                p.copy_(h.reshape(p.shape))
+        else:
+            lpmm.adamw4_step(pair.state, pair.params, grads, step=t, **hyper)
+            assert pair.state.last_launches == 1
+        for i, g in enumerate(grads):
+            oracle.adamw4_step(pair.w_ref[i], g.float().cpu().numpy().ravel(), pair.ostate[i], step=t, **hyper)
+        torch.cuda.synchronize()
+        pair.compare(tol=1e-6)
+
+
 def test_attach_refuses_an_arena_that_is_something_else():
     specs = [_mat(128, 512), _vec(5000)]
     cfg = lpmm.default_config()
@@ -538,13 +571,13 @@ def _nd(*dims):
     return workloads.TensorSpec("t" + "x".join(map(str, dims)), rows, dims[-1], len(dims), dims=tuple(dims))
 
 
-@SCHEDULES
+@SCHEDULES3
 @pytest.mark.parametrize("grad_dtype,update_math", [(torch.float32, lpmm.UPDATE_IEEE), (torch.bfloat16, lpmm.UPDATE_FAST)])
 def test_tensors_with_three_and_four_axes_match_oracle(grad_dtype, update_math, schedule):
     # Alg. 4 in its general form: one vector of maxima per axis, scale = minimum over the element's axes.
     # Codes, block scales and every axis' statistics bit-exact; parameters bit-exact with IEEE update math,
     # within 1e-6 * max(|w|, lr) with the approximate one. A matrix rides along to cover mixed lists.
-    cfg = lpmm.default_config(update_math=update_math, schedule=schedule)
+    cfg = lpmm.default_config(update_math=update_math, schedule=schedule, overlap_groups=3)
     # (under the two-pass schedule the tensors whose trailing axes multiply to whole 128-blocks - the last five - run on
     # the tiled kernels as composite matrices with expanded statistics; the others, and all of them under the fused
     # schedule, on the element-indexed ones)
@@ -588,13 +621,16 @@ def test_tensors_with_three_and_four_axes_match_oracle(grad_dtype, update_math, 
     assert ei.value.status == lpmm.ERR_UNSUPPORTED
 
 
-@pytest.mark.parametrize("grad_dtype,m_block", [(torch.bfloat16, 128), (torch.float32, 2048)])
-def test_bf16_copy_of_the_parameters(grad_dtype, m_block):
+@pytest.mark.parametrize("grad_dtype,m_block,schedule", [(torch.bfloat16, 128, lpmm.SCHEDULE_AUTO), (torch.float32, 2048, lpmm.SCHEDULE_AUTO),
+                                                         (torch.bfloat16, 128, lpmm.SCHEDULE_TWO_PASS)])
+def test_bf16_copy_of_the_parameters(grad_dtype, m_block, schedule):
     # lpmm_adamw4_step_bf16w: states and fp32 parameters exactly as the plain step leaves them, plus a bfloat16 copy
     # that is the nearest-even rounding of the new fp32 parameters, on every kind of tensor and on ragged tails.
-    cfg = lpmm.default_config(m_block=m_block)
+    # (AUTO puts this small list on the fused schedule for the plain step, so the two states also compare the schedules;
+    # under TWO_PASS the tensors with three axes whose trailing axes fill 128-blocks are composite matrices in both)
+    cfg = lpmm.default_config(m_block=m_block, schedule=schedule)
     specs = [_mat(96, 256), _mat(64, 2048), _mat(130, 384), _mat(33, 77), _mat(257, 129), _vec(50265), _vec(4097), _vec(300), _vec(1),
-             _nd(6, 10, 200), _vec(196608)]      # the last one is folded into rows and updated by a launch of its own
+             _nd(6, 10, 200), _nd(5, 3, 384), _vec(196608)]      # the last one is folded into rows and updated by a launch of its own
     hyper = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01)
     pa = [workloads.make_param(s, 15, i, device="cuda") for i, s in enumerate(specs)]
     pb = [p.clone() for p in pa]
@@ -616,8 +652,8 @@ def test_bf16_copy_of_the_parameters(grad_dtype, m_block):
             got = copies[i].view(torch.int16).cpu().numpy().view(np.uint16)
             assert np.array_equal(got, want), (s.name, t)
     # (the bfloat16 copy always runs the two-pass schedule: maxima, reciprocals, tiled update, element-indexed update, and
-    # the folded tensor's own update launch)
-    assert sb.last_launches == 5
+    # the folded tensor's own update launch; three more small kernels where a composite tensor is present)
+    assert sb.last_launches == (8 if schedule == lpmm.SCHEDULE_TWO_PASS else 5)
     # refused with the factorized second moment, and with a missing pointer array
     sf = lpmm.state_init(lpmm.default_config(v_mode=lpmm.V_FACTORED), [_mat(96, 256)])
     with pytest.raises(lpmm.LpmmError) as ei:
