@@ -136,3 +136,49 @@ def test_llama_7b_flat_full_size_sampled_tensors():
             w_ref[i][:] = w
         del grads
     assert lpmm.device_status(state) == 0
+
+
+@pytest.mark.parametrize("m_block", [128, 2048])
+@pytest.mark.parametrize("v_mode", [lpmm.V_RANK1, lpmm.V_BLOCK, lpmm.V_FACTORED], ids=["rank1", "block", "factored"])
+def test_square_8192_sweep_variants_full_size(m_block, v_mode):
+    # The quantizer / normalizer sweep as the benchmark runs it: one 8192 x 8192 matrix (67 M elements, many tiles and
+    # tile rows), first-moment blocks of 128 and 2048, second moment rank-1, block-wise or factorized; the oracle
+    # follows the whole matrix for two steps from a shared state.
+    wl = workloads.square_8192()
+    hyper = hyper_of(wl)
+    spec = wl.tensors[0]
+    cfg = lpmm.default_config(m_block=m_block, v_mode=v_mode)
+    p = workloads.make_param(spec, wl.index, 0, device="cuda")
+    state = lpmm.state_init(cfg, wl.tensors)
+    w_ref = p.cpu().numpy().ravel().copy()
+    factored = v_mode == lpmm.V_FACTORED
+    okind = oracle.BLOCK if v_mode == lpmm.V_BLOCK else oracle.RANK1
+    ost = oracle.state_init(spec.rows, spec.cols, okind, m_block=m_block)
+    R, Cc = np.zeros(spec.rows, np.float32), np.zeros(spec.cols, np.float32)
+    for step in (1, 2):
+        g = workloads.make_grad(spec, wl.index, 0, step, device="cuda")
+        lpmm.adamw4_step(state, [p], [g], step=step, **hyper)
+        torch.cuda.synchronize()
+        assert lpmm.device_status(state) == 0
+        g_host = g.cpu().numpy().ravel()
+        w_prev = w_ref.copy()
+        view = lpmm.state_view(state, 0)
+        if factored:
+            oracle.adamw4_factor_step(w_ref, g_host, ost, R, Cc, step=step, **hyper)
+            np.testing.assert_allclose(view["v_s0"].cpu().numpy(), R, rtol=1e-6, atol=0)
+            np.testing.assert_allclose(view["v_s1"].cpu().numpy(), Cc, rtol=1e-6, atol=0)
+            names = ("m_codes", "m_scale")
+        else:
+            oracle.adamw4_step(w_ref, g_host, ost, step=step, **hyper)
+            names = ("m_codes", "m_scale", "v_codes", "v_s0", "v_s1")
+        for name in names:
+            ref = getattr(ost, name)
+            if ref is not None:
+                assert np.array_equal(view[name].cpu().numpy().view(np.uint8), ref.view(np.uint8)), (name, step)
+        w = p.cpu().numpy().ravel()
+        scale = np.maximum(np.abs(w_ref), hyper["lr"])
+        if factored:       # the step an element took joins the normaliser (see the factorized test in test_gpu_parity.py)
+            scale = np.maximum(scale, np.abs(w_ref - w_prev))
+        err = float(np.max(np.abs(w - w_ref) / scale))
+        assert err <= 1e-6, (step, err)
+        w_ref[:] = w
