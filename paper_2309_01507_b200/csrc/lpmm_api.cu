@@ -211,10 +211,12 @@ TileSizes choose_tile_sizes(const lpmm_config& cfg, int64_t total_elems, int64_t
     TileSizes ts;
     ts.update = 2048;
     while (ts.update * 2 <= target && ts.update < cap2) ts.update *= 2;
+    if (fused && ts.update < 8192) ts.update = 8192;   // (one 1024x4096 matrix: 41.7 us with 8 Ki / 16 Ki tiles, 45.3 with 2 Ki / 4 Ki)
     if (cfg.tile_elems > 0) ts.update = cfg.tile_elems < hard2 ? cfg.tile_elems : hard2;
     ts.maxima = ts.update;
     while (ts.maxima * 2 <= target && ts.maxima < cap1) ts.maxima *= 2;
     if (fused && ts.maxima < cap1 && ts.maxima * 2 <= 2 * target) ts.maxima *= 2;
+    if (fused && ts.maxima < 16384) ts.maxima = 16384;
     if (cfg.tile_elems_maxima > 0) ts.maxima = cfg.tile_elems_maxima;
     if (ts.maxima < ts.update) ts.maxima = ts.update;
     // the element-indexed tensors are sized by their own total: their kernel is a separate launch, and a few long tiles
