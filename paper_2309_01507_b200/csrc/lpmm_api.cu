@@ -374,8 +374,20 @@ void compute_layout(const lpmm_config& cfg, const lpmm_shape* shapes, int32_t n,
                 if (c % 128 != 0 || c % cfg.m_block != 0 || c > ((int64_t)1 << 24)) continue;
                 if (best == 0 || (best_cols < 1024 && c > best_cols)) { best = sp; best_cols = c; }   // the narrowest one that fills a tile
             }
+            bool whole_blocks = best != 0;
+            if (!whole_blocks && cfg.m_block == 128) {
+                // no split makes rows of whole first-moment blocks: rows of whole lanes (cols % 8 == 0, at least 256) still get
+                // the tiled maxima pass and the stepped interior loop of the element-indexed update
+                for (int32_t sp = t.nd - 1; sp >= 1; --sp) {
+                    int64_t c = 1;
+                    for (int32_t a = sp; a < t.nd; ++a) c *= t.nd_dim[a];
+                    if (c % 8 != 0 || c < 256 || c > ((int64_t)1 << 24)) continue;
+                    if (best == 0 || (best_cols < 1024 && c > best_cols)) { best = sp; best_cols = c; }
+                }
+            }
             if (best == 0) continue;
-            t.kind = K_RANK1_FAST;
+            if (whole_blocks) t.kind = K_RANK1_FAST;
+            else t.p1_tiled = true;
             t.nd_split = best;
             t.cols = best_cols;
             t.rows = t.numel / best_cols;

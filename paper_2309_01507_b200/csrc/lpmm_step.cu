@@ -719,7 +719,7 @@ __device__ __forceinline__ void pass2_flat_interior(const TensorDesc& d, float* 
                                                     const Hyper2& h2, const LaneTables& lt, const unsigned char* s_lut) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t base = (int64_t)tile * d.flat_chunks * (kWarps * kWarpElems);
-    const float* rc_old = rc_pick(d, sel.old_i);
+    const float* rc_old = stats_old(d, sel);
     const float* rcp_new = d.rcp_new;
     float* wb = w + base;
     uint16_t* w16b = WB ? w16 + base : nullptr;
@@ -775,7 +775,7 @@ __device__ __forceinline__ void pass2_flat(const TensorDesc& d, float* __restric
                                            int tile, RcSel sel, const Hyper& h, const Hyper2& h2, const LaneTables& lt,
                                            const unsigned char* s_lut, float* s_red, uint32_t& red_step) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const float* rc_old = rc_pick(d, sel.old_i);
+    const float* rc_old = stats_old(d, sel);
     const float* rcp_new = d.rcp_new;
     const int64_t m_mask = ((int64_t)1 << MSHIFT) - 1;
     // checking build: the tile starts inside the tensor (B2048: recorded only, the CTA-wide barrier needs every warp)

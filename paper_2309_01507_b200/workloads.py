@@ -172,6 +172,7 @@ WORKLOADS = {
     "odd_64x128x8192": lambda: odd_shape(64, 128, 8192),
     "odd_2048x2048x4x4": lambda: odd_shape(2048, 2048, 4, 4),
     "odd_4096x4096x3": lambda: odd_shape(4096, 4096, 3),
+    "odd_1024x1000x3x3": lambda: odd_shape(1024, 1000, 3, 3),     # rows of whole lanes, not of whole blocks (9000 = 8 * 1125)
 }
 
 
