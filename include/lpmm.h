@@ -151,14 +151,17 @@ lpmm_status lpmm_state_attach(const lpmm_config* cfg, const lpmm_shape* shapes, 
  * Both arrays are HOST arrays of n device pointers, each 16-byte aligned (when all of them are 32-byte aligned, as
  * framework allocations are, the update pass uses 256-bit accesses and is ~6 % faster). step is t >= 1.
  * Requires 0 <= beta1, beta2 < 1, lr >= 0, eps >= 0, weight_decay >= 0, all finite.
- * Kernels launched: one pass over the rank-1 tensors that reduces the new row/column maxima, one
- * small pass that inverts them, one pass over all tensors that updates and re-quantizes; one more update
- * launch when the state holds 1-D tensors of 65536 elements or more whose length is a multiple of 128 (they are
- * folded into rows and updated by the block-wise form of the tiled kernel) and its matrices are not block-wise.
+ * Kernels launched (two-pass schedule; see lpmm_schedule for the others): one pass over the rank-1 tensors that
+ * reduces the new row/column maxima, one small pass that inverts them, one pass that updates and re-quantizes the
+ * tensors on the tiled path (rows of whole first-moment blocks) and the small fp32 ones; one more update launch each
+ * for the element-indexed tensors (other shapes) and for 1-D tensors of 65536 elements or more whose length is a
+ * multiple of 128 (folded into rows and updated by the block-wise form of the tiled kernel) when the state's matrices
+ * are not block-wise; three more small launches when tensors with three or four axes run as composite matrices
+ * (their per-axis statistics are expanded per step). lpmm_state_last_launches() reports the count.
  * LPMM_V_FACTORED (reading of Sec. 4.3, which gives no formula): R <- b2 R + (1-b2) rowsum(g^2), C likewise,
- * v_ij = R_i C_j / sum(R), then Eq. 1 as usual; the first pass reduces the sums (fp32 atomics, so R and C are
- * reproducible to rounding only), a fourth small kernel updates R, C and sum(R). Such tensors need
- * cols % m_block == 0 (else LPMM_ERR_UNSUPPORTED at state creation). */
+ * v_ij = R_i C_j / sum(R), then Eq. 1 as usual. The first pass writes per-tile partial sums of g^2, a small kernel adds
+ * them in a fixed order and updates R, C and sum(R): R and C are reproducible bit for bit (no floating-point atomics).
+ * Such tensors need cols % m_block == 0 (else LPMM_ERR_UNSUPPORTED at state creation). */
 lpmm_status lpmm_adamw4_step(lpmm_state* st, void* const* d_params, const void* const* d_grads,
                              int32_t grad_dtype, float lr, float beta1, float beta2, float eps,
                              float weight_decay, int64_t step, void* stream);
