@@ -59,17 +59,19 @@ typedef enum { LPMM_UPDATE_FAST = 0, LPMM_UPDATE_IEEE = 1 } lpmm_update_math;
 
 /* Order of the work inside one step (Sec. 4.2: the row and column maxima of the NEW second moment depend on the whole
  * tensor, so every rank-1 tensor is read twice: once to reduce r', c' and once to update and re-quantize).
- *   TWO_PASS: the maxima pass over all tensors, then the update pass over all tensors (three launches). The second read
- *             of the gradient and the second-moment codes comes from DRAM.
- *   FUSED:    one launch whose work list interleaves the maxima tiles of a tensor closely before its update tiles, with
- *             L2 eviction priorities on every access, so that the second read is served by L2 where the tensor (or its
- *             tail) fits. Needs the default quantizers (LPMM_V_RANK1, m_block 128); other states and
- *             lpmm_adamw4_step_bf16w / lpmm_adamw4_step_host run TWO_PASS. CTAs wait for one another through
- *             counters in the arena; every wait is bounded (see lpmm_state_device_status).
- *   AUTO:     by measurement: FUSED for eligible states of fewer than 63 Mi elements, else TWO_PASS.
- * The stored states and the parameters are bit-identical under both schedules. */
-/*   OVERLAP:  TWO_PASS on groups of tensors, with the maxima pass of group k + 1 launched on a second stream (owned by the
- *             handle) beside the update pass of group k; ordered by events, no device-side waiting. */
+ *   TWO_PASS: the maxima pass over all tensors, then the update pass over all tensors (three launches, see
+ *             lpmm_adamw4_step). The second read of the gradient and the second-moment codes comes from DRAM.
+ *   FUSED:    one launch whose work list puts the update tiles of a tensor closely behind its maxima tiles (the maxima
+ *             pass loads the tail of a tensor with the "evict last" L2 priority), so that part of the second read is
+ *             served by L2, and that needs no memset node. Needs the default quantizers (LPMM_V_RANK1, m_block 128);
+ *             other states and lpmm_adamw4_step_bf16w / lpmm_adamw4_step_host run TWO_PASS. CTAs wait for one
+ *             another through counters in the arena; every wait is bounded (see lpmm_state_device_status).
+ *   OVERLAP:  TWO_PASS on groups of tensors, with the maxima pass of group k + 1 launched on a second stream (owned by
+ *             the handle) beside the update pass of group k; ordered by events, no device-side waiting.
+ *   AUTO:     by measurement on B200: FUSED for eligible states of fewer than 63 Mi elements (it is 11-14 % faster
+ *             there: fewer launches), else TWO_PASS (faster from there on; the L2-resident re-read saves DRAM bytes
+ *             but not time).
+ * The stored states and the parameters are bit-identical under all schedules. */
 typedef enum { LPMM_SCHEDULE_AUTO = 0, LPMM_SCHEDULE_TWO_PASS = 1, LPMM_SCHEDULE_FUSED = 2, LPMM_SCHEDULE_OVERLAP = 3 } lpmm_schedule;
 
 /* lpmm_shape.flags */
