@@ -994,7 +994,6 @@ lpmm_status enqueue_range(lpmm_state* st, StepArgs a, int32_t t0, int32_t t1, bo
 //   aux:  maxima(0) | maxima(1) after update(-)... each maxima(k+1) starts when update(k-1) has finished
 //   main: update(k) after maxima(k)
 lpmm_status enqueue_overlapped(lpmm_state* st, const StepArgs& a, bool bf16, bool ieee_update, cudaStream_t s, int32_t* launches) {
-    const int32_t n = st->n;
     if (!st->aux) LPMM_CUDA(cudaStreamCreateWithFlags(&st->aux, cudaStreamNonBlocking));
     const std::vector<int32_t>& cut = st->group_cut;
     const size_t groups = cut.size() - 1;
@@ -1022,7 +1021,6 @@ lpmm_status enqueue_overlapped(lpmm_state* st, const StepArgs& a, bool bf16, boo
         if (rc != LPMM_OK) return rc;
         LPMM_CUDA(cudaEventRecord(ev_u, s));
     }
-    (void)n;
     return LPMM_OK;   // the caller's stream ends after the last update; the second stream has nothing left in flight
 }
 
