@@ -40,8 +40,9 @@ PASS1_BYTES = {"bf16": 2.5, "f32": 4.5}
 PASS2_TRAFFIC_BYTES_PER_PARAM = {"bf16": 12.009, "f32": 14.125}
 # DRAM traffic of the whole step per parameter by schedule (ncu, same metrics): two-pass = the update pass above plus
 # the maxima pass (2.503 B/param, profiles/pass1_llama_7b_1l.txt); fused = one launch, from the capture of the
-# four-decoder-layer LLaMA slice summarised in profiles/step_fused_llama_7b_4l.txt.
-STEP_TRAFFIC_BYTES_PER_PARAM = {"two_pass": {"bf16": 14.512}, "fused": {"bf16": None}}
+# four-decoder-layer LLaMA slice (817.96 M params) summarised in profiles/schedules_llama_7b.txt, at the library's default
+# tuning (7.931 GB read + 4.092 GB written; 13.98 B/param at the tuning that keeps most in L2).
+STEP_TRAFFIC_BYTES_PER_PARAM = {"two_pass": {"bf16": 14.512}, "fused": {"bf16": 14.699}}
 
 
 def parse_args():
