@@ -365,6 +365,49 @@ def test_fused_state_interleaved_with_two_pass_steps():
         pair.compare(tol=1e-6)
 
 
+def test_fused_work_list_invariants():
+    # The fused launch's correctness rests on its host-built list: every tile of either pass exactly once, and every
+    # update tile of a rank-1 tensor behind all of that tensor's maxima tiles (its CTA waits for them; items are handed
+    # out in list order). The list lies behind the states in the arena: two words per item (tensor | flags, tile).
+    for wl, kw in ((workloads.transformer_base(), {}), (workloads.single_matrix(), {}),
+                   (workloads.transformer_base(), dict(lead_melems=1, gap_items=7, tile_elems=4096, tile_elems_maxima=8192))):
+        cfg = lpmm.default_config(schedule=lpmm.SCHEDULE_FUSED, **kw)
+        st = lpmm.state_init(cfg, wl.tensors)
+        torch.cuda.synchronize()
+        states_end = lpmm.state_bytes(lpmm.default_config(schedule=lpmm.SCHEDULE_TWO_PASS, **kw), wl.tensors)
+        words = st.arena[states_end:].view(torch.int32).cpu().numpy().view(np.uint32).reshape(-1, 2)
+        tensor = words[:, 0] & 0x0fffffff
+        update = (words[:, 0] & 0x40000000) != 0
+        keep = (words[:, 0] & 0x80000000) != 0
+        kinds = [lpmm.state_view(st, i)["kind"] for i in range(len(wl.tensors))]
+        seen = {}
+        last_maxima, first_update = {}, {}
+        pos = 0
+        for pos in range(len(words)):
+            t, u, tile = int(tensor[pos]), bool(update[pos]), int(words[pos, 1])
+            if t >= len(wl.tensors):
+                break
+            key = (t, u, tile)
+            if key in seen:
+                break                      # padding behind the list (zeros repeat item (0, maxima, 0))
+            seen[key] = pos
+            if u:
+                first_update.setdefault(t, pos)
+            else:
+                last_maxima[t] = pos
+                assert kinds[t] == lpmm.KIND_RANK1
+        for t, k in enumerate(kinds):
+            ups = sorted(tile for (tt, u, tile) in seen if tt == t and u)
+            assert ups == list(range(len(ups))) and len(ups) > 0, t          # every update tile once, none missing
+            mxs = sorted(tile for (tt, u, tile) in seen if tt == t and not u)
+            assert mxs == list(range(len(mxs)))
+            if k == lpmm.KIND_RANK1:
+                assert len(mxs) > 0 and last_maxima[t] < first_update[t], t  # dependency order
+            else:
+                assert len(mxs) == 0
+        assert not np.any(keep & update)                                     # only maxima tiles carry the keep flag
+
+
 def test_attach_refuses_an_arena_that_is_something_else():
     specs = [_mat(128, 512), _vec(5000)]
     cfg = lpmm.default_config()
