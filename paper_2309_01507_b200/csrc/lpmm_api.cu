@@ -1166,7 +1166,7 @@ lpmm_status lpmm_adamw4_step_host(lpmm_state* st, void* const* h_params, const v
     {
         int64_t total = 0;
         for (int32_t i = 0; i < n; ++i) total += st->L.t[i].numel;
-        const int64_t per_group = total / 16 + 1;
+        const int64_t per_group = total / 32 + 1;
         int64_t acc = 0;
         for (int32_t i = 0; i < n; ++i) {
             acc += st->L.t[i].numel;
